@@ -1,0 +1,520 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, invariants and
+brute force on tiny inputs.  None of these re-types an oracle formula; each one checks
+the oracle against something fixed outside it."""
+
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.special
+import torch
+from scipy.spatial import cKDTree
+
+from oracle import dpa4c as orc
+from workloads import SMALL_PROFILES, make_blob, make_system
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden_rows(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+TOL = {k: float(v) for k, v in _golden_rows("verification_tolerances.txt")}
+
+
+def _rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def _rand_unitish(n, seed):
+    return torch.from_numpy(_rng(seed).standard_normal((n, 3)))
+
+
+# ---------------------------------------------------------------- printed tables
+
+def test_widths_table():
+    for row in _golden_rows("widths_table.txt"):
+        C0, C1, C2, K1, K2 = map(int, row[:5])
+        for k, L in enumerate((2, 3, 4)):
+            w = orc.widths(C0, L)
+            assert (w["C1"], w["C2"], w["K1"], w["K2"]) == (C1, C2, K1, K2)
+            assert w["S"] == int(row[5 + k])
+            assert w["D_out"] == int(row[8 + k])
+
+
+def test_worked_examples():
+    w = orc.widths(32, 2)
+    assert (w["C1"], w["C2"], w["S"], w["D_out"]) == (8, 4, 76, 144)
+
+
+def test_parameter_counts():
+    # 118 elements plus the zero padding row of the type table
+    for name, C0, L, R, F, n in _golden_rows("parameter_counts.txt"):
+        assert orc.parameter_count(int(C0), int(L), int(R), 16, 3, int(F), 119) == int(n), name
+
+
+def test_triples_for_L4():
+    assert orc.triples(4) == [(1, 1, 2), (1, 2, 3), (1, 3, 4), (2, 2, 2), (2, 2, 4), (2, 3, 3),
+                              (2, 4, 4), (3, 3, 4), (4, 4, 4)]
+    assert orc.triples(2) == [(1, 1, 2), (2, 2, 2)]
+    assert orc.triples(3) == [(1, 1, 2), (1, 2, 3), (2, 2, 2), (2, 3, 3)]
+
+
+def test_bispectrum_counts():
+    # Eq. "bispectrum-count"
+    for C0 in (8, 32, 128):
+        K = orc.probe_ranks(C0, 4)
+        for tr in orc.triples(4):
+            l1, l2, l3 = tr
+            n = len(orc.retained_entries(tr, K))
+            if l1 == l2 == l3:
+                k = K[l1]
+                assert n == k * (k + 1) * (k + 2) // 6
+            elif l1 == l2:
+                assert n == K[l1] * (K[l1] + 1) // 2 * K[l3]
+            elif l2 == l3:
+                assert n == K[l2] * (K[l2] + 1) // 2 * K[l1]
+            else:
+                assert n == K[l1] * K[l2] * K[l3]
+
+
+# ---------------------------------------------------------------- envelope
+
+def test_envelope_is_incomplete_beta():
+    rc = 6.0
+    rho = torch.linspace(0.0, 7.0, 1401, dtype=torch.float64)
+    chi = orc.envelope(rho, rc).numpy()
+    x = np.clip(rho.numpy() / rc, 0, 1)
+    ref = 1.0 - scipy.special.betainc(5, 4, x)
+    assert np.abs(chi - ref).max() < 1e-15 * 8
+    assert chi[0] == 1.0 and (chi[rho.numpy() >= rc] == 0).all()
+
+
+def test_envelope_derivative_closed_form():
+    rc = 6.0
+    rho = torch.linspace(0.05, 5.95, 300, dtype=torch.float64, requires_grad=True)
+    (d,) = torch.autograd.grad(orc.envelope(rho, rc).sum(), rho)
+    x = rho.detach() / rc
+    ref = -280.0 * x ** 4 * (1 - x) ** 3 / rc
+    assert (d - ref).abs().max() < 1e-14
+
+
+def test_envelope_c3_at_cutoff():
+    rc = 6.0
+    h = 1e-3
+    for k in (1, 2, 3):
+        # one-sided k-th difference quotient just inside the cutoff vanishes like h^(4-k)
+        pts = torch.tensor([rc - j * h for j in range(k + 1)], dtype=torch.float64)
+        vals = orc.envelope(pts, rc).numpy()
+        coef = [(-1) ** j * math.comb(k, j) for j in range(k + 1)]
+        dq = sum(c * v for c, v in zip(coef, vals)) / h ** k
+        assert abs(dq) < 50 * h ** (4 - k)
+
+
+# ---------------------------------------------------------------- radial basis
+
+def test_bessel_basis_values_and_limit():
+    omega = torch.tensor([0.5, 1.0, 3.0], dtype=torch.float64)
+    rho = torch.tensor([0.0, 1e-9, 0.7, 5.0], dtype=torch.float64)
+    f = orc.bessel_basis(rho, omega).numpy()
+    assert np.allclose(f[0], omega.numpy(), rtol=0, atol=0)
+    assert np.allclose(f[1], omega.numpy(), rtol=1e-15)
+    assert np.allclose(f[2], np.sin(omega.numpy() * 0.7) / 0.7, rtol=1e-15)
+    assert np.allclose(f[3], np.sin(omega.numpy() * 5.0) / 5.0, rtol=1e-14, atol=1e-17)
+
+
+# ---------------------------------------------------------------- harmonics
+
+def test_addition_theorem_degrees_0_to_4():
+    u, v = _rand_unitish(200, 1), _rand_unitish(200, 2)
+    Bu, Bv = orc.harmonics(u, 4), orc.harmonics(v, 4)
+    nu, nv = u.norm(dim=1), v.norm(dim=1)
+    c = ((u * v).sum(1) / (nu * nv)).numpy()
+    for l in range(5):
+        lhs = (Bu[l] * Bv[l]).sum(1).numpy()
+        rhs = (nu * nv).numpy() ** l * scipy.special.eval_legendre(l, c)
+        scale = np.maximum(1.0, np.abs(rhs))
+        assert (np.abs(lhs - rhs) / scale).max() < 10 * TOL["addition_theorem"]
+
+
+def test_harmonics_parity_exact():
+    u = _rand_unitish(100, 3)
+    Bp, Bm = orc.harmonics(u, 4), orc.harmonics(-u, 4)
+    for l in range(5):
+        assert torch.equal(Bm[l], (-1) ** l * Bp[l])
+
+
+def test_harmonic_blocks_are_harmonic_and_orthogonal():
+    # Laplacian of each component vanishes (solid harmonics) and distinct components are
+    # orthogonal over the sphere with equal norms 4 pi / (2l+1) (from the addition theorem)
+    xs, ws = np.polynomial.legendre.leggauss(16)
+    ph = (np.arange(32) + 0.5) * (2 * math.pi / 32)
+    ct, phg = np.meshgrid(xs, ph, indexing="ij")
+    st = np.sqrt(1 - ct * ct)
+    u = torch.from_numpy(np.stack([st * np.cos(phg), st * np.sin(phg), ct], -1).reshape(-1, 3))
+    w = torch.from_numpy((ws[:, None] * np.full((1, 32), 2 * math.pi / 32)).reshape(-1))
+    B = orc.harmonics(u, 4)
+    for l in range(5):
+        gram = torch.einsum("p,pa,pb->ab", w, B[l], B[l])
+        assert (gram - torch.eye(2 * l + 1, dtype=torch.float64) * 4 * math.pi / (2 * l + 1)).abs().max() < 1e-13
+    for l1, l2 in itertools.combinations(range(5), 2):
+        assert torch.einsum("p,pa,pb->ab", w, B[l1], B[l2]).abs().max() < 1e-13
+
+
+# ---------------------------------------------------------------- STF map
+
+def test_stf_quadrupolar_form():
+    u = _rand_unitish(100, 4)
+    Q = orc.stf(orc.harmonics(u, 2)[2])
+    s = (u * u).sum(1)
+    ref = math.sqrt(1.5) * (u[:, :, None] * u[:, None, :] - s[:, None, None] / 3 * torch.eye(3, dtype=torch.float64))
+    assert (Q - ref).abs().max() < 10 * TOL["quadrupolar_form"]
+
+
+def test_stf_isometry_symmetric_tracefree():
+    z = torch.from_numpy(_rng(5).standard_normal((100, 5)))
+    z2 = torch.from_numpy(_rng(6).standard_normal((100, 5)))
+    Q, Q2 = orc.stf(z), orc.stf(z2)
+    assert ((Q * Q2).sum((1, 2)) - (z * z2).sum(1)).abs().max() < 10 * TOL["stf_isometry"]
+    assert (Q - Q.transpose(1, 2)).abs().max() == 0
+    assert Q.diagonal(dim1=1, dim2=2).sum(1).abs().max() < 1e-15
+
+
+# ---------------------------------------------------------------- Gaunt couplings
+
+def test_gaunt_unit_norm_and_axis_symmetry():
+    for tr in orc.triples(4):
+        Cc = orc.gaunt_coupling(tr)
+        assert abs(torch.linalg.norm(Cc).item() - 1) < 1e-14
+        if tr[0] == tr[1]:
+            assert (Cc - Cc.permute(1, 0, 2)).abs().max() < 1e-15
+        if tr[1] == tr[2]:
+            assert (Cc - Cc.permute(0, 2, 1)).abs().max() < 1e-15
+
+
+def test_gaunt_rotation_invariant_trilinear_form():
+    # the coupling is an invariant trilinear form: contracting three rotated harmonic
+    # blocks gives the same number as contracting the originals
+    rng = _rng(7)
+    A = rng.standard_normal((3, 3))
+    Rm, _ = np.linalg.qr(A)
+    Rm = torch.from_numpy(Rm * np.sign(np.linalg.det(Rm)))
+    pts = [_rand_unitish(20, 8 + k) for k in range(3)]
+    for tr in orc.triples(4):
+        Cc = orc.gaunt_coupling(tr)
+        a = torch.einsum("abc,na,nb,nc->n", Cc, *[orc.harmonics(p, 4)[l] for p, l in zip(pts, tr)])
+        b = torch.einsum("abc,na,nb,nc->n", Cc, *[orc.harmonics(p @ Rm.T, 4)[l] for p, l in zip(pts, tr)])
+        assert (a - b).abs().max() < 1e-12 * max(1.0, a.abs().max().item())
+
+
+def test_closed_forms_against_gaunt_contraction():
+    rng = _rng(9)
+    v1 = torch.from_numpy(rng.standard_normal((50, 3)))
+    v2 = torch.from_numpy(rng.standard_normal((50, 3)))
+    z = [torch.from_numpy(rng.standard_normal((50, 5))) for _ in range(3)]
+    Q = [orc.stf(t) for t in z]
+    j112 = torch.einsum("abc,na,nb,nc->n", orc.gaunt_coupling((1, 1, 2)), v1, v2, z[0])
+    ref112 = -(1 / math.sqrt(5)) * torch.einsum("na,nab,nb->n", v1, Q[0], v2)
+    assert (j112 - ref112).abs().max() < 10 * TOL["closed_forms_vs_gaunt"]
+    j222 = torch.einsum("abc,na,nb,nc->n", orc.gaunt_coupling((2, 2, 2)), z[0], z[1], z[2])
+    ref222 = -math.sqrt(12 / 35) * torch.einsum("nab,nbc,nca->n", Q[0], Q[1], Q[2])
+    assert (j222 - ref222).abs().max() < 10 * TOL["closed_forms_vs_gaunt"]
+
+
+# ---------------------------------------------------------------- neighbor search
+
+def _python_neighbors(pos, cell, pbc, r_list):
+    """Independent plain-loop search over atoms and images."""
+    N = len(pos)
+    rng_ = orc.image_range(cell, pbc, r_list)
+    rows = []
+    for i in range(N):
+        ent = []
+        for j in range(N):
+            for nx in range(-rng_[0], rng_[0] + 1):
+                for ny in range(-rng_[1], rng_[1] + 1):
+                    for nz in range(-rng_[2], rng_[2] + 1):
+                        if j == i and nx == 0 and ny == 0 and nz == 0:
+                            continue
+                        s = nx * cell[0] + ny * cell[1] + nz * cell[2]
+                        d = (pos[j] + s) - pos[i]
+                        if math.sqrt(float(d @ d)) < r_list:
+                            ent.append((j, nx, ny, nz))
+        rows.append(sorted(ent))
+    return rows
+
+
+@pytest.mark.parametrize("edges,n,r_list", [((4.0, 4.5, 5.0), 6, 6.0), ((9.0, 13.0, 12.5), 14, 6.0),
+                                            ((3.1, 14.0, 7.3), 8, 7.0)])
+def test_neighbor_rows_match_plain_loops(edges, n, r_list):
+    s = make_system(dict(kind="random_box", atoms=n, edges=edges, min_dist=1.2, seed=11, n_types=1,
+                         masses=[1.0], shift=True))
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    assert (pos >= 0).all() and (pos <= np.diag(s["cell"])).all()
+    rows = orc.neighbor_rows(pos, s["cell"], s["pbc"], r_list)
+    ref = _python_neighbors(pos, s["cell"], s["pbc"], r_list)
+    for a, b in zip(rows, ref):
+        assert [tuple(x) for x in a.tolist()] == b
+    # list is symmetric: (i <- j, n) iff (j <- i, -n)
+    have = {(i, *e) for i, r in enumerate(rows) for e in map(tuple, r.tolist())}
+    assert all((j, i, -nx, -ny, -nz) in have for (i, j, nx, ny, nz) in have)
+
+
+def test_neighbor_rows_match_kdtree_counts():
+    s = make_system(dict(kind="random_box", atoms=300, edges=(14.0, 15.0, 16.0), min_dist=1.5, seed=12,
+                         n_types=1, masses=[1.0]))
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    rows = orc.neighbor_rows(pos, s["cell"], s["pbc"], 6.0)
+    tree = cKDTree(pos % np.diag(s["cell"]), boxsize=np.diag(s["cell"]))
+    counts = np.array([len(x) - 1 for x in tree.query_ball_point(pos % np.diag(s["cell"]), 6.0 - 1e-12)])
+    assert (np.array([len(r) for r in rows]) == counts).all()
+
+
+def test_non_periodic_cluster_has_no_images():
+    s = make_system(dict(kind="random_box", atoms=12, edges=(6.0, 6.0, 6.0), min_dist=1.5, seed=13,
+                         n_types=1, masses=[1.0], pbc=[0, 0, 0]))
+    rows = orc.neighbor_rows(s["pos"], s["cell"], s["pbc"], 6.0)
+    assert all((r[:, 1:] == 0).all() for r in rows)
+
+
+# ---------------------------------------------------------------- model-level pins
+
+def _small_case(profile="p16_3_2", n=24, edges=(7.5, 8.0, 9.1), seed=21, pbc=(1, 1, 1), **kw):
+    p = SMALL_PROFILES[profile]
+    blob = make_blob(p, seed=seed, bias_scale=0.3, e_ref_scale=0.5, **kw)
+    s = make_system(dict(kind="random_box", atoms=n, edges=edges, min_dist=1.6, seed=seed + 1,
+                         n_types=p["T"], masses=[1.0] * p["T"], pbc=list(pbc)))
+    return orc.Oracle(blob), s
+
+
+def _raw_descriptors(o, pos, types, cell, pbc):
+    out = o.compute(pos, types, cell, pbc, want_grad=False)
+    return out["D_raw"], out["E_i"]
+
+
+def _random_rotation(seed, proper=True):
+    A = _rng(seed).standard_normal((3, 3))
+    Rm, _ = np.linalg.qr(A)
+    if (np.linalg.det(Rm) > 0) != proper:
+        Rm[:, 0] *= -1
+    return Rm
+
+
+def test_invariance_rotation_translation_permutation():
+    o, s = _small_case()
+    D0, E0 = _raw_descriptors(o, s["pos"], s["types"], s["cell"], s["pbc"])
+    scale = np.abs(D0).max()
+    Rm = _random_rotation(31, proper=True)
+    D1, E1 = _raw_descriptors(o, s["pos"] @ Rm.T, s["types"], s["cell"] @ Rm.T, s["pbc"])
+    assert np.abs(D1 - D0).max() / scale < 20 * TOL["rotation"]
+    t = np.array([0.37, -1.9, 11.3])
+    D2, E2 = _raw_descriptors(o, s["pos"] + t, s["types"], s["cell"], s["pbc"])
+    assert np.abs(D2 - D0).max() / scale < 20 * TOL["translation"]
+    perm = _rng(32).permutation(len(s["pos"]))
+    D3, E3 = _raw_descriptors(o, s["pos"][perm], s["types"][perm], s["cell"], s["pbc"])
+    assert np.abs(D3 - D0[perm]).max() / scale < 20 * TOL["permutation"]
+    for E in (E1, E2):
+        assert np.abs(E - E0).max() < 1e-12 * max(1.0, np.abs(E0).max())
+    assert np.abs(E3 - E0[perm]).max() < 1e-12 * max(1.0, np.abs(E0).max())
+
+
+def test_invariance_improper_rotation_and_inversion_on_cluster():
+    o, s = _small_case(n=12, edges=(6.0, 6.0, 6.0), pbc=(0, 0, 0))
+    D0, E0 = _raw_descriptors(o, s["pos"], s["types"], s["cell"], s["pbc"])
+    D1, _ = _raw_descriptors(o, -s["pos"], s["types"], s["cell"], s["pbc"])
+    assert np.abs(D1 - D0).max() == TOL["inversion"]
+    Rm = _random_rotation(33, proper=False)
+    D2, _ = _raw_descriptors(o, s["pos"] @ Rm.T, s["types"], s["cell"], s["pbc"])
+    assert np.abs(D2 - D0).max() / np.abs(D0).max() < 20 * TOL["rotation"]
+
+
+def test_odd_triple_would_not_be_invariant():
+    # guards the parity selection rule: the (1,1,1) contraction with the Levi-Civita
+    # tensor changes sign under inversion, which is why T_L keeps even sums only
+    assert all(sum(t) % 2 == 0 for t in orc.triples(4))
+
+
+def test_single_aggregation_equals_per_degree_sums():
+    o, s = _small_case()
+    p, prm = o.p, o.prm
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    rows = orc.neighbor_rows(pos, s["cell"], s["pbc"], p["rc"])
+    dst, src, rij = orc.rows_to_edges(rows, np.arange(len(pos)), pos, s["cell"])
+    ty = torch.from_numpy(s["types"].astype(np.int64))
+    dst_t, r = torch.from_numpy(dst), torch.from_numpy(rij)
+    A, s0, s1 = orc.aggregate(p, prm, o.pair, len(pos), dst_t, ty[dst_t], ty[torch.from_numpy(src)], r)
+    # per-centre, per-degree plain loops over that centre's neighbours
+    rho = torch.sqrt((r * r).sum(1) + orc.EPS_REG ** 2)
+    chi = orc.envelope(rho, p["rc"]).numpy()
+    for i in (0, 5, 17):
+        sel = dst == i
+        assert abs(s0[i].item() - (chi[sel] ** 2).sum()) < 1e-14 * max(1, s0[i].item())
+        assert abs(s1[i].item() - (chi[sel] ** 4).sum()) < 1e-14 * max(1, s1[i].item())
+    # order independence: shuffling the edge list leaves the sums unchanged to rounding
+    perm = torch.from_numpy(_rng(41).permutation(len(dst)))
+    A2, s02, s12 = orc.aggregate(p, prm, o.pair, len(pos), dst_t[perm], ty[dst_t][perm],
+                                 ty[torch.from_numpy(src)][perm], r[perm])
+    for a, b in zip(A, A2):
+        assert (a - b).abs().max() < 20 * TOL["single_aggregation"] * max(1.0, a.abs().max().item())
+
+
+def test_zeroed_learned_maps_reduce_to_envelope_sums():
+    # With W_out = 0 and W_p_out = 0: g = 0, gamma = 1, beta = X0_i + X0_j, U = 0, so
+    # psi = beta and A_{0,c} = sum_j chi_j (X0_i + X0_j)_c: pure envelope sums that plain
+    # numpy reproduces from distances alone.
+    p = SMALL_PROFILES["p16_2_0"]
+    blob = bytearray(make_blob(p, seed=50))
+    _, prm = orc.parse_blob(bytes(blob))
+    o = orc.Oracle(bytes(blob))
+    o.prm["W_out"].zero_()
+    o.prm["W_p_out"].zero_()
+    with torch.no_grad():
+        o.pair = orc.pair_modulation(o.p, o.prm)
+    s = make_system(dict(kind="random_box", atoms=20, edges=(8.0, 8.5, 9.0), min_dist=1.6, seed=51,
+                         n_types=p["T"], masses=[1.0] * p["T"]))
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"], want_grad=False)
+    X0 = o.prm["X0"].numpy()
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    C0, C1 = p["C0"], p["C1"]
+    for i in (0, 7, 19):
+        sel = out["dst"] == i
+        d = np.sqrt((out["rij"][sel] ** 2).sum(1))       # eps changes d by 1e-15
+        x = d / p["rc"]
+        chi = 1.0 - scipy.special.betainc(5, 4, np.clip(x, 0, 1))
+        beta = X0[s["types"][i]][None, :] + X0[s["types"][out["src"][sel]]]
+        M0 = math.sqrt(0.25 + (chi ** 2).sum())
+        M1 = math.sqrt(0.25 + (chi ** 4).sum())
+        A0 = (chi[:, None] * beta).sum(0)
+        Dr = out["D_raw"][i]
+        assert np.allclose(Dr[:C0], X0[s["types"][i]], rtol=0, atol=0)
+        assert np.allclose(Dr[C0:2 * C0], A0 / M0, rtol=1e-12, atol=1e-14)
+        assert abs(Dr[2 * C0] - M0) < 1e-13 and abs(Dr[2 * C0 + 1] - M1) < 1e-13
+        # degree one: X_1[m, c] = sum chi^2 beta_c u_m / M1 ; G_1 = X~^T X~ with W_1 as drawn
+        u = out["rij"][sel] / d[:, None]
+        X1 = np.einsum("e,ec,em->mc", chi ** 2, beta[:, :C1], u) / M1
+        Xt = X1 @ (np.eye(C1) + o.prm["W_1"].numpy())
+        G = Xt.T @ Xt
+        vech = [G[a, b] * (1 if a == b else math.sqrt(2)) for a in range(C1) for b in range(a, C1)]
+        got = Dr[2 * C0 + 2:2 * C0 + 2 + len(vech)]
+        assert np.allclose(got, vech, rtol=1e-10, atol=1e-13)
+        # the half-vectorisation preserves the Frobenius norm
+        assert abs(np.linalg.norm(got) - np.linalg.norm(G)) < 1e-12
+
+
+def test_retained_bispectrum_preserves_tensor_norm():
+    rng = _rng(60)
+    K = orc.probe_ranks(128, 3)
+    Z = {l: torch.from_numpy(rng.standard_normal((2 * l + 1, K[l]))) for l in (1, 2, 3)}
+    for tr in orc.triples(3):
+        J = torch.einsum("abc,ai,bj,ck->ijk", orc.gaunt_coupling(tr), Z[tr[0]], Z[tr[1]], Z[tr[2]])
+        kept = torch.stack([J[i, j, k] * w for ((i, j, k), w) in orc.retained_entries(tr, K)])
+        assert abs(kept.norm().item() - J.norm().item()) < 1e-13
+
+
+def test_mlp_residual_layers_with_zero_weights_are_identity():
+    p = dict(SMALL_PROFILES["p16_2_0"])
+    blob = make_blob(p, seed=70, bias_scale=0.2, e_ref_scale=0.4)
+    o, _ = orc.Oracle(blob), None
+    D = torch.from_numpy(_rng(71).standard_normal((5, p["D_out"])))
+    ty = torch.tensor([0, 1, 2, 1, 0])
+    E_full = orc.mlp_energy(o.p, o.prm, D, ty)
+    o.prm["Theta_2"].zero_()
+    o.prm["b_2"].zero_()
+    E_res = orc.mlp_energy(o.p, o.prm, D, ty)
+    p1 = dict(o.p, n_hidden=1)
+    E_one = orc.mlp_energy(p1, o.prm, D, ty)
+    assert (E_res - E_one).abs().max() == 0 and (E_full - E_one).abs().max() > 1e-6
+    # dead first layer: only head bias and reference energy remain
+    o.prm["Theta_1"].zero_()
+    o.prm["b_1"].zero_()
+    E0 = orc.mlp_energy(o.p, o.prm, D, ty)
+    assert (E0 - (o.prm["b_head"][0] + o.prm["E_ref"][ty])).abs().max() == 0
+
+
+def test_first_layer_residual_only_when_widths_agree():
+    p = SMALL_PROFILES["p32_2_0_res"]
+    o = orc.Oracle(make_blob(p, seed=72))
+    D = torch.from_numpy(_rng(73).standard_normal((3, p["D_out"])))
+    ty = torch.zeros(3, dtype=torch.int64)
+    o.prm["Theta_1"].zero_()
+    o.prm["Theta_2"].zero_()
+    E = orc.mlp_energy(o.p, o.prm, D, ty)
+    assert (E - (D @ o.prm["w_head"] + o.prm["b_head"][0])).abs().max() < 1e-14
+
+
+def test_pair_modulation_ranges_and_order():
+    p = SMALL_PROFILES["p32_3_2"]
+    o = orc.Oracle(make_blob(p, seed=74))
+    gamma, beta, U = o.pair
+    assert ((gamma > 0) & (gamma < 2)).all() and (U.abs() < 1).all()
+    X0 = o.prm["X0"]
+    assert ((beta - X0[:, None, :] - X0[None, :, :]).abs() < 1).all()
+    assert (gamma[0, 1] - gamma[1, 0]).abs().max() > 1e-6          # ordered pairs differ
+    assert U.shape == (p["T"], p["T"], p["C0"], p["R"])
+
+
+# ---------------------------------------------------------------- forces and virial
+
+def _energy(o, pos, s, cell=None):
+    return o.compute(pos, s["types"], s["cell"] if cell is None else cell, s["pbc"], want_grad=False)["E"]
+
+
+@pytest.mark.parametrize("profile", ["p16_3_2", "p32_2_4"])
+def test_forces_sum_to_zero_and_match_finite_differences(profile):
+    o, s = _small_case(profile=profile, n=16, edges=(7.0, 7.7, 8.1), seed=80)
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    F = out["F"]
+    assert np.abs(F.sum(0)).max() < 1e-12 * max(1.0, np.abs(F).max())
+    h = 1e-4
+    fscale = np.abs(F).max()
+    for (k, a) in [(0, 0), (3, 1), (7, 2), (15, 0), (9, 1)]:
+        pp, pm = s["pos"].copy(), s["pos"].copy()
+        pp[k, a] += h
+        pm[k, a] -= h
+        fd = -(_energy(o, pp, s) - _energy(o, pm, s)) / (2 * h)
+        assert abs(fd - F[k, a]) < 1e-6 * fscale, (k, a, fd, F[k, a])
+
+
+def test_virial_is_strain_derivative_and_symmetric():
+    o, s = _small_case(profile="p16_3_2", n=16, edges=(7.0, 7.7, 8.1), seed=81)
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    Xi = out["virial"]
+    assert np.abs(Xi - Xi.T).max() < 1e-11 * max(1.0, np.abs(Xi).max())
+    h = 1e-5
+    for a in range(3):
+        for b in range(3):
+            eps = np.zeros((3, 3))
+            eps[a, b] = h
+            Ep = _energy(o, s["pos"] @ (np.eye(3) + eps).T, s, s["cell"] @ (np.eye(3) + eps).T)
+            Em = _energy(o, s["pos"] @ (np.eye(3) - eps).T, s, s["cell"] @ (np.eye(3) - eps).T)
+            dE = (Ep - Em) / (2 * h)
+            assert abs(dE + Xi[a, b]) < 1e-6 * max(1.0, np.abs(Xi).max()), (a, b, dE, Xi[a, b])
+
+
+def test_skin_shell_edges_contribute_nothing():
+    o, s = _small_case(n=16, edges=(7.0, 7.7, 8.1), seed=82)
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    cs = np.arange(len(pos))
+    r0 = orc.neighbor_rows(pos, s["cell"], s["pbc"], o.p["rc"])
+    r1 = orc.neighbor_rows(pos, s["cell"], s["pbc"], o.p["rc"] + 1.0)
+    assert sum(map(len, r1)) > sum(map(len, r0))
+    E0 = o.evaluate_rows(pos, s["types"], s["cell"], r0, cs, want_grad=False)[0]
+    E1 = o.evaluate_rows(pos, s["types"], s["cell"], r1, cs, want_grad=False)[0]
+    assert np.abs(E0 - E1).max() < 1e-13 * max(1.0, np.abs(E0).max())
+
+
+def test_force_on_single_atom_matches_whole_system():
+    o, s = _small_case(n=20, edges=(12.5, 13.0, 12.2), seed=83)
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    Fk, Ei = o.force_on(s["pos"], s["types"], s["cell"], s["pbc"], 4)
+    assert np.abs(Fk - out["F"][4]).max() < 1e-12 * max(1.0, np.abs(out["F"]).max())
+    assert abs(Ei[4] - out["E_i"][4]) < 1e-13 * max(1.0, abs(out["E_i"][4]))
