@@ -1,0 +1,191 @@
+/*
+ * umlmd.h -- C ABI of libumlmd: energy, force and virial evaluation of the DPA4C
+ * machine-learning interatomic potential on one NVIDIA B200 (sm_100a), plus a
+ * velocity-Verlet NVE driver.
+ *
+ * Conventions
+ *   - Every function returns an int status: UMLMD_OK (0) or a negative UMLMD_E_* code.
+ *     Nothing throws, aborts or traps on the device.  umlmd_last_error() returns a
+ *     human-readable message for the last failure on a handle.
+ *   - Pointers whose name starts with d_ are CUDA device pointers owned by the caller
+ *     (for instance a torch tensor's data_ptr()); every other pointer is host memory.
+ *     The library never frees or keeps caller memory beyond the call, except the MD state
+ *     registered with umlmd_set_md_state, which must stay valid until it is replaced or
+ *     the handle is destroyed.
+ *   - The handle owns the model constants and all workspace; it allocates device memory
+ *     in the first umlmd_build_neighbors call and grows it there when a system needs more.
+ *   - All work is enqueued on the CUDA stream given to umlmd_create.  Calls that return
+ *     host values (energy, virial, counts) synchronise that stream before returning.
+ *   - Units are "metal": Angstrom, eV, ps, amu, K.  Species are 0-based indices into the
+ *     blob's type table.
+ *   - Arrays are row-major.  Positions, velocities and forces are double [N][3].
+ */
+#ifndef UMLMD_H
+#define UMLMD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct umlmd umlmd_t;
+
+enum {
+    UMLMD_OK = 0,
+    UMLMD_E_INVALID_ARG = -1,         /* NULL pointer, negative size, bad option            */
+    UMLMD_E_BAD_BLOB = -2,            /* magic / version / size mismatch, non-finite weight */
+    UMLMD_E_UNSUPPORTED_PROFILE = -3, /* C0 not in {8,16,32,64,128}, L not in {2,3},
+                                         R not in {0,2,4,8}, F % 4 != 0, ...                */
+    UMLMD_E_UNSUPPORTED_CELL = -4,    /* non-orthorhombic cell, non-positive edge           */
+    UMLMD_E_NO_NEIGHBORS = -5,        /* compute/step called before build_neighbors         */
+    UMLMD_E_STALE_NEIGHBORS = -6,     /* an atom moved more than skin/2 since the build     */
+    UMLMD_E_NONFINITE = -7,           /* NaN or Inf in positions, energy or forces          */
+    UMLMD_E_CUDA = -8,                /* a CUDA runtime call failed (message has details)   */
+    UMLMD_E_CAPACITY = -9,            /* caller buffer too small (see umlmd_get_neighbors)  */
+    UMLMD_E_NO_MD_STATE = -10         /* step called before set_md_state                    */
+};
+
+/* Optional settings for umlmd_create.  Zero-initialise, set struct_bytes = sizeof, then
+ * override fields; a zero field means "default". */
+typedef struct umlmd_options {
+    uint32_t struct_bytes;
+    double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
+    int32_t  node_tile;  /* atoms per workspace tile; 0 = 131072                            */
+    int32_t  mlp_path;   /* 0 = default, 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM  */
+} umlmd_options;
+
+/* Structural widths of a model, all derived from (C0, L, R) by the paper's formulas
+ * (degree-wise channel widths, probe ranks, feature-state width S, feature-vector width
+ * D_out, gated hidden widths H and H_pair). */
+typedef struct umlmd_info {
+    int32_t C0, L, R, N_rbf, n_hidden, F, T;
+    int32_t C1, C2, K1, K2, S, D_out, H, H_pair;
+    int32_t table_rows;
+    double  rc, table_dx;
+    int64_t n_atoms, n_edges;          /* of the current neighbor list (0 before a build)  */
+    int64_t device_bytes;              /* device memory currently held by the handle       */
+} umlmd_info;
+
+/* Widths for a (C0, L, R) triple without a handle; fills only the width fields.
+ * Returns UMLMD_E_UNSUPPORTED_PROFILE for an unsupported triple. */
+int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out);
+
+/*
+ * Create a model from a weight blob (host memory, little-endian):
+ *   char[8] "UMLMD1\0\0"; u32 version = 1; u32 C0, L, R, N_rbf, n_hidden, F, T, basis (0 =
+ *   Bessel); f64 rc, table_dx; then float32 arrays, row-major, y = x W convention:
+ *   X0[T,C0], omega[N_rbf], W_in[N_rbf,2H], W_out[H,C0], W_mode[H,R], W_p_in[2C0,2Hp],
+ *   W_p_out[Hp,C0(2+R)] (column blocks scale|shift|mode), W_1[C1,C1], W_2[C2,C2],
+ *   A_1[C1,K1], A_2[C2,K2], mu[D_out], sigma[D_out], Theta_1[D_out,F], b_1[F],
+ *   {Theta_t[F,F], b_t[F]} t = 2..n_hidden, w_head[F], b_head, E_ref[T].
+ * The create step evaluates, once and in double precision on the host, everything the
+ * paper's compressed inference precomputes: the quintic-Hermite radial table of the shared
+ * radial map and modes on [0, rc] (value, first and second derivative at each knot), the
+ * ordered type-pair scale / shift / mode-mixing cache, and the unit-norm Gaunt coupling
+ * tensors of the admissible degree triples.
+ *   stream: a cudaStream_t passed as void* (NULL = the default stream).
+ * umlmd_create itself touches no device: the constants are uploaded by the first
+ * umlmd_build_neighbors call, so creation and the host-side diagnostics below also work on
+ * a machine without a GPU.
+ */
+int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, void* stream,
+                 umlmd_t** out);
+int umlmd_destroy(umlmd_t* h);
+int umlmd_query(const umlmd_t* h, umlmd_info* out);
+const char* umlmd_last_error(const umlmd_t* h);
+
+/*
+ * Build the directed neighbor graph of the paper's neighbor-set definition with list
+ * radius r_list = rc + skin: edge (i <- j, n) exists iff (j, n) != (i, 0) and
+ * |(r_j + n.cell) - r_i|^2 < r_list^2 (true distance, strict), periodic images being
+ * distinct neighbor instances, both orientations stored, no capacity limit.
+ *   d_pos   [N,3] double, any image of each atom; folded into the cell internally with
+ *           frac - floor(frac) along periodic directions (n refers to folded positions)
+ *   d_type  [N] int32 species
+ *   cell    9 doubles, rows are cell vectors; must be orthorhombic (diagonal)
+ *   pbc     3 ints, non-zero = periodic along that cell vector
+ *   skin    extra list radius in Angstrom (>= 0); edges beyond rc carry zero weight
+ * The predicate is evaluated in double precision as ((xj + n*L) - xi), d2 = (dx*dx +
+ * dy*dy) + dz*dz, d2 < r_list*r_list, without fused multiply-add, so that the edge set is
+ * reproducible bit for bit.  Atoms are renumbered internally in cell order; all outputs
+ * of this library are in the caller's numbering.
+ */
+int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type,
+                          const double cell[9], const int pbc[3], double skin);
+
+/*
+ * Copy the current neighbor list out in the caller's atom numbering (for verification).
+ *   d_row_ptr [N+1] int32, d_src [cap] int32, d_shift [cap,3] int8; row i holds the
+ *   neighbor instances (j, n) of centre i in no particular order.
+ * Pass cap = 0 (pointers may be NULL) to only query *n_edges.  UMLMD_E_CAPACITY if the
+ * list has more than cap edges.
+ */
+int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
+                        int64_t cap, int64_t* n_edges);
+
+/*
+ * Energy, forces and virial for positions d_pos [N,3] (same atoms, species and cell as
+ * the last build; each atom within skin/2 of where it was at the build, else
+ * UMLMD_E_STALE_NEIGHBORS).
+ *   energy         host, eV: sum of atomic energies (MLP output + per-species reference)
+ *   d_force        [N,3] double, eV/Angstrom: F_k = sum_{j in N_k} g_kj - sum_{i: k in N_i} g_ik
+ *                  with g_ij = dE/dr_ij; may be NULL
+ *   virial         host, 9 doubles, eV: Xi_ab = - sum_edges g_a r_b; may be NULL
+ *   d_atom_energy  [N] double, eV; may be NULL
+ * The whole chain runs in the library's CUDA kernels: per-edge radial table / pair
+ * modulation / envelope / harmonics and per-destination aggregation, polynomial
+ * invariants, the residual SiLU MLP, its vector-Jacobian product, the invariant
+ * vector-Jacobian product, the edge recomputation pass and the atomic-free force and
+ * virial assembly.
+ */
+int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_force,
+                  double virial[9], double* d_atom_energy);
+
+/*
+ * Register MD state for umlmd_step: d_pos and d_vel [N,3] double (Angstrom, Angstrom/ps)
+ * are advanced in place; mass_per_type is T doubles (amu, host; copied).  N, species and
+ * cell are those of the last umlmd_build_neighbors call.
+ */
+int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* mass_per_type);
+
+/*
+ * Advance nsteps of velocity-Verlet NVE with time step dt_ps.  The neighbor list is
+ * rebuilt (with the skin of the last build) every rebuild_every steps, counted from the
+ * last build; rebuild_every <= 0 never rebuilds.  On return e_pot / e_kin (host, eV; may
+ * be NULL) hold the potential and kinetic energy after the last step.
+ */
+int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* e_pot,
+               double* e_kin);
+
+/*
+ * Diagnostics used by the parity tests: copy out per-atom intermediates of the last
+ * umlmd_compute, in the caller's numbering.  Each pointer may be NULL.
+ *   d_state  [N, S+2] float: unnormalised sums A (degree, then m, then channel), s0, s1
+ *   d_desc   [N, D_out] float: calibrated feature vector D
+ * Only valid when N <= node tile (single-tile evaluation); otherwise UMLMD_E_CAPACITY.
+ * These hold forward values only if umlmd_compute was called with d_force == NULL and
+ * virial == NULL (the backward pass reuses both buffers).
+ */
+int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc);
+
+/*
+ * Evaluate the tabulated radial map at n distances (host arrays): out_g [n, C0+R] holds
+ * g(rho) then q(rho), out_dg their derivatives, from the same quintic polynomials the
+ * kernels use (evaluated on the host from the device table's float32 coefficients).
+ */
+int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, double* out_g,
+                            double* out_dg);
+
+/*
+ * Read one entry of the ordered type-pair cache (host): out receives (2+R)*C0 doubles,
+ * the scale gamma[C0], the shift beta[C0], then the mode mixing as R rows U[:, mu] of C0
+ * values, for centre species type_i and neighbour species type_j.
+ */
+int umlmd_eval_pair_cache(const umlmd_t* h, int32_t type_i, int32_t type_j, double* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UMLMD_H */

@@ -1,0 +1,234 @@
+"""Thin ctypes binding of libumlmd.so: argument marshalling only.
+
+Every computation runs inside the library's CUDA kernels.  Importing this module loads the
+shared library and fails loudly if it has not been built
+(``python -m paper_2608_19041_b200.build``); there is no fallback path.
+"""
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libumlmd.so")
+
+OK = 0
+ERRORS = {
+    -1: "INVALID_ARG", -2: "BAD_BLOB", -3: "UNSUPPORTED_PROFILE", -4: "UNSUPPORTED_CELL",
+    -5: "NO_NEIGHBORS", -6: "STALE_NEIGHBORS", -7: "NONFINITE", -8: "CUDA", -9: "CAPACITY",
+    -10: "NO_MD_STATE",
+}
+
+EXPORTS = [
+    "umlmd_profile_widths", "umlmd_create", "umlmd_destroy", "umlmd_query", "umlmd_last_error",
+    "umlmd_build_neighbors", "umlmd_get_neighbors", "umlmd_compute", "umlmd_set_md_state", "umlmd_step",
+    "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache",
+]
+
+
+class UmlmdError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__(f"{ERRORS.get(code, code)}: {message}")
+        self.code = code
+
+
+class Options(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_uint32), ("table_dx", ctypes.c_double),
+                ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32)]
+
+
+class Info(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T", "C1", "C2", "K1", "K2", "S", "D_out", "H",
+                 "H_pair", "table_rows")] + \
+               [("rc", ctypes.c_double), ("table_dx", ctypes.c_double), ("n_atoms", ctypes.c_int64),
+                ("n_edges", ctypes.c_int64), ("device_bytes", ctypes.c_int64)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+def load_library(path=_LIB_PATH):
+    if not os.path.exists(path):
+        raise ImportError(f"{path} not found: build it with `python -m paper_2608_19041_b200.build`")
+    lib = ctypes.CDLL(path)
+    vp, i64, i32, dbl = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double
+    lib.umlmd_profile_widths.argtypes = [i32, i32, i32, ctypes.POINTER(Info)]
+    lib.umlmd_create.argtypes = [vp, ctypes.c_size_t, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
+    lib.umlmd_destroy.argtypes = [vp]
+    lib.umlmd_query.argtypes = [vp, ctypes.POINTER(Info)]
+    lib.umlmd_last_error.argtypes = [vp]
+    lib.umlmd_last_error.restype = ctypes.c_char_p
+    lib.umlmd_build_neighbors.argtypes = [vp, i64, vp, vp, ctypes.POINTER(dbl), ctypes.POINTER(ctypes.c_int), dbl]
+    lib.umlmd_get_neighbors.argtypes = [vp, vp, vp, vp, i64, ctypes.POINTER(i64)]
+    lib.umlmd_compute.argtypes = [vp, vp, ctypes.POINTER(dbl), vp, ctypes.POINTER(dbl), vp]
+    lib.umlmd_set_md_state.argtypes = [vp, vp, vp, ctypes.POINTER(dbl)]
+    lib.umlmd_step.argtypes = [vp, ctypes.c_int, dbl, ctypes.c_int, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.umlmd_get_intermediates.argtypes = [vp, vp, vp]
+    lib.umlmd_eval_radial_table.argtypes = [vp, i64, ctypes.POINTER(dbl), ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.umlmd_eval_pair_cache.argtypes = [vp, i32, i32, ctypes.POINTER(dbl)]
+    for name in EXPORTS:
+        if name != "umlmd_last_error":
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = load_library()
+    return _lib
+
+
+def profile_widths(C0, L, R=0):
+    info = Info()
+    rc = lib().umlmd_profile_widths(C0, L, R, ctypes.byref(info))
+    if rc != OK:
+        raise UmlmdError(rc, f"unsupported profile ({C0}, {L}, {R})")
+    return {k: v for k, v in info.as_dict().items() if k in
+            ("C1", "C2", "K1", "K2", "S", "D_out", "H", "H_pair")}
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _check_dev(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+
+
+class Model:
+    """A DPA4C model on the current CUDA device, created from a weight blob."""
+
+    def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, stream=None):
+        self._lib = lib()
+        self._h = ctypes.c_void_p()
+        opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path))
+        # creation is host-only; a stream is only meaningful when a device is present
+        self._stream = stream if stream is not None else (
+            torch.cuda.current_stream() if torch.cuda.is_available() else None)
+        stream_ptr = ctypes.c_void_p(self._stream.cuda_stream if self._stream is not None else 0)
+        buf = (ctypes.c_char * len(blob)).from_buffer_copy(blob)
+        rc = self._lib.umlmd_create(buf, len(blob), ctypes.byref(opt), stream_ptr,
+                                    ctypes.byref(self._h))
+        if rc != OK:
+            self._h = ctypes.c_void_p()
+            raise UmlmdError(rc, "umlmd_create failed (bad blob or unsupported profile)")
+        self._keep = []
+        self.n_atoms = 0
+
+    def _raise(self, rc):
+        raise UmlmdError(rc, self._lib.umlmd_last_error(self._h).decode())
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            self._lib.umlmd_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def query(self):
+        info = Info()
+        rc = self._lib.umlmd_query(self._h, ctypes.byref(info))
+        if rc != OK:
+            self._raise(rc)
+        return info.as_dict()
+
+    def build_neighbors(self, pos, types, cell, pbc=(1, 1, 1), skin=0.0):
+        _check_dev(pos, torch.float64, "pos")
+        _check_dev(types, torch.int32, "types")
+        n = pos.shape[0]
+        cell9 = (ctypes.c_double * 9)(*np.asarray(cell, dtype=np.float64).reshape(9))
+        pbc3 = (ctypes.c_int * 3)(*[int(x) for x in pbc])
+        rc = self._lib.umlmd_build_neighbors(self._h, n, _ptr(pos), _ptr(types), cell9, pbc3, float(skin))
+        if rc != OK:
+            self._raise(rc)
+        self.n_atoms = n
+
+    def get_neighbors(self):
+        """(row_ptr [N+1], src [E], shift [E,3]) as CUDA tensors, caller numbering."""
+        ne = ctypes.c_int64()
+        rc = self._lib.umlmd_get_neighbors(self._h, None, None, None, 0, ctypes.byref(ne))
+        if rc != OK:
+            self._raise(rc)
+        E = ne.value
+        row_ptr = torch.empty(self.n_atoms + 1, dtype=torch.int32, device="cuda")
+        src = torch.empty(max(E, 1), dtype=torch.int32, device="cuda")
+        shift = torch.empty((max(E, 1), 3), dtype=torch.int8, device="cuda")
+        rc = self._lib.umlmd_get_neighbors(self._h, _ptr(row_ptr), _ptr(src), _ptr(shift), max(E, 1), ctypes.byref(ne))
+        if rc != OK:
+            self._raise(rc)
+        return row_ptr, src[:E], shift[:E]
+
+    def compute(self, pos, forces=True, virial=True, atom_energy=False):
+        """Returns dict(energy=float, forces=CUDA tensor or None, virial=np [3,3] or None,
+        atom_energy=CUDA tensor or None)."""
+        _check_dev(pos, torch.float64, "pos")
+        n = self.n_atoms
+        e = ctypes.c_double()
+        f = torch.empty((n, 3), dtype=torch.float64, device="cuda") if forces else None
+        ea = torch.empty(n, dtype=torch.float64, device="cuda") if atom_energy else None
+        vir = (ctypes.c_double * 9)() if virial else None
+        rc = self._lib.umlmd_compute(self._h, _ptr(pos), ctypes.byref(e), _ptr(f), vir, _ptr(ea))
+        if rc != OK:
+            self._raise(rc)
+        return dict(energy=e.value, forces=f, atom_energy=ea,
+                    virial=np.array(list(vir), dtype=np.float64).reshape(3, 3) if virial else None)
+
+    def set_md_state(self, pos, vel, masses):
+        _check_dev(pos, torch.float64, "pos")
+        _check_dev(vel, torch.float64, "vel")
+        m = np.asarray(masses, dtype=np.float64)
+        arr = (ctypes.c_double * len(m))(*m)
+        rc = self._lib.umlmd_set_md_state(self._h, _ptr(pos), _ptr(vel), arr)
+        if rc != OK:
+            self._raise(rc)
+        self._keep = [pos, vel]
+
+    def step(self, nsteps, dt_ps, rebuild_every=0):
+        ep, ek = ctypes.c_double(), ctypes.c_double()
+        rc = self._lib.umlmd_step(self._h, int(nsteps), float(dt_ps), int(rebuild_every), ctypes.byref(ep),
+                                  ctypes.byref(ek))
+        if rc != OK:
+            self._raise(rc)
+        return ep.value, ek.value
+
+    def get_intermediates(self):
+        q = self.query()
+        state = torch.empty((self.n_atoms, q["S"] + 2), dtype=torch.float32, device="cuda")
+        desc = torch.empty((self.n_atoms, q["D_out"]), dtype=torch.float32, device="cuda")
+        rc = self._lib.umlmd_get_intermediates(self._h, _ptr(state), _ptr(desc))
+        if rc != OK:
+            self._raise(rc)
+        return state, desc
+
+    def eval_pair_cache(self, type_i, type_j):
+        q = self.query()
+        out = np.empty(((2 + q["R"]), q["C0"]), dtype=np.float64)
+        rc = self._lib.umlmd_eval_pair_cache(self._h, int(type_i), int(type_j),
+                                             out.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
+        if rc != OK:
+            self._raise(rc)
+        return out
+
+    def eval_radial_table(self, rho):
+        rho = np.ascontiguousarray(rho, dtype=np.float64)
+        q = self.query()
+        nc = q["C0"] + q["R"]
+        g = np.empty((len(rho), nc), dtype=np.float64)
+        dg = np.empty((len(rho), nc), dtype=np.float64)
+        P = ctypes.POINTER(ctypes.c_double)
+        rc = self._lib.umlmd_eval_radial_table(self._h, len(rho), rho.ctypes.data_as(P), g.ctypes.data_as(P),
+                                               dg.ctypes.data_as(P))
+        if rc != OK:
+            self._raise(rc)
+        return g, dg

@@ -1,0 +1,409 @@
+// extern "C" entry points of libumlmd (see include/umlmd.h for the contract).
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "alloc.h"
+#include "kernels.h"
+#include "model.h"
+
+using namespace umd;
+
+struct umlmd {
+    HostModel hm;
+    ModelDev md{};
+    Dims d{};
+    cudaStream_t st = nullptr;
+    std::string err;
+    NeighborDev nb;
+    int node_tile = 131072;
+    int mlp_path = 1;
+    bool have_list = false;
+    bool on_device = false;
+    std::vector<void*> model_allocs;
+    // workspace
+    float* state = nullptr; float* desc = nullptr; float* pre = nullptr; float* hbuf = nullptr;
+    int64_t tile_cap = 0;
+    float* g = nullptr; int64_t g_cap = 0;
+    double* e_atom = nullptr; double* f_sorted = nullptr; int* type_o = nullptr; int64_t n_cap = 0;
+    double* virial_part = nullptr; int64_t vpart_cap = 0;
+    double* scratch = nullptr; double* d_out = nullptr; int* d_err = nullptr;
+    double* h_out = nullptr; int* h_err = nullptr;      // pinned
+    // MD
+    double* md_pos = nullptr; double* md_vel = nullptr; double* md_force = nullptr; int64_t md_cap = 0;
+    double* d_mass = nullptr; double* d_inv_mass = nullptr;
+    bool have_md = false, have_force = false;
+    int steps_since_build = 0;
+};
+
+namespace {
+
+int fail(umlmd_t* h, int code, const std::string& msg) {
+    if (h) h->err = msg;
+    return code;
+}
+
+#define API_CUDA(h, call)                                                                     \
+    do {                                                                                      \
+        cudaError_t e__ = (call);                                                             \
+        if (e__ != cudaSuccess)                                                               \
+            return fail(h, UMLMD_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__)); \
+    } while (0)
+
+template <typename T>
+cudaError_t upload(umlmd_t* h, const std::vector<T>& v, T** out) {
+    *out = nullptr;
+    void* p = nullptr;
+    cudaError_t e = dev_malloc(&p, v.size() * sizeof(T) + 16);
+    if (e != cudaSuccess) return e;
+    h->model_allocs.push_back(p);
+    if (!v.empty()) e = cudaMemcpyAsync(p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice, h->st);
+    *out = static_cast<T*>(p);
+    return e;
+}
+
+void fill_info(const Dims& d, umlmd_info* o) {
+    o->C0 = d.C0; o->L = d.L; o->R = d.R; o->N_rbf = d.N_rbf; o->n_hidden = d.n_hidden; o->F = d.F; o->T = d.T;
+    o->C1 = d.C[1]; o->C2 = d.C[2]; o->K1 = d.K[1]; o->K2 = d.K[2]; o->S = d.S; o->D_out = d.D_out;
+    o->H = d.H; o->H_pair = d.Hp; o->table_rows = d.n_rows;
+}
+
+int ensure_workspace(umlmd_t* h) {
+    const Dims& d = h->d;
+    const int64_t N = h->nb.N, E = h->nb.E;
+    const int64_t B = N < h->node_tile ? N : h->node_tile;
+    if (B > h->tile_cap || !h->state) {
+        int64_t c;
+        c = 0; API_CUDA(h, dev_ensure(&h->state, &c, B * d.SP));
+        c = 0; API_CUDA(h, dev_ensure(&h->desc, &c, B * d.DP));
+        c = 0; API_CUDA(h, dev_ensure(&h->pre, &c, B * d.F * d.n_hidden));
+        c = 0; API_CUDA(h, dev_ensure(&h->hbuf, &c, B * d.F * 2));
+        h->tile_cap = B;
+    }
+    if (E > h->g_cap || !h->g) { API_CUDA(h, dev_ensure(&h->g, &h->g_cap, E * 3, 1.1)); h->g_cap /= 3; }
+    if (N > h->n_cap || !h->e_atom) {
+        int64_t c;
+        c = 0; API_CUDA(h, dev_ensure(&h->e_atom, &c, N));
+        c = 0; API_CUDA(h, dev_ensure(&h->f_sorted, &c, N * 3));
+        c = 0; API_CUDA(h, dev_ensure(&h->type_o, &c, N));
+        h->n_cap = N;
+    }
+    const int64_t n_tiles = B > 0 ? (N + B - 1) / B : 0;
+    const int64_t vneed = (N / 8 + n_tiles + 2) * 9;
+    if (vneed > h->vpart_cap || !h->virial_part) API_CUDA(h, dev_ensure(&h->virial_part, &h->vpart_cap, vneed));
+    return UMLMD_OK;
+}
+
+int decode_device_errors(umlmd_t* h, int word) {
+    if (word & kErrNonFinite) return fail(h, UMLMD_E_NONFINITE, "non-finite value in positions, energy or forces");
+    if (word & kErrShiftRange) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "periodic image index outside [-127, 127]");
+    if (word & kErrStale)
+        return fail(h, UMLMD_E_STALE_NEIGHBORS, "an atom moved more than skin/2 since the neighbor list was built");
+    return UMLMD_OK;
+}
+
+// enqueue one full evaluation; results stay on the device (d_out[0] energy, d_out[1..9] virial)
+int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_force, double* d_atom_energy) {
+    const Dims& d = h->d;
+    NeighborDev& nb = h->nb;
+    const int N = (int)nb.N;
+    API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st));
+    const int B = N < h->node_tile ? N : h->node_tile;
+    int vpart_used = 0;
+    for (int a0 = 0; a0 < N; a0 += B) {
+        const int n = N - a0 < B ? N - a0 : B;
+        EdgeArgs ea;
+        ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.type_s = nb.type_s;
+        ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
+        ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
+        ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
+        ea.virial_part = h->virial_part + (size_t)vpart_used * 9;
+        API_CUDA(h, launch_edge_forward(ea, h->st));
+        InvArgs ia;
+        ia.d = d; ia.m = h->md; ia.type_s = nb.type_s; ia.a0 = a0; ia.n = n; ia.state = h->state; ia.desc = h->desc;
+        API_CUDA(h, launch_invariants_forward(ia, h->st));
+        MlpArgs ma;
+        ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
+        ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
+        API_CUDA(h, launch_mlp(ma, h->st));
+        if (want_grad) {
+            API_CUDA(h, launch_invariants_backward(ia, h->st));
+            int blocks = 0;
+            API_CUDA(h, launch_edge_backward(ea, &blocks, h->st));
+            vpart_used += blocks;
+        }
+    }
+    if (want_grad) {
+        API_CUDA(h, launch_force_assembly(nb, h->g, h->f_sorted, h->st));
+        if (d_force) API_CUDA(h, launch_scatter_forces(nb, h->f_sorted, d_force, h->d_err, h->st));
+    }
+    API_CUDA(h, launch_reduce_energy_virial(h->e_atom, N, h->virial_part, vpart_used, h->scratch, h->d_out,
+                                            h->d_err, h->st));
+    if (d_atom_energy) API_CUDA(h, launch_scatter_atom_energy(nb, h->e_atom, d_atom_energy, h->st));
+    return UMLMD_OK;
+}
+
+// copy results and the error word to the host, synchronise, clear the error word
+int fetch_results(umlmd_t* h, int n_out) {
+    API_CUDA(h, cudaMemcpyAsync(h->h_out, h->d_out, sizeof(double) * n_out, cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    return decode_device_errors(h, *h->h_err);
+}
+
+// first use on a device: upload the model constants and allocate the small result buffers
+int ensure_device_model(umlmd_t* h) {
+    if (h->on_device) return UMLMD_OK;
+    const HostModel& m = h->hm;
+    ModelDev& md = h->md;
+    cudaError_t e = cudaSuccess;
+    auto up = [&](const std::vector<float>& v, float** p) { if (e == cudaSuccess) e = upload(h, v, p); };
+    up(m.table, &md.table); up(m.pairmod, &md.pairmod); up(m.X0, &md.X0); up(m.W1p, &md.W1p); up(m.W2p, &md.W2p);
+    up(m.A1, &md.A1); up(m.A2, &md.A2); up(m.mu, &md.mu); up(m.inv_sigma, &md.inv_sigma);
+    for (int t = 0; t < h->d.n_hidden; ++t) { up(m.theta[t], &md.theta[t]); up(m.thetaT[t], &md.thetaT[t]); up(m.bias[t], &md.bias[t]); }
+    up(m.w_head, &md.w_head); up(m.e_ref, &md.e_ref);
+    md.b_head = m.b_head;
+    if (e == cudaSuccess && h->d.L >= 3) {
+        std::vector<GauntSparse> g1(1, m.g123), g2(1, m.g233);
+        e = upload(h, g1, &md.g123);
+        if (e == cudaSuccess) e = upload(h, g2, &md.g233);
+    }
+    void* p = nullptr;
+    if (e == cudaSuccess) { e = dev_malloc(&p, sizeof(double) * (reduce_scratch_doubles(0) + 16)); h->scratch = (double*)p; }
+    if (e == cudaSuccess) { e = dev_malloc(&p, sizeof(double) * 16); h->d_out = (double*)p; }
+    if (e == cudaSuccess) { e = dev_malloc(&p, sizeof(int) * 4); h->d_err = (int*)p; }
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->d_err, 0, sizeof(int) * 4, h->st);
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&h->h_out, sizeof(double) * 16);
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&h->h_err, sizeof(int) * 4);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->st);
+    if (e != cudaSuccess) return fail(h, UMLMD_E_CUDA, std::string("model upload: ") + cudaGetErrorString(e));
+    h->on_device = true;
+    return UMLMD_OK;
+}
+
+int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type, const double L[3],
+               const int pbc[3], double skin) {
+    int rc = ensure_device_model(h);
+    if (rc != UMLMD_OK) return rc;
+    rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err);
+    if (rc != UMLMD_OK) { h->have_list = false; return rc; }
+    h->have_list = true;
+    h->steps_since_build = 0;
+    return ensure_workspace(h);
+}
+
+}  // namespace
+
+extern "C" {
+
+int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out) {
+    if (!out) return UMLMD_E_INVALID_ARG;
+    Dims d;
+    if (!derive_dims(C0, L, R, &d)) return UMLMD_E_UNSUPPORTED_PROFILE;
+    std::memset(out, 0, sizeof(*out));
+    fill_info(d, out);
+    return UMLMD_OK;
+}
+
+int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, void* stream, umlmd_t** out) {
+    if (!blob || !out) return UMLMD_E_INVALID_ARG;
+    *out = nullptr;
+    umlmd_t* h = new (std::nothrow) umlmd();
+    if (!h) return UMLMD_E_INVALID_ARG;
+    h->st = static_cast<cudaStream_t>(stream);
+    double dx_override = 0;
+    if (opt) {
+        if (opt->struct_bytes != sizeof(umlmd_options)) { delete h; return UMLMD_E_INVALID_ARG; }
+        if (opt->table_dx < 0 || opt->node_tile < 0 || opt->mlp_path < 0 || opt->mlp_path > 2) { delete h; return UMLMD_E_INVALID_ARG; }
+        dx_override = opt->table_dx;
+        if (opt->node_tile > 0) h->node_tile = opt->node_tile;
+        if (opt->mlp_path > 0) h->mlp_path = opt->mlp_path;
+    }
+    int rc = build_host_model(blob, blob_bytes, dx_override, &h->hm, &h->err);
+    if (rc != UMLMD_OK) { delete h; return rc; }
+    h->d = h->hm.d;
+    *out = h;
+    return UMLMD_OK;
+}
+
+int umlmd_destroy(umlmd_t* h) {
+    if (!h) return UMLMD_OK;
+    if (h->on_device) cudaStreamSynchronize(h->st);
+    for (void* p : h->model_allocs) dev_free(p);
+    neighbor_free(&h->nb);
+    void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
+                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass};
+    for (void* p : ptrs) dev_free(p);
+    if (h->h_out) cudaFreeHost(h->h_out);
+    if (h->h_err) cudaFreeHost(h->h_err);
+    delete h;
+    return UMLMD_OK;
+}
+
+int umlmd_query(const umlmd_t* h, umlmd_info* out) {
+    if (!h || !out) return UMLMD_E_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    fill_info(h->d, out);
+    out->rc = h->hm.rc; out->table_dx = h->hm.dx;
+    out->n_atoms = h->have_list ? h->nb.N : 0;
+    out->n_edges = h->have_list ? h->nb.E : 0;
+    out->device_bytes = dev_bytes_held();
+    return UMLMD_OK;
+}
+
+const char* umlmd_last_error(const umlmd_t* h) { return h ? h->err.c_str() : "null handle"; }
+
+int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type, const double cell[9],
+                          const int pbc[3], double skin) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (N < 0 || !cell || !pbc || !(skin >= 0) || !std::isfinite(skin) || (N > 0 && (!d_pos || !d_type)))
+        return fail(h, UMLMD_E_INVALID_ARG, "bad argument to umlmd_build_neighbors");
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) {
+            const double v = cell[3 * i + j];
+            if (!std::isfinite(v)) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "non-finite cell");
+            if (i != j && v != 0.0) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "only orthorhombic cells are supported");
+            if (i == j && !(v > 0.0)) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "cell edges must be positive");
+        }
+    const double L[3] = {cell[0], cell[4], cell[8]};
+    h->have_md = false;
+    int rc = build_list(h, N, d_pos, d_type, L, pbc, skin);
+    if (rc != UMLMD_OK) return rc;
+    if (N > 0) API_CUDA(h, cudaMemcpyAsync(h->type_o, d_type, sizeof(int) * N, cudaMemcpyDeviceToDevice, h->st));
+    // surface device-side findings of the build (non-finite positions, image range)
+    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    rc = decode_device_errors(h, *h->h_err);
+    if (rc != UMLMD_OK) h->have_list = false;
+    return rc;
+}
+
+int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift, int64_t cap,
+                        int64_t* n_edges) {
+    if (!h || !n_edges) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "no neighbor list built");
+    *n_edges = h->nb.E;
+    if (cap == 0) return UMLMD_OK;
+    if (cap < h->nb.E) return fail(h, UMLMD_E_CAPACITY, "edge buffers smaller than the list");
+    if (!d_row_ptr || (h->nb.E > 0 && (!d_src || !d_shift))) return fail(h, UMLMD_E_INVALID_ARG, "null output buffer");
+    int rc = neighbor_export(&h->nb, d_row_ptr, d_src, d_shift, h->st, &h->err);
+    if (rc != UMLMD_OK) return rc;
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    return UMLMD_OK;
+}
+
+int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_force, double virial[9],
+                  double* d_atom_energy) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
+    if (h->nb.N > 0 && !d_pos) return fail(h, UMLMD_E_INVALID_ARG, "null positions");
+    const bool want_grad = d_force != nullptr || virial != nullptr;
+    if (h->nb.N == 0) {
+        if (energy) *energy = 0;
+        if (virial) for (int k = 0; k < 9; ++k) virial[k] = 0;
+        return UMLMD_OK;
+    }
+    int rc = enqueue_compute(h, d_pos, want_grad, d_force, d_atom_energy);
+    if (rc != UMLMD_OK) return rc;
+    rc = fetch_results(h, 10);
+    if (rc != UMLMD_OK) return rc;
+    if (energy) *energy = h->h_out[0];
+    if (virial) for (int k = 0; k < 9; ++k) virial[k] = h->h_out[1 + k];
+    return UMLMD_OK;
+}
+
+int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* mass_per_type) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
+    if (!d_pos || !d_vel || !mass_per_type) return fail(h, UMLMD_E_INVALID_ARG, "null MD state");
+    const int T = h->d.T;
+    std::vector<double> m(T), im(T);
+    for (int t = 0; t < T; ++t) {
+        if (!(mass_per_type[t] > 0) || !std::isfinite(mass_per_type[t])) return fail(h, UMLMD_E_INVALID_ARG, "masses must be positive");
+        m[t] = mass_per_type[t]; im[t] = 1.0 / mass_per_type[t];
+    }
+    int64_t c;
+    if (!h->d_mass) { c = 0; API_CUDA(h, dev_ensure(&h->d_mass, &c, T)); c = 0; API_CUDA(h, dev_ensure(&h->d_inv_mass, &c, T)); }
+    API_CUDA(h, cudaMemcpyAsync(h->d_mass, m.data(), sizeof(double) * T, cudaMemcpyHostToDevice, h->st));
+    API_CUDA(h, cudaMemcpyAsync(h->d_inv_mass, im.data(), sizeof(double) * T, cudaMemcpyHostToDevice, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    if (h->nb.N > h->md_cap || !h->md_force) API_CUDA(h, dev_ensure(&h->md_force, &h->md_cap, h->nb.N * 3));
+    h->md_pos = d_pos; h->md_vel = d_vel;
+    h->have_md = true; h->have_force = false;
+    return UMLMD_OK;
+}
+
+int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* e_pot, double* e_kin) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
+    if (!h->have_md) return fail(h, UMLMD_E_NO_MD_STATE, "umlmd_set_md_state must be called first");
+    if (nsteps < 0 || !(dt_ps > 0) || !std::isfinite(dt_ps)) return fail(h, UMLMD_E_INVALID_ARG, "bad step count or time step");
+    const int64_t N = h->nb.N;
+    int rc;
+    if (!h->have_force) {
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        h->have_force = true;
+    }
+    for (int s = 0; s < nsteps; ++s) {
+        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, true, h->st));
+        ++h->steps_since_build;
+        if (rebuild_every > 0 && h->steps_since_build >= rebuild_every) {
+            const double skin = h->nb.skin;
+            const double L[3] = {h->nb.L[0], h->nb.L[1], h->nb.L[2]};
+            const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};
+            if ((rc = build_list(h, N, h->md_pos, h->type_o, L, pbc, skin)) != UMLMD_OK) return rc;
+        }
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, false, h->st));
+    }
+    API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st));
+    rc = fetch_results(h, 11);
+    if (rc != UMLMD_OK) return rc;
+    if (e_pot) *e_pot = h->h_out[0];
+    if (e_kin) *e_kin = h->h_out[10];
+    return UMLMD_OK;
+}
+
+int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "no neighbor list built");
+    if (h->nb.N > h->node_tile) return fail(h, UMLMD_E_CAPACITY, "intermediates are only kept for single-tile systems");
+    if (d_state) API_CUDA(h, launch_unsort_state(h->nb, h->state, h->d.SP, h->d.S + 2, d_state, h->st));
+    if (d_desc) API_CUDA(h, launch_unsort_state(h->nb, h->desc, h->d.DP, h->d.D_out, d_desc, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    return UMLMD_OK;
+}
+
+int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, double* out_g, double* out_dg) {
+    if (!h || n < 0 || (n > 0 && (!rho || !out_g))) return UMLMD_E_INVALID_ARG;
+    const Dims& d = h->d;
+    const int NC = d.C0 + d.R;
+    for (int64_t i = 0; i < n; ++i) {
+        int row = (int)std::floor(rho[i] / h->hm.dx);
+        if (row < 0) row = 0;
+        if (row > d.n_rows - 1) row = d.n_rows - 1;
+        const double t = rho[i] - row * h->hm.dx;
+        const float* p = &h->hm.table[(size_t)row * 6 * d.CP];
+        for (int c = 0; c < NC; ++c) {
+            const double c0 = p[c], c1 = p[d.CP + c], c2 = p[2 * d.CP + c], c3 = p[3 * d.CP + c], c4 = p[4 * d.CP + c],
+                         c5 = p[5 * d.CP + c];
+            out_g[i * NC + c] = ((((c5 * t + c4) * t + c3) * t + c2) * t + c1) * t + c0;
+            if (out_dg) out_dg[i * NC + c] = (((5 * c5 * t + 4 * c4) * t + 3 * c3) * t + 2 * c2) * t + c1;
+        }
+    }
+    return UMLMD_OK;
+}
+
+int umlmd_eval_pair_cache(const umlmd_t* h, int32_t type_i, int32_t type_j, double* out) {
+    if (!h || !out) return UMLMD_E_INVALID_ARG;
+    const Dims& d = h->d;
+    if (type_i < 0 || type_j < 0 || type_i >= d.T || type_j >= d.T) return UMLMD_E_INVALID_ARG;
+    const size_t n = (size_t)(2 + d.R) * d.C0;
+    const float* p = &h->hm.pairmod[(size_t)(type_i * d.T + type_j) * n];
+    for (size_t k = 0; k < n; ++k) out[k] = p[k];
+    return UMLMD_OK;
+}
+
+}  // extern "C"

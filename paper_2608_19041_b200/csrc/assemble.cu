@@ -1,0 +1,215 @@
+// Force / virial / energy assembly and the velocity-Verlet update.
+//
+// Forces: each atom is written by exactly one warp, which sums, over the atom's own CSR
+// row, the gradient of each edge minus the gradient of its reverse edge (the reverse-edge
+// map turns the source-sorted view into a gather).  No floating-point atomics anywhere,
+// sums in double, fixed order, so results are bitwise reproducible.
+#include "kernels.h"
+
+namespace umd {
+
+namespace {
+
+constexpr int kRedBlock = 256;
+constexpr int kRedMaxBlocks = 1024;
+
+__global__ void k_force_rows(int N, const int* __restrict__ row_ptr, const int* __restrict__ rev,
+                             const float* __restrict__ g, double* __restrict__ f) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int e0 = row_ptr[warp], e1 = row_ptr[warp + 1];
+    double fx = 0, fy = 0, fz = 0;
+    for (int e = e0 + lane; e < e1; e += 32) {
+        const float* a = g + 3 * (size_t)e;
+        float bx = 0.f, by = 0.f, bz = 0.f;
+        const int r = rev[e];
+        if (r >= 0) { const float* b = g + 3 * (size_t)r; bx = b[0]; by = b[1]; bz = b[2]; }
+        fx += (double)a[0] - (double)bx;
+        fy += (double)a[1] - (double)by;
+        fz += (double)a[2] - (double)bz;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        fx += __shfl_xor_sync(0xffffffffu, fx, off);
+        fy += __shfl_xor_sync(0xffffffffu, fy, off);
+        fz += __shfl_xor_sync(0xffffffffu, fz, off);
+    }
+    if (lane == 0) { f[3 * (size_t)warp] = fx; f[3 * (size_t)warp + 1] = fy; f[3 * (size_t)warp + 2] = fz; }
+}
+
+__global__ void k_scatter3(int N, const int* __restrict__ perm, const double* __restrict__ in,
+                           double* __restrict__ out, int* __restrict__ err) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int o = perm[i];
+    bool bad = false;
+    for (int k = 0; k < 3; ++k) {
+        const double v = in[3 * (size_t)i + k];
+        if (!isfinite(v)) bad = true;
+        out[3 * (size_t)o + k] = v;
+    }
+    if (bad) atomicOr(err, kErrNonFinite);
+}
+
+__global__ void k_scatter1(int N, const int* __restrict__ perm, const double* __restrict__ in,
+                           double* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N) out[perm[i]] = in[i];
+}
+
+__global__ void k_unsort_rows(int N, const int* __restrict__ perm, const float* __restrict__ in, int stride,
+                              int width, float* __restrict__ out) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const float* r = in + (size_t)warp * stride;
+    float* w = out + (size_t)perm[warp] * width;
+    for (int k = lane; k < width; k += 32) w[k] = r[k];
+}
+
+__device__ __forceinline__ double block_sum(double v, double* sh) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    double s = 0;
+    if (threadIdx.x == 0) for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += sh[w];
+    return s;   // valid in thread 0
+}
+
+// pass 1: block b sums the contiguous slice [b*chunk, (b+1)*chunk) of x
+__global__ void __launch_bounds__(kRedBlock) k_sum_slices(const double* __restrict__ x, int64_t N, int64_t chunk,
+                                                          double* __restrict__ part) {
+    __shared__ double sh[kRedBlock / 32];
+    const int64_t lo = (int64_t)blockIdx.x * chunk;
+    const int64_t hi = lo + chunk < N ? lo + chunk : N;
+    double v = 0;
+    for (int64_t i = lo + threadIdx.x; i < hi; i += kRedBlock) v += x[i];
+    const double s = block_sum(v, sh);
+    if (threadIdx.x == 0) part[blockIdx.x] = s;
+}
+
+// pass 2 (one block): out[0] = sum of slice partials; out[1..9] = -sum of virial partials
+__global__ void __launch_bounds__(kRedBlock) k_final_reduce(const double* __restrict__ part, int n_part,
+                                                            const double* __restrict__ vpart, int n_vpart,
+                                                            double* __restrict__ out, int* __restrict__ err) {
+    __shared__ double sh[kRedBlock / 32];
+    double v = 0;
+    for (int i = threadIdx.x; i < n_part; i += kRedBlock) v += part[i];
+    double s = block_sum(v, sh);
+    if (threadIdx.x == 0) {
+        out[0] = s;
+        if (!isfinite(s)) atomicOr(err, kErrNonFinite);
+    }
+    for (int k = 0; k < 9; ++k) {
+        v = 0;
+        for (int i = threadIdx.x; i < n_vpart; i += kRedBlock) v += vpart[(size_t)i * 9 + k];
+        s = block_sum(v, sh);
+        if (threadIdx.x == 0) out[1 + k] = -s;
+    }
+}
+
+__global__ void k_vv(int64_t N, double* __restrict__ pos, double* __restrict__ vel, const double* __restrict__ force,
+                     const int* __restrict__ type, const double* __restrict__ inv_mass, double dt, bool drift) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const double c = 0.5 * dt * kAccelUnit * inv_mass[type[i]];
+    for (int k = 0; k < 3; ++k) {
+        double v = vel[3 * i + k] + c * force[3 * i + k];
+        vel[3 * i + k] = v;
+        if (drift) pos[3 * i + k] += dt * v;
+    }
+}
+
+__global__ void __launch_bounds__(kRedBlock) k_ke_slices(const double* __restrict__ vel, const int* __restrict__ type,
+                                                         const double* __restrict__ mass, int64_t N, int64_t chunk,
+                                                         double* __restrict__ part) {
+    __shared__ double sh[kRedBlock / 32];
+    const int64_t lo = (int64_t)blockIdx.x * chunk;
+    const int64_t hi = lo + chunk < N ? lo + chunk : N;
+    double v = 0;
+    for (int64_t i = lo + threadIdx.x; i < hi; i += kRedBlock) {
+        const double vx = vel[3 * i], vy = vel[3 * i + 1], vz = vel[3 * i + 2];
+        v += 0.5 * mass[type[i]] * (vx * vx + vy * vy + vz * vz) / kAccelUnit;
+    }
+    const double s = block_sum(v, sh);
+    if (threadIdx.x == 0) part[blockIdx.x] = s;
+}
+
+__global__ void __launch_bounds__(kRedBlock) k_sum_small(const double* __restrict__ part, int n, double* out) {
+    __shared__ double sh[kRedBlock / 32];
+    double v = 0;
+    for (int i = threadIdx.x; i < n; i += kRedBlock) v += part[i];
+    const double s = block_sum(v, sh);
+    if (threadIdx.x == 0) *out = s;
+}
+
+inline void slices(int64_t N, int* blocks, int64_t* chunk) {
+    int64_t b = (N + 4095) / 4096;
+    if (b < 1) b = 1;
+    if (b > kRedMaxBlocks) b = kRedMaxBlocks;
+    *blocks = (int)b;
+    *chunk = (N + b - 1) / b;
+}
+
+}  // namespace
+
+int reduce_scratch_doubles(int64_t) { return kRedMaxBlocks; }
+
+cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* f_sorted, cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    k_force_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.row_ptr, nb.rev, g, f_sorted);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force, int* d_err,
+                                  cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    k_scatter3<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, f_sorted, d_force, d_err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_atom_energy(const NeighborDev& nb, const double* e_sorted, double* d_out, cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    k_scatter1<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, e_sorted, d_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_energy_virial(const double* e_atom, int64_t N, const double* virial_part, int n_part,
+                                        double* scratch, double* out, int* d_err, cudaStream_t st) {
+    int blocks; int64_t chunk;
+    slices(N, &blocks, &chunk);
+    k_sum_slices<<<blocks, kRedBlock, 0, st>>>(e_atom, N, chunk, scratch);
+    k_final_reduce<<<1, kRedBlock, 0, st>>>(scratch, blocks, virial_part, n_part, out, d_err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stride, int width, float* out,
+                                cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    k_unsort_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.perm, in, stride, width, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force, const int* type,
+                                 const double* inv_mass, double dt, bool drift, cudaStream_t st) {
+    if (N == 0) return cudaSuccess;
+    k_vv<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, pos, vel, force, type, inv_mass, dt, drift);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_kinetic_energy(int64_t N, const double* vel, const int* type, const double* mass,
+                                  double* scratch, double* out, cudaStream_t st) {
+    int blocks; int64_t chunk;
+    slices(N, &blocks, &chunk);
+    k_ke_slices<<<blocks, kRedBlock, 0, st>>>(vel, type, mass, N, chunk, scratch);
+    k_sum_small<<<1, kRedBlock, 0, st>>>(scratch, blocks, out);
+    return cudaGetLastError();
+}
+
+}  // namespace umd

@@ -1,0 +1,97 @@
+// Shared declarations of the library's translation units: structural widths, the
+// device-resident model constants, the per-handle workspace and the kernel launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+#include <string>
+#include <vector>
+
+#include "../../include/umlmd.h"
+
+namespace umd {
+
+constexpr float kEpsReg = 1.0e-7f;     // direction regulariser, Angstrom (edge geometry)
+constexpr int kMaxDeg = 3;             // highest angular degree compiled in
+constexpr int kMaxR = 8;               // most shared radial modes
+constexpr int kMaxGaunt = 96;          // non-zeros kept per generic coupling tensor
+constexpr double kAccelUnit = 9648.53321;   // (eV/Angstrom/amu) in Angstrom/ps^2
+constexpr double kBoltzmann = 8.617333262e-5;
+
+// error word bits set by kernels (read back at synchronisation points)
+enum : int { kErrStale = 1, kErrNonFinite = 2, kErrEdgeOverflow = 4, kErrShiftRange = 8 };
+
+// Widths derived from (C0, L, R): degree-wise channels, probe ranks, feature-state width
+// S, feature-vector width D_out, gated hidden widths, and the flat offsets used by the
+// kernels.  Host and device both read this struct (it is passed by value).
+struct Dims {
+    int C0, L, R, N_rbf, n_hidden, F, T;
+    int C[kMaxDeg + 1];      // channels per degree
+    int K[kMaxDeg + 1];      // probe ranks (index 0 unused)
+    int S, SP;               // state width S; row stride SP >= S+2, multiple of 4
+    int offA[kMaxDeg + 1];   // offset of degree block in the state row
+    int D_out, DP;           // feature-vector width; row stride (multiple of 32)
+    int oG[kMaxDeg + 1];     // offsets of vech(G_l) in D
+    int oJ112, oJ123, oJ222, oJ233, oPi;
+    int H, Hp;
+    int CP;                  // table channels C0+R rounded up to 4
+    int n_rows;              // table intervals
+    float rc, dx, inv_dx;
+};
+
+struct GauntSparse {         // non-zeros of one unit-norm coupling tensor
+    int n;
+    unsigned char m1[kMaxGaunt], m2[kMaxGaunt], m3[kMaxGaunt];
+    float v[kMaxGaunt];
+};
+
+// Device-resident constants of one model.
+struct ModelDev {
+    float* table;     // [n_rows][6][CP] quintic coefficients c0..c5 of [g, q]
+    float* pairmod;   // [T*T][2+R][C0]: scale gamma, shift beta, mode mixing U[:, mu]
+    float* X0;        // [T][C0]
+    float* W1p;       // [C1][C1]  I + W_1
+    float* W2p;       // [C2][C2]  I + W_2
+    float* A1;        // [C1][K1]
+    float* A2;        // [C2][K2]
+    float* mu;        // [D_out]
+    float* inv_sigma; // [D_out]
+    float* theta[8];  // Theta_t, row-major [K_in (padded)][F]; theta[0] has DP rows
+    float* thetaT[8]; // transposes, [F][K_in (padded)]
+    float* bias[8];   // b_t [F]
+    float* w_head;    // [F]
+    float* e_ref;     // [T]
+    float b_head;
+    GauntSparse* g123;   // device copies (NULL when L < 3)
+    GauntSparse* g233;
+};
+
+struct Handle;  // defined in api.cu
+
+// ---- launchers (each enqueues on `st`; none synchronises) ---------------------------
+
+struct NeighborDev {
+    int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;
+    double L[3] = {0, 0, 0};
+    int pbc[3] = {1, 1, 1};
+    double skin = 0, r_list = 0;
+    double* wpos = nullptr;      // [N][3] folded positions, caller order (build time)
+    int* img = nullptr;          // [N][3] floor(frac) per atom, sorted order
+    int* perm = nullptr;         // [N] sorted index -> caller index
+    int* type_s = nullptr;       // [N] species, sorted order
+    double* xs0 = nullptr;       // [N][3] folded positions at build time, sorted order
+    double* xs = nullptr;        // [N][3] current positions minus img*L, sorted order
+    int* row_ptr = nullptr;      // [N+1]
+    int* src = nullptr;          // [E] sorted index of the neighbour
+    int* shift = nullptr;        // [E] packed int8 x3 image n
+    int* rev = nullptr;          // [E] index of the reverse edge, -1 if absent
+    // scratch
+    int* key = nullptr; int* key2 = nullptr; int* idx = nullptr; int* idx2 = nullptr;
+    int* cell_start = nullptr; int64_t ncell_cap = 0;
+    int* deg = nullptr;
+    void* cub_tmp = nullptr; size_t cub_bytes = 0;
+};
+
+}  // namespace umd

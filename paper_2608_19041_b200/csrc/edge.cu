@@ -1,0 +1,477 @@
+// Fused per-edge kernels: edge featurisation + per-destination aggregation (forward) and
+// the recomputing edge backward pass that returns dE/dr_ij for every edge.
+//
+// One warp owns one destination atom and walks its contiguous CSR interval.  Edges are
+// taken in batches of 32: first each lane computes the geometry of one edge (displacement
+// from double-precision positions, regularised length, direction, cutoff envelope, table
+// row), then the batch is replayed with lanes split over channels -- a group of C0/4 lanes
+// handles one edge, each lane holding four consecutive channels, so table and pair-cache
+// reads are 16-byte vector loads that a group issues as one contiguous segment.  The S+2
+// sums live in registers and are written once per destination; nothing per-edge is stored
+// in the forward pass.  The backward pass recomputes the same per-edge quantities from the
+// same quintic polynomial (so the force is the exact derivative of the interpolated
+// energy), contracts them with dE/d(sums) and writes one 3-vector per edge; the virial is
+// accumulated in the same pass.
+//
+// Harmonics are evaluated with |u|^2 set to one; the regularised direction differs from a
+// unit vector by eps^2/rho^2, far below single precision.
+#include "kernels.h"
+
+namespace umd {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+
+struct Geom {
+    float dx, dy, dz, rho, inv_rho, ux, uy, uz, chi, dchi, t;
+    int row, pair;
+    bool valid;
+};
+
+// phase 1: one lane, one edge
+__device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, int e, bool in_range, double xi, double yi,
+                                              double zi, int ti) {
+    Geom g;
+    g.valid = false;
+    g.dx = g.dy = g.dz = 0.f; g.rho = 1.f; g.inv_rho = 1.f; g.ux = g.uy = g.uz = 0.f;
+    g.chi = 0.f; g.dchi = 0.f; g.t = 0.f; g.row = 0; g.pair = 0;
+    if (!in_range) return g;
+    const int j = a.src[e];
+    const int s = a.shift[e];
+    const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff),
+              nz = (int)(signed char)((s >> 16) & 0xff);
+    const double* xj = a.xs + 3 * (size_t)j;
+    g.dx = (float)((xj[0] + nx * a.Lx) - xi);
+    g.dy = (float)((xj[1] + ny * a.Ly) - yi);
+    g.dz = (float)((xj[2] + nz * a.Lz) - zi);
+    const float r2 = g.dx * g.dx + g.dy * g.dy + g.dz * g.dz + kEpsReg * kEpsReg;
+    g.rho = sqrtf(r2);
+    if (!(g.rho < a.d.rc)) return g;       // skin-shell edge: zero weight
+    g.valid = true;
+    g.inv_rho = 1.0f / g.rho;
+    g.ux = g.dx * g.inv_rho; g.uy = g.dy * g.inv_rho; g.uz = g.dz * g.inv_rho;
+    const float inv_rc = 1.0f / a.d.rc;
+    const float x = g.rho * inv_rc, t = 1.0f - x;
+    const float t2 = t * t, x2 = x * x;
+    const float poly = 1.0f + x * (4.0f + x * (10.0f + x * (20.0f + 35.0f * x)));
+    g.chi = t2 * t2 * poly;
+    g.dchi = -280.0f * x2 * x2 * t2 * t * inv_rc;
+    int row = (int)(g.rho * a.d.inv_dx);
+    row = row < a.d.n_rows - 1 ? row : a.d.n_rows - 1;
+    g.row = row;
+    g.t = g.rho - (float)row * a.d.dx;
+    g.pair = ti * a.d.T + a.type_s[j];
+    return g;
+}
+
+template <int L>
+__device__ __forceinline__ void harmonics_s1(float x, float y, float z, float* B1, float* B2, float* B3) {
+    const float r3 = 1.7320508075688772f;
+    B1[0] = x; B1[1] = y; B1[2] = z;
+    B2[0] = r3 * x * y; B2[1] = r3 * y * z; B2[2] = 0.5f * (3.0f * z * z - 1.0f); B2[3] = r3 * x * z;
+    B2[4] = 0.5f * r3 * (x * x - y * y);
+    if (L >= 3) {
+        const float a = 0.7905694150420949f, b = 3.872983346207417f, c = 0.6123724356957945f;
+        B3[0] = a * y * (3.0f * x * x - y * y);
+        B3[1] = b * x * y * z;
+        B3[2] = c * y * (5.0f * z * z - 1.0f);
+        B3[3] = 0.5f * z * (5.0f * z * z - 3.0f);
+        B3[4] = c * x * (5.0f * z * z - 1.0f);
+        B3[5] = 0.5f * b * z * (x * x - y * y);
+        B3[6] = a * x * (x * x - 3.0f * y * y);
+    }
+}
+
+// sum over l >= 1 of t_lm * grad_u B_lm (|u|^2 = 1 convention)
+template <int L>
+__device__ __forceinline__ void harmonics_grad_contract(float x, float y, float z, const float* t1,
+                                                        const float* t2, const float* t3, float* gx,
+                                                        float* gy, float* gz) {
+    const float r3 = 1.7320508075688772f;
+    float ax = t1[0], ay = t1[1], az = t1[2];
+    ax += r3 * (t2[0] * y + t2[3] * z + t2[4] * x);
+    ay += r3 * (t2[0] * x + t2[1] * z - t2[4] * y);
+    az += r3 * (t2[1] * y + t2[3] * x) + 3.0f * t2[2] * z;
+    if (L >= 3) {
+        const float a = 0.7905694150420949f, b = 3.872983346207417f, c = 0.6123724356957945f;
+        const float xx = x * x, yy = y * y, zz = z * z;
+        ax += t3[0] * (6.0f * a * x * y) + t3[1] * (b * y * z) + t3[4] * (c * (5.0f * zz - 1.0f)) +
+              t3[5] * (b * x * z) + t3[6] * (3.0f * a * (xx - yy));
+        ay += t3[0] * (3.0f * a * (xx - yy)) + t3[1] * (b * x * z) + t3[2] * (c * (5.0f * zz - 1.0f)) -
+              t3[5] * (b * y * z) - t3[6] * (6.0f * a * x * y);
+        az += t3[1] * (b * x * y) + t3[2] * (10.0f * c * y * z) + t3[3] * (0.5f * (15.0f * zz - 3.0f)) +
+              t3[4] * (10.0f * c * x * z) + t3[5] * (0.5f * b * (xx - yy));
+    }
+    *gx = ax; *gy = ay; *gz = az;
+}
+
+// value (and derivative) of four consecutive table channels at offset t in row `row`
+template <bool DERIV>
+__device__ __forceinline__ void table_eval4(const float* __restrict__ table, int CP, int row, int c, float t,
+                                            float* v, float* dv) {
+    const float* p = table + (size_t)row * 6 * CP + c;
+    const float4 c0 = ldg4(p), c1 = ldg4(p + CP), c2 = ldg4(p + 2 * CP), c3 = ldg4(p + 3 * CP),
+                 c4 = ldg4(p + 4 * CP), c5 = ldg4(p + 5 * CP);
+#define UMLMD_HORNER(k, f)                                                                             \
+    v[k] = ((((c5.f * t + c4.f) * t + c3.f) * t + c2.f) * t + c1.f) * t + c0.f;                        \
+    if (DERIV) dv[k] = (((5.0f * c5.f * t + 4.0f * c4.f) * t + 3.0f * c3.f) * t + 2.0f * c2.f) * t + c1.f;
+    UMLMD_HORNER(0, x) UMLMD_HORNER(1, y) UMLMD_HORNER(2, z) UMLMD_HORNER(3, w)
+#undef UMLMD_HORNER
+}
+
+template <bool DERIV>
+__device__ __forceinline__ void table_eval1(const float* __restrict__ table, int CP, int row, int c, float t,
+                                            float* v, float* dv) {
+    const float* p = table + (size_t)row * 6 * CP + c;
+    const float c0 = __ldg(p), c1 = __ldg(p + CP), c2 = __ldg(p + 2 * CP), c3 = __ldg(p + 3 * CP),
+                c4 = __ldg(p + 4 * CP), c5 = __ldg(p + 5 * CP);
+    *v = ((((c5 * t + c4) * t + c3) * t + c2) * t + c1) * t + c0;
+    if (DERIV) *dv = (((5.0f * c5 * t + 4.0f * c4) * t + 3.0f * c3) * t + 2.0f * c2) * t + c1;
+}
+
+// amplitude psi (and d psi / d rho) of this lane's four channels for one edge
+template <int C0, bool HASR, bool DERIV>
+__device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, int pair, int c, float* psi,
+                                           float* dpsi) {
+    float g[4], dg[4];
+    table_eval4<DERIV>(a.table, a.d.CP, row, c, t, g, dg);
+    const int R = HASR ? a.d.R : 0;
+    const float* pm = a.pairmod + (size_t)pair * (2 + R) * C0 + c;
+    const float4 ga = ldg4(pm), be = ldg4(pm + C0);
+    psi[0] = ga.x * g[0] + be.x; psi[1] = ga.y * g[1] + be.y;
+    psi[2] = ga.z * g[2] + be.z; psi[3] = ga.w * g[3] + be.w;
+    if (DERIV) { dpsi[0] = ga.x * dg[0]; dpsi[1] = ga.y * dg[1]; dpsi[2] = ga.z * dg[2]; dpsi[3] = ga.w * dg[3]; }
+    if (HASR) {
+        for (int q = 0; q < R; ++q) {
+            float qv, dqv = 0.f;
+            table_eval1<DERIV>(a.table, a.d.CP, row, C0 + q, t, &qv, &dqv);
+            const float4 U = ldg4(pm + (size_t)(2 + q) * C0);
+            psi[0] += U.x * qv; psi[1] += U.y * qv; psi[2] += U.z * qv; psi[3] += U.w * qv;
+            if (DERIV) { dpsi[0] += U.x * dqv; dpsi[1] += U.y * dqv; dpsi[2] += U.z * dqv; dpsi[3] += U.w * dqv; }
+        }
+    }
+}
+
+template <int C0> struct Widths {
+    static constexpr int C1 = C0 <= 16 ? 4 : (C0 <= 64 ? 8 : 16);
+    static constexpr int C2 = C1 / 2 > 4 ? C1 / 2 : 4;
+    static constexpr int LPE = C0 / 4;          // lanes per edge
+    static constexpr int EPI = 32 / LPE;        // edges per replay step
+    static constexpr int NL1 = C1 / 4;          // lanes of a group that hold degree-1 channels
+    static constexpr int NL2 = C2 / 4;
+};
+
+// ------------------------------------------------------------------------------- forward
+template <int C0, int L, bool HASR>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+k_edge_forward(const EdgeArgs a) {
+    using W = Widths<C0>;
+    const int lane = threadIdx.x & 31;
+    const int i = a.a0 + blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (i >= a.a1) return;
+    const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
+    const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
+    const int ti = a.type_s[i];
+    const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
+
+    float acc0[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc1[3][4], acc2[5][4], acc3[7];
+#pragma unroll
+    for (int m = 0; m < 3; ++m)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc1[m][k] = 0.f;
+#pragma unroll
+    for (int m = 0; m < 5; ++m)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc2[m][k] = 0.f;
+#pragma unroll
+    for (int m = 0; m < 7; ++m) acc3[m] = 0.f;
+    float s0 = 0.f, s1 = 0.f;
+
+    for (int base = e0; base < e1; base += 32) {
+        const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
+        if (g.valid) { const float c2 = g.chi * g.chi; s0 += c2; s1 += c2 * c2; }
+        const int nb = min(32, e1 - base);
+        for (int it = 0; it * W::EPI < nb; ++it) {
+            const int b = it * W::EPI + sub;
+            const bool v = __shfl_sync(kFull, (int)g.valid, b) != 0;
+            const int row = __shfl_sync(kFull, g.row, b);
+            const int pair = __shfl_sync(kFull, g.pair, b);
+            const float t = __shfl_sync(kFull, g.t, b);
+            const float chi = __shfl_sync(kFull, g.chi, b);
+            const float ux = __shfl_sync(kFull, g.ux, b);
+            const float uy = __shfl_sync(kFull, g.uy, b);
+            const float uz = __shfl_sync(kFull, g.uz, b);
+            if (!v) continue;
+            float psi[4];
+            amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc0[k] += chi * psi[k];
+            if (cl < W::NL1) {
+                float B1[3], B2[5], B3[7];
+                harmonics_s1<L>(ux, uy, uz, B1, B2, B3);
+                const float w = chi * chi;
+#pragma unroll
+                for (int m = 0; m < 3; ++m) {
+                    const float wb = w * B1[m];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) acc1[m][k] += wb * psi[k];
+                }
+                if (cl < W::NL2) {
+#pragma unroll
+                    for (int m = 0; m < 5; ++m) {
+                        const float wb = w * B2[m];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) acc2[m][k] += wb * psi[k];
+                    }
+                }
+                if (L >= 3 && cl == 0) {
+#pragma unroll
+                    for (int m = 0; m < 7; ++m) acc3[m] += w * B3[m] * psi[0];
+                }
+            }
+        }
+    }
+    // combine the edge slots of the warp (lanes with equal channel offset)
+#pragma unroll
+    for (int off = W::LPE; off < 32; off <<= 1) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc0[k] += __shfl_xor_sync(kFull, acc0[k], off);
+#pragma unroll
+        for (int m = 0; m < 3; ++m)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc1[m][k] += __shfl_xor_sync(kFull, acc1[m][k], off);
+#pragma unroll
+        for (int m = 0; m < 5; ++m)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc2[m][k] += __shfl_xor_sync(kFull, acc2[m][k], off);
+        if (L >= 3) {
+#pragma unroll
+            for (int m = 0; m < 7; ++m) acc3[m] += __shfl_xor_sync(kFull, acc3[m], off);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        s0 += __shfl_xor_sync(kFull, s0, off);
+        s1 += __shfl_xor_sync(kFull, s1, off);
+    }
+    float* row_out = a.state + (size_t)(i - a.a0) * a.d.SP;
+    if (sub == 0) {
+        *reinterpret_cast<float4*>(row_out + c) = make_float4(acc0[0], acc0[1], acc0[2], acc0[3]);
+        if (cl < W::NL1) {
+#pragma unroll
+            for (int m = 0; m < 3; ++m)
+                *reinterpret_cast<float4*>(row_out + a.d.offA[1] + m * W::C1 + c) =
+                    make_float4(acc1[m][0], acc1[m][1], acc1[m][2], acc1[m][3]);
+        }
+        if (cl < W::NL2) {
+#pragma unroll
+            for (int m = 0; m < 5; ++m)
+                *reinterpret_cast<float4*>(row_out + a.d.offA[2] + m * W::C2 + c) =
+                    make_float4(acc2[m][0], acc2[m][1], acc2[m][2], acc2[m][3]);
+        }
+        if (L >= 3 && cl == 0) {
+#pragma unroll
+            for (int m = 0; m < 7; ++m) row_out[a.d.offA[3] + m] = acc3[m];
+        }
+        if (cl == 0) { row_out[a.d.S] = s0; row_out[a.d.S + 1] = s1; }
+    }
+}
+
+// ------------------------------------------------------------------------------ backward
+template <int C0, int L, bool HASR>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+k_edge_backward(const EdgeArgs a) {
+    using W = Widths<C0>;
+    __shared__ float red[kWarpsPerBlock][32][5];
+    __shared__ double vsum[kWarpsPerBlock][9];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
+    const bool active = i < a.a1;
+    const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
+    float vir[9];
+#pragma unroll
+    for (int k = 0; k < 9; ++k) vir[k] = 0.f;
+
+    if (active) {
+        const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
+        const int ti = a.type_s[i];
+        const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
+        const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
+        // dE/d(sums) of this lane's channels
+        float h0[4], h1[3][4], h2[5][4], h3[7];
+        {
+            const float4 v = *reinterpret_cast<const float4*>(grow + c);
+            h0[0] = v.x; h0[1] = v.y; h0[2] = v.z; h0[3] = v.w;
+        }
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (cl < W::NL1) v = *reinterpret_cast<const float4*>(grow + a.d.offA[1] + m * W::C1 + c);
+            h1[m][0] = v.x; h1[m][1] = v.y; h1[m][2] = v.z; h1[m][3] = v.w;
+        }
+#pragma unroll
+        for (int m = 0; m < 5; ++m) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (cl < W::NL2) v = *reinterpret_cast<const float4*>(grow + a.d.offA[2] + m * W::C2 + c);
+            h2[m][0] = v.x; h2[m][1] = v.y; h2[m][2] = v.z; h2[m][3] = v.w;
+        }
+#pragma unroll
+        for (int m = 0; m < 7; ++m) h3[m] = (L >= 3 && cl == 0) ? grow[a.d.offA[3] + m] : 0.f;
+        const float ds0 = grow[a.d.S], ds1 = grow[a.d.S + 1];
+
+        for (int base = e0; base < e1; base += 32) {
+            const int e = base + lane;
+            const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
+            const int nb = min(32, e1 - base);
+            for (int it = 0; it * W::EPI < nb; ++it) {
+                const int b = it * W::EPI + sub;
+                const bool v = __shfl_sync(kFull, (int)g.valid, b) != 0;
+                const int row = __shfl_sync(kFull, g.row, b);
+                const int pair = __shfl_sync(kFull, g.pair, b);
+                const float t = __shfl_sync(kFull, g.t, b);
+                const float chi = __shfl_sync(kFull, g.chi, b);
+                const float ux = __shfl_sync(kFull, g.ux, b);
+                const float uy = __shfl_sync(kFull, g.uy, b);
+                const float uz = __shfl_sync(kFull, g.uz, b);
+                float p_rho = 0.f, p_chi = 0.f, pux = 0.f, puy = 0.f, puz = 0.f;
+                if (v) {
+                    float psi[4], dpsi[4];
+                    amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi);
+                    float ec[4];   // dE/dpsi_c
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) { ec[k] = chi * h0[k]; p_chi += psi[k] * h0[k]; }
+                    if (cl < W::NL1) {
+                        float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
+                        harmonics_s1<L>(ux, uy, uz, B1, B2, B3);
+                        const float w = chi * chi;
+                        float bt = 0.f;   // sum_lm B_lm t_lm
+#pragma unroll
+                        for (int m = 0; m < 3; ++m) {
+                            float tm = 0.f;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) { tm += psi[k] * h1[m][k]; ec[k] += w * B1[m] * h1[m][k]; }
+                            t1[m] = tm; bt += B1[m] * tm;
+                        }
+#pragma unroll
+                        for (int m = 0; m < 5; ++m) {
+                            float tm = 0.f;
+                            if (cl < W::NL2) {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) { tm += psi[k] * h2[m][k]; ec[k] += w * B2[m] * h2[m][k]; }
+                            }
+                            t2[m] = tm; bt += B2[m] * tm;
+                        }
+#pragma unroll
+                        for (int m = 0; m < 7; ++m) {
+                            float tm = 0.f;
+                            if (L >= 3 && cl == 0) { tm = psi[0] * h3[m]; ec[0] += w * B3[m] * h3[m]; }
+                            t3[m] = tm;
+                            if (L >= 3) bt += B3[m] * tm;
+                        }
+                        p_chi += 2.0f * chi * bt;
+                        float gx, gy, gz;
+                        harmonics_grad_contract<L>(ux, uy, uz, t1, t2, t3, &gx, &gy, &gz);
+                        pux = w * gx; puy = w * gy; puz = w * gz;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) p_rho += ec[k] * dpsi[k];
+                }
+                // sum over the lanes of the group
+#pragma unroll
+                for (int off = 1; off < W::LPE; off <<= 1) {
+                    p_rho += __shfl_xor_sync(kFull, p_rho, off);
+                    p_chi += __shfl_xor_sync(kFull, p_chi, off);
+                    pux += __shfl_xor_sync(kFull, pux, off);
+                    puy += __shfl_xor_sync(kFull, puy, off);
+                    puz += __shfl_xor_sync(kFull, puz, off);
+                }
+                if (cl == 0 && b < 32) {
+                    red[wid][b][0] = p_rho; red[wid][b][1] = p_chi;
+                    red[wid][b][2] = pux; red[wid][b][3] = puy; red[wid][b][4] = puz;
+                }
+            }
+            __syncwarp();
+            if (e < e1) {
+                float gx = 0.f, gy = 0.f, gz = 0.f;
+                if (g.valid) {
+                    const float p_rho = red[wid][lane][0], p_chi = red[wid][lane][1];
+                    const float pux = red[wid][lane][2], puy = red[wid][lane][3], puz = red[wid][lane][4];
+                    const float c2 = g.chi * g.chi;
+                    const float dEdrho = p_rho + (p_chi + 2.0f * g.chi * ds0 + 4.0f * c2 * g.chi * ds1) * g.dchi;
+                    const float dot = pux * g.ux + puy * g.uy + puz * g.uz;
+                    gx = dEdrho * g.ux + (pux - dot * g.ux) * g.inv_rho;
+                    gy = dEdrho * g.uy + (puy - dot * g.uy) * g.inv_rho;
+                    gz = dEdrho * g.uz + (puz - dot * g.uz) * g.inv_rho;
+                    vir[0] += gx * g.dx; vir[1] += gx * g.dy; vir[2] += gx * g.dz;
+                    vir[3] += gy * g.dx; vir[4] += gy * g.dy; vir[5] += gy * g.dz;
+                    vir[6] += gz * g.dx; vir[7] += gz * g.dy; vir[8] += gz * g.dz;
+                }
+                float* go = a.g + 3 * (size_t)e;
+                go[0] = gx; go[1] = gy; go[2] = gz;
+            }
+            __syncwarp();
+        }
+    }
+    // block partial of sum_e g (x) r, in double, fixed order
+#pragma unroll
+    for (int k = 0; k < 9; ++k) {
+        double v = (double)vir[k];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFull, v, off);
+        if (lane == 0) vsum[wid][k] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < 9) {
+        double v = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) v += vsum[w][threadIdx.x];
+        a.virial_part[(size_t)blockIdx.x * 9 + threadIdx.x] = v;
+    }
+}
+
+template <int C0, int L>
+cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
+    if (a.d.R > 0) k_edge_forward<C0, L, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    else k_edge_forward<C0, L, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template <int C0, int L>
+cudaError_t launch_bwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
+    if (a.d.R > 0) k_edge_backward<C0, L, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    else k_edge_backward<C0, L, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <bool FWD>
+cudaError_t dispatch(const EdgeArgs& a, int blocks, cudaStream_t st) {
+#define UMLMD_CASE(C0v, Lv)                                                       \
+    if (a.d.C0 == C0v && a.d.L == Lv)                                             \
+        return FWD ? launch_fwd_r<C0v, Lv>(a, blocks, st) : launch_bwd_r<C0v, Lv>(a, blocks, st);
+    UMLMD_CASE(8, 2) UMLMD_CASE(8, 3) UMLMD_CASE(16, 2) UMLMD_CASE(16, 3) UMLMD_CASE(32, 2)
+    UMLMD_CASE(32, 3) UMLMD_CASE(64, 2) UMLMD_CASE(64, 3) UMLMD_CASE(128, 2) UMLMD_CASE(128, 3)
+#undef UMLMD_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+int edge_backward_blocks(int n_rows) { return (n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock; }
+
+cudaError_t launch_edge_forward(const EdgeArgs& a, cudaStream_t st) {
+    const int rows = a.a1 - a.a0;
+    if (rows <= 0) return cudaSuccess;
+    return dispatch<true>(a, (rows + kWarpsPerBlock - 1) / kWarpsPerBlock, st);
+}
+
+cudaError_t launch_edge_backward(const EdgeArgs& a, int* n_blocks, cudaStream_t st) {
+    const int rows = a.a1 - a.a0;
+    *n_blocks = edge_backward_blocks(rows);
+    if (rows <= 0) return cudaSuccess;
+    return dispatch<false>(a, *n_blocks, st);
+}
+
+}  // namespace umd

@@ -1,0 +1,92 @@
+// Launchers implemented across the .cu files.  Every launcher enqueues work on the given
+// stream and returns the CUDA status of the launch; none of them synchronises unless
+// stated.
+#pragma once
+
+#include "common.cuh"
+
+namespace umd {
+
+// ---- neighbor.cu ---------------------------------------------------------------------
+// Full build: fold + bin + sort + count + scan + fill + reverse map.  Synchronises once
+// (to learn the edge count and grow the edge arrays).  Returns a UMLMD_* code.
+int neighbor_build(NeighborDev* nb, int64_t N, const double* d_pos, const int32_t* d_type,
+                   const double L[3], const int pbc[3], double skin, double rc, int* d_err,
+                   cudaStream_t st, std::string* err);
+void neighbor_free(NeighborDev* nb);
+// Export the list in caller numbering (device buffers of the caller).
+int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
+                    cudaStream_t st, std::string* err);
+// xs[i] = pos[perm[i]] - img[i]*L; flags stale / non-finite atoms in *d_err.
+cudaError_t launch_gather_positions(const NeighborDev& nb, const double* d_pos, int* d_err,
+                                    cudaStream_t st);
+
+// ---- edge.cu ---------------------------------------------------------------------------
+struct EdgeArgs {
+    Dims d;
+    const float* table;
+    const float* pairmod;
+    const double* xs;       // [N][3] sorted positions
+    const int* type_s;
+    const int* row_ptr;
+    const int* src;
+    const int* shift;
+    double Lx, Ly, Lz;
+    int a0, a1;             // destination range [a0, a1) of this tile
+    float* state;           // [a1-a0][SP]: forward writes sums; backward reads dE/d(sums)
+    float* g;               // [E][3] per-edge gradient (backward)
+    double* virial_part;    // [blocks][9] partial virial sums (backward)
+};
+cudaError_t launch_edge_forward(const EdgeArgs& a, cudaStream_t st);
+cudaError_t launch_edge_backward(const EdgeArgs& a, int* n_blocks, cudaStream_t st);
+int edge_backward_blocks(int n_rows_in_tile);
+
+// ---- invariants.cu -------------------------------------------------------------------
+struct InvArgs {
+    Dims d;
+    ModelDev m;
+    const int* type_s;
+    int a0, n;              // tile start (sorted index) and atom count
+    float* state;           // [n][SP]
+    float* desc;            // [n][DP]
+};
+cudaError_t launch_invariants_forward(const InvArgs& a, cudaStream_t st);
+cudaError_t launch_invariants_backward(const InvArgs& a, cudaStream_t st);
+
+// ---- mlp.cu ----------------------------------------------------------------------------
+struct MlpArgs {
+    Dims d;
+    ModelDev m;
+    const int* type_s;
+    int a0, n;
+    float* desc;            // [n][DP]  in: D, out (backward): dE/dD
+    float* pre;             // [n_hidden][n][F] pre-activations, overwritten by dE/dY
+    float* hbuf;            // [2][n][F] ping-pong activations / hidden gradients
+    double* e_atom;         // [N] sorted order, eV (written at a0..a0+n)
+    int path;               // 1 = CUDA-core fp32, 2 = tcgen05
+    bool want_grad;
+};
+cudaError_t launch_mlp(const MlpArgs& a, cudaStream_t st);
+
+// ---- assemble.cu ---------------------------------------------------------------------
+cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted,
+                                  cudaStream_t st);
+cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,
+                                  int* d_err, cudaStream_t st);
+cudaError_t launch_scatter_atom_energy(const NeighborDev& nb, const double* e_sorted, double* d_out,
+                                       cudaStream_t st);
+// out[0] = sum e_atom, out[1..9] = -sum virial partials (fixed order, double)
+cudaError_t launch_reduce_energy_virial(const double* e_atom, int64_t N, const double* virial_part,
+                                        int n_part, double* scratch, double* out, int* d_err,
+                                        cudaStream_t st);
+int reduce_scratch_doubles(int64_t N);
+cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stride, int width,
+                                float* out, cudaStream_t st);
+// velocity Verlet pieces (caller order, double)
+cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force,
+                                 const int* type, const double* inv_mass, double dt, bool drift,
+                                 cudaStream_t st);
+cudaError_t launch_kinetic_energy(int64_t N, const double* vel, const int* type, const double* mass,
+                                  double* scratch, double* out, cudaStream_t st);
+
+}  // namespace umd

@@ -1,0 +1,159 @@
+// Atomic-energy MLP: residual SiLU layers, scalar head, and the input vector-Jacobian
+// product (no weight gradients).  Each dense layer is one GEMM whose epilogue applies
+// bias / SiLU / identity residual (forward) or the residual add and the SiLU derivative
+// (backward), so activations make one trip through memory per layer.
+//
+// This file holds the CUDA-core fp32 GEMM (any width that is a multiple of 4) and the
+// layer schedule; the tensor-core GEMM lives in mlp_tc.cu and plugs into the same
+// schedule and epilogues.
+#include "kernels.h"
+#include "mlp_gemm.h"
+
+namespace umd {
+
+namespace {
+
+constexpr int BM = 64, BN = 64, BK = 16;
+
+__global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    // loader coordinates: A tile 64 rows x 16 k (float4 along k), B tile 16 k x 64 cols
+    const int ar = tid >> 2, ak = (tid & 3) * 4;
+    const int bk = tid >> 4, bc = (tid & 15) * 4;
+    for (int k0 = 0; k0 < g.K; k0 += BK) {
+        float4 av = make_float4(0.f, 0.f, 0.f, 0.f), bv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m0 + ar < g.M && k0 + ak < g.K)
+            av = *reinterpret_cast<const float4*>(g.A + (size_t)(m0 + ar) * g.lda + k0 + ak);
+        if (k0 + bk < g.K && n0 + bc < g.N)
+            bv = __ldg(reinterpret_cast<const float4*>(g.B + (size_t)(k0 + bk) * g.ldb + n0 + bc));
+        As[ak][ar] = av.x; As[ak + 1][ar] = av.y; As[ak + 2][ar] = av.z; As[ak + 3][ar] = av.w;
+        *reinterpret_cast<float4*>(&Bs[bk][bc]) = bv;
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] += a[i] * b[j];
+        }
+        __syncthreads();
+    }
+    const int n = n0 + tx * 4;
+    if (n >= g.N) return;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= g.M) continue;
+        float v[4] = {acc[i][0], acc[i][1], acc[i][2], acc[i][3]};
+        gemm_epilogue4(g, m, n, v);
+    }
+}
+
+// scalar head: E_i = h . w_head + b_head + E_ref[type]; seeds the backward pass with
+// dE/dY_last = w_head * SiLU'(Y_last)
+__global__ void k_head(int n, int F, const float* __restrict__ h, const float* __restrict__ w, float b_head,
+                       const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
+                       float* __restrict__ pre_last, double* __restrict__ e_atom, bool want_grad) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= n) return;
+    const float* hr = h + (size_t)warp * F;
+    float s = 0.f;
+    for (int f = lane; f < F; f += 32) s += hr[f] * __ldg(w + f);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0)
+        e_atom[a0 + warp] = (double)s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + warp]);
+    if (want_grad) {
+        float* pr = pre_last + (size_t)warp * F;
+        for (int f = lane; f < F; f += 32) pr[f] = __ldg(w + f) * silu_grad(pr[f]);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {
+    if (g.M <= 0 || g.N <= 0) return cudaSuccess;
+    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
+    k_gemm_simt<<<grid, 256, 0, st>>>(g);
+    return cudaGetLastError();
+}
+
+static cudaError_t run_gemm(const GemmArgs& g, int path, cudaStream_t st) {
+    if (path == 2 && gemm_tc_supported(g)) return launch_gemm_tc(g, st);
+    return launch_gemm_simt(g, st);
+}
+
+cudaError_t launch_mlp(const MlpArgs& a, cudaStream_t st) {
+    const Dims& d = a.d;
+    const int n = a.n, F = d.F, NH = d.n_hidden;
+    if (n <= 0) return cudaSuccess;
+    const size_t layer = (size_t)n * F;
+    float* hb[2] = {a.hbuf, a.hbuf + layer};
+    const bool res0 = (d.D_out == F);
+    cudaError_t e;
+    // ---- forward --------------------------------------------------------------------
+    for (int t = 0; t < NH; ++t) {
+        GemmArgs g = {};
+        g.mode = 0;
+        g.M = n; g.N = F;
+        if (t == 0) { g.A = a.desc; g.lda = d.DP; g.K = d.DP; g.res = res0 ? a.desc : nullptr; g.ldres = d.DP; }
+        else { g.A = hb[(t - 1) & 1]; g.lda = F; g.K = F; g.res = hb[(t - 1) & 1]; g.ldres = F; }
+        g.B = a.m.theta[t]; g.ldb = F;
+        g.bias = a.m.bias[t];
+        g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
+        g.out = hb[t & 1]; g.ldout = F;
+        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+    }
+    {
+        const int warps = 8, blocks = (n + warps - 1) / warps;
+        k_head<<<blocks, warps * 32, 0, st>>>(n, F, hb[(NH - 1) & 1], a.m.w_head, a.m.b_head, a.m.e_ref, a.type_s,
+                                             a.a0, a.want_grad ? a.pre + (size_t)(NH - 1) * layer : nullptr,
+                                             a.e_atom, a.want_grad);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    if (!a.want_grad) return cudaSuccess;
+    // ---- backward: dE/dY_t sits in pre[t]; dE/dh_t alternates between the two hbuf slots
+    int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
+    bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
+    for (int t = NH - 1; t >= 1; --t) {
+        GemmArgs g = {};
+        g.mode = 1;
+        g.M = n; g.N = F; g.K = F;
+        g.A = a.pre + (size_t)t * layer; g.lda = F;
+        g.B = a.m.thetaT[t]; g.ldb = F;
+        if (vec_grad) g.rvec = a.m.w_head; else { g.res = hb[slot]; g.ldres = F; }
+        const int out_slot = vec_grad ? 0 : 1 - slot;
+        const bool need_dh = (t - 1 >= 1) || res0;
+        g.out = need_dh ? hb[out_slot] : nullptr; g.ldout = F;
+        g.pre = a.pre + (size_t)(t - 1) * layer; g.ldpre = F;
+        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+        slot = out_slot; vec_grad = false;
+    }
+    {
+        GemmArgs g = {};
+        g.mode = 1;
+        g.M = n; g.N = d.DP; g.K = F;
+        g.A = a.pre; g.lda = F;
+        g.B = a.m.thetaT[0]; g.ldb = d.DP;
+        if (res0) {
+            if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
+            else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }
+        }
+        g.out = a.desc; g.ldout = d.DP;
+        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace umd

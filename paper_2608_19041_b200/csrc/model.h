@@ -1,0 +1,32 @@
+// Host-side model construction: blob parsing and the create-time precomputation that the
+// paper's compressed inference performs once per model (radial table, pair cache, Gaunt
+// couplings).  Plain C++, double precision.
+#pragma once
+
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+namespace umd {
+
+struct HostModel {
+    Dims d;
+    double rc = 0, dx = 0;
+    std::vector<float> table;      // [n_rows][6][CP]
+    std::vector<float> pairmod;    // [T*T][2+R][C0]
+    std::vector<float> X0, W1p, W2p, A1, A2, mu, inv_sigma;
+    std::vector<std::vector<float>> theta, thetaT, bias;   // per hidden layer
+    std::vector<float> w_head, e_ref;
+    float b_head = 0;
+    GauntSparse g123, g233;
+};
+
+// Fills `d` widths for (C0, L, R); false when the triple is unsupported.
+bool derive_dims(int C0, int L, int R, Dims* d);
+
+// Returns UMLMD_OK or an error code with `err` set.
+int build_host_model(const void* blob, size_t bytes, double table_dx_override, HostModel* out,
+                     std::string* err);
+
+}  // namespace umd

@@ -1,0 +1,409 @@
+// Cell-list neighbor builder producing destination-sorted CSR edges.
+//
+// Atoms are folded into the cell, binned into cells at least r_list wide, sorted by cell
+// (stable radix sort, so the internal numbering is deterministic) and renumbered in that
+// order.  One warp per centre then walks the surrounding cells twice -- a count pass and a
+// fill pass with an in-warp prefix count that keeps candidates in traversal order -- so the
+// edge list comes out grouped by destination with no atomics and a reproducible order.
+// A last pass finds, for every edge (i <- j, n), the slot of its reverse (j <- i, -n).
+//
+// The distance predicate is the paper's neighbor-set definition evaluated in double
+// precision with explicit round-to-nearest adds and multiplies (no contraction into fused
+// multiply-adds), which makes the edge set reproducible bit for bit.
+#include <cub/cub.cuh>
+
+#include <cmath>
+
+#include "alloc.h"
+#include "kernels.h"
+
+namespace umd {
+
+namespace {
+
+struct Grid {
+    double L[3];        // cell edge lengths
+    double lo[3];       // binning origin
+    double inv_cw[3];   // 1 / bin width
+    int nc[3];          // bins per direction
+    int m[3];           // bin reach per direction
+    int pbc[3];
+};
+
+__device__ __forceinline__ int floor_div(int a, int b) {
+    int q = a / b;
+    if ((a % b != 0) && ((a < 0) != (b < 0))) --q;
+    return q;
+}
+
+__device__ __forceinline__ int pack_shift(int nx, int ny, int nz) {
+    return (nx & 0xff) | ((ny & 0xff) << 8) | ((nz & 0xff) << 16);
+}
+
+// fold positions into the cell, bin them
+__global__ void k_fold_bin(int N, const double* __restrict__ pos, Grid g, double* __restrict__ wpos,
+                           int* __restrict__ img_o, int* __restrict__ key, int* __restrict__ idx,
+                           int* __restrict__ err) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    int c[3];
+    bool bad = false;
+    for (int k = 0; k < 3; ++k) {
+        const double x = pos[3 * (size_t)i + k];
+        if (!isfinite(x)) bad = true;
+        double w = x;
+        int fl = 0;
+        if (g.pbc[k]) {
+            const double frac = x / g.L[k];
+            const double f = floor(frac);
+            w = __dmul_rn(__dsub_rn(frac, f), g.L[k]);
+            fl = (int)f;
+            if (fabs(f) > 1.0e6) bad = true;
+        }
+        wpos[3 * (size_t)i + k] = w;
+        img_o[3 * (size_t)i + k] = fl;
+        int ck = (int)floor((w - g.lo[k]) * g.inv_cw[k]);
+        ck = ck < 0 ? 0 : (ck >= g.nc[k] ? g.nc[k] - 1 : ck);
+        c[k] = ck;
+    }
+    if (bad) {
+        atomicOr(err, kErrNonFinite);
+        c[0] = c[1] = c[2] = 0;
+    }
+    key[i] = (c[2] * g.nc[1] + c[1]) * g.nc[0] + c[0];
+    idx[i] = i;
+}
+
+__global__ void k_cell_start(int ncell, int N, const int* __restrict__ skey, int* __restrict__ cell_start) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c > ncell) return;
+    int lo = 0, hi = N;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (skey[mid] < c) lo = mid + 1; else hi = mid;
+    }
+    cell_start[c] = lo;
+}
+
+__global__ void k_gather_sorted(int N, const int* __restrict__ sidx, const double* __restrict__ wpos,
+                                const int* __restrict__ img_o, const int* __restrict__ type,
+                                int* __restrict__ perm, double* __restrict__ xs0, double* __restrict__ xs,
+                                int* __restrict__ img, int* __restrict__ type_s) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int o = sidx[i];
+    perm[i] = o;
+    type_s[i] = type[o];
+    for (int k = 0; k < 3; ++k) {
+        const double w = wpos[3 * (size_t)o + k];
+        xs0[3 * (size_t)i + k] = w;
+        xs[3 * (size_t)i + k] = w;
+        img[3 * (size_t)i + k] = img_o[3 * (size_t)o + k];
+    }
+}
+
+// One warp per centre.  FILL = false: count accepted candidates.  FILL = true: write them.
+template <bool FILL>
+__global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ skey,
+                             const int* __restrict__ cell_start, const double* __restrict__ xs0,
+                             int* __restrict__ deg, const int* __restrict__ row_ptr,
+                             int* __restrict__ src, int* __restrict__ shift, int* __restrict__ err) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int i = warp;
+    const int key = skey[i];
+    const int cx = key % g.nc[0], cy = (key / g.nc[0]) % g.nc[1], cz = key / (g.nc[0] * g.nc[1]);
+    const double xi = xs0[3 * (size_t)i], yi = xs0[3 * (size_t)i + 1], zi = xs0[3 * (size_t)i + 2];
+    int count = 0;
+    const int base_out = FILL ? row_ptr[i] : 0;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    for (int dz = -g.m[2]; dz <= g.m[2]; ++dz) {
+        int zc = cz + dz, nz = 0;
+        if (g.pbc[2]) { nz = floor_div(zc, g.nc[2]); zc -= nz * g.nc[2]; }
+        else if (zc < 0 || zc >= g.nc[2]) continue;
+        const double sz = __dmul_rn((double)nz, g.L[2]);
+        for (int dy = -g.m[1]; dy <= g.m[1]; ++dy) {
+            int yc = cy + dy, ny = 0;
+            if (g.pbc[1]) { ny = floor_div(yc, g.nc[1]); yc -= ny * g.nc[1]; }
+            else if (yc < 0 || yc >= g.nc[1]) continue;
+            const double sy = __dmul_rn((double)ny, g.L[1]);
+            for (int dx = -g.m[0]; dx <= g.m[0]; ++dx) {
+                int xc = cx + dx, nx = 0;
+                if (g.pbc[0]) { nx = floor_div(xc, g.nc[0]); xc -= nx * g.nc[0]; }
+                else if (xc < 0 || xc >= g.nc[0]) continue;
+                const double sx = __dmul_rn((double)nx, g.L[0]);
+                const int cell = (zc * g.nc[1] + yc) * g.nc[0] + xc;
+                const int beg = cell_start[cell], end = cell_start[cell + 1];
+                const bool self_img = (nx == 0 && ny == 0 && nz == 0);
+                for (int b = beg; b < end; b += 32) {
+                    const int j = b + lane;
+                    bool ok = false;
+                    if (j < end) {
+                        const double ddx = __dsub_rn(__dadd_rn(xs0[3 * (size_t)j], sx), xi);
+                        const double ddy = __dsub_rn(__dadd_rn(xs0[3 * (size_t)j + 1], sy), yi);
+                        const double ddz = __dsub_rn(__dadd_rn(xs0[3 * (size_t)j + 2], sz), zi);
+                        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(ddx, ddx), __dmul_rn(ddy, ddy)),
+                                                    __dmul_rn(ddz, ddz));
+                        ok = (d2 < rl2) && !(self_img && j == i);
+                    }
+                    const unsigned mask = __ballot_sync(0xffffffffu, ok);
+                    if (FILL && ok) {
+                        const int p = base_out + count + __popc(mask & lt_mask);
+                        src[p] = j;
+                        shift[p] = pack_shift(nx, ny, nz);
+                    }
+                    count += __popc(mask);
+                }
+                if (nx < -127 || nx > 127 || ny < -127 || ny > 127 || nz < -127 || nz > 127)
+                    if (lane == 0) atomicOr(err, kErrShiftRange);
+            }
+        }
+    }
+    if (!FILL && lane == 0) deg[i] = count;
+}
+
+// rev[e] = slot of (j <- i, -n) for e = (i <- j, n); -1 when absent (can only happen for
+// pairs whose two orientations round to opposite sides of the list radius).
+__global__ void k_reverse_map(int N, const int* __restrict__ row_ptr, const int* __restrict__ src,
+                              const int* __restrict__ shift, int* __restrict__ rev) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int i = warp;
+    const int e0 = row_ptr[i], e1 = row_ptr[i + 1];
+    for (int e = e0 + lane; e < e1; e += 32) {
+        const int j = src[e];
+        const int s = shift[e];
+        const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff),
+                  nz = (int)(signed char)((s >> 16) & 0xff);
+        const int want = pack_shift(-nx, -ny, -nz);
+        int found = -1;
+        const int f0 = row_ptr[j], f1 = row_ptr[j + 1];
+        for (int f = f0; f < f1; ++f) {
+            if (src[f] == i && shift[f] == want) { found = f; break; }
+        }
+        rev[e] = found;
+    }
+}
+
+__global__ void k_gather_positions(int N, const int* __restrict__ perm, const int* __restrict__ img,
+                                   const double* __restrict__ pos, const double* __restrict__ xs0,
+                                   double Lx, double Ly, double Lz, double max_disp2,
+                                   double* __restrict__ xs, int* __restrict__ err) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int o = perm[i];
+    const double L[3] = {Lx, Ly, Lz};
+    double d2 = 0;
+    bool bad = false;
+    for (int k = 0; k < 3; ++k) {
+        const double x = pos[3 * (size_t)o + k] - (double)img[3 * (size_t)i + k] * L[k];
+        if (!isfinite(x)) bad = true;
+        xs[3 * (size_t)i + k] = x;
+        const double d = x - xs0[3 * (size_t)i + k];
+        d2 += d * d;
+    }
+    if (bad) atomicOr(err, kErrNonFinite);
+    else if (d2 > max_disp2) atomicOr(err, kErrStale);
+}
+
+// ---- export in caller numbering ------------------------------------------------------
+__global__ void k_export_deg(int N, const int* __restrict__ perm, const int* __restrict__ row_ptr,
+                             int* __restrict__ deg_o) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    deg_o[perm[i]] = row_ptr[i + 1] - row_ptr[i];
+    if (i == 0) deg_o[N] = 0;
+}
+
+__global__ void k_export_rows(int N, const int* __restrict__ perm, const int* __restrict__ row_ptr,
+                              const int* __restrict__ src, const int* __restrict__ shift,
+                              const int* __restrict__ row_ptr_o, int* __restrict__ src_o,
+                              signed char* __restrict__ shift_o) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int i = warp, o = perm[i];
+    const int e0 = row_ptr[i], n = row_ptr[i + 1] - e0, q0 = row_ptr_o[o];
+    for (int k = lane; k < n; k += 32) {
+        const int s = shift[e0 + k];
+        src_o[q0 + k] = perm[src[e0 + k]];
+        shift_o[3 * (size_t)(q0 + k)] = (signed char)(s & 0xff);
+        shift_o[3 * (size_t)(q0 + k) + 1] = (signed char)((s >> 8) & 0xff);
+        shift_o[3 * (size_t)(q0 + k) + 2] = (signed char)((s >> 16) & 0xff);
+    }
+}
+
+#define NB_CHECK(call)                                                              \
+    do {                                                                            \
+        cudaError_t e__ = (call);                                                   \
+        if (e__ != cudaSuccess) {                                                   \
+            *err = std::string(#call) + ": " + cudaGetErrorString(e__);             \
+            return UMLMD_E_CUDA;                                                    \
+        }                                                                           \
+    } while (0)
+
+}  // namespace
+
+void neighbor_free(NeighborDev* nb) {
+    void* ptrs[] = {nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
+                    nb->shift, nb->rev, nb->key, nb->key2, nb->idx, nb->idx2, nb->cell_start, nb->deg,
+                    nb->cub_tmp};
+    for (void* p : ptrs)
+        dev_free(p);
+    *nb = NeighborDev();
+}
+
+int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int32_t* d_type,
+                   const double L[3], const int pbc[3], double skin, double rc, int* d_err,
+                   cudaStream_t st, std::string* err) {
+    if (N64 > 0x7fff0000LL) { *err = "too many atoms for 32-bit indices"; return UMLMD_E_INVALID_ARG; }
+    const int N = (int)N64;
+    const double r_list = rc + skin;
+    Grid g;
+    // per-direction bounding interval for non-periodic directions (host reduction of a
+    // device min/max would cost a sync as well; the list build synchronises anyway)
+    double lo[3] = {0, 0, 0}, ext[3] = {L[0], L[1], L[2]};
+    if (!(pbc[0] && pbc[1] && pbc[2]) && N > 0) {
+        std::vector<double> hp((size_t)N * 3);
+        NB_CHECK(cudaMemcpyAsync(hp.data(), d_pos, sizeof(double) * 3 * (size_t)N, cudaMemcpyDeviceToHost, st));
+        NB_CHECK(cudaStreamSynchronize(st));
+        for (int k = 0; k < 3; ++k) {
+            if (pbc[k]) continue;
+            double mn = hp[k], mx = hp[k];
+            for (int i = 1; i < N; ++i) { const double v = hp[3 * (size_t)i + k]; if (v < mn) mn = v; if (v > mx) mx = v; }
+            if (!std::isfinite(mn) || !std::isfinite(mx)) { *err = "non-finite position"; return UMLMD_E_NONFINITE; }
+            lo[k] = mn; ext[k] = (mx - mn) + 1e-6;
+        }
+    }
+    int64_t ncell = 1;
+    const double rl_pad = r_list * (1.0 + 1e-9) + 1e-12;
+    for (int k = 0; k < 3; ++k) {
+        g.L[k] = L[k]; g.lo[k] = lo[k]; g.pbc[k] = pbc[k] ? 1 : 0;
+        int nc = (int)std::floor(ext[k] / rl_pad);
+        if (nc < 1) nc = 1;
+        if (nc > 1024) nc = 1024;
+        g.nc[k] = nc;
+    }
+    // keep the cell table modest relative to the atom count
+    while ((int64_t)g.nc[0] * g.nc[1] * g.nc[2] > 8 * (int64_t)N + 64) {
+        int kmax = 0;
+        for (int k = 1; k < 3; ++k) if (g.nc[k] > g.nc[kmax]) kmax = k;
+        if (g.nc[kmax] == 1) break;
+        g.nc[kmax] = (g.nc[kmax] + 1) / 2;
+    }
+    for (int k = 0; k < 3; ++k) {
+        const double cw = ext[k] / g.nc[k];
+        g.inv_cw[k] = 1.0 / cw;
+        g.m[k] = pbc[k] || g.nc[k] > 1 ? (int)std::ceil(r_list / cw) : 0;
+        if (!pbc[k] && g.m[k] > g.nc[k] - 1) g.m[k] = g.nc[k] - 1;
+        if (g.m[k] > 127) { *err = "cell much smaller than the list radius (more than 127 images)"; return UMLMD_E_UNSUPPORTED_CELL; }
+        ncell *= g.nc[k];
+    }
+
+    nb->N = N; nb->skin = skin; nb->r_list = r_list;
+    for (int k = 0; k < 3; ++k) { nb->L[k] = L[k]; nb->pbc[k] = pbc[k] ? 1 : 0; }
+    if (N == 0) { nb->E = 0; return UMLMD_OK; }
+
+    // per-atom arrays (all sized from one capacity)
+    if (N > nb->N_cap || !nb->wpos) {
+        const int64_t need = N + 1;
+        int64_t c;
+        c = 0; NB_CHECK(dev_ensure(&nb->wpos, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->xs0, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->xs, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->img, &c, need * 6));   // sorted-order and caller-order halves
+        c = 0; NB_CHECK(dev_ensure(&nb->perm, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->type_s, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->row_ptr, &c, need + 1));
+        c = 0; NB_CHECK(dev_ensure(&nb->key, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->key2, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->idx, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->idx2, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->deg, &c, need + 1));
+        nb->N_cap = N;
+    }
+    NB_CHECK(dev_ensure(&nb->cell_start, &nb->ncell_cap, ncell + 2));
+    int* img_o = nb->img + 3 * (size_t)(N + 1);
+
+    const int TB = 256;
+    k_fold_bin<<<(N + TB - 1) / TB, TB, 0, st>>>(N, d_pos, g, nb->wpos, img_o, nb->key, nb->idx, d_err);
+    int end_bit = 1;
+    while ((1LL << end_bit) < ncell) ++end_bit;
+    size_t need_tmp = 0, need_scan = 0;
+    cub::DeviceRadixSort::SortPairs(nullptr, need_tmp, nb->key, nb->key2, nb->idx, nb->idx2, N, 0, end_bit, st);
+    cub::DeviceScan::ExclusiveSum(nullptr, need_scan, nb->deg, nb->row_ptr, N + 1, st);
+    if (need_scan > need_tmp) need_tmp = need_scan;
+    if (need_tmp > nb->cub_bytes) {
+        if (nb->cub_tmp) dev_free(nb->cub_tmp);
+        nb->cub_tmp = nullptr; nb->cub_bytes = 0;
+        NB_CHECK(dev_malloc(&nb->cub_tmp, need_tmp + 256));
+        nb->cub_bytes = need_tmp + 256;
+    }
+    size_t tmp_bytes = nb->cub_bytes;
+    NB_CHECK(cub::DeviceRadixSort::SortPairs(nb->cub_tmp, tmp_bytes, nb->key, nb->key2, nb->idx, nb->idx2, N,
+                                             0, end_bit, st));
+    k_cell_start<<<(int)((ncell + 1 + TB - 1) / TB), TB, 0, st>>>((int)ncell, N, nb->key2, nb->cell_start);
+    k_gather_sorted<<<(N + TB - 1) / TB, TB, 0, st>>>(N, nb->idx2, nb->wpos, img_o, d_type, nb->perm, nb->xs0,
+                                                      nb->xs, nb->img, nb->type_s);
+    const double rl2 = r_list * r_list;
+    const int warps_per_block = TB / 32;
+    const int wb = (N + warps_per_block - 1) / warps_per_block;
+    k_scan_cells<false><<<wb, TB, 0, st>>>(N, g, rl2, nb->key2, nb->cell_start, nb->xs0, nb->deg, nullptr,
+                                           nullptr, nullptr, d_err);
+    NB_CHECK(cudaMemsetAsync(nb->deg + N, 0, sizeof(int), st));
+    tmp_bytes = nb->cub_bytes;
+    NB_CHECK(cub::DeviceScan::ExclusiveSum(nb->cub_tmp, tmp_bytes, nb->deg, nb->row_ptr, N + 1, st));
+    int total = 0;
+    NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(int), cudaMemcpyDeviceToHost, st));
+    NB_CHECK(cudaStreamSynchronize(st));
+    if (total < 0) { *err = "edge count overflows 32-bit indices"; return UMLMD_E_INVALID_ARG; }
+    nb->E = total;
+    if (total > nb->E_cap) {
+        int64_t c;
+        c = 0; NB_CHECK(dev_ensure(&nb->src, &c, total, 1.1));
+        c = 0; NB_CHECK(dev_ensure(&nb->shift, &c, total, 1.1));
+        c = 0; NB_CHECK(dev_ensure(&nb->rev, &c, total, 1.1));
+        nb->E_cap = c;
+    }
+    if (total > 0) {
+        k_scan_cells<true><<<wb, TB, 0, st>>>(N, g, rl2, nb->key2, nb->cell_start, nb->xs0, nullptr,
+                                              nb->row_ptr, nb->src, nb->shift, d_err);
+        k_reverse_map<<<wb, TB, 0, st>>>(N, nb->row_ptr, nb->src, nb->shift, nb->rev);
+    }
+    NB_CHECK(cudaGetLastError());
+    return UMLMD_OK;
+}
+
+int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
+                    cudaStream_t st, std::string* err) {
+    const int N = (int)nb->N;
+    if (N == 0) {
+        NB_CHECK(cudaMemsetAsync(d_row_ptr, 0, sizeof(int), st));
+        return UMLMD_OK;
+    }
+    const int TB = 256;
+    k_export_deg<<<(N + TB - 1) / TB, TB, 0, st>>>(N, nb->perm, nb->row_ptr, nb->deg);
+    size_t tmp_bytes = nb->cub_bytes;
+    NB_CHECK(cub::DeviceScan::ExclusiveSum(nb->cub_tmp, tmp_bytes, nb->deg, d_row_ptr, N + 1, st));
+    const int wb = (N + TB / 32 - 1) / (TB / 32);
+    if (nb->E > 0)
+        k_export_rows<<<wb, TB, 0, st>>>(N, nb->perm, nb->row_ptr, nb->src, nb->shift, d_row_ptr, d_src,
+                                         (signed char*)d_shift);
+    NB_CHECK(cudaGetLastError());
+    return UMLMD_OK;
+}
+
+cudaError_t launch_gather_positions(const NeighborDev& nb, const double* d_pos, int* d_err, cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    const double half = 0.5 * nb.skin;
+    // a tiny slack keeps a fresh build with zero skin from tripping on its own rounding
+    const double max_disp2 = half * half + 1e-20;
+    k_gather_positions<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, nb.img, d_pos, nb.xs0, nb.L[0], nb.L[1],
+                                                        nb.L[2], max_disp2, nb.xs, d_err);
+    return cudaGetLastError();
+}
+
+}  // namespace umd

@@ -1,0 +1,212 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on
+the same seeded inputs.
+
+Tolerances (fp32 kernels against an fp64 reference):
+  * neighbor lists: identical as sorted sets of (j, n) per centre;
+  * aggregated sums and feature vector: 2e-5 of the largest entry of the block compared;
+  * atomic energies: |dE_i| <= 1e-5 * max(|E_i|, rms(E));   total energy likewise per atom;
+  * forces: max |dF| <= 1e-4 eV/Angstrom;   virial: |dXi| / N <= 1e-5 eV.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dpa4c as orc
+from workloads import CONFIGS, SMALL_PROFILES, load_calibration, make_blob, make_system
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_19041_b200 import binding
+    return binding
+
+
+def _dev(a, dtype):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype).cuda().contiguous()
+
+
+def _rows_from_gpu(model, N):
+    row_ptr, src, shift = model.get_neighbors()
+    row_ptr, src, shift = row_ptr.cpu().numpy(), src.cpu().numpy(), shift.cpu().numpy()
+    rows = []
+    for i in range(N):
+        a, b = row_ptr[i], row_ptr[i + 1]
+        ent = np.concatenate([src[a:b, None].astype(np.int64), shift[a:b].astype(np.int64)], axis=1)
+        order = np.lexsort((ent[:, 3], ent[:, 2], ent[:, 1], ent[:, 0]))
+        rows.append(ent[order])
+    return rows
+
+
+def _build(blob, s, skin=0.0, **kw):
+    m = _binding().Model(blob, **kw)
+    pos = _dev(s["pos"], torch.float64)
+    types = _dev(s["types"], torch.int32)
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], skin)
+    return m, pos
+
+
+TINY = [
+    dict(kind="random_box", atoms=6, edges=(4.0, 4.5, 5.0), min_dist=1.2, seed=11, n_types=1, masses=[1.0], shift=True),
+    dict(kind="random_box", atoms=14, edges=(9.0, 13.0, 12.5), min_dist=1.2, seed=12, n_types=1, masses=[1.0], shift=True),
+    dict(kind="random_box", atoms=8, edges=(3.1, 14.0, 7.3), min_dist=1.2, seed=13, n_types=1, masses=[1.0]),
+    dict(kind="random_box", atoms=40, edges=(14.5, 12.1, 19.0), min_dist=1.2, seed=14, n_types=1, masses=[1.0]),
+    dict(kind="random_box", atoms=12, edges=(6.0, 6.0, 6.0), min_dist=1.5, seed=15, n_types=1, masses=[1.0], pbc=[0, 0, 0]),
+    dict(kind="random_box", atoms=30, edges=(20.0, 7.0, 9.0), min_dist=1.5, seed=16, n_types=1, masses=[1.0], pbc=[0, 1, 1]),
+    dict(kind="random_box", atoms=300, edges=(21.0, 22.5, 30.0), min_dist=1.5, seed=17, n_types=1, masses=[1.0], shift=True),
+]
+
+
+@pytest.mark.parametrize("desc", TINY, ids=lambda d: f"n{d['atoms']}_{'x'.join(map(str, d['edges']))}")
+@pytest.mark.parametrize("skin", [0.0, 1.0])
+def test_neighbor_lists_bit_exact_on_small_cells(desc, skin):
+    s = make_system(desc)
+    blob = make_blob(SMALL_PROFILES["p8_2_0"], seed=1)
+    m, _ = _build(blob, s, skin=skin)
+    got = _rows_from_gpu(m, len(s["pos"]))
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    ref = orc.neighbor_rows(pos, s["cell"], s["pbc"], 6.0 + skin)
+    assert m.query()["n_edges"] == sum(len(r) for r in ref)
+    for a, b in zip(got, ref):
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["cfg1_al108", "cfg2_cu4000"])
+def test_neighbor_lists_bit_exact_on_workloads(name):
+    cfg = CONFIGS[name]
+    s = make_system(cfg["system"])
+    blob = make_blob(SMALL_PROFILES["p8_2_0"], seed=1)
+    for skin in (0.0, 1.0):
+        m, _ = _build(blob, s, skin=skin)
+        got = _rows_from_gpu(m, len(s["pos"]))
+        pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+        ref = orc.neighbor_rows(pos, s["cell"], s["pbc"], 6.0 + skin)
+        assert all(np.array_equal(a, b) for a, b in zip(got, ref))
+        m.close()
+
+
+def test_empty_system_and_single_atom():
+    blob = make_blob(SMALL_PROFILES["p8_2_0"], seed=1, e_ref_scale=0.5, bias_scale=0.2)
+    B = _binding()
+    m = B.Model(blob)
+    pos = torch.zeros((0, 3), dtype=torch.float64, device="cuda")
+    types = torch.zeros((0,), dtype=torch.int32, device="cuda")
+    m.build_neighbors(pos, types, np.eye(3) * 20.0)
+    out = m.compute(pos)
+    assert out["energy"] == 0.0 and np.all(out["virial"] == 0)
+    # one isolated atom: no edges, energy = MLP of the empty-neighbourhood features
+    s = dict(pos=np.array([[1.0, 2.0, 3.0]]), types=np.array([1], dtype=np.int32), cell=np.eye(3) * 20.0,
+             pbc=np.array([1, 1, 1]))
+    m, pos = _build(blob, s)
+    assert m.query()["n_edges"] == 0
+    out = m.compute(pos, atom_energy=True)
+    ref = orc.Oracle(blob).compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    assert abs(out["energy"] - ref["E"]) < 1e-5 * max(1.0, abs(ref["E"]))
+    assert out["forces"].abs().max().item() == 0.0
+
+
+def _compare(blob, s, tol_scale=1.0, skin=0.0, check_intermediates=True, **kw):
+    o = orc.Oracle(blob)
+    ref = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    m, pos = _build(blob, s, skin=skin, **kw)
+    N = len(s["pos"])
+    if check_intermediates:
+        m.compute(pos, forces=False, virial=False)
+        state, desc = m.get_intermediates()
+        state, desc = state.cpu().numpy().astype(np.float64), desc.cpu().numpy().astype(np.float64)
+        ty = torch.from_numpy(s["types"].astype(np.int64))
+        dst_t = torch.from_numpy(ref["dst"])
+        A, s0, s1 = orc.aggregate(o.p, o.prm, o.pair, N, dst_t, ty[dst_t], ty[torch.from_numpy(ref["src"])],
+                                  torch.from_numpy(ref["rij"]))
+        flat = torch.cat([a.reshape(N, -1) for a in A] + [s0[:, None], s1[:, None]], dim=1).numpy()
+        off = 0
+        for l, a in enumerate(A):
+            w = a[0].numel()
+            blk = flat[:, off:off + w]
+            assert np.abs(state[:, off:off + w] - blk).max() <= 2e-5 * tol_scale * max(np.abs(blk).max(), 1e-30), f"A_{l}"
+            off += w
+        assert np.abs(state[:, off:] - flat[:, off:]).max() <= 2e-5 * np.abs(flat[:, off:]).max()
+        Dref = (ref["D_raw"] - o.prm["mu"].numpy()) / o.prm["sigma"].numpy()
+        err = np.abs(desc - Dref)
+        assert err.max() <= 5e-5 * tol_scale * np.abs(Dref).max(), (err.max(), np.unravel_index(err.argmax(), err.shape))
+    out = m.compute(pos, atom_energy=True)
+    Ei = out["atom_energy"].cpu().numpy()
+    F = out["forces"].cpu().numpy()
+    rms = np.sqrt(np.mean(ref["E_i"] ** 2))
+    assert (np.abs(Ei - ref["E_i"]) <= 1e-5 * tol_scale * np.maximum(np.abs(ref["E_i"]), rms)).all(), \
+        np.abs(Ei - ref["E_i"]).max() / rms
+    assert abs(out["energy"] - ref["E"]) / N <= 1e-5 * tol_scale * max(abs(ref["E"]) / N, rms)
+    assert np.abs(F - ref["F"]).max() <= 1e-4 * tol_scale, np.abs(F - ref["F"]).max()
+    assert np.abs(out["virial"] - ref["virial"]).max() / N <= 1e-5 * tol_scale
+    m.close()
+    return ref, out
+
+
+SYS_SMALL = dict(kind="random_box", atoms=60, edges=(9.5, 10.5, 12.0), min_dist=1.7, seed=31, masses=[1.0] * 3)
+
+
+@pytest.mark.parametrize("name", sorted(SMALL_PROFILES))
+def test_energy_force_virial_parity_small_profiles(name):
+    p = SMALL_PROFILES[name]
+    blob = make_blob(p, seed=40, bias_scale=0.2, e_ref_scale=0.5)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    _compare(blob, s)
+
+
+def test_parity_with_skin_and_multi_image_box():
+    p = SMALL_PROFILES["p16_3_2"]
+    blob = make_blob(p, seed=41, bias_scale=0.2)
+    s = make_system(dict(kind="random_box", atoms=16, edges=(5.0, 7.7, 8.1), min_dist=1.6, seed=32,
+                         n_types=p["T"], masses=[1.0] * p["T"], shift=True))
+    _compare(blob, s, skin=1.0)
+
+
+def test_parity_isolated_cluster():
+    p = SMALL_PROFILES["p32_2_4"]
+    blob = make_blob(p, seed=42)
+    s = make_system(dict(kind="random_box", atoms=20, edges=(7.0, 7.0, 7.0), min_dist=1.6, seed=33,
+                         n_types=p["T"], masses=[1.0] * p["T"], pbc=[0, 0, 0]))
+    _compare(blob, s)
+
+
+def test_parity_with_node_tiling():
+    # several workspace tiles with a ragged last tile
+    p = SMALL_PROFILES["p16_2_0"]
+    blob = make_blob(p, seed=43, bias_scale=0.2)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"], atoms=75))
+    _compare(blob, s, check_intermediates=False, node_tile=32)
+
+
+@pytest.mark.parametrize("name", ["cfg1_al108", "cfg2_cu4000"])
+def test_parity_on_workloads(name):
+    cfg = CONFIGS[name]
+    s = make_system(cfg["system"])
+    blob = make_blob(cfg["profile"], cfg["weights_seed"], calibration=load_calibration(name))
+    _compare(blob, s)
+
+
+def test_results_are_bitwise_reproducible():
+    cfg = CONFIGS["cfg1_al108"]
+    s = make_system(cfg["system"])
+    blob = make_blob(cfg["profile"], cfg["weights_seed"], calibration=load_calibration("cfg1_al108"))
+    m, pos = _build(blob, s)
+    a = m.compute(pos)
+    b = m.compute(pos)
+    assert a["energy"] == b["energy"] and torch.equal(a["forces"], b["forces"])
+    assert np.array_equal(a["virial"], b["virial"])
+
+
+def test_stale_list_is_reported():
+    p = SMALL_PROFILES["p8_2_0"]
+    blob = make_blob(p, seed=44)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    m, pos = _build(blob, s, skin=0.4)
+    moved = pos.clone()
+    moved[3, 0] += 0.15
+    m.compute(moved)                       # within skin/2
+    moved[3, 0] += 0.2
+    with pytest.raises(_binding().UmlmdError) as e:
+        m.compute(moved)
+    assert e.value.code == -6
+    m.compute(pos)                         # the handle stays usable
