@@ -65,7 +65,8 @@ typedef struct umlmd_info {
     int32_t table_rows;
     double  rc, table_dx;
     int64_t n_atoms, n_edges;          /* of the current neighbor list (0 before a build)  */
-    int64_t device_bytes;              /* device memory currently held by the handle       */
+    int64_t device_bytes;              /* device memory currently held by the library      */
+    int64_t kernel_launches;           /* kernels of this library launched by the handle   */
 } umlmd_info;
 
 /* Widths for a (C0, L, R) triple without a handle; fills only the width fields.
@@ -177,6 +178,20 @@ int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc);
  */
 int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, double* out_g,
                             double* out_dg);
+
+/*
+ * Per-kernel-class accounting.  The handle always counts the kernels it launches; with
+ * profiling enabled it also brackets each class with CUDA events on its stream (a few
+ * microseconds of overhead per launch group, so leave it off when timing whole steps).
+ * umlmd_get_profile synchronises the stream, returns accumulated milliseconds and launch
+ * counts per class since the previous call (arrays of max_classes entries; *n_classes
+ * receives the number of classes) and resets them.  Class names: gather_positions,
+ * edge_forward, invariants_forward, mlp_forward, mlp_backward, invariants_backward,
+ * edge_backward, force_assembly, energy_virial_reduce, integrate, neighbor_build.
+ */
+int umlmd_set_profiling(umlmd_t* h, int enabled);
+int umlmd_get_profile(umlmd_t* h, int32_t max_classes, double* ms, int64_t* launches, int32_t* n_classes);
+const char* umlmd_profile_class_name(int32_t cls);
 
 /*
  * Read one entry of the ordered type-pair cache (host): out receives (2+R)*C0 doubles,

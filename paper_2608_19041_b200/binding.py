@@ -23,7 +23,8 @@ ERRORS = {
 EXPORTS = [
     "umlmd_profile_widths", "umlmd_create", "umlmd_destroy", "umlmd_query", "umlmd_last_error",
     "umlmd_build_neighbors", "umlmd_get_neighbors", "umlmd_compute", "umlmd_set_md_state", "umlmd_step",
-    "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache",
+    "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
+    "umlmd_get_profile", "umlmd_profile_class_name",
 ]
 
 
@@ -43,7 +44,7 @@ class Info(ctypes.Structure):
                 ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T", "C1", "C2", "K1", "K2", "S", "D_out", "H",
                  "H_pair", "table_rows")] + \
                [("rc", ctypes.c_double), ("table_dx", ctypes.c_double), ("n_atoms", ctypes.c_int64),
-                ("n_edges", ctypes.c_int64), ("device_bytes", ctypes.c_int64)]
+                ("n_edges", ctypes.c_int64), ("device_bytes", ctypes.c_int64), ("kernel_launches", ctypes.c_int64)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -68,8 +69,12 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_get_intermediates.argtypes = [vp, vp, vp]
     lib.umlmd_eval_radial_table.argtypes = [vp, i64, ctypes.POINTER(dbl), ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.umlmd_eval_pair_cache.argtypes = [vp, i32, i32, ctypes.POINTER(dbl)]
+    lib.umlmd_set_profiling.argtypes = [vp, ctypes.c_int]
+    lib.umlmd_get_profile.argtypes = [vp, i32, ctypes.POINTER(dbl), ctypes.POINTER(i64), ctypes.POINTER(i32)]
+    lib.umlmd_profile_class_name.argtypes = [i32]
+    lib.umlmd_profile_class_name.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name != "umlmd_last_error":
+        if name not in ("umlmd_last_error", "umlmd_profile_class_name"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -210,6 +215,21 @@ class Model:
         if rc != OK:
             self._raise(rc)
         return state, desc
+
+    def set_profiling(self, enabled):
+        rc = self._lib.umlmd_set_profiling(self._h, int(bool(enabled)))
+        if rc != OK:
+            self._raise(rc)
+
+    def get_profile(self):
+        """{class name: (milliseconds, launches)} since the previous call; resets the counters."""
+        ms = (ctypes.c_double * 16)()
+        ln = (ctypes.c_int64 * 16)()
+        n = ctypes.c_int32()
+        rc = self._lib.umlmd_get_profile(self._h, 16, ms, ln, ctypes.byref(n))
+        if rc != OK:
+            self._raise(rc)
+        return {self._lib.umlmd_profile_class_name(k).decode(): (ms[k], ln[k]) for k in range(n.value)}
 
     def eval_pair_cache(self, type_i, type_j):
         q = self.query()

@@ -34,9 +34,41 @@ struct umlmd {
     double* d_mass = nullptr; double* d_inv_mass = nullptr;
     bool have_md = false, have_force = false;
     int steps_since_build = 0;
+    // launch accounting and optional per-class timing
+    bool prof_on = false;
+    struct Span { int cls; cudaEvent_t a, b; };
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> free_events;
+    double prof_ms[16] = {0};
+    int64_t prof_launches[16] = {0};
+    int64_t launches_total = 0;
 };
 
+enum KernelClass { kGather = 0, kEdgeFwd, kInvFwd, kMlpFwd, kMlpBwd, kInvBwd, kEdgeBwd, kForce, kReduce, kIntegrate,
+                   kNeighbor, kClassCount };
+static const char* const kClassNames[kClassCount] = {
+    "gather_positions", "edge_forward", "invariants_forward", "mlp_forward", "mlp_backward", "invariants_backward",
+    "edge_backward", "force_assembly", "energy_virial_reduce", "integrate", "neighbor_build"};
+
 namespace {
+
+// counts the kernels a call site launches and, when profiling is on, brackets them with events
+struct Scope {
+    umlmd_t* h; int cls; cudaEvent_t a = nullptr;
+    static cudaEvent_t get(umlmd_t* h) {
+        cudaEvent_t e = nullptr;
+        if (!h->free_events.empty()) { e = h->free_events.back(); h->free_events.pop_back(); }
+        else cudaEventCreate(&e);
+        return e;
+    }
+    Scope(umlmd_t* h_, int cls_, int n) : h(h_), cls(cls_) {
+        h->launches_total += n; h->prof_launches[cls] += n;
+        if (h->prof_on) { a = get(h); cudaEventRecord(a, h->st); }
+    }
+    ~Scope() {
+        if (a) { cudaEvent_t b = get(h); cudaEventRecord(b, h->st); h->spans.push_back({cls, a, b}); }
+    }
+};
 
 int fail(umlmd_t* h, int code, const std::string& msg) {
     if (h) h->err = msg;
@@ -107,7 +139,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
     const Dims& d = h->d;
     NeighborDev& nb = h->nb;
     const int N = (int)nb.N;
-    API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st));
+    { Scope sc(h, kGather, 1); API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st)); }
     const int B = N < h->node_tile ? N : h->node_tile;
     int vpart_used = 0;
     for (int a0 = 0; a0 < N; a0 += B) {
@@ -118,25 +150,28 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
         ea.virial_part = h->virial_part + (size_t)vpart_used * 9;
-        API_CUDA(h, launch_edge_forward(ea, h->st));
+        { Scope sc(h, kEdgeFwd, 1); API_CUDA(h, launch_edge_forward(ea, h->st)); }
         InvArgs ia;
         ia.d = d; ia.m = h->md; ia.type_s = nb.type_s; ia.a0 = a0; ia.n = n; ia.state = h->state; ia.desc = h->desc;
-        API_CUDA(h, launch_invariants_forward(ia, h->st));
+        { Scope sc(h, kInvFwd, 1); API_CUDA(h, launch_invariants_forward(ia, h->st)); }
         MlpArgs ma;
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
-        API_CUDA(h, launch_mlp(ma, h->st));
+        { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
-            API_CUDA(h, launch_invariants_backward(ia, h->st));
+            { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
+            { Scope sc(h, kInvBwd, 1); API_CUDA(h, launch_invariants_backward(ia, h->st)); }
             int blocks = 0;
-            API_CUDA(h, launch_edge_backward(ea, &blocks, h->st));
+            { Scope sc(h, kEdgeBwd, 1); API_CUDA(h, launch_edge_backward(ea, &blocks, h->st)); }
             vpart_used += blocks;
         }
     }
     if (want_grad) {
+        Scope sc(h, kForce, d_force ? 2 : 1);
         API_CUDA(h, launch_force_assembly(nb, h->g, h->f_sorted, h->st));
         if (d_force) API_CUDA(h, launch_scatter_forces(nb, h->f_sorted, d_force, h->d_err, h->st));
     }
+    Scope sc(h, kReduce, d_atom_energy ? 3 : 2);
     API_CUDA(h, launch_reduce_energy_virial(h->e_atom, N, h->virial_part, vpart_used, h->scratch, h->d_out,
                                             h->d_err, h->st));
     if (d_atom_energy) API_CUDA(h, launch_scatter_atom_energy(nb, h->e_atom, d_atom_energy, h->st));
@@ -186,7 +221,7 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
                const int pbc[3], double skin) {
     int rc = ensure_device_model(h);
     if (rc != UMLMD_OK) return rc;
-    rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err);
+    { Scope sc(h, kNeighbor, 6); rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
     h->have_list = true;
     h->steps_since_build = 0;
@@ -235,6 +270,8 @@ int umlmd_destroy(umlmd_t* h) {
     void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
                     h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass};
     for (void* p : ptrs) dev_free(p);
+    for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
     if (h->h_out) cudaFreeHost(h->h_out);
     if (h->h_err) cudaFreeHost(h->h_err);
     delete h;
@@ -249,6 +286,7 @@ int umlmd_query(const umlmd_t* h, umlmd_info* out) {
     out->n_atoms = h->have_list ? h->nb.N : 0;
     out->n_edges = h->have_list ? h->nb.E : 0;
     out->device_bytes = dev_bytes_held();
+    out->kernel_launches = h->launches_total;
     return UMLMD_OK;
 }
 
@@ -347,7 +385,7 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
         h->have_force = true;
     }
     for (int s = 0; s < nsteps; ++s) {
-        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, true, h->st));
+        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, true, h->st)); }
         ++h->steps_since_build;
         if (rebuild_every > 0 && h->steps_since_build >= rebuild_every) {
             const double skin = h->nb.skin;
@@ -356,9 +394,9 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
             if ((rc = build_list(h, N, h->md_pos, h->type_o, L, pbc, skin)) != UMLMD_OK) return rc;
         }
         if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
-        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, false, h->st));
+        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, false, h->st)); }
     }
-    API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st));
+    { Scope sc(h, kIntegrate, 2); API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st)); }
     rc = fetch_results(h, 11);
     if (rc != UMLMD_OK) return rc;
     if (e_pot) *e_pot = h->h_out[0];
@@ -394,6 +432,35 @@ int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, doub
         }
     }
     return UMLMD_OK;
+}
+
+int umlmd_set_profiling(umlmd_t* h, int enabled) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    h->prof_on = enabled != 0;
+    return UMLMD_OK;
+}
+
+int umlmd_get_profile(umlmd_t* h, int32_t max_classes, double* ms, int64_t* launches, int32_t* n_classes) {
+    if (!h || !n_classes || max_classes < 0) return UMLMD_E_INVALID_ARG;
+    if (h->on_device) API_CUDA(h, cudaStreamSynchronize(h->st));
+    for (auto& sp : h->spans) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, sp.a, sp.b) == cudaSuccess) h->prof_ms[sp.cls] += t;
+        h->free_events.push_back(sp.a);
+        h->free_events.push_back(sp.b);
+    }
+    h->spans.clear();
+    *n_classes = kClassCount;
+    for (int k = 0; k < kClassCount && k < max_classes; ++k) {
+        if (ms) ms[k] = h->prof_ms[k];
+        if (launches) launches[k] = h->prof_launches[k];
+    }
+    for (int k = 0; k < kClassCount; ++k) { h->prof_ms[k] = 0; h->prof_launches[k] = 0; }
+    return UMLMD_OK;
+}
+
+const char* umlmd_profile_class_name(int32_t cls) {
+    return (cls >= 0 && cls < kClassCount) ? kClassNames[cls] : "";
 }
 
 int umlmd_eval_pair_cache(const umlmd_t* h, int32_t type_i, int32_t type_j, double* out) {

@@ -66,7 +66,8 @@ struct MlpArgs {
     int path;               // 1 = CUDA-core fp32, 2 = tcgen05
     bool want_grad;
 };
-cudaError_t launch_mlp(const MlpArgs& a, cudaStream_t st);
+cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)
+cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad
 
 // ---- assemble.cu ---------------------------------------------------------------------
 cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted,

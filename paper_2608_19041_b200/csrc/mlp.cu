@@ -94,7 +94,7 @@ static cudaError_t run_gemm(const GemmArgs& g, int path, cudaStream_t st) {
     return launch_gemm_simt(g, st);
 }
 
-cudaError_t launch_mlp(const MlpArgs& a, cudaStream_t st) {
+cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     const Dims& d = a.d;
     const int n = a.n, F = d.F, NH = d.n_hidden;
     if (n <= 0) return cudaSuccess;
@@ -122,8 +122,18 @@ cudaError_t launch_mlp(const MlpArgs& a, cudaStream_t st) {
                                              a.e_atom, a.want_grad);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    if (!a.want_grad) return cudaSuccess;
-    // ---- backward: dE/dY_t sits in pre[t]; dE/dh_t alternates between the two hbuf slots
+    return cudaSuccess;
+}
+
+// backward: dE/dY_t sits in pre[t]; dE/dh_t alternates between the two hbuf slots
+cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
+    const Dims& d = a.d;
+    const int n = a.n, F = d.F, NH = d.n_hidden;
+    if (n <= 0) return cudaSuccess;
+    const size_t layer = (size_t)n * F;
+    float* hb[2] = {a.hbuf, a.hbuf + layer};
+    const bool res0 = (d.D_out == F);
+    cudaError_t e;
     int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
     bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
     for (int t = NH - 1; t >= 1; --t) {
