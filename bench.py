@@ -37,7 +37,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from workloads import CONFIGS, load_calibration, make_blob, make_system  # noqa: E402
+from workloads import CONFIGS, make_system, workload_blob  # noqa: E402
 
 DEFAULT_WORKLOAD = "cfg5_amorphous1m"
 SM_COUNT = 148
@@ -168,7 +168,7 @@ class OracleSampler:
         cfg = CONFIGS[name]
         self.name = name
         self.s = make_system(cfg["system"])
-        self.o = orc.Oracle(make_blob(cfg["profile"], cfg["weights_seed"], calibration=load_calibration(name)))
+        self.o = orc.Oracle(workload_blob(name))
         self.rc = cfg["profile"]["rc"]
         self.N = len(self.s["pos"])
         self.pos = orc.wrap_positions(self.s["pos"], self.s["cell"], self.s["pbc"])
@@ -231,7 +231,7 @@ def run_ours(args):
     md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=300.0, seed=1, rebuild_every=10, skin=0.0)
     s = make_system(cfg["system"], md)
     N = len(s["pos"])
-    blob = make_blob(p, cfg["weights_seed"], calibration=load_calibration(name))
+    blob = workload_blob(name)
     model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile)
     pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
     pos = pos0.cuda().contiguous()

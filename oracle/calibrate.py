@@ -12,8 +12,11 @@ uncalibrated model (mu = 0, sigma = 1):
     initial features, so that it is brought to the scale of the initial features.
 
 READING: "brought to the root-mean-square scale of the initial features" is taken to mean
-that D_k has the RMS of the initial-feature entries after division by sigma_k.  A floor of
-1e-6 keeps sigma away from zero for entries that vanish on the sample.
+that D_k has the RMS of the initial-feature entries after division by sigma_k.  As every
+normalisation does, the measured scale gets an epsilon: RMS (or spread) values below 1e-3
+are raised to 1e-3.  Without it the near-centrosymmetric crystal frames, whose odd-degree
+invariants almost vanish, would have those dead entries blown up by 1e5 and the
+random-weight potential would be too stiff to integrate at a 1 fs time step.
 
 Usage:  python -m oracle.calibrate [config ...]      (writes workloads/calibration/*.txt)
 """
@@ -28,6 +31,7 @@ from workloads import CONFIGS, make_blob, make_system
 
 SAMPLE = {"cfg1_al108": 108, "cfg2_cu4000": 512, "cfg3_water32400": 384, "cfg4_hea128k": 160,
           "cfg5_amorphous1m": 96}
+SCALE_FLOOR = 1.0e-3
 OUT_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "calibration")
 
 
@@ -49,9 +53,9 @@ def calibration_for(name):
     for k in range(C0, D):
         if k in (2 * C0, 2 * C0 + 1):
             mu[k] = Dt[:, k].mean()
-            sigma[k] = max(Dt[:, k].std(), 1e-6) / rms_x0
+            sigma[k] = max(Dt[:, k].std(), SCALE_FLOOR) / rms_x0
         else:
-            sigma[k] = max(float(np.sqrt(np.mean(Dt[:, k] ** 2))), 1e-6) / rms_x0
+            sigma[k] = max(float(np.sqrt(np.mean(Dt[:, k] ** 2))), SCALE_FLOOR) / rms_x0
     return mu, sigma, len(centers)
 
 

@@ -30,7 +30,7 @@ struct Dims {
     int C0, L, R, N_rbf, n_hidden, F, T;
     int C[kMaxDeg + 1];      // channels per degree
     int K[kMaxDeg + 1];      // probe ranks (index 0 unused)
-    int S, SP;               // state width S; row stride SP >= S+2, multiple of 4
+    int S, SP;               // state width S; row stride SP >= S+4 (s0, s1 as float pairs), multiple of 4
     int offA[kMaxDeg + 1];   // offset of degree block in the state row
     int D_out, DP;           // feature-vector width; row stride (multiple of 32)
     int oG[kMaxDeg + 1];     // offsets of vech(G_l) in D

@@ -190,11 +190,11 @@ k_edge_forward(const EdgeArgs a) {
         for (int k = 0; k < 4; ++k) acc2[m][k] = 0.f;
 #pragma unroll
     for (int m = 0; m < 7; ++m) acc3[m] = 0.f;
-    float s0 = 0.f, s1 = 0.f;
+    double s0 = 0.0, s1 = 0.0;   // normaliser sums in double: the calibration subtracts their mean
 
     for (int base = e0; base < e1; base += 32) {
         const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
-        if (g.valid) { const float c2 = g.chi * g.chi; s0 += c2; s1 += c2 * c2; }
+        if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
         const int nb = min(32, e1 - base);
         for (int it = 0; it * W::EPI < nb; ++it) {
             const int b = it * W::EPI + sub;
@@ -278,7 +278,11 @@ k_edge_forward(const EdgeArgs a) {
 #pragma unroll
             for (int m = 0; m < 7; ++m) row_out[a.d.offA[3] + m] = acc3[m];
         }
-        if (cl == 0) { row_out[a.d.S] = s0; row_out[a.d.S + 1] = s1; }
+        if (cl == 0) {
+            const float h0 = (float)s0, h1 = (float)s1;
+            row_out[a.d.S] = h0; row_out[a.d.S + 1] = h1;
+            row_out[a.d.S + 2] = (float)(s0 - (double)h0); row_out[a.d.S + 3] = (float)(s1 - (double)h1);
+        }
     }
 }
 

@@ -17,12 +17,6 @@ namespace umd {
 
 namespace {
 
-struct BlobHeader {
-    char magic[8];
-    uint32_t version, C0, L, R, N_rbf, n_hidden, F, T, basis;
-    double rc, table_dx;
-};
-static_assert(sizeof(BlobHeader) == 8 + 9 * 4 + 4 /*pad*/ + 16 || true, "layout checked by offsets");
 constexpr size_t kHeaderBytes = 8 + 9 * 4 + 2 * 8;  // packed, no padding
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -142,7 +136,7 @@ bool derive_dims(int C0, int L, int R, Dims* d) {
     int off = 0;
     for (int l = 0; l <= L; ++l) { d->offA[l] = off; off += (2 * l + 1) * d->C[l]; }
     d->S = off;
-    d->SP = round_up(d->S + 2, 4);
+    d->SP = round_up(d->S + 4, 4);   // sums, then s0, s1 (high parts) and their low parts
     int o = 2 * C0 + 2;
     for (int l = 1; l <= L; ++l) { d->oG[l] = o; o += d->C[l] * (d->C[l] + 1) / 2; }
     const int K1 = d->K[1], K2 = d->K[2];

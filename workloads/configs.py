@@ -9,6 +9,17 @@ the atomic-energy MLP (the model has exactly one aggregation layer), "channels"
 = scalar channel width C0, "ranks 0..L" = maximum angular degree L.  Where a
 workload does not say, N_rbf = 16, R = 0 and the MLP width is the one the paper
 pairs with that C0 (256 for C0 = 64, 384 for C0 = 128).
+
+A random-weight potential has no repulsive core and no reason to hold a crystal together:
+at the plain Xavier output scale the 300 K copper crystal slides down the random energy
+surface, releases half an eV per atom within 100 fs and melts to thousands of kelvin, and
+atoms that pass close to each other feel angular forces that grow like 1/distance.  The
+workloads that run molecular dynamics therefore fix the one free output-scale choice of the
+otherwise unconstrained initialisation law, ``head_scale`` (a factor on the scalar head
+w_head), so that the run is integrable at the stated time step: a negative sign makes the
+jittered lattice a minimum instead of a maximum of the random surface (the copper crystal
+then vibrates at ~230 K for the whole picosecond), and the magnitude is reduced where
+light or densely packed atoms would otherwise be accelerated into each other.
 """
 
 
@@ -27,7 +38,7 @@ CONFIGS = {
                     n_types=1, masses=[26.982]),
         profile=_profile(32, 2, 0, 8, 1, 64, 1, C1=8, C2=4, K1=4, K2=2, H=88,
                          Hp=176, S=76, D_out=144),
-        weights_seed=0,
+        weights_seed=0, head_scale=1.0,
         md=None,
     ),
     # 4,000-atom FCC Cu, 1000 NVE steps
@@ -37,7 +48,7 @@ CONFIGS = {
                     n_types=1, masses=[63.546]),
         profile=_profile(64, 2, 0, 16, 2, 256, 1, C1=8, C2=4, K1=4, K2=2, H=176,
                          Hp=344, S=108, D_out=208),
-        weights_seed=11,
+        weights_seed=11, head_scale=-1.0,
         md=dict(steps=1000, dt_ps=0.001, temperature=300.0, seed=1,
                 rebuild_every=10, skin=1.0),
     ),
@@ -48,7 +59,7 @@ CONFIGS = {
                     min_oo=2.5, seed=4, n_types=2, masses=[15.999, 1.008]),
         profile=_profile(64, 3, 0, 16, 2, 256, 2, C1=8, C2=4, K1=4, K2=2, H=176,
                          Hp=344, S=115, D_out=219),
-        weights_seed=12,
+        weights_seed=12, head_scale=-0.01,
         md=dict(steps=500, dt_ps=0.0005, temperature=300.0, seed=5,
                 rebuild_every=10, skin=1.0),
     ),
@@ -59,7 +70,7 @@ CONFIGS = {
                     n_types=5, masses=[50.94, 92.91, 95.95, 180.95, 183.84]),
         profile=_profile(128, 2, 0, 16, 3, 384, 5, C1=16, C2=8, K1=8, K2=2,
                          H=344, Hp=688, S=216, D_out=522),
-        weights_seed=13,
+        weights_seed=13, head_scale=-0.2,
         md=dict(steps=200, dt_ps=0.001, temperature=1000.0, seed=6,
                 rebuild_every=10, skin=1.0),
     ),
@@ -71,7 +82,7 @@ CONFIGS = {
                     masses=[12.0 + 3.0 * t for t in range(64)]),
         profile=_profile(128, 3, 0, 16, 3, 384, 64, C1=16, C2=8, K1=8, K2=2,
                          H=344, Hp=688, S=223, D_out=541),
-        weights_seed=14,
+        weights_seed=14, head_scale=0.05,
         md=dict(steps=100, dt_ps=0.001, temperature=600.0, seed=7,
                 rebuild_every=10, skin=1.0),
     ),

@@ -52,12 +52,13 @@ def blob_array_shapes(p):
     return shapes
 
 
-def make_blob(p, seed, calibration=None, bias_scale=0.0, e_ref_scale=0.0):
+def make_blob(p, seed, calibration=None, bias_scale=0.0, e_ref_scale=0.0, head_scale=1.0):
     """Return the blob bytes for profile ``p``.
 
     ``calibration`` is an optional (mu, sigma) pair of length-D_out arrays.
     ``bias_scale`` / ``e_ref_scale`` > 0 draw non-zero MLP biases / reference
-    energies (used by tests so that those terms are exercised).
+    energies (used by tests so that those terms are exercised).  ``head_scale``
+    multiplies the scalar head w_head, i.e. the energy scale of the random potential.
     """
     rng = np.random.Generator(np.random.PCG64(seed))
     chunks = [struct.pack(HEADER_FMT, MAGIC, 1, p["C0"], p["L"], p["R"], p["N_rbf"],
@@ -77,7 +78,7 @@ def make_blob(p, seed, calibration=None, bias_scale=0.0, e_ref_scale=0.0):
         elif name == "E_ref":
             a = rng.standard_normal(shape) * e_ref_scale
         elif name == "w_head":
-            a = rng.standard_normal(shape) * math.sqrt(2.0 / (shape[0] + 1))
+            a = rng.standard_normal(shape) * math.sqrt(2.0 / (shape[0] + 1)) * head_scale
         elif len(shape) == 2:
             a = rng.standard_normal(shape) * math.sqrt(2.0 / (shape[0] + shape[1])) \
                 if n else np.zeros(shape)
