@@ -17,12 +17,13 @@ struct umlmd {
     std::string err;
     NeighborDev nb;
     int node_tile = 131072;
-    int mlp_path = 1;
+    int mlp_path = 2;   // tensor-core GEMM wherever it applies, CUDA-core GEMM otherwise
     bool have_list = false;
     bool on_device = false;
     std::vector<void*> model_allocs;
     // workspace
     float* state = nullptr; float* desc = nullptr; float* pre = nullptr; float* hbuf = nullptr;
+    float* tc_hi = nullptr; float* tc_lo = nullptr;   // TF32 split of the current GEMM's activations
     int64_t tile_cap = 0;
     float* g = nullptr; int64_t g_cap = 0;
     double* e_atom = nullptr; double* f_sorted = nullptr; int* type_o = nullptr; int64_t n_cap = 0;
@@ -110,6 +111,9 @@ int ensure_workspace(umlmd_t* h) {
         c = 0; API_CUDA(h, dev_ensure(&h->desc, &c, B * d.DP));
         c = 0; API_CUDA(h, dev_ensure(&h->pre, &c, B * d.F * d.n_hidden));
         c = 0; API_CUDA(h, dev_ensure(&h->hbuf, &c, B * d.F * 2));
+        const int64_t wmax = d.DP > d.F ? d.DP : d.F;
+        c = 0; API_CUDA(h, dev_ensure(&h->tc_hi, &c, B * wmax));
+        c = 0; API_CUDA(h, dev_ensure(&h->tc_lo, &c, B * wmax));
         h->tile_cap = B;
     }
     if (E > h->g_cap || !h->g) { API_CUDA(h, dev_ensure(&h->g, &h->g_cap, E * 3, 1.1)); h->g_cap /= 3; }
@@ -128,6 +132,7 @@ int ensure_workspace(umlmd_t* h) {
 
 int decode_device_errors(umlmd_t* h, int word) {
     if (word & kErrNonFinite) return fail(h, UMLMD_E_NONFINITE, "non-finite value in positions, energy or forces");
+    if (word & kErrPipelineTimeout) return fail(h, UMLMD_E_CUDA, "tensor-core GEMM pipeline wait expired");
     if (word & kErrShiftRange) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "periodic image index outside [-127, 127]");
     if (word & kErrStale)
         return fail(h, UMLMD_E_STALE_NEIGHBORS, "an atom moved more than skin/2 since the neighbor list was built");
@@ -157,6 +162,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         MlpArgs ma;
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
+        ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err;
         { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
@@ -196,7 +202,9 @@ int ensure_device_model(umlmd_t* h) {
     auto up = [&](const std::vector<float>& v, float** p) { if (e == cudaSuccess) e = upload(h, v, p); };
     up(m.table, &md.table); up(m.pairmod, &md.pairmod); up(m.X0, &md.X0); up(m.W1p, &md.W1p); up(m.W2p, &md.W2p);
     up(m.A1, &md.A1); up(m.A2, &md.A2); up(m.mu, &md.mu); up(m.inv_sigma, &md.inv_sigma);
-    for (int t = 0; t < h->d.n_hidden; ++t) { up(m.theta[t], &md.theta[t]); up(m.thetaT[t], &md.thetaT[t]); up(m.bias[t], &md.bias[t]); }
+    for (int t = 0; t < h->d.n_hidden; ++t) { up(m.theta[t], &md.theta[t]); up(m.thetaT[t], &md.thetaT[t]); up(m.bias[t], &md.bias[t]);
+        up(m.theta_hi[t], &md.theta_hi[t]); up(m.theta_lo[t], &md.theta_lo[t]);
+        up(m.thetaT_hi[t], &md.thetaT_hi[t]); up(m.thetaT_lo[t], &md.thetaT_lo[t]); }
     up(m.w_head, &md.w_head); up(m.e_ref, &md.e_ref);
     md.b_head = m.b_head;
     if (e == cudaSuccess && h->d.L >= 3) {
@@ -267,7 +275,7 @@ int umlmd_destroy(umlmd_t* h) {
     if (h->on_device) cudaStreamSynchronize(h->st);
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
-    void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
+    void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
                     h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }

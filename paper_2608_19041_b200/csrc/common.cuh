@@ -21,7 +21,7 @@ constexpr double kAccelUnit = 9648.53321;   // (eV/Angstrom/amu) in Angstrom/ps^
 constexpr double kBoltzmann = 8.617333262e-5;
 
 // error word bits set by kernels (read back at synchronisation points)
-enum : int { kErrStale = 1, kErrNonFinite = 2, kErrEdgeOverflow = 4, kErrShiftRange = 8 };
+enum : int { kErrStale = 1, kErrNonFinite = 2, kErrEdgeOverflow = 4, kErrShiftRange = 8, kErrPipelineTimeout = 16 };
 
 // Widths derived from (C0, L, R): degree-wise channels, probe ranks, feature-state width
 // S, feature-vector width D_out, gated hidden widths, and the flat offsets used by the
@@ -60,6 +60,8 @@ struct ModelDev {
     float* inv_sigma; // [D_out]
     float* theta[8];  // Theta_t, row-major [K_in (padded)][F]; theta[0] has DP rows
     float* thetaT[8]; // transposes, [F][K_in (padded)]
+    float* theta_hi[8];  float* theta_lo[8];    // TF32 split of theta  (x = hi + lo)
+    float* thetaT_hi[8]; float* thetaT_lo[8];   // TF32 split of thetaT
     float* bias[8];   // b_t [F]
     float* w_head;    // [F]
     float* e_ref;     // [T]

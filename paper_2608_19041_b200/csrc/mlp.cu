@@ -110,6 +110,8 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         if (t == 0) { g.A = a.desc; g.lda = d.DP; g.K = d.DP; g.res = res0 ? a.desc : nullptr; g.ldres = d.DP; }
         else { g.A = hb[(t - 1) & 1]; g.lda = F; g.K = F; g.res = hb[(t - 1) & 1]; g.ldres = F; }
         g.B = a.m.theta[t]; g.ldb = F;
+        g.Bt_hi = a.m.thetaT_hi[t]; g.Bt_lo = a.m.thetaT_lo[t]; g.ldbt = t == 0 ? d.DP : F;
+        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
         g.bias = a.m.bias[t];
         g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
         g.out = hb[t & 1]; g.ldout = F;
@@ -142,6 +144,8 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.M = n; g.N = F; g.K = F;
         g.A = a.pre + (size_t)t * layer; g.lda = F;
         g.B = a.m.thetaT[t]; g.ldb = F;
+        g.Bt_hi = a.m.theta_hi[t]; g.Bt_lo = a.m.theta_lo[t]; g.ldbt = F;
+        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
         if (vec_grad) g.rvec = a.m.w_head; else { g.res = hb[slot]; g.ldres = F; }
         const int out_slot = vec_grad ? 0 : 1 - slot;
         const bool need_dh = (t - 1 >= 1) || res0;
@@ -156,6 +160,8 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.M = n; g.N = d.DP; g.K = F;
         g.A = a.pre; g.lda = F;
         g.B = a.m.thetaT[0]; g.ldb = d.DP;
+        g.Bt_hi = a.m.theta_hi[0]; g.Bt_lo = a.m.theta_lo[0]; g.ldbt = F;
+        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
         if (res0) {
             if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }

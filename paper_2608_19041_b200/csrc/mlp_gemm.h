@@ -23,6 +23,8 @@ struct GemmArgs {
     float* out; int ldout;
     // tensor-core path only: pre-split copies of B (hi / lo TF32 parts), K-major [N][K]
     const float* Bt_hi; const float* Bt_lo; int ldbt;
+    float* A_hi; float* A_lo;     // scratch [M][K] for the split of A
+    int* err;                     // device error word (bounded-wait expiry)
 };
 
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.0f / (1.0f + expf(-x)); }

@@ -1,9 +1,275 @@
-// Tensor-core GEMM for the MLP layers (tcgen05 / TMEM / TMA, 3xTF32 split).
+// Tensor-core GEMM for the MLP layers on sm_100a: TMA loads into 128-byte-swizzled shared
+// memory, tcgen05.mma (kind::tf32) issued by one thread, fp32 accumulator in tensor memory,
+// tcgen05.ld epilogue with the fused bias / SiLU / residual (or SiLU-derivative) step.
+//
+// Precision: a single TF32 product carries 11 significant bits, far short of the 1e-5
+// parity target, so every operand is split into two TF32 numbers, x = hi + lo with
+// hi = round_tf32(x) and lo = round_tf32(x - hi), and each K step issues three MMAs,
+// A_lo B_hi + A_hi B_lo + A_hi B_hi (the lo*lo term, ~2^-22, is dropped).  Both parts are
+// exactly representable in TF32, so the result does not depend on how the tensor core
+// treats the low mantissa bits.  Weights are split once on the host; activations are split
+// by a small kernel in front of each GEMM.
+//
+// Tiling: one CTA computes a 128 x 128 output tile; K advances in blocks of 32 floats (one
+// 128-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (64 KB
+// per stage).  Warp 0 is the TMA producer, warp 1 issues the MMAs and owns the tensor-memory
+// allocation, warps 2-5 run the epilogue (one 32-lane quarter of tensor memory each).
+// Every mbarrier wait is bounded: on expiry the kernel flags an error word and carries on,
+// so a wedged pipeline ends with a wrong result and an error code instead of a hang, and
+// tensor memory is always released.
+#include <cuda.h>
+
+#include <cstdint>
+
+#include "common.cuh"
 #include "mlp_gemm.h"
 
 namespace umd {
 
-bool gemm_tc_supported(const GemmArgs&) { return false; }
-cudaError_t launch_gemm_tc(const GemmArgs&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 32, STAGES = 3;
+constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 16 KB, also BN * BK * 4
+constexpr uint32_t STAGE_BYTES = 4 * TILE_BYTES;      // A_hi, A_lo, B_hi, B_lo
+constexpr uint32_t BAR_BYTES = 128;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + BAR_BYTES;
+constexpr uint32_t TMEM_COLS = 128;
+constexpr int kSpinLimit = 4000000;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bounded wait: flags the error word and returns after kSpinLimit polls
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* err) {
+    for (int i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, parity)) return;
+        if (i > 64) __nanosleep(32);
+    }
+    if (err) atomicOr(err, kErrPipelineTimeout);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, 8-row
+// groups 1024 B apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// instruction descriptor: D = F32, A = B = TF32, both K-major, N = 128, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__global__ void __launch_bounds__(192, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUtensorMap mAl,
+          const __grid_constant__ CUtensorMap mBh, const __grid_constant__ CUtensorMap mBl, const GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t bars = tiles + STAGES * STAGE_BYTES;       // full[s], empty[s], accum, then the tmem slot
+    const uint32_t accum_bar = bars + 8 * (2 * STAGES);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars - raw) + 8 * (2 * STAGES + 1));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int KB = (g.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(bars + 8 * s, 1); mbar_init(bars + 8 * (STAGES + s), 1); }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {                                   // TMA producer
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % STAGES, u = kb / STAGES;
+                if (u > 0) mbar_wait(bars + 8 * (STAGES + s), (u - 1) & 1, g.err);
+                const uint32_t full = bars + 8 * s, sa = tiles + s * STAGE_BYTES;
+                mbar_expect_tx(full, STAGE_BYTES);
+                tma_load_2d(sa, &mAh, kb * BK, m0, full);
+                tma_load_2d(sa + TILE_BYTES, &mAl, kb * BK, m0, full);
+                tma_load_2d(sa + 2 * TILE_BYTES, &mBh, kb * BK, n0, full);
+                tma_load_2d(sa + 3 * TILE_BYTES, &mBl, kb * BK, n0, full);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {                                   // MMA issuer
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % STAGES, u = kb / STAGES;
+                mbar_wait(bars + 8 * s, u & 1, g.err);
+                tc_fence_after();
+                const uint32_t sa = tiles + s * STAGE_BYTES;
+#pragma unroll
+                for (int k = 0; k < BK / 8; ++k) {
+                    const uint64_t ah = umma_desc(sa + k * 32), al = umma_desc(sa + TILE_BYTES + k * 32);
+                    const uint64_t bh = umma_desc(sa + 2 * TILE_BYTES + k * 32), bl = umma_desc(sa + 3 * TILE_BYTES + k * 32);
+                    umma_tf32(tmem, al, bh, kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_tf32(tmem, ah, bl, kIdesc, 1u);
+                    umma_tf32(tmem, ah, bh, kIdesc, 1u);
+                }
+                umma_commit(bars + 8 * (STAGES + s));      // frees the stage when these MMAs retire
+            }
+            umma_commit(accum_bar);
+        }
+    } else {                                               // epilogue: warps 2..5 -> lane quarters 2,3,0,1
+        const int q = warp & 3;
+        mbar_wait(accum_bar, 0, g.err);
+        tc_fence_after();
+        const int m = m0 + q * 32 + lane;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            float v[32];
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+            if (m < g.M) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int n = n0 + c0 + 4 * j;
+                    if (n < g.N) gemm_epilogue4(g, m, n, v + 4 * j);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// hi = round-to-nearest TF32 of x, lo = round-to-nearest TF32 of (x - hi); rows [M][K]
+__global__ void k_split_tf32(const float* __restrict__ A, int lda, int M, int K, float* __restrict__ hi,
+                             float* __restrict__ lo) {
+    const int k4 = K >> 2;
+    const size_t total = (size_t)M * k4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / k4), k = (int)(i - (size_t)m * k4) * 4;
+        const float4 x = *reinterpret_cast<const float4*>(A + (size_t)m * lda + k);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+        float h[4], l[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t hb, lb;
+            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hb) : "f"(xs[j]));
+            h[j] = __uint_as_float(hb);
+            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lb) : "f"(xs[j] - h[j]));
+            l[j] = __uint_as_float(lb);
+        }
+        *reinterpret_cast<float4*>(hi + (size_t)m * K + k) = make_float4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<float4*>(lo + (size_t)m * K + k) = make_float4(l[0], l[1], l[2], l[3]);
+    }
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// 2-D map over a row-major [rows][cols] float matrix with row pitch ld; box = 32 cols x 128 rows
+bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    const cuuint32_t box[2] = {BK, BM};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const GemmArgs& g) {
+    return g.A_hi && g.A_lo && g.Bt_hi && g.Bt_lo && g.M > 0 && g.N >= 4 && g.K >= 4 && (g.K & 3) == 0 &&
+           (g.N & 3) == 0 && (g.lda & 3) == 0 && (g.ldbt & 3) == 0 && encode_fn() != nullptr;
+}
+
+cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    {
+        const size_t total = (size_t)g.M * (g.K >> 2);
+        int blocks = (int)((total + 255) / 256);
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        k_split_tf32<<<blocks, 256, 0, st>>>(g.A, g.lda, g.M, g.K, g.A_hi, g.A_lo);
+    }
+    CUtensorMap mAh, mAl, mBh, mBl;
+    if (!make_map(&mAh, g.A_hi, g.M, g.K, g.K) || !make_map(&mAl, g.A_lo, g.M, g.K, g.K) ||
+        !make_map(&mBh, g.Bt_hi, g.N, g.K, g.ldbt) || !make_map(&mBl, g.Bt_lo, g.N, g.K, g.ldbt))
+        return cudaErrorInvalidValue;
+    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
+    k_gemm_tc<<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    return cudaGetLastError();
+}
 
 }  // namespace umd

@@ -358,6 +358,26 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
             }
         m->bias[t] = to_f(b);
     }
+    // TF32 splits for the tensor-core GEMM: hi = round-to-nearest-even to 10 mantissa bits,
+    // lo = the same rounding of (x - hi); both are exactly representable in TF32
+    auto tf32 = [](float x) {
+        uint32_t u;
+        std::memcpy(&u, &x, 4);
+        u += 0x00000FFFu + ((u >> 13) & 1u);
+        u &= 0xFFFFE000u;
+        float y;
+        std::memcpy(&y, &u, 4);
+        return y;
+    };
+    auto split = [&](const std::vector<float>& w, std::vector<float>* hi, std::vector<float>* lo) {
+        hi->resize(w.size()); lo->resize(w.size());
+        for (size_t i = 0; i < w.size(); ++i) { (*hi)[i] = tf32(w[i]); (*lo)[i] = tf32(w[i] - (*hi)[i]); }
+    };
+    m->theta_hi.resize(NH); m->theta_lo.resize(NH); m->thetaT_hi.resize(NH); m->thetaT_lo.resize(NH);
+    for (int t = 0; t < NH; ++t) {
+        split(m->theta[t], &m->theta_hi[t], &m->theta_lo[t]);
+        split(m->thetaT[t], &m->thetaT_hi[t], &m->thetaT_lo[t]);
+    }
     const size_t tail = 13 + 2 * NH;
     m->w_head = to_f(arr[tail]);
     m->b_head = (float)arr[tail + 1][0];

@@ -17,6 +17,7 @@ struct HostModel {
     std::vector<float> pairmod;    // [T*T][2+R][C0]
     std::vector<float> X0, W1p, W2p, A1, A2, mu, inv_sigma;
     std::vector<std::vector<float>> theta, thetaT, bias;   // per hidden layer
+    std::vector<std::vector<float>> theta_hi, theta_lo, thetaT_hi, thetaT_lo;   // TF32 splits
     std::vector<float> w_head, e_ref;
     float b_head = 0;
     GauntSparse g123, g233;

@@ -216,3 +216,30 @@ def test_stale_list_is_reported():
         m.compute(moved)
     assert e.value.code == -6
     m.compute(pos)                         # the handle stays usable
+
+
+@pytest.mark.parametrize("name", ["p16_3_2", "p32_2_4", "p32_2_0_res"])
+def test_tensor_core_mlp_path_small_profiles(name):
+    # ragged everything: fewer rows than a tile, widths that are not multiples of the tile
+    p = SMALL_PROFILES[name]
+    blob = make_blob(p, seed=45, bias_scale=0.2, e_ref_scale=0.5)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"], atoms=150, edges=(12.5, 13.5, 14.0)))
+    _compare(blob, s, check_intermediates=False, mlp_path=2)
+
+
+def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
+    name = "cfg2_cu4000"
+    s = make_system(CONFIGS[name]["system"])
+    blob = workload_blob(name)
+    outs = []
+    for path in (1, 2):
+        m, pos = _build(blob, s, mlp_path=path, node_tile=1536)    # three tiles, ragged last one
+        outs.append(m.compute(pos, atom_energy=True))
+        m.close()
+    a, b = outs
+    e_scale = a["atom_energy"].abs().max().item()
+    f_scale = a["forces"].abs().max().item()
+    # the tensor core truncates when it aligns partial sums, a ~2e-6 relative one-sided bias
+    assert (a["atom_energy"] - b["atom_energy"]).abs().max().item() <= 5e-6 * e_scale
+    assert (a["forces"] - b["forces"]).abs().max().item() <= 1e-5 * f_scale
+    assert np.abs(a["virial"] - b["virial"]).max() <= 1e-5 * np.abs(a["virial"]).max()
