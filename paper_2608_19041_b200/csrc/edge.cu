@@ -156,40 +156,57 @@ __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, 
     }
 }
 
-template <int C0> struct Widths {
+template <int C0, int L> struct Widths {
     static constexpr int C1 = C0 <= 16 ? 4 : (C0 <= 64 ? 8 : 16);
     static constexpr int C2 = C1 / 2 > 4 ? C1 / 2 : 4;
-    static constexpr int LPE = C0 / 4;          // lanes per edge
+    static constexpr int LPE = C0 / 4;          // lanes per edge in the channel-parallel phase
     static constexpr int EPI = 32 / LPE;        // edges per replay step
     static constexpr int NL1 = C1 / 4;          // lanes of a group that hold degree-1 channels
-    static constexpr int NL2 = C2 / 4;
+    static constexpr int NHI = 3 * C1 + 5 * C2 + (L >= 3 ? 7 : 0);   // sums of degree >= 1
+    static constexpr int NCH = (NHI + 31) / 32;
+    // row pitch (floats) of the per-edge amplitude staging; pitch/4 odd keeps 16-byte
+    // accesses of 8 consecutive lanes on distinct bank groups
+    static constexpr int PF = ((C1 / 4 + 1) & 1) ? C1 + 4 : C1 + 8;          // forward: psi
+    static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
+};
+
+template <int C0, int L> struct BwdSmem {          // dynamic shared memory of the backward kernel
+    using W = Widths<C0, L>;
+    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LPE + 1) + W::NHI + 3) / 4 * 4;   // floats
+    static constexpr size_t bytes = kWarpsPerBlock * 9 * sizeof(double) + sizeof(float) * kWarpsPerBlock * per_warp;
 };
 
 // ------------------------------------------------------------------------------- forward
+//
+// Per batch of 32 edges:
+//   1. lane = edge: geometry.
+//   2. lanes = channels (a group of C0/4 lanes per edge): amplitude psi of all C0 channels,
+//      degree-0 sums accumulated in registers; the leading C1 amplitudes of each edge are
+//      parked in shared memory.
+//   3. lane = edge again: harmonics and the chi^2 psi_c B_lm products of degree >= 1 for the
+//      lane's own edge, summed over the batch by a shared-memory transpose (32 values at a
+//      time), so that lane v ends up owning sums v, v+32, v+64 of the flattened block.
 template <int C0, int L, bool HASR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_forward(const EdgeArgs a) {
-    using W = Widths<C0>;
-    const int lane = threadIdx.x & 31;
-    const int i = a.a0 + blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    using W = Widths<C0, L>;
+    // one 32 x 33 float scratch per warp: first the parked amplitudes (row pitch PF), then,
+    // once every lane has read its own row, the transpose buffer
+    __shared__ __align__(16) float scratch[kWarpsPerBlock][32 * 33];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     if (i >= a.a1) return;
+    float* const psi_s = scratch[wid];      // [32][PF]
+    float* const tr = scratch[wid];         // [32][33]
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
     const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
     const int ti = a.type_s[i];
     const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
 
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
-    float acc1[3][4], acc2[5][4], acc3[7];
+    float accH[W::NCH];
 #pragma unroll
-    for (int m = 0; m < 3; ++m)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc1[m][k] = 0.f;
-#pragma unroll
-    for (int m = 0; m < 5; ++m)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc2[m][k] = 0.f;
-#pragma unroll
-    for (int m = 0; m < 7; ++m) acc3[m] = 0.f;
+    for (int j = 0; j < W::NCH; ++j) accH[j] = 0.f;
     double s0 = 0.0, s1 = 0.0;   // normaliser sums in double: the calibration subtracts their mean
 
     for (int base = e0; base < e1; base += 32) {
@@ -203,37 +220,66 @@ k_edge_forward(const EdgeArgs a) {
             const int pair = __shfl_sync(kFull, g.pair, b);
             const float t = __shfl_sync(kFull, g.t, b);
             const float chi = __shfl_sync(kFull, g.chi, b);
-            const float ux = __shfl_sync(kFull, g.ux, b);
-            const float uy = __shfl_sync(kFull, g.uy, b);
-            const float uz = __shfl_sync(kFull, g.uz, b);
             if (!v) continue;
             float psi[4];
             amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr);
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc0[k] += chi * psi[k];
-            if (cl < W::NL1) {
-                float B1[3], B2[5], B3[7];
-                harmonics_s1<L>(ux, uy, uz, B1, B2, B3);
-                const float w = chi * chi;
+            if (cl < W::NL1)
+                *reinterpret_cast<float4*>(psi_s + b * W::PF + c) = make_float4(psi[0], psi[1], psi[2], psi[3]);
+        }
+        __syncwarp();
+        // lane = edge: products of degree >= 1, then batch sums by transposition
+        float ps[W::C1];
+        float B1[3], B2[5], B3[7];
+        float w = 0.f;
+        if (g.valid) {
 #pragma unroll
-                for (int m = 0; m < 3; ++m) {
-                    const float wb = w * B1[m];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) acc1[m][k] += wb * psi[k];
-                }
-                if (cl < W::NL2) {
-#pragma unroll
-                    for (int m = 0; m < 5; ++m) {
-                        const float wb = w * B2[m];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) acc2[m][k] += wb * psi[k];
-                    }
-                }
-                if (L >= 3 && cl == 0) {
-#pragma unroll
-                    for (int m = 0; m < 7; ++m) acc3[m] += w * B3[m] * psi[0];
-                }
+            for (int q = 0; q < W::C1 / 4; ++q) {
+                const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PF + 4 * q);
+                ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
             }
+            harmonics_s1<L>(g.ux, g.uy, g.uz, B1, B2, B3);
+            w = g.chi * g.chi;
+        } else {
+#pragma unroll
+            for (int q = 0; q < W::C1; ++q) ps[q] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 3; ++q) B1[q] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 5; ++q) B2[q] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 7; ++q) B3[q] = 0.f;
+        }
+        __syncwarp();                           // amplitudes are in registers: reuse the scratch
+        int vv = 0;
+        auto emit = [&](float val) {
+            tr[(vv & 31) * 33 + lane] = val;
+            ++vv;
+            if ((vv & 31) == 0 || vv == W::NHI) {
+                __syncwarp();
+                float s = 0.f;
+#pragma unroll
+                for (int l = 0; l < 32; ++l) s += tr[lane * 33 + l];
+                accH[(vv - 1) >> 5] += s;
+                __syncwarp();
+            }
+        };
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const float wb = w * B1[m];
+#pragma unroll
+            for (int k = 0; k < W::C1; ++k) emit(wb * ps[k]);
+        }
+#pragma unroll
+        for (int m = 0; m < 5; ++m) {
+            const float wb = w * B2[m];
+#pragma unroll
+            for (int k = 0; k < W::C2; ++k) emit(wb * ps[k]);
+        }
+        if (L >= 3) {
+#pragma unroll
+            for (int m = 0; m < 7; ++m) emit(w * B3[m] * ps[0]);
         }
     }
     // combine the edge slots of the warp (lanes with equal channel offset)
@@ -241,18 +287,6 @@ k_edge_forward(const EdgeArgs a) {
     for (int off = W::LPE; off < 32; off <<= 1) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) acc0[k] += __shfl_xor_sync(kFull, acc0[k], off);
-#pragma unroll
-        for (int m = 0; m < 3; ++m)
-#pragma unroll
-            for (int k = 0; k < 4; ++k) acc1[m][k] += __shfl_xor_sync(kFull, acc1[m][k], off);
-#pragma unroll
-        for (int m = 0; m < 5; ++m)
-#pragma unroll
-            for (int k = 0; k < 4; ++k) acc2[m][k] += __shfl_xor_sync(kFull, acc2[m][k], off);
-        if (L >= 3) {
-#pragma unroll
-            for (int m = 0; m < 7; ++m) acc3[m] += __shfl_xor_sync(kFull, acc3[m], off);
-        }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -260,40 +294,37 @@ k_edge_forward(const EdgeArgs a) {
         s1 += __shfl_xor_sync(kFull, s1, off);
     }
     float* row_out = a.state + (size_t)(i - a.a0) * a.d.SP;
-    if (sub == 0) {
-        *reinterpret_cast<float4*>(row_out + c) = make_float4(acc0[0], acc0[1], acc0[2], acc0[3]);
-        if (cl < W::NL1) {
+    if (sub == 0) *reinterpret_cast<float4*>(row_out + c) = make_float4(acc0[0], acc0[1], acc0[2], acc0[3]);
 #pragma unroll
-            for (int m = 0; m < 3; ++m)
-                *reinterpret_cast<float4*>(row_out + a.d.offA[1] + m * W::C1 + c) =
-                    make_float4(acc1[m][0], acc1[m][1], acc1[m][2], acc1[m][3]);
-        }
-        if (cl < W::NL2) {
-#pragma unroll
-            for (int m = 0; m < 5; ++m)
-                *reinterpret_cast<float4*>(row_out + a.d.offA[2] + m * W::C2 + c) =
-                    make_float4(acc2[m][0], acc2[m][1], acc2[m][2], acc2[m][3]);
-        }
-        if (L >= 3 && cl == 0) {
-#pragma unroll
-            for (int m = 0; m < 7; ++m) row_out[a.d.offA[3] + m] = acc3[m];
-        }
-        if (cl == 0) {
-            const float h0 = (float)s0, h1 = (float)s1;
-            row_out[a.d.S] = h0; row_out[a.d.S + 1] = h1;
-            row_out[a.d.S + 2] = (float)(s0 - (double)h0); row_out[a.d.S + 3] = (float)(s1 - (double)h1);
-        }
+    for (int j = 0; j < W::NCH; ++j) {
+        const int v = lane + 32 * j;
+        if (v < W::NHI) row_out[a.d.offA[1] + v] = accH[j];
+    }
+    if (lane == 0) {
+        const float h0 = (float)s0, h1 = (float)s1;
+        row_out[a.d.S] = h0; row_out[a.d.S + 1] = h1;
+        row_out[a.d.S + 2] = (float)(s0 - (double)h0); row_out[a.d.S + 3] = (float)(s1 - (double)h1);
     }
 }
 
 // ------------------------------------------------------------------------------ backward
+//
+// Same three phases.  The channel-parallel phase produces, per edge, the two degree-0 dot
+// products sum_c G0_c psi_c and sum_c G0_c dpsi_c (partial sums parked in shared memory and
+// finished by the edge's own lane) and parks psi, dpsi of the leading C1 channels; the
+// edge's lane then does the whole degree >= 1 contraction by itself against the
+// destination's gradient block held in shared memory, and assembles dE/dr_ij.
 template <int C0, int L, bool HASR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_backward(const EdgeArgs a) {
-    using W = Widths<C0>;
-    __shared__ float red[kWarpsPerBlock][32][5];
-    __shared__ double vsum[kWarpsPerBlock][9];
+    using W = Widths<C0, L>;
+    extern __shared__ __align__(16) unsigned char dsm[];
+    double (*vsum)[9] = reinterpret_cast<double (*)[9]>(dsm);
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    float* const wbase = reinterpret_cast<float*>(dsm + kWarpsPerBlock * 9 * sizeof(double)) + wid * BwdSmem<C0, L>::per_warp;
+    float* const psi_s = wbase;                                  // [32][PB]: psi, dpsi of the leading channels
+    float* const red = psi_s + 32 * W::PB;                       // [2][32][LPE+1] partial dot products
+    float* const hi_s = red + 2 * 32 * (W::LPE + 1);             // [NHI] gradient of the degree >= 1 sums
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     const bool active = i < a.a1;
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
@@ -306,27 +337,17 @@ k_edge_backward(const EdgeArgs a) {
         const int ti = a.type_s[i];
         const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
-        // dE/d(sums) of this lane's channels
-        float h0[4], h1[3][4], h2[5][4], h3[7];
+        float h0[4];
         {
             const float4 v = *reinterpret_cast<const float4*>(grow + c);
             h0[0] = v.x; h0[1] = v.y; h0[2] = v.z; h0[3] = v.w;
         }
-#pragma unroll
-        for (int m = 0; m < 3; ++m) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (cl < W::NL1) v = *reinterpret_cast<const float4*>(grow + a.d.offA[1] + m * W::C1 + c);
-            h1[m][0] = v.x; h1[m][1] = v.y; h1[m][2] = v.z; h1[m][3] = v.w;
-        }
-#pragma unroll
-        for (int m = 0; m < 5; ++m) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (cl < W::NL2) v = *reinterpret_cast<const float4*>(grow + a.d.offA[2] + m * W::C2 + c);
-            h2[m][0] = v.x; h2[m][1] = v.y; h2[m][2] = v.z; h2[m][3] = v.w;
-        }
-#pragma unroll
-        for (int m = 0; m < 7; ++m) h3[m] = (L >= 3 && cl == 0) ? grow[a.d.offA[3] + m] : 0.f;
+        for (int v = lane; v < W::NHI; v += 32) hi_s[v] = grow[a.d.offA[1] + v];
         const float ds0 = grow[a.d.S], ds1 = grow[a.d.S + 1];
+        __syncwarp();
+        const float* H1 = hi_s;
+        const float* H2 = H1 + 3 * W::C1;
+        const float* H3 = H2 + 5 * W::C2;
 
         for (int base = e0; base < e1; base += 32) {
             const int e = base + lane;
@@ -338,75 +359,70 @@ k_edge_backward(const EdgeArgs a) {
                 const int row = __shfl_sync(kFull, g.row, b);
                 const int pair = __shfl_sync(kFull, g.pair, b);
                 const float t = __shfl_sync(kFull, g.t, b);
-                const float chi = __shfl_sync(kFull, g.chi, b);
-                const float ux = __shfl_sync(kFull, g.ux, b);
-                const float uy = __shfl_sync(kFull, g.uy, b);
-                const float uz = __shfl_sync(kFull, g.uz, b);
-                float p_rho = 0.f, p_chi = 0.f, pux = 0.f, puy = 0.f, puz = 0.f;
+                float pa = 0.f, pb = 0.f;
                 if (v) {
                     float psi[4], dpsi[4];
                     amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi);
-                    float ec[4];   // dE/dpsi_c
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) { ec[k] = chi * h0[k]; p_chi += psi[k] * h0[k]; }
+                    for (int k = 0; k < 4; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
                     if (cl < W::NL1) {
-                        float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
-                        harmonics_s1<L>(ux, uy, uz, B1, B2, B3);
-                        const float w = chi * chi;
-                        float bt = 0.f;   // sum_lm B_lm t_lm
-#pragma unroll
-                        for (int m = 0; m < 3; ++m) {
-                            float tm = 0.f;
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) { tm += psi[k] * h1[m][k]; ec[k] += w * B1[m] * h1[m][k]; }
-                            t1[m] = tm; bt += B1[m] * tm;
-                        }
-#pragma unroll
-                        for (int m = 0; m < 5; ++m) {
-                            float tm = 0.f;
-                            if (cl < W::NL2) {
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) { tm += psi[k] * h2[m][k]; ec[k] += w * B2[m] * h2[m][k]; }
-                            }
-                            t2[m] = tm; bt += B2[m] * tm;
-                        }
-#pragma unroll
-                        for (int m = 0; m < 7; ++m) {
-                            float tm = 0.f;
-                            if (L >= 3 && cl == 0) { tm = psi[0] * h3[m]; ec[0] += w * B3[m] * h3[m]; }
-                            t3[m] = tm;
-                            if (L >= 3) bt += B3[m] * tm;
-                        }
-                        p_chi += 2.0f * chi * bt;
-                        float gx, gy, gz;
-                        harmonics_grad_contract<L>(ux, uy, uz, t1, t2, t3, &gx, &gy, &gz);
-                        pux = w * gx; puy = w * gy; puz = w * gz;
+                        *reinterpret_cast<float4*>(psi_s + b * W::PB + c) = make_float4(psi[0], psi[1], psi[2], psi[3]);
+                        *reinterpret_cast<float4*>(psi_s + b * W::PB + W::C1 + c) = make_float4(dpsi[0], dpsi[1], dpsi[2], dpsi[3]);
                     }
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) p_rho += ec[k] * dpsi[k];
                 }
-                // sum over the lanes of the group
-#pragma unroll
-                for (int off = 1; off < W::LPE; off <<= 1) {
-                    p_rho += __shfl_xor_sync(kFull, p_rho, off);
-                    p_chi += __shfl_xor_sync(kFull, p_chi, off);
-                    pux += __shfl_xor_sync(kFull, pux, off);
-                    puy += __shfl_xor_sync(kFull, puy, off);
-                    puz += __shfl_xor_sync(kFull, puz, off);
-                }
-                if (cl == 0 && b < 32) {
-                    red[wid][b][0] = p_rho; red[wid][b][1] = p_chi;
-                    red[wid][b][2] = pux; red[wid][b][3] = puy; red[wid][b][4] = puz;
-                }
+                red[b * (W::LPE + 1) + cl] = pa;
+                red[(32 + b) * (W::LPE + 1) + cl] = pb;
             }
             __syncwarp();
             if (e < e1) {
                 float gx = 0.f, gy = 0.f, gz = 0.f;
                 if (g.valid) {
-                    const float p_rho = red[wid][lane][0], p_chi = red[wid][lane][1];
-                    const float pux = red[wid][lane][2], puy = red[wid][lane][3], puz = red[wid][lane][4];
-                    const float c2 = g.chi * g.chi;
-                    const float dEdrho = p_rho + (p_chi + 2.0f * g.chi * ds0 + 4.0f * c2 * g.chi * ds1) * g.dchi;
+                    float sa = 0.f, sb = 0.f;
+#pragma unroll
+                    for (int j = 0; j < W::LPE; ++j) { sa += red[lane * (W::LPE + 1) + j]; sb += red[(32 + lane) * (W::LPE + 1) + j]; }
+                    float ps[W::C1], dps[W::C1], ec[W::C1];
+#pragma unroll
+                    for (int q = 0; q < W::C1 / 4; ++q) {
+                        const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + 4 * q);
+                        const float4 d4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + W::C1 + 4 * q);
+                        ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
+                        dps[4 * q] = d4.x; dps[4 * q + 1] = d4.y; dps[4 * q + 2] = d4.z; dps[4 * q + 3] = d4.w;
+                    }
+#pragma unroll
+                    for (int k = 0; k < W::C1; ++k) ec[k] = 0.f;
+                    float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
+                    harmonics_s1<L>(g.ux, g.uy, g.uz, B1, B2, B3);
+                    float bt = 0.f;    // sum_lm B_lm t_lm,  t_lm = sum_c psi_c G_lmc
+#pragma unroll
+                    for (int m = 0; m < 3; ++m) {
+                        float tm = 0.f;
+#pragma unroll
+                        for (int k = 0; k < W::C1; ++k) { const float hv = H1[m * W::C1 + k]; tm += ps[k] * hv; ec[k] += B1[m] * hv; }
+                        t1[m] = tm; bt += B1[m] * tm;
+                    }
+#pragma unroll
+                    for (int m = 0; m < 5; ++m) {
+                        float tm = 0.f;
+#pragma unroll
+                        for (int k = 0; k < W::C2; ++k) { const float hv = H2[m * W::C2 + k]; tm += ps[k] * hv; ec[k] += B2[m] * hv; }
+                        t2[m] = tm; bt += B2[m] * tm;
+                    }
+#pragma unroll
+                    for (int m = 0; m < 7; ++m) {
+                        float tm = 0.f;
+                        if (L >= 3) { const float hv = H3[m]; tm = ps[0] * hv; ec[0] += B3[m] * hv; bt += B3[m] * tm; }
+                        t3[m] = tm;
+                    }
+                    const float w = g.chi * g.chi;
+                    float pr1 = 0.f;
+#pragma unroll
+                    for (int k = 0; k < W::C1; ++k) pr1 += ec[k] * dps[k];
+                    float ux, uy, uz;
+                    harmonics_grad_contract<L>(g.ux, g.uy, g.uz, t1, t2, t3, &ux, &uy, &uz);
+                    const float pux = w * ux, puy = w * uy, puz = w * uz;
+                    const float p_rho = g.chi * sa + w * pr1;
+                    const float p_chi = sb + 2.0f * g.chi * bt;
+                    const float dEdrho = p_rho + (p_chi + 2.0f * g.chi * ds0 + 4.0f * w * g.chi * ds1) * g.dchi;
                     const float dot = pux * g.ux + puy * g.uy + puz * g.uz;
                     gx = dEdrho * g.ux + (pux - dot * g.ux) * g.inv_rho;
                     gy = dEdrho * g.uy + (puy - dot * g.uy) * g.inv_rho;
@@ -437,6 +453,7 @@ k_edge_backward(const EdgeArgs a) {
     }
 }
 
+
 template <int C0, int L>
 cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
     if (a.d.R > 0) k_edge_forward<C0, L, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
@@ -445,8 +462,11 @@ cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
 }
 template <int C0, int L>
 cudaError_t launch_bwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
-    if (a.d.R > 0) k_edge_backward<C0, L, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
-    else k_edge_backward<C0, L, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    constexpr size_t bytes = BwdSmem<C0, L>::bytes;
+    auto kern = a.d.R > 0 ? k_edge_backward<C0, L, true> : k_edge_backward<C0, L, false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    kern<<<blocks, kWarpsPerBlock * 32, bytes, st>>>(a);
     return cudaGetLastError();
 }
 
