@@ -1,4 +1,4 @@
-// Tensor-core GEMM for the MLP layers on sm_100a: TMA loads into 128-byte-swizzled shared
+// Tensor-core GEMM for the MLP layers on sm_100a: TMA loads into 64-byte-swizzled shared
 // memory, tcgen05.mma (kind::tf32) issued by one thread, fp32 accumulator in tensor memory,
 // tcgen05.ld epilogue with the fused bias / SiLU / residual (or SiLU-derivative) step.
 //
@@ -10,9 +10,11 @@
 // treats the low mantissa bits.  Weights are split once on the host; activations are split
 // by a small kernel in front of each GEMM.
 //
-// Tiling: one CTA computes a 128 x 128 output tile; K advances in blocks of 32 floats (one
-// 128-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (64 KB
-// per stage).  Warp 0 is the TMA producer, warp 1 issues the MMAs and owns the tensor-memory
+// Tiling: one CTA computes a 128 x 128 output tile; K advances in blocks of 16 floats (one
+// 64-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (32 KB per
+// stage), so two CTAs fit on an SM and one CTA's epilogue overlaps the other's main loop
+// (a 128 x 128 x 8 TF32 MMA reads 8 KB of shared memory and is bound by that, ~94 cycles).
+// Warp 0 is the TMA producer, warp 1 issues the MMAs and owns the tensor-memory
 // allocation, warps 2-5 run the epilogue (one 32-lane quarter of tensor memory each).
 // Every mbarrier wait is bounded: on expiry the kernel flags an error word and carries on,
 // so a wedged pipeline ends with a wrong result and an error code instead of a hang, and
@@ -28,12 +30,13 @@ namespace umd {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 32, STAGES = 3;
-constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 16 KB, also BN * BK * 4
+constexpr int BM = 128, BN = 128, BK = 16, STAGES = 3;
+constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 8 KB, also BN * BK * 4
 constexpr uint32_t STAGE_BYTES = 4 * TILE_BYTES;      // A_hi, A_lo, B_hi, B_lo
 constexpr uint32_t BAR_BYTES = 128;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + BAR_BYTES;
 constexpr uint32_t TMEM_COLS = 128;
+constexpr int EPITCH = BN + 4;                        // epilogue staging pitch: 16-byte rows, odd in 16-byte units
 constexpr int kSpinLimit = 4000000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -66,11 +69,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
-// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, 8-row
-// groups 1024 B apart
+// shared-memory matrix descriptor: K-major tile, 64-byte swizzle, rows 64 B apart, 8-row
+// groups 512 B apart
 __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
-    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(512 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)4 << 61);
 }
 __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
     asm volatile(
@@ -104,7 +107,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 // instruction descriptor: D = F32, A = B = TF32, both K-major, N = 128, M = 128
 constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUtensorMap mAl,
           const __grid_constant__ CUtensorMap mBh, const __grid_constant__ CUtensorMap mBl, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
@@ -165,19 +168,50 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
             umma_commit(accum_bar);
         }
     } else {                                               // epilogue: warps 2..5 -> lane quarters 2,3,0,1
+        // Tensor memory hands each thread one accumulator row; global memory wants a warp
+        // on one row.  The tile is therefore turned through shared memory (the operand
+        // ring is free once the accumulator barrier has fired): each warp parks its 32
+        // rows with a padded pitch, then walks them row by row, lanes across columns, so
+        // every global access of the fused epilogue is one contiguous 512-byte segment.
         const int q = warp & 3;
         mbar_wait(accum_bar, 0, g.err);
         tc_fence_after();
-        const int m = m0 + q * 32 + lane;
+        float* stage = reinterpret_cast<float*>(smem_raw + (tiles - raw)) + (size_t)q * 32 * EPITCH;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
             float v[32];
             tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-            if (m < g.M) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int n = n0 + c0 + 4 * j;
-                    if (n < g.N) gemm_epilogue4(g, m, n, v + 4 * j);
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(stage + lane * EPITCH + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        }
+        __syncwarp();
+        const int n = n0 + 4 * lane;
+        if (n < g.N) {
+            float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias;
+            if (g.mode == 0) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+            const bool use_res = g.res && (g.res_n == 0 || n < g.res_n);
+            if (g.mode == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+            const int rows = min(32, g.M - (m0 + q * 32));
+#pragma unroll 4
+            for (int r = 0; r < rows; ++r) {
+                const size_t m = (size_t)(m0 + q * 32 + r);
+                float4 a = *reinterpret_cast<const float4*>(stage + r * EPITCH + 4 * lane);
+                float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (use_res) res = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
+                if (g.mode == 0) {
+                    a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
+                    if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
+                    *reinterpret_cast<float4*>(g.out + m * g.ldout + n) =
+                        make_float4(silu(a.x) + res.x, silu(a.y) + res.y, silu(a.z) + res.z, silu(a.w) + res.w);
+                } else {
+                    a.x += res.x + rvec.x; a.y += res.y + rvec.y; a.z += res.z + rvec.z; a.w += res.w + rvec.w;
+                    if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
+                    if (g.pre) {
+                        float4* pp = reinterpret_cast<float4*>(g.pre + m * g.ldpre + n);
+                        const float4 y = *pp;
+                        *pp = make_float4(a.x * silu_grad(y.x), a.y * silu_grad(y.y), a.z * silu_grad(y.z), a.w * silu_grad(y.w));
+                    }
                 }
             }
         }
@@ -230,7 +264,7 @@ EncodeFn encode_fn() {
     return fn;
 }
 
-// 2-D map over a row-major [rows][cols] float matrix with row pitch ld; box = 32 cols x 128 rows
+// 2-D map over a row-major [rows][cols] float matrix with row pitch ld; box = 16 cols x 128 rows
 bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
@@ -239,7 +273,7 @@ bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
     const cuuint32_t box[2] = {BK, BM};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
