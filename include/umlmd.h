@@ -194,6 +194,38 @@ int umlmd_get_profile(umlmd_t* h, int32_t max_classes, double* ms, int64_t* laun
 const char* umlmd_profile_class_name(int32_t cls);
 
 /*
+ * Kinetic energy sum_i m_i |v_i|^2 / 2 (eV) for callers that must not allocate.  (The
+ * paper has no counterpart: its integrator is LAMMPS'.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they need a number
+ * from it: a plugin running inside another program's real-time or memory-pooled loop,
+ * where the embedding application owns all device memory and forbids allocator calls (they
+ * can synchronise the whole device), or code that runs after its memory budget has been
+ * handed out.  Every other entry point may grow the handle's workspace; this one never
+ * does.  It calls no cudaMalloc, cudaFree or allocating library routine and needs no
+ * handle.  It is the same two-pass, fixed-order, double-precision reduction that
+ * umlmd_step uses for e_kin, with the per-block partial sums kept in a fixed 8 KB array
+ * inside the library's device image instead of allocated workspace.
+ *   N                 atoms, at most UMLMD_STATIC_MAX_ATOMS; more is rejected with
+ *                     UMLMD_E_CAPACITY and a message (umlmd_static_last_error)
+ *   d_vel             [N,3] double, Angstrom/ps           (device, caller-owned)
+ *   d_type            [N] int32 species                   (device, caller-owned)
+ *   d_mass_per_type   masses in amu indexed by species    (device, caller-owned)
+ *   d_e_kin           one double, receives the result     (device, caller-owned)
+ *   stream            cudaStream_t as void*; the call only enqueues work
+ * The first call on each device looks up the device address of the fixed array (current
+ * device = the one the stream belongs to); make that first call before starting any
+ * stream capture.  All calls on a device share the array: it keeps the previous call's
+ * partial sums, every entry that a call reads is first written by that same call so
+ * nothing needs clearing, and two calls whose kernels overlap on the GPU (different
+ * streams) race on it -- serialise them.
+ */
+#define UMLMD_STATIC_MAX_ATOMS 4194304
+int umlmd_kinetic_energy_static(int64_t N, const double* d_vel, const int32_t* d_type,
+                                const double* d_mass_per_type, double* d_e_kin, void* stream);
+const char* umlmd_static_last_error(void);
+
+/*
  * Read one entry of the ordered type-pair cache (host): out receives (2+R)*C0 doubles,
  * the scale gamma[C0], the shift beta[C0], then the mode mixing as R rows U[:, mu] of C0
  * values, for centre species type_i and neighbour species type_j.

@@ -24,7 +24,7 @@ EXPORTS = [
     "umlmd_profile_widths", "umlmd_create", "umlmd_destroy", "umlmd_query", "umlmd_last_error",
     "umlmd_build_neighbors", "umlmd_get_neighbors", "umlmd_compute", "umlmd_set_md_state", "umlmd_step",
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
-    "umlmd_get_profile", "umlmd_profile_class_name",
+    "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
 ]
 
 
@@ -73,8 +73,11 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_get_profile.argtypes = [vp, i32, ctypes.POINTER(dbl), ctypes.POINTER(i64), ctypes.POINTER(i32)]
     lib.umlmd_profile_class_name.argtypes = [i32]
     lib.umlmd_profile_class_name.restype = ctypes.c_char_p
+    lib.umlmd_kinetic_energy_static.argtypes = [i64, vp, vp, vp, vp, vp]
+    lib.umlmd_static_last_error.argtypes = []
+    lib.umlmd_static_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("umlmd_last_error", "umlmd_profile_class_name"):
+        if name not in ("umlmd_last_error", "umlmd_profile_class_name", "umlmd_static_last_error"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 

@@ -213,3 +213,71 @@ cudaError_t launch_kinetic_energy(int64_t N, const double* vel, const int* type,
 }
 
 }  // namespace umd
+
+// ---------------------------------------------------------------------------------------
+// Kinetic energy without any allocation (see umlmd_kinetic_energy_static in umlmd.h).
+//
+// Same two kernels as launch_kinetic_energy; the only difference is where the per-block
+// partial sums live: in a fixed array inside this library's device image instead of
+// workspace obtained from cudaMalloc.
+// ---------------------------------------------------------------------------------------
+namespace umd {
+namespace {
+
+constexpr int64_t kStaticMaxAtoms = (int64_t)kRedMaxBlocks * 4096;      // 4,194,304
+constexpr int kMaxDevices = 64;
+
+// Partial sums of one reduction (8 KB).  Every GPU that loads the library holds a copy
+// until the process exits.
+static __device__ __align__(256) double g_static_partials[kRedMaxBlocks];
+
+// g_static_partials is only a host-side handle in host code; the device address has to be
+// asked for, once per device, with that device current.
+double* g_static_partials_dev[kMaxDevices] = {nullptr};
+thread_local char g_static_err[256] = "";
+
+int static_fail(int code, const char* msg) {
+    snprintf(g_static_err, sizeof(g_static_err), "%s", msg);
+    return code;
+}
+
+}  // namespace
+}  // namespace umd
+
+extern "C" int umlmd_kinetic_energy_static(int64_t N, const double* d_vel, const int32_t* d_type,
+                                           const double* d_mass_per_type, double* d_e_kin, void* stream) {
+    using namespace umd;
+    if (N < 0 || !d_e_kin || (N > 0 && (!d_vel || !d_type || !d_mass_per_type)))
+        return static_fail(UMLMD_E_INVALID_ARG, "umlmd_kinetic_energy_static: null pointer or negative atom count");
+    if (N > kStaticMaxAtoms) {
+        char msg[200];
+        snprintf(msg, sizeof(msg), "umlmd_kinetic_energy_static: %lld atoms exceed the fixed scratch limit of %lld",
+                 (long long)N, (long long)kStaticMaxAtoms);
+        return static_fail(UMLMD_E_CAPACITY, msg);
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return static_fail(UMLMD_E_CUDA, "umlmd_kinetic_energy_static: no current CUDA device");
+    if (!g_static_partials_dev[dev]) {
+        double* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void**)&p, g_static_partials);
+        if (e != cudaSuccess || !p) {
+            char msg[200];
+            snprintf(msg, sizeof(msg), "umlmd_kinetic_energy_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            return static_fail(UMLMD_E_CUDA, msg);
+        }
+        g_static_partials_dev[dev] = p;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // every partial that the final pass reads is written by the first pass of the same call,
+    // so nothing left over from an earlier call needs clearing
+    cudaError_t e = launch_kinetic_energy(N, d_vel, d_type, d_mass_per_type, g_static_partials_dev[dev], d_e_kin, st);
+    if (e != cudaSuccess) {
+        char msg[200];
+        snprintf(msg, sizeof(msg), "umlmd_kinetic_energy_static: launch failed: %s", cudaGetErrorString(e));
+        return static_fail(UMLMD_E_CUDA, msg);
+    }
+    return UMLMD_OK;
+}
+
+extern "C" const char* umlmd_static_last_error(void) { return umd::g_static_err; }
