@@ -76,7 +76,8 @@ struct Lay {                                  // shared-memory plan, in floats
     static constexpr int nMat = C1 * C1 + C2 * C2 + C1 * K1 + C2 * K2;
     static constexpr int work_fwd = nZ1 + nZ2;
     static constexpr int work_bwd = nZ1 + nZ2 + 3 * C1 + 5 * C2 + 7 + nZ1 + nZ2;
-    static int floats(int SP, bool bwd) { return (SP + (bwd ? work_bwd : work_fwd) + CHUNK) * PITCH + nMat; }
+    static constexpr int nGaunt = L >= 3 ? 2 * (int)((sizeof(GauntSparse) + 3) / 4) : 0;
+    static int floats(int SP, bool bwd) { return (SP + (bwd ? work_bwd : work_fwd) + CHUNK) * PITCH + nMat + nGaunt; }
 };
 
 // Shared setup of both passes: stage matrices and the block's state slice, then per thread
@@ -86,6 +87,7 @@ template <int C1, int C2, int L>
 struct Front {
     static constexpr int K1 = C2, K2 = 2;
     float* tile; float* mW1; float* mW2; float* mA1; float* mA2;
+    const GauntSparse* G123; const GauntSparse* G233;     // shared-memory copies of the sparse couplings
     SCol T, Z1, Z2;
     double M0d, M1d;
     float iM0, iM1;
@@ -101,6 +103,17 @@ struct Front {
         for (int i = tid; i < C2 * C2; i += BLK) mW2[i] = __ldg(a.m.W2p + i);
         for (int i = tid; i < C1 * K1; i += BLK) mA1[i] = __ldg(a.m.A1 + i);
         for (int i = tid; i < C2 * K2; i += BLK) mA2[i] = __ldg(a.m.A2 + i);
+        G123 = nullptr; G233 = nullptr;
+        if (L >= 3) {
+            constexpr int nw = (int)((sizeof(GauntSparse) + 3) / 4);
+            unsigned* g1 = reinterpret_cast<unsigned*>(mA2 + C2 * K2);
+            unsigned* g2 = g1 + nw;
+            const unsigned* s1 = reinterpret_cast<const unsigned*>(a.m.g123);
+            const unsigned* s2 = reinterpret_cast<const unsigned*>(a.m.g233);
+            for (int i = tid; i < nw; i += BLK) { g1[i] = __ldg(s1 + i); g2[i] = __ldg(s2 + i); }
+            G123 = reinterpret_cast<const GauntSparse*>(g1);
+            G233 = reinterpret_cast<const GauntSparse*>(g2);
+        }
         b0 = blockIdx.x * BLK;
         nv = a.n - b0 < BLK ? a.n - b0 : BLK;
         const float* src = a.state + (size_t)b0 * d.SP;
@@ -185,22 +198,39 @@ __global__ void __launch_bounds__(BLK) k_inv_forward(const InvArgs a) {
     float* Dg = a.desc + (size_t)b0 * d.DP;
     const int ty = a.type_s[a.a0 + (b0 + tid < a.n ? b0 + tid : a.n - 1)];
 
-    // feature-vector columns are produced in increasing order; every 32nd one flushes
+    // feature-vector columns are produced in increasing order; every 32nd one flushes.  The
+    // calibration (v - mu) / sigma is applied by the flushing lane, which owns one column, so
+    // the per-thread code never waits on a global load; the two normalising scales arrive
+    // already calibrated (they are formed in double precision).
+    const int kM0 = 2 * C0, kM1 = 2 * C0 + 1;
     auto store = [&](int k, float v) {
         chunk[(k & (CHUNK - 1)) * PITCH + tid] = v;
         if ((k & (CHUNK - 1)) == CHUNK - 1) {
-            const int kb = k - (CHUNK - 1);
+            const int kb = k - (CHUNK - 1), col = kb + lane;
+            float mu_c = 0.f, is_c = 1.f;
+            if (col < d.D_out && col != kM0 && col != kM1) { mu_c = __ldg(m.mu + col); is_c = __ldg(m.inv_sigma + col); }
             __syncthreads();
-            for (int at = warp; at < nv; at += BLK / 32) Dg[(size_t)at * d.DP + kb + lane] = chunk[lane * PITCH + at];
+            for (int at = warp; at < nv; at += BLK / 32) Dg[(size_t)at * d.DP + col] = (chunk[lane * PITCH + at] - mu_c) * is_c;
             __syncthreads();
         }
     };
-    auto put = [&](int k, float v) { store(k, (v - __ldg(m.mu + k)) * __ldg(m.inv_sigma + k)); };
+    auto put = store;
 
-    for (int c = 0; c < C0; ++c) put(c, __ldg(m.X0 + ty * C0 + c));
+    // centre's initial-feature block: a plain gather, done by whole warps (lane = column) for
+    // every complete group of 32 columns; a trailing partial group goes through the stream
+    const int c_full = (C0 / CHUNK) * CHUNK;
+    for (int cb = 0; cb < c_full; cb += CHUNK) {
+        const int col = cb + lane;
+        const float mu_c = __ldg(m.mu + col), is_c = __ldg(m.inv_sigma + col);
+        for (int at = warp; at < nv; at += BLK / 32) {
+            const int tt = a.type_s[a.a0 + b0 + at];
+            Dg[(size_t)at * d.DP + col] = (__ldg(m.X0 + tt * C0 + col) - mu_c) * is_c;
+        }
+    }
+    for (int c = c_full; c < C0; ++c) put(c, __ldg(m.X0 + ty * C0 + c));
     for (int c = 0; c < C0; ++c) put(C0 + c, T[c] * f.iM0);
-    store(2 * C0, (float)((f.M0d - (double)__ldg(m.mu + 2 * C0)) * (double)__ldg(m.inv_sigma + 2 * C0)));
-    store(2 * C0 + 1, (float)((f.M1d - (double)__ldg(m.mu + 2 * C0 + 1)) * (double)__ldg(m.inv_sigma + 2 * C0 + 1)));
+    store(kM0, (float)((f.M0d - (double)__ldg(m.mu + kM0)) * (double)__ldg(m.inv_sigma + kM0)));
+    store(kM1, (float)((f.M1d - (double)__ldg(m.mu + kM1)) * (double)__ldg(m.inv_sigma + kM1)));
     const int o1 = d.offA[1], o2 = d.offA[2], o3 = d.offA[3];
     {   // Gram blocks, row-major upper triangle, strict off-diagonals times sqrt 2
         int k = d.oG[1];
@@ -240,7 +270,7 @@ __global__ void __launch_bounds__(BLK) k_inv_forward(const InvArgs a) {
             }
     }
     if (L >= 3) {   // (1,2,3): sparse Gaunt contraction
-        const GauntSparse* G = m.g123;
+        const GauntSparse* G = f.G123;
         const int nn = G->n;
         int k = d.oJ123;
         for (int k1 = 0; k1 < K1; ++k1)
@@ -264,7 +294,7 @@ __global__ void __launch_bounds__(BLK) k_inv_forward(const InvArgs a) {
             }
     }
     if (L >= 3) {   // (2,3,3)
-        const GauntSparse* G = m.g233;
+        const GauntSparse* G = f.G233;
         const int nn = G->n;
         int k = d.oJ233;
         for (int e = 0; e < K2; ++e) {
@@ -322,11 +352,13 @@ __global__ void __launch_bounds__(BLK) k_inv_backward(const InvArgs a) {
         const int c = k >> 5;
         if (c != cur) {
             __syncthreads();
-            for (int at = warp; at < nv; at += BLK / 32) chunk[lane * PITCH + at] = dDg[(size_t)at * d.DP + c * CHUNK + lane];
+            const int col = c * CHUNK + lane;
+            const float is_c = col < d.D_out ? __ldg(m.inv_sigma + col) : 0.f;
+            for (int at = warp; at < nv; at += BLK / 32) chunk[lane * PITCH + at] = dDg[(size_t)at * d.DP + col] * is_c;
             __syncthreads();
             cur = c;
         }
-        return chunk[(k & (CHUNK - 1)) * PITCH + tid] * __ldg(m.inv_sigma + k);
+        return chunk[(k & (CHUNK - 1)) * PITCH + tid];
     };
 
     const int o1 = d.offA[1], o2 = d.offA[2], o3 = d.offA[3];
@@ -388,7 +420,7 @@ __global__ void __launch_bounds__(BLK) k_inv_backward(const InvArgs a) {
             }
     }
     if (L >= 3) {   // (1,2,3)
-        const GauntSparse* G = m.g123;
+        const GauntSparse* G = f.G123;
         const int nn = G->n;
         int k = d.oJ123;
         for (int k1 = 0; k1 < K1; ++k1)
@@ -432,7 +464,7 @@ __global__ void __launch_bounds__(BLK) k_inv_backward(const InvArgs a) {
                 }
     }
     if (L >= 3) {   // (2,3,3)
-        const GauntSparse* G = m.g233;
+        const GauntSparse* G = f.G233;
         const int nn = G->n;
         int k = d.oJ233;
         for (int e = 0; e < K2; ++e) {

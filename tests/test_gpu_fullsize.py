@@ -1,0 +1,67 @@
+"""Full-size parity: the three large workloads in the configuration bench.py times (list
+radius r_c + skin, default node tiling, default MLP path), checked against the oracle on
+sampled outputs that it can compute one by one, plus properties that hold at any size."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dpa4c as orc
+from workloads import CONFIGS, make_system, workload_blob
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_19041_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("name,n_force,n_rows", [("cfg3_water32400", 3, 48), ("cfg4_hea128k", 3, 48),
+                                                 ("cfg5_amorphous1m", 2, 24)])
+def test_fullsize_sampled_parity(name, n_force, n_rows):
+    cfg = CONFIGS[name]
+    s = make_system(cfg["system"])
+    N = len(s["pos"])
+    blob = workload_blob(name)
+    skin = cfg["md"]["skin"]
+    m = _binding().Model(blob)
+    pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
+    types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], skin)
+    out = m.compute(pos, atom_energy=True)
+    Ei = out["atom_energy"].cpu().numpy()
+    F = out["forces"].cpu().numpy()
+    assert np.isfinite(Ei).all() and np.isfinite(F).all()
+
+    # ---- properties that hold at any size
+    f_scale, e_scale = np.abs(F).max(), np.abs(Ei).max()
+    assert abs(Ei.sum() - out["energy"]) <= 1e-9 * max(1.0, np.abs(Ei).sum())
+    assert np.abs(F.sum(axis=0)).max() <= 2e-6 * f_scale * np.sqrt(N) * 10       # sum of forces ~ fp32 noise
+    V = out["virial"]
+    assert np.abs(V - V.T).max() <= 1e-5 * max(np.abs(V).max(), 1e-12)
+
+    # ---- neighbor rows of sampled centres, bit-exact as sorted sets
+    rng = np.random.Generator(np.random.PCG64(2024 + cfg["index"]))
+    centers = np.sort(rng.choice(N, size=n_rows, replace=False))
+    pos_w = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    ref_rows = orc.neighbor_rows(pos_w, s["cell"], s["pbc"], cfg["profile"]["rc"] + skin, centers=centers)
+    row_ptr, src, shift = m.get_neighbors()
+    rp = row_ptr.cpu().numpy()
+    assert rp[-1] == m.query()["n_edges"]
+    for c, ref in zip(centers, ref_rows):
+        a, b = int(rp[c]), int(rp[c + 1])
+        ent = np.concatenate([src[a:b].cpu().numpy()[:, None].astype(np.int64),
+                              shift[a:b].cpu().numpy().astype(np.int64)], axis=1)
+        ent = ent[np.lexsort((ent[:, 3], ent[:, 2], ent[:, 1], ent[:, 0]))]
+        assert np.array_equal(ent, ref), c
+    del row_ptr, src, shift
+
+    # ---- forces on sampled atoms and energies of their whole neighbourhoods
+    o = orc.Oracle(blob)
+    for k in rng.choice(N, size=n_force, replace=False):
+        Fk, E_near = o.force_on(s["pos"], s["types"], s["cell"], s["pbc"], int(k))
+        assert np.abs(F[k] - Fk).max() <= min(1e-4, 2e-5 * f_scale + 2e-7), (k, F[k], Fk)
+        for a, ea in E_near.items():
+            assert abs(Ei[a] - ea) <= 1e-5 * e_scale, (a, Ei[a], ea)
+    m.close()
