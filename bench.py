@@ -229,9 +229,17 @@ def run_ours(args):
     cfg = CONFIGS[name]
     p = cfg["profile"]
     md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=300.0, seed=1, rebuild_every=10, skin=0.0)
-    s = make_system(cfg["system"], md)
+    desc = dict(cfg["system"])
+    if args.atoms:
+        # a smaller box of the same recipe (density, exclusion radius, species mix): the size one
+        # node tile of the full workload has, for profiler captures that must stay small
+        if desc.get("kind") != "poisson_disk":
+            raise SystemExit("--atoms applies to the amorphous workload only")
+        desc["atoms"] = int(args.atoms)
+        name = f"{name}[atoms={int(args.atoms)}]"
+    s = make_system(desc, md)
     N = len(s["pos"])
-    blob = workload_blob(name)
+    blob = workload_blob(args.workload)
     model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile)
     pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
     pos = pos0.cuda().contiguous()
@@ -292,8 +300,7 @@ def run_ours(args):
     dom = dict(kernels[0]) if kernels else None
     if dom:
         dom["peak_source"] = peaks["source"]
-        traffic = load_traffic(name, dom["kernel"])
-        dom["traffic"] = traffic
+        dom["traffic"] = load_traffic(args.workload, dom["kernel"])
 
     # ---- end to end from host buffers: upload positions, evaluate, download forces
     k_e2e = max(1, min(args.steps, 10))
@@ -325,7 +332,7 @@ def run_ours(args):
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        smp = OracleSampler(name)
+        smp = OracleSampler(args.workload)
         n_s = smp.sized_for(args.cpu_seconds)
         t_s = smp.run(n_s, offset=8)
         cpu = dict(value=n_s / t_s, unit="atom-steps/s", cores=smp.cores, kind="oracle",
@@ -349,15 +356,18 @@ def run_ours(args):
 
 
 def load_traffic(workload, kernel):
-    """DRAM bytes per launch from a stored ncu capture (profiles/traffic.json), if any."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of one kernel class on
+    one workload, from the stored summary of an ncu capture: lines "workload class bytes" in
+    profiles/dram_traffic_per_launch.txt.  None when no capture is stored."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
     if not os.path.exists(path):
         return None
-    try:
-        with open(path) as f:
-            return json.load(f).get(workload, {}).get(kernel)
-    except Exception:
-        return None
+    with open(path) as f:
+        for ln in f:
+            w = ln.split()
+            if len(w) >= 3 and not ln.startswith("#") and w[0] == workload and w[1] == kernel:
+                return float(w[2])
+    return None
 
 
 def main():
@@ -369,6 +379,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
     ap.add_argument("--mlp-path", type=int, default=0)
     ap.add_argument("--node-tile", type=int, default=0)
+    ap.add_argument("--atoms", type=int, default=0, help="amorphous workload only: atoms of a smaller box of the same recipe")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
