@@ -193,24 +193,41 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
             const bool use_res = g.res && (g.res_n == 0 || n < g.res_n);
             if (g.mode == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
             const int rows = min(32, g.M - (m0 + q * 32));
-#pragma unroll 4
-            for (int r = 0; r < rows; ++r) {
-                const size_t m = (size_t)(m0 + q * 32 + r);
-                float4 a = *reinterpret_cast<const float4*>(stage + r * EPITCH + 4 * lane);
-                float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (use_res) res = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
-                if (g.mode == 0) {
-                    a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
-                    if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
-                    *reinterpret_cast<float4*>(g.out + m * g.ldout + n) =
-                        make_float4(silu(a.x) + res.x, silu(a.y) + res.y, silu(a.z) + res.z, silu(a.w) + res.w);
-                } else {
-                    a.x += res.x + rvec.x; a.y += res.y + rvec.y; a.z += res.z + rvec.z; a.w += res.w + rvec.w;
-                    if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
-                    if (g.pre) {
-                        float4* pp = reinterpret_cast<float4*>(g.pre + m * g.ldpre + n);
-                        const float4 y = *pp;
-                        *pp = make_float4(a.x * silu_grad(y.x), a.y * silu_grad(y.y), a.z * silu_grad(y.z), a.w * silu_grad(y.w));
+            // The stores below may alias the loads as far as the compiler knows, so the rows
+            // are taken in batches: all global loads of a batch are issued before its first
+            // store, which keeps RB rows (not one) in flight per warp.
+            constexpr int RB = 8;
+            const bool rd_pre = g.mode == 1 && g.pre;
+#pragma unroll 1
+            for (int r0 = 0; r0 < rows; r0 += RB) {
+                float4 res[RB], y[RB];
+#pragma unroll
+                for (int j = 0; j < RB; ++j) {
+                    const size_t m = (size_t)(m0 + q * 32 + r0 + j);
+                    res[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    y[j] = res[j];
+                    if (r0 + j < rows) {
+                        if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
+                        if (rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < RB; ++j) {
+                    if (r0 + j >= rows) break;
+                    const size_t m = (size_t)(m0 + q * 32 + r0 + j);
+                    float4 a = *reinterpret_cast<const float4*>(stage + (r0 + j) * EPITCH + 4 * lane);
+                    if (g.mode == 0) {
+                        a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
+                        if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
+                        *reinterpret_cast<float4*>(g.out + m * g.ldout + n) =
+                            make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z, silu(a.w) + res[j].w);
+                    } else {
+                        a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
+                        if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
+                        if (g.pre)
+                            *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) =
+                                make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y), a.z * silu_grad(y[j].z),
+                                            a.w * silu_grad(y[j].w));
                     }
                 }
             }
