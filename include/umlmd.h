@@ -82,8 +82,9 @@ int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out);
  *   A_1[C1,K1], A_2[C2,K2], mu[D_out], sigma[D_out], Theta_1[D_out,F], b_1[F],
  *   {Theta_t[F,F], b_t[F]} t = 2..n_hidden, w_head[F], b_head, E_ref[T].
  * The create step evaluates, once and in double precision on the host, everything the
- * paper's compressed inference precomputes: the quintic-Hermite radial table of the shared
- * radial map and modes on [0, rc] (value, first and second derivative at each knot), the
+ * paper's compressed inference precomputes: the Hermite radial table of the shared radial
+ * map and modes on [0, rc] (the cubic through value and first derivative at each knot; the
+ * paper stores the quintic that also matches the second derivative), the
  * ordered type-pair scale / shift / mode-mixing cache, and the unit-norm Gaunt coupling
  * tensors of the admissible degree triples.
  *   stream: a cudaStream_t passed as void* (NULL = the default stream).
@@ -173,7 +174,7 @@ int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc);
 
 /*
  * Evaluate the tabulated radial map at n distances (host arrays): out_g [n, C0+R] holds
- * g(rho) then q(rho), out_dg their derivatives, from the same quintic polynomials the
+ * g(rho) then q(rho), out_dg their derivatives, from the same cubic polynomials the
  * kernels use (evaluated on the host from the device table's float32 coefficients).
  */
 int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, double* out_g,

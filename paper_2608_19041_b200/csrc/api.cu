@@ -112,8 +112,8 @@ int ensure_workspace(umlmd_t* h) {
         c = 0; API_CUDA(h, dev_ensure(&h->pre, &c, B * d.F * d.n_hidden));
         c = 0; API_CUDA(h, dev_ensure(&h->hbuf, &c, B * d.F * 2));
         const int64_t wmax = d.DP > d.F ? d.DP : d.F;
-        c = 0; API_CUDA(h, dev_ensure(&h->tc_hi, &c, B * wmax));
-        c = 0; API_CUDA(h, dev_ensure(&h->tc_lo, &c, B * wmax));
+        c = 0; API_CUDA(h, dev_ensure(&h->tc_hi, &c, 2 * B * wmax));
+        c = 0; API_CUDA(h, dev_ensure(&h->tc_lo, &c, 2 * B * wmax));
         h->tile_cap = B;
     }
     if (E > h->g_cap || !h->g) { API_CUDA(h, dev_ensure(&h->g, &h->g_cap, E * 3, 1.1)); h->g_cap /= 3; }
@@ -163,7 +163,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err;
-        { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
+        ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
+        { Scope sc(h, kMlpFwd, d.n_hidden + (h->mlp_path == 2 ? 2 : 1)); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
             { Scope sc(h, kInvBwd, 1); API_CUDA(h, launch_invariants_backward(ia, h->st)); }
@@ -431,12 +432,11 @@ int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, doub
         if (row < 0) row = 0;
         if (row > d.n_rows - 1) row = d.n_rows - 1;
         const double t = rho[i] - row * h->hm.dx;
-        const float* p = &h->hm.table[(size_t)row * 6 * d.CP];
+        const float* p = &h->hm.table[(size_t)row * 4 * d.CP];
         for (int c = 0; c < NC; ++c) {
-            const double c0 = p[c], c1 = p[d.CP + c], c2 = p[2 * d.CP + c], c3 = p[3 * d.CP + c], c4 = p[4 * d.CP + c],
-                         c5 = p[5 * d.CP + c];
-            out_g[i * NC + c] = ((((c5 * t + c4) * t + c3) * t + c2) * t + c1) * t + c0;
-            if (out_dg) out_dg[i * NC + c] = (((5 * c5 * t + 4 * c4) * t + 3 * c3) * t + 2 * c2) * t + c1;
+            const double c0 = p[c], c1 = p[d.CP + c], c2 = p[2 * d.CP + c], c3 = p[3 * d.CP + c];
+            out_g[i * NC + c] = ((c3 * t + c2) * t + c1) * t + c0;
+            if (out_dg) out_dg[i * NC + c] = (3 * c3 * t + 2 * c2) * t + c1;
         }
     }
     return UMLMD_OK;

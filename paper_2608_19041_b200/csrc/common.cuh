@@ -49,7 +49,7 @@ struct GauntSparse {         // non-zeros of one unit-norm coupling tensor
 
 // Device-resident constants of one model.
 struct ModelDev {
-    float* table;     // [n_rows][6][CP] quintic coefficients c0..c5 of [g, q]
+    float* table;     // [n_rows][4][CP] cubic Hermite coefficients c0..c3 of [g, q]
     float* pairmod;   // [T*T][2+R][C0]: scale gamma, shift beta, mode mixing U[:, mu]
     float* X0;        // [T][C0]
     float* W1p;       // [C1][C1]  I + W_1

@@ -9,7 +9,7 @@
 // reads are 16-byte vector loads that a group issues as one contiguous segment.  The S+2
 // sums live in registers and are written once per destination; nothing per-edge is stored
 // in the forward pass.  The backward pass recomputes the same per-edge quantities from the
-// same quintic polynomial (so the force is the exact derivative of the interpolated
+// same cubic polynomial (so the force is the exact derivative of the interpolated
 // energy), contracts them with dE/d(sums) and writes one 3-vector per edge; the virial is
 // accumulated in the same pass.
 //
@@ -113,12 +113,11 @@ __device__ __forceinline__ void harmonics_grad_contract(float x, float y, float 
 template <bool DERIV>
 __device__ __forceinline__ void table_eval4(const float* __restrict__ table, int CP, int row, int c, float t,
                                             float* v, float* dv) {
-    const float* p = table + (size_t)row * 6 * CP + c;
-    const float4 c0 = ldg4(p), c1 = ldg4(p + CP), c2 = ldg4(p + 2 * CP), c3 = ldg4(p + 3 * CP),
-                 c4 = ldg4(p + 4 * CP), c5 = ldg4(p + 5 * CP);
+    const float* p = table + (size_t)row * 4 * CP + c;
+    const float4 c0 = ldg4(p), c1 = ldg4(p + CP), c2 = ldg4(p + 2 * CP), c3 = ldg4(p + 3 * CP);
 #define UMLMD_HORNER(k, f)                                                                             \
-    v[k] = ((((c5.f * t + c4.f) * t + c3.f) * t + c2.f) * t + c1.f) * t + c0.f;                        \
-    if (DERIV) dv[k] = (((5.0f * c5.f * t + 4.0f * c4.f) * t + 3.0f * c3.f) * t + 2.0f * c2.f) * t + c1.f;
+    v[k] = ((c3.f * t + c2.f) * t + c1.f) * t + c0.f;                                                  \
+    if (DERIV) dv[k] = (3.0f * c3.f * t + 2.0f * c2.f) * t + c1.f;
     UMLMD_HORNER(0, x) UMLMD_HORNER(1, y) UMLMD_HORNER(2, z) UMLMD_HORNER(3, w)
 #undef UMLMD_HORNER
 }
@@ -126,11 +125,10 @@ __device__ __forceinline__ void table_eval4(const float* __restrict__ table, int
 template <bool DERIV>
 __device__ __forceinline__ void table_eval1(const float* __restrict__ table, int CP, int row, int c, float t,
                                             float* v, float* dv) {
-    const float* p = table + (size_t)row * 6 * CP + c;
-    const float c0 = __ldg(p), c1 = __ldg(p + CP), c2 = __ldg(p + 2 * CP), c3 = __ldg(p + 3 * CP),
-                c4 = __ldg(p + 4 * CP), c5 = __ldg(p + 5 * CP);
-    *v = ((((c5 * t + c4) * t + c3) * t + c2) * t + c1) * t + c0;
-    if (DERIV) *dv = (((5.0f * c5 * t + 4.0f * c4) * t + 3.0f * c3) * t + 2.0f * c2) * t + c1;
+    const float* p = table + (size_t)row * 4 * CP + c;
+    const float c0 = __ldg(p), c1 = __ldg(p + CP), c2 = __ldg(p + 2 * CP), c3 = __ldg(p + 3 * CP);
+    *v = ((c3 * t + c2) * t + c1) * t + c0;
+    if (DERIV) *dv = (3.0f * c3 * t + 2.0f * c2) * t + c1;
 }
 
 // amplitude psi (and d psi / d rho) of this lane's four channels for one edge

@@ -65,8 +65,9 @@ struct MlpArgs {
     double* e_atom;         // [N] sorted order, eV (written at a0..a0+n)
     int path;               // 1 = CUDA-core fp32, 2 = tcgen05
     bool want_grad;
-    float* tc_hi;           // [n][max(DP, F)] scratch for the tensor-core path
+    float* tc_hi;           // two slots of [n][max(DP, F)]: TF32 splits of the activations (tensor-core path)
     float* tc_lo;
+    size_t tc_slot;         // floats per slot
     int* err;               // device error word
 };
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)

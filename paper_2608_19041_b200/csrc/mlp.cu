@@ -61,10 +61,11 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
 }
 
 // scalar head: E_i = h . w_head + b_head + E_ref[type]; seeds the backward pass with
-// dE/dY_last = w_head * SiLU'(Y_last)
+// dE/dY_last = w_head * SiLU'(Y_last) (also as a TF32 split for the tensor-core path)
 __global__ void k_head(int n, int F, const float* __restrict__ h, const float* __restrict__ w, float b_head,
                        const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
-                       float* __restrict__ pre_last, double* __restrict__ e_atom, bool want_grad) {
+                       float* __restrict__ pre_last, float* __restrict__ seed_hi, float* __restrict__ seed_lo,
+                       double* __restrict__ e_atom, bool want_grad) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= n) return;
     const float* hr = h + (size_t)warp * F;
@@ -76,7 +77,11 @@ __global__ void k_head(int n, int F, const float* __restrict__ h, const float* _
         e_atom[a0 + warp] = (double)s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + warp]);
     if (want_grad) {
         float* pr = pre_last + (size_t)warp * F;
-        for (int f = lane; f < F; f += 32) pr[f] = __ldg(w + f) * silu_grad(pr[f]);
+        for (int f = lane; f < F; f += 32) {
+            const float v = __ldg(w + f) * silu_grad(pr[f]);
+            pr[f] = v;
+            if (seed_hi) split_tf32(v, seed_hi[(size_t)warp * F + f], seed_lo[(size_t)warp * F + f]);
+        }
     }
 }
 
@@ -101,6 +106,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     const size_t layer = (size_t)n * F;
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
+    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo;
     cudaError_t e;
     // ---- forward --------------------------------------------------------------------
     for (int t = 0; t < NH; ++t) {
@@ -111,7 +117,14 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         else { g.A = hb[(t - 1) & 1]; g.lda = F; g.K = F; g.res = hb[(t - 1) & 1]; g.ldres = F; }
         g.B = a.m.theta[t]; g.ldb = F;
         g.Bt_hi = a.m.thetaT_hi[t]; g.Bt_lo = a.m.thetaT_lo[t]; g.ldbt = t == 0 ? d.DP : F;
-        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
+        // tensor-core path: the split of layer t's input sits in slot t & 1 (layer 0's is made by
+        // the split kernel), and the epilogue leaves the split of its output in the other slot
+        g.A_hi = a.tc_hi + (size_t)(t & 1) * a.tc_slot; g.A_lo = a.tc_lo + (size_t)(t & 1) * a.tc_slot;
+        g.a_presplit = t > 0; g.err = a.err;
+        if (tc && t + 1 < NH) {
+            g.nxt_hi = a.tc_hi + (size_t)((t + 1) & 1) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)((t + 1) & 1) * a.tc_slot;
+            g.ldnxt = F;
+        }
         g.bias = a.m.bias[t];
         g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
         g.out = hb[t & 1]; g.ldout = F;
@@ -121,7 +134,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         const int warps = 8, blocks = (n + warps - 1) / warps;
         k_head<<<blocks, warps * 32, 0, st>>>(n, F, hb[(NH - 1) & 1], a.m.w_head, a.m.b_head, a.m.e_ref, a.type_s,
                                              a.a0, a.want_grad ? a.pre + (size_t)(NH - 1) * layer : nullptr,
-                                             a.e_atom, a.want_grad);
+                                             tc ? a.tc_hi : nullptr, tc ? a.tc_lo : nullptr, a.e_atom, a.want_grad);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -136,6 +149,8 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
     cudaError_t e;
+    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo;
+    int sp = 0;                // tensor-core path: slot with the TF32 split of pre[t] (the head kernel fills slot 0)
     int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
     bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
     for (int t = NH - 1; t >= 1; --t) {
@@ -145,7 +160,10 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.A = a.pre + (size_t)t * layer; g.lda = F;
         g.B = a.m.thetaT[t]; g.ldb = F;
         g.Bt_hi = a.m.theta_hi[t]; g.Bt_lo = a.m.theta_lo[t]; g.ldbt = F;
-        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
+        g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
+        g.a_presplit = tc; g.err = a.err;
+        if (tc) { g.nxt_hi = a.tc_hi + (size_t)(1 - sp) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)(1 - sp) * a.tc_slot; g.ldnxt = F; }
+        sp = 1 - sp;
         if (vec_grad) g.rvec = a.m.w_head; else { g.res = hb[slot]; g.ldres = F; }
         const int out_slot = vec_grad ? 0 : 1 - slot;
         const bool need_dh = (t - 1 >= 1) || res0;
@@ -161,7 +179,8 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.A = a.pre; g.lda = F;
         g.B = a.m.thetaT[0]; g.ldb = d.DP;
         g.Bt_hi = a.m.theta_hi[0]; g.Bt_lo = a.m.theta_lo[0]; g.ldbt = F;
-        g.A_hi = a.tc_hi; g.A_lo = a.tc_lo; g.err = a.err;
+        g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
+        g.a_presplit = tc; g.err = a.err;
         if (res0) {
             if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }

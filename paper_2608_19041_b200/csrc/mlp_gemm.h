@@ -4,6 +4,8 @@
 
 #include <cuda_runtime.h>
 
+#include <cstdint>
+
 namespace umd {
 
 // C[M,N] = A[M,K] (row-major, lda) x B[K,N] (row-major, ldb), then
@@ -23,7 +25,11 @@ struct GemmArgs {
     float* out; int ldout;
     // tensor-core path only: pre-split copies of B (hi / lo TF32 parts), K-major [N][K]
     const float* Bt_hi; const float* Bt_lo; int ldbt;
-    float* A_hi; float* A_lo;     // scratch [M][K] for the split of A
+    float* A_hi; float* A_lo;     // [M][K] TF32 split of A: filled by the caller if a_presplit, else by a split kernel
+    int a_presplit;
+    // TF32 split of the value the next GEMM of the chain consumes (mode 0: out, mode 1: the new
+    // pre), written by the epilogue with row pitch ldnxt when non-null
+    float* nxt_hi; float* nxt_lo; int ldnxt;
     int* err;                     // device error word (bounded-wait expiry)
 };
 
@@ -34,6 +40,21 @@ __device__ __forceinline__ float silu_grad(float x) {
     return s * (1.0f + x * (1.0f - s));
 }
 
+// x = hi + lo with hi = round-to-nearest TF32 of x and lo = round-to-nearest TF32 of (x - hi)
+__device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
+    uint32_t hb, lb;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hb) : "f"(x));
+    hi = __uint_as_float(hb);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lb) : "f"(x - hi));
+    lo = __uint_as_float(lb);
+}
+__device__ __forceinline__ void store_split4(float* hi, float* lo, size_t off, float4 v) {
+    float4 h, l;
+    split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
+    *reinterpret_cast<float4*>(hi + off) = h;
+    *reinterpret_cast<float4*>(lo + off) = l;
+}
+
 // epilogue for four consecutive columns n..n+3 of row m (n multiple of 4, n < N)
 __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, float* v) {
     if (g.mode == 0) {
@@ -42,8 +63,9 @@ __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, 
         if (g.pre) *reinterpret_cast<float4*>(g.pre + (size_t)m * g.ldpre + n) = make_float4(v[0], v[1], v[2], v[3]);
         float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
         if (g.res) r = *reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n);
-        *reinterpret_cast<float4*>(g.out + (size_t)m * g.ldout + n) =
-            make_float4(silu(v[0]) + r.x, silu(v[1]) + r.y, silu(v[2]) + r.z, silu(v[3]) + r.w);
+        const float4 o = make_float4(silu(v[0]) + r.x, silu(v[1]) + r.y, silu(v[2]) + r.z, silu(v[3]) + r.w);
+        *reinterpret_cast<float4*>(g.out + (size_t)m * g.ldout + n) = o;
+        if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, (size_t)m * g.ldnxt + n, o);
     } else {
         if (g.res && (g.res_n == 0 || n < g.res_n)) {
             const float4 r = *reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n);
@@ -57,8 +79,10 @@ __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, 
         if (g.pre) {
             float4* p = reinterpret_cast<float4*>(g.pre + (size_t)m * g.ldpre + n);
             const float4 y = *p;
-            *p = make_float4(v[0] * silu_grad(y.x), v[1] * silu_grad(y.y), v[2] * silu_grad(y.z),
-                             v[3] * silu_grad(y.w));
+            const float4 o = make_float4(v[0] * silu_grad(y.x), v[1] * silu_grad(y.y), v[2] * silu_grad(y.z),
+                                         v[3] * silu_grad(y.w));
+            *p = o;
+            if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, (size_t)m * g.ldnxt + n, o);
         }
     }
 }

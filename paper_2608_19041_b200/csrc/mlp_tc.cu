@@ -8,7 +8,7 @@
 // A_lo B_hi + A_hi B_lo + A_hi B_hi (the lo*lo term, ~2^-22, is dropped).  Both parts are
 // exactly representable in TF32, so the result does not depend on how the tensor core
 // treats the low mantissa bits.  Weights are split once on the host; activations are split
-// by a small kernel in front of each GEMM.
+// by the epilogue that produces them (or, for the first GEMM of a chain, by a small kernel).
 //
 // Tiling: one CTA computes a 128 x 128 output tile; K advances in blocks of 16 floats (one
 // 64-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (32 KB per
@@ -219,15 +219,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     if (g.mode == 0) {
                         a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
                         if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
-                        *reinterpret_cast<float4*>(g.out + m * g.ldout + n) =
-                            make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z, silu(a.w) + res[j].w);
+                        const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
+                                                     silu(a.w) + res[j].w);
+                        *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
+                        if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
                     } else {
                         a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
                         if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
-                        if (g.pre)
-                            *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) =
-                                make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y), a.z * silu_grad(y[j].z),
-                                            a.w * silu_grad(y[j].w));
+                        if (g.pre) {
+                            const float4 o = make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y),
+                                                         a.z * silu_grad(y[j].z), a.w * silu_grad(y[j].w));
+                            *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
+                            if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
+                        }
                     }
                 }
             }
@@ -248,18 +252,7 @@ __global__ void k_split_tf32(const float* __restrict__ A, int lda, int M, int K,
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int m = (int)(i / k4), k = (int)(i - (size_t)m * k4) * 4;
         const float4 x = *reinterpret_cast<const float4*>(A + (size_t)m * lda + k);
-        const float xs[4] = {x.x, x.y, x.z, x.w};
-        float h[4], l[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t hb, lb;
-            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hb) : "f"(xs[j]));
-            h[j] = __uint_as_float(hb);
-            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lb) : "f"(xs[j] - h[j]));
-            l[j] = __uint_as_float(lb);
-        }
-        *reinterpret_cast<float4*>(hi + (size_t)m * K + k) = make_float4(h[0], h[1], h[2], h[3]);
-        *reinterpret_cast<float4*>(lo + (size_t)m * K + k) = make_float4(l[0], l[1], l[2], l[3]);
+        store_split4(hi, lo, (size_t)m * K + k, x);
     }
 }
 
@@ -308,7 +301,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    {
+    if (!g.a_presplit) {
         const size_t total = (size_t)g.M * (g.K >> 2);
         int blocks = (int)((total + 255) / 256);
         if (blocks > 148 * 16) blocks = 148 * 16;
