@@ -117,8 +117,10 @@ class ClockSampler:
 def work_model(p, n_atoms, e_rc, e_list):
     """Algorithmic FLOPs (FMA = 2) and compulsory HBM bytes per evaluation, per kernel class."""
     C0, R, S, D, F, NH, C1 = p["C0"], p["R"], p["S"], p["D_out"], p["F"], p["n_hidden"], p["C1"]
-    fwd_edge = 10 * (C0 + R) + 2 * C0 * (1 + R) + 2 * S + C0 + C1 + 60
-    bwd_edge = 18 * (C0 + R) + 4 * C0 * (1 + R) + 4 * S + 2 * C0 + 250
+    # per edge: cubic Horner of the table channels (6 flops a value, 4 more for its derivative),
+    # pair modulation, the S+2 accumulations, envelope and harmonics
+    fwd_edge = 6 * (C0 + R) + 2 * C0 * (1 + R) + 2 * S + C0 + C1 + 60
+    bwd_edge = 10 * (C0 + R) + 4 * C0 * (1 + R) + 4 * S + 2 * C0 + 250
     mlp = 2 * (D * F + (NH - 1) * F * F + F)
     return {
         "edge_forward": dict(flops=fwd_edge * e_rc, bytes=8 * e_list + n_atoms * (28 + 4 * (S + 2)), pipe="alu"),
