@@ -4,15 +4,22 @@
 // invariant, assembly and diagonal calibration -- and the matching vector-Jacobian
 // product, which turns dE/dD into dE/d(sums) in place of the saved sums.
 //
-// A block handles 64 atoms with 256 threads: four adjacent lanes share one atom.  All
-// per-atom tensors live in shared memory in an [index][atom] layout with an odd row pitch
-// (conflict-free for a warp's accesses).  Work is divided among an atom's four lanes so
-// that no two lanes ever accumulate into the same entry: forward outputs are dealt out
-// round-robin, backward accumulators are owned by harmonic row (each lane owns one
-// degree-1 row and one or two degree-2 rows), so there are no atomics and the result is
-// bitwise reproducible.  Global memory is only touched by block-cooperative, coalesced
-// transfers: the block's slice of the state array is staged in one pass, and the feature
-// vector streams through a 32-column staging buffer in increasing column order.
+// A block handles 32 atoms with eight warps, lane = atom.  All per-atom tensors live in
+// shared memory in an [index][atom] layout with row pitch 33, so a warp that reads or
+// writes one index for its 32 atoms touches 32 distinct banks, and every index computation
+// is uniform over the warp.  The work of a phase is cut into units (an output row, a pair
+// of Gram rows, one probe index ...) that are dealt round-robin to the warps; each output
+// entry has exactly one writer and a fixed summation order, so there are no atomics and the
+// result is bitwise reproducible.  Phases are separated by block barriers.  Global memory
+// is only touched by block-cooperative, coalesced transfers (lane = column): the state
+// slice and the feature rows are staged once per block.
+//
+// The sparse Gaunt triples are contracted through small intermediates instead of per
+// entry: with the non-zeros (m1, m2, m3, v) of the (1,2,3) coupling,
+//   U[m1][e] = sum_n v Z2[m2][e] X3[m3],   J123[k][e] = sum_m1 Z1[m1][k] U[m1][e],
+// and with those of the (2,3,3) coupling
+//   Y[m1] = sum_n v X3[m2] X3[m3],         J233[e] = sum_m1 Z2[m1][e] Y[m1];
+// the backward pass uses the same factorisation.
 //
 // The two normalising scales are standardised by the calibration, (M - mu) / sigma with
 // mu ~ M, so they are formed in double precision from sums accumulated in double (stored
@@ -23,11 +30,10 @@ namespace umd {
 
 namespace {
 
-constexpr int ATOMS = 64;            // atoms per block
-constexpr int LPA = 4;               // lanes per atom
-constexpr int NT = ATOMS * LPA;      // threads per block
-constexpr int PITCH = ATOMS + 1;
-constexpr int CHUNK = 32;
+constexpr int AT = 32;               // atoms per block = lanes
+constexpr int NW = 8;                // warps per block
+constexpr int NT = AT * NW;
+constexpr int P = AT + 1;            // row pitch of the [index][atom] layout
 constexpr unsigned kFull = 0xffffffffu;
 
 constexpr float kR2 = 1.4142135623730951f;
@@ -36,17 +42,6 @@ constexpr float kInvR6 = 0.4082482904638631f;
 constexpr float kC112 = -0.4472135954999579f;    // -1/sqrt(5)
 constexpr float kC222 = -0.5855400437691199f;    // -sqrt(12/35)
 constexpr float kR3 = 1.7320508075688772f;
-
-// column of the [index][atom] shared-memory layout belonging to one atom
-struct SCol {
-    float* p;
-    __device__ __forceinline__ float& operator[](int i) const { return p[i * PITCH]; }
-};
-
-// which of an atom's four lanes owns a harmonic row
-__device__ __forceinline__ int own1(int m) { return m; }             // degree 1: rows 0,1,2 -> lanes 0,1,2
-__device__ __forceinline__ int own2(int m) { return (m + 3) & 3; }   // degree 2: rows 0..4 -> lanes 3,0,1,2,3
-__device__ __forceinline__ int own3(int m) { return m & 3; }         // degree 3: rows 0..6 round-robin
 
 // symmetric trace-free matrix of a packed degree-2 vector, row-major 3x3
 __device__ __forceinline__ void stf9(float z1, float z2, float z3, float z4, float z5, float* Q) {
@@ -79,92 +74,73 @@ __device__ __forceinline__ float fam3(int a, int b, int c) {
     if (a == b || b == c) return kR3;
     return 2.449489742783178f;
 }
-// picks component i of a 3-vector held in registers without a dynamic register index
-__device__ __forceinline__ float pick3(const float* v, int i) { return i == 0 ? v[0] : (i == 1 ? v[1] : v[2]); }
-
-// ---- feature-vector streaming through the 32-column staging buffer --------------------
-// The per-column paths are force-inlined so that their state stays in registers; only the
-// block-wide transfers (once per 32 columns) are real calls.
-
-// write columns [kb, kb+32) of the block's feature vectors: lane = column, calibrated
-__device__ __noinline__ void flush_columns(const float* chunk, float* Dg, const float* mu, const float* inv_sigma,
-                                           int kb, int nv, int DP, int D_out, int k_skip0, int k_skip1) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int col = kb + lane;
-    float mu_c = 0.f, is_c = 1.f;
-    if (col < D_out && col != k_skip0 && col != k_skip1) { mu_c = __ldg(mu + col); is_c = __ldg(inv_sigma + col); }
-    __syncthreads();
-    for (int aa = warp; aa < nv; aa += NT / 32) Dg[(size_t)aa * DP + col] = (chunk[lane * PITCH + aa] - mu_c) * is_c;
-    __syncthreads();
-}
-__device__ __forceinline__ void put_column(float* chunk, int at, int k, float v, bool own, float* Dg, const float* mu,
-                                           const float* inv_sigma, int nv, int DP, int D_out, int k_skip0, int k_skip1) {
-    if (own) chunk[(k & (CHUNK - 1)) * PITCH + at] = v;
-    if ((k & (CHUNK - 1)) == CHUNK - 1) flush_columns(chunk, Dg, mu, inv_sigma, k - (CHUNK - 1), nv, DP, D_out, k_skip0, k_skip1);
-}
-// Backward streaming: columns [32c, 32c+32) of the block's dE/dD rows are fetched with
-// asynchronous copies into one of two staging buffers while the previous 32 columns are
-// being consumed, so the DRAM latency of the fetch is off the critical path.
-__device__ __forceinline__ void issue_columns(float* buf, const float* dDg, int c, int nv, int DP) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int col = c * CHUNK + lane;
-    if (col < DP) {
-        for (int aa = warp; aa < nv; aa += NT / 32) {
-            const unsigned dst = (unsigned)__cvta_generic_to_shared(buf + lane * PITCH + aa);
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(dDg + (size_t)aa * DP + col) : "memory");
-        }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-}
-// make chunk c current (its copy was issued earlier) and start fetching chunk c + 1
-__device__ __noinline__ void advance_columns(float* chunk2, const float* dDg, int c, int nv, int DP) {
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();                       // chunk c landed for everyone; everyone is done with chunk c - 1
-    if ((c + 1) * CHUNK < DP) issue_columns(chunk2 + ((c + 1) & 1) * CHUNK * PITCH, dDg, c + 1, nv, DP);
-}
-__device__ __forceinline__ float get_column(float* chunk2, const float* isig_s, int at, int k, int& cur, const float* dDg,
-                                            int nv, int DP) {
-    const int c = k >> 5;
-    if (c != cur) { advance_columns(chunk2, dDg, c, nv, DP); cur = c; }
-    return chunk2[(c & 1) * CHUNK * PITCH + (k & (CHUNK - 1)) * PITCH + at] * isig_s[k];
-}
+// position of (p, q), p <= q, in the row-major upper triangle of a C x C matrix
+__device__ __forceinline__ int tri(int p, int q, int C) { return p * C - (p * (p - 1)) / 2 + (q - p); }
+__device__ __forceinline__ int tri_sym(int p, int q, int C) { return p <= q ? tri(p, q, C) : tri(q, p, C); }
 
 template <int C1, int C2, int L>
-struct Lay {                                  // shared-memory plan, in floats
+struct Plan {                                 // widths and the shared-memory plan, in rows of P floats
     static constexpr int K1 = C2, K2 = 2;
-    static constexpr int nZ1 = 3 * K1, nZ2 = 5 * K2;
+    static constexpr int nX1 = 3 * C1, nX2 = 5 * C2, nX3 = L >= 3 ? 7 : 0, nX = nX1 + nX2 + nX3;
+    static constexpr int nZ1 = 3 * K1, nZ2 = 5 * K2, nZ = nZ1 + nZ2;
+    static constexpr int nU = L >= 3 ? 3 * K2 : 0, nY = L >= 3 ? 5 : 0;          // forward intermediates
+    static constexpr int nPreF = nU + nY;
+    static constexpr int nW = nU, nZg = nY, nYQ = K2 * K1 * 3;                   // backward adds W, Zg, Q v
+    static constexpr int nPreB = nPreF + nW + nZg + nYQ;
+    static constexpr int nAux = 12;                                              // dot0, nine partial dots
     static constexpr int nMat = C1 * C1 + C2 * C2 + C1 * K1 + C2 * K2;
     static constexpr int nGaunt = L >= 3 ? 2 * (int)((sizeof(GauntSparse) + 3) / 4) : 0;
-    // work rows: per-atom scalars (1/M0, dot0), Z1, Z2 [, dXt1, dXt2, dX3, dZ1, dZ2]
-    static constexpr int nAux = 2;
-    static constexpr int work_fwd = nAux + nZ1 + nZ2;
-    static constexpr int work_bwd = nAux + nZ1 + nZ2 + 3 * C1 + 5 * C2 + 7 + nZ1 + nZ2;
-    // the tile holds the state row without its leading C0 scalar sums (those are handled by
-    // whole warps straight from global memory)
-    static int floats(int SP, int C0, int DP, bool bwd) {
-        return (SP - C0 + (bwd ? work_bwd + CHUNK : work_fwd) + CHUNK) * PITCH + nMat + nGaunt + (bwd ? DP : 0);
+    static constexpr int nMatP = (nMat + nGaunt + 3) / 4 * 4;                    // matrices come first: 16-byte rows
+    static int rows(int TW, int nDS, bool bwd) {
+        return TW + nX + nZ + nDS + (bwd ? nPreB + nX + nX3 + nZ + 18 + nAux : nPreF);
     }
+    static size_t bytes(int TW, int nDS, bool bwd) { return sizeof(float) * ((size_t)rows(TW, nDS, bwd) * P + nMatP); }
 };
 
-// Shared setup of both passes: stage matrices and the block's state slice, then per atom
-// normalise and align in place:  tile[offA1..] <- X1 (I + W1),  tile[offA2..] <- X2 (I + W2),
-// tile[offA3..] <- X3, and form the probes Z1, Z2 (each row by its owner lane) and Q.
+// Shared front of both passes: stage the small matrices and the block's slice of the state
+// array (everything behind the C0 scalar sums), then, one warp per harmonic row, normalise
+// and align it, XT = (X / M_1)(I + W), and project it on the probes, Z = XT A.
 template <int C1, int C2, int L>
 struct Front {
+    using PL = Plan<C1, C2, L>;
     static constexpr int K1 = C2, K2 = 2;
-    float* tile; float* mW1; float* mW2; float* mA1; float* mA2;
-    const GauntSparse* G123; const GauntSparse* G233;     // shared-memory copies of the sparse couplings
-    SCol T, Z1, Z2, AUX;         // T[k] = state entry C0 + k of this atom
-    double M0d, M1d;
-    float iM0, iM1;
-    float Q[K2][9];
-    int nv, b0, at, r;
+    float *ST, *XT, *ZZ;
+    float *mW1, *mW2, *mA1, *mA2;
+    const GauntSparse *G123, *G233;
+    int nv, b0, lane, warp, C0, TW, o1, o2, o3, oS;
+    float iM1;
+    double M1d;
 
-    __device__ __forceinline__ void setup(const InvArgs& a, float* sm, float* work, float* mats) {
+    template <int C, int K>
+    __device__ __forceinline__ void align_row(const float* xr, const float* W, const float* A, float* xt, float* z) const {
+        float rr[C];
+#pragma unroll
+        for (int b = 0; b < C; ++b) rr[b] = 0.f;
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            const float x = xr[c * P] * iM1;
+#pragma unroll
+            for (int b = 0; b < C; b += 4) {
+                const float4 w = *reinterpret_cast<const float4*>(W + c * C + b);
+                rr[b] += x * w.x; rr[b + 1] += x * w.y; rr[b + 2] += x * w.z; rr[b + 3] += x * w.w;
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < C; ++b) xt[b * P] = rr[b];
+#pragma unroll
+        for (int kk = 0; kk < K; ++kk) {
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < C; ++c) s += rr[c] * A[c * K + kk];
+            z[kk * P] = s;
+        }
+    }
+
+    __device__ __forceinline__ void setup(const InvArgs& a, float* st, float* xt, float* zz, float* mats) {
         const Dims& d = a.d;
         const int tid = threadIdx.x;
-        at = tid >> 2; r = tid & 3;
-        tile = sm;
+        lane = tid & 31; warp = tid >> 5;
+        ST = st; XT = xt; ZZ = zz;
         mW1 = mats; mW2 = mW1 + C1 * C1; mA1 = mW2 + C2 * C2; mA2 = mA1 + C1 * K1;
         for (int i = tid; i < C1 * C1; i += NT) mW1[i] = __ldg(a.m.W1p + i);
         for (int i = tid; i < C2 * C2; i += NT) mW2[i] = __ldg(a.m.W2p + i);
@@ -181,593 +157,675 @@ struct Front {
             G123 = reinterpret_cast<const GauntSparse*>(g1);
             G233 = reinterpret_cast<const GauntSparse*>(g2);
         }
-        b0 = blockIdx.x * ATOMS;
-        nv = a.n - b0 < ATOMS ? a.n - b0 : ATOMS;
-        const float* src = a.state + (size_t)b0 * d.SP;
-        const int C0 = d.C0, TW = d.SP - C0;     // tile rows per atom
-        const int total = ATOMS * TW;
-        constexpr int US = 5;                    // loads in flight per thread
-        for (int e0 = tid; e0 < total; e0 += US * NT) {
-            float v[US];
-            int slot[US];
+        b0 = blockIdx.x * AT;
+        nv = a.n - b0 < AT ? a.n - b0 : AT;
+        C0 = d.C0; TW = d.SP - C0;
+        o1 = d.offA[1] - C0; o2 = d.offA[2] - C0; o3 = d.offA[3] - C0; oS = d.S - C0;
+        // state slice: a warp reads 32 consecutive entries of one atom's row; four atoms'
+        // loads are issued before the first store
+        const float* src = a.state + (size_t)b0 * d.SP + C0;
+        for (int k0 = 0; k0 < TW; k0 += 32) {
+            const int k = k0 + lane;
+            float v[AT / NW];
 #pragma unroll
-            for (int u = 0; u < US; ++u) {
-                const int e = e0 + u * NT;
-                const int atom = e / TW, k = e - atom * TW;
-                slot[u] = e < total ? k * PITCH + atom : -1;
-                v[u] = (e < total && atom < nv) ? src[(size_t)atom * d.SP + C0 + k] : 0.f;
+            for (int i = 0; i < AT / NW; ++i) {
+                const int aa = warp + i * NW;
+                v[i] = (k < TW && aa < nv) ? src[(size_t)aa * d.SP + k] : 0.f;
             }
+            if (k < TW) {
 #pragma unroll
-            for (int u = 0; u < US; ++u)
-                if (slot[u] >= 0) tile[slot[u]] = v[u];
+                for (int i = 0; i < AT / NW; ++i) ST[k * P + warp + i * NW] = v[i];
+            }
         }
         __syncthreads();
-        T.p = tile + at;
-        AUX.p = work + at;
-        Z1.p = work + 2 * PITCH + at;
-        Z2.p = work + (2 + 3 * K1) * PITCH + at;
-        const int oS = d.S - C0;
-        M0d = sqrt(0.25 + (double)T[oS] + (double)T[oS + 2]);
-        M1d = sqrt(0.25 + (double)T[oS + 1] + (double)T[oS + 3]);
-        iM0 = (float)(1.0 / M0d); iM1 = (float)(1.0 / M1d);
-        if (r == 0) AUX[0] = iM0;
-        const int o1 = d.offA[1] - C0, o2 = d.offA[2] - C0, o3 = d.offA[3] - C0;
+        M1d = sqrt(0.25 + (double)ST[(oS + 1) * P + lane] + (double)ST[(oS + 3) * P + lane]);
+        iM1 = (float)(1.0 / M1d);
+        for (int u = warp; u < 9; u += NW) {
+            if (u < 3) align_row<C1, K1>(ST + (o1 + u * C1) * P + lane, mW1, mA1, XT + u * C1 * P + lane, ZZ + u * K1 * P + lane);
+            else if (u < 8)
+                align_row<C2, K2>(ST + (o2 + (u - 3) * C2) * P + lane, mW2, mA2, XT + (PL::nX1 + (u - 3) * C2) * P + lane,
+                                  ZZ + (PL::nZ1 + (u - 3) * K2) * P + lane);
+            else if (L >= 3) {
 #pragma unroll
-        for (int mm = 0; mm < 3; ++mm) {
-            if (own1(mm) != r) continue;
-            float x[C1], rr[C1];
-#pragma unroll
-            for (int c = 0; c < C1; ++c) { x[c] = T[o1 + mm * C1 + c] * iM1; rr[c] = 0.f; }
-#pragma unroll
-            for (int c = 0; c < C1; ++c)
-#pragma unroll
-                for (int b = 0; b < C1; ++b) rr[b] += x[c] * mW1[c * C1 + b];
-#pragma unroll
-            for (int b = 0; b < C1; ++b) T[o1 + mm * C1 + b] = rr[b];
-#pragma unroll
-            for (int kk = 0; kk < K1; ++kk) {
-                float s = 0.f;
-#pragma unroll
-                for (int c = 0; c < C1; ++c) s += rr[c] * mA1[c * K1 + kk];
-                Z1[mm * K1 + kk] = s;
+                for (int mm = 0; mm < 7; ++mm) XT[(PL::nX1 + PL::nX2 + mm) * P + lane] = ST[(o3 + mm) * P + lane] * iM1;
             }
         }
-#pragma unroll
-        for (int mm = 0; mm < 5; ++mm) {
-            if (own2(mm) != r) continue;
-            float x[C2], rr[C2];
-#pragma unroll
-            for (int c = 0; c < C2; ++c) { x[c] = T[o2 + mm * C2 + c] * iM1; rr[c] = 0.f; }
-#pragma unroll
-            for (int c = 0; c < C2; ++c)
-#pragma unroll
-                for (int b = 0; b < C2; ++b) rr[b] += x[c] * mW2[c * C2 + b];
-#pragma unroll
-            for (int b = 0; b < C2; ++b) T[o2 + mm * C2 + b] = rr[b];
-#pragma unroll
-            for (int kk = 0; kk < K2; ++kk) {
-                float s = 0.f;
-#pragma unroll
-                for (int c = 0; c < C2; ++c) s += rr[c] * mA2[c * K2 + kk];
-                Z2[mm * K2 + kk] = s;
+        __syncthreads();
+    }
+    // 1 / M_0 of atom aa (the same value in every lane)
+    __device__ __forceinline__ double M0_of(int aa) const {
+        return sqrt(0.25 + (double)ST[oS * P + aa] + (double)ST[(oS + 2) * P + aa]);
+    }
+    // U[m1][e] and Y[m1] of the sparse couplings, one unit per m1
+    __device__ __forceinline__ void gaunt_pre(float* PRE, int& uctr) const {
+        if (L < 3) return;
+        const float* Z2 = ZZ + PL::nZ1 * P + lane;
+        const float* X3 = XT + (PL::nX1 + PL::nX2) * P + lane;
+        for (int m1 = 0; m1 < 3; ++m1) {
+            if ((uctr++ % NW) != warp) continue;
+            float u0 = 0.f, u1 = 0.f;
+            const int nn = G123->n;
+            for (int n = 0; n < nn; ++n) {
+                if (G123->m1[n] != m1) continue;
+                const float t = G123->v[n] * X3[G123->m3[n] * P];
+                u0 += t * Z2[(G123->m2[n] * K2) * P];
+                u1 += t * Z2[(G123->m2[n] * K2 + 1) * P];
             }
+            PRE[(m1 * K2) * P + lane] = u0;
+            PRE[(m1 * K2 + 1) * P + lane] = u1;
         }
-        if (L >= 3) {
-#pragma unroll
-            for (int mm = 0; mm < 7; ++mm)
-                if (own3(mm) == r) T[o3 + mm] = T[o3 + mm] * iM1;
+        for (int m1 = 0; m1 < 5; ++m1) {
+            if ((uctr++ % NW) != warp) continue;
+            float y = 0.f;
+            const int nn = G233->n;
+            for (int n = 0; n < nn; ++n) {
+                if (G233->m1[n] != m1) continue;
+                y += G233->v[n] * X3[G233->m2[n] * P] * X3[G233->m3[n] * P];
+            }
+            PRE[(PL::nU + m1) * P + lane] = y;
         }
-        __syncthreads();                         // rows, probes and 1/M0 visible to the whole block
-#pragma unroll
-        for (int e = 0; e < K2; ++e) stf9(Z2[e], Z2[K2 + e], Z2[2 * K2 + e], Z2[3 * K2 + e], Z2[4 * K2 + e], Q[e]);
     }
 };
 
 template <int C1, int C2, int L>
-__global__ void __launch_bounds__(NT, 2) k_inv_forward(const InvArgs a) {
+__global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
+    using PL = Plan<C1, C2, L>;
     constexpr int K1 = C2, K2 = 2;
-    using LY = Lay<C1, C2, L>;
     extern __shared__ float sm[];
     const Dims& d = a.d;
     const ModelDev& m = a.m;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float* work = sm + (d.SP - d.C0) * PITCH;
-    float* chunk = work + LY::work_fwd * PITCH;
-    float* mats = chunk + CHUNK * PITCH;
+    const int C0 = d.C0, TW = d.SP - C0;
+    const int c_full = (2 * C0 / 32) * 32;         // columns [0, c_full) go straight from global to global
+    const int nDS = d.DP - c_full;
+    float* mats = sm;
+    float* ST = sm + PL::nMatP;
+    float* XT = ST + TW * P;
+    float* ZZ = XT + PL::nX * P;
+    float* PRE = ZZ + PL::nZ * P;
+    float* DS = PRE + PL::nPreF * P;               // feature columns [c_full, DP), [column][atom]
     Front<C1, C2, L> f;
-    f.setup(a, sm, work, mats);
-    const SCol T = f.T, Z1 = f.Z1, Z2 = f.Z2;
-    const int nv = f.nv, b0 = f.b0, C0 = d.C0, at = f.at, r = f.r;
+    f.setup(a, ST, XT, ZZ, mats);
+    const int lane = f.lane, warp = f.warp, nv = f.nv, b0 = f.b0;
     float* Dg = a.desc + (size_t)b0 * d.DP;
-    const int ty = a.type_s[a.a0 + (b0 + at < a.n ? b0 + at : a.n - 1)];
+    int uctr = 0;
+#define TAKE() ((uctr++ % NW) == warp)
+#define DSK(k) DS[((k) - c_full) * P + lane]
 
-    // Feature-vector columns are produced in increasing order, dealt round-robin to the
-    // atom's four lanes; every 32nd column flushes the staging buffer.  The calibration
-    // (v - mu) / sigma is applied by the flushing lane, which owns one column; the two
-    // normalising scales arrive already calibrated (formed in double precision).
+    f.gaunt_pre(PRE, uctr);
+
+    // Columns [0, c_full): the centre's initial features (a gather by species) and the
+    // normalised scalar sums A_0 / M_0.  A warp takes one atom at a time, lane = column.
+    {
+        const float* st_g = a.state + (size_t)b0 * d.SP;
+        float im0[AT / NW];
+        int ty[AT / NW];
+#pragma unroll
+        for (int i = 0; i < AT / NW; ++i) {
+            const int aa = warp + i * NW;
+            im0[i] = (float)(1.0 / f.M0_of(aa));
+            ty[i] = aa < nv ? a.type_s[a.a0 + b0 + aa] : 0;
+        }
+        for (int cb = 0; cb < c_full; cb += 64) {
+            float v[2][AT / NW];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int col = cb + 32 * h + lane;
+#pragma unroll
+                for (int i = 0; i < AT / NW; ++i) {
+                    const int aa = warp + i * NW;
+                    v[h][i] = 0.f;
+                    if (aa < nv && col < c_full) {
+                        if (col < C0) v[h][i] = __ldg(m.X0 + ty[i] * C0 + col);
+                        else v[h][i] = st_g[(size_t)aa * d.SP + (col - C0)] * im0[i];
+                    }
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int col = cb + 32 * h + lane;
+                if (col >= c_full) continue;
+                const float mu_c = __ldg(m.mu + col), is_c = __ldg(m.inv_sigma + col);
+#pragma unroll
+                for (int i = 0; i < AT / NW; ++i) {
+                    const int aa = warp + i * NW;
+                    if (aa < nv) Dg[(size_t)aa * d.DP + col] = (v[h][i] - mu_c) * is_c;
+                }
+            }
+        }
+    }
+    __syncthreads();                               // U, Y visible
+
+    // ---- the remaining columns, by units dealt to the warps; lane = atom -------------
+    const float* X1 = XT + lane;                               // [mm * C1 + c]
+    const float* X2 = XT + PL::nX1 * P + lane;                 // [mm * C2 + c]
+    const float* X3 = XT + (PL::nX1 + PL::nX2) * P + lane;     // [mm]
+    const float* Z1 = ZZ + lane;                               // [mm * K1 + k]
+    const float* Z2 = ZZ + PL::nZ1 * P + lane;                 // [mm * K2 + e]
+    float Q[K2][9];
+#pragma unroll
+    for (int e = 0; e < K2; ++e) stf9(Z2[e * P], Z2[(K2 + e) * P], Z2[(2 * K2 + e) * P], Z2[(3 * K2 + e) * P], Z2[(4 * K2 + e) * P], Q[e]);
+
     const int kM0 = 2 * C0, kM1 = 2 * C0 + 1;
-    int oc = 0;                                               // running output counter
-#define mine() (((oc++) & 3) == r)
-    const float* mu_g = m.mu;
-    const float* is_g = m.inv_sigma;
-    const int DPv = d.DP, Dov = d.D_out;
-#define put(k, v, own) put_column(chunk, at, (k), (v), (own), Dg, mu_g, is_g, nv, DPv, Dov, kM0, kM1)
-
-    // The first 2*C0 columns are plain per-column work -- the centre's initial features (a
-    // gather by species) and the normalised scalar sums A_0 / M_0 -- so whole warps write
-    // them straight from global memory, lane = column, for every complete group of 32
-    // columns; a trailing partial group (only for C0 = 8) goes through the stream.
-    const float* st_g = a.state + (size_t)b0 * d.SP;
-    const int c_full = (2 * C0 / CHUNK) * CHUNK;
-    for (int cb = 0; cb < c_full; cb += CHUNK) {
-        const int col = cb + lane;
-        const float mu_c = __ldg(m.mu + col), is_c = __ldg(m.inv_sigma + col);
-        constexpr int UA = 8;
-        float v[UA];
-#pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const int aa = warp + u * (NT / 32);
-            v[u] = 0.f;
-            if (aa < nv) {
-                if (col < C0) v[u] = __ldg(m.X0 + a.type_s[a.a0 + b0 + aa] * C0 + col);
-                else v[u] = st_g[(size_t)aa * d.SP + (col - C0)];
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < UA; ++u) {
-            const int aa = warp + u * (NT / 32);
-            if (aa < nv) {
-                const float x = col < C0 ? v[u] : v[u] * f.AUX.p[aa - at];
-                Dg[(size_t)aa * d.DP + col] = (x - mu_c) * is_c;
-            }
-        }
-    }
+    // columns of a trailing partial group of 32 (only for C0 = 8)
     for (int c = c_full; c < 2 * C0; ++c) {
-        const bool own = mine();
+        if (!TAKE()) continue;
         float v = 0.f;
-        if (own && at < nv) v = c < C0 ? __ldg(m.X0 + ty * C0 + c) : st_g[(size_t)at * d.SP + (c - C0)] * f.iM0;
-        put(c, v, own);
+        if (lane < nv) {
+            if (c < C0) v = __ldg(m.X0 + a.type_s[a.a0 + b0 + lane] * C0 + c);
+            else v = a.state[(size_t)(b0 + lane) * d.SP + (c - C0)] * (float)(1.0 / f.M0_of(lane));
+        }
+        DSK(c) = v;
     }
-    put(kM0, (float)((f.M0d - (double)__ldg(m.mu + kM0)) * (double)__ldg(m.inv_sigma + kM0)), r == 0);
-    put(kM1, (float)((f.M1d - (double)__ldg(m.mu + kM1)) * (double)__ldg(m.inv_sigma + kM1)), r == 0);
-    const int o1 = d.offA[1] - C0, o2 = d.offA[2] - C0, o3 = d.offA[3] - C0;
-    {   // Gram blocks, row-major upper triangle, strict off-diagonals times sqrt 2
-        int k = d.oG[1];
-        for (int p = 0; p < C1; ++p)
-            for (int q = p; q < C1; ++q) {
-                const bool own = mine();
-                float s = 0.f;
-                if (own) {
-#pragma unroll
-                    for (int mm = 0; mm < 3; ++mm) s += T[o1 + mm * C1 + p] * T[o1 + mm * C1 + q];
-                }
-                put(k++, p == q ? s : kR2 * s, own);
+    if (TAKE()) {   // the two normalising scales, calibrated here in double precision
+        const double M0d = f.M0_of(lane);
+        DSK(kM0) = (float)((M0d - (double)__ldg(m.mu + kM0)) * (double)__ldg(m.inv_sigma + kM0));
+        DSK(kM1) = (float)((f.M1d - (double)__ldg(m.mu + kM1)) * (double)__ldg(m.inv_sigma + kM1));
+        for (int k = d.D_out; k < d.DP; ++k) DSK(k) = 0.f;
+    }
+    // Gram blocks, row-major upper triangle, strict off-diagonals times sqrt 2; a unit is
+    // rows u and C-1-u, which together hold C+1 entries
+    for (int u = 0; u < C1 / 2; ++u) {
+        if (!TAKE()) continue;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+            const int p = h ? C1 - 1 - u : u;
+            const float x0 = X1[p * P], x1 = X1[(C1 + p) * P], x2 = X1[(2 * C1 + p) * P];
+            int k = d.oG[1] + tri(p, p, C1);
+            DSK(k) = x0 * x0 + x1 * x1 + x2 * x2;
+            for (int q = p + 1; q < C1; ++q) {
+                ++k;
+                DSK(k) = kR2 * (x0 * X1[q * P] + x1 * X1[(C1 + q) * P] + x2 * X1[(2 * C1 + q) * P]);
             }
-        for (int p = 0; p < C2; ++p)
-            for (int q = p; q < C2; ++q) {
-                const bool own = mine();
-                float s = 0.f;
-                if (own) {
-#pragma unroll
-                    for (int mm = 0; mm < 5; ++mm) s += T[o2 + mm * C2 + p] * T[o2 + mm * C2 + q];
-                }
-                put(k++, p == q ? s : kR2 * s, own);
-            }
-        if (L >= 3) {
-            const bool own = mine();
-            float s = 0.f;
-            if (own) {
-#pragma unroll
-                for (int mm = 0; mm < 7; ++mm) s += T[o3 + mm] * T[o3 + mm];
-            }
-            put(k++, s, own);
         }
     }
-    {   // (1,1,2): -(1/sqrt5) v_k1^T Q_eta v_k2, k1 <= k2
-        int k = d.oJ112;
-        for (int k1 = 0; k1 < K1; ++k1)
+    for (int u = 0; u < C2 / 2; ++u) {
+        if (!TAKE()) continue;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+            const int p = h ? C2 - 1 - u : u;
+            float x[5];
+#pragma unroll
+            for (int mm = 0; mm < 5; ++mm) x[mm] = X2[(mm * C2 + p) * P];
+            int k = d.oG[2] + tri(p, p, C2);
+            for (int q = p; q < C2; ++q) {
+                float s = 0.f;
+#pragma unroll
+                for (int mm = 0; mm < 5; ++mm) s += x[mm] * X2[(mm * C2 + q) * P];
+                DSK(k) = q == p ? s : kR2 * s;
+                ++k;
+            }
+        }
+    }
+    if (L >= 3) {
+        if (TAKE()) {
+            float s = 0.f;
+#pragma unroll
+            for (int mm = 0; mm < 7; ++mm) s += X3[mm * P] * X3[mm * P];
+            DSK(d.oG[3]) = s;
+        }
+    }
+    // (1,1,2): -(1/sqrt5) v_k1^T Q_eta v_k2, k1 <= k2; a unit is rows u and K1-1-u
+    for (int u = 0; u < (K1 + 1) / 2; ++u) {
+        if (!TAKE()) continue;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+            const int k1 = h ? K1 - 1 - u : u;
+            if (h && k1 == u) break;
+            const float a0 = Z1[k1 * P], a1 = Z1[(K1 + k1) * P], a2 = Z1[(2 * K1 + k1) * P];
+            int k = d.oJ112 + tri(k1, k1, K1) * K2;
             for (int k2 = k1; k2 < K1; ++k2) {
+                const float b0v = Z1[k2 * P], b1v = Z1[(K1 + k2) * P], b2v = Z1[(2 * K1 + k2) * P];
+                const float w = kC112 * (k1 == k2 ? 1.0f : kR2);
 #pragma unroll
                 for (int e = 0; e < K2; ++e) {
-                    const bool own = mine();
-                    float val = 0.f;
-                    if (own) {
-                        float y[3];
-                        matvec3(f.Q[e], Z1[k2], Z1[K1 + k2], Z1[2 * K1 + k2], y);
-                        val = kC112 * (k1 == k2 ? 1.0f : kR2) * (Z1[k1] * y[0] + Z1[K1 + k1] * y[1] + Z1[2 * K1 + k1] * y[2]);
-                    }
-                    put(k++, val, own);
+                    float y[3];
+                    matvec3(Q[e], b0v, b1v, b2v, y);
+                    DSK(k) = w * (a0 * y[0] + a1 * y[1] + a2 * y[2]);
+                    ++k;
                 }
             }
+        }
     }
-    if (L >= 3) {   // (1,2,3): sparse Gaunt contraction
-        const GauntSparse* G = f.G123;
-        const int nn = G->n;
-        int k = d.oJ123;
-        for (int k1 = 0; k1 < K1; ++k1)
+    if (L >= 3) {   // (1,2,3) and (2,3,3) from the intermediates
+        for (int e = 0; e < K2; ++e) {
+            if (!TAKE()) continue;
+            const float u0 = PRE[(0 * K2 + e) * P + lane], u1 = PRE[(1 * K2 + e) * P + lane], u2 = PRE[(2 * K2 + e) * P + lane];
+            for (int k1 = 0; k1 < K1; ++k1)
+                DSK(d.oJ123 + k1 * K2 + e) = Z1[k1 * P] * u0 + Z1[(K1 + k1) * P] * u1 + Z1[(2 * K1 + k1) * P] * u2;
+        }
+        if (TAKE()) {
+#pragma unroll
             for (int e = 0; e < K2; ++e) {
-                const bool own = mine();
                 float s = 0.f;
-                if (own)
-                    for (int n = 0; n < nn; ++n)
-                        s += G->v[n] * Z1[G->m1[n] * K1 + k1] * Z2[G->m2[n] * K2 + e] * T[o3 + G->m3[n]];
-                put(k++, s, own);
+#pragma unroll
+                for (int m1 = 0; m1 < 5; ++m1) s += Z2[(m1 * K2 + e) * P] * PRE[(PL::nU + m1) * P + lane];
+                DSK(d.oJ233 + e) = s;
             }
+        }
     }
-    {   // (2,2,2): -sqrt(12/35) tr(Q Q Q), non-decreasing index triples
+    if (TAKE()) {   // (2,2,2): -sqrt(12/35) tr(Q Q Q), non-decreasing index triples
         int k = d.oJ222;
 #pragma unroll
         for (int e1 = 0; e1 < K2; ++e1)
 #pragma unroll
             for (int e2 = e1; e2 < K2; ++e2) {
-                float P[9];
-                matmul3(f.Q[e1], f.Q[e2], P);
+                float Pm[9];
+                matmul3(Q[e1], Q[e2], Pm);
 #pragma unroll
                 for (int e3 = e2; e3 < K2; ++e3) {
-                    const bool own = mine();
-                    put(k++, kC222 * fam3(e1, e2, e3) * trace_prod(P, f.Q[e3]), own);
+                    DSK(k) = kC222 * fam3(e1, e2, e3) * trace_prod(Pm, Q[e3]);
+                    ++k;
                 }
             }
     }
-    if (L >= 3) {   // (2,3,3)
-        const GauntSparse* G = f.G233;
-        const int nn = G->n;
-        int k = d.oJ233;
-        for (int e = 0; e < K2; ++e) {
-            const bool own = mine();
-            float s = 0.f;
-            if (own)
-                for (int n = 0; n < nn; ++n) s += G->v[n] * Z2[G->m1[n] * K2 + e] * T[o3 + G->m2[n]] * T[o3 + G->m3[n]];
-            put(k++, s, own);
+#pragma unroll
+    for (int e = 0; e < K2; ++e) {   // projected quartic |Q_eta v_k|^2, eta-major
+        if (!TAKE()) continue;
+        for (int k1 = 0; k1 < K1; ++k1) {
+            float y[3];
+            matvec3(Q[e], Z1[k1 * P], Z1[(K1 + k1) * P], Z1[(2 * K1 + k1) * P], y);
+            DSK(d.oPi + e * K1 + k1) = y[0] * y[0] + y[1] * y[1] + y[2] * y[2];
         }
     }
-    {   // projected quartic |Q_eta v_k|^2, eta-major
-        int k = d.oPi;
+    __syncthreads();
+
+    // ---- calibrate and write out, lane = column ----------------------------------------
+    for (int cb = c_full; cb < d.DP; cb += 32) {
+        const int col = cb + lane;
+        float mu_c = 0.f, is_c = 1.f;
+        if (col < d.D_out && col != kM0 && col != kM1) { mu_c = __ldg(m.mu + col); is_c = __ldg(m.inv_sigma + col); }
 #pragma unroll
-        for (int e = 0; e < K2; ++e)
-            for (int k1 = 0; k1 < K1; ++k1) {
-                const bool own = mine();
-                float val = 0.f;
-                if (own) {
-                    float y[3];
-                    matvec3(f.Q[e], Z1[k1], Z1[K1 + k1], Z1[2 * K1 + k1], y);
-                    val = y[0] * y[0] + y[1] * y[1] + y[2] * y[2];
-                }
-                put(k++, val, own);
-            }
+        for (int i = 0; i < AT / NW; ++i) {
+            const int aa = warp + i * NW;
+            if (aa < nv) Dg[(size_t)aa * d.DP + col] = (DS[(col - c_full) * P + aa] - mu_c) * is_c;
+        }
     }
-    for (int k = d.D_out; k < d.DP; ++k) put(k, 0.f, r == 0);    // DP is a multiple of 32: ends on a flush
-#undef put
-#undef mine
+#undef TAKE
+#undef DSK
+}
+
+// transpose of the alignment and probe maps for one harmonic row: g = dXt + dZ A^T,
+// dX = g (I + W)^T / M_1; returns the row's share of sum g . Xt
+template <int C, int K>
+__device__ __forceinline__ float back_row(const float* dxt, const float* dz, const float* A, const float* W,
+                                          const float* xt, float* out, float iM1) {
+    float zz[K], g[C];
+#pragma unroll
+    for (int kk = 0; kk < K; ++kk) zz[kk] = dz[kk * P];
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        float s = dxt[c * P];
+#pragma unroll
+        for (int kk = 0; kk < K; ++kk) s += zz[kk] * A[c * K + kk];
+        g[c] = s;
+        dot += s * xt[c * P];
+    }
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        float s = 0.f;
+#pragma unroll
+        for (int b = 0; b < C; b += 4) {
+            const float4 w = *reinterpret_cast<const float4*>(W + c * C + b);
+            s += g[b] * w.x + g[b + 1] * w.y + g[b + 2] * w.z + g[b + 3] * w.w;
+        }
+        out[c * P] = s * iM1;
+    }
+    return dot;
 }
 
 template <int C1, int C2, int L>
-__global__ void __launch_bounds__(NT, 2) k_inv_backward(const InvArgs a) {
+__global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
+    using PL = Plan<C1, C2, L>;
     constexpr int K1 = C2, K2 = 2;
-    using LY = Lay<C1, C2, L>;
     extern __shared__ float sm[];
     const Dims& d = a.d;
     const ModelDev& m = a.m;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float* work = sm + (d.SP - d.C0) * PITCH;
-    float* chunk = work + LY::work_bwd * PITCH;            // two staging buffers of 32 columns
-    float* mats = chunk + 2 * CHUNK * PITCH;
-    float* isig_s = mats + LY::nMat + LY::nGaunt;          // 1 / sigma per column (0 beyond D_out)
-    for (int k = threadIdx.x; k < d.DP; k += NT) isig_s[k] = k < d.D_out ? __ldg(a.m.inv_sigma + k) : 0.f;
-    // start fetching the first streamed chunk (the one that holds column 2*C0) right away
-    issue_columns(chunk + (((2 * d.C0) >> 5) & 1) * CHUNK * PITCH, a.desc + (size_t)blockIdx.x * ATOMS * d.DP, (2 * d.C0) >> 5,
-                  a.n - (int)blockIdx.x * ATOMS < ATOMS ? a.n - (int)blockIdx.x * ATOMS : ATOMS, d.DP);
-    Front<C1, C2, L> f;
-    f.setup(a, sm, work, mats);
-    const SCol T = f.T, Z1 = f.Z1, Z2 = f.Z2;
-    const int nv = f.nv, b0 = f.b0, C0 = d.C0, at = f.at, r = f.r;
+    const int C0 = d.C0, TW = d.SP - C0;
+    const int c_full = (2 * C0 / 32) * 32;
+    const int nDS = d.DP - c_full;
+    float* mats = sm;
+    float* ST = sm + PL::nMatP;
+    float* XT = ST + TW * P;
+    float* ZZ = XT + PL::nX * P;
+    float* DS = ZZ + PL::nZ * P;                   // dE/dD / sigma, columns [c_full, DP), [column][atom]
+    float* PRE = DS + nDS * P;                     // U, Y, W, Zg, Q v
+    float* GX = PRE + PL::nPreB * P;               // dE/dXt (degree-3 rows twice: the two couplings' shares)
+    float* DZ = GX + (PL::nX + PL::nX3) * P;
+    float* DQ = DZ + PL::nZ * P;
+    float* AUX = DQ + 18 * P;                      // row 0: sum_c X_0 dE/dX_0; rows 1..9: partial dots
+    float* Ws = PRE + PL::nPreF * P;               // [m1 * K2 + e]
+    float* Zg = Ws + PL::nW * P;                   // [m1]
+    float* YQ = Zg + PL::nZg * P;                  // [(e * K1 + k) * 3 + m]
+    const int b0 = blockIdx.x * AT;
     const float* dDg = a.desc + (size_t)b0 * d.DP;
-    float* wp = work + (LY::nAux + LY::nZ1 + LY::nZ2) * PITCH + at;
-    const SCol dXt1{wp}, dXt2{wp + 3 * C1 * PITCH}, dX3{wp + (3 * C1 + 5 * C2) * PITCH},
-        dZ1{wp + (3 * C1 + 5 * C2 + 7) * PITCH}, dZ2{wp + (3 * C1 + 5 * C2 + 7 + LY::nZ1) * PITCH},
-        dQs{chunk + at};          // the staging buffer is free once the last column has been consumed
-    // each lane clears the accumulators it owns
+    {   // stage the gradient rows, lane = column, divided by sigma (zero beyond D_out)
+        const int ln = threadIdx.x & 31, wp = threadIdx.x >> 5;
+        const int nv0 = a.n - b0 < AT ? a.n - b0 : AT;
+        for (int cb = c_full; cb < d.DP; cb += 64) {
+            float v[2][AT / NW];
 #pragma unroll
-    for (int mm = 0; mm < 3; ++mm)
-        if (own1(mm) == r) {
-            for (int k = 0; k < C1; ++k) dXt1[mm * C1 + k] = 0.f;
-            for (int k = 0; k < K1; ++k) dZ1[mm * K1 + k] = 0.f;
+            for (int h = 0; h < 2; ++h) {
+                const int col = cb + 32 * h + ln;
+#pragma unroll
+                for (int i = 0; i < AT / NW; ++i) {
+                    const int aa = wp + i * NW;
+                    v[h][i] = (col < d.DP && aa < nv0) ? dDg[(size_t)aa * d.DP + col] : 0.f;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int col = cb + 32 * h + ln;
+                if (col >= d.DP) continue;
+                const float is_c = col < d.D_out ? __ldg(m.inv_sigma + col) : 0.f;
+#pragma unroll
+                for (int i = 0; i < AT / NW; ++i) DS[(col - c_full) * P + wp + i * NW] = v[h][i] * is_c;
+            }
         }
+    }
+    Front<C1, C2, L> f;
+    f.setup(a, ST, XT, ZZ, mats);                  // its barriers also publish DS
+    const int lane = f.lane, warp = f.warp, nv = f.nv;
+    int uctr = 0;
+#define TAKE() ((uctr++ % NW) == warp)
+#define DSK(k) DS[((k) - c_full) * P + lane]
+
+    const float* X1 = XT + lane;
+    const float* X2 = XT + PL::nX1 * P + lane;
+    const float* X3 = XT + (PL::nX1 + PL::nX2) * P + lane;
+    const float* Z1 = ZZ + lane;
+    const float* Z2 = ZZ + PL::nZ1 * P + lane;
+    float Q[K2][9];
 #pragma unroll
-    for (int mm = 0; mm < 5; ++mm)
-        if (own2(mm) == r) {
-            for (int k = 0; k < C2; ++k) dXt2[mm * C2 + k] = 0.f;
-            for (int k = 0; k < K2; ++k) dZ2[mm * K2 + k] = 0.f;
+    for (int e = 0; e < K2; ++e) stf9(Z2[e * P], Z2[(K2 + e) * P], Z2[(2 * K2 + e) * P], Z2[(3 * K2 + e) * P], Z2[(4 * K2 + e) * P], Q[e]);
+
+    // ---- intermediates --------------------------------------------------------------
+    f.gaunt_pre(PRE, uctr);
+    if (L >= 3) {
+        for (int m1 = 0; m1 < 3; ++m1) {           // W[m1][e] = sum_k g123[k][e] Z1[m1][k]
+            if (!TAKE()) continue;
+            float w0 = 0.f, w1 = 0.f;
+            for (int k1 = 0; k1 < K1; ++k1) {
+                const float z = Z1[(m1 * K1 + k1) * P];
+                w0 += DSK(d.oJ123 + k1 * K2) * z;
+                w1 += DSK(d.oJ123 + k1 * K2 + 1) * z;
+            }
+            Ws[(m1 * K2) * P + lane] = w0;
+            Ws[(m1 * K2 + 1) * P + lane] = w1;
         }
+        if (TAKE()) {                              // Zg[m1] = sum_e g233[e] Z2[m1][e]
+            const float g0 = DSK(d.oJ233), g1 = DSK(d.oJ233 + 1);
 #pragma unroll
-    for (int mm = 0; mm < 7; ++mm)
-        if (own3(mm) == r) dX3[mm] = 0.f;
-    // gradient of the two matrices Q: lane i < 3 accumulates row i of both in registers
-    float dQ[K2][3];
+            for (int m1 = 0; m1 < 5; ++m1) Zg[m1 * P + lane] = g0 * Z2[(m1 * K2) * P] + g1 * Z2[(m1 * K2 + 1) * P];
+        }
+    }
 #pragma unroll
-    for (int e = 0; e < K2; ++e) { dQ[e][0] = 0.f; dQ[e][1] = 0.f; dQ[e][2] = 0.f; }
-
-    // dE/dD columns are consumed in increasing order, 32 at a time, already divided by sigma
-    int cur = -1;
-    const int DPv = d.DP;
-#define get(k) get_column(chunk, isig_s, at, (k), cur, dDg, nv, DPv)
-
-    const int o1 = d.offA[1] - C0, o2 = d.offA[2] - C0, o3 = d.offA[3] - C0;
-    // scalar block, X_0 = A_0 / M_0: whole warps, lane = channel, straight from / to global
-    // memory; the per-atom sum over channels of X_0 dE/dX_0 lands in the second scalar row
+    for (int e = 0; e < K2; ++e) {                 // Q_e v_k for every probe
+        if (!TAKE()) continue;
+        for (int k1 = 0; k1 < K1; ++k1) {
+            float y[3];
+            matvec3(Q[e], Z1[k1 * P], Z1[(K1 + k1) * P], Z1[(2 * K1 + k1) * P], y);
+            YQ[((e * K1 + k1) * 3 + 0) * P + lane] = y[0];
+            YQ[((e * K1 + k1) * 3 + 1) * P + lane] = y[1];
+            YQ[((e * K1 + k1) * 3 + 2) * P + lane] = y[2];
+        }
+    }
+    // scalar block, X_0 = A_0 / M_0: a warp takes its four atoms, lane = channel, straight
+    // from / to global memory; sum_c X_0 dE/dX_0 of each atom lands in the first scratch row
     {
         float* __restrict__ st_g = a.state + (size_t)b0 * d.SP;
         const float* __restrict__ dd_g = dDg;
-        constexpr int UA = 4;                           // atoms per batch: 4 x C0/32 x 2 loads in flight
+        constexpr int UA = AT / NW;
         float isg[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) isg[j] = lane + 32 * j < C0 ? __ldg(m.inv_sigma + C0 + lane + 32 * j) : 0.f;
-        for (int aa0 = warp; aa0 < nv; aa0 += UA * (NT / 32)) {
-            float dx[UA][4], a0v[UA][4];
+        float dx[UA][4], a0v[UA][4];
 #pragma unroll
-            for (int u = 0; u < UA; ++u) {
-                const int aa = aa0 + u * (NT / 32);
+        for (int u = 0; u < UA; ++u) {
+            const int aa = warp + u * NW;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int c = lane + 32 * j;
-                    const bool ok = aa < nv && c < C0;
-                    dx[u][j] = ok ? dd_g[(size_t)aa * d.DP + C0 + c] : 0.f;
-                    a0v[u][j] = ok ? st_g[(size_t)aa * d.SP + c] : 0.f;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < UA; ++u) {
-                const int aa = aa0 + u * (NT / 32);
-                if (aa >= nv) continue;
-                const float im0 = f.AUX.p[aa - at];
-                float part = 0.f;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int c = lane + 32 * j;
-                    const float dxs = dx[u][j] * isg[j];
-                    part += a0v[u][j] * im0 * dxs;
-                    if (c < C0) st_g[(size_t)aa * d.SP + c] = dxs * im0;
-                }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
-                if (lane == 0) f.AUX.p[PITCH + aa - at] = part;
+            for (int j = 0; j < 4; ++j) {
+                const int c = lane + 32 * j;
+                const bool ok = aa < nv && c < C0;
+                dx[u][j] = ok ? dd_g[(size_t)aa * d.DP + C0 + c] : 0.f;
+                a0v[u][j] = ok ? st_g[(size_t)aa * d.SP + c] : 0.f;
             }
         }
-        __syncthreads();
-    }
-    const float dot0 = f.AUX[1];
-    const float dM0 = get(2 * C0), dM1 = get(2 * C0 + 1);
-    {   // Gram: every lane walks all pairs and updates the rows it owns
-        int k = d.oG[1];
-        for (int p = 0; p < C1; ++p)
-            for (int q = p; q < C1; ++q) {
-                const float g = get(k++) * (p == q ? 1.0f : kR2);
-                if (r < 3) {
-                    const int mm = r;
-                    const float xp = T[o1 + mm * C1 + p], xq = T[o1 + mm * C1 + q];
-                    dXt1[mm * C1 + p] += g * xq;
-                    dXt1[mm * C1 + q] += g * xp;
-                }
+#pragma unroll
+        for (int u = 0; u < UA; ++u) {
+            const int aa = warp + u * NW;
+            const float im0 = (float)(1.0 / f.M0_of(aa));
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int c = lane + 32 * j;
+                const float dxs = dx[u][j] * isg[j];
+                part += a0v[u][j] * im0 * dxs;
+                if (aa < nv && c < C0) st_g[(size_t)aa * d.SP + c] = dxs * im0;
             }
-        for (int p = 0; p < C2; ++p)
-            for (int q = p; q < C2; ++q) {
-                const float g = get(k++) * (p == q ? 1.0f : kR2);
 #pragma unroll
-                for (int mm = 0; mm < 5; ++mm) {
-                    if (own2(mm) != r) continue;
-                    const float xp = T[o2 + mm * C2 + p], xq = T[o2 + mm * C2 + q];
-                    dXt2[mm * C2 + p] += g * xq;
-                    dXt2[mm * C2 + q] += g * xp;
-                }
-            }
-        if (L >= 3) {
-            const float g = get(k++);
-#pragma unroll
-            for (int mm = 0; mm < 7; ++mm)
-                if (own3(mm) == r) dX3[mm] += 2.0f * g * T[o3 + mm];
+            for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+            if (lane == 0) AUX[aa] = part;
         }
-    }
-    {   // (1,1,2): lane i < 3 owns component i of every probe gradient and row i of dQ
-        int k = d.oJ112;
-        for (int k1 = 0; k1 < K1; ++k1)
-            for (int k2 = k1; k2 < K1; ++k2) {
-                const float v1[3] = {Z1[k1], Z1[K1 + k1], Z1[2 * K1 + k1]};
-                const float v2[3] = {Z1[k2], Z1[K1 + k2], Z1[2 * K1 + k2]};
-#pragma unroll
-                for (int e = 0; e < K2; ++e) {
-                    const float cf = get(k++) * kC112 * (k1 == k2 ? 1.0f : kR2);
-                    if (r < 3) {
-                        const float q0 = pick3(f.Q[e], r), q1 = pick3(f.Q[e] + 3, r), q2 = pick3(f.Q[e] + 6, r);   // row r (Q symmetric)
-                        const float y2 = q0 * v2[0] + q1 * v2[1] + q2 * v2[2];
-                        const float y1 = q0 * v1[0] + q1 * v1[1] + q2 * v1[2];
-                        dZ1[r * K1 + k1] += cf * y2;
-                        dZ1[r * K1 + k2] += cf * y1;
-                        const float vr = pick3(v1, r);
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) dQ[e][j] += cf * vr * v2[j];
-                    }
-                }
-            }
-    }
-    if (L >= 3) {   // (1,2,3): each lane updates the targets whose rows it owns
-        const GauntSparse* G = f.G123;
-        const int nn = G->n;
-        int k = d.oJ123;
-        for (int k1 = 0; k1 < K1; ++k1)
-            for (int e = 0; e < K2; ++e) {
-                const float g = get(k++);
-                for (int n = 0; n < nn; ++n) {
-                    const int m1 = G->m1[n], m2 = G->m2[n], m3 = G->m3[n];
-                    const bool w1 = own1(m1) == r, w2 = own2(m2) == r, w3 = own3(m3) == r;
-                    if (!(w1 || w2 || w3)) continue;
-                    const float cv = g * G->v[n];
-                    const float z1 = Z1[m1 * K1 + k1], z2 = Z2[m2 * K2 + e], x3 = T[o3 + m3];
-                    if (w1) dZ1[m1 * K1 + k1] += cv * z2 * x3;
-                    if (w2) dZ2[m2 * K2 + e] += cv * z1 * x3;
-                    if (w3) dX3[m3] += cv * z1 * z2;
-                }
-            }
-    }
-    {   // (2,2,2): d tr(Qa Qb Qc)/dQa_ij = (Qb Qc)_ji, and cyclically; lane i takes row i
-        int k = d.oJ222;
-#pragma unroll
-        for (int e1 = 0; e1 < K2; ++e1)
-#pragma unroll
-            for (int e2 = e1; e2 < K2; ++e2)
-#pragma unroll
-                for (int e3 = e2; e3 < K2; ++e3) {
-                    const float cf = get(k++) * kC222 * fam3(e1, e2, e3);
-                    if (r < 3) {
-                        float P[9];
-                        matmul3(f.Q[e2], f.Q[e3], P);
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) dQ[e1][j] += cf * pick3(P + 3 * j, r);
-                        matmul3(f.Q[e3], f.Q[e1], P);
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) dQ[e2][j] += cf * pick3(P + 3 * j, r);
-                        matmul3(f.Q[e1], f.Q[e2], P);
-#pragma unroll
-                        for (int j = 0; j < 3; ++j) dQ[e3][j] += cf * pick3(P + 3 * j, r);
-                    }
-                }
-    }
-    if (L >= 3) {   // (2,3,3)
-        const GauntSparse* G = f.G233;
-        const int nn = G->n;
-        int k = d.oJ233;
-        for (int e = 0; e < K2; ++e) {
-            const float g = get(k++);
-            for (int n = 0; n < nn; ++n) {
-                const int m1 = G->m1[n], m2 = G->m2[n], m3 = G->m3[n];
-                const bool w1 = own2(m1) == r, w2 = own3(m2) == r, w3 = own3(m3) == r;
-                if (!(w1 || w2 || w3)) continue;
-                const float cv = g * G->v[n];
-                const float z2 = Z2[m1 * K2 + e], xa = T[o3 + m2], xb = T[o3 + m3];
-                if (w1) dZ2[m1 * K2 + e] += cv * xa * xb;
-                if (w2) dX3[m2] += cv * z2 * xb;
-                if (w3) dX3[m3] += cv * z2 * xa;
-            }
-        }
-    }
-    {   // quartic: y = Q v, Pi = y.y; lane i takes component i
-        int k = d.oPi;
-#pragma unroll
-        for (int e = 0; e < K2; ++e)
-            for (int k1 = 0; k1 < K1; ++k1) {
-                const float g2 = 2.0f * get(k++);
-                if (r < 3) {
-                    const float v[3] = {Z1[k1], Z1[K1 + k1], Z1[2 * K1 + k1]};
-                    float y[3];
-                    matvec3(f.Q[e], v[0], v[1], v[2], y);
-                    const float q0 = pick3(f.Q[e], r), q1 = pick3(f.Q[e] + 3, r), q2 = pick3(f.Q[e] + 6, r);
-                    const float qy = q0 * y[0] + q1 * y[1] + q2 * y[2];
-                    dZ1[r * K1 + k1] += g2 * qy;
-                    const float yr = pick3(y, r);
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) dQ[e][j] += g2 * yr * v[j];
-                }
-            }
-    }
-    // hand the rows of dQ to the degree-2 row owners through shared memory
-    __syncwarp();
-    if (r < 3) {
-#pragma unroll
-        for (int e = 0; e < K2; ++e)
-#pragma unroll
-            for (int j = 0; j < 3; ++j) dQs[e * 9 + 3 * r + j] = dQ[e][j];
-    }
-    __syncwarp();
-    // transpose of the symmetric-trace-free map, then probes -> aligned features.
-    // dot1 = sum dXt . Xt = sum dX . X (the alignment is linear)
-    float dot1 = 0.f;
-#pragma unroll
-    for (int mm = 0; mm < 5; ++mm) {
-        if (own2(mm) != r) continue;
-#pragma unroll
-        for (int e = 0; e < K2; ++e) {
-            const float q0 = dQs[e * 9], q1 = dQs[e * 9 + 1], q2 = dQs[e * 9 + 2], q3 = dQs[e * 9 + 3], q4 = dQs[e * 9 + 4],
-                        q5 = dQs[e * 9 + 5], q6 = dQs[e * 9 + 6], q7 = dQs[e * 9 + 7], q8 = dQs[e * 9 + 8];
-            float add;
-            if (mm == 0) add = kInvR2 * (q1 + q3);
-            else if (mm == 1) add = kInvR2 * (q5 + q7);
-            else if (mm == 2) add = kInvR6 * (2.0f * q8 - q0 - q4);
-            else if (mm == 3) add = kInvR2 * (q2 + q6);
-            else add = kInvR2 * (q0 - q4);
-            dZ2[mm * K2 + e] += add;
-        }
-        float g[C2];
-#pragma unroll
-        for (int c = 0; c < C2; ++c) {
-            float s = dXt2[mm * C2 + c];
-#pragma unroll
-            for (int kk = 0; kk < K2; ++kk) s += dZ2[mm * K2 + kk] * f.mA2[c * K2 + kk];
-            g[c] = s;
-            dot1 += s * T[o2 + mm * C2 + c];
-        }
-#pragma unroll
-        for (int c = 0; c < C2; ++c) {         // dX = dXt (I + W)^T, then / M_1
-            float s = 0.f;
-#pragma unroll
-            for (int b = 0; b < C2; ++b) s += g[b] * f.mW2[c * C2 + b];
-            T[o2 + mm * C2 + c] = s * f.iM1;
-        }
-    }
-#pragma unroll
-    for (int mm = 0; mm < 3; ++mm) {
-        if (own1(mm) != r) continue;
-        float g[C1];
-#pragma unroll
-        for (int c = 0; c < C1; ++c) {
-            float s = dXt1[mm * C1 + c];
-#pragma unroll
-            for (int kk = 0; kk < K1; ++kk) s += dZ1[mm * K1 + kk] * f.mA1[c * K1 + kk];
-            g[c] = s;
-            dot1 += s * T[o1 + mm * C1 + c];
-        }
-#pragma unroll
-        for (int c = 0; c < C1; ++c) {
-            float s = 0.f;
-#pragma unroll
-            for (int b = 0; b < C1; ++b) s += g[b] * f.mW1[c * C1 + b];
-            T[o1 + mm * C1 + c] = s * f.iM1;
-        }
-    }
-    if (L >= 3) {
-#pragma unroll
-        for (int mm = 0; mm < 7; ++mm) {
-            if (own3(mm) != r) continue;
-            const float g = dX3[mm];
-            dot1 += g * T[o3 + mm];
-            T[o3 + mm] = g * f.iM1;
-        }
-    }
-    // combine the four lanes' partial dot products (fixed order)
-    dot1 += __shfl_xor_sync(kFull, dot1, 1); dot1 += __shfl_xor_sync(kFull, dot1, 2);
-    if (r == 0) {
-        T[d.S - C0] = (dM0 - dot0 * f.iM0) * 0.5f * f.iM0;
-        T[d.S - C0 + 1] = (dM1 - dot1 * f.iM1) * 0.5f * f.iM1;
     }
     __syncthreads();
-    // write the block's slice back, coalesced
-    float* dst = a.state + (size_t)b0 * d.SP;
-    const int TW = d.SP - C0, total = nv * TW;
-    int atom = 0, k = tid;
-    for (int e = tid; e < total; e += NT) {
-        while (k >= TW) { k -= TW; ++atom; }
-        dst[(size_t)atom * d.SP + C0 + k] = f.tile[k * PITCH + atom];
-        k += NT;
+
+    // ---- gradients of the aligned rows, the probes and the two matrices Q --------------
+    for (int p = 0; p < C1; ++p) {                 // Gram of degree 1: a symmetric matrix-vector product per row
+        if (!TAKE()) continue;
+        float acc[3] = {0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int q = 0; q < C1; ++q) {
+            const float g = DSK(d.oG[1] + tri_sym(p, q, C1)) * (p == q ? 2.0f : kR2);
+#pragma unroll
+            for (int mm = 0; mm < 3; ++mm) acc[mm] += g * X1[(mm * C1 + q) * P];
+        }
+#pragma unroll
+        for (int mm = 0; mm < 3; ++mm) GX[(mm * C1 + p) * P + lane] = acc[mm];
     }
-#undef get
+    for (int p = 0; p < C2; ++p) {
+        if (!TAKE()) continue;
+        float acc[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int q = 0; q < C2; ++q) {
+            const float g = DSK(d.oG[2] + tri_sym(p, q, C2)) * (p == q ? 2.0f : kR2);
+#pragma unroll
+            for (int mm = 0; mm < 5; ++mm) acc[mm] += g * X2[(mm * C2 + q) * P];
+        }
+#pragma unroll
+        for (int mm = 0; mm < 5; ++mm) GX[(PL::nX1 + mm * C2 + p) * P + lane] = acc[mm];
+    }
+    if (L >= 3) {
+        float* G3a = GX + (PL::nX1 + PL::nX2) * P + lane;      // squared norm and (1,2,3)
+        float* G3b = GX + PL::nX * P + lane;                   // (2,3,3)
+        if (TAKE()) {
+            const float g2 = 2.0f * DSK(d.oG[3]);
+#pragma unroll
+            for (int mm = 0; mm < 7; ++mm) G3a[mm * P] = g2 * X3[mm * P];
+            const int nn = f.G123->n;
+            for (int n = 0; n < nn; ++n) {
+                const int m1 = f.G123->m1[n], m2 = f.G123->m2[n], m3 = f.G123->m3[n];
+                G3a[m3 * P] += f.G123->v[n] * (Ws[(m1 * K2) * P + lane] * Z2[(m2 * K2) * P] +
+                                               Ws[(m1 * K2 + 1) * P + lane] * Z2[(m2 * K2 + 1) * P]);
+            }
+        }
+        if (TAKE()) {
+#pragma unroll
+            for (int mm = 0; mm < 7; ++mm) G3b[mm * P] = 0.f;
+            const int nn = f.G233->n;
+            for (int n = 0; n < nn; ++n) {
+                const int m1 = f.G233->m1[n], m2 = f.G233->m2[n], m3 = f.G233->m3[n];
+                const float c = f.G233->v[n] * Zg[m1 * P + lane];
+                const float xa = X3[m2 * P], xb = X3[m3 * P];
+                G3b[m2 * P] += c * xb;
+                G3b[m3 * P] += c * xa;
+            }
+        }
+    }
+    for (int k = 0; k < K1; ++k) {                 // dE/dZ1[., k]: (1,1,2), quartic and (1,2,3) shares
+        if (!TAKE()) continue;
+        float acc[3] = {0.f, 0.f, 0.f};
+        for (int k2 = 0; k2 < K1; ++k2) {
+            const int t = tri_sym(k, k2, K1) * K2;
+            const float w = kC112 * (k == k2 ? 2.0f : kR2);
+#pragma unroll
+            for (int e = 0; e < K2; ++e) {
+                const float cf = DSK(d.oJ112 + t + e) * w;
+                const float* y = YQ + ((e * K1 + k2) * 3) * P + lane;
+                acc[0] += cf * y[0]; acc[1] += cf * y[P]; acc[2] += cf * y[2 * P];
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < K2; ++e) {
+            const float g2 = 2.0f * DSK(d.oPi + e * K1 + k);
+            const float* y = YQ + ((e * K1 + k) * 3) * P + lane;
+            float qy[3];
+            matvec3(Q[e], y[0], y[P], y[2 * P], qy);
+            acc[0] += g2 * qy[0]; acc[1] += g2 * qy[1]; acc[2] += g2 * qy[2];
+        }
+        if (L >= 3) {
+#pragma unroll
+            for (int e = 0; e < K2; ++e) {
+                const float g = DSK(d.oJ123 + k * K2 + e);
+#pragma unroll
+                for (int mm = 0; mm < 3; ++mm) acc[mm] += g * PRE[(mm * K2 + e) * P + lane];
+            }
+        }
+#pragma unroll
+        for (int mm = 0; mm < 3; ++mm) DZ[(mm * K1 + k) * P + lane] = acc[mm];
+    }
+#pragma unroll
+    for (int e = 0; e < K2; ++e) {                 // dE/dQ_e, one row i per unit
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            if (!TAKE()) continue;
+            float out[3] = {0.f, 0.f, 0.f};
+            for (int k1 = 0; k1 < K1; ++k1) {
+                const float vi = Z1[(i * K1 + k1) * P];
+                for (int k2 = k1; k2 < K1; ++k2) {
+                    const float cf = DSK(d.oJ112 + tri(k1, k2, K1) * K2 + e) * kC112 * (k1 == k2 ? 1.0f : kR2) * vi;
+                    out[0] += cf * Z1[k2 * P]; out[1] += cf * Z1[(K1 + k2) * P]; out[2] += cf * Z1[(2 * K1 + k2) * P];
+                }
+                const float gy = 2.0f * DSK(d.oPi + e * K1 + k1) * YQ[((e * K1 + k1) * 3 + i) * P + lane];
+                out[0] += gy * Z1[k1 * P]; out[1] += gy * Z1[(K1 + k1) * P]; out[2] += gy * Z1[(2 * K1 + k1) * P];
+            }
+            {   // (2,2,2): d tr(Qa Qb Qc) / dQa_ij = (Qb Qc)_ji, and cyclically
+                int k = d.oJ222;
+#pragma unroll
+                for (int e1 = 0; e1 < K2; ++e1)
+#pragma unroll
+                    for (int e2 = e1; e2 < K2; ++e2)
+#pragma unroll
+                        for (int e3 = e2; e3 < K2; ++e3) {
+                            const float cf = DSK(k) * kC222 * fam3(e1, e2, e3);
+                            ++k;
+#pragma unroll
+                            for (int j = 0; j < 3; ++j) {
+                                float s = 0.f;
+#pragma unroll
+                                for (int t = 0; t < 3; ++t) {
+                                    if (e1 == e) s += Q[e2][3 * j + t] * Q[e3][3 * t + i];
+                                    if (e2 == e) s += Q[e3][3 * j + t] * Q[e1][3 * t + i];
+                                    if (e3 == e) s += Q[e1][3 * j + t] * Q[e2][3 * t + i];
+                                }
+                                out[j] += cf * s;
+                            }
+                        }
+            }
+#pragma unroll
+            for (int j = 0; j < 3; ++j) DQ[(e * 9 + 3 * i + j) * P + lane] = out[j];
+        }
+    }
+    __syncthreads();
+
+    // ---- dE/dZ2: sparse couplings plus the transpose of the trace-free map -------------
+    for (int m2 = 0; m2 < 5; ++m2) {
+        if (!TAKE()) continue;
+        float acc[K2];
+#pragma unroll
+        for (int e = 0; e < K2; ++e) acc[e] = 0.f;
+        if (L >= 3) {
+            const int nn = f.G123->n;
+            for (int n = 0; n < nn; ++n) {
+                if (f.G123->m2[n] != m2) continue;
+                const float t = f.G123->v[n] * X3[f.G123->m3[n] * P];
+                const int m1 = f.G123->m1[n];
+#pragma unroll
+                for (int e = 0; e < K2; ++e) acc[e] += t * Ws[(m1 * K2 + e) * P + lane];
+            }
+            const float y = PRE[(PL::nU + m2) * P + lane];
+#pragma unroll
+            for (int e = 0; e < K2; ++e) acc[e] += DSK(d.oJ233 + e) * y;
+        }
+#pragma unroll
+        for (int e = 0; e < K2; ++e) {
+            const float* q = DQ + (e * 9) * P + lane;
+            float add;
+            if (m2 == 0) add = kInvR2 * (q[1 * P] + q[3 * P]);
+            else if (m2 == 1) add = kInvR2 * (q[5 * P] + q[7 * P]);
+            else if (m2 == 2) add = kInvR6 * (2.0f * q[8 * P] - q[0] - q[4 * P]);
+            else if (m2 == 3) add = kInvR2 * (q[2 * P] + q[6 * P]);
+            else add = kInvR2 * (q[0] - q[4 * P]);
+            DZ[(PL::nZ1 + m2 * K2 + e) * P + lane] = acc[e] + add;
+        }
+    }
+    __syncthreads();
+
+    // ---- probes and alignment transposed, row by row; dot1 = sum dXt . Xt = sum dX . X --
+    for (int u = 0; u < 9; ++u) {
+        if (!TAKE()) continue;
+        float dot = 0.f;
+        if (u < 3)
+            dot = back_row<C1, K1>(GX + (u * C1) * P + lane, DZ + (u * K1) * P + lane, f.mA1, f.mW1, X1 + (u * C1) * P,
+                                   ST + (f.o1 + u * C1) * P + lane, f.iM1);
+        else if (u < 8)
+            dot = back_row<C2, K2>(GX + (PL::nX1 + (u - 3) * C2) * P + lane, DZ + (PL::nZ1 + (u - 3) * K2) * P + lane, f.mA2,
+                                   f.mW2, X2 + ((u - 3) * C2) * P, ST + (f.o2 + (u - 3) * C2) * P + lane, f.iM1);
+        else if (L >= 3) {
+#pragma unroll
+            for (int mm = 0; mm < 7; ++mm) {
+                const float g = GX[(PL::nX1 + PL::nX2 + mm) * P + lane] + GX[(PL::nX + mm) * P + lane];
+                dot += g * X3[mm * P];
+                ST[(f.o3 + mm) * P + lane] = g * f.iM1;
+            }
+        }
+        AUX[(1 + u) * P + lane] = dot;
+    }
+    __syncthreads();
+    if (warp == 0) {   // gradients of the two sums of squared envelopes, fixed summation order
+        float dot1 = 0.f;
+#pragma unroll
+        for (int u = 0; u < 9; ++u) dot1 += AUX[(1 + u) * P + lane];
+        const float iM0 = (float)(1.0 / f.M0_of(lane));
+        const float dM0 = DSK(2 * C0), dM1 = DSK(2 * C0 + 1), dot0 = AUX[lane];
+        ST[f.oS * P + lane] = (dM0 - dot0 * iM0) * 0.5f * iM0;
+        ST[(f.oS + 1) * P + lane] = (dM1 - dot1 * f.iM1) * 0.5f * f.iM1;
+    }
+    __syncthreads();
+    // write the block's slice back, lane = state entry
+    float* dst = a.state + (size_t)b0 * d.SP + C0;
+    for (int k0 = 0; k0 < TW; k0 += 32) {
+        const int k = k0 + lane;
+        if (k >= TW) continue;
+#pragma unroll
+        for (int i = 0; i < AT / NW; ++i) {
+            const int aa = warp + i * NW;
+            if (aa < nv) dst[(size_t)aa * d.SP + k] = ST[k * P + aa];
+        }
+    }
+#undef TAKE
+#undef DSK
 }
 
 template <bool FWD>
 cudaError_t dispatch(const InvArgs& a, cudaStream_t st) {
     if (a.n <= 0) return cudaSuccess;
-    const int blocks = (a.n + ATOMS - 1) / ATOMS;
+    const int blocks = (a.n + AT - 1) / AT;
     const int C1 = a.d.C[1], C2 = a.d.C[2], L = a.d.L;
+    const int TW = a.d.SP - a.d.C0, nDS = a.d.DP - (2 * a.d.C0 / 32) * 32;
 #define UMLMD_CASE(c1, c2, l)                                                                   \
     if (C1 == c1 && C2 == c2 && L == l) {                                                       \
-        const size_t bytes = sizeof(float) * Lay<c1, c2, l>::floats(a.d.SP, a.d.C0, a.d.DP, !FWD);              \
+        const size_t bytes = Plan<c1, c2, l>::bytes(TW, nDS, !FWD);                             \
         auto kern = FWD ? k_inv_forward<c1, c2, l> : k_inv_backward<c1, c2, l>;                 \
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes); \
         if (e != cudaSuccess) return e;                                                         \
