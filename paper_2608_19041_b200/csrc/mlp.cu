@@ -85,6 +85,17 @@ __global__ void k_head(int n, int F, const float* __restrict__ h, const float* _
     }
 }
 
+// tensor-core path: the last layer's epilogue left one partial dot product per column tile
+__global__ void k_head_finish(int n, int parts, const float* __restrict__ part, float b_head,
+                              const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
+                              double* __restrict__ e_atom) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    double s = 0.0;
+    for (int p = 0; p < parts; ++p) s += (double)part[(size_t)i * parts + p];
+    e_atom[a0 + i] = s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + i]);
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {
@@ -106,7 +117,9 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     const size_t layer = (size_t)n * F;
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
-    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo;
+    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    // the backward seed goes to the slot the last layer does not read its input from
+    const int seed_slot = NH & 1;
     cudaError_t e;
     // ---- forward --------------------------------------------------------------------
     for (int t = 0; t < NH; ++t) {
@@ -128,13 +141,28 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         g.bias = a.m.bias[t];
         g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
         g.out = hb[t & 1]; g.ldout = F;
+        if (tc && t == NH - 1) {
+            // last layer: the epilogue takes the head's dot product and the backward seed, so
+            // neither the activations nor the pre-activations of this layer are stored
+            g.head_w = a.m.w_head; g.head_part = hb[t & 1]; g.head_parts = (F + kGemmTcBN - 1) / kGemmTcBN;
+            g.out = nullptr; g.pre = nullptr;
+            if (a.want_grad) {
+                g.nxt_hi = a.tc_hi + (size_t)seed_slot * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)seed_slot * a.tc_slot;
+                g.ldnxt = F;
+            }
+        }
         if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
     }
-    {
+    if (tc) {
+        const int parts = (F + kGemmTcBN - 1) / kGemmTcBN;
+        k_head_finish<<<(n + 255) / 256, 256, 0, st>>>(n, parts, hb[(NH - 1) & 1], a.m.b_head, a.m.e_ref, a.type_s, a.a0,
+                                                        a.e_atom);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    } else {
         const int warps = 8, blocks = (n + warps - 1) / warps;
         k_head<<<blocks, warps * 32, 0, st>>>(n, F, hb[(NH - 1) & 1], a.m.w_head, a.m.b_head, a.m.e_ref, a.type_s,
                                              a.a0, a.want_grad ? a.pre + (size_t)(NH - 1) * layer : nullptr,
-                                             tc ? a.tc_hi : nullptr, tc ? a.tc_lo : nullptr, a.e_atom, a.want_grad);
+                                             nullptr, nullptr, a.e_atom, a.want_grad);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -149,8 +177,8 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
     cudaError_t e;
-    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo;
-    int sp = 0;                // tensor-core path: slot with the TF32 split of pre[t] (the head kernel fills slot 0)
+    const bool tc = a.path == 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    int sp = NH & 1;           // tensor-core path: slot with the TF32 split of pre[t] (the forward pass left the seed here)
     int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
     bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
     for (int t = NH - 1; t >= 1; --t) {

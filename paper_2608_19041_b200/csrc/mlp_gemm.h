@@ -30,6 +30,11 @@ struct GemmArgs {
     // TF32 split of the value the next GEMM of the chain consumes (mode 0: out, mode 1: the new
     // pre), written by the epilogue with row pitch ldnxt when non-null
     float* nxt_hi; float* nxt_lo; int ldnxt;
+    // tensor-core path, mode 0, last layer: instead of storing out (and pre), the epilogue dots
+    // each output row with head_w over the CTA's columns, head_part[m * head_parts + column
+    // tile], and, when nxt_hi is set, leaves the split of head_w[n] * SiLU'(y[m,n]) there (the
+    // seed of the backward pass)
+    const float* head_w; float* head_part; int head_parts;
     int* err;                     // device error word (bounded-wait expiry)
 };
 
@@ -89,6 +94,8 @@ __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, 
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
+bool gemm_tc_available();      // the driver's tensor-map encoder could be resolved
+constexpr int kGemmTcBN = 128;  // column tile of the tensor-core GEMM
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st);
 
 }  // namespace umd

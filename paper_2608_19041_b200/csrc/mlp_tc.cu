@@ -30,7 +30,7 @@ namespace umd {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 16, STAGES = 3;
+constexpr int BM = 128, BN = kGemmTcBN, BK = 16, STAGES = 3;
 constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 8 KB, also BN * BK * 4
 constexpr uint32_t STAGE_BYTES = 4 * TILE_BYTES;      // A_hi, A_lo, B_hi, B_lo
 constexpr uint32_t BAR_BYTES = 128;
@@ -107,6 +107,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 // instruction descriptor: D = F32, A = B = TF32, both K-major, N = 128, M = 128
 constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+// MODE 0: forward layer, 1: backward layer, 2: last forward layer with the fused head
+template <int MODE>
 __global__ void __launch_bounds__(192, 2)
 k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUtensorMap mAl,
           const __grid_constant__ CUtensorMap mBh, const __grid_constant__ CUtensorMap mBl, const GemmArgs g) {
@@ -187,17 +189,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
         }
         __syncwarp();
         const int n = n0 + 4 * lane;
-        if (n < g.N) {
-            float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias;
-            if (g.mode == 0) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
-            const bool use_res = g.res && (g.res_n == 0 || n < g.res_n);
-            if (g.mode == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+        const bool valid = n < g.N;
+        {
+            float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
+            if (valid && MODE != 1) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+            if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
+            const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
+            if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
             const int rows = min(32, g.M - (m0 + q * 32));
             // The stores below may alias the loads as far as the compiler knows, so the rows
             // are taken in batches: all global loads of a batch are issued before its first
             // store, which keeps RB rows (not one) in flight per warp.
             constexpr int RB = 8;
-            const bool rd_pre = g.mode == 1 && g.pre;
+            const bool rd_pre = valid && MODE == 1 && g.pre;
 #pragma unroll 1
             for (int r0 = 0; r0 < rows; r0 += RB) {
                 float4 res[RB], y[RB];
@@ -208,7 +212,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     y[j] = res[j];
                     if (r0 + j < rows) {
                         if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
-                        if (rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n);
+                        if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n);
                     }
                 }
 #pragma unroll
@@ -216,21 +220,34 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     if (r0 + j >= rows) break;
                     const size_t m = (size_t)(m0 + q * 32 + r0 + j);
                     float4 a = *reinterpret_cast<const float4*>(stage + (r0 + j) * EPITCH + 4 * lane);
-                    if (g.mode == 0) {
+                    if (MODE != 1) {
                         a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
-                        if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
                         const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
                                                      silu(a.w) + res[j].w);
-                        *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
-                        if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
-                    } else {
+                        if (MODE == 2) {           // last layer: row . w_head, and the backward seed
+                            float part = valid ? o.x * hw.x + o.y * hw.y + o.z * hw.z + o.w * hw.w : 0.f;
+#pragma unroll
+                            for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                            if (lane == 0) g.head_part[m * g.head_parts + blockIdx.x] = part;
+                            if (valid && g.nxt_hi)
+                                store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n,
+                                             make_float4(hw.x * silu_grad(a.x), hw.y * silu_grad(a.y), hw.z * silu_grad(a.z),
+                                                         hw.w * silu_grad(a.w)));
+                        } else if (valid) {
+                            if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
+                            *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
+                            if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
+                        }
+                    } else if (valid) {
                         a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
                         if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
                         if (g.pre) {
                             const float4 o = make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y),
                                                          a.z * silu_grad(y[j].z), a.w * silu_grad(y[j].w));
-                            *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
+                            // the next GEMM of the chain reads the split; the fp32 copy is only
+                            // kept when nothing else will carry the value
                             if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
+                            else *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
                         }
                     }
                 }
@@ -289,6 +306,8 @@ bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
 
 }  // namespace
 
+bool gemm_tc_available() { return encode_fn() != nullptr; }
+
 bool gemm_tc_supported(const GemmArgs& g) {
     return g.A_hi && g.A_lo && g.Bt_hi && g.Bt_lo && g.M > 0 && g.N >= 4 && g.K >= 4 && (g.K & 3) == 0 &&
            (g.N & 3) == 0 && (g.lda & 3) == 0 && (g.ldbt & 3) == 0 && encode_fn() != nullptr;
@@ -297,7 +316,9 @@ bool gemm_tc_supported(const GemmArgs& g) {
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -312,7 +333,9 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
         !make_map(&mBh, g.Bt_hi, g.N, g.K, g.ldbt) || !make_map(&mBl, g.Bt_lo, g.N, g.K, g.ldbt))
         return cudaErrorInvalidValue;
     dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
-    k_gemm_tc<<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    if (g.mode == 1) k_gemm_tc<1><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    else if (g.head_w) k_gemm_tc<2><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    else k_gemm_tc<0><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
     return cudaGetLastError();
 }
 
