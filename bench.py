@@ -230,7 +230,10 @@ def run_ours(args):
     name = args.workload
     cfg = CONFIGS[name]
     p = cfg["profile"]
-    md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=300.0, seed=1, rebuild_every=10, skin=0.0)
+    # a workload without an MD recipe is timed as repeated single evaluations (energy + forces +
+    # virial of the same frame, list built once): velocities are zero and nothing moves
+    static = cfg["md"] is None
+    md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=0.0, seed=1, rebuild_every=1 << 30, skin=0.0)
     desc = dict(cfg["system"])
     if args.atoms:
         # a smaller box of the same recipe (density, exclusion radius, species mix): the size one
@@ -239,13 +242,13 @@ def run_ours(args):
             raise SystemExit("--atoms applies to the amorphous workload only")
         desc["atoms"] = int(args.atoms)
         name = f"{name}[atoms={int(args.atoms)}]"
-    s = make_system(desc, md)
+    s = make_system(desc, None if static else md)
     N = len(s["pos"])
     blob = workload_blob(args.workload)
     model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile)
     pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
     pos = pos0.cuda().contiguous()
-    vel = torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
+    vel = None if static else torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
     types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
     skin, every, dt = md["skin"], md["rebuild_every"], md["dt_ps"]
 
@@ -253,7 +256,8 @@ def run_ours(args):
     e_rc = model.query()["n_edges"]
     model.build_neighbors(pos, types, s["cell"], s["pbc"], skin)
     e_list = model.query()["n_edges"]
-    model.set_md_state(pos, vel, s["masses"])
+    if not static:
+        model.set_md_state(pos, vel, s["masses"])
 
     def sync_all():
         torch.cuda.synchronize()
@@ -261,14 +265,21 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    model.step(args.warmup, dt, every)
+    def run_steps(k):
+        if not static:
+            return model.step(k, dt, every)
+        for _ in range(k):
+            out = model.compute(pos, forces=True, virial=True)
+        return out["energy"], 0.0
+
+    run_steps(args.warmup)
     launches0 = model.query()["kernel_launches"]
     sampler = ClockSampler(local)
     sync_all()
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    e_pot, e_kin = model.step(args.steps, dt, every)
+    e_pot, e_kin = run_steps(args.steps)
     ev1.record()
     sync_all()
     clocks = sampler.stop()
@@ -283,7 +294,7 @@ def run_ours(args):
     # ---- second pass with per-class events: where the time goes, roofline per class
     model.get_profile()
     model.set_profiling(True)
-    model.step(args.steps, dt, every)
+    run_steps(args.steps)
     prof = model.get_profile()
     model.set_profiling(False)
     peaks = measured_peaks()

@@ -53,7 +53,7 @@ typedef struct umlmd_options {
     uint32_t struct_bytes;
     double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
     int32_t  node_tile;  /* atoms per workspace tile; 0 = 131072                            */
-    int32_t  mlp_path;   /* 0 = default, 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM  */
+    int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM, persistent, 3 = tcgen05 3xTF32 GEMM, one tile per CTA */
 } umlmd_options;
 
 /* Structural widths of a model, all derived from (C0, L, R) by the paper's formulas

@@ -164,7 +164,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
-        { Scope sc(h, kMlpFwd, d.n_hidden + (h->mlp_path == 2 ? 2 : 1)); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
+        { Scope sc(h, kMlpFwd, d.n_hidden + (h->mlp_path >= 2 ? 2 : 1)); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
             { Scope sc(h, kInvBwd, 1); API_CUDA(h, launch_invariants_backward(ia, h->st)); }
@@ -259,7 +259,7 @@ int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, 
     double dx_override = 0;
     if (opt) {
         if (opt->struct_bytes != sizeof(umlmd_options)) { delete h; return UMLMD_E_INVALID_ARG; }
-        if (opt->table_dx < 0 || opt->node_tile < 0 || opt->mlp_path < 0 || opt->mlp_path > 2) { delete h; return UMLMD_E_INVALID_ARG; }
+        if (opt->table_dx < 0 || opt->node_tile < 0 || opt->mlp_path < 0 || opt->mlp_path > 3) { delete h; return UMLMD_E_INVALID_ARG; }
         dx_override = opt->table_dx;
         if (opt->node_tile > 0) h->node_tile = opt->node_tile;
         if (opt->mlp_path > 0) h->mlp_path = opt->mlp_path;

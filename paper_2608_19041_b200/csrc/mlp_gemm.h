@@ -35,6 +35,7 @@ struct GemmArgs {
     // tile], and, when nxt_hi is set, leaves the split of head_w[n] * SiLU'(y[m,n]) there (the
     // seed of the backward pass)
     const float* head_w; float* head_part; int head_parts;
+    int variant;                  // tensor-core kernel: 3 = one tile per CTA, otherwise the persistent one
     int* err;                     // device error word (bounded-wait expiry)
 };
 
@@ -96,6 +97,8 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
 bool gemm_tc_available();      // the driver's tensor-map encoder could be resolved
 constexpr int kGemmTcBN = 128;  // column tile of the tensor-core GEMM
+// partial head sums per row that the fused last-layer epilogue of a variant leaves
+inline int gemm_tc_head_parts(int N, int variant) { return (variant == 3 ? 1 : 2) * ((N + kGemmTcBN - 1) / kGemmTcBN); }
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st);
 
 }  // namespace umd

@@ -261,6 +261,218 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Persistent variant: one CTA per SM walks work items of 256 rows x 128 columns.  An item
+// uses two accumulators (rows 0..127 and 128..255) that share every B tile, so the weights
+// cross L2 -> shared memory half as often as with one 128 x 128 tile per CTA; tensor memory
+// holds two such pairs (512 columns), so the epilogue of item i overlaps the main loop of
+// item i + 1.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2..9: epilogue (warp % 4 =
+// lane quarter of tensor memory, (warp - 2) / 4 = which accumulator of the pair).
+// The epilogue turns the tile through a staging area of its own, 64 columns at a time.
+constexpr int P_STAGES = 3;
+constexpr uint32_t P_STAGE_BYTES = 6 * TILE_BYTES;    // A0_hi, A0_lo, A1_hi, A1_lo, B_hi, B_lo
+constexpr int P_EPW = 8;                               // epilogue warps
+constexpr int P_SPITCH = 64 + 4;                       // staging row pitch (floats)
+constexpr uint32_t P_STAGING_BYTES = P_EPW * 32 * P_SPITCH * 4;
+constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_STAGING_BYTES + 1024 + BAR_BYTES;
+constexpr int P_THREADS = (2 + P_EPW) * 32;
+
+// bounded wait that gives up at once after any wait of this CTA has expired
+__device__ __forceinline__ void mbar_wait_a(uint32_t bar, uint32_t parity, int* err, volatile int* abort_flag) {
+    if (*abort_flag) return;
+    for (int i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, parity)) return;
+        if (i > 64) __nanosleep(32);
+    }
+    *abort_flag = 1;
+    if (err) atomicOr(err, kErrPipelineTimeout);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(P_THREADS, 1)
+k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUtensorMap mAl,
+           const __grid_constant__ CUtensorMap mBh, const __grid_constant__ CUtensorMap mBl, const GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t staging = tiles + P_STAGES * P_STAGE_BYTES;
+    const uint32_t bars = staging + P_STAGING_BYTES;   // full[3], empty[3], acc_full[2], acc_empty[2], tmem slot, abort flag
+    const uint32_t acc_full = bars + 8 * (2 * P_STAGES), acc_empty = acc_full + 16;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + (acc_empty + 16 - raw));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (acc_empty + 24 - raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KB = (g.K + BK - 1) / BK;
+    const int ntn = (g.N + BN - 1) / BN, ntm = (g.M + 2 * BM - 1) / (2 * BM);
+    const int items = ntn * ntm;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(bars + 8 * s, 1); mbar_init(bars + 8 * (P_STAGES + s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full + 8 * b, 1); mbar_init(acc_empty + 8 * b, P_EPW); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {                                   // TMA producer
+            int gk = 0;
+            for (int it = blockIdx.x; it < items; it += gridDim.x) {
+                const int m0 = (it / ntn) * 2 * BM, n0 = (it % ntn) * BN;
+                for (int kb = 0; kb < KB; ++kb, ++gk) {
+                    const int s = gk % P_STAGES, u = gk / P_STAGES;
+                    if (u > 0) mbar_wait_a(bars + 8 * (P_STAGES + s), (u - 1) & 1, g.err, abort_flag);
+                    const uint32_t full = bars + 8 * s, sa = tiles + s * P_STAGE_BYTES;
+                    mbar_expect_tx(full, P_STAGE_BYTES);
+                    tma_load_2d(sa, &mAh, kb * BK, m0, full);
+                    tma_load_2d(sa + TILE_BYTES, &mAl, kb * BK, m0, full);
+                    tma_load_2d(sa + 2 * TILE_BYTES, &mAh, kb * BK, m0 + BM, full);
+                    tma_load_2d(sa + 3 * TILE_BYTES, &mAl, kb * BK, m0 + BM, full);
+                    tma_load_2d(sa + 4 * TILE_BYTES, &mBh, kb * BK, n0, full);
+                    tma_load_2d(sa + 5 * TILE_BYTES, &mBl, kb * BK, n0, full);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {                                   // MMA issuer
+            int gk = 0, li = 0;
+            for (int it = blockIdx.x; it < items; it += gridDim.x, ++li) {
+                const int b = li & 1, v = li >> 1;
+                if (v > 0) mbar_wait_a(acc_empty + 8 * b, (v - 1) & 1, g.err, abort_flag);
+                tc_fence_after();
+                const uint32_t d0 = tmem + (uint32_t)(b * 256), d1 = d0 + 128u;
+                for (int kb = 0; kb < KB; ++kb, ++gk) {
+                    const int s = gk % P_STAGES, u = gk / P_STAGES;
+                    mbar_wait_a(bars + 8 * s, u & 1, g.err, abort_flag);
+                    tc_fence_after();
+                    const uint32_t sa = tiles + s * P_STAGE_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 8; ++k) {
+                        const uint64_t bh = umma_desc(sa + 4 * TILE_BYTES + k * 32), bl = umma_desc(sa + 5 * TILE_BYTES + k * 32);
+                        const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                        {
+                            const uint64_t ah = umma_desc(sa + k * 32), al = umma_desc(sa + TILE_BYTES + k * 32);
+                            umma_tf32(d0, al, bh, kIdesc, acc);
+                            umma_tf32(d0, ah, bl, kIdesc, 1u);
+                            umma_tf32(d0, ah, bh, kIdesc, 1u);
+                        }
+                        {
+                            const uint64_t ah = umma_desc(sa + 2 * TILE_BYTES + k * 32), al = umma_desc(sa + 3 * TILE_BYTES + k * 32);
+                            umma_tf32(d1, al, bh, kIdesc, acc);
+                            umma_tf32(d1, ah, bl, kIdesc, 1u);
+                            umma_tf32(d1, ah, bh, kIdesc, 1u);
+                        }
+                    }
+                    umma_commit(bars + 8 * (P_STAGES + s));    // frees the stage when these MMAs retire
+                }
+                umma_commit(acc_full + 8 * b);
+            }
+        }
+    } else {                                               // epilogue
+        const int e = warp - 2, q = warp & 3, h = e >> 2;
+        float* stage = reinterpret_cast<float*>(smem_raw + (staging - raw)) + (size_t)e * 32 * P_SPITCH;
+        const int hr = lane >> 4, c4 = (lane & 15) * 4;      // half-warp per row, four columns per lane
+        int li = 0;
+        for (int it = blockIdx.x; it < items; it += gridDim.x, ++li) {
+            const int b = li & 1, v = li >> 1;
+            const int ct = it % ntn;
+            const int mrow0 = (it / ntn) * 2 * BM + h * BM + q * 32, n0 = ct * BN;
+            mbar_wait_a(acc_full + 8 * b, v & 1, g.err, abort_flag);
+            tc_fence_after();
+            const uint32_t tacc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 256 + h * 128);
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    float vv[32];
+                    tmem_ld32(tacc + (uint32_t)(pass * 64 + c0), vv);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4*>(stage + lane * P_SPITCH + c0 + 4 * j) =
+                            make_float4(vv[4 * j], vv[4 * j + 1], vv[4 * j + 2], vv[4 * j + 3]);
+                }
+                if (pass == 1) {                           // the accumulator has been read out: hand it back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty + 8 * b) : "memory");
+                }
+                __syncwarp();
+                const int n = n0 + pass * 64 + c4;
+                const bool valid = n < g.N;
+                float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
+                if (valid && MODE != 1) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+                if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
+                const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
+                if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+                const bool rd_pre = valid && MODE == 1 && g.pre;
+                constexpr int RB = 4;                      // iterations (two rows each) whose loads are issued together
+#pragma unroll 1
+                for (int i0 = 0; i0 < 16; i0 += RB) {
+                    float4 res[RB], y[RB];
+#pragma unroll
+                    for (int j = 0; j < RB; ++j) {
+                        const int m = mrow0 + 2 * (i0 + j) + hr;
+                        res[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        y[j] = res[j];
+                        if (m < g.M) {
+                            if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n);
+                            if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + (size_t)m * g.ldpre + n);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < RB; ++j) {
+                        const int r = 2 * (i0 + j) + hr;
+                        const size_t m = (size_t)(mrow0 + r);
+                        const bool okm = mrow0 + r < g.M;
+                        float4 a = *reinterpret_cast<const float4*>(stage + r * P_SPITCH + c4);
+                        if (MODE != 1) {
+                            a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
+                            const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
+                                                         silu(a.w) + res[j].w);
+                            if (MODE == 2) {               // last layer: row . w_head over these 64 columns, and the seed
+                                float part = valid ? o.x * hw.x + o.y * hw.y + o.z * hw.z + o.w * hw.w : 0.f;
+#pragma unroll
+                                for (int off = 8; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                                if ((lane & 15) == 0 && okm) g.head_part[m * g.head_parts + 2 * ct + pass] = part;
+                                if (valid && okm && g.nxt_hi)
+                                    store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n,
+                                                 make_float4(hw.x * silu_grad(a.x), hw.y * silu_grad(a.y), hw.z * silu_grad(a.z),
+                                                             hw.w * silu_grad(a.w)));
+                            } else if (valid && okm) {
+                                if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
+                                *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
+                                if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
+                            }
+                        } else if (valid && okm) {
+                            a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
+                            if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
+                            if (g.pre) {
+                                const float4 o = make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y),
+                                                             a.z * silu_grad(y[j].z), a.w * silu_grad(y[j].w));
+                                if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
+                                else *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
+                            }
+                        }
+                    }
+                }
+                __syncwarp();                              // staging rows are rewritten by the next pass
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
 // hi = round-to-nearest TF32 of x, lo = round-to-nearest TF32 of (x - hi); rows [M][K]
 __global__ void k_split_tf32(const float* __restrict__ A, int lda, int M, int K, float* __restrict__ hi,
                              float* __restrict__ lo) {
@@ -315,10 +527,17 @@ bool gemm_tc_supported(const GemmArgs& g) {
 
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
     static bool attr_set = false;
+    static int n_sm = 0;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tcp<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tcp<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tcp<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+        int dev = 0;
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -332,10 +551,19 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
     if (!make_map(&mAh, g.A_hi, g.M, g.K, g.K) || !make_map(&mAl, g.A_lo, g.M, g.K, g.K) ||
         !make_map(&mBh, g.Bt_hi, g.N, g.K, g.ldbt) || !make_map(&mBl, g.Bt_lo, g.N, g.K, g.ldbt))
         return cudaErrorInvalidValue;
-    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
-    if (g.mode == 1) k_gemm_tc<1><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
-    else if (g.head_w) k_gemm_tc<2><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
-    else k_gemm_tc<0><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    const int mode = g.mode == 1 ? 1 : (g.head_w ? 2 : 0);
+    if (g.variant == 3) {                                  // one 128 x 128 tile per CTA, two CTAs per SM
+        dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM);
+        if (mode == 1) k_gemm_tc<1><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+        else if (mode == 2) k_gemm_tc<2><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+        else k_gemm_tc<0><<<grid, 192, SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    } else {                                               // persistent, 256 x 128 items
+        const int items = ((g.N + BN - 1) / BN) * ((g.M + 2 * BM - 1) / (2 * BM));
+        const int grid = items < n_sm ? items : n_sm;
+        if (mode == 1) k_gemm_tcp<1><<<grid, P_THREADS, P_SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+        else if (mode == 2) k_gemm_tcp<2><<<grid, P_THREADS, P_SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+        else k_gemm_tcp<0><<<grid, P_THREADS, P_SMEM_BYTES, st>>>(mAh, mAl, mBh, mBl, g);
+    }
     return cudaGetLastError();
 }
 
