@@ -90,22 +90,24 @@ __global__ void __launch_bounds__(kRedBlock) k_sum_slices(const double* __restri
     if (threadIdx.x == 0) part[blockIdx.x] = s;
 }
 
-// pass 2 (one block): out[0] = sum of slice partials; out[1..9] = -sum of virial partials
+// pass 2 (ten blocks): block 0: out[0] = sum of slice partials; block 1 + k: out[1 + k] = -sum of
+// the k-th component of the virial partials
 __global__ void __launch_bounds__(kRedBlock) k_final_reduce(const double* __restrict__ part, int n_part,
                                                             const double* __restrict__ vpart, int n_vpart,
                                                             double* __restrict__ out, int* __restrict__ err) {
     __shared__ double sh[kRedBlock / 32];
     double v = 0;
-    for (int i = threadIdx.x; i < n_part; i += kRedBlock) v += part[i];
-    double s = block_sum(v, sh);
-    if (threadIdx.x == 0) {
-        out[0] = s;
-        if (!isfinite(s)) atomicOr(err, kErrNonFinite);
-    }
-    for (int k = 0; k < 9; ++k) {
-        v = 0;
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < n_part; i += kRedBlock) v += part[i];
+        const double s = block_sum(v, sh);
+        if (threadIdx.x == 0) {
+            out[0] = s;
+            if (!isfinite(s)) atomicOr(err, kErrNonFinite);
+        }
+    } else {
+        const int k = blockIdx.x - 1;
         for (int i = threadIdx.x; i < n_vpart; i += kRedBlock) v += vpart[(size_t)i * 9 + k];
-        s = block_sum(v, sh);
+        const double s = block_sum(v, sh);
         if (threadIdx.x == 0) out[1 + k] = -s;
     }
 }
@@ -184,7 +186,7 @@ cudaError_t launch_reduce_energy_virial(const double* e_atom, int64_t N, const d
     int blocks; int64_t chunk;
     slices(N, &blocks, &chunk);
     k_sum_slices<<<blocks, kRedBlock, 0, st>>>(e_atom, N, chunk, scratch);
-    k_final_reduce<<<1, kRedBlock, 0, st>>>(scratch, blocks, virial_part, n_part, out, d_err);
+    k_final_reduce<<<10, kRedBlock, 0, st>>>(scratch, blocks, virial_part, n_part, out, d_err);
     return cudaGetLastError();
 }
 

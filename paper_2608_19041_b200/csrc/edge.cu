@@ -170,7 +170,7 @@ template <int C0, int L> struct Widths {
 
 template <int C0, int L> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L>;
-    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LPE + 1) + W::NHI + 3) / 4 * 4;   // floats
+    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LPE + 1) + W::NHI + 3) / 4 * 4 + 32 * 4;   // floats
     static constexpr size_t bytes = kWarpsPerBlock * 9 * sizeof(double) + sizeof(float) * kWarpsPerBlock * per_warp;
 };
 
@@ -191,6 +191,7 @@ k_edge_forward(const EdgeArgs a) {
     // one 32 x 33 float scratch per warp: first the parked amplitudes (row pitch PF), then,
     // once every lane has read its own row, the transpose buffer
     __shared__ __align__(16) float scratch[kWarpsPerBlock][32 * 33];
+    __shared__ int4 edge_s[kWarpsPerBlock][32];         // per-edge scalars of the batch: row, pair, t, chi
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     if (i >= a.a1) return;
@@ -210,15 +211,25 @@ k_edge_forward(const EdgeArgs a) {
     for (int base = e0; base < e1; base += 32) {
         const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
         if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
-        const int nb = min(32, e1 - base);
-        for (int it = 0; it * W::EPI < nb; ++it) {
-            const int b = it * W::EPI + sub;
-            const bool v = __shfl_sync(kFull, (int)g.valid, b) != 0;
-            const int row = __shfl_sync(kFull, g.row, b);
-            const int pair = __shfl_sync(kFull, g.pair, b);
-            const float t = __shfl_sync(kFull, g.t, b);
-            const float chi = __shfl_sync(kFull, g.chi, b);
-            if (!v) continue;
+        // The channel-parallel phase visits only the edges inside the cutoff; their scalars
+        // are parked in shared memory and fetched with one 16-byte broadcast load (shuffles
+        // would go through the same L1 data pipe as the table reads, five at a time).
+        edge_s[wid][lane] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
+        const unsigned vmask = __ballot_sync(kFull, g.valid);
+        const int nvalid = __popc(vmask);
+        __syncwarp();
+        unsigned mrun = vmask;
+        for (int it = 0; it * W::EPI < nvalid; ++it) {
+            int b;
+            if (W::EPI == 1) { b = __ffs(mrun) - 1; mrun &= mrun - 1; }      // next edge inside the cutoff
+            else {
+                const int idx = it * W::EPI + sub;
+                if (idx >= nvalid) continue;
+                b = (int)__fns(vmask, 0, idx + 1);
+            }
+            const int4 es = edge_s[wid][b];
+            const int row = es.x, pair = es.y;
+            const float t = __int_as_float(es.z), chi = __int_as_float(es.w);
             float psi[4];
             amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr);
 #pragma unroll
@@ -323,6 +334,7 @@ k_edge_backward(const EdgeArgs a) {
     float* const psi_s = wbase;                                  // [32][PB]: psi, dpsi of the leading channels
     float* const red = psi_s + 32 * W::PB;                       // [2][32][LPE+1] partial dot products
     float* const hi_s = red + 2 * 32 * (W::LPE + 1);             // [NHI] gradient of the degree >= 1 sums
+    int4* const edge_s = reinterpret_cast<int4*>(wbase + BwdSmem<C0, L>::per_warp - 32 * 4);   // [32] row, pair, t of the batch
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     const bool active = i < a.a1;
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
@@ -350,15 +362,24 @@ k_edge_backward(const EdgeArgs a) {
         for (int base = e0; base < e1; base += 32) {
             const int e = base + lane;
             const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
-            const int nb = min(32, e1 - base);
-            for (int it = 0; it * W::EPI < nb; ++it) {
-                const int b = it * W::EPI + sub;
-                const bool v = __shfl_sync(kFull, (int)g.valid, b) != 0;
-                const int row = __shfl_sync(kFull, g.row, b);
-                const int pair = __shfl_sync(kFull, g.pair, b);
-                const float t = __shfl_sync(kFull, g.t, b);
+            edge_s[lane] = make_int4(g.row, g.pair, __float_as_int(g.t), 0);
+            const unsigned vmask = __ballot_sync(kFull, g.valid);
+            const int nvalid = __popc(vmask);
+            __syncwarp();
+            unsigned mrun = vmask;
+            for (int it = 0; it * W::EPI < nvalid; ++it) {
+                int b;
+                if (W::EPI == 1) { b = __ffs(mrun) - 1; mrun &= mrun - 1; }
+                else {
+                    const int idx = it * W::EPI + sub;
+                    if (idx >= nvalid) continue;
+                    b = (int)__fns(vmask, 0, idx + 1);
+                }
+                const int4 es = edge_s[b];
+                const int row = es.x, pair = es.y;
+                const float t = __int_as_float(es.z);
                 float pa = 0.f, pb = 0.f;
-                if (v) {
+                {
                     float psi[4], dpsi[4];
                     amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi);
 #pragma unroll
