@@ -37,7 +37,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from workloads import CONFIGS, make_system, workload_blob  # noqa: E402
+from workloads import CONFIGS, make_system, workload_blob, workload_profile  # noqa: E402
 
 DEFAULT_WORKLOAD = "cfg5_amorphous1m"
 SM_COUNT = 148
@@ -162,7 +162,7 @@ class OracleSampler:
     """The fp64 oracle on bounded samples of a workload: brute-force neighbor rows of the
     sampled atoms plus their energies and edge gradients.  Rate = atom evaluations / s."""
 
-    def __init__(self, name):
+    def __init__(self, name, modes=None):
         import torch
 
         from oracle import dpa4c as orc
@@ -170,7 +170,7 @@ class OracleSampler:
         cfg = CONFIGS[name]
         self.name = name
         self.s = make_system(cfg["system"])
-        self.o = orc.Oracle(workload_blob(name))
+        self.o = orc.Oracle(workload_blob(name, modes))
         self.rc = cfg["profile"]["rc"]
         self.N = len(self.s["pos"])
         self.pos = orc.wrap_positions(self.s["pos"], self.s["cell"], self.s["pbc"])
@@ -193,7 +193,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    smp = OracleSampler(args.workload)
+    smp = OracleSampler(args.workload, args.modes if args.modes >= 0 else None)
     total_steps = max(1, args.steps + args.warmup)
     n = smp.sized_for(min(20.0, 150.0 / total_steps))
     for w in range(args.warmup):
@@ -229,7 +229,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     name = args.workload
     cfg = CONFIGS[name]
-    p = cfg["profile"]
+    modes = args.modes if args.modes >= 0 else None
+    p = workload_profile(name, modes)
     # a workload without an MD recipe is timed as repeated single evaluations (energy + forces +
     # virial of the same frame, list built once): velocities are zero and nothing moves
     static = cfg["md"] is None
@@ -244,7 +245,9 @@ def run_ours(args):
         name = f"{name}[atoms={int(args.atoms)}]"
     s = make_system(desc, None if static else md)
     N = len(s["pos"])
-    blob = workload_blob(args.workload)
+    blob = workload_blob(args.workload, modes)
+    if modes is not None:
+        name = f"{name}[R={modes}]"
     model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile)
     pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
     pos = pos0.cuda().contiguous()
@@ -345,7 +348,7 @@ def run_ours(args):
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        smp = OracleSampler(args.workload)
+        smp = OracleSampler(args.workload, args.modes if args.modes >= 0 else None)
         n_s = smp.sized_for(args.cpu_seconds)
         t_s = smp.run(n_s, offset=8)
         cpu = dict(value=n_s / t_s, unit="atom-steps/s", cores=smp.cores, kind="oracle",
@@ -393,6 +396,7 @@ def main():
     ap.add_argument("--mlp-path", type=int, default=0)
     ap.add_argument("--node-tile", type=int, default=0)
     ap.add_argument("--atoms", type=int, default=0, help="amorphous workload only: atoms of a smaller box of the same recipe")
+    ap.add_argument("--modes", type=int, default=-1, help="override the number R of shared radial modes of the workload's profile")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -17,13 +17,14 @@ def _binding():
     return binding
 
 
-@pytest.mark.parametrize("name,n_force,n_rows", [("cfg3_water32400", 3, 48), ("cfg4_hea128k", 3, 48),
-                                                 ("cfg5_amorphous1m", 2, 24)])
-def test_fullsize_sampled_parity(name, n_force, n_rows):
+@pytest.mark.parametrize("name,n_force,n_rows,modes", [("cfg3_water32400", 3, 48, None), ("cfg4_hea128k", 3, 48, None),
+                                                       ("cfg5_amorphous1m", 2, 24, None),
+                                                       ("cfg3_water32400", 2, 24, 4)])   # R = 4: the profile with shared radial modes
+def test_fullsize_sampled_parity(name, n_force, n_rows, modes):
     cfg = CONFIGS[name]
     s = make_system(cfg["system"])
     N = len(s["pos"])
-    blob = workload_blob(name)
+    blob = workload_blob(name, modes)
     skin = cfg["md"]["skin"]
     m = _binding().Model(blob)
     pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()

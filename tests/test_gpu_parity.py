@@ -218,13 +218,15 @@ def test_stale_list_is_reported():
     m.compute(pos)                         # the handle stays usable
 
 
+@pytest.mark.parametrize("path", [2, 3])
 @pytest.mark.parametrize("name", ["p16_3_2", "p32_2_4", "p32_2_0_res"])
-def test_tensor_core_mlp_path_small_profiles(name):
+def test_tensor_core_mlp_path_small_profiles(name, path):
+    # both tensor-core GEMM variants (2: persistent 256-row items, 3: one tile per CTA) with
     # ragged everything: fewer rows than a tile, widths that are not multiples of the tile
     p = SMALL_PROFILES[name]
     blob = make_blob(p, seed=45, bias_scale=0.2, e_ref_scale=0.5)
     s = make_system(dict(SYS_SMALL, n_types=p["T"], atoms=150, edges=(12.5, 13.5, 14.0)))
-    _compare(blob, s, check_intermediates=False, mlp_path=2)
+    _compare(blob, s, check_intermediates=False, mlp_path=path)
 
 
 def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
@@ -232,14 +234,19 @@ def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
     s = make_system(CONFIGS[name]["system"])
     blob = workload_blob(name)
     outs = []
-    for path in (1, 2):
-        m, pos = _build(blob, s, mlp_path=path, node_tile=1536)    # three tiles, ragged last one
+    for path in (1, 2, 3):
+        m, pos = _build(blob, s, mlp_path=path, node_tile=1536)    # three tiles, ragged last one (928 = 3 * 256 + 160 rows)
         outs.append(m.compute(pos, atom_energy=True))
         m.close()
-    a, b = outs
+    a = outs[0]
     e_scale = a["atom_energy"].abs().max().item()
     f_scale = a["forces"].abs().max().item()
-    # the tensor core truncates when it aligns partial sums, a ~2e-6 relative one-sided bias
-    assert (a["atom_energy"] - b["atom_energy"]).abs().max().item() <= 5e-6 * e_scale
-    assert (a["forces"] - b["forces"]).abs().max().item() <= 1e-5 * f_scale
-    assert np.abs(a["virial"] - b["virial"]).max() <= 1e-5 * np.abs(a["virial"]).max()
+    for b in outs[1:]:
+        # the tensor core truncates when it aligns partial sums, a ~2e-6 relative one-sided bias
+        assert (a["atom_energy"] - b["atom_energy"]).abs().max().item() <= 5e-6 * e_scale
+        assert (a["forces"] - b["forces"]).abs().max().item() <= 1e-5 * f_scale
+        assert np.abs(a["virial"] - b["virial"]).max() <= 1e-5 * np.abs(a["virial"]).max()
+    # the two tensor-core variants issue the same products in the same order per output element;
+    # only the head's partial sums are grouped differently
+    assert (outs[1]["forces"] - outs[2]["forces"]).abs().max().item() <= 1e-7 * f_scale
+    assert (outs[1]["atom_energy"] - outs[2]["atom_energy"]).abs().max().item() <= 1e-6 * e_scale
