@@ -30,7 +30,8 @@ from oracle import dpa4c as orc
 from workloads import CONFIGS, make_blob, make_system
 
 SAMPLE = {"cfg1_al108": 108, "cfg2_cu4000": 512, "cfg3_water32400": 384, "cfg4_hea128k": 160,
-          "cfg5_amorphous1m": 96}
+          "cfg5_amorphous1m": 96, "paper_nano_c1m": 64, "paper_mini_c1m": 64, "paper_neo_c1m": 64,
+          "paper_air_c1m": 64, "paper_plus_c1m": 64}
 SCALE_FLOOR = 1.0e-3
 OUT_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "workloads", "calibration")
 

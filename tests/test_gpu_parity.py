@@ -18,7 +18,7 @@ import pytest
 import torch
 
 from oracle import dpa4c as orc
-from workloads import CONFIGS, SMALL_PROFILES, make_blob, make_system, workload_blob
+from workloads import CONFIGS, SMALL_PROFILES, load_calibration, make_blob, make_system, workload_blob
 
 pytestmark = pytest.mark.gpu
 
@@ -227,6 +227,18 @@ def test_tensor_core_mlp_path_small_profiles(name, path):
     blob = make_blob(p, seed=45, bias_scale=0.2, e_ref_scale=0.5)
     s = make_system(dict(SYS_SMALL, n_types=p["T"], atoms=150, edges=(12.5, 13.5, 14.0)))
     _compare(blob, s, check_intermediates=False, mlp_path=path)
+
+
+@pytest.mark.parametrize("name", ["paper_nano_c1m", "paper_air_c1m", "paper_plus_c1m"])
+def test_paper_variants_on_small_diamond_cell(name):
+    # the paper's model variants (118-species type table, carbon only) on a 512-atom cell of its
+    # jittered-diamond workload: 158 neighbours per atom, box < 2 (r_c + skin)
+    cfg = CONFIGS[name]
+    s = make_system(dict(cfg["system"], cells=4))
+    blob = make_blob(cfg["profile"], seed=cfg["weights_seed"], calibration=load_calibration(name), bias_scale=0.1,
+                     e_ref_scale=0.5)
+    _compare(blob, s, check_intermediates=False)
+    _compare(blob, s, check_intermediates=False, skin=1.0)
 
 
 def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():

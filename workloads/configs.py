@@ -88,6 +88,39 @@ CONFIGS = {
     ),
 }
 
+# The paper's own throughput workload: jittered diamond carbon (a = 3.567, sigma = 0.03, seed 0; 158
+# neighbours within 6 A), 50^3 conventional cells = 1,000,000 atoms, with its five model variants
+# (C0, L, R, F) = Nano (8,2,0,96), Mini (32,2,0,192), Neo (64,2,0,256), Air (64,3,4,256), Plus
+# (128,3,4,384); three hidden layers, 16 radial functions, a 118-species type table of which only
+# carbon (index 5) occurs.  ``published`` is the paper's rate at 1,000,000 atoms on one H20 (complete
+# NVT steps in LAMMPS/Kokkos, trained weights): context for the rate measured here with random
+# weights and the library's own NVE driver, not a like-for-like target.
+def _paper_variant(index, seed, published, *profile_args, **profile_kw):
+    return dict(
+        index=index,
+        system=dict(kind="diamond", cells=50, a=3.567, jitter=0.03, seed=0, n_types=118, type_index=5,
+                    masses=[12.011] * 118),
+        profile=_profile(*profile_args, **profile_kw),
+        weights_seed=seed, head_scale=-0.02,
+        md=dict(steps=100, dt_ps=0.001, temperature=300.0, seed=8, rebuild_every=10, skin=1.0),
+        published=dict(value=published, unit="atom-steps/s", hardware="1x NVIDIA H20, fp32",
+                       source="paper, supplementary table of rates at 1,000,000 atoms"),
+    )
+
+
+CONFIGS.update({
+    "paper_nano_c1m": _paper_variant(5, 21, 16.72e6, 8, 2, 0, 16, 3, 96, 118, C1=4, C2=4, K1=4, K2=2,
+                                     H=24, Hp=48, S=40, D_out=70),
+    "paper_mini_c1m": _paper_variant(6, 22, 10.37e6, 32, 2, 0, 16, 3, 192, 118, C1=8, C2=4, K1=4, K2=2,
+                                     H=88, Hp=176, S=76, D_out=144),
+    "paper_neo_c1m": _paper_variant(7, 23, 7.12e6, 64, 2, 0, 16, 3, 256, 118, C1=8, C2=4, K1=4, K2=2,
+                                    H=176, Hp=344, S=108, D_out=208),
+    "paper_air_c1m": _paper_variant(8, 24, 3.82e6, 64, 3, 4, 16, 3, 256, 118, C1=8, C2=4, K1=4, K2=2,
+                                    H=176, Hp=344, S=115, D_out=219),
+    "paper_plus_c1m": _paper_variant(9, 25, 2.16e6, 128, 3, 4, 16, 3, 384, 118, C1=16, C2=8, K1=8, K2=2,
+                                     H=344, Hp=688, S=223, D_out=541),
+})
+
 # Small profiles for unit and parity tests (shape coverage: identity A_1 at the two
 # narrowest widths, R > 0, L = 3, several species).
 SMALL_PROFILES = {

@@ -15,6 +15,7 @@ EV_PER_AMU_IN_A2_PS2 = 9648.53321
 
 _FCC_BASIS = np.array([[0.0, 0.0, 0.0], [0.5, 0.5, 0.0], [0.5, 0.0, 0.5], [0.0, 0.5, 0.5]])
 _BCC_BASIS = np.array([[0.0, 0.0, 0.0], [0.5, 0.5, 0.5]])
+_DIAMOND_BASIS = np.concatenate([_FCC_BASIS, _FCC_BASIS + 0.25])
 
 
 def _lattice(basis, cells, a):
@@ -149,11 +150,15 @@ def make_system(desc, md=None):
     rng = np.random.Generator(np.random.PCG64(desc["seed"]))
     pbc = np.array(desc.get("pbc", [1, 1, 1]), dtype=np.int32)
     n_types = desc["n_types"]
-    if kind in ("fcc", "bcc"):
-        basis = _FCC_BASIS if kind == "fcc" else _BCC_BASIS
+    if kind in ("fcc", "bcc", "diamond"):
+        basis = {"fcc": _FCC_BASIS, "bcc": _BCC_BASIS, "diamond": _DIAMOND_BASIS}[kind]
         pos, cell = _lattice(basis, desc["cells"], desc["a"])
-        types = rng.integers(0, n_types, size=len(pos)).astype(np.int32) if n_types > 1 \
-            else np.zeros(len(pos), dtype=np.int32)
+        if "type_index" in desc:         # one species out of a larger type table
+            types = np.full(len(pos), desc["type_index"], dtype=np.int32)
+        elif n_types > 1:
+            types = rng.integers(0, n_types, size=len(pos)).astype(np.int32)
+        else:
+            types = np.zeros(len(pos), dtype=np.int32)
         pos = pos + rng.standard_normal(pos.shape) * desc["jitter"]
     elif kind == "water":
         nmol = desc["molecules"]
