@@ -28,7 +28,18 @@ struct Grid {
     int nc[3];          // bins per direction
     int m[3];           // bin reach per direction
     int pbc[3];
+    int sorted;         // every periodic direction has at least 2 m + 1 bins: bins are visited in
+                        // increasing bin index, so each row comes out sorted by neighbour index
 };
+
+// first offset of the walk over the 2 m + 1 bins around bin c of a direction: the one whose wrapped
+// bin index is smallest, so that the walk (continuing cyclically) visits bins in increasing index
+__device__ __forceinline__ int walk_start(int c, int m, int nc, int pbc, int sorted) {
+    if (!sorted || !pbc) return -m;
+    if (c - m < 0) return -c;
+    if (c + m >= nc) return nc - c;
+    return -m;
+}
 
 __device__ __forceinline__ int floor_div(int a, int b) {
     int q = a / b;
@@ -118,17 +129,27 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     int count = 0;
     const int base_out = FILL ? row_ptr[i] : 0;
     const unsigned lt_mask = (1u << lane) - 1u;
-    for (int dz = -g.m[2]; dz <= g.m[2]; ++dz) {
+    const int wz = 2 * g.m[2] + 1, wy = 2 * g.m[1] + 1, wx = 2 * g.m[0] + 1;
+    const int sz0 = walk_start(cz, g.m[2], g.nc[2], g.pbc[2], g.sorted);
+    const int sy0 = walk_start(cy, g.m[1], g.nc[1], g.pbc[1], g.sorted);
+    const int sx0 = walk_start(cx, g.m[0], g.nc[0], g.pbc[0], g.sorted);
+    for (int tz = 0; tz < wz; ++tz) {
+        int dz = sz0 + tz;
+        if (dz > g.m[2]) dz -= wz;
         int zc = cz + dz, nz = 0;
         if (g.pbc[2]) { nz = floor_div(zc, g.nc[2]); zc -= nz * g.nc[2]; }
         else if (zc < 0 || zc >= g.nc[2]) continue;
         const double sz = __dmul_rn((double)nz, g.L[2]);
-        for (int dy = -g.m[1]; dy <= g.m[1]; ++dy) {
+        for (int ty = 0; ty < wy; ++ty) {
+            int dy = sy0 + ty;
+            if (dy > g.m[1]) dy -= wy;
             int yc = cy + dy, ny = 0;
             if (g.pbc[1]) { ny = floor_div(yc, g.nc[1]); yc -= ny * g.nc[1]; }
             else if (yc < 0 || yc >= g.nc[1]) continue;
             const double sy = __dmul_rn((double)ny, g.L[1]);
-            for (int dx = -g.m[0]; dx <= g.m[0]; ++dx) {
+            for (int tx = 0; tx < wx; ++tx) {
+                int dx = sx0 + tx;
+                if (dx > g.m[0]) dx -= wx;
                 int xc = cx + dx, nx = 0;
                 if (g.pbc[0]) { nx = floor_div(xc, g.nc[0]); xc -= nx * g.nc[0]; }
                 else if (xc < 0 || xc >= g.nc[0]) continue;
@@ -165,7 +186,7 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
 
 // rev[e] = slot of (j <- i, -n) for e = (i <- j, n); -1 when absent (can only happen for
 // pairs whose two orientations round to opposite sides of the list radius).
-__global__ void k_reverse_map(int N, const int* __restrict__ row_ptr, const int* __restrict__ src,
+__global__ void k_reverse_map(int N, int sorted, const int* __restrict__ row_ptr, const int* __restrict__ src,
                               const int* __restrict__ shift, int* __restrict__ rev) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -180,8 +201,17 @@ __global__ void k_reverse_map(int N, const int* __restrict__ row_ptr, const int*
         const int want = pack_shift(-nx, -ny, -nz);
         int found = -1;
         const int f0 = row_ptr[j], f1 = row_ptr[j + 1];
-        for (int f = f0; f < f1; ++f) {
-            if (src[f] == i && shift[f] == want) { found = f; break; }
+        if (sorted) {          // rows ascend in the neighbour index, each neighbour at most once
+            int lo = f0, hi = f1;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (src[mid] < i) lo = mid + 1; else hi = mid;
+            }
+            if (lo < f1 && src[lo] == i && shift[lo] == want) found = lo;
+        } else {
+            for (int f = f0; f < f1; ++f) {
+                if (src[f] == i && shift[f] == want) { found = f; break; }
+            }
         }
         rev[e] = found;
     }
@@ -301,6 +331,9 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
         if (g.m[k] > 127) { *err = "cell much smaller than the list radius (more than 127 images)"; return UMLMD_E_UNSUPPORTED_CELL; }
         ncell *= g.nc[k];
     }
+    g.sorted = 1;
+    for (int k = 0; k < 3; ++k)
+        if (g.pbc[k] && g.nc[k] < 2 * g.m[k] + 1) g.sorted = 0;
 
     nb->N = N; nb->skin = skin; nb->r_list = r_list;
     for (int k = 0; k < 3; ++k) { nb->L[k] = L[k]; nb->pbc[k] = pbc[k] ? 1 : 0; }
@@ -370,7 +403,7 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     if (total > 0) {
         k_scan_cells<true><<<wb, TB, 0, st>>>(N, g, rl2, nb->key2, nb->cell_start, nb->xs0, nullptr,
                                               nb->row_ptr, nb->src, nb->shift, d_err);
-        k_reverse_map<<<wb, TB, 0, st>>>(N, nb->row_ptr, nb->src, nb->shift, nb->rev);
+        k_reverse_map<<<wb, TB, 0, st>>>(N, g.sorted, nb->row_ptr, nb->src, nb->shift, nb->rev);
     }
     NB_CHECK(cudaGetLastError());
     return UMLMD_OK;
