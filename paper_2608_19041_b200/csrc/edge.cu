@@ -158,6 +158,7 @@ template <int C0, int L> struct Widths {
     static constexpr int C1 = C0 <= 16 ? 4 : (C0 <= 64 ? 8 : 16);
     static constexpr int C2 = C1 / 2 > 4 ? C1 / 2 : 4;
     static constexpr int LPE = C0 / 4;          // lanes per edge in the channel-parallel phase
+    static constexpr int LH = LPE / 2;          // parked partial dot products per edge (lanes paired)
     static constexpr int EPI = 32 / LPE;        // edges per replay step
     static constexpr int NL1 = C1 / 4;          // lanes of a group that hold degree-1 channels
     static constexpr int NHI = 3 * C1 + 5 * C2 + (L >= 3 ? 7 : 0);   // sums of degree >= 1
@@ -170,14 +171,17 @@ template <int C0, int L> struct Widths {
 
 template <int C0, int L> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L>;
-    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LPE + 1) + W::NHI + 3) / 4 * 4 + 32 * 4;   // floats
+    static constexpr int queue_floats = 64 * 4 + 5 * 64;    // queue of in-range edges: int4 and five scalars per slot
+    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LH + 1) + W::NHI + 3) / 4 * 4 + queue_floats;   // floats
     static constexpr size_t bytes = kWarpsPerBlock * 9 * sizeof(double) + sizeof(float) * kWarpsPerBlock * per_warp;
 };
 
 // ------------------------------------------------------------------------------- forward
 //
-// Per batch of 32 edges:
-//   1. lane = edge: geometry.
+// The row is scanned 32 listed edges at a time (lane = edge: geometry); the edges that fall
+// inside the cutoff are appended to a per-warp queue in shared memory, and whenever the queue
+// holds 32 of them (and once more at the end of the row) a full batch is processed, so the
+// later phases never run on skin-shell edges:
 //   2. lanes = channels (a group of C0/4 lanes per edge): amplitude psi of all C0 channels,
 //      degree-0 sums accumulated in registers; the leading C1 amplitudes of each edge are
 //      parked in shared memory.
@@ -191,16 +195,23 @@ k_edge_forward(const EdgeArgs a) {
     // one 32 x 33 float scratch per warp: first the parked amplitudes (row pitch PF), then,
     // once every lane has read its own row, the transpose buffer
     __shared__ __align__(16) float scratch[kWarpsPerBlock][32 * 33];
-    __shared__ int4 edge_s[kWarpsPerBlock][32];         // per-edge scalars of the batch: row, pair, t, chi
+    // queue of edges inside the cutoff: row, pair, t, chi (fetched with one 16-byte broadcast
+    // load in the channel-parallel phase; shuffles would go through the same L1 data pipe as
+    // the table reads) and the edge vector
+    __shared__ int4 q_es[kWarpsPerBlock][64];
+    __shared__ float q_d[kWarpsPerBlock][3 * 64];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     if (i >= a.a1) return;
     float* const psi_s = scratch[wid];      // [32][PF]
     float* const tr = scratch[wid];         // [32][33]
+    int4* const qes = q_es[wid];
+    float* const qd = q_d[wid];
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
     const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
     const int ti = a.type_s[i];
     const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
+    const unsigned lt_mask = (1u << lane) - 1u;
 
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
     float accH[W::NCH];
@@ -208,26 +219,11 @@ k_edge_forward(const EdgeArgs a) {
     for (int j = 0; j < W::NCH; ++j) accH[j] = 0.f;
     double s0 = 0.0, s1 = 0.0;   // normaliser sums in double: the calibration subtracts their mean
 
-    for (int base = e0; base < e1; base += 32) {
-        const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
-        if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
-        // The channel-parallel phase visits only the edges inside the cutoff; their scalars
-        // are parked in shared memory and fetched with one 16-byte broadcast load (shuffles
-        // would go through the same L1 data pipe as the table reads, five at a time).
-        edge_s[wid][lane] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
-        const unsigned vmask = __ballot_sync(kFull, g.valid);
-        const int nvalid = __popc(vmask);
-        __syncwarp();
-        unsigned mrun = vmask;
-        for (int it = 0; it * W::EPI < nvalid; ++it) {
-            int b;
-            if (W::EPI == 1) { b = __ffs(mrun) - 1; mrun &= mrun - 1; }      // next edge inside the cutoff
-            else {
-                const int idx = it * W::EPI + sub;
-                if (idx >= nvalid) continue;
-                b = (int)__fns(vmask, 0, idx + 1);
-            }
-            const int4 es = edge_s[wid][b];
+    auto run_batch = [&](const int nb) {     // the first nb queue slots
+        for (int it = 0; it * W::EPI < nb; ++it) {
+            const int b = it * W::EPI + sub;
+            if (b >= nb) continue;
+            const int4 es = qes[b];
             const int row = es.x, pair = es.y;
             const float t = __int_as_float(es.z), chi = __int_as_float(es.w);
             float psi[4];
@@ -242,14 +238,17 @@ k_edge_forward(const EdgeArgs a) {
         float ps[W::C1];
         float B1[3], B2[5], B3[7];
         float w = 0.f;
-        if (g.valid) {
+        if (lane < nb) {
 #pragma unroll
             for (int q = 0; q < W::C1 / 4; ++q) {
                 const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PF + 4 * q);
                 ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
             }
-            harmonics_s1<L>(g.ux, g.uy, g.uz, B1, B2, B3);
-            w = g.chi * g.chi;
+            const float dx = qd[lane], dy = qd[64 + lane], dz = qd[128 + lane];
+            const float inv_rho = 1.0f / sqrtf(dx * dx + dy * dy + dz * dz + kEpsReg * kEpsReg);
+            harmonics_s1<L>(dx * inv_rho, dy * inv_rho, dz * inv_rho, B1, B2, B3);
+            const float chi = __int_as_float(qes[lane].w);
+            w = chi * chi;
         } else {
 #pragma unroll
             for (int q = 0; q < W::C1; ++q) ps[q] = 0.f;
@@ -290,7 +289,34 @@ k_edge_forward(const EdgeArgs a) {
 #pragma unroll
             for (int m = 0; m < 7; ++m) emit(w * B3[m] * ps[0]);
         }
+    };
+
+    int qn = 0;
+    for (int base = e0; base < e1; base += 32) {
+        const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
+        const unsigned vmask = __ballot_sync(kFull, g.valid);
+        if (g.valid) {
+            const double c2 = (double)g.chi * (double)g.chi;
+            s0 += c2; s1 += c2 * c2;
+            const int p = qn + __popc(vmask & lt_mask);
+            qes[p] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
+            qd[p] = g.dx; qd[64 + p] = g.dy; qd[128 + p] = g.dz;
+        }
+        qn += __popc(vmask);
+        __syncwarp();
+        if (qn >= 32) {
+            run_batch(32);
+            const int rem = qn - 32;            // move the tail of the queue to its front
+            int4 tes = make_int4(0, 0, 0, 0);
+            float t0 = 0.f, t1 = 0.f, t2 = 0.f;
+            if (lane < rem) { tes = qes[32 + lane]; t0 = qd[32 + lane]; t1 = qd[96 + lane]; t2 = qd[160 + lane]; }
+            __syncwarp();
+            if (lane < rem) { qes[lane] = tes; qd[lane] = t0; qd[64 + lane] = t1; qd[128 + lane] = t2; }
+            __syncwarp();
+            qn = rem;
+        }
     }
+    if (qn > 0) run_batch(qn);
     // combine the edge slots of the warp (lanes with equal channel offset)
 #pragma unroll
     for (int off = W::LPE; off < 32; off <<= 1) {
@@ -318,11 +344,12 @@ k_edge_forward(const EdgeArgs a) {
 
 // ------------------------------------------------------------------------------ backward
 //
-// Same three phases.  The channel-parallel phase produces, per edge, the two degree-0 dot
-// products sum_c G0_c psi_c and sum_c G0_c dpsi_c (partial sums parked in shared memory and
-// finished by the edge's own lane) and parks psi, dpsi of the leading C1 channels; the
-// edge's lane then does the whole degree >= 1 contraction by itself against the
-// destination's gradient block held in shared memory, and assembles dE/dr_ij.
+// Same scan, queue and phases.  The channel-parallel phase produces, per edge, the two
+// degree-0 dot products sum_c G0_c psi_c and sum_c G0_c dpsi_c (partial sums parked in shared
+// memory and finished by the edge's own lane) and parks psi, dpsi of the leading C1 channels;
+// the edge's lane then does the whole degree >= 1 contraction by itself against the
+// destination's gradient block held in shared memory, and assembles dE/dr_ij.  Edges in the
+// skin shell get a zero gradient as soon as their geometry is known.
 template <int C0, int L, bool HASR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_backward(const EdgeArgs a) {
@@ -332,12 +359,15 @@ k_edge_backward(const EdgeArgs a) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float* const wbase = reinterpret_cast<float*>(dsm + kWarpsPerBlock * 9 * sizeof(double)) + wid * BwdSmem<C0, L>::per_warp;
     float* const psi_s = wbase;                                  // [32][PB]: psi, dpsi of the leading channels
-    float* const red = psi_s + 32 * W::PB;                       // [2][32][LPE+1] partial dot products
-    float* const hi_s = red + 2 * 32 * (W::LPE + 1);             // [NHI] gradient of the degree >= 1 sums
-    int4* const edge_s = reinterpret_cast<int4*>(wbase + BwdSmem<C0, L>::per_warp - 32 * 4);   // [32] row, pair, t of the batch
+    float* const red = psi_s + 32 * W::PB;                       // [2][32][LH+1] partial dot products
+    float* const hi_s = red + 2 * 32 * (W::LH + 1);              // [NHI] gradient of the degree >= 1 sums
+    // queue of edges inside the cutoff: (row, pair, t, chi), then dx, dy, dz, dchi, edge index
+    int4* const qes = reinterpret_cast<int4*>(wbase + BwdSmem<C0, L>::per_warp - BwdSmem<C0, L>::queue_floats);
+    float* const qd = reinterpret_cast<float*>(qes + 64);        // [5][64]
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     const bool active = i < a.a1;
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
+    const unsigned lt_mask = (1u << lane) - 1u;
     float vir[9];
 #pragma unroll
     for (int k = 0; k < 9; ++k) vir[k] = 0.f;
@@ -359,27 +389,15 @@ k_edge_backward(const EdgeArgs a) {
         const float* H2 = H1 + 3 * W::C1;
         const float* H3 = H2 + 5 * W::C2;
 
-        for (int base = e0; base < e1; base += 32) {
-            const int e = base + lane;
-            const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
-            edge_s[lane] = make_int4(g.row, g.pair, __float_as_int(g.t), 0);
-            const unsigned vmask = __ballot_sync(kFull, g.valid);
-            const int nvalid = __popc(vmask);
-            __syncwarp();
-            unsigned mrun = vmask;
-            for (int it = 0; it * W::EPI < nvalid; ++it) {
-                int b;
-                if (W::EPI == 1) { b = __ffs(mrun) - 1; mrun &= mrun - 1; }
-                else {
-                    const int idx = it * W::EPI + sub;
-                    if (idx >= nvalid) continue;
-                    b = (int)__fns(vmask, 0, idx + 1);
-                }
-                const int4 es = edge_s[b];
-                const int row = es.x, pair = es.y;
-                const float t = __int_as_float(es.z);
+        auto run_batch = [&](const int nb) {     // the first nb queue slots
+            for (int it = 0; it * W::EPI < nb; ++it) {
+                const int b = it * W::EPI + sub;
+                const bool act = b < nb;
                 float pa = 0.f, pb = 0.f;
-                {
+                if (act) {
+                    const int4 es = qes[b];
+                    const int row = es.x, pair = es.y;
+                    const float t = __int_as_float(es.z);
                     float psi[4], dpsi[4];
                     amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi);
 #pragma unroll
@@ -389,72 +407,118 @@ k_edge_backward(const EdgeArgs a) {
                         *reinterpret_cast<float4*>(psi_s + b * W::PB + W::C1 + c) = make_float4(dpsi[0], dpsi[1], dpsi[2], dpsi[3]);
                     }
                 }
-                red[b * (W::LPE + 1) + cl] = pa;
-                red[(32 + b) * (W::LPE + 1) + cl] = pb;
+                // neighbouring lanes are paired before the partial sums are parked, which halves
+                // the parking area (it decides how many blocks fit on an SM)
+                pa += __shfl_xor_sync(kFull, pa, 1);
+                pb += __shfl_xor_sync(kFull, pb, 1);
+                if (act && !(cl & 1)) {
+                    red[b * (W::LH + 1) + (cl >> 1)] = pa;
+                    red[(32 + b) * (W::LH + 1) + (cl >> 1)] = pb;
+                }
             }
             __syncwarp();
-            if (e < e1) {
-                float gx = 0.f, gy = 0.f, gz = 0.f;
-                if (g.valid) {
-                    float sa = 0.f, sb = 0.f;
+            if (lane < nb) {
+                const float gdx = qd[lane], gdy = qd[64 + lane], gdz = qd[128 + lane], dchi = qd[192 + lane];
+                const int e = __float_as_int(qd[256 + lane]);
+                const float chi = __int_as_float(qes[lane].w);
+                const float inv_rho = 1.0f / sqrtf(gdx * gdx + gdy * gdy + gdz * gdz + kEpsReg * kEpsReg);
+                const float gux = gdx * inv_rho, guy = gdy * inv_rho, guz = gdz * inv_rho;
+                float sa = 0.f, sb = 0.f;
 #pragma unroll
-                    for (int j = 0; j < W::LPE; ++j) { sa += red[lane * (W::LPE + 1) + j]; sb += red[(32 + lane) * (W::LPE + 1) + j]; }
-                    float ps[W::C1], dps[W::C1], ec[W::C1];
+                for (int j = 0; j < W::LH; ++j) { sa += red[lane * (W::LH + 1) + j]; sb += red[(32 + lane) * (W::LH + 1) + j]; }
+                float ps[W::C1], dps[W::C1], ec[W::C1];
 #pragma unroll
-                    for (int q = 0; q < W::C1 / 4; ++q) {
-                        const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + 4 * q);
-                        const float4 d4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + W::C1 + 4 * q);
-                        ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
-                        dps[4 * q] = d4.x; dps[4 * q + 1] = d4.y; dps[4 * q + 2] = d4.z; dps[4 * q + 3] = d4.w;
-                    }
-#pragma unroll
-                    for (int k = 0; k < W::C1; ++k) ec[k] = 0.f;
-                    float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
-                    harmonics_s1<L>(g.ux, g.uy, g.uz, B1, B2, B3);
-                    float bt = 0.f;    // sum_lm B_lm t_lm,  t_lm = sum_c psi_c G_lmc
-#pragma unroll
-                    for (int m = 0; m < 3; ++m) {
-                        float tm = 0.f;
-#pragma unroll
-                        for (int k = 0; k < W::C1; ++k) { const float hv = H1[m * W::C1 + k]; tm += ps[k] * hv; ec[k] += B1[m] * hv; }
-                        t1[m] = tm; bt += B1[m] * tm;
-                    }
-#pragma unroll
-                    for (int m = 0; m < 5; ++m) {
-                        float tm = 0.f;
-#pragma unroll
-                        for (int k = 0; k < W::C2; ++k) { const float hv = H2[m * W::C2 + k]; tm += ps[k] * hv; ec[k] += B2[m] * hv; }
-                        t2[m] = tm; bt += B2[m] * tm;
-                    }
-#pragma unroll
-                    for (int m = 0; m < 7; ++m) {
-                        float tm = 0.f;
-                        if (L >= 3) { const float hv = H3[m]; tm = ps[0] * hv; ec[0] += B3[m] * hv; bt += B3[m] * tm; }
-                        t3[m] = tm;
-                    }
-                    const float w = g.chi * g.chi;
-                    float pr1 = 0.f;
-#pragma unroll
-                    for (int k = 0; k < W::C1; ++k) pr1 += ec[k] * dps[k];
-                    float ux, uy, uz;
-                    harmonics_grad_contract<L>(g.ux, g.uy, g.uz, t1, t2, t3, &ux, &uy, &uz);
-                    const float pux = w * ux, puy = w * uy, puz = w * uz;
-                    const float p_rho = g.chi * sa + w * pr1;
-                    const float p_chi = sb + 2.0f * g.chi * bt;
-                    const float dEdrho = p_rho + (p_chi + 2.0f * g.chi * ds0 + 4.0f * w * g.chi * ds1) * g.dchi;
-                    const float dot = pux * g.ux + puy * g.uy + puz * g.uz;
-                    gx = dEdrho * g.ux + (pux - dot * g.ux) * g.inv_rho;
-                    gy = dEdrho * g.uy + (puy - dot * g.uy) * g.inv_rho;
-                    gz = dEdrho * g.uz + (puz - dot * g.uz) * g.inv_rho;
-                    vir[0] += gx * g.dx; vir[1] += gx * g.dy; vir[2] += gx * g.dz;
-                    vir[3] += gy * g.dx; vir[4] += gy * g.dy; vir[5] += gy * g.dz;
-                    vir[6] += gz * g.dx; vir[7] += gz * g.dy; vir[8] += gz * g.dz;
+                for (int q = 0; q < W::C1 / 4; ++q) {
+                    const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + 4 * q);
+                    const float4 d4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PB + W::C1 + 4 * q);
+                    ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
+                    dps[4 * q] = d4.x; dps[4 * q + 1] = d4.y; dps[4 * q + 2] = d4.z; dps[4 * q + 3] = d4.w;
                 }
+#pragma unroll
+                for (int k = 0; k < W::C1; ++k) ec[k] = 0.f;
+                float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
+                harmonics_s1<L>(gux, guy, guz, B1, B2, B3);
+                float bt = 0.f;    // sum_lm B_lm t_lm,  t_lm = sum_c psi_c G_lmc
+#pragma unroll
+                for (int m = 0; m < 3; ++m) {
+                    float tm = 0.f;
+#pragma unroll
+                    for (int k = 0; k < W::C1; ++k) { const float hv = H1[m * W::C1 + k]; tm += ps[k] * hv; ec[k] += B1[m] * hv; }
+                    t1[m] = tm; bt += B1[m] * tm;
+                }
+#pragma unroll
+                for (int m = 0; m < 5; ++m) {
+                    float tm = 0.f;
+#pragma unroll
+                    for (int k = 0; k < W::C2; ++k) { const float hv = H2[m * W::C2 + k]; tm += ps[k] * hv; ec[k] += B2[m] * hv; }
+                    t2[m] = tm; bt += B2[m] * tm;
+                }
+#pragma unroll
+                for (int m = 0; m < 7; ++m) {
+                    float tm = 0.f;
+                    if (L >= 3) { const float hv = H3[m]; tm = ps[0] * hv; ec[0] += B3[m] * hv; bt += B3[m] * tm; }
+                    t3[m] = tm;
+                }
+                const float w = chi * chi;
+                float pr1 = 0.f;
+#pragma unroll
+                for (int k = 0; k < W::C1; ++k) pr1 += ec[k] * dps[k];
+                float ux, uy, uz;
+                harmonics_grad_contract<L>(gux, guy, guz, t1, t2, t3, &ux, &uy, &uz);
+                const float pux = w * ux, puy = w * uy, puz = w * uz;
+                const float p_rho = chi * sa + w * pr1;
+                const float p_chi = sb + 2.0f * chi * bt;
+                const float dEdrho = p_rho + (p_chi + 2.0f * chi * ds0 + 4.0f * w * chi * ds1) * dchi;
+                const float dot = pux * gux + puy * guy + puz * guz;
+                const float gx = dEdrho * gux + (pux - dot * gux) * inv_rho;
+                const float gy = dEdrho * guy + (puy - dot * guy) * inv_rho;
+                const float gz = dEdrho * guz + (puz - dot * guz) * inv_rho;
+                vir[0] += gx * gdx; vir[1] += gx * gdy; vir[2] += gx * gdz;
+                vir[3] += gy * gdx; vir[4] += gy * gdy; vir[5] += gy * gdz;
+                vir[6] += gz * gdx; vir[7] += gz * gdy; vir[8] += gz * gdz;
                 float* go = a.g + 3 * (size_t)e;
                 go[0] = gx; go[1] = gy; go[2] = gz;
             }
             __syncwarp();
+        };
+
+        int qn = 0;
+        for (int base = e0; base < e1; base += 32) {
+            const int e = base + lane;
+            const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
+            const unsigned vmask = __ballot_sync(kFull, g.valid);
+            if (g.valid) {
+                const int p = qn + __popc(vmask & lt_mask);
+                qes[p] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
+                qd[p] = g.dx; qd[64 + p] = g.dy; qd[128 + p] = g.dz; qd[192 + p] = g.dchi;
+                qd[256 + p] = __int_as_float(e);
+            } else if (e < e1) {
+                float* go = a.g + 3 * (size_t)e;
+                go[0] = 0.f; go[1] = 0.f; go[2] = 0.f;
+            }
+            qn += __popc(vmask);
+            __syncwarp();
+            if (qn >= 32) {
+                run_batch(32);
+                const int rem = qn - 32;        // move the tail of the queue to its front
+                int4 tes = make_int4(0, 0, 0, 0);
+                float tq[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+                if (lane < rem) {
+                    tes = qes[32 + lane];
+#pragma unroll
+                    for (int k = 0; k < 5; ++k) tq[k] = qd[64 * k + 32 + lane];
+                }
+                __syncwarp();
+                if (lane < rem) {
+                    qes[lane] = tes;
+#pragma unroll
+                    for (int k = 0; k < 5; ++k) qd[64 * k + lane] = tq[k];
+                }
+                __syncwarp();
+                qn = rem;
+            }
         }
+        if (qn > 0) run_batch(qn);
     }
     // block partial of sum_e g (x) r, in double, fixed order
 #pragma unroll
