@@ -239,9 +239,13 @@ def run_ours(args):
     if args.atoms:
         # a smaller box of the same recipe (density, exclusion radius, species mix): the size one
         # node tile of the full workload has, for profiler captures that must stay small
-        if desc.get("kind") != "poisson_disk":
-            raise SystemExit("--atoms applies to the amorphous workload only")
-        desc["atoms"] = int(args.atoms)
+        if desc.get("kind") == "poisson_disk":
+            desc["atoms"] = int(args.atoms)
+        elif desc.get("kind") in ("fcc", "bcc", "diamond"):
+            per_cell = {"fcc": 4, "bcc": 2, "diamond": 8}[desc["kind"]]
+            desc["cells"] = max(1, round((args.atoms / per_cell) ** (1.0 / 3.0)))
+        else:
+            raise SystemExit("--atoms applies to the amorphous and the lattice workloads only")
         name = f"{name}[atoms={int(args.atoms)}]"
     s = make_system(desc, None if static else md)
     N = len(s["pos"])
@@ -400,7 +404,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
     ap.add_argument("--mlp-path", type=int, default=0)
     ap.add_argument("--node-tile", type=int, default=0)
-    ap.add_argument("--atoms", type=int, default=0, help="amorphous workload only: atoms of a smaller box of the same recipe")
+    ap.add_argument("--atoms", type=int, default=0, help="amorphous and lattice workloads: (about) this many atoms in a smaller box of the same recipe")
     ap.add_argument("--modes", type=int, default=-1, help="override the number R of shared radial modes of the workload's profile")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -131,10 +131,27 @@ __device__ __forceinline__ void table_eval1(const float* __restrict__ table, int
     if (DERIV) *dv = (3.0f * c3 * t + 2.0f * c2) * t + c1;
 }
 
-// amplitude psi (and d psi / d rho) of this lane's four channels for one edge
+// Shared radial modes q_mu(rho) (and derivatives) of the first nb queued edges, one (edge, mode)
+// pair per lane, parked as qm[edge * kMaxR + mu]: evaluated once per edge here instead of once
+// per lane in the channel-parallel phase.
+template <bool DERIV>
+__device__ __forceinline__ void eval_modes(const EdgeArgs& a, const int4* qes, int nb, int lane, float* qm, float* dqm) {
+    const int R = a.d.R;
+    for (int idx = lane; idx < nb * R; idx += 32) {
+        const int b = idx / R, q = idx - b * R;
+        const int4 es = qes[b];
+        float qv, dqv = 0.f;
+        table_eval1<DERIV>(a.table, a.d.CP, es.x, a.d.C0 + q, __int_as_float(es.z), &qv, &dqv);
+        qm[b * kMaxR + q] = qv;
+        if (DERIV) dqm[b * kMaxR + q] = dqv;
+    }
+}
+
+// amplitude psi (and d psi / d rho) of this lane's four channels for one edge; qm / dqm: the
+// edge's parked radial modes (only read when HASR)
 template <int C0, bool HASR, bool DERIV>
 __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, int pair, int c, float* psi,
-                                           float* dpsi) {
+                                           float* dpsi, const float* qm, const float* dqm) {
     float g[4], dg[4];
     table_eval4<DERIV>(a.table, a.d.CP, row, c, t, g, dg);
     const int R = HASR ? a.d.R : 0;
@@ -144,12 +161,23 @@ __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, 
     psi[2] = ga.z * g[2] + be.z; psi[3] = ga.w * g[3] + be.w;
     if (DERIV) { dpsi[0] = ga.x * dg[0]; dpsi[1] = ga.y * dg[1]; dpsi[2] = ga.z * dg[2]; dpsi[3] = ga.w * dg[3]; }
     if (HASR) {
-        for (int q = 0; q < R; ++q) {
-            float qv, dqv = 0.f;
-            table_eval1<DERIV>(a.table, a.d.CP, row, C0 + q, t, &qv, &dqv);
+        float qv[kMaxR], dqv[kMaxR];
+        {
+            const float4 v0 = *reinterpret_cast<const float4*>(qm);
+            qv[0] = v0.x; qv[1] = v0.y; qv[2] = v0.z; qv[3] = v0.w;
+            if (R > 4) { const float4 v1 = *reinterpret_cast<const float4*>(qm + 4); qv[4] = v1.x; qv[5] = v1.y; qv[6] = v1.z; qv[7] = v1.w; }
+            if (DERIV) {
+                const float4 d0 = *reinterpret_cast<const float4*>(dqm);
+                dqv[0] = d0.x; dqv[1] = d0.y; dqv[2] = d0.z; dqv[3] = d0.w;
+                if (R > 4) { const float4 d1 = *reinterpret_cast<const float4*>(dqm + 4); dqv[4] = d1.x; dqv[5] = d1.y; dqv[6] = d1.z; dqv[7] = d1.w; }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kMaxR; ++q) {
+            if (q >= R) break;
             const float4 U = ldg4(pm + (size_t)(2 + q) * C0);
-            psi[0] += U.x * qv; psi[1] += U.y * qv; psi[2] += U.z * qv; psi[3] += U.w * qv;
-            if (DERIV) { dpsi[0] += U.x * dqv; dpsi[1] += U.y * dqv; dpsi[2] += U.z * dqv; dpsi[3] += U.w * dqv; }
+            psi[0] += U.x * qv[q]; psi[1] += U.y * qv[q]; psi[2] += U.z * qv[q]; psi[3] += U.w * qv[q];
+            if (DERIV) { dpsi[0] += U.x * dqv[q]; dpsi[1] += U.y * dqv[q]; dpsi[2] += U.z * dqv[q]; dpsi[3] += U.w * dqv[q]; }
         }
     }
 }
@@ -169,19 +197,20 @@ template <int C0, int L> struct Widths {
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
 };
 
-template <int C0, int L> struct BwdSmem {          // dynamic shared memory of the backward kernel
+template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L>;
-    static constexpr int queue_floats = 64 * 4 + 5 * 64;    // queue of in-range edges: int4 and five scalars per slot
-    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LH + 1) + W::NHI + 3) / 4 * 4 + queue_floats;   // floats
+    static constexpr int queue_floats = 32 * 4 + 5 * 32;    // queue of in-range edges: int4 and five scalars per slot
+    static constexpr int mode_floats = HASR ? 2 * 32 * kMaxR : 0;   // parked radial modes and their derivatives
+    static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LH + 1) + W::NHI + 3) / 4 * 4 + mode_floats + queue_floats;   // floats
     static constexpr size_t bytes = kWarpsPerBlock * 9 * sizeof(double) + sizeof(float) * kWarpsPerBlock * per_warp;
 };
 
 // ------------------------------------------------------------------------------- forward
 //
 // The row is scanned 32 listed edges at a time (lane = edge: geometry); the edges that fall
-// inside the cutoff are appended to a per-warp queue in shared memory, and whenever the queue
-// holds 32 of them (and once more at the end of the row) a full batch is processed, so the
-// later phases never run on skin-shell edges:
+// inside the cutoff are appended to a 32-slot per-warp queue in shared memory (edges that do
+// not fit wait in their lane's registers), and whenever 32 are there (and once more at the end
+// of the row) a full batch is processed, so the later phases never run on skin-shell edges:
 //   2. lanes = channels (a group of C0/4 lanes per edge): amplitude psi of all C0 channels,
 //      degree-0 sums accumulated in registers; the leading C1 amplitudes of each edge are
 //      parked in shared memory.
@@ -198,13 +227,15 @@ k_edge_forward(const EdgeArgs a) {
     // queue of edges inside the cutoff: row, pair, t, chi (fetched with one 16-byte broadcast
     // load in the channel-parallel phase; shuffles would go through the same L1 data pipe as
     // the table reads) and the edge vector
-    __shared__ int4 q_es[kWarpsPerBlock][64];
-    __shared__ float q_d[kWarpsPerBlock][3 * 64];
+    __shared__ int4 q_es[kWarpsPerBlock][32];
+    __shared__ float q_d[kWarpsPerBlock][3 * 32];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     if (i >= a.a1) return;
     float* const psi_s = scratch[wid];      // [32][PF]
     float* const tr = scratch[wid];         // [32][33]
+    float* const qm = scratch[wid] + 32 * W::PF;   // [32][kMaxR] radial modes, behind the parked amplitudes
+    static_assert(32 * W::PF + 32 * kMaxR <= 32 * 33, "scratch too small for the parked radial modes");
     int4* const qes = q_es[wid];
     float* const qd = q_d[wid];
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
@@ -220,6 +251,10 @@ k_edge_forward(const EdgeArgs a) {
     double s0 = 0.0, s1 = 0.0;   // normaliser sums in double: the calibration subtracts their mean
 
     auto run_batch = [&](const int nb) {     // the first nb queue slots
+        if (HASR) {
+            eval_modes<false>(a, qes, nb, lane, qm, nullptr);
+            __syncwarp();
+        }
         for (int it = 0; it * W::EPI < nb; ++it) {
             const int b = it * W::EPI + sub;
             if (b >= nb) continue;
@@ -227,7 +262,7 @@ k_edge_forward(const EdgeArgs a) {
             const int row = es.x, pair = es.y;
             const float t = __int_as_float(es.z), chi = __int_as_float(es.w);
             float psi[4];
-            amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr);
+            amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr, qm + b * kMaxR, nullptr);
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc0[k] += chi * psi[k];
             if (cl < W::NL1)
@@ -244,7 +279,7 @@ k_edge_forward(const EdgeArgs a) {
                 const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PF + 4 * q);
                 ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
             }
-            const float dx = qd[lane], dy = qd[64 + lane], dz = qd[128 + lane];
+            const float dx = qd[lane], dy = qd[32 + lane], dz = qd[64 + lane];
             const float inv_rho = 1.0f / sqrtf(dx * dx + dy * dy + dz * dz + kEpsReg * kEpsReg);
             harmonics_s1<L>(dx * inv_rho, dy * inv_rho, dz * inv_rho, B1, B2, B3);
             const float chi = __int_as_float(qes[lane].w);
@@ -295,25 +330,22 @@ k_edge_forward(const EdgeArgs a) {
     for (int base = e0; base < e1; base += 32) {
         const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
         const unsigned vmask = __ballot_sync(kFull, g.valid);
-        if (g.valid) {
-            const double c2 = (double)g.chi * (double)g.chi;
-            s0 += c2; s1 += c2 * c2;
-            const int p = qn + __popc(vmask & lt_mask);
+        const int p = qn + __popc(vmask & lt_mask);       // queue slot of this lane's edge, if it has one
+        if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
+        if (g.valid && p < 32) {
             qes[p] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
-            qd[p] = g.dx; qd[64 + p] = g.dy; qd[128 + p] = g.dz;
+            qd[p] = g.dx; qd[32 + p] = g.dy; qd[64 + p] = g.dz;
         }
         qn += __popc(vmask);
         __syncwarp();
-        if (qn >= 32) {
+        if (qn >= 32) {                                   // a full batch; the overflow waits in registers
             run_batch(32);
-            const int rem = qn - 32;            // move the tail of the queue to its front
-            int4 tes = make_int4(0, 0, 0, 0);
-            float t0 = 0.f, t1 = 0.f, t2 = 0.f;
-            if (lane < rem) { tes = qes[32 + lane]; t0 = qd[32 + lane]; t1 = qd[96 + lane]; t2 = qd[160 + lane]; }
+            if (g.valid && p >= 32) {
+                qes[p - 32] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
+                qd[p - 32] = g.dx; qd[p] = g.dy; qd[32 + p] = g.dz;
+            }
+            qn -= 32;
             __syncwarp();
-            if (lane < rem) { qes[lane] = tes; qd[lane] = t0; qd[64 + lane] = t1; qd[128 + lane] = t2; }
-            __syncwarp();
-            qn = rem;
         }
     }
     if (qn > 0) run_batch(qn);
@@ -357,13 +389,14 @@ k_edge_backward(const EdgeArgs a) {
     extern __shared__ __align__(16) unsigned char dsm[];
     double (*vsum)[9] = reinterpret_cast<double (*)[9]>(dsm);
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    float* const wbase = reinterpret_cast<float*>(dsm + kWarpsPerBlock * 9 * sizeof(double)) + wid * BwdSmem<C0, L>::per_warp;
+    float* const wbase = reinterpret_cast<float*>(dsm + kWarpsPerBlock * 9 * sizeof(double)) + wid * BwdSmem<C0, L, HASR>::per_warp;
     float* const psi_s = wbase;                                  // [32][PB]: psi, dpsi of the leading channels
     float* const red = psi_s + 32 * W::PB;                       // [2][32][LH+1] partial dot products
     float* const hi_s = red + 2 * 32 * (W::LH + 1);              // [NHI] gradient of the degree >= 1 sums
     // queue of edges inside the cutoff: (row, pair, t, chi), then dx, dy, dz, dchi, edge index
-    int4* const qes = reinterpret_cast<int4*>(wbase + BwdSmem<C0, L>::per_warp - BwdSmem<C0, L>::queue_floats);
-    float* const qd = reinterpret_cast<float*>(qes + 64);        // [5][64]
+    int4* const qes = reinterpret_cast<int4*>(wbase + BwdSmem<C0, L, HASR>::per_warp - BwdSmem<C0, L, HASR>::queue_floats);
+    float* const qm = reinterpret_cast<float*>(qes) - BwdSmem<C0, L, HASR>::mode_floats;   // [2][32][kMaxR]
+    float* const qd = reinterpret_cast<float*>(qes + 32);        // [5][32]
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     const bool active = i < a.a1;
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
@@ -390,6 +423,10 @@ k_edge_backward(const EdgeArgs a) {
         const float* H3 = H2 + 5 * W::C2;
 
         auto run_batch = [&](const int nb) {     // the first nb queue slots
+            if (HASR) {
+                eval_modes<true>(a, qes, nb, lane, qm, qm + 32 * kMaxR);
+                __syncwarp();
+            }
             for (int it = 0; it * W::EPI < nb; ++it) {
                 const int b = it * W::EPI + sub;
                 const bool act = b < nb;
@@ -399,7 +436,7 @@ k_edge_backward(const EdgeArgs a) {
                     const int row = es.x, pair = es.y;
                     const float t = __int_as_float(es.z);
                     float psi[4], dpsi[4];
-                    amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi);
+                    amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi, qm + b * kMaxR, qm + (32 + b) * kMaxR);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
                     if (cl < W::NL1) {
@@ -418,8 +455,8 @@ k_edge_backward(const EdgeArgs a) {
             }
             __syncwarp();
             if (lane < nb) {
-                const float gdx = qd[lane], gdy = qd[64 + lane], gdz = qd[128 + lane], dchi = qd[192 + lane];
-                const int e = __float_as_int(qd[256 + lane]);
+                const float gdx = qd[lane], gdy = qd[32 + lane], gdz = qd[64 + lane], dchi = qd[96 + lane];
+                const int e = __float_as_int(qd[128 + lane]);
                 const float chi = __int_as_float(qes[lane].w);
                 const float inv_rho = 1.0f / sqrtf(gdx * gdx + gdy * gdy + gdz * gdz + kEpsReg * kEpsReg);
                 const float gux = gdx * inv_rho, guy = gdy * inv_rho, guz = gdz * inv_rho;
@@ -487,35 +524,27 @@ k_edge_backward(const EdgeArgs a) {
             const int e = base + lane;
             const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
             const unsigned vmask = __ballot_sync(kFull, g.valid);
-            if (g.valid) {
-                const int p = qn + __popc(vmask & lt_mask);
+            const int p = qn + __popc(vmask & lt_mask);   // queue slot of this lane's edge, if it has one
+            if (g.valid && p < 32) {
                 qes[p] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
-                qd[p] = g.dx; qd[64 + p] = g.dy; qd[128 + p] = g.dz; qd[192 + p] = g.dchi;
-                qd[256 + p] = __int_as_float(e);
-            } else if (e < e1) {
+                qd[p] = g.dx; qd[32 + p] = g.dy; qd[64 + p] = g.dz; qd[96 + p] = g.dchi;
+                qd[128 + p] = __int_as_float(e);
+            } else if (!g.valid && e < e1) {
                 float* go = a.g + 3 * (size_t)e;
                 go[0] = 0.f; go[1] = 0.f; go[2] = 0.f;
             }
             qn += __popc(vmask);
             __syncwarp();
-            if (qn >= 32) {
+            if (qn >= 32) {                               // a full batch; the overflow waits in registers
                 run_batch(32);
-                const int rem = qn - 32;        // move the tail of the queue to its front
-                int4 tes = make_int4(0, 0, 0, 0);
-                float tq[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-                if (lane < rem) {
-                    tes = qes[32 + lane];
-#pragma unroll
-                    for (int k = 0; k < 5; ++k) tq[k] = qd[64 * k + 32 + lane];
+                if (g.valid && p >= 32) {
+                    const int r = p - 32;
+                    qes[r] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
+                    qd[r] = g.dx; qd[32 + r] = g.dy; qd[64 + r] = g.dz; qd[96 + r] = g.dchi;
+                    qd[128 + r] = __int_as_float(e);
                 }
+                qn -= 32;
                 __syncwarp();
-                if (lane < rem) {
-                    qes[lane] = tes;
-#pragma unroll
-                    for (int k = 0; k < 5; ++k) qd[64 * k + lane] = tq[k];
-                }
-                __syncwarp();
-                qn = rem;
             }
         }
         if (qn > 0) run_batch(qn);
@@ -545,8 +574,9 @@ cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
 }
 template <int C0, int L>
 cudaError_t launch_bwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
-    constexpr size_t bytes = BwdSmem<C0, L>::bytes;
-    auto kern = a.d.R > 0 ? k_edge_backward<C0, L, true> : k_edge_backward<C0, L, false>;
+    const bool hasr = a.d.R > 0;
+    const size_t bytes = hasr ? BwdSmem<C0, L, true>::bytes : BwdSmem<C0, L, false>::bytes;
+    auto kern = hasr ? k_edge_backward<C0, L, true> : k_edge_backward<C0, L, false>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e != cudaSuccess) return e;
     kern<<<blocks, kWarpsPerBlock * 32, bytes, st>>>(a);
