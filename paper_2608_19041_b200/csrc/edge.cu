@@ -255,7 +255,27 @@ k_edge_forward(const EdgeArgs a) {
             eval_modes<false>(a, qes, nb, lane, qm, nullptr);
             __syncwarp();
         }
-        for (int it = 0; it * W::EPI < nb; ++it) {
+        int it = 0;
+        if (W::EPI == 1 && !HASR) {
+            // whole warp per edge: two edges per step, so that twelve 16-byte table and pair
+            // loads are in flight per lane instead of six (the phase waits on their latency)
+            for (; it + 1 < nb; it += 2) {
+                const int4 ea = qes[it], eb = qes[it + 1];
+                float pa[4], pb[4];
+                amplitude4<C0, HASR, false>(a, ea.x, __int_as_float(ea.z), ea.y, c, pa, nullptr, nullptr, nullptr);
+                amplitude4<C0, HASR, false>(a, eb.x, __int_as_float(eb.z), eb.y, c, pb, nullptr, nullptr, nullptr);
+                const float ca = __int_as_float(ea.w), cb = __int_as_float(eb.w);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc0[k] += ca * pa[k];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc0[k] += cb * pb[k];
+                if (cl < W::NL1) {
+                    *reinterpret_cast<float4*>(psi_s + it * W::PF + c) = make_float4(pa[0], pa[1], pa[2], pa[3]);
+                    *reinterpret_cast<float4*>(psi_s + (it + 1) * W::PF + c) = make_float4(pb[0], pb[1], pb[2], pb[3]);
+                }
+            }
+        }
+        for (; it * W::EPI < nb; ++it) {
             const int b = it * W::EPI + sub;
             if (b >= nb) continue;
             const int4 es = qes[b];
