@@ -155,8 +155,11 @@ int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* m
 /*
  * Advance nsteps of velocity-Verlet NVE with time step dt_ps.  The neighbor list is
  * rebuilt (with the skin of the last build) every rebuild_every steps, counted from the
- * last build; rebuild_every <= 0 never rebuilds.  On return e_pot / e_kin (host, eV; may
- * be NULL) hold the potential and kinetic energy after the last step.
+ * last build; rebuild_every == 0 never rebuilds (a step in which an atom has moved more
+ * than skin/2 since the build then fails with UMLMD_E_STALE_NEIGHBORS); rebuild_every < 0
+ * rebuilds exactly when that displacement criterion trips, at the price of one host
+ * synchronisation per step.  On return e_pot / e_kin (host, eV; may be NULL) hold the
+ * potential and kinetic energy after the last step.
  */
 int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* e_pot,
                double* e_kin);

@@ -396,7 +396,24 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
     for (int s = 0; s < nsteps; ++s) {
         { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, true, h->st)); }
         ++h->steps_since_build;
-        if (rebuild_every > 0 && h->steps_since_build >= rebuild_every) {
+        bool rebuild = rebuild_every > 0 && h->steps_since_build >= rebuild_every;
+        if (rebuild_every < 0) {
+            // displacement-triggered: the gather pass flags any atom that has moved more than half
+            // the skin since the build; read the flag (one host synchronisation per step)
+            API_CUDA(h, launch_gather_positions(h->nb, h->md_pos, h->d_err, h->st));
+            API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+            API_CUDA(h, cudaStreamSynchronize(h->st));
+            const int word = *h->h_err;
+            if (word & ~kErrStale) {
+                API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+                return decode_device_errors(h, word & ~kErrStale);
+            }
+            if (word & kErrStale) {
+                API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+                rebuild = true;
+            }
+        }
+        if (rebuild) {
             const double skin = h->nb.skin;
             const double L[3] = {h->nb.L[0], h->nb.L[1], h->nb.L[2]};
             const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};

@@ -118,3 +118,33 @@ def test_rebuild_keeps_results_continuous():
         res.append((pos.clone(), ep, ek))
     assert (res[0][0] - res[1][0]).abs().max().item() < 1e-6
     assert abs(res[0][1] - res[1][1]) < 1e-6 * max(1.0, abs(res[0][1]))
+
+
+def test_displacement_triggered_rebuild():
+    # a thin skin that the motion outruns: a fixed list fails as stale, the displacement-triggered
+    # mode (rebuild_every < 0) rebuilds when needed and follows the frequently rebuilt trajectory
+    p = SMALL_PROFILES["p16_2_0"]
+    blob = make_blob(p, seed=60)
+    s = make_system(dict(kind="random_box", atoms=80, edges=(13.0, 14.0, 15.0), min_dist=1.8, seed=61,
+                         n_types=p["T"], masses=[20.0, 30.0, 40.0]),
+                    dict(seed=62, temperature=3000.0))
+    res = {}
+    for every in (0, -1, 1):
+        m = _binding().Model(blob)
+        pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
+        vel = torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
+        types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+        m.build_neighbors(pos, types, s["cell"], s["pbc"], 0.2)
+        m.set_md_state(pos, vel, s["masses"])
+        if every == 0:
+            with pytest.raises(_binding().UmlmdError) as e:
+                m.step(60, 0.001, every)
+            assert e.value.code == -6
+        else:
+            ep, ek = m.step(60, 0.001, every)
+            res[every] = (pos.clone(), ep, ek, m.query()["kernel_launches"])
+        m.close()
+    assert (res[-1][0] - res[1][0]).abs().max().item() < 1e-6
+    assert abs(res[-1][1] - res[1][1]) < 1e-6 * max(1.0, abs(res[1][1]))
+    assert res[-1][3] < res[1][3]          # fewer builds than one per step
+

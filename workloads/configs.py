@@ -101,7 +101,7 @@ def _paper_variant(index, seed, published, *profile_args, **profile_kw):
         system=dict(kind="diamond", cells=50, a=3.567, jitter=0.03, seed=0, n_types=118, type_index=5,
                     masses=[12.011] * 118),
         profile=_profile(*profile_args, **profile_kw),
-        weights_seed=seed, head_scale=-0.02,
+        weights_seed=seed, head_scale=-0.002,
         md=dict(steps=100, dt_ps=0.001, temperature=300.0, seed=8, rebuild_every=10, skin=1.0),
         published=dict(value=published, unit="atom-steps/s", hardware="1x NVIDIA H20, fp32",
                        source="paper, supplementary table of rates at 1,000,000 atoms"),
