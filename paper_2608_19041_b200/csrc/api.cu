@@ -5,6 +5,7 @@
 
 #include "alloc.h"
 #include "kernels.h"
+#include "mlp_gemm.h"
 #include "model.h"
 
 using namespace umd;
@@ -158,13 +159,20 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         { Scope sc(h, kEdgeFwd, 1); API_CUDA(h, launch_edge_forward(ea, h->st)); }
         InvArgs ia;
         ia.d = d; ia.m = h->md; ia.type_s = nb.type_s; ia.a0 = a0; ia.n = n; ia.state = h->state; ia.desc = h->desc;
+        // tensor-core MLP: the invariants kernel writes the first GEMM's operand split itself; the
+        // fp32 feature rows are then only kept where something still reads them (the identity
+        // residual of a first layer as wide as the feature vector, or the intermediates query of a
+        // single-tile system)
+        const bool presplit = h->mlp_path >= 2 && gemm_tc_available();
+        ia.desc_hi = presplit ? h->tc_hi : nullptr; ia.desc_lo = presplit ? h->tc_lo : nullptr;
+        ia.write_desc = !presplit || d.D_out == d.F || N <= h->node_tile;
         { Scope sc(h, kInvFwd, 1); API_CUDA(h, launch_invariants_forward(ia, h->st)); }
         MlpArgs ma;
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
-        ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err;
+        ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
-        { Scope sc(h, kMlpFwd, d.n_hidden + (h->mlp_path >= 2 ? 2 : 1)); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
+        { Scope sc(h, kMlpFwd, d.n_hidden + (presplit ? 1 : (h->mlp_path >= 2 ? 2 : 1))); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
             { Scope sc(h, kInvBwd, 1); API_CUDA(h, launch_invariants_backward(ia, h->st)); }

@@ -25,6 +25,7 @@
 // mu ~ M, so they are formed in double precision from sums accumulated in double (stored
 // as a float pair) to keep the subtraction from cancelling single-precision digits.
 #include "kernels.h"
+#include "mlp_gemm.h"
 
 namespace umd {
 
@@ -227,6 +228,12 @@ struct Front {
     }
 };
 
+// one calibrated feature-vector entry: fp32 and / or its TF32 split
+__device__ __forceinline__ void put_feature(const InvArgs& a, size_t off, float v) {
+    if (a.write_desc) a.desc[off] = v;
+    if (a.desc_hi) split_tf32(v, a.desc_hi[off], a.desc_lo[off]);
+}
+
 template <int C1, int C2, int L>
 __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
     using PL = Plan<C1, C2, L>;
@@ -236,7 +243,6 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
     const ModelDev& m = a.m;
     const int C0 = d.C0, TW = d.SP - C0;
     const int c_full = (2 * C0 / 32) * 32;         // columns [0, c_full) go straight from global to global
-    const int nDS = d.DP - c_full;
     float* mats = sm;
     float* ST = sm + PL::nMatP;
     float* XT = ST + TW * P;
@@ -246,7 +252,6 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
     Front<C1, C2, L> f;
     f.setup(a, ST, XT, ZZ, mats);
     const int lane = f.lane, warp = f.warp, nv = f.nv, b0 = f.b0;
-    float* Dg = a.desc + (size_t)b0 * d.DP;
     int uctr = 0;
 #define TAKE() ((uctr++ % NW) == warp)
 #define DSK(k) DS[((k) - c_full) * P + lane]
@@ -288,7 +293,7 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
 #pragma unroll
                 for (int i = 0; i < AT / NW; ++i) {
                     const int aa = warp + i * NW;
-                    if (aa < nv) Dg[(size_t)aa * d.DP + col] = (v[h][i] - mu_c) * is_c;
+                    if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (v[h][i] - mu_c) * is_c);
                 }
             }
         }
@@ -437,7 +442,7 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
 #pragma unroll
         for (int i = 0; i < AT / NW; ++i) {
             const int aa = warp + i * NW;
-            if (aa < nv) Dg[(size_t)aa * d.DP + col] = (DS[(col - c_full) * P + aa] - mu_c) * is_c;
+            if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (DS[(col - c_full) * P + aa] - mu_c) * is_c);
         }
     }
 #undef TAKE

@@ -49,6 +49,11 @@ struct InvArgs {
     int a0, n;              // tile start (sorted index) and atom count
     float* state;           // [n][SP]
     float* desc;            // [n][DP]
+    // forward only: when non-null the feature rows are also written as their TF32 split (row pitch
+    // DP), the form the tensor-core MLP reads; write_desc = false then skips the fp32 copy
+    float* desc_hi;
+    float* desc_lo;
+    bool write_desc;
 };
 cudaError_t launch_invariants_forward(const InvArgs& a, cudaStream_t st);
 cudaError_t launch_invariants_backward(const InvArgs& a, cudaStream_t st);
@@ -67,6 +72,7 @@ struct MlpArgs {
     bool want_grad;
     float* tc_hi;           // two slots of [n][max(DP, F)]: TF32 splits of the activations (tensor-core path)
     float* tc_lo;
+    bool desc_presplit;     // slot 0 already holds the split of desc (written by the invariants kernel)
     size_t tc_slot;         // floats per slot
     int* err;               // device error word
 };

@@ -133,7 +133,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         // tensor-core path: the split of layer t's input sits in slot t & 1 (layer 0's is made by
         // the split kernel), and the epilogue leaves the split of its output in the other slot
         g.A_hi = a.tc_hi + (size_t)(t & 1) * a.tc_slot; g.A_lo = a.tc_lo + (size_t)(t & 1) * a.tc_slot;
-        g.a_presplit = t > 0; g.err = a.err; g.variant = a.path;
+        g.a_presplit = t > 0 || (tc && a.desc_presplit); g.err = a.err; g.variant = a.path;
         if (tc && t + 1 < NH) {
             g.nxt_hi = a.tc_hi + (size_t)((t + 1) & 1) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)((t + 1) & 1) * a.tc_slot;
             g.ldnxt = F;
