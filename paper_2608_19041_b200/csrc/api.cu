@@ -162,10 +162,10 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         // tensor-core MLP: the invariants kernel writes the first GEMM's operand split itself; the
         // fp32 feature rows are then only kept where something still reads them (the identity
         // residual of a first layer as wide as the feature vector, or the intermediates query of a
-        // single-tile system)
+        // system smaller than one node tile)
         const bool presplit = h->mlp_path >= 2 && gemm_tc_available();
         ia.desc_hi = presplit ? h->tc_hi : nullptr; ia.desc_lo = presplit ? h->tc_lo : nullptr;
-        ia.write_desc = !presplit || d.D_out == d.F || N <= h->node_tile;
+        ia.write_desc = !presplit || d.D_out == d.F || N < h->node_tile;
         { Scope sc(h, kInvFwd, 1); API_CUDA(h, launch_invariants_forward(ia, h->st)); }
         MlpArgs ma;
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
@@ -441,7 +441,7 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
 int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc) {
     if (!h) return UMLMD_E_INVALID_ARG;
     if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "no neighbor list built");
-    if (h->nb.N > h->node_tile) return fail(h, UMLMD_E_CAPACITY, "intermediates are only kept for single-tile systems");
+    if (h->nb.N >= h->node_tile) return fail(h, UMLMD_E_CAPACITY, "intermediates are only kept for systems smaller than one node tile");
     if (d_state) API_CUDA(h, launch_unsort_state(h->nb, h->state, h->d.SP, h->d.S + 2, d_state, h->st));
     if (d_desc) API_CUDA(h, launch_unsort_state(h->nb, h->desc, h->d.DP, h->d.D_out, d_desc, h->st));
     API_CUDA(h, cudaStreamSynchronize(h->st));

@@ -229,6 +229,34 @@ def test_tensor_core_mlp_path_small_profiles(name, path):
     _compare(blob, s, check_intermediates=False, mlp_path=path)
 
 
+def test_table_spacing_sweep_against_the_continuous_model():
+    # the paper's fidelity experiment on random weights: the tabulated path against the
+    # continuous model for a range of table spacings.  The library stores the cubic two-point
+    # interpolant, whose error grows like the fourth power of the spacing (third for the
+    # derivative); up to 0.005 A the result sits at the single-precision floor, and the forces,
+    # which see the derivative of the table, resolve the spacing first.
+    p = SMALL_PROFILES["p32_3_2"]
+    blob = make_blob(p, seed=46)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    o = orc.Oracle(blob)
+    ref = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    Dref = (ref["D_raw"] - o.prm["mu"].numpy()) / o.prm["sigma"].numpy()
+    dev = {}
+    for dx in (0.0005, 0.002, 0.005, 0.01, 0.02, 0.05):
+        m, pos = _build(blob, s, table_dx=dx)
+        m.compute(pos, forces=False, virial=False)
+        _, desc = m.get_intermediates()
+        desc = desc.cpu().numpy().astype(np.float64)
+        out = m.compute(pos)
+        dev[dx] = (np.abs(desc - Dref).max() / np.abs(Dref).max(),
+                   np.abs(out["forces"].cpu().numpy() - ref["F"]).max() / np.abs(ref["F"]).max())
+        m.close()
+    for dx in (0.0005, 0.002, 0.005):
+        assert dev[dx][0] <= 2e-6 and dev[dx][1] <= 5e-6, (dx, dev[dx])
+    assert dev[0.01][1] <= 1e-5 and dev[0.02][1] <= 1e-4 and dev[0.05][1] <= 2e-3, dev
+    assert dev[0.05][1] > 10 * dev[0.002][1]                 # the coarse end is resolvably worse
+
+
 @pytest.mark.parametrize("name", ["paper_nano_c1m", "paper_air_c1m", "paper_plus_c1m"])
 def test_paper_variants_on_small_diamond_cell(name):
     # the paper's model variants (118-species type table, carbon only) on a 512-atom cell of its
