@@ -118,6 +118,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
     const bool tc = a.path >= 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    const int variant = tc ? gemm_tc_pick_variant(n, F, a.path) : a.path;
     // the backward seed goes to the slot the last layer does not read its input from
     const int seed_slot = NH & 1;
     cudaError_t e;
@@ -133,7 +134,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         // tensor-core path: the split of layer t's input sits in slot t & 1 (layer 0's is made by
         // the split kernel), and the epilogue leaves the split of its output in the other slot
         g.A_hi = a.tc_hi + (size_t)(t & 1) * a.tc_slot; g.A_lo = a.tc_lo + (size_t)(t & 1) * a.tc_slot;
-        g.a_presplit = t > 0 || (tc && a.desc_presplit); g.err = a.err; g.variant = a.path;
+        g.a_presplit = t > 0 || (tc && a.desc_presplit); g.err = a.err; g.variant = variant;
         if (tc && t + 1 < NH) {
             g.nxt_hi = a.tc_hi + (size_t)((t + 1) & 1) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)((t + 1) & 1) * a.tc_slot;
             g.ldnxt = F;
@@ -144,7 +145,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         if (tc && t == NH - 1) {
             // last layer: the epilogue takes the head's dot product and the backward seed, so
             // neither the activations nor the pre-activations of this layer are stored
-            g.head_w = a.m.w_head; g.head_part = hb[t & 1]; g.head_parts = gemm_tc_head_parts(F, a.path);
+            g.head_w = a.m.w_head; g.head_part = hb[t & 1]; g.head_parts = gemm_tc_head_parts(F, variant);
             g.out = nullptr; g.pre = nullptr;
             if (a.want_grad) {
                 g.nxt_hi = a.tc_hi + (size_t)seed_slot * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)seed_slot * a.tc_slot;
@@ -154,7 +155,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
     }
     if (tc) {
-        const int parts = gemm_tc_head_parts(F, a.path);
+        const int parts = gemm_tc_head_parts(F, variant);
         k_head_finish<<<(n + 255) / 256, 256, 0, st>>>(n, parts, hb[(NH - 1) & 1], a.m.b_head, a.m.e_ref, a.type_s, a.a0,
                                                         a.e_atom);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -178,6 +179,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
     const bool res0 = (d.D_out == F);
     cudaError_t e;
     const bool tc = a.path >= 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    const int variant = tc ? gemm_tc_pick_variant(n, F, a.path) : a.path;
     int sp = NH & 1;           // tensor-core path: slot with the TF32 split of pre[t] (the forward pass left the seed here)
     int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
     bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
@@ -189,7 +191,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.B = a.m.thetaT[t]; g.ldb = F;
         g.Bt_hi = a.m.theta_hi[t]; g.Bt_lo = a.m.theta_lo[t]; g.ldbt = F;
         g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
-        g.a_presplit = tc; g.err = a.err; g.variant = a.path;
+        g.a_presplit = tc; g.err = a.err; g.variant = variant;
         if (tc) { g.nxt_hi = a.tc_hi + (size_t)(1 - sp) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)(1 - sp) * a.tc_slot; g.ldnxt = F; }
         sp = 1 - sp;
         if (vec_grad) g.rvec = a.m.w_head; else { g.res = hb[slot]; g.ldres = F; }
@@ -208,7 +210,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.B = a.m.thetaT[0]; g.ldb = d.DP;
         g.Bt_hi = a.m.theta_hi[0]; g.Bt_lo = a.m.theta_lo[0]; g.ldbt = F;
         g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
-        g.a_presplit = tc; g.err = a.err; g.variant = a.path;
+        g.a_presplit = tc; g.err = a.err; g.variant = variant;
         if (res0) {
             if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }

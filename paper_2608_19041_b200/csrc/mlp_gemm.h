@@ -96,6 +96,7 @@ __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
 bool gemm_tc_available();      // the driver's tensor-map encoder could be resolved
+int gemm_tc_pick_variant(int M, int N, int requested);   // 2 (persistent) or 3 (one tile per CTA) for path 2
 constexpr int kGemmTcBN = 128;  // column tile of the tensor-core GEMM
 // partial head sums per row that the fused last-layer epilogue of a variant leaves
 inline int gemm_tc_head_parts(int N, int variant) { return (variant == 3 ? 1 : 2) * ((N + kGemmTcBN - 1) / kGemmTcBN); }

@@ -520,6 +520,20 @@ bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
 
 bool gemm_tc_available() { return encode_fn() != nullptr; }
 
+// The persistent kernel needs about one 256 x 128 item per SM to fill the machine; below half of
+// that the one-tile-per-CTA kernel, with twice as many and half as long CTAs, finishes sooner.
+int gemm_tc_pick_variant(int M, int N, int requested) {
+    if (requested != 2) return requested;
+    static int n_sm = 0;
+    if (n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n_sm = 148;
+    }
+    const int items = ((N + BN - 1) / BN) * ((M + 2 * BM - 1) / (2 * BM));
+    return 2 * items <= n_sm ? 3 : 2;
+}
+
 bool gemm_tc_supported(const GemmArgs& g) {
     return g.A_hi && g.A_lo && g.Bt_hi && g.Bt_lo && g.M > 0 && g.N >= 4 && g.K >= 4 && (g.K & 3) == 0 &&
            (g.N & 3) == 0 && (g.lda & 3) == 0 && (g.ldbt & 3) == 0 && encode_fn() != nullptr;
