@@ -213,6 +213,26 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ replicas on several ranks
+
+def max_over_ranks(ms, device):
+    """Time of the slowest rank (the job's time): all-reduce MAX over the default process group;
+    the value itself for a single process."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_rate(units_per_rank, ms, world):
+    """Whole-job rate of `world` independent replicas that each did `units_per_rank` units of work,
+    over the slowest rank's time `ms` (milliseconds)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------ our arm
 
 def run_ours(args):
@@ -292,11 +312,8 @@ def run_ours(args):
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1)
     launches = model.query()["kernel_launches"] - launches0
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * N * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, "cuda")
+    value = job_rate(N * args.steps, ms, world)
 
     # ---- second pass with per-class events: where the time goes, roofline per class
     model.get_profile()
@@ -343,11 +360,8 @@ def run_ours(args):
     t1.record()
     sync_all()
     ms_e2e = t0.elapsed_time(t1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e = dict(value=world * N * k_e2e / (ms_e2e * 1e-3), unit="atom-steps/s", h2d_bytes_per_step=N * 24,
+    ms_e2e = max_over_ranks(ms_e2e, "cuda")
+    e2e = dict(value=job_rate(N * k_e2e, ms_e2e, world), unit="atom-steps/s", h2d_bytes_per_step=N * 24,
                d2h_bytes_per_step=N * 24 + 80, steps=k_e2e)
 
     cpu = None
