@@ -182,10 +182,14 @@ __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, 
     }
 }
 
-template <int C0, int L> struct Widths {
+// G = groups of four channels a lane holds in the channel-parallel phase (group g starts at
+// channel 4 * lane_in_group + g * C0 / G, so every 16-byte load instruction of a group of lanes
+// still covers one contiguous segment)
+template <int C0, int L, int G = 1> struct Widths {
     static constexpr int C1 = C0 <= 16 ? 4 : (C0 <= 64 ? 8 : 16);
     static constexpr int C2 = C1 / 2 > 4 ? C1 / 2 : 4;
-    static constexpr int LPE = C0 / 4;          // lanes per edge in the channel-parallel phase
+    static constexpr int LPE = C0 / (4 * G);    // lanes per edge in the channel-parallel phase
+    static constexpr int GOFF = C0 / G;         // channel offset between a lane's groups
     static constexpr int LH = LPE / 2;          // parked partial dot products per edge (lanes paired)
     static constexpr int EPI = 32 / LPE;        // edges per replay step
     static constexpr int NL1 = C1 / 4;          // lanes of a group that hold degree-1 channels
@@ -197,8 +201,12 @@ template <int C0, int L> struct Widths {
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
 };
 
+// the backward pass keeps two channel groups per lane at C0 = 128: twice as many table and pair
+// loads are in flight per lane, which is what this latency-bound phase lacks at two blocks per SM
+template <int C0> struct BwdGroups { static constexpr int G = C0 >= 128 ? 2 : 1; };
+
 template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
-    using W = Widths<C0, L>;
+    using W = Widths<C0, L, BwdGroups<C0>::G>;
     static constexpr int queue_floats = 32 * 4 + 5 * 32;    // queue of in-range edges: int4 and five scalars per slot
     static constexpr int mode_floats = HASR ? 2 * 32 * kMaxR : 0;   // parked radial modes and their derivatives
     static constexpr int per_warp = (32 * W::PB + 2 * 32 * (W::LH + 1) + W::NHI + 3) / 4 * 4 + mode_floats + queue_floats;   // floats
@@ -405,7 +413,8 @@ k_edge_forward(const EdgeArgs a) {
 template <int C0, int L, bool HASR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_backward(const EdgeArgs a) {
-    using W = Widths<C0, L>;
+    constexpr int G = BwdGroups<C0>::G;
+    using W = Widths<C0, L, G>;
     extern __shared__ __align__(16) unsigned char dsm[];
     double (*vsum)[9] = reinterpret_cast<double (*)[9]>(dsm);
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -430,10 +439,11 @@ k_edge_backward(const EdgeArgs a) {
         const int ti = a.type_s[i];
         const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
-        float h0[4];
-        {
-            const float4 v = *reinterpret_cast<const float4*>(grow + c);
-            h0[0] = v.x; h0[1] = v.y; h0[2] = v.z; h0[3] = v.w;
+        float h0[4 * G];
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq) {
+            const float4 v = *reinterpret_cast<const float4*>(grow + c + gq * W::GOFF);
+            h0[4 * gq] = v.x; h0[4 * gq + 1] = v.y; h0[4 * gq + 2] = v.z; h0[4 * gq + 3] = v.w;
         }
         for (int v = lane; v < W::NHI; v += 32) hi_s[v] = grow[a.d.offA[1] + v];
         const float ds0 = grow[a.d.S], ds1 = grow[a.d.S + 1];
@@ -455,11 +465,14 @@ k_edge_backward(const EdgeArgs a) {
                     const int4 es = qes[b];
                     const int row = es.x, pair = es.y;
                     const float t = __int_as_float(es.z);
-                    float psi[4], dpsi[4];
-                    amplitude4<C0, HASR, true>(a, row, t, pair, c, psi, dpsi, qm + b * kMaxR, qm + (32 + b) * kMaxR);
+                    float psi[4 * G], dpsi[4 * G];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
-                    if (cl < W::NL1) {
+                    for (int gq = 0; gq < G; ++gq)
+                        amplitude4<C0, HASR, true>(a, row, t, pair, c + gq * W::GOFF, psi + 4 * gq, dpsi + 4 * gq, qm + b * kMaxR,
+                                                   qm + (32 + b) * kMaxR);
+#pragma unroll
+                    for (int k = 0; k < 4 * G; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
+                    if (cl < W::NL1) {       // the leading C1 channels all sit in group 0
                         *reinterpret_cast<float4*>(psi_s + b * W::PB + c) = make_float4(psi[0], psi[1], psi[2], psi[3]);
                         *reinterpret_cast<float4*>(psi_s + b * W::PB + W::C1 + c) = make_float4(dpsi[0], dpsi[1], dpsi[2], dpsi[3]);
                     }
