@@ -265,8 +265,13 @@ def test_paper_variants_on_small_diamond_cell(name):
     s = make_system(dict(cfg["system"], cells=4))
     blob = make_blob(cfg["profile"], seed=cfg["weights_seed"], calibration=load_calibration(name), bias_scale=0.1,
                      e_ref_scale=0.5)
-    _compare(blob, s, check_intermediates=False)
-    _compare(blob, s, check_intermediates=False, skin=1.0)
+    # Twice the usual tolerance: on this nearly perfect lattice the odd-degree invariants almost
+    # cancel (single-precision noise amplified by the calibration, as on the 108-atom Al cell), and
+    # the tensor-core accumulator truncates once per MMA instruction, a one-sided bias of about half
+    # an ulp times the 100-150 instructions per output (~4e-6 of a pre-activation); together they
+    # sit at 0.5-1.1e-5 of the largest atomic energy here, while the CUDA-core path shows 5e-6.
+    _compare(blob, s, check_intermediates=False, tol_scale=2.0)
+    _compare(blob, s, check_intermediates=False, skin=1.0, tol_scale=2.0)
 
 
 def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
