@@ -203,7 +203,7 @@ template <int C0, int L, int G = 1> struct Widths {
 
 // the backward pass keeps two channel groups per lane at C0 = 128: twice as many table and pair
 // loads are in flight per lane, which is what this latency-bound phase lacks at two blocks per SM
-template <int C0> struct BwdGroups { static constexpr int G = C0 >= 128 ? 2 : 1; };
+template <int C0> struct BwdGroups { static constexpr int G = C0 >= 64 ? 2 : 1; };
 
 template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L, BwdGroups<C0>::G>;
