@@ -166,11 +166,13 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         const bool presplit = h->mlp_path >= 2 && gemm_tc_available();
         ia.desc_hi = presplit ? h->tc_hi : nullptr; ia.desc_lo = presplit ? h->tc_lo : nullptr;
         ia.write_desc = !presplit || d.D_out == d.F || N < h->node_tile;
+        const bool fold_x0 = presplit && d.D_out != d.F;      // first GEMM skips the per-species constant columns
+        ia.skip_x0_split = fold_x0;
         { Scope sc(h, kInvFwd, 1); API_CUDA(h, launch_invariants_forward(ia, h->st)); }
         MlpArgs ma;
         ma.d = d; ma.m = h->md; ma.type_s = nb.type_s; ma.a0 = a0; ma.n = n; ma.desc = h->desc; ma.pre = h->pre;
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
-        ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit;
+        ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit; ma.fold_x0 = fold_x0;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
         { Scope sc(h, kMlpFwd, d.n_hidden + (presplit ? 1 : (h->mlp_path >= 2 ? 2 : 1))); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
@@ -211,6 +213,7 @@ int ensure_device_model(umlmd_t* h) {
     auto up = [&](const std::vector<float>& v, float** p) { if (e == cudaSuccess) e = upload(h, v, p); };
     up(m.table, &md.table); up(m.pairmod, &md.pairmod); up(m.X0, &md.X0); up(m.W1p, &md.W1p); up(m.W2p, &md.W2p);
     up(m.A1, &md.A1); up(m.A2, &md.A2); up(m.mu, &md.mu); up(m.inv_sigma, &md.inv_sigma);
+    up(m.type_bias, &md.type_bias);
     for (int t = 0; t < h->d.n_hidden; ++t) { up(m.theta[t], &md.theta[t]); up(m.thetaT[t], &md.thetaT[t]); up(m.bias[t], &md.bias[t]);
         up(m.theta_hi[t], &md.theta_hi[t]); up(m.theta_lo[t], &md.theta_lo[t]);
         up(m.thetaT_hi[t], &md.thetaT_hi[t]); up(m.thetaT_lo[t], &md.thetaT_lo[t]); }

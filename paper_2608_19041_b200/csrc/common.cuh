@@ -63,6 +63,7 @@ struct ModelDev {
     float* theta_hi[8];  float* theta_lo[8];    // TF32 split of theta  (x = hi + lo)
     float* thetaT_hi[8]; float* thetaT_lo[8];   // TF32 split of thetaT
     float* bias[8];   // b_t [F]
+    float* type_bias; // [T][F] first-layer bias with the centre's initial features folded in
     float* w_head;    // [F]
     float* e_ref;     // [T]
     float b_head;

@@ -229,9 +229,9 @@ struct Front {
 };
 
 // one calibrated feature-vector entry: fp32 and / or its TF32 split
-__device__ __forceinline__ void put_feature(const InvArgs& a, size_t off, float v) {
+__device__ __forceinline__ void put_feature(const InvArgs& a, size_t off, float v, bool split_ok) {
     if (a.write_desc) a.desc[off] = v;
-    if (a.desc_hi) split_tf32(v, a.desc_hi[off], a.desc_lo[off]);
+    if (a.desc_hi && split_ok) split_tf32(v, a.desc_hi[off], a.desc_lo[off]);
 }
 
 template <int C1, int C2, int L>
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
                     const int aa = warp + i * NW;
                     v[h][i] = 0.f;
                     if (aa < nv && col < c_full) {
-                        if (col < C0) v[h][i] = __ldg(m.X0 + ty[i] * C0 + col);
+                        if (col < C0) { if (a.write_desc || !a.skip_x0_split) v[h][i] = __ldg(m.X0 + ty[i] * C0 + col); }
                         else v[h][i] = st_g[(size_t)aa * d.SP + (col - C0)] * im0[i];
                     }
                 }
@@ -290,10 +290,11 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
                 const int col = cb + 32 * h + lane;
                 if (col >= c_full) continue;
                 const float mu_c = __ldg(m.mu + col), is_c = __ldg(m.inv_sigma + col);
+                const bool split_col = !(a.skip_x0_split && col < C0);
 #pragma unroll
                 for (int i = 0; i < AT / NW; ++i) {
                     const int aa = warp + i * NW;
-                    if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (v[h][i] - mu_c) * is_c);
+                    if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (v[h][i] - mu_c) * is_c, split_col);
                 }
             }
         }
@@ -439,10 +440,11 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
         const int col = cb + lane;
         float mu_c = 0.f, is_c = 1.f;
         if (col < d.D_out && col != kM0 && col != kM1) { mu_c = __ldg(m.mu + col); is_c = __ldg(m.inv_sigma + col); }
+        const bool split_col = !(a.skip_x0_split && col < C0);
 #pragma unroll
         for (int i = 0; i < AT / NW; ++i) {
             const int aa = warp + i * NW;
-            if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (DS[(col - c_full) * P + aa] - mu_c) * is_c);
+            if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (DS[(col - c_full) * P + aa] - mu_c) * is_c, split_col);
         }
     }
 #undef TAKE

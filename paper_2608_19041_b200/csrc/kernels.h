@@ -54,6 +54,7 @@ struct InvArgs {
     float* desc_hi;
     float* desc_lo;
     bool write_desc;
+    bool skip_x0_split;     // the split omits the first C0 columns (the MLP folds them into a per-species bias)
 };
 cudaError_t launch_invariants_forward(const InvArgs& a, cudaStream_t st);
 cudaError_t launch_invariants_backward(const InvArgs& a, cudaStream_t st);
@@ -73,6 +74,7 @@ struct MlpArgs {
     float* tc_hi;           // two slots of [n][max(DP, F)]: TF32 splits of the activations (tensor-core path)
     float* tc_lo;
     bool desc_presplit;     // slot 0 already holds the split of desc (written by the invariants kernel)
+    bool fold_x0;           // tensor-core path: the first C0 feature columns enter through m.type_bias instead of the GEMM
     size_t tc_slot;         // floats per slot
     int* err;               // device error word
 };

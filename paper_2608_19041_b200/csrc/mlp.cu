@@ -140,6 +140,13 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
             g.ldnxt = F;
         }
         g.bias = a.m.bias[t];
+        if (tc && t == 0 && a.fold_x0) {
+            // the first C0 feature columns are constants per species: their share of the product
+            // sits in the per-species bias, and the GEMM starts at column C0 of A and of Theta_1^T
+            g.A_hi += d.C0; g.A_lo += d.C0; g.lda_split = d.DP; g.K = d.DP - d.C0;
+            g.Bt_hi += d.C0; g.Bt_lo += d.C0;
+            g.bias_rows = a.m.type_bias; g.row_type = a.type_s + a.a0;
+        }
         g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
         g.out = hb[t & 1]; g.ldout = F;
         if (tc && t == NH - 1) {
@@ -216,6 +223,11 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }
         }
         g.out = a.desc; g.ldout = d.DP;
+        if (tc && a.fold_x0) {        // no gradient is needed for the per-species constant columns
+            g.N = d.DP - d.C0;
+            g.Bt_hi += (size_t)d.C0 * F; g.Bt_lo += (size_t)d.C0 * F;
+            g.out = a.desc + d.C0;
+        }
         if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
     }
     return cudaSuccess;

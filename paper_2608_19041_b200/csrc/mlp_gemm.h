@@ -35,6 +35,9 @@ struct GemmArgs {
     // tile], and, when nxt_hi is set, leaves the split of head_w[n] * SiLU'(y[m,n]) there (the
     // seed of the backward pass)
     const float* head_w; float* head_part; int head_parts;
+    // tensor-core path, mode 0 / head: per-row bias bias_rows[row_type[m] * N + n] instead of bias[n]
+    const float* bias_rows; const int* row_type;
+    int lda_split;                // row pitch of A_hi / A_lo (0 = K)
     int variant;                  // tensor-core kernel: 3 = one tile per CTA, otherwise the persistent one
     int* err;                     // device error word (bounded-wait expiry)
 };

@@ -192,7 +192,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
         const bool valid = n < g.N;
         {
             float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
-            if (valid && MODE != 1) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+            if (valid && MODE != 1 && !g.bias_rows) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
             if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
             const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
             if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
@@ -213,6 +213,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     if (r0 + j < rows) {
                         if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
                         if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n);
+                        if (MODE != 1 && valid && g.bias_rows)      // per-species bias: carried in the y slot
+                            y[j] = __ldg(reinterpret_cast<const float4*>(g.bias_rows + (size_t)g.row_type[m] * g.N + n));
                     }
                 }
 #pragma unroll
@@ -221,7 +223,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     const size_t m = (size_t)(m0 + q * 32 + r0 + j);
                     float4 a = *reinterpret_cast<const float4*>(stage + (r0 + j) * EPITCH + 4 * lane);
                     if (MODE != 1) {
-                        a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
+                        const float4 bb = g.bias_rows ? y[j] : bias;
+                        a.x += bb.x; a.y += bb.y; a.z += bb.z; a.w += bb.w;
                         const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
                                                      silu(a.w) + res[j].w);
                         if (MODE == 2) {           // last layer: row . w_head, and the backward seed
@@ -407,7 +410,7 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                 const int n = n0 + pass * 64 + c4;
                 const bool valid = n < g.N;
                 float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
-                if (valid && MODE != 1) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+                if (valid && MODE != 1 && !g.bias_rows) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
                 if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
                 const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
                 if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
@@ -424,6 +427,8 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                         if (m < g.M) {
                             if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n);
                             if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + (size_t)m * g.ldpre + n);
+                            if (MODE != 1 && valid && g.bias_rows)  // per-species bias: carried in the y slot
+                                y[j] = __ldg(reinterpret_cast<const float4*>(g.bias_rows + (size_t)g.row_type[m] * g.N + n));
                         }
                     }
 #pragma unroll
@@ -433,7 +438,8 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                         const bool okm = mrow0 + r < g.M;
                         float4 a = *reinterpret_cast<const float4*>(stage + r * P_SPITCH + c4);
                         if (MODE != 1) {
-                            a.x += bias.x; a.y += bias.y; a.z += bias.z; a.w += bias.w;
+                            const float4 bb = g.bias_rows ? y[j] : bias;
+                            a.x += bb.x; a.y += bb.y; a.z += bb.z; a.w += bb.w;
                             const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
                                                          silu(a.w) + res[j].w);
                             if (MODE == 2) {               // last layer: row . w_head over these 64 columns, and the seed
@@ -562,7 +568,8 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
         k_split_tf32<<<blocks, 256, 0, st>>>(g.A, g.lda, g.M, g.K, g.A_hi, g.A_lo);
     }
     CUtensorMap mAh, mAl, mBh, mBl;
-    if (!make_map(&mAh, g.A_hi, g.M, g.K, g.K) || !make_map(&mAl, g.A_lo, g.M, g.K, g.K) ||
+    const int lda_s = g.lda_split ? g.lda_split : g.K;
+    if (!make_map(&mAh, g.A_hi, g.M, g.K, lda_s) || !make_map(&mAl, g.A_lo, g.M, g.K, lda_s) ||
         !make_map(&mBh, g.Bt_hi, g.N, g.K, g.ldbt) || !make_map(&mBl, g.Bt_lo, g.N, g.K, g.ldbt))
         return cudaErrorInvalidValue;
     const int mode = g.mode == 1 ? 1 : (g.head_w ? 2 : 0);

@@ -353,6 +353,23 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
             }
         m->bias[t] = to_f(b);
     }
+    // The first C0 entries of the feature vector are the centre's initial features, a constant per
+    // species; their image under the first layer is folded into a per-species bias so that the
+    // tensor-core GEMM can skip those K columns.
+    {
+        const std::vector<double>& Th = arr[13];
+        const std::vector<double>& b = arr[14];
+        m->type_bias.assign((size_t)T * F, 0.0f);
+        for (int t = 0; t < T; ++t)
+            for (int f = 0; f < F; ++f) {
+                double s = b[f];
+                for (int c = 0; c < C0; ++c) {
+                    const double x = ((double)m->X0[(size_t)t * C0 + c] - (double)m->mu[c]) * (double)m->inv_sigma[c];
+                    s += x * (double)(float)Th[(size_t)c * F + f];
+                }
+                m->type_bias[(size_t)t * F + f] = (float)s;
+            }
+    }
     // TF32 splits for the tensor-core GEMM: hi = round-to-nearest-even to 10 mantissa bits,
     // lo = the same rounding of (x - hi); both are exactly representable in TF32
     auto tf32 = [](float x) {

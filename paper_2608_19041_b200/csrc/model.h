@@ -18,6 +18,7 @@ struct HostModel {
     std::vector<float> X0, W1p, W2p, A1, A2, mu, inv_sigma;
     std::vector<std::vector<float>> theta, thetaT, bias;   // per hidden layer
     std::vector<std::vector<float>> theta_hi, theta_lo, thetaT_hi, thetaT_lo;   // TF32 splits
+    std::vector<float> type_bias;  // [T][F]: b_1 plus the first layer's image of the centre's calibrated initial features
     std::vector<float> w_head, e_ref;
     float b_head = 0;
     GauntSparse g123, g233;
