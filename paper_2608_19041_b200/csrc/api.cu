@@ -184,9 +184,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         }
     }
     if (want_grad) {
-        Scope sc(h, kForce, d_force ? 2 : 1);
-        API_CUDA(h, launch_force_assembly(nb, h->g, h->f_sorted, h->st));
-        if (d_force) API_CUDA(h, launch_scatter_forces(nb, h->f_sorted, d_force, h->d_err, h->st));
+        Scope sc(h, kForce, 1);
+        API_CUDA(h, launch_force_assembly(nb, h->g, d_force ? nullptr : h->f_sorted, d_force, h->d_err, h->st));
     }
     Scope sc(h, kReduce, d_atom_energy ? 3 : 2);
     API_CUDA(h, launch_reduce_energy_virial(h->e_atom, N, h->virial_part, vpart_used, h->scratch, h->d_out,
@@ -405,7 +404,9 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
         h->have_force = true;
     }
     for (int s = 0; s < nsteps; ++s) {
-        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, true, h->st)); }
+        // opening half kick and drift; from the second step on they were fused with the previous
+        // step's closing half kick
+        if (s == 0) { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, h->st)); }
         ++h->steps_since_build;
         bool rebuild = rebuild_every > 0 && h->steps_since_build >= rebuild_every;
         if (rebuild_every < 0) {
@@ -431,7 +432,8 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
             if ((rc = build_list(h, N, h->md_pos, h->type_o, L, pbc, skin)) != UMLMD_OK) return rc;
         }
         if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
-        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, false, h->st)); }
+        const bool last = s + 1 == nsteps;
+        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, h->st)); }
     }
     { Scope sc(h, kIntegrate, 2); API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st)); }
     rc = fetch_results(h, 11);

@@ -13,8 +13,10 @@ namespace {
 constexpr int kRedBlock = 256;
 constexpr int kRedMaxBlocks = 1024;
 
+// out (caller numbering, through perm) and / or f (sorted numbering) may be null
 __global__ void k_force_rows(int N, const int* __restrict__ row_ptr, const int* __restrict__ rev,
-                             const float* __restrict__ g, double* __restrict__ f) {
+                             const float* __restrict__ g, double* __restrict__ f, const int* __restrict__ perm,
+                             double* __restrict__ out, int* __restrict__ err) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= N) return;
     const int e0 = row_ptr[warp], e1 = row_ptr[warp + 1];
@@ -34,7 +36,14 @@ __global__ void k_force_rows(int N, const int* __restrict__ row_ptr, const int* 
         fy += __shfl_xor_sync(0xffffffffu, fy, off);
         fz += __shfl_xor_sync(0xffffffffu, fz, off);
     }
-    if (lane == 0) { f[3 * (size_t)warp] = fx; f[3 * (size_t)warp + 1] = fy; f[3 * (size_t)warp + 2] = fz; }
+    if (lane == 0) {
+        if (f) { f[3 * (size_t)warp] = fx; f[3 * (size_t)warp + 1] = fy; f[3 * (size_t)warp + 2] = fz; }
+        if (out) {
+            const size_t o = 3 * (size_t)perm[warp];
+            out[o] = fx; out[o + 1] = fy; out[o + 2] = fz;
+            if (!isfinite(fx) || !isfinite(fy) || !isfinite(fz)) atomicOr(err, kErrNonFinite);
+        }
+    }
 }
 
 __global__ void k_scatter3(int N, const int* __restrict__ perm, const double* __restrict__ in,
@@ -112,13 +121,17 @@ __global__ void __launch_bounds__(kRedBlock) k_final_reduce(const double* __rest
     }
 }
 
+// kicks = 1: v += (dt/2) a; kicks = 2: the closing half kick of one step and the opening half kick
+// of the next, applied one after the other exactly as two launches would; drift: x += dt v after them
 __global__ void k_vv(int64_t N, double* __restrict__ pos, double* __restrict__ vel, const double* __restrict__ force,
-                     const int* __restrict__ type, const double* __restrict__ inv_mass, double dt, bool drift) {
+                     const int* __restrict__ type, const double* __restrict__ inv_mass, double dt, int kicks, bool drift) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const double c = 0.5 * dt * kAccelUnit * inv_mass[type[i]];
     for (int k = 0; k < 3; ++k) {
-        double v = vel[3 * i + k] + c * force[3 * i + k];
+        const double f = force[3 * i + k];
+        double v = vel[3 * i + k] + c * f;
+        if (kicks == 2) v = v + c * f;
         vel[3 * i + k] = v;
         if (drift) pos[3 * i + k] += dt * v;
     }
@@ -159,10 +172,12 @@ inline void slices(int64_t N, int* blocks, int64_t* chunk) {
 
 int reduce_scratch_doubles(int64_t) { return kRedMaxBlocks; }
 
-cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* f_sorted, cudaStream_t st) {
+// forces in sorted numbering (f_sorted) and / or scattered to the caller's numbering (d_force)
+cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* f_sorted, double* d_force,
+                                  int* d_err, cudaStream_t st) {
     const int N = (int)nb.N;
     if (N == 0) return cudaSuccess;
-    k_force_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.row_ptr, nb.rev, g, f_sorted);
+    k_force_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.row_ptr, nb.rev, g, f_sorted, nb.perm, d_force, d_err);
     return cudaGetLastError();
 }
 
@@ -199,9 +214,9 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
 }
 
 cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force, const int* type,
-                                 const double* inv_mass, double dt, bool drift, cudaStream_t st) {
+                                 const double* inv_mass, double dt, int kicks, bool drift, cudaStream_t st) {
     if (N == 0) return cudaSuccess;
-    k_vv<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, pos, vel, force, type, inv_mass, dt, drift);
+    k_vv<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, pos, vel, force, type, inv_mass, dt, kicks, drift);
     return cudaGetLastError();
 }
 

@@ -82,8 +82,8 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers +
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad
 
 // ---- assemble.cu ---------------------------------------------------------------------
-cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted,
-                                  cudaStream_t st);
+cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted, double* d_force,
+                                  int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_atom_energy(const NeighborDev& nb, const double* e_sorted, double* d_out,
@@ -96,9 +96,8 @@ int reduce_scratch_doubles(int64_t N);
 cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stride, int width,
                                 float* out, cudaStream_t st);
 // velocity Verlet pieces (caller order, double)
-cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force,
-                                 const int* type, const double* inv_mass, double dt, bool drift,
-                                 cudaStream_t st);
+cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force, const int* type,
+                                 const double* inv_mass, double dt, int kicks, bool drift, cudaStream_t st);
 cudaError_t launch_kinetic_energy(int64_t N, const double* vel, const int* type, const double* mass,
                                   double* scratch, double* out, cudaStream_t st);
 
