@@ -66,3 +66,32 @@ def test_fullsize_sampled_parity(name, n_force, n_rows, modes):
         for a, ea in E_near.items():
             assert abs(Ei[a] - ea) <= 1e-5 * e_scale, (a, Ei[a], ea)
     m.close()
+
+
+@pytest.mark.parametrize("name", ["cfg3_water32400", "cfg4_hea128k", "cfg5_amorphous1m"])
+def test_fullsize_nve_drift_over_the_configured_run(name):
+    # the workload's own MD recipe (steps, time step, temperature, rebuild interval, skin) in the
+    # configuration bench.py times; drift = slope of a least-squares line through (E_pot + E_kin) / N
+    cfg = CONFIGS[name]
+    md = cfg["md"]
+    s = make_system(cfg["system"], md)
+    N = len(s["pos"])
+    m = _binding().Model(workload_blob(name))
+    pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
+    vel = torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
+    types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], md["skin"])
+    m.set_md_state(pos, vel, s["masses"])
+    chunk = max(1, md["steps"] // 10)
+    t, e = [0.0], []
+    ep, ek = m.step(0, md["dt_ps"], md["rebuild_every"])
+    e.append((ep + ek) / N)
+    for k in range(md["steps"] // chunk):
+        ep, ek = m.step(chunk, md["dt_ps"], md["rebuild_every"])
+        t.append((k + 1) * chunk * md["dt_ps"])
+        e.append((ep + ek) / N)
+    slope = np.polyfit(np.array(t), np.array(e), 1)[0]
+    print(f"{name}: NVE drift {slope:.3e} eV/atom/ps over {t[-1]:.3f} ps, E/N {min(e):.8f}..{max(e):.8f}")
+    assert np.isfinite(e).all()
+    assert abs(slope) <= 1e-5
+    m.close()
