@@ -14,6 +14,9 @@
 // 64-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (32 KB per
 // stage), so two CTAs fit on an SM and one CTA's epilogue overlaps the other's main loop
 // (a 128 x 128 x 8 TF32 MMA reads 8 KB of shared memory and is bound by that, ~94 cycles).
+// This kernel keeps the hi*hi sum and the cross terms in two accumulators (256 columns of
+// tensor memory per CTA); the persistent kernel further down, which needs all 512 columns
+// for its double buffering, sums all three products into one.
 // Warp 0 is the TMA producer, warp 1 issues the MMAs and owns the tensor-memory
 // allocation, warps 2-5 run the epilogue (one 32-lane quarter of tensor memory each).
 // Every mbarrier wait is bounded: on expiry the kernel flags an error word and carries on,
@@ -35,7 +38,7 @@ constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 8 KB, also BN * BK * 4
 constexpr uint32_t STAGE_BYTES = 4 * TILE_BYTES;      // A_hi, A_lo, B_hi, B_lo
 constexpr uint32_t BAR_BYTES = 128;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + BAR_BYTES;
-constexpr uint32_t TMEM_COLS = 128;
+constexpr uint32_t TMEM_COLS = 256;                   // two accumulators: hi*hi, and the two cross terms
 constexpr int EPITCH = BN + 4;                        // epilogue staging pitch: 16-byte rows, odd in 16-byte units
 constexpr int kSpinLimit = 4000000;
 
@@ -161,9 +164,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                 for (int k = 0; k < BK / 8; ++k) {
                     const uint64_t ah = umma_desc(sa + k * 32), al = umma_desc(sa + TILE_BYTES + k * 32);
                     const uint64_t bh = umma_desc(sa + 2 * TILE_BYTES + k * 32), bl = umma_desc(sa + 3 * TILE_BYTES + k * 32);
-                    umma_tf32(tmem, al, bh, kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    umma_tf32(tmem, ah, bl, kIdesc, 1u);
-                    umma_tf32(tmem, ah, bh, kIdesc, 1u);
+                    // The accumulator truncates once per instruction.  The cross terms, 2^-11 of
+                    // the result, get an accumulator of their own, where that loss is 2^-11 as
+                    // small, and the main sum sees a third of the instructions.
+                    const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                    umma_tf32(tmem + BN, al, bh, kIdesc, acc);
+                    umma_tf32(tmem + BN, ah, bl, kIdesc, 1u);
+                    umma_tf32(tmem, ah, bh, kIdesc, acc);
                 }
                 umma_commit(bars + 8 * (STAGES + s));      // frees the stage when these MMAs retire
             }
@@ -181,11 +188,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
         float* stage = reinterpret_cast<float*>(smem_raw + (tiles - raw)) + (size_t)q * 32 * EPITCH;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
-            float v[32];
+            float v[32], w[32];
             tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN + c0), w);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(stage + lane * EPITCH + c0 + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                *reinterpret_cast<float4*>(stage + lane * EPITCH + c0 + 4 * j) =
+                    make_float4(v[4 * j] + w[4 * j], v[4 * j + 1] + w[4 * j + 1], v[4 * j + 2] + w[4 * j + 2], v[4 * j + 3] + w[4 * j + 3]);
         }
         __syncwarp();
         const int n = n0 + 4 * lane;
