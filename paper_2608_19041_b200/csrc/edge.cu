@@ -1,17 +1,18 @@
 // Fused per-edge kernels: edge featurisation + per-destination aggregation (forward) and
 // the recomputing edge backward pass that returns dE/dr_ij for every edge.
 //
-// One warp owns one destination atom and walks its contiguous CSR interval.  Edges are
-// taken in batches of 32: first each lane computes the geometry of one edge (displacement
-// from double-precision positions, regularised length, direction, cutoff envelope, table
-// row), then the batch is replayed with lanes split over channels -- a group of C0/4 lanes
-// handles one edge, each lane holding four consecutive channels, so table and pair-cache
-// reads are 16-byte vector loads that a group issues as one contiguous segment.  The S+2
-// sums live in registers and are written once per destination; nothing per-edge is stored
-// in the forward pass.  The backward pass recomputes the same per-edge quantities from the
-// same cubic polynomial (so the force is the exact derivative of the interpolated
-// energy), contracts them with dE/d(sums) and writes one 3-vector per edge; the virial is
-// accumulated in the same pass.
+// One warp owns one destination atom and walks its contiguous CSR interval, 32 listed edges
+// at a time: each lane computes the geometry of one edge (displacement from double-precision
+// positions, regularised length, direction, cutoff envelope, table row) and the edges inside
+// the cutoff are queued in shared memory.  Full batches of queued edges are then processed
+// with lanes split over channels -- a group of lanes handles one edge, each lane holding one
+// or two runs of four consecutive channels, so table and pair-cache reads are 16-byte vector
+// loads that a group issues as contiguous segments -- followed by a lane-per-edge phase for
+// the degree >= 1 blocks.  The S+2 sums live in registers and are written once per
+// destination; nothing per-edge is stored in the forward pass.  The backward pass recomputes
+// the same per-edge quantities from the same cubic polynomial (so the force is the exact
+// derivative of the interpolated energy), contracts them with dE/d(sums) and writes one
+// 3-vector per edge; the virial is accumulated in the same pass.
 //
 // Harmonics are evaluated with |u|^2 set to one; the regularised direction differs from a
 // unit vector by eps^2/rho^2, far below single precision.

@@ -8,9 +8,10 @@
 // A_lo B_hi + A_hi B_lo + A_hi B_hi (the lo*lo term, ~2^-22, is dropped).  Both parts are
 // exactly representable in TF32, so the result does not depend on how the tensor core
 // treats the low mantissa bits.  Weights are split once on the host; activations are split
-// by the epilogue that produces them (or, for the first GEMM of a chain, by a small kernel).
+// by the kernel that produces them (the invariants kernel, a GEMM epilogue; a small split kernel
+// remains for callers that hand in an unsplit operand).
 //
-// Tiling: one CTA computes a 128 x 128 output tile; K advances in blocks of 16 floats (one
+// Tiling of the first kernel below: one CTA computes a 128 x 128 output tile; K advances in blocks of 16 floats (one
 // 64-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (32 KB per
 // stage), so two CTAs fit on an SM and one CTA's epilogue overlaps the other's main loop
 // (a 128 x 128 x 8 TF32 MMA reads 8 KB of shared memory and is bound by that, ~94 cycles).
