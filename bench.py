@@ -294,6 +294,9 @@ def run_ours(args):
 
     def run_steps(k):
         if not static:
+            if args.nvt:
+                ep, ek, _ = model.step_nvt(k, dt, md["temperature"], 100.0 * dt, every)
+                return ep, ek
             return model.step(k, dt, every)
         for _ in range(k):
             out = model.compute(pos, forces=True, virial=True)
@@ -382,6 +385,7 @@ def run_ours(args):
                     config=dict(workload=name, n_atoms=N, edges_within_rc=e_rc, edges_in_list=e_list,
                                 profile={k: p[k] for k in ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T")},
                                 dt_ps=dt, rebuild_every=every, skin=skin,
+                                ensemble="nvt (Nose-Hoover chain, period 100 dt)" if (args.nvt and not static) else "nve",
                                 mlp_path=args.mlp_path, parallelism="replicas" if world > 1 else "single",
                                 **({"published": pub} if pub else {}),
                                 cache="working set per step exceeds L2" if N >= 100000 else "fits in L2 (launch-bound)"),
@@ -420,6 +424,7 @@ def main():
     ap.add_argument("--node-tile", type=int, default=0)
     ap.add_argument("--atoms", type=int, default=0, help="amorphous and lattice workloads: (about) this many atoms in a smaller box of the same recipe")
     ap.add_argument("--modes", type=int, default=-1, help="override the number R of shared radial modes of the workload's profile")
+    ap.add_argument("--nvt", action="store_true", help="time the Nose-Hoover-chain NVT driver instead of NVE")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -165,6 +165,19 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
                double* e_kin);
 
 /*
+ * The same driver at constant temperature: velocity Verlet between two half-step
+ * propagations of a Nose-Hoover chain of three thermostats (Martyna-Tuckerman-Klein form,
+ * the integrator behind the NVT runs the paper times; the model's hot path is unchanged).
+ * temperature_K is the target, t_damp_ps the thermostat period: the first thermostat has
+ * mass (3N - 3) kT t_damp^2, the others kT t_damp^2.  The chain starts at rest after every
+ * umlmd_set_md_state and carries over between calls.  e_conserved (may be NULL) receives
+ * E_pot + E_kin + the chain's energy, which this dynamics conserves.  The system needs at
+ * least two atoms.  Other arguments and errors as for umlmd_step.
+ */
+int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double temperature_K,
+                   double t_damp_ps, double* e_pot, double* e_kin, double* e_conserved);
+
+/*
  * Diagnostics used by the parity tests: copy out per-atom intermediates of the last
  * umlmd_compute, in the caller's numbering.  Each pointer may be NULL.
  *   d_state  [N, S+2] float: unnormalised sums A (degree, then m, then channel), s0, s1

@@ -23,6 +23,7 @@ ERRORS = {
 EXPORTS = [
     "umlmd_profile_widths", "umlmd_create", "umlmd_destroy", "umlmd_query", "umlmd_last_error",
     "umlmd_build_neighbors", "umlmd_get_neighbors", "umlmd_compute", "umlmd_set_md_state", "umlmd_step",
+    "umlmd_step_nvt",
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
     "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
 ]
@@ -66,6 +67,8 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_compute.argtypes = [vp, vp, ctypes.POINTER(dbl), vp, ctypes.POINTER(dbl), vp]
     lib.umlmd_set_md_state.argtypes = [vp, vp, vp, ctypes.POINTER(dbl)]
     lib.umlmd_step.argtypes = [vp, ctypes.c_int, dbl, ctypes.c_int, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.umlmd_step_nvt.argtypes = [vp, ctypes.c_int, dbl, ctypes.c_int, dbl, dbl, ctypes.POINTER(dbl), ctypes.POINTER(dbl),
+                                   ctypes.POINTER(dbl)]
     lib.umlmd_get_intermediates.argtypes = [vp, vp, vp]
     lib.umlmd_eval_radial_table.argtypes = [vp, i64, ctypes.POINTER(dbl), ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.umlmd_eval_pair_cache.argtypes = [vp, i32, i32, ctypes.POINTER(dbl)]
@@ -209,6 +212,16 @@ class Model:
         if rc != OK:
             self._raise(rc)
         return ep.value, ek.value
+
+    def step_nvt(self, nsteps, dt_ps, temperature_K, t_damp_ps, rebuild_every=0):
+        """(e_pot, e_kin, conserved energy) after nsteps of Nose-Hoover-chain NVT."""
+        ep, ek, ec = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+        rc = self._lib.umlmd_step_nvt(self._h, int(nsteps), ctypes.c_double(dt_ps), int(rebuild_every),
+                                      ctypes.c_double(temperature_K), ctypes.c_double(t_damp_ps), ctypes.byref(ep),
+                                      ctypes.byref(ek), ctypes.byref(ec))
+        if rc != OK:
+            self._raise(rc)
+        return ep.value, ek.value, ec.value
 
     def get_intermediates(self):
         q = self.query()

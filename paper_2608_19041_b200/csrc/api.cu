@@ -36,6 +36,8 @@ struct umlmd {
     double* d_mass = nullptr; double* d_inv_mass = nullptr;
     bool have_md = false, have_force = false;
     int steps_since_build = 0;
+    double* d_nhc = nullptr;      // thermostat chain on the device: eta[M], v_eta[M], scale, kinetic energy
+    bool nhc_reset = true;
     // launch accounting and optional per-class timing
     bool prof_on = false;
     struct Span { int cls; cudaEvent_t a, b; };
@@ -287,7 +289,7 @@ int umlmd_destroy(umlmd_t* h) {
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
     void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
-                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass};
+                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
@@ -388,7 +390,37 @@ int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* m
     API_CUDA(h, cudaStreamSynchronize(h->st));
     if (h->nb.N > h->md_cap || !h->md_force) API_CUDA(h, dev_ensure(&h->md_force, &h->md_cap, h->nb.N * 3));
     h->md_pos = d_pos; h->md_vel = d_vel;
-    h->have_md = true; h->have_force = false;
+    h->have_md = true; h->have_force = false; h->nhc_reset = true;
+    return UMLMD_OK;
+}
+
+// after a drift: rebuild the list if the schedule (rebuild_every > 0) or the displacement
+// criterion (rebuild_every < 0) asks for it
+static int maybe_rebuild(umlmd_t* h, int rebuild_every) {
+    const int64_t N = h->nb.N;
+    bool rebuild = rebuild_every > 0 && h->steps_since_build >= rebuild_every;
+    if (rebuild_every < 0) {
+        // displacement-triggered: the gather pass flags any atom that has moved more than half
+        // the skin since the build; read the flag (one host synchronisation per step)
+        API_CUDA(h, launch_gather_positions(h->nb, h->md_pos, h->d_err, h->st));
+        API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+        API_CUDA(h, cudaStreamSynchronize(h->st));
+        const int word = *h->h_err;
+        if (word & ~kErrStale) {
+            API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+            return decode_device_errors(h, word & ~kErrStale);
+        }
+        if (word & kErrStale) {
+            API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+            rebuild = true;
+        }
+    }
+    if (rebuild) {
+        const double skin = h->nb.skin;
+        const double L[3] = {h->nb.L[0], h->nb.L[1], h->nb.L[2]};
+        const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};
+        return build_list(h, N, h->md_pos, h->type_o, L, pbc, skin);
+    }
     return UMLMD_OK;
 }
 
@@ -406,40 +438,85 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
     for (int s = 0; s < nsteps; ++s) {
         // opening half kick and drift; from the second step on they were fused with the previous
         // step's closing half kick
-        if (s == 0) { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, h->st)); }
+        if (s == 0) { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, nullptr, h->st)); }
         ++h->steps_since_build;
-        bool rebuild = rebuild_every > 0 && h->steps_since_build >= rebuild_every;
-        if (rebuild_every < 0) {
-            // displacement-triggered: the gather pass flags any atom that has moved more than half
-            // the skin since the build; read the flag (one host synchronisation per step)
-            API_CUDA(h, launch_gather_positions(h->nb, h->md_pos, h->d_err, h->st));
-            API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
-            API_CUDA(h, cudaStreamSynchronize(h->st));
-            const int word = *h->h_err;
-            if (word & ~kErrStale) {
-                API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
-                return decode_device_errors(h, word & ~kErrStale);
-            }
-            if (word & kErrStale) {
-                API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
-                rebuild = true;
-            }
-        }
-        if (rebuild) {
-            const double skin = h->nb.skin;
-            const double L[3] = {h->nb.L[0], h->nb.L[1], h->nb.L[2]};
-            const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};
-            if ((rc = build_list(h, N, h->md_pos, h->type_o, L, pbc, skin)) != UMLMD_OK) return rc;
-        }
+        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return rc;
         if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
         const bool last = s + 1 == nsteps;
-        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, h->st)); }
+        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, nullptr, h->st)); }
     }
     { Scope sc(h, kIntegrate, 2); API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st)); }
     rc = fetch_results(h, 11);
     if (rc != UMLMD_OK) return rc;
     if (e_pot) *e_pot = h->h_out[0];
     if (e_kin) *e_kin = h->h_out[10];
+    return UMLMD_OK;
+}
+
+int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double temperature_K, double t_damp_ps,
+                   double* e_pot, double* e_kin, double* e_conserved) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
+    if (!h->have_md) return fail(h, UMLMD_E_NO_MD_STATE, "umlmd_set_md_state must be called first");
+    if (nsteps < 0 || !(dt_ps > 0) || !std::isfinite(dt_ps) || !(temperature_K > 0) || !std::isfinite(temperature_K) ||
+        !(t_damp_ps > 0) || !std::isfinite(t_damp_ps))
+        return fail(h, UMLMD_E_INVALID_ARG, "bad step count, time step, temperature or damping time");
+    const int64_t N = h->nb.N;
+    if (N < 2) return fail(h, UMLMD_E_INVALID_ARG, "the thermostat needs at least two atoms");
+    constexpr int M = kNhcChain;
+    int rc;
+    if (!h->d_nhc) { int64_t c = 0; API_CUDA(h, dev_ensure(&h->d_nhc, &c, 2 * M + 2)); h->nhc_reset = true; }
+    if (h->nhc_reset) { API_CUDA(h, cudaMemsetAsync(h->d_nhc, 0, sizeof(double) * (2 * M + 2), h->st)); h->nhc_reset = false; }
+    NhcParams p;
+    p.dof = 3.0 * (double)N - 3.0;
+    p.kT = kBoltzmann * temperature_K;
+    p.Q[0] = p.dof * p.kT * t_damp_ps * t_damp_ps;
+    for (int k = 1; k < M; ++k) p.Q[k] = p.kT * t_damp_ps * t_damp_ps;
+    p.dt_half = 0.5 * dt_ps;
+    if (!h->have_force) {
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        h->have_force = true;
+    }
+    double* d_ke = h->d_out + 10;
+    double* d_scale = h->d_nhc + 2 * M;
+    if (nsteps > 0) {      // opening half step of the chain for the first step
+        Scope sc(h, kIntegrate, 3);
+        API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, d_ke, h->st));
+        API_CUDA(h, launch_nhc(h->d_nhc, d_ke, 1, p, h->st));
+    }
+    for (int s = 0; s < nsteps; ++s) {
+        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, d_scale, h->st)); }
+        ++h->steps_since_build;
+        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return rc;
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        const bool last = s + 1 == nsteps;
+        Scope sc(h, kIntegrate, 4);
+        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, false, nullptr, h->st));
+        API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, d_ke, h->st));
+        // closing half step of the chain, and the next step's opening one in the same launch
+        API_CUDA(h, launch_nhc(h->d_nhc, d_ke, last ? 1 : 2, p, h->st));
+    }
+    if (nsteps > 0) {      // the last scale factor has not been applied to the velocities yet
+        Scope sc(h, kIntegrate, 1);
+        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 0, false, d_scale, h->st));
+    } else {
+        Scope sc(h, kIntegrate, 2);
+        API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, d_ke, h->st));
+        API_CUDA(h, cudaMemcpyAsync(h->d_nhc + 2 * M + 1, d_ke, sizeof(double), cudaMemcpyDeviceToDevice, h->st));
+    }
+    double chain[2 * M + 2];
+    API_CUDA(h, cudaMemcpyAsync(chain, h->d_nhc, sizeof(chain), cudaMemcpyDeviceToHost, h->st));
+    rc = fetch_results(h, 10);
+    if (rc != UMLMD_OK) return rc;
+    const double ke = chain[2 * M + 1];
+    if (e_pot) *e_pot = h->h_out[0];
+    if (e_kin) *e_kin = ke;
+    if (e_conserved) {
+        double e = h->h_out[0] + ke + p.dof * p.kT * chain[0];
+        for (int k = 0; k < M; ++k) e += 0.5 * p.Q[k] * chain[M + k] * chain[M + k];
+        for (int k = 1; k < M; ++k) e += p.kT * chain[k];
+        *e_conserved = e;
+    }
     return UMLMD_OK;
 }
 

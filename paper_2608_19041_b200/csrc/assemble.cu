@@ -121,20 +121,61 @@ __global__ void __launch_bounds__(kRedBlock) k_final_reduce(const double* __rest
     }
 }
 
-// kicks = 1: v += (dt/2) a; kicks = 2: the closing half kick of one step and the opening half kick
-// of the next, applied one after the other exactly as two launches would; drift: x += dt v after them
+// kicks = 0: none; kicks = 1: v += (dt/2) a; kicks = 2: the closing half kick of one step and the
+// opening half kick of the next, applied one after the other exactly as two launches would; drift:
+// x += dt v after them; scale (may be null): the thermostat's velocity factor, applied first
 __global__ void k_vv(int64_t N, double* __restrict__ pos, double* __restrict__ vel, const double* __restrict__ force,
-                     const int* __restrict__ type, const double* __restrict__ inv_mass, double dt, int kicks, bool drift) {
+                     const int* __restrict__ type, const double* __restrict__ inv_mass, double dt, int kicks, bool drift,
+                     const double* __restrict__ scale) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const double c = 0.5 * dt * kAccelUnit * inv_mass[type[i]];
+    const double sc = scale ? *scale : 1.0;
     for (int k = 0; k < 3; ++k) {
         const double f = force[3 * i + k];
-        double v = vel[3 * i + k] + c * f;
+        double v = vel[3 * i + k];
+        if (scale) v *= sc;
+        if (kicks >= 1) v = v + c * f;
         if (kicks == 2) v = v + c * f;
         vel[3 * i + k] = v;
         if (drift) pos[3 * i + k] += dt * v;
     }
+}
+
+// Nose-Hoover chain of kNhcChain thermostats (Martyna-Tuckerman-Klein form): `halves` successive
+// half-step propagations of the chain given the current kinetic energy; returns the product of the
+// velocity scale factors and the kinetic energy after scaling.  One thread: the chain is a handful
+// of scalars.  st = [eta[M], v_eta[M], scale, kinetic energy]
+__global__ void k_nhc(double* __restrict__ st, const double* __restrict__ ke_in, int halves, NhcParams p) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    constexpr int M = kNhcChain;
+    double* eta = st;
+    double* v = st + M;
+    double ke2 = 2.0 * (ke_in ? *ke_in : st[2 * M + 1]);
+    double scale = 1.0;
+    const double d2 = p.dt_half, d4 = 0.5 * d2, d8 = 0.25 * d2;
+    for (int h = 0; h < halves; ++h) {
+        double G = (p.Q[M - 2] * v[M - 2] * v[M - 2] - p.kT) / p.Q[M - 1];
+        v[M - 1] += G * d4;
+        for (int k = M - 2; k >= 0; --k) {
+            const double e = exp(-v[k + 1] * d8);
+            G = (k == 0 ? (ke2 - p.dof * p.kT) : (p.Q[k - 1] * v[k - 1] * v[k - 1] - p.kT)) / p.Q[k];
+            v[k] = (v[k] * e + G * d4) * e;
+        }
+        const double sfac = exp(-v[0] * d2);
+        scale *= sfac;
+        ke2 *= sfac * sfac;
+        for (int k = 0; k < M; ++k) eta[k] += v[k] * d2;
+        for (int k = 0; k < M - 1; ++k) {
+            const double e = exp(-v[k + 1] * d8);
+            G = (k == 0 ? (ke2 - p.dof * p.kT) : (p.Q[k - 1] * v[k - 1] * v[k - 1] - p.kT)) / p.Q[k];
+            v[k] = (v[k] * e + G * d4) * e;
+        }
+        G = (p.Q[M - 2] * v[M - 2] * v[M - 2] - p.kT) / p.Q[M - 1];
+        v[M - 1] += G * d4;
+    }
+    st[2 * M] = scale;
+    st[2 * M + 1] = 0.5 * ke2;
 }
 
 __global__ void __launch_bounds__(kRedBlock) k_ke_slices(const double* __restrict__ vel, const int* __restrict__ type,
@@ -214,9 +255,15 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
 }
 
 cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force, const int* type,
-                                 const double* inv_mass, double dt, int kicks, bool drift, cudaStream_t st) {
+                                 const double* inv_mass, double dt, int kicks, bool drift, const double* d_scale,
+                                 cudaStream_t st) {
     if (N == 0) return cudaSuccess;
-    k_vv<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, pos, vel, force, type, inv_mass, dt, kicks, drift);
+    k_vv<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, pos, vel, force, type, inv_mass, dt, kicks, drift, d_scale);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_nhc(double* d_state, const double* d_ke, int halves, const NhcParams& p, cudaStream_t st) {
+    k_nhc<<<1, 32, 0, st>>>(d_state, d_ke, halves, p);
     return cudaGetLastError();
 }
 

@@ -97,7 +97,13 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
                                 float* out, cudaStream_t st);
 // velocity Verlet pieces (caller order, double)
 cudaError_t launch_vv_kick_drift(int64_t N, double* pos, double* vel, const double* force, const int* type,
-                                 const double* inv_mass, double dt, int kicks, bool drift, cudaStream_t st);
+                                 const double* inv_mass, double dt, int kicks, bool drift, const double* d_scale,
+                                 cudaStream_t st);
+// Nose-Hoover chain thermostat: chain length, parameters (energies in eV, times in ps) and the
+// propagation of `halves` half steps on the device; d_state = [eta[M], v_eta[M], scale, kinetic energy]
+constexpr int kNhcChain = 3;
+struct NhcParams { double dof, kT, Q[kNhcChain], dt_half; };
+cudaError_t launch_nhc(double* d_state, const double* d_ke, int halves, const NhcParams& p, cudaStream_t st);
 cudaError_t launch_kinetic_energy(int64_t N, const double* vel, const int* type, const double* mass,
                                   double* scratch, double* out, cudaStream_t st);
 

@@ -148,3 +148,85 @@ def test_displacement_triggered_rebuild():
     assert abs(res[-1][1] - res[1][1]) < 1e-6 * max(1.0, abs(res[1][1]))
     assert res[-1][3] < res[1][3]          # fewer builds than one per step
 
+
+
+def _nhc_half(ke2, eta, veta, Q, dof, kT, dt_half):
+    """One half-step propagation of a Nose-Hoover chain (Martyna-Tuckerman-Klein), written out from
+    the equations of motion; returns the velocity scale factor and 2 * KE after scaling."""
+    M = len(Q)
+    d2, d4, d8 = dt_half, 0.5 * dt_half, 0.25 * dt_half
+
+    def force(k):
+        return ((ke2 - dof * kT) if k == 0 else (Q[k - 1] * veta[k - 1] ** 2 - kT)) / Q[k]
+
+    veta[M - 1] += force(M - 1) * d4
+    for k in range(M - 2, -1, -1):
+        e = np.exp(-veta[k + 1] * d8)
+        veta[k] = (veta[k] * e + force(k) * d4) * e
+    s = np.exp(-veta[0] * d2)
+    ke2 = ke2 * s * s
+    for k in range(M):
+        eta[k] += veta[k] * d2
+    for k in range(M - 1):
+        e = np.exp(-veta[k + 1] * d8)
+        veta[k] = (veta[k] * e + force(k) * d4) * e
+    veta[M - 1] += force(M - 1) * d4
+    return s, ke2
+
+
+def test_nvt_step_equals_hand_written_nose_hoover_chain():
+    cfg, s, blob, m, pos, vel, types = _setup("cfg2_cu4000")
+    dt, T, tdamp = cfg["md"]["dt_ps"], 450.0, 0.05
+    N = len(s["pos"])
+    m2 = _binding().Model(blob)
+    p2, v2 = pos.clone(), vel.clone()
+    m2.build_neighbors(p2, types, s["cell"], s["pbc"], cfg["md"]["skin"])
+    mass = torch.as_tensor(s["masses"][s["types"]], dtype=torch.float64).cuda()[:, None]
+    inv_m = 1.0 / mass
+
+    def ke2_of(v):
+        return (mass * v ** 2).sum().item() / EV_PER_AMU_IN_A2_PS2
+
+    dof, kT = 3.0 * N - 3.0, KB_EV_PER_K * T
+    Q = [dof * kT * tdamp ** 2, kT * tdamp ** 2, kT * tdamp ** 2]
+    eta, veta = [0.0] * 3, [0.0] * 3
+    f = m2.compute(p2)["forces"]
+    nsteps = 5
+    for _ in range(nsteps):
+        sc, _ = _nhc_half(ke2_of(v2), eta, veta, Q, dof, kT, 0.5 * dt)
+        v2 *= sc
+        v2 += 0.5 * dt * EV_PER_AMU_IN_A2_PS2 * inv_m * f
+        p2 += dt * v2
+        out = m2.compute(p2)
+        f = out["forces"]
+        v2 += 0.5 * dt * EV_PER_AMU_IN_A2_PS2 * inv_m * f
+        sc, _ = _nhc_half(ke2_of(v2), eta, veta, Q, dof, kT, 0.5 * dt)
+        v2 *= sc
+    e_pot, e_kin, e_cons = m.step_nvt(nsteps, dt, T, tdamp)
+    assert (pos - p2).abs().max().item() < 1e-11
+    assert (vel - v2).abs().max().item() < 1e-9
+    ke = 0.5 * ke2_of(v2)
+    assert abs(e_kin - ke) < 1e-9 * ke
+    cons = out["energy"] + ke + sum(0.5 * Q[k] * veta[k] ** 2 for k in range(3)) + dof * kT * eta[0] + kT * (eta[1] + eta[2])
+    assert abs(e_cons - cons) < 1e-8 * max(1.0, abs(cons))
+
+
+def test_nvt_drives_the_temperature_to_the_target_and_conserves_its_energy():
+    # The jittered crystal starts with 300 K of kinetic energy and, left alone, settles near 225 K
+    # as it equipartitions; the thermostat (period 0.1 ps = 100 steps) brings it back to 300 K.
+    # The conserved energy of the extended system is held to second order in the time step
+    # (measured: 1e-6 eV/atom here, 1e-4 when the target is doubled with a 0.05 ps period,
+    # a quarter of that at half the time step).
+    cfg, s, blob, m, pos, vel, types = _setup("cfg2_cu4000")
+    md = cfg["md"]
+    N = len(s["pos"])
+    T, tdamp = 300.0, 0.1
+    temps, cons = [], []
+    _, _, c0 = m.step_nvt(0, md["dt_ps"], T, tdamp, md["rebuild_every"])
+    for _ in range(10):
+        ep, ek, ec = m.step_nvt(50, md["dt_ps"], T, tdamp, md["rebuild_every"])
+        temps.append(2 * ek / ((3 * N - 3) * KB_EV_PER_K))
+        cons.append(ec)
+    print("T:", " ".join(f"{t:.0f}" for t in temps), " conserved/N drift:", (cons[-1] - c0) / N)
+    assert abs(np.mean(temps[5:]) - T) < 0.1 * T                    # thermostatted to the target
+    assert max(abs(c - c0) for c in cons) / N < 5e-6                 # over 0.5 ps
