@@ -89,6 +89,8 @@ def test_calls_before_a_neighbor_build_fail_cleanly():
     e = ctypes.c_double()
     assert lib.umlmd_compute(m._h, None, ctypes.byref(e), None, None, None) == -5
     assert lib.umlmd_step(m._h, 1, 0.001, 0, None, None) == -5
+    assert lib.umlmd_step_nvt(m._h, 1, 0.001, 0, 300.0, 0.1, None, None, None) == -5
+    assert lib.umlmd_step_nvt(None, 1, 0.001, 0, 300.0, 0.1, None, None, None) == -1
     assert b"build_neighbors" in lib.umlmd_last_error(m._h)
     q = m.query()
     assert q["n_atoms"] == 0 and q["table_rows"] == 3000 and q["rc"] == 6.0
