@@ -114,13 +114,18 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ algorithmic work
 
-def work_model(p, n_atoms, e_rc, e_list):
-    """Algorithmic FLOPs (FMA = 2) and compulsory HBM bytes per evaluation, per kernel class."""
+def work_model(p, n_atoms, e_rc, e_list, one_species=False):
+    """Algorithmic FLOPs (FMA = 2) and compulsory HBM bytes per evaluation, per kernel class.
+    With one species the library tabulates the amplitude of that pair directly, so an edge costs
+    the Horner evaluation of C0 channels and no modes or pair modulation: count that, not more."""
     C0, R, S, D, F, NH, C1 = p["C0"], p["R"], p["S"], p["D_out"], p["F"], p["n_hidden"], p["C1"]
     # per edge: cubic Horner of the table channels (6 flops a value, 4 more for its derivative),
     # pair modulation, the S+2 accumulations, envelope and harmonics
     fwd_edge = 6 * (C0 + R) + 2 * C0 * (1 + R) + 2 * S + C0 + C1 + 60
     bwd_edge = 10 * (C0 + R) + 4 * C0 * (1 + R) + 4 * S + 2 * C0 + 250
+    if one_species:
+        fwd_edge = 6 * C0 + 2 * S + C0 + C1 + 60
+        bwd_edge = 10 * C0 + 4 * S + 2 * C0 + 250
     mlp = 2 * (D * F + (NH - 1) * F * F + F)
     return {
         "edge_forward": dict(flops=fwd_edge * e_rc, bytes=8 * e_list + n_atoms * (28 + 4 * (S + 2)), pipe="alu"),
@@ -325,7 +330,7 @@ def run_ours(args):
     prof = model.get_profile()
     model.set_profiling(False)
     peaks = measured_peaks()
-    work = work_model(p, N, e_rc, e_list)
+    work = work_model(p, N, e_rc, e_list, one_species=len(np.unique(s["types"])) == 1)
     total_ms = sum(v[0] for v in prof.values()) or 1.0
     kernels = []
     for cname, (kms, kl) in prof.items():

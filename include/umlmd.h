@@ -113,6 +113,11 @@ const char* umlmd_last_error(const umlmd_t* h);
  * dy*dy) + dz*dz, d2 < r_list*r_list, without fused multiply-add, so that the edge set is
  * reproducible bit for bit.  Atoms are renumbered internally in cell order; all outputs
  * of this library are in the caller's numbering.
+ * When all N atoms have the same species s, the call also tabulates the edge amplitude of
+ * the one ordered pair (s, s), psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu
+ * q_mu(rho), as its own cubic table (the same linear combination of the coefficient rows of
+ * the radial table), and umlmd_compute reads that table instead of the radial table, the
+ * pair cache and the shared modes.  The species are re-examined at every call.
  */
 int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type,
                           const double cell[9], const int pbc[3], double skin);

@@ -31,6 +31,8 @@ struct umlmd {
     double* virial_part = nullptr; int64_t vpart_cap = 0;
     double* scratch = nullptr; double* d_out = nullptr; int* d_err = nullptr;
     double* h_out = nullptr; int* h_err = nullptr;      // pinned
+    bool one_species = false;                           // set by umlmd_build_neighbors
+    float* table_uni = nullptr;                         // amplitude table of the one pair, when one_species
     // MD
     double* md_pos = nullptr; double* md_vel = nullptr; double* md_force = nullptr; int64_t md_cap = 0;
     double* d_mass = nullptr; double* d_inv_mass = nullptr;
@@ -154,6 +156,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         const int n = N - a0 < B ? N - a0 : B;
         EdgeArgs ea;
         ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.type_s = nb.type_s;
+        ea.table_uni = h->one_species ? h->table_uni : nullptr;
         ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
@@ -289,7 +292,7 @@ int umlmd_destroy(umlmd_t* h) {
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
     void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
-                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc};
+                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
@@ -330,12 +333,25 @@ int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int3
     int rc = build_list(h, N, d_pos, d_type, L, pbc, skin);
     if (rc != UMLMD_OK) return rc;
     if (N > 0) API_CUDA(h, cudaMemcpyAsync(h->type_o, d_type, sizeof(int) * N, cudaMemcpyDeviceToDevice, h->st));
+    // one species throughout: the edge kernels then keep the pair rows in registers
+    API_CUDA(h, launch_species_differ(N, d_type, h->d_err + 1, h->st));
+    h->launches_total += N > 0;
     // surface device-side findings of the build (non-finite positions, image range)
-    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, 2 * sizeof(int), cudaMemcpyDeviceToHost, h->st));
     API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
     API_CUDA(h, cudaStreamSynchronize(h->st));
+    h->one_species = N > 0 && h->h_err[1] == 0;
     rc = decode_device_errors(h, *h->h_err);
-    if (rc != UMLMD_OK) h->have_list = false;
+    if (rc != UMLMD_OK) { h->have_list = false; return rc; }
+    if (h->one_species) {
+        if (!h->table_uni) {
+            void* p = nullptr;
+            API_CUDA(h, dev_malloc(&p, sizeof(float) * (size_t)h->d.n_rows * 4 * h->d.C0));
+            h->table_uni = (float*)p;
+        }
+        API_CUDA(h, launch_fuse_pair_table(h->d, h->md.table, h->md.pairmod, h->type_o, h->table_uni, h->st));
+        h->launches_total += 1;
+    }
     return rc;
 }
 

@@ -75,6 +75,13 @@ __global__ void k_unsort_rows(int N, const int* __restrict__ perm, const float* 
     for (int k = lane; k < width; k += 32) w[k] = r[k];
 }
 
+// *flag = 1 when some atom's species differs from the first atom's (flag cleared by the caller)
+__global__ void k_species_differ(int64_t N, const int* __restrict__ type, int* __restrict__ flag) {
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const bool differs = i < N && type[i] != type[0];
+    if (__any_sync(0xffffffffu, differs) && (threadIdx.x & 31) == 0) *flag = 1;
+}
+
 __device__ __forceinline__ double block_sum(double v, double* sh) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
@@ -251,6 +258,13 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
     const int N = (int)nb.N;
     if (N == 0) return cudaSuccess;
     k_unsort_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.perm, in, stride, width, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_species_differ(int64_t N, const int* type, int* d_flag, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(d_flag, 0, sizeof(int), st);
+    if (e != cudaSuccess || N == 0) return e;
+    k_species_differ<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, type, d_flag);
     return cudaGetLastError();
 }
 

@@ -149,10 +149,16 @@ __device__ __forceinline__ void eval_modes(const EdgeArgs& a, const int4* qes, i
 }
 
 // amplitude psi (and d psi / d rho) of this lane's four channels for one edge; qm / dqm: the
-// edge's parked radial modes (only read when HASR)
-template <int C0, bool HASR, bool DERIV>
+// edge's parked radial modes (only read when HASR).  UNI: the system has one species, so psi is
+// a function of rho alone and comes from the table of that pair (a.table_uni, row pitch C0),
+// without pair rows or modes
+template <int C0, bool HASR, bool DERIV, bool UNI>
 __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, int pair, int c, float* psi,
                                            float* dpsi, const float* qm, const float* dqm) {
+    if (UNI) {
+        table_eval4<DERIV>(a.table_uni, C0, row, c, t, psi, dpsi);
+        return;
+    }
     float g[4], dg[4];
     table_eval4<DERIV>(a.table, a.d.CP, row, c, t, g, dg);
     const int R = HASR ? a.d.R : 0;
@@ -226,7 +232,7 @@ template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared 
 //   3. lane = edge again: harmonics and the chi^2 psi_c B_lm products of degree >= 1 for the
 //      lane's own edge, summed over the batch by a shared-memory transpose (32 values at a
 //      time), so that lane v ends up owning sums v, v+32, v+64 of the flattened block.
-template <int C0, int L, bool HASR>
+template <int C0, int L, bool HASR, bool UNI>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_forward(const EdgeArgs a) {
     using W = Widths<C0, L>;
@@ -252,7 +258,6 @@ k_edge_forward(const EdgeArgs a) {
     const int ti = a.type_s[i];
     const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
     const unsigned lt_mask = (1u << lane) - 1u;
-
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
     float accH[W::NCH];
 #pragma unroll
@@ -271,8 +276,8 @@ k_edge_forward(const EdgeArgs a) {
             for (; it + 1 < nb; it += 2) {
                 const int4 ea = qes[it], eb = qes[it + 1];
                 float pa[4], pb[4];
-                amplitude4<C0, HASR, false>(a, ea.x, __int_as_float(ea.z), ea.y, c, pa, nullptr, nullptr, nullptr);
-                amplitude4<C0, HASR, false>(a, eb.x, __int_as_float(eb.z), eb.y, c, pb, nullptr, nullptr, nullptr);
+                amplitude4<C0, HASR, false, UNI>(a, ea.x, __int_as_float(ea.z), ea.y, c, pa, nullptr, nullptr, nullptr);
+                amplitude4<C0, HASR, false, UNI>(a, eb.x, __int_as_float(eb.z), eb.y, c, pb, nullptr, nullptr, nullptr);
                 const float ca = __int_as_float(ea.w), cb = __int_as_float(eb.w);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) acc0[k] += ca * pa[k];
@@ -291,7 +296,7 @@ k_edge_forward(const EdgeArgs a) {
             const int row = es.x, pair = es.y;
             const float t = __int_as_float(es.z), chi = __int_as_float(es.w);
             float psi[4];
-            amplitude4<C0, HASR, false>(a, row, t, pair, c, psi, nullptr, qm + b * kMaxR, nullptr);
+            amplitude4<C0, HASR, false, UNI>(a, row, t, pair, c, psi, nullptr, qm + b * kMaxR, nullptr);
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc0[k] += chi * psi[k];
             if (cl < W::NL1)
@@ -411,7 +416,7 @@ k_edge_forward(const EdgeArgs a) {
 // the edge's lane then does the whole degree >= 1 contraction by itself against the
 // destination's gradient block held in shared memory, and assembles dE/dr_ij.  Edges in the
 // skin shell get a zero gradient as soon as their geometry is known.
-template <int C0, int L, bool HASR>
+template <int C0, int L, bool HASR, bool UNI>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 k_edge_backward(const EdgeArgs a) {
     constexpr int G = BwdGroups<C0>::G;
@@ -469,8 +474,8 @@ k_edge_backward(const EdgeArgs a) {
                     float psi[4 * G], dpsi[4 * G];
 #pragma unroll
                     for (int gq = 0; gq < G; ++gq)
-                        amplitude4<C0, HASR, true>(a, row, t, pair, c + gq * W::GOFF, psi + 4 * gq, dpsi + 4 * gq, qm + b * kMaxR,
-                                                   qm + (32 + b) * kMaxR);
+                        amplitude4<C0, HASR, true, UNI>(a, row, t, pair, c + gq * W::GOFF, psi + 4 * gq, dpsi + 4 * gq,
+                                                        qm + b * kMaxR, qm + (32 + b) * kMaxR);
 #pragma unroll
                     for (int k = 0; k < 4 * G; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
                     if (cl < W::NL1) {       // the leading C1 channels all sit in group 0
@@ -600,17 +605,20 @@ k_edge_backward(const EdgeArgs a) {
 }
 
 
+// one species: the fused table already holds the modes, so the kernels without them are used
 template <int C0, int L>
 cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
-    if (a.d.R > 0) k_edge_forward<C0, L, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
-    else k_edge_forward<C0, L, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    if (a.table_uni) k_edge_forward<C0, L, false, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    else if (a.d.R > 0) k_edge_forward<C0, L, true, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
+    else k_edge_forward<C0, L, false, false><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
     return cudaGetLastError();
 }
 template <int C0, int L>
 cudaError_t launch_bwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
-    const bool hasr = a.d.R > 0;
+    const bool hasr = a.d.R > 0 && !a.table_uni;
     const size_t bytes = hasr ? BwdSmem<C0, L, true>::bytes : BwdSmem<C0, L, false>::bytes;
-    auto kern = hasr ? k_edge_backward<C0, L, true> : k_edge_backward<C0, L, false>;
+    auto kern = a.table_uni ? k_edge_backward<C0, L, false, true>
+                            : (hasr ? k_edge_backward<C0, L, true, false> : k_edge_backward<C0, L, false, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e != cudaSuccess) return e;
     kern<<<blocks, kWarpsPerBlock * 32, bytes, st>>>(a);
@@ -628,7 +636,32 @@ cudaError_t dispatch(const EdgeArgs& a, int blocks, cudaStream_t st) {
     return cudaErrorInvalidValue;
 }
 
+// Table of psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu q_mu(rho) for the ordered pair
+// (s, s), s = the species of atom 0: the cubic coefficients are linear in the tabulated
+// functions, so the same combination of the coefficient rows of [g, q] gives them exactly.
+__global__ void k_fuse_pair_table(Dims d, const float* __restrict__ table, const float* __restrict__ pairmod,
+                                  const int* __restrict__ type, float* __restrict__ out) {
+    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;   // over [row][k][c]
+    if (idx >= (int64_t)d.n_rows * 4 * d.C0) return;
+    const int c = (int)(idx % d.C0);
+    const int64_t rk = idx / d.C0;              // row * 4 + k
+    const int s = type[0];
+    const float* pm = pairmod + (size_t)(s * d.T + s) * (2 + d.R) * d.C0 + c;
+    const float* tr = table + (size_t)rk * d.CP;
+    double v = (double)pm[0] * (double)tr[c];
+    if ((rk & 3) == 0) v += (double)pm[d.C0];
+    for (int q = 0; q < d.R; ++q) v += (double)pm[(size_t)(2 + q) * d.C0] * (double)tr[d.C0 + q];
+    out[idx] = (float)v;
+}
+
 }  // namespace
+
+cudaError_t launch_fuse_pair_table(const Dims& d, const float* table, const float* pairmod, const int* type,
+                                   float* out, cudaStream_t st) {
+    const int64_t n = (int64_t)d.n_rows * 4 * d.C0;
+    k_fuse_pair_table<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d, table, pairmod, type, out);
+    return cudaGetLastError();
+}
 
 int edge_backward_blocks(int n_rows) { return (n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock; }
 

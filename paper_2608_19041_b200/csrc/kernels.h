@@ -36,7 +36,13 @@ struct EdgeArgs {
     float* state;           // [a1-a0][SP]: forward writes sums; backward reads dE/d(sums)
     float* g;               // [E][3] per-edge gradient (backward)
     double* virial_part;    // [blocks][9] partial virial sums (backward)
+    // non-null when every atom has the same species: [n_rows][4][C0] cubic coefficients of the
+    // amplitude psi_c(rho) of that one ordered pair (launch_fuse_pair_table), read instead of
+    // table, pairmod and the radial modes
+    const float* table_uni;
 };
+cudaError_t launch_fuse_pair_table(const Dims& d, const float* table, const float* pairmod, const int* type,
+                                   float* out, cudaStream_t st);
 cudaError_t launch_edge_forward(const EdgeArgs& a, cudaStream_t st);
 cudaError_t launch_edge_backward(const EdgeArgs& a, int* n_blocks, cudaStream_t st);
 int edge_backward_blocks(int n_rows_in_tile);
@@ -82,6 +88,8 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers +
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad
 
 // ---- assemble.cu ---------------------------------------------------------------------
+// *d_flag = 0 when all N species indices are equal (or N == 0), 1 otherwise
+cudaError_t launch_species_differ(int64_t N, const int* type, int* d_flag, cudaStream_t st);
 cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,

@@ -176,6 +176,35 @@ def test_parity_isolated_cluster():
     _compare(blob, s)
 
 
+@pytest.mark.parametrize("name", ["p16_3_2", "p32_2_4", "p8_2_0"])
+def test_parity_one_species_uses_the_fused_pair_table(name):
+    # all atoms of one species (not index 0): the library tabulates that pair's amplitude,
+    # shared radial modes included, and must still agree with the oracle, which knows no such path
+    p = SMALL_PROFILES[name]
+    blob = make_blob(p, seed=44, bias_scale=0.2, e_ref_scale=0.5)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    s["types"] = np.full_like(s["types"], p["T"] - 1)
+    _compare(blob, s)
+
+
+def test_species_mix_may_change_between_builds_on_one_handle():
+    p = SMALL_PROFILES["p32_2_4"]
+    blob = make_blob(p, seed=45, bias_scale=0.2)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    assert len(np.unique(s["types"])) > 1
+    one = dict(s, types=np.full_like(s["types"], 1 % p["T"]))
+    o = orc.Oracle(blob)
+    m, pos = _build(blob, one)
+    for sysd in (one, s, one):
+        m.build_neighbors(pos, _dev(sysd["types"], torch.int32), s["cell"], s["pbc"], 0.0)
+        ref = o.compute(s["pos"], sysd["types"], s["cell"], s["pbc"])
+        out = m.compute(pos)
+        f_scale = np.abs(ref["F"]).max()
+        assert np.abs(out["forces"].cpu().numpy() - ref["F"]).max() <= 2e-5 * f_scale + 2e-7
+        assert abs(out["energy"] - ref["E"]) <= 1e-5 * len(s["pos"]) * np.abs(ref["E_i"]).max()
+    m.close()
+
+
 def test_parity_with_node_tiling():
     # several workspace tiles with a ragged last tile
     p = SMALL_PROFILES["p16_2_0"]
