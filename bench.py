@@ -277,7 +277,8 @@ def run_ours(args):
     blob = workload_blob(args.workload, modes)
     if modes is not None:
         name = f"{name}[R={modes}]"
-    model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile)
+    model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile, pair_table_mb=args.pair_table_mb,
+                          table_dx=args.table_dx)
     pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
     pos = pos0.cuda().contiguous()
     vel = None if static else torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
@@ -391,7 +392,7 @@ def run_ours(args):
                                 profile={k: p[k] for k in ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T")},
                                 dt_ps=dt, rebuild_every=every, skin=skin,
                                 ensemble="nvt (Nose-Hoover chain, period 100 dt)" if (args.nvt and not static) else "nve",
-                                mlp_path=args.mlp_path, parallelism="replicas" if world > 1 else "single",
+                                mlp_path=args.mlp_path, pair_table_mb=args.pair_table_mb, table_dx=args.table_dx, parallelism="replicas" if world > 1 else "single",
                                 **({"published": pub} if pub else {}),
                                 cache="working set per step exceeds L2" if N >= 100000 else "fits in L2 (launch-bound)"),
                     e_pot_per_atom=e_pot / N, e_kin_per_atom=e_kin / N,
@@ -426,6 +427,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(CONFIGS))
     ap.add_argument("--mlp-path", type=int, default=0)
+    ap.add_argument("--table-dx", type=float, default=0.0, help="radial table spacing in Angstrom (0 = the workload's)")
+    ap.add_argument("--pair-table-mb", type=int, default=0,
+                    help="memory for per-pair amplitude tables in MiB (0 = library default, negative = off)")
     ap.add_argument("--node-tile", type=int, default=0)
     ap.add_argument("--atoms", type=int, default=0, help="amorphous and lattice workloads: (about) this many atoms in a smaller box of the same recipe")
     ap.add_argument("--modes", type=int, default=-1, help="override the number R of shared radial modes of the workload's profile")

@@ -54,6 +54,8 @@ typedef struct umlmd_options {
     double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
     int32_t  node_tile;  /* atoms per workspace tile; 0 = 131072                            */
     int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM, persistent, 3 = tcgen05 3xTF32 GEMM, one tile per CTA */
+    int32_t  pair_table_mb;  /* device memory, MiB, that per-pair amplitude tables may take
+                                (see umlmd_build_neighbors); 0 = 192, negative = never build them */
 } umlmd_options;
 
 /* Structural widths of a model, all derived from (C0, L, R) by the paper's formulas
@@ -113,11 +115,13 @@ const char* umlmd_last_error(const umlmd_t* h);
  * dy*dy) + dz*dz, d2 < r_list*r_list, without fused multiply-add, so that the edge set is
  * reproducible bit for bit.  Atoms are renumbered internally in cell order; all outputs
  * of this library are in the caller's numbering.
- * When all N atoms have the same species s, the call also tabulates the edge amplitude of
- * the one ordered pair (s, s), psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu
- * q_mu(rho), as its own cubic table (the same linear combination of the coefficient rows of
- * the radial table), and umlmd_compute reads that table instead of the radial table, the
- * pair cache and the shared modes.  The species are re-examined at every call.
+ * The call also finds which species occur.  When the P species present are few enough that
+ * P^2 tables of table_rows x 4 x C0 floats fit in umlmd_options.pair_table_mb, the edge
+ * amplitude of every ordered pair (s, s') among them, psi_c(rho) = gamma_c g_c(rho) + beta_c +
+ * sum_mu U_c,mu q_mu(rho), is tabulated as a cubic table of its own (the same linear
+ * combination of the coefficient rows of the radial table), and umlmd_compute reads one row of
+ * that table per edge instead of the radial table, the pair cache and the shared modes.  The
+ * species are re-examined at every call; the tables are kept while the set does not change.
  */
 int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type,
                           const double cell[9], const int pbc[3], double skin);

@@ -37,7 +37,7 @@ class UmlmdError(RuntimeError):
 
 class Options(ctypes.Structure):
     _fields_ = [("struct_bytes", ctypes.c_uint32), ("table_dx", ctypes.c_double),
-                ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32)]
+                ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32), ("pair_table_mb", ctypes.c_int32)]
 
 
 class Info(ctypes.Structure):
@@ -116,10 +116,10 @@ def _check_dev(t, dtype, name):
 class Model:
     """A DPA4C model on the current CUDA device, created from a weight blob."""
 
-    def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, stream=None):
+    def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, pair_table_mb=0, stream=None):
         self._lib = lib()
         self._h = ctypes.c_void_p()
-        opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path))
+        opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path), int(pair_table_mb))
         # creation is host-only; a stream is only meaningful when a device is present
         self._stream = stream if stream is not None else (
             torch.cuda.current_stream() if torch.cuda.is_available() else None)

@@ -31,8 +31,13 @@ struct umlmd {
     double* virial_part = nullptr; int64_t vpart_cap = 0;
     double* scratch = nullptr; double* d_out = nullptr; int* d_err = nullptr;
     double* h_out = nullptr; int* h_err = nullptr;      // pinned
-    bool one_species = false;                           // set by umlmd_build_neighbors
-    float* table_uni = nullptr;                         // amplitude table of the one pair, when one_species
+    // per-pair amplitude tables of the species present (set up by umlmd_build_neighbors)
+    int64_t pair_table_budget = 192ll << 20;            // bytes; negative = never build them
+    bool pair_tables = false;                           // in use for the current system
+    std::vector<int> present;                           // species the tables were built for, ascending
+    float* table_uni = nullptr; size_t table_uni_cap = 0;   // [present^2][n_rows][4][C0], capacity in floats
+    int* d_species = nullptr;                           // [3T]: occurrence flags, species -> slot, present list
+    int* h_species = nullptr;                           // pinned [T]
     // MD
     double* md_pos = nullptr; double* md_vel = nullptr; double* md_force = nullptr; int64_t md_cap = 0;
     double* d_mass = nullptr; double* d_inv_mass = nullptr;
@@ -156,7 +161,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         const int n = N - a0 < B ? N - a0 : B;
         EdgeArgs ea;
         ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.type_s = nb.type_s;
-        ea.table_uni = h->one_species ? h->table_uni : nullptr;
+        ea.table_uni = h->pair_tables ? h->table_uni : nullptr;
+        ea.species_slot = h->d_species + d.T; ea.n_present = (int)h->present.size();
         ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
@@ -252,6 +258,33 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
     return ensure_workspace(h);
 }
 
+// With few species present, psi_c(rho) of every ordered pair among them is tabulated by itself,
+// so that the edge kernels read one table row per edge and neither pair rows nor shared modes.
+// The tables depend on the model and the set of species only, so they are kept across builds.
+int setup_pair_tables(umlmd_t* h) {
+    const Dims& d = h->d;
+    std::vector<int> present;
+    for (int t = 0; t < d.T; ++t) if (h->h_species[t]) present.push_back(t);
+    const size_t np = present.size();
+    const size_t floats = np * np * (size_t)d.n_rows * 4 * d.C0;
+    h->pair_tables = np > 0 && h->pair_table_budget >= 0 && floats * sizeof(float) <= (size_t)h->pair_table_budget;
+    if (!h->pair_tables || present == h->present) return UMLMD_OK;
+    if (floats > h->table_uni_cap) {
+        dev_free(h->table_uni); h->table_uni = nullptr; h->table_uni_cap = 0;
+        void* p = nullptr;
+        API_CUDA(h, dev_malloc(&p, sizeof(float) * floats));
+        h->table_uni = (float*)p; h->table_uni_cap = floats;
+    }
+    std::vector<int> up(2 * (size_t)d.T, 0);          // species -> slot, then the present list
+    for (size_t k = 0; k < np; ++k) { up[present[k]] = (int)k; up[d.T + k] = present[k]; }
+    API_CUDA(h, cudaMemcpyAsync(h->d_species + d.T, up.data(), sizeof(int) * up.size(), cudaMemcpyHostToDevice, h->st));
+    API_CUDA(h, launch_fuse_pair_tables(d, h->md.table, h->md.pairmod, h->d_species + 2 * d.T, (int)np, h->table_uni, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));       // `up` is pageable host memory
+    h->launches_total += 1;
+    h->present = present;
+    return UMLMD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -278,6 +311,7 @@ int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, 
         dx_override = opt->table_dx;
         if (opt->node_tile > 0) h->node_tile = opt->node_tile;
         if (opt->mlp_path > 0) h->mlp_path = opt->mlp_path;
+        if (opt->pair_table_mb != 0) h->pair_table_budget = opt->pair_table_mb < 0 ? -1 : (int64_t)opt->pair_table_mb << 20;
     }
     int rc = build_host_model(blob, blob_bytes, dx_override, &h->hm, &h->err);
     if (rc != UMLMD_OK) { delete h; return rc; }
@@ -292,12 +326,13 @@ int umlmd_destroy(umlmd_t* h) {
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
     void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
-                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni};
+                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni, h->d_species};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
     if (h->h_out) cudaFreeHost(h->h_out);
     if (h->h_err) cudaFreeHost(h->h_err);
+    if (h->h_species) cudaFreeHost(h->h_species);
     delete h;
     return UMLMD_OK;
 }
@@ -333,26 +368,24 @@ int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int3
     int rc = build_list(h, N, d_pos, d_type, L, pbc, skin);
     if (rc != UMLMD_OK) return rc;
     if (N > 0) API_CUDA(h, cudaMemcpyAsync(h->type_o, d_type, sizeof(int) * N, cudaMemcpyDeviceToDevice, h->st));
-    // one species throughout: the edge kernels then keep the pair rows in registers
-    API_CUDA(h, launch_species_differ(N, d_type, h->d_err + 1, h->st));
+    // which species occur: few enough of them get per-pair amplitude tables (see below)
+    const int T = h->d.T;
+    if (!h->d_species) {
+        void* p = nullptr;
+        API_CUDA(h, dev_malloc(&p, sizeof(int) * 3 * (size_t)T));
+        h->d_species = (int*)p;
+        API_CUDA(h, cudaMallocHost((void**)&h->h_species, sizeof(int) * (size_t)T));
+    }
+    API_CUDA(h, launch_species_present(N, d_type, T, h->d_species, h->st));
     h->launches_total += N > 0;
+    API_CUDA(h, cudaMemcpyAsync(h->h_species, h->d_species, sizeof(int) * (size_t)T, cudaMemcpyDeviceToHost, h->st));
     // surface device-side findings of the build (non-finite positions, image range)
-    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, 2 * sizeof(int), cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
     API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
     API_CUDA(h, cudaStreamSynchronize(h->st));
-    h->one_species = N > 0 && h->h_err[1] == 0;
     rc = decode_device_errors(h, *h->h_err);
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
-    if (h->one_species) {
-        if (!h->table_uni) {
-            void* p = nullptr;
-            API_CUDA(h, dev_malloc(&p, sizeof(float) * (size_t)h->d.n_rows * 4 * h->d.C0));
-            h->table_uni = (float*)p;
-        }
-        API_CUDA(h, launch_fuse_pair_table(h->d, h->md.table, h->md.pairmod, h->type_o, h->table_uni, h->st));
-        h->launches_total += 1;
-    }
-    return rc;
+    return setup_pair_tables(h);
 }
 
 int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift, int64_t cap,

@@ -75,11 +75,12 @@ __global__ void k_unsort_rows(int N, const int* __restrict__ perm, const float* 
     for (int k = lane; k < width; k += 32) w[k] = r[k];
 }
 
-// *flag = 1 when some atom's species differs from the first atom's (flag cleared by the caller)
-__global__ void k_species_differ(int64_t N, const int* __restrict__ type, int* __restrict__ flag) {
+// flags[t] = 1 for every species that occurs (flags cleared by the caller)
+__global__ void k_species_present(int64_t N, const int* __restrict__ type, int T, int* __restrict__ flags) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    const bool differs = i < N && type[i] != type[0];
-    if (__any_sync(0xffffffffu, differs) && (threadIdx.x & 31) == 0) *flag = 1;
+    if (i >= N) return;
+    const int t = type[i];
+    if (t >= 0 && t < T && flags[t] == 0) flags[t] = 1;
 }
 
 __device__ __forceinline__ double block_sum(double v, double* sh) {
@@ -261,10 +262,10 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
     return cudaGetLastError();
 }
 
-cudaError_t launch_species_differ(int64_t N, const int* type, int* d_flag, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(d_flag, 0, sizeof(int), st);
+cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(d_flags, 0, sizeof(int) * T, st);
     if (e != cudaSuccess || N == 0) return e;
-    k_species_differ<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, type, d_flag);
+    k_species_present<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, type, T, d_flags);
     return cudaGetLastError();
 }
 

@@ -65,7 +65,14 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, int e, bool in_
     row = row < a.d.n_rows - 1 ? row : a.d.n_rows - 1;
     g.row = row;
     g.t = g.rho - (float)row * a.d.dx;
-    g.pair = ti * a.d.T + a.type_s[j];
+    if (a.table_uni) {
+        // per-pair amplitude tables, one after another: the pair selects the table (ti is
+        // already the compact index of the centre's species)
+        g.pair = ti * a.n_present + a.species_slot[a.type_s[j]];
+        g.row += g.pair * a.d.n_rows;
+    } else {
+        g.pair = ti * a.d.T + a.type_s[j];
+    }
     return g;
 }
 
@@ -149,9 +156,9 @@ __device__ __forceinline__ void eval_modes(const EdgeArgs& a, const int4* qes, i
 }
 
 // amplitude psi (and d psi / d rho) of this lane's four channels for one edge; qm / dqm: the
-// edge's parked radial modes (only read when HASR).  UNI: the system has one species, so psi is
-// a function of rho alone and comes from the table of that pair (a.table_uni, row pitch C0),
-// without pair rows or modes
+// edge's parked radial modes (only read when HASR).  UNI: psi_c(rho) of every ordered pair of
+// species present is tabulated by itself (a.table_uni, row pitch C0; `row` already points into
+// the edge's pair), so neither pair rows nor modes are read
 template <int C0, bool HASR, bool DERIV, bool UNI>
 __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, int pair, int c, float* psi,
                                            float* dpsi, const float* qm, const float* dqm) {
@@ -255,7 +262,7 @@ k_edge_forward(const EdgeArgs a) {
     float* const qd = q_d[wid];
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
     const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
-    const int ti = a.type_s[i];
+    const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
     const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
     const unsigned lt_mask = (1u << lane) - 1u;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
@@ -442,7 +449,7 @@ k_edge_backward(const EdgeArgs a) {
 
     if (active) {
         const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
-        const int ti = a.type_s[i];
+        const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
         const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
         float h0[4 * G];
@@ -605,7 +612,7 @@ k_edge_backward(const EdgeArgs a) {
 }
 
 
-// one species: the fused table already holds the modes, so the kernels without them are used
+// per-pair amplitude tables already hold the modes, so the kernels without them are used
 template <int C0, int L>
 cudaError_t launch_fwd_r(const EdgeArgs& a, int blocks, cudaStream_t st) {
     if (a.table_uni) k_edge_forward<C0, L, false, true><<<blocks, kWarpsPerBlock * 32, 0, st>>>(a);
@@ -636,17 +643,21 @@ cudaError_t dispatch(const EdgeArgs& a, int blocks, cudaStream_t st) {
     return cudaErrorInvalidValue;
 }
 
-// Table of psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu q_mu(rho) for the ordered pair
-// (s, s), s = the species of atom 0: the cubic coefficients are linear in the tabulated
-// functions, so the same combination of the coefficient rows of [g, q] gives them exactly.
-__global__ void k_fuse_pair_table(Dims d, const float* __restrict__ table, const float* __restrict__ pairmod,
-                                  const int* __restrict__ type, float* __restrict__ out) {
-    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;   // over [row][k][c]
-    if (idx >= (int64_t)d.n_rows * 4 * d.C0) return;
-    const int c = (int)(idx % d.C0);
-    const int64_t rk = idx / d.C0;              // row * 4 + k
-    const int s = type[0];
-    const float* pm = pairmod + (size_t)(s * d.T + s) * (2 + d.R) * d.C0 + c;
+// Tables of psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu q_mu(rho) for the ordered
+// pairs (present[a], present[b]), stored as [a * n_present + b][row][k][c]: the cubic
+// coefficients are linear in the tabulated functions, so the same combination of the
+// coefficient rows of [g, q] gives them exactly.
+__global__ void k_fuse_pair_tables(Dims d, const float* __restrict__ table, const float* __restrict__ pairmod,
+                                   const int* __restrict__ present, int n_present, float* __restrict__ out) {
+    const int64_t per_pair = (int64_t)d.n_rows * 4 * d.C0;
+    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;   // over [pair][row][k][c]
+    if (idx >= per_pair * n_present * n_present) return;
+    const int pr = (int)(idx / per_pair);
+    const int64_t in_pair = idx - pr * per_pair;
+    const int c = (int)(in_pair % d.C0);
+    const int64_t rk = in_pair / d.C0;          // row * 4 + k
+    const int si = present[pr / n_present], sj = present[pr % n_present];
+    const float* pm = pairmod + (size_t)(si * d.T + sj) * (2 + d.R) * d.C0 + c;
     const float* tr = table + (size_t)rk * d.CP;
     double v = (double)pm[0] * (double)tr[c];
     if ((rk & 3) == 0) v += (double)pm[d.C0];
@@ -656,10 +667,11 @@ __global__ void k_fuse_pair_table(Dims d, const float* __restrict__ table, const
 
 }  // namespace
 
-cudaError_t launch_fuse_pair_table(const Dims& d, const float* table, const float* pairmod, const int* type,
-                                   float* out, cudaStream_t st) {
-    const int64_t n = (int64_t)d.n_rows * 4 * d.C0;
-    k_fuse_pair_table<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d, table, pairmod, type, out);
+cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
+                                    int n_present, float* out, cudaStream_t st) {
+    const int64_t n = (int64_t)d.n_rows * 4 * d.C0 * n_present * n_present;
+    if (n == 0) return cudaSuccess;
+    k_fuse_pair_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d, table, pairmod, present, n_present, out);
     return cudaGetLastError();
 }
 

@@ -36,13 +36,16 @@ struct EdgeArgs {
     float* state;           // [a1-a0][SP]: forward writes sums; backward reads dE/d(sums)
     float* g;               // [E][3] per-edge gradient (backward)
     double* virial_part;    // [blocks][9] partial virial sums (backward)
-    // non-null when every atom has the same species: [n_rows][4][C0] cubic coefficients of the
-    // amplitude psi_c(rho) of that one ordered pair (launch_fuse_pair_table), read instead of
-    // table, pairmod and the radial modes
+    // non-null when the species present are few enough for per-pair amplitude tables:
+    // [n_present^2][n_rows][4][C0] cubic coefficients of psi_c(rho) of each ordered pair
+    // (launch_fuse_pair_tables), read instead of table, pairmod and the radial modes
     const float* table_uni;
+    const int* species_slot;    // [T] species -> index among the species present
+    int n_present;
 };
-cudaError_t launch_fuse_pair_table(const Dims& d, const float* table, const float* pairmod, const int* type,
-                                   float* out, cudaStream_t st);
+// present: device array of the n_present species indices, ascending
+cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
+                                    int n_present, float* out, cudaStream_t st);
 cudaError_t launch_edge_forward(const EdgeArgs& a, cudaStream_t st);
 cudaError_t launch_edge_backward(const EdgeArgs& a, int* n_blocks, cudaStream_t st);
 int edge_backward_blocks(int n_rows_in_tile);
@@ -88,8 +91,8 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers +
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad
 
 // ---- assemble.cu ---------------------------------------------------------------------
-// *d_flag = 0 when all N species indices are equal (or N == 0), 1 otherwise
-cudaError_t launch_species_differ(int64_t N, const int* type, int* d_flag, cudaStream_t st);
+// d_flags[t] = 1 for every species t in [0, T) that occurs among the N atoms, 0 otherwise
+cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, cudaStream_t st);
 cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,

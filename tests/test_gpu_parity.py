@@ -152,12 +152,15 @@ def _compare(blob, s, tol_scale=1.0, skin=0.0, check_intermediates=True, **kw):
 SYS_SMALL = dict(kind="random_box", atoms=60, edges=(9.5, 10.5, 12.0), min_dist=1.7, seed=31, masses=[1.0] * 3)
 
 
+@pytest.mark.parametrize("pair_table_mb", [-1, 0], ids=["pair_cache", "pair_tables"])
 @pytest.mark.parametrize("name", sorted(SMALL_PROFILES))
-def test_energy_force_virial_parity_small_profiles(name):
+def test_energy_force_virial_parity_small_profiles(name, pair_table_mb):
+    # with and without the per-pair amplitude tables that the library builds when few species
+    # are present (the oracle knows no such path)
     p = SMALL_PROFILES[name]
     blob = make_blob(p, seed=40, bias_scale=0.2, e_ref_scale=0.5)
     s = make_system(dict(SYS_SMALL, n_types=p["T"]))
-    _compare(blob, s)
+    _compare(blob, s, pair_table_mb=pair_table_mb)
 
 
 def test_parity_with_skin_and_multi_image_box():
@@ -177,9 +180,8 @@ def test_parity_isolated_cluster():
 
 
 @pytest.mark.parametrize("name", ["p16_3_2", "p32_2_4", "p8_2_0"])
-def test_parity_one_species_uses_the_fused_pair_table(name):
-    # all atoms of one species (not index 0): the library tabulates that pair's amplitude,
-    # shared radial modes included, and must still agree with the oracle, which knows no such path
+def test_parity_one_species_present_out_of_several(name):
+    # all atoms of one species (not index 0): a single pair table, shared radial modes included
     p = SMALL_PROFILES[name]
     blob = make_blob(p, seed=44, bias_scale=0.2, e_ref_scale=0.5)
     s = make_system(dict(SYS_SMALL, n_types=p["T"]))
@@ -188,14 +190,15 @@ def test_parity_one_species_uses_the_fused_pair_table(name):
 
 
 def test_species_mix_may_change_between_builds_on_one_handle():
-    p = SMALL_PROFILES["p32_2_4"]
+    p = SMALL_PROFILES["p32_3_2"]
     blob = make_blob(p, seed=45, bias_scale=0.2)
     s = make_system(dict(SYS_SMALL, n_types=p["T"]))
     assert len(np.unique(s["types"])) > 1
     one = dict(s, types=np.full_like(s["types"], 1 % p["T"]))
     o = orc.Oracle(blob)
     m, pos = _build(blob, one)
-    for sysd in (one, s, one):
+    two = dict(s, types=np.where(s["types"] == s["types"][0], 0, p["T"] - 1).astype(s["types"].dtype))
+    for sysd in (one, s, two, one):
         m.build_neighbors(pos, _dev(sysd["types"], torch.int32), s["cell"], s["pbc"], 0.0)
         ref = o.compute(s["pos"], sysd["types"], s["cell"], s["pbc"])
         out = m.compute(pos)
