@@ -68,8 +68,10 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, int e, bool in_
     if (a.table_uni) {
         // per-pair amplitude tables, one after another: the pair selects the table (ti is
         // already the compact index of the centre's species)
-        g.pair = ti * a.n_present + a.species_slot[a.type_s[j]];
-        g.row += g.pair * a.d.n_rows;
+        if (a.n_present > 1) {           // with one species there is one table and no lookup
+            g.pair = ti * a.n_present + a.species_slot[a.type_s[j]];
+            g.row += g.pair * a.d.n_rows;
+        }
     } else {
         g.pair = ti * a.d.T + a.type_s[j];
     }
