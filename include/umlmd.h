@@ -107,7 +107,7 @@ const char* umlmd_last_error(const umlmd_t* h);
  * distinct neighbor instances, both orientations stored, no capacity limit.
  *   d_pos   [N,3] double, any image of each atom; folded into the cell internally with
  *           frac - floor(frac) along periodic directions (n refers to folded positions)
- *   d_type  [N] int32 species
+ *   d_type  [N] int32 species, each in [0, T) (checked: UMLMD_E_INVALID_ARG otherwise)
  *   cell    9 doubles, rows are cell vectors; must be orthorhombic (diagonal)
  *   pbc     3 ints, non-zero = periodic along that cell vector
  *   skin    extra list radius in Angstrom (>= 0); edges beyond rc carry zero weight

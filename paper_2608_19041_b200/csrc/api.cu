@@ -141,6 +141,7 @@ int ensure_workspace(umlmd_t* h) {
 }
 
 int decode_device_errors(umlmd_t* h, int word) {
+    if (word & kErrSpecies) return fail(h, UMLMD_E_INVALID_ARG, "species index outside [0, T)");
     if (word & kErrNonFinite) return fail(h, UMLMD_E_NONFINITE, "non-finite value in positions, energy or forces");
     if (word & kErrPipelineTimeout) return fail(h, UMLMD_E_CUDA, "tensor-core GEMM pipeline wait expired");
     if (word & kErrShiftRange) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "periodic image index outside [-127, 127]");
@@ -376,7 +377,7 @@ int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int3
         h->d_species = (int*)p;
         API_CUDA(h, cudaMallocHost((void**)&h->h_species, sizeof(int) * (size_t)T));
     }
-    API_CUDA(h, launch_species_present(N, d_type, T, h->d_species, h->st));
+    API_CUDA(h, launch_species_present(N, d_type, T, h->d_species, h->d_err, h->st));
     h->launches_total += N > 0;
     API_CUDA(h, cudaMemcpyAsync(h->h_species, h->d_species, sizeof(int) * (size_t)T, cudaMemcpyDeviceToHost, h->st));
     // surface device-side findings of the build (non-finite positions, image range)

@@ -75,12 +75,15 @@ __global__ void k_unsort_rows(int N, const int* __restrict__ perm, const float* 
     for (int k = lane; k < width; k += 32) w[k] = r[k];
 }
 
-// flags[t] = 1 for every species that occurs (flags cleared by the caller)
-__global__ void k_species_present(int64_t N, const int* __restrict__ type, int T, int* __restrict__ flags) {
+// flags[t] = 1 for every species that occurs (flags cleared by the caller); an index outside
+// [0, T) is reported in the error word
+__global__ void k_species_present(int64_t N, const int* __restrict__ type, int T, int* __restrict__ flags,
+                                  int* __restrict__ err) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (i >= N) return;
     const int t = type[i];
-    if (t >= 0 && t < T && flags[t] == 0) flags[t] = 1;
+    if (t < 0 || t >= T) atomicOr(err, kErrSpecies);
+    else if (flags[t] == 0) flags[t] = 1;
 }
 
 __device__ __forceinline__ double block_sum(double v, double* sh) {
@@ -262,10 +265,10 @@ cudaError_t launch_unsort_state(const NeighborDev& nb, const float* in, int stri
     return cudaGetLastError();
 }
 
-cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, cudaStream_t st) {
+cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, int* d_err, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(d_flags, 0, sizeof(int) * T, st);
     if (e != cudaSuccess || N == 0) return e;
-    k_species_present<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, type, T, d_flags);
+    k_species_present<<<(unsigned)((N + 255) / 256), 256, 0, st>>>(N, type, T, d_flags, d_err);
     return cudaGetLastError();
 }
 

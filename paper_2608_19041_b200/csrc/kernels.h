@@ -91,8 +91,9 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers +
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad
 
 // ---- assemble.cu ---------------------------------------------------------------------
-// d_flags[t] = 1 for every species t in [0, T) that occurs among the N atoms, 0 otherwise
-cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, cudaStream_t st);
+// d_flags[t] = 1 for every species t in [0, T) that occurs among the N atoms, 0 otherwise;
+// kErrSpecies is or-ed into *d_err when an index lies outside [0, T)
+cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, int* d_err, cudaStream_t st);
 cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,

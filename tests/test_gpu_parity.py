@@ -250,6 +250,27 @@ def test_stale_list_is_reported():
     m.compute(pos)                         # the handle stays usable
 
 
+@pytest.mark.parametrize("bad", [-1, 2])
+def test_species_index_out_of_range_is_refused(bad):
+    # the index would address the pair cache out of bounds: the build reports it, nothing reads it
+    p = SMALL_PROFILES["p8_2_0"]
+    assert p["T"] == 2
+    blob = make_blob(p, seed=44)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    m, pos = _build(blob, s)
+    types = s["types"].copy()
+    types[7] = bad
+    with pytest.raises(_binding().UmlmdError) as e:
+        m.build_neighbors(pos, _dev(types, torch.int32), s["cell"], s["pbc"], 0.0)
+    assert e.value.code == -1
+    with pytest.raises(_binding().UmlmdError) as e:
+        m.compute(pos)                     # no list: the failed build left none
+    assert e.value.code == -5
+    m.build_neighbors(pos, _dev(s["types"], torch.int32), s["cell"], s["pbc"], 0.0)
+    m.compute(pos)                         # the handle stays usable
+    m.close()
+
+
 @pytest.mark.parametrize("path", [2, 3])
 @pytest.mark.parametrize("name", ["p16_3_2", "p32_2_4", "p32_2_0_res"])
 def test_tensor_core_mlp_path_small_profiles(name, path):
