@@ -43,7 +43,8 @@ enum {
     UMLMD_E_STALE_NEIGHBORS = -6,     /* an atom moved more than skin/2 since the build     */
     UMLMD_E_NONFINITE = -7,           /* NaN or Inf in positions, energy or forces          */
     UMLMD_E_CUDA = -8,                /* a CUDA runtime call failed (message has details)   */
-    UMLMD_E_CAPACITY = -9,            /* caller buffer too small (see umlmd_get_neighbors)  */
+    UMLMD_E_CAPACITY = -9,            /* caller buffer too small (see umlmd_get_neighbors);
+                                         neighbor list beyond 2^31 - 1 edges                */
     UMLMD_E_NO_MD_STATE = -10         /* step called before set_md_state                    */
 };
 

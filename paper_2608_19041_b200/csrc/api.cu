@@ -252,7 +252,7 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
                const int pbc[3], double skin) {
     int rc = ensure_device_model(h);
     if (rc != UMLMD_OK) return rc;
-    { Scope sc(h, kNeighbor, 6); rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
+    { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
     h->have_list = true;
     h->steps_since_build = 0;

@@ -90,7 +90,7 @@ __global__ void k_cell_start(int ncell, int N, const int* __restrict__ skey, int
     if (c > ncell) return;
     int lo = 0, hi = N;
     while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
+        const int mid = lo + ((hi - lo) >> 1);     // lo + hi would pass 2^31 in a long list
         if (skey[mid] < c) lo = mid + 1; else hi = mid;
     }
     cell_start[c] = lo;
@@ -184,6 +184,16 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     if (!FILL && lane == 0) deg[i] = count;
 }
 
+// 64-bit sum of the row lengths: the 32-bit prefix sum wraps silently once a list passes 2^31
+// edges, and what wrapped must not size the edge arrays
+__global__ void k_sum_deg64(int N, const int* __restrict__ deg, unsigned long long* __restrict__ out) {
+    unsigned long long v = 0;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) v += (unsigned)deg[i];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    if ((threadIdx.x & 31) == 0 && v) atomicAdd(out, v);
+}
+
 // rev[e] = slot of (j <- i, -n) for e = (i <- j, n); -1 when absent (can only happen for
 // pairs whose two orientations round to opposite sides of the list radius).
 __global__ void k_reverse_map(int N, int sorted, const int* __restrict__ row_ptr, const int* __restrict__ src,
@@ -204,7 +214,7 @@ __global__ void k_reverse_map(int N, int sorted, const int* __restrict__ row_ptr
         if (sorted) {          // rows ascend in the neighbour index, each neighbour at most once
             int lo = f0, hi = f1;
             while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
+                const int mid = lo + ((hi - lo) >> 1);     // lo + hi would pass 2^31 in a long list
                 if (src[mid] < i) lo = mid + 1; else hi = mid;
             }
             if (lo < f1 && src[lo] == i && shift[lo] == want) found = lo;
@@ -388,10 +398,18 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     NB_CHECK(cudaMemsetAsync(nb->deg + N, 0, sizeof(int), st));
     tmp_bytes = nb->cub_bytes;
     NB_CHECK(cub::DeviceScan::ExclusiveSum(nb->cub_tmp, tmp_bytes, nb->deg, nb->row_ptr, N + 1, st));
-    int total = 0;
-    NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(int), cudaMemcpyDeviceToHost, st));
+    // the unsorted keys are no longer needed: their buffer holds the 64-bit total
+    unsigned long long* d_total = reinterpret_cast<unsigned long long*>(nb->key);
+    NB_CHECK(cudaMemsetAsync(d_total, 0, sizeof(unsigned long long), st));
+    k_sum_deg64<<<(N + 4 * TB - 1) / (4 * TB) < 1024 ? (N + 4 * TB - 1) / (4 * TB) : 1024, TB, 0, st>>>(N, nb->deg, d_total);
+    unsigned long long total64 = 0;
+    NB_CHECK(cudaMemcpyAsync(&total64, d_total, sizeof(total64), cudaMemcpyDeviceToHost, st));
     NB_CHECK(cudaStreamSynchronize(st));
-    if (total < 0) { *err = "edge count overflows 32-bit indices"; return UMLMD_E_INVALID_ARG; }
+    if (total64 > 0x7fffffffull - 64) {      // the margin keeps "edge index + lane" inside int as well
+        *err = "neighbor list has " + std::to_string(total64) + " edges; edge indices are 32-bit (at most 2147483583)";
+        return UMLMD_E_CAPACITY;
+    }
+    const int total = (int)total64;
     nb->E = total;
     if (total > nb->E_cap) {
         int64_t c;
