@@ -43,8 +43,8 @@ enum {
     UMLMD_E_STALE_NEIGHBORS = -6,     /* an atom moved more than skin/2 since the build     */
     UMLMD_E_NONFINITE = -7,           /* NaN or Inf in positions, energy or forces          */
     UMLMD_E_CUDA = -8,                /* a CUDA runtime call failed (message has details)   */
-    UMLMD_E_CAPACITY = -9,            /* caller buffer too small (see umlmd_get_neighbors);
-                                         neighbor list beyond 2^31 - 1 edges                */
+    UMLMD_E_CAPACITY = -9,            /* caller buffer too small, or a list too long for the
+                                         32-bit export (see umlmd_get_neighbors)             */
     UMLMD_E_NO_MD_STATE = -10         /* step called before set_md_state                    */
 };
 
@@ -131,6 +131,8 @@ int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int3
  * Copy the current neighbor list out in the caller's atom numbering (for verification).
  *   d_row_ptr [N+1] int32, d_src [cap] int32, d_shift [cap,3] int8; row i holds the
  *   neighbor instances (j, n) of centre i in no particular order.
+ * Internally edge offsets are 64-bit and a list may hold more than 2^31 - 1 edges; this export
+ * then fails with UMLMD_E_CAPACITY, *n_edges still being set.
  * Pass cap = 0 (pointers may be NULL) to only query *n_edges.  UMLMD_E_CAPACITY if the
  * list has more than cap edges.
  */

@@ -396,6 +396,7 @@ int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* 
     *n_edges = h->nb.E;
     if (cap == 0) return UMLMD_OK;
     if (cap < h->nb.E) return fail(h, UMLMD_E_CAPACITY, "edge buffers smaller than the list");
+    if (h->nb.E > 0x7fffffffll) return fail(h, UMLMD_E_CAPACITY, "the export has 32-bit row pointers; this list has more than 2^31 - 1 edges");
     if (!d_row_ptr || (h->nb.E > 0 && (!d_src || !d_shift))) return fail(h, UMLMD_E_INVALID_ARG, "null output buffer");
     int rc = neighbor_export(&h->nb, d_row_ptr, d_src, d_shift, h->st, &h->err);
     if (rc != UMLMD_OK) return rc;

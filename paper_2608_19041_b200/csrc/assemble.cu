@@ -14,17 +14,19 @@ constexpr int kRedBlock = 256;
 constexpr int kRedMaxBlocks = 1024;
 
 // out (caller numbering, through perm) and / or f (sorted numbering) may be null
-__global__ void k_force_rows(int N, const int* __restrict__ row_ptr, const int* __restrict__ rev,
+__global__ void k_force_rows(int N, const eidx_t* __restrict__ row_ptr, const eidx_t* __restrict__ rev,
                              const float* __restrict__ g, double* __restrict__ f, const int* __restrict__ perm,
                              double* __restrict__ out, int* __restrict__ err) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= N) return;
-    const int e0 = row_ptr[warp], e1 = row_ptr[warp + 1];
+    const eidx_t e0 = row_ptr[warp];
+    const int len = (int)(row_ptr[warp + 1] - e0);
     double fx = 0, fy = 0, fz = 0;
-    for (int e = e0 + lane; e < e1; e += 32) {
+    for (int k = lane; k < len; k += 32) {
+        const eidx_t e = e0 + k;
         const float* a = g + 3 * (size_t)e;
         float bx = 0.f, by = 0.f, bz = 0.f;
-        const int r = rev[e];
+        const eidx_t r = rev[e];
         if (r >= 0) { const float* b = g + 3 * (size_t)r; bx = b[0]; by = b[1]; bz = b[2]; }
         fx += (double)a[0] - (double)bx;
         fy += (double)a[1] - (double)by;

@@ -75,6 +75,8 @@ struct Handle;  // defined in api.cu
 
 // ---- launchers (each enqueues on `st`; none synchronises) ---------------------------
 
+typedef long long eidx_t;      // edge offsets are 64-bit: a list may hold more than 2^31 edges
+
 struct NeighborDev {
     int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;
     double L[3] = {0, 0, 0};
@@ -86,10 +88,10 @@ struct NeighborDev {
     int* type_s = nullptr;       // [N] species, sorted order
     double* xs0 = nullptr;       // [N][3] folded positions at build time, sorted order
     double* xs = nullptr;        // [N][3] current positions minus img*L, sorted order
-    int* row_ptr = nullptr;      // [N+1]
+    eidx_t* row_ptr = nullptr;   // [N+1]
     int* src = nullptr;          // [E] sorted index of the neighbour
     int* shift = nullptr;        // [E] packed int8 x3 image n
-    int* rev = nullptr;          // [E] index of the reverse edge, -1 if absent
+    eidx_t* rev = nullptr;       // [E] index of the reverse edge, -1 if absent
     // scratch
     int* key = nullptr; int* key2 = nullptr; int* idx = nullptr; int* idx2 = nullptr;
     int* cell_start = nullptr; int64_t ncell_cap = 0;

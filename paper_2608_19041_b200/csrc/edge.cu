@@ -34,7 +34,7 @@ struct Geom {
 };
 
 // phase 1: one lane, one edge
-__device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, int e, bool in_range, double xi, double yi,
+__device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool in_range, double xi, double yi,
                                               double zi, int ti) {
     Geom g;
     g.valid = false;
@@ -265,7 +265,8 @@ k_edge_forward(const EdgeArgs a) {
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
     const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
     const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
-    const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
+    const eidx_t e0 = a.row_ptr[i];
+    const int len = (int)(a.row_ptr[i + 1] - e0);      // edge offsets are 64-bit, offsets inside a row are not
     const unsigned lt_mask = (1u << lane) - 1u;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
     float accH[W::NCH];
@@ -370,8 +371,8 @@ k_edge_forward(const EdgeArgs a) {
     };
 
     int qn = 0;
-    for (int base = e0; base < e1; base += 32) {
-        const Geom g = edge_geometry(a, base + lane, base + lane < e1, xi, yi, zi, ti);
+    for (int base = 0; base < len; base += 32) {
+        const Geom g = edge_geometry(a, e0 + base + lane, base + lane < len, xi, yi, zi, ti);
         const unsigned vmask = __ballot_sync(kFull, g.valid);
         const int p = qn + __popc(vmask & lt_mask);       // queue slot of this lane's edge, if it has one
         if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
@@ -452,7 +453,8 @@ k_edge_backward(const EdgeArgs a) {
     if (active) {
         const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
         const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
-        const int e0 = a.row_ptr[i], e1 = a.row_ptr[i + 1];
+        const eidx_t e0 = a.row_ptr[i];
+        const int len = (int)(a.row_ptr[i + 1] - e0);
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
         float h0[4 * G];
 #pragma unroll
@@ -504,7 +506,7 @@ k_edge_backward(const EdgeArgs a) {
             __syncwarp();
             if (lane < nb) {
                 const float gdx = qd[lane], gdy = qd[32 + lane], gdz = qd[64 + lane], dchi = qd[96 + lane];
-                const int e = __float_as_int(qd[128 + lane]);
+                const int e = __float_as_int(qd[128 + lane]);       // offset inside the row
                 const float chi = __int_as_float(qes[lane].w);
                 const float inv_rho = 1.0f / sqrtf(gdx * gdx + gdy * gdy + gdz * gdz + kEpsReg * kEpsReg);
                 const float gux = gdx * inv_rho, guy = gdy * inv_rho, guz = gdz * inv_rho;
@@ -561,24 +563,24 @@ k_edge_backward(const EdgeArgs a) {
                 vir[0] += gx * gdx; vir[1] += gx * gdy; vir[2] += gx * gdz;
                 vir[3] += gy * gdx; vir[4] += gy * gdy; vir[5] += gy * gdz;
                 vir[6] += gz * gdx; vir[7] += gz * gdy; vir[8] += gz * gdz;
-                float* go = a.g + 3 * (size_t)e;
+                float* go = a.g + 3 * (size_t)(e0 + e);
                 go[0] = gx; go[1] = gy; go[2] = gz;
             }
             __syncwarp();
         };
 
         int qn = 0;
-        for (int base = e0; base < e1; base += 32) {
-            const int e = base + lane;
-            const Geom g = edge_geometry(a, e, e < e1, xi, yi, zi, ti);
+        for (int base = 0; base < len; base += 32) {
+            const int e = base + lane;                                // offset inside the row
+            const Geom g = edge_geometry(a, e0 + e, e < len, xi, yi, zi, ti);
             const unsigned vmask = __ballot_sync(kFull, g.valid);
             const int p = qn + __popc(vmask & lt_mask);   // queue slot of this lane's edge, if it has one
             if (g.valid && p < 32) {
                 qes[p] = make_int4(g.row, g.pair, __float_as_int(g.t), __float_as_int(g.chi));
                 qd[p] = g.dx; qd[32 + p] = g.dy; qd[64 + p] = g.dz; qd[96 + p] = g.dchi;
                 qd[128 + p] = __int_as_float(e);
-            } else if (!g.valid && e < e1) {
-                float* go = a.g + 3 * (size_t)e;
+            } else if (!g.valid && e < len) {
+                float* go = a.g + 3 * (size_t)(e0 + e);
                 go[0] = 0.f; go[1] = 0.f; go[2] = 0.f;
             }
             qn += __popc(vmask);

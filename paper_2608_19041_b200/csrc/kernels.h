@@ -28,7 +28,7 @@ struct EdgeArgs {
     const float* pairmod;
     const double* xs;       // [N][3] sorted positions
     const int* type_s;
-    const int* row_ptr;
+    const eidx_t* row_ptr;
     const int* src;
     const int* shift;
     double Lx, Ly, Lz;

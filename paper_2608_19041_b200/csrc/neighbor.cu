@@ -11,6 +11,7 @@
 // precision with explicit round-to-nearest adds and multiplies (no contraction into fused
 // multiply-adds), which makes the edge set reproducible bit for bit.
 #include <cub/cub.cuh>
+#include <thrust/iterator/transform_iterator.h>
 
 #include <cmath>
 
@@ -117,7 +118,7 @@ __global__ void k_gather_sorted(int N, const int* __restrict__ sidx, const doubl
 template <bool FILL>
 __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ skey,
                              const int* __restrict__ cell_start, const double* __restrict__ xs0,
-                             int* __restrict__ deg, const int* __restrict__ row_ptr,
+                             int* __restrict__ deg, const eidx_t* __restrict__ row_ptr,
                              int* __restrict__ src, int* __restrict__ shift, int* __restrict__ err) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -127,7 +128,7 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     const int cx = key % g.nc[0], cy = (key / g.nc[0]) % g.nc[1], cz = key / (g.nc[0] * g.nc[1]);
     const double xi = xs0[3 * (size_t)i], yi = xs0[3 * (size_t)i + 1], zi = xs0[3 * (size_t)i + 2];
     int count = 0;
-    const int base_out = FILL ? row_ptr[i] : 0;
+    const eidx_t base_out = FILL ? row_ptr[i] : 0;
     const unsigned lt_mask = (1u << lane) - 1u;
     const int wz = 2 * g.m[2] + 1, wy = 2 * g.m[1] + 1, wx = 2 * g.m[0] + 1;
     const int sz0 = walk_start(cz, g.m[2], g.nc[2], g.pbc[2], g.sorted);
@@ -170,7 +171,7 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
                     }
                     const unsigned mask = __ballot_sync(0xffffffffu, ok);
                     if (FILL && ok) {
-                        const int p = base_out + count + __popc(mask & lt_mask);
+                        const eidx_t p = base_out + count + __popc(mask & lt_mask);
                         src[p] = j;
                         shift[p] = pack_shift(nx, ny, nz);
                     }
@@ -184,43 +185,38 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     if (!FILL && lane == 0) deg[i] = count;
 }
 
-// 64-bit sum of the row lengths: the 32-bit prefix sum wraps silently once a list passes 2^31
-// edges, and what wrapped must not size the edge arrays
-__global__ void k_sum_deg64(int N, const int* __restrict__ deg, unsigned long long* __restrict__ out) {
-    unsigned long long v = 0;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) v += (unsigned)deg[i];
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    if ((threadIdx.x & 31) == 0 && v) atomicAdd(out, v);
-}
-
 // rev[e] = slot of (j <- i, -n) for e = (i <- j, n); -1 when absent (can only happen for
 // pairs whose two orientations round to opposite sides of the list radius).
-__global__ void k_reverse_map(int N, int sorted, const int* __restrict__ row_ptr, const int* __restrict__ src,
-                              const int* __restrict__ shift, int* __restrict__ rev) {
+__global__ void k_reverse_map(int N, int sorted, const eidx_t* __restrict__ row_ptr, const int* __restrict__ src,
+                              const int* __restrict__ shift, eidx_t* __restrict__ rev) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= N) return;
     const int i = warp;
-    const int e0 = row_ptr[i], e1 = row_ptr[i + 1];
-    for (int e = e0 + lane; e < e1; e += 32) {
+    const eidx_t e0 = row_ptr[i];
+    const int len = (int)(row_ptr[i + 1] - e0);
+    for (int k = lane; k < len; k += 32) {
+        const eidx_t e = e0 + k;
         const int j = src[e];
         const int s = shift[e];
         const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff),
                   nz = (int)(signed char)((s >> 16) & 0xff);
         const int want = pack_shift(-nx, -ny, -nz);
-        int found = -1;
-        const int f0 = row_ptr[j], f1 = row_ptr[j + 1];
+        eidx_t found = -1;
+        const eidx_t f0 = row_ptr[j];
+        const int flen = (int)(row_ptr[j + 1] - f0);
+        const int* srow = src + f0;
+        const int* hrow = shift + f0;
         if (sorted) {          // rows ascend in the neighbour index, each neighbour at most once
-            int lo = f0, hi = f1;
+            int lo = 0, hi = flen;
             while (lo < hi) {
-                const int mid = lo + ((hi - lo) >> 1);     // lo + hi would pass 2^31 in a long list
-                if (src[mid] < i) lo = mid + 1; else hi = mid;
+                const int mid = (lo + hi) >> 1;            // offsets inside one row: no overflow
+                if (srow[mid] < i) lo = mid + 1; else hi = mid;
             }
-            if (lo < f1 && src[lo] == i && shift[lo] == want) found = lo;
+            if (lo < flen && srow[lo] == i && hrow[lo] == want) found = f0 + lo;
         } else {
-            for (int f = f0; f < f1; ++f) {
-                if (src[f] == i && shift[f] == want) { found = f; break; }
+            for (int f = 0; f < flen; ++f) {
+                if (srow[f] == i && hrow[f] == want) { found = f0 + f; break; }
             }
         }
         rev[e] = found;
@@ -249,15 +245,15 @@ __global__ void k_gather_positions(int N, const int* __restrict__ perm, const in
 }
 
 // ---- export in caller numbering ------------------------------------------------------
-__global__ void k_export_deg(int N, const int* __restrict__ perm, const int* __restrict__ row_ptr,
+__global__ void k_export_deg(int N, const int* __restrict__ perm, const eidx_t* __restrict__ row_ptr,
                              int* __restrict__ deg_o) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
-    deg_o[perm[i]] = row_ptr[i + 1] - row_ptr[i];
+    deg_o[perm[i]] = (int)(row_ptr[i + 1] - row_ptr[i]);
     if (i == 0) deg_o[N] = 0;
 }
 
-__global__ void k_export_rows(int N, const int* __restrict__ perm, const int* __restrict__ row_ptr,
+__global__ void k_export_rows(int N, const int* __restrict__ perm, const eidx_t* __restrict__ row_ptr,
                               const int* __restrict__ src, const int* __restrict__ shift,
                               const int* __restrict__ row_ptr_o, int* __restrict__ src_o,
                               signed char* __restrict__ shift_o) {
@@ -265,7 +261,8 @@ __global__ void k_export_rows(int N, const int* __restrict__ perm, const int* __
     const int lane = threadIdx.x & 31;
     if (warp >= N) return;
     const int i = warp, o = perm[i];
-    const int e0 = row_ptr[i], n = row_ptr[i + 1] - e0, q0 = row_ptr_o[o];
+    const eidx_t e0 = row_ptr[i];
+    const int n = (int)(row_ptr[i + 1] - e0), q0 = row_ptr_o[o];
     for (int k = lane; k < n; k += 32) {
         const int s = shift[e0 + k];
         src_o[q0 + k] = perm[src[e0 + k]];
@@ -274,6 +271,10 @@ __global__ void k_export_rows(int N, const int* __restrict__ perm, const int* __
         shift_o[3 * (size_t)(q0 + k) + 2] = (signed char)((s >> 16) & 0xff);
     }
 }
+
+struct WidenDeg {
+    __host__ __device__ eidx_t operator()(int v) const { return (eidx_t)v; }
+};
 
 #define NB_CHECK(call)                                                              \
     do {                                                                            \
@@ -376,7 +377,12 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     while ((1LL << end_bit) < ncell) ++end_bit;
     size_t need_tmp = 0, need_scan = 0;
     cub::DeviceRadixSort::SortPairs(nullptr, need_tmp, nb->key, nb->key2, nb->idx, nb->idx2, N, 0, end_bit, st);
-    cub::DeviceScan::ExclusiveSum(nullptr, need_scan, nb->deg, nb->row_ptr, N + 1, st);
+    // row offsets are accumulated in 64 bits from the 32-bit row lengths
+    auto deg_wide = thrust::make_transform_iterator(static_cast<const int*>(nb->deg), WidenDeg());
+    cub::DeviceScan::ExclusiveScan(nullptr, need_scan, deg_wide, nb->row_ptr, cub::Sum(), (eidx_t)0, N + 1, st);
+    size_t need_scan32 = 0;                     // the export scans into the caller's 32-bit row pointers
+    cub::DeviceScan::ExclusiveSum(nullptr, need_scan32, nb->deg, (int*)nullptr, N + 1, st);
+    if (need_scan32 > need_scan) need_scan = need_scan32;
     if (need_scan > need_tmp) need_tmp = need_scan;
     if (need_tmp > nb->cub_bytes) {
         if (nb->cub_tmp) dev_free(nb->cub_tmp);
@@ -397,19 +403,10 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
                                            nullptr, nullptr, d_err);
     NB_CHECK(cudaMemsetAsync(nb->deg + N, 0, sizeof(int), st));
     tmp_bytes = nb->cub_bytes;
-    NB_CHECK(cub::DeviceScan::ExclusiveSum(nb->cub_tmp, tmp_bytes, nb->deg, nb->row_ptr, N + 1, st));
-    // the unsorted keys are no longer needed: their buffer holds the 64-bit total
-    unsigned long long* d_total = reinterpret_cast<unsigned long long*>(nb->key);
-    NB_CHECK(cudaMemsetAsync(d_total, 0, sizeof(unsigned long long), st));
-    k_sum_deg64<<<(N + 4 * TB - 1) / (4 * TB) < 1024 ? (N + 4 * TB - 1) / (4 * TB) : 1024, TB, 0, st>>>(N, nb->deg, d_total);
-    unsigned long long total64 = 0;
-    NB_CHECK(cudaMemcpyAsync(&total64, d_total, sizeof(total64), cudaMemcpyDeviceToHost, st));
+    NB_CHECK(cub::DeviceScan::ExclusiveScan(nb->cub_tmp, tmp_bytes, deg_wide, nb->row_ptr, cub::Sum(), (eidx_t)0, N + 1, st));
+    eidx_t total = 0;
+    NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(total), cudaMemcpyDeviceToHost, st));
     NB_CHECK(cudaStreamSynchronize(st));
-    if (total64 > 0x7fffffffull - 64) {      // the margin keeps "edge index + lane" inside int as well
-        *err = "neighbor list has " + std::to_string(total64) + " edges; edge indices are 32-bit (at most 2147483583)";
-        return UMLMD_E_CAPACITY;
-    }
-    const int total = (int)total64;
     nb->E = total;
     if (total > nb->E_cap) {
         int64_t c;

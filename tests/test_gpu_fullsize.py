@@ -108,8 +108,8 @@ def _cluster_around(pos_w, cell, k, radius):
     return idx, d[idx] + 0.5 * L
 
 
-def test_near_the_32_bit_edge_limit():
-    # the largest jittered-diamond box whose neighbor list still fits 32-bit edge indices
+def test_just_below_2_31_edges():
+    # the largest jittered-diamond box whose neighbor list the 32-bit verification export still takes
     # (6,859,000 atoms, 1.88e9 listed edges, 3 E > 2^32): properties that hold at any size, sampled
     # rows against brute force, and energies and forces of sampled atoms against the oracle run
     # on the isolated cluster that determines them (radius 2 r_c around the atom)
@@ -161,18 +161,40 @@ def test_near_the_32_bit_edge_limit():
     m.close()
 
 
-def test_more_than_2_31_edges_is_refused_not_wrapped():
-    # 8,000,000 diamond atoms with the 1 A skin list 2.19e9 edges: the build must say so (the
-    # 32-bit prefix sum alone would wrap) and leave the handle usable
+def test_more_than_2_31_edges():
+    # 8,000,000 diamond atoms with the 1 A skin list 2.19e9 edges, more than a 32-bit offset holds:
+    # edge offsets are 64-bit inside the library (only the verification export is 32-bit and says
+    # so); energies and forces of sampled atoms against the oracle on their isolated clusters
     name = "paper_nano_c1m"
     cfg = CONFIGS[name]
     s = make_system(dict(cfg["system"], cells=100))
-    m = _binding().Model(workload_blob(name))
+    N = len(s["pos"])
+    rc = cfg["profile"]["rc"]
+    blob = workload_blob(name)
+    m = _binding().Model(blob)
     pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
     types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], cfg["md"]["skin"])
+    assert m.query()["n_edges"] > 2 ** 31
     with pytest.raises(_binding().UmlmdError) as e:
-        m.build_neighbors(pos, types, s["cell"], s["pbc"], cfg["md"]["skin"])
+        m.get_neighbors()
     assert e.value.code == -9
-    m.build_neighbors(pos, types, s["cell"], s["pbc"], 0.0)      # about 158 neighbours each: 1.26e9 edges fit
-    assert 1.2e9 < m.query()["n_edges"] < 2 ** 31
+    out = m.compute(pos, atom_energy=True)
+    Ei = out["atom_energy"].cpu().numpy()
+    F = out["forces"].cpu().numpy()
+    assert np.isfinite(Ei).all() and np.isfinite(F).all()
+    f_scale, e_scale = np.abs(F).max(), np.abs(Ei).max()
+    assert abs(Ei.sum() - out["energy"]) <= 1e-9 * max(1.0, np.abs(Ei).sum())
+    assert np.abs(F.sum(axis=0)).max() <= 2e-6 * f_scale * np.sqrt(N) * 10
+    rng = np.random.Generator(np.random.PCG64(100))
+    pos_w = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    o = orc.Oracle(blob)
+    big = [[1000.0, 0, 0], [0, 1000.0, 0], [0, 0, 1000.0]]
+    # one atom from the end of the caller's numbering and two anywhere (the internal order is by cell)
+    for k in [N - 1] + list(rng.choice(N, size=2, replace=False)):
+        idx, xyz = _cluster_around(pos_w, s["cell"], int(k), 2 * rc + 0.5)
+        ref = o.compute(xyz, s["types"][idx], big, (0, 0, 0))
+        assert np.abs(F[k] - ref["F"][0]).max() <= min(1e-4, 2e-5 * f_scale + 2e-7), (k, F[k], ref["F"][0])
+        near = np.nonzero(((xyz - xyz[0]) ** 2).sum(axis=1) < rc * rc)[0]
+        assert np.abs(Ei[idx[near]] - ref["E_i"][near]).max() <= 1e-5 * e_scale
     m.close()
