@@ -134,11 +134,11 @@ def work_model(p, n_atoms, e_rc, e_list, one_species=False):
         "mlp_backward": dict(flops=mlp * n_atoms, bytes=4 * n_atoms * (D + 2 * NH * F), pipe="tensor"),
         "invariants_forward": dict(flops=0, bytes=4 * n_atoms * (S + 2 + D), pipe="hbm"),
         "invariants_backward": dict(flops=0, bytes=4 * n_atoms * (2 * (S + 2) + D), pipe="hbm"),
-        "force_assembly": dict(flops=0, bytes=e_list * (12 + 12 + 4) + n_atoms * 72, pipe="hbm"),
+        "force_assembly": dict(flops=0, bytes=e_list * (12 + 12 + 8) + n_atoms * 72, pipe="hbm"),
         "gather_positions": dict(flops=0, bytes=n_atoms * (24 * 3 + 16), pipe="hbm"),
         "energy_virial_reduce": dict(flops=0, bytes=n_atoms * 8, pipe="hbm"),
         "integrate": dict(flops=0, bytes=n_atoms * 2 * (24 * 5 + 4), pipe="hbm"),
-        "neighbor_build": dict(flops=0, bytes=e_list * 12 + n_atoms * 200, pipe="hbm"),
+        "neighbor_build": dict(flops=0, bytes=e_list * 16 + n_atoms * 200, pipe="hbm"),
     }
 
 
