@@ -79,7 +79,9 @@ int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out);
 /*
  * Create a model from a weight blob (host memory, little-endian):
  *   char[8] "UMLMD1\0\0"; u32 version = 1; u32 C0, L, R, N_rbf, n_hidden, F, T, basis (0 =
- *   Bessel); f64 rc, table_dx; then float32 arrays, row-major, y = x W convention:
+ *   Bessel, f_n = sin(omega_n rho) / rho; 1 = Gaussian, f_n = exp(-(rho - c_n)^2 / (2 s^2)) with
+ *   s = rc / (N_rbf - 1), the centres c_n in the place of omega); f64 rc, table_dx; then float32
+ *   arrays, row-major, y = x W convention:
  *   X0[T,C0], omega[N_rbf], W_in[N_rbf,2H], W_out[H,C0], W_mode[H,R], W_p_in[2C0,2Hp],
  *   W_p_out[Hp,C0(2+R)] (column blocks scale|shift|mode), W_1[C1,C1], W_2[C2,C2],
  *   A_1[C1,K1], A_2[C2,K2], mu[D_out], sigma[D_out], Theta_1[D_out,F], b_1[F],

@@ -124,10 +124,11 @@ def parse_blob(blob):
     hb = struct.calcsize(_HEADER_FMT)
     magic, version, C0, L, R, N_rbf, n_hidden, F, T, basis, rc, table_dx = struct.unpack(
         _HEADER_FMT, blob[:hb])
-    if magic != MAGIC or version != 1 or basis != 0:
+    if magic != MAGIC or version != 1 or basis not in (0, 1):
         raise ValueError("bad blob header")
     w = widths(C0, L, R)
-    p = dict(C0=C0, L=L, R=R, N_rbf=N_rbf, n_hidden=n_hidden, F=F, T=T, rc=rc, table_dx=table_dx, **w)
+    p = dict(C0=C0, L=L, R=R, N_rbf=N_rbf, n_hidden=n_hidden, F=F, T=T, rc=rc, table_dx=table_dx,
+             basis=("bessel", "gaussian")[basis], **w)
     H, Hp, C1, C2, K1, K2, D = w["H"], w["Hp"], w["C1"], w["C2"], w["K1"], w["K2"], w["D_out"]
     shapes = [("X0", (T, C0)), ("omega", (N_rbf,)), ("W_in", (N_rbf, 2 * H)), ("W_out", (H, C0)),
               ("W_mode", (H, R)), ("W_p_in", (2 * C0, 2 * Hp)), ("W_p_out", (Hp, C0 * (2 + R))),
@@ -351,6 +352,15 @@ def silu(x):
     return x * torch.sigmoid(x)
 
 
+def gaussian_basis(rho, centers, rc):
+    """The Gaussian family of the radial-basis paragraph: f_n = exp(-(rho - c_n)^2 / (2 sigma_g^2))
+    with the fixed width sigma_g = rc / (N_rbf - 1); like the Bessel family, no cutoff factor.
+    The centres c_n take the blob slot of the Bessel frequencies."""
+    sg = rc / (centers.shape[0] - 1)
+    d = rho[:, None] - centers[None, :]
+    return torch.exp(-d * d / (2.0 * sg * sg))
+
+
 def swiglu(x, W):
     """Eq. "swiglu": [x_g, x_v] = x W, SiLU(x_g) * x_v; gate = first H columns."""
     a = x @ W
@@ -358,9 +368,10 @@ def swiglu(x, W):
     return silu(a[..., :H]) * a[..., H:]
 
 
-def radial_map(rho, prm):
+def radial_map(rho, prm, basis="bessel", rc=None):
     """Eqs. "radial-map", "radial-modes": g(rho) in R^C0 and q(rho) in R^R."""
-    h = swiglu(bessel_basis(rho, prm["omega"]), prm["W_in"])
+    f = bessel_basis(rho, prm["omega"]) if basis == "bessel" else gaussian_basis(rho, prm["omega"], rc)
+    h = swiglu(f, prm["W_in"])
     return h @ prm["W_out"], h @ prm["W_mode"]
 
 
@@ -396,7 +407,7 @@ def aggregate(p, prm, pair, n_centers, dst, type_i, type_j, rij):
     rho = torch.sqrt((rij * rij).sum(dim=1) + EPS_REG ** 2)
     u = rij / rho[:, None]
     chi = envelope(rho, rc)
-    g, q = radial_map(rho, prm)
+    g, q = radial_map(rho, prm, p.get("basis", "bessel"), rc)
     psi = gamma[type_i, type_j] * g + beta[type_i, type_j]              # Eq. "amplitude"
     if p["R"] > 0:
         psi = psi + torch.einsum("ecm,em->ec", U[type_i, type_j], q)

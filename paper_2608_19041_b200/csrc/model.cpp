@@ -169,7 +169,8 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
     if (u[0] != 1) { *err = "unsupported blob version"; return UMLMD_E_BAD_BLOB; }
     const int C0 = (int)u[1], L = (int)u[2], R = (int)u[3], N_rbf = (int)u[4], NH = (int)u[5],
               F = (int)u[6], T = (int)u[7];
-    if (u[8] != 0) { *err = "only the Bessel radial family is supported"; return UMLMD_E_UNSUPPORTED_PROFILE; }
+    if (u[8] > 1) { *err = "radial family must be 0 (Bessel) or 1 (Gaussian)"; return UMLMD_E_UNSUPPORTED_PROFILE; }
+    const bool gaussian = u[8] == 1;
     Dims& d = m->d;
     if (!derive_dims(C0, L, R, &d)) {
         *err = "unsupported (C0, L, R): C0 in {8,16,32,64,128}, L in {2,3}, R in {0,2,4,8}";
@@ -180,6 +181,7 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
         *err = "unsupported N_rbf / hidden layers / width / type count";
         return UMLMD_E_UNSUPPORTED_PROFILE;
     }
+    if (gaussian && N_rbf < 2) { *err = "the Gaussian family needs at least two basis functions"; return UMLMD_E_UNSUPPORTED_PROFILE; }
     d.N_rbf = N_rbf; d.n_hidden = NH; d.F = F; d.T = T;
     m->rc = rd[0];
     m->dx = dx_override > 0 ? dx_override : rd[1];
@@ -231,6 +233,11 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
         for (int s = 0; s <= n_rows; ++s) {
             const double rho = s * m->dx;
             for (int n = 0; n < N_rbf; ++n) {
+                if (gaussian) {   // f_n = exp(-(rho - c_n)^2 / (2 s^2)), s = rc / (N_rbf - 1); centres in the omega slot
+                    const double sg = m->rc / (N_rbf - 1), t = (rho - omega[n]) / sg;
+                    f[n] = std::exp(-0.5 * t * t); f1[n] = -t / sg * f[n];
+                    continue;
+                }
                 double j, j1;
                 const double w = omega[n];
                 j0_derivs(w * rho, &j, &j1);

@@ -208,6 +208,15 @@ def test_species_mix_may_change_between_builds_on_one_handle():
     m.close()
 
 
+@pytest.mark.parametrize("name", ["p16_3_2", "p32_2_0_res"])
+def test_parity_gaussian_radial_family(name):
+    # only the create-time table differs: Gaussian basis functions with the centres in the blob
+    p = SMALL_PROFILES[name]
+    blob = make_blob(p, seed=47, bias_scale=0.2, basis="gaussian")
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    _compare(blob, s)
+
+
 def test_parity_with_node_tiling():
     # several workspace tiles with a ragged last tile
     p = SMALL_PROFILES["p16_2_0"]

@@ -96,19 +96,21 @@ def test_calls_before_a_neighbor_build_fail_cleanly():
     assert q["n_atoms"] == 0 and q["table_rows"] == 3000 and q["rc"] == 6.0
 
 
+@pytest.mark.parametrize("basis", ["bessel", "gaussian"])
 @pytest.mark.parametrize("name", ["p16_2_0", "p32_2_4", "p32_3_2"])
-def test_radial_table_reproduces_continuous_radial_map(name):
+def test_radial_table_reproduces_continuous_radial_map(name, basis):
     # the paper reports 1.3e-7 .. 1.8e-7 (relative to the largest entry) for these three
     # (C0, L, R) at a spacing of 0.002 Angstrom in single precision
     p = SMALL_PROFILES[name]
-    blob = make_blob(p, seed=5)
+    blob = make_blob(p, seed=5, basis=basis)
     m = binding.Model(blob)
     o = orc.Oracle(blob)
+    assert o.p["basis"] == basis
     rho = np.random.default_rng(0).uniform(0.0, p["rc"], 4000)
     rho[:3] = [0.0, 1e-9, p["rc"] - 1e-9]
     g, dg = m.eval_radial_table(rho)
     r = torch.from_numpy(rho).requires_grad_(True)
-    go, qo = orc.radial_map(r, o.prm)
+    go, qo = orc.radial_map(r, o.prm, basis, p["rc"])
     ref = torch.cat([go, qo], dim=1)
     scale = ref.abs().max().item()
     assert np.abs(g - ref.detach().numpy()).max() / scale < 3e-7

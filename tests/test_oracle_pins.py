@@ -132,6 +132,31 @@ def test_bessel_basis_values_and_limit():
     assert np.allclose(f[3], np.sin(omega.numpy() * 5.0) / 5.0, rtol=1e-14, atol=1e-17)
 
 
+def test_gaussian_basis_against_the_normal_density():
+    # fixed width sigma_g = rc / (N_rbf - 1): f_n is the normal density of that width, centred on
+    # c_n, rescaled to 1 at its maximum; half maximum at sigma_g sqrt(2 ln 2); the family has no
+    # cutoff factor, so it does not vanish at rc
+    import scipy.stats
+    rc, centers = 6.0, torch.tensor([0.0, 1.3, 2.0, 4.4, 6.0], dtype=torch.float64)
+    sg = rc / 4
+    rho = torch.tensor([0.0, 0.9, 2.0, 2.0 + sg, 2.0 - sg * math.sqrt(2 * math.log(2)), 6.0], dtype=torch.float64)
+    f = orc.gaussian_basis(rho, centers, rc).numpy()
+    ref = scipy.stats.norm.pdf(rho.numpy()[:, None], loc=centers.numpy()[None, :], scale=sg) * sg * math.sqrt(2 * math.pi)
+    assert np.allclose(f, ref, rtol=1e-14, atol=0)
+    assert f[2, 2] == 1.0 and abs(f[3, 2] - math.exp(-0.5)) < 1e-15 and abs(f[4, 2] - 0.5) < 1e-15
+    assert f[5, 3] > 0.5                                  # at rho = rc, centre 4.4: no cutoff factor
+    # the radial map routes through the family named in the blob header
+    p = SMALL_PROFILES["p16_2_0"]
+    ob, og = orc.Oracle(make_blob(p, seed=3)), orc.Oracle(make_blob(p, seed=3, basis="gaussian"))
+    assert ob.p["basis"] == "bessel" and og.p["basis"] == "gaussian"
+    r = torch.tensor([0.3, 2.5, 5.9], dtype=torch.float64)
+    g, _ = orc.radial_map(r, og.prm, "gaussian", p["rc"])
+    h = orc.swiglu(torch.from_numpy(scipy.stats.norm.pdf(r.numpy()[:, None], loc=og.prm["omega"].numpy()[None, :],
+                                                         scale=p["rc"] / (p["N_rbf"] - 1))
+                                    * p["rc"] / (p["N_rbf"] - 1) * math.sqrt(2 * math.pi)), og.prm["W_in"])
+    assert np.allclose(g.numpy(), (h @ og.prm["W_out"]).numpy(), rtol=1e-13, atol=1e-15)
+
+
 # ---------------------------------------------------------------- harmonics
 
 def test_addition_theorem_degrees_0_to_4():

@@ -4,7 +4,7 @@ Blob layout (little-endian):
 
     char[8]  magic  "UMLMD1\\0\\0"
     u32      version (=1)
-    u32      C0, L, R, N_rbf, n_hidden, F, T, basis (0 = Bessel)
+    u32      C0, L, R, N_rbf, n_hidden, F, T, basis (0 = Bessel, 1 = Gaussian)
     f64      rc, table_dx
     f32[]    arrays, row-major, right-multiplication convention y = x W, in the
              order given by ``blob_array_shapes``.
@@ -52,20 +52,24 @@ def blob_array_shapes(p):
     return shapes
 
 
-def make_blob(p, seed, calibration=None, bias_scale=0.0, e_ref_scale=0.0, head_scale=1.0):
+def make_blob(p, seed, calibration=None, bias_scale=0.0, e_ref_scale=0.0, head_scale=1.0, basis="bessel"):
     """Return the blob bytes for profile ``p``.
 
     ``calibration`` is an optional (mu, sigma) pair of length-D_out arrays.
     ``bias_scale`` / ``e_ref_scale`` > 0 draw non-zero MLP biases / reference
     energies (used by tests so that those terms are exercised).  ``head_scale``
     multiplies the scalar head w_head, i.e. the energy scale of the random potential.
+    ``basis`` = "gaussian" sets the header's radial-family field to 1 and fills the frequency
+    slot with N_rbf centres, evenly spaced on [0, rc] and then jittered (they are trainable).
     """
     rng = np.random.Generator(np.random.PCG64(seed))
     chunks = [struct.pack(HEADER_FMT, MAGIC, 1, p["C0"], p["L"], p["R"], p["N_rbf"],
-                          p["n_hidden"], p["F"], p["T"], 0, p["rc"], p["table_dx"])]
+                          p["n_hidden"], p["F"], p["T"], {"bessel": 0, "gaussian": 1}[basis], p["rc"], p["table_dx"])]
     for name, shape in blob_array_shapes(p):
         n = int(np.prod(shape)) if len(shape) else 1
-        if name == "omega":
+        if name == "omega" and basis == "gaussian":
+            a = np.linspace(0.0, p["rc"], shape[0]) + 0.1 * p["rc"] / shape[0] * rng.standard_normal(shape)
+        elif name == "omega":
             a = np.arange(1, shape[0] + 1, dtype=np.float64) * math.pi / p["rc"]
         elif name == "A_1" and shape[0] == shape[1]:
             a = np.eye(shape[0])
