@@ -38,7 +38,8 @@ enum {
     UMLMD_E_BAD_BLOB = -2,            /* magic / version / size mismatch, non-finite weight */
     UMLMD_E_UNSUPPORTED_PROFILE = -3, /* C0 not in {8,16,32,64,128}, L not in {2,3},
                                          R not in {0,2,4,8}, F % 4 != 0, ...                */
-    UMLMD_E_UNSUPPORTED_CELL = -4,    /* non-orthorhombic cell, non-positive edge           */
+    UMLMD_E_UNSUPPORTED_CELL = -4,    /* singular or non-finite cell, non-positive edge,
+                                         more than 127 periodic images along a direction     */
     UMLMD_E_NO_NEIGHBORS = -5,        /* compute/step called before build_neighbors         */
     UMLMD_E_STALE_NEIGHBORS = -6,     /* an atom moved more than skin/2 since the build     */
     UMLMD_E_NONFINITE = -7,           /* NaN or Inf in positions, energy or forces          */
@@ -109,9 +110,12 @@ const char* umlmd_last_error(const umlmd_t* h);
  * |(r_j + n.cell) - r_i|^2 < r_list^2 (true distance, strict), periodic images being
  * distinct neighbor instances, both orientations stored, no capacity limit.
  *   d_pos   [N,3] double, any image of each atom; folded into the cell internally with
- *           frac - floor(frac) along periodic directions (n refers to folded positions)
+ *           frac - floor(frac) along periodic directions (n refers to folded positions);
+ *           periodicity of direction k means translation by cell vector k
  *   d_type  [N] int32 species, each in [0, T) (checked: UMLMD_E_INVALID_ARG otherwise)
- *   cell    9 doubles, rows are cell vectors; must be orthorhombic (diagonal)
+ *   cell    9 doubles, rows are the cell vectors a, b, c; any non-singular cell.  A diagonal
+ *           (orthorhombic) cell takes the exactly reproducible path below; a general cell is
+ *           folded with f = r cell^-1, r - floor(f) . cell, and images are offset by n . cell
  *   pbc     3 ints, non-zero = periodic along that cell vector
  *   skin    extra list radius in Angstrom (>= 0); edges beyond rc carry zero weight
  * The predicate is evaluated in double precision as ((xj + n*L) - xi), d2 = (dx*dx +

@@ -166,6 +166,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ea.species_slot = h->d_species + d.T; ea.n_present = (int)h->present.size();
         ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
+        for (int k = 0; k < 9; ++k) ea.H[k] = nb.H[k];
+        ea.tri = nb.tri;
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
         ea.virial_part = h->virial_part + (size_t)vpart_used * 9;
         { Scope sc(h, kEdgeFwd, 1); API_CUDA(h, launch_edge_forward(ea, h->st)); }
@@ -248,11 +250,11 @@ int ensure_device_model(umlmd_t* h) {
     return UMLMD_OK;
 }
 
-int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type, const double L[3],
+int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type, const double cell[9],
                const int pbc[3], double skin) {
     int rc = ensure_device_model(h);
     if (rc != UMLMD_OK) return rc;
-    { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, d_pos, d_type, L, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
+    { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, d_pos, d_type, cell, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
     h->have_list = true;
     h->steps_since_build = 0;
@@ -357,16 +359,18 @@ int umlmd_build_neighbors(umlmd_t* h, int64_t N, const double* d_pos, const int3
     if (!h) return UMLMD_E_INVALID_ARG;
     if (N < 0 || !cell || !pbc || !(skin >= 0) || !std::isfinite(skin) || (N > 0 && (!d_pos || !d_type)))
         return fail(h, UMLMD_E_INVALID_ARG, "bad argument to umlmd_build_neighbors");
+    bool diagonal = true;
     for (int i = 0; i < 3; ++i)
         for (int j = 0; j < 3; ++j) {
             const double v = cell[3 * i + j];
             if (!std::isfinite(v)) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "non-finite cell");
-            if (i != j && v != 0.0) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "only orthorhombic cells are supported");
-            if (i == j && !(v > 0.0)) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "cell edges must be positive");
+            if (i != j && v != 0.0) diagonal = false;
         }
-    const double L[3] = {cell[0], cell[4], cell[8]};
+    if (diagonal)
+        for (int i = 0; i < 3; ++i)
+            if (!(cell[4 * i] > 0.0)) return fail(h, UMLMD_E_UNSUPPORTED_CELL, "cell edges must be positive");
     h->have_md = false;
-    int rc = build_list(h, N, d_pos, d_type, L, pbc, skin);
+    int rc = build_list(h, N, d_pos, d_type, cell, pbc, skin);
     if (rc != UMLMD_OK) return rc;
     if (N > 0) API_CUDA(h, cudaMemcpyAsync(h->type_o, d_type, sizeof(int) * N, cudaMemcpyDeviceToDevice, h->st));
     // which species occur: few enough of them get per-pair amplitude tables (see below)
@@ -468,9 +472,10 @@ static int maybe_rebuild(umlmd_t* h, int rebuild_every) {
     }
     if (rebuild) {
         const double skin = h->nb.skin;
-        const double L[3] = {h->nb.L[0], h->nb.L[1], h->nb.L[2]};
+        double cell[9];
+        for (int k = 0; k < 9; ++k) cell[k] = h->nb.H[k];
         const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};
-        return build_list(h, N, h->md_pos, h->type_o, L, pbc, skin);
+        return build_list(h, N, h->md_pos, h->type_o, cell, pbc, skin);
     }
     return UMLMD_OK;
 }

@@ -79,7 +79,9 @@ typedef long long eidx_t;      // edge offsets are 64-bit: a list may hold more 
 
 struct NeighborDev {
     int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;
-    double L[3] = {0, 0, 0};
+    double L[3] = {0, 0, 0};     // cell edge lengths (the diagonal of H)
+    double H[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // cell vectors as rows
+    int tri = 0;                 // the cell has off-diagonal components
     int pbc[3] = {1, 1, 1};
     double skin = 0, r_list = 0;
     double* wpos = nullptr;      // [N][3] folded positions, caller order (build time)

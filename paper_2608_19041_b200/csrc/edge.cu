@@ -46,9 +46,15 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool 
     const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff),
               nz = (int)(signed char)((s >> 16) & 0xff);
     const double* xj = a.xs + 3 * (size_t)j;
-    g.dx = (float)((xj[0] + nx * a.Lx) - xi);
-    g.dy = (float)((xj[1] + ny * a.Ly) - yi);
-    g.dz = (float)((xj[2] + nz * a.Lz) - zi);
+    if (a.tri) {        // general cell: the image offset is n . H
+        g.dx = (float)((xj[0] + ((nx * a.H[0] + ny * a.H[3]) + nz * a.H[6])) - xi);
+        g.dy = (float)((xj[1] + ((nx * a.H[1] + ny * a.H[4]) + nz * a.H[7])) - yi);
+        g.dz = (float)((xj[2] + ((nx * a.H[2] + ny * a.H[5]) + nz * a.H[8])) - zi);
+    } else {
+        g.dx = (float)((xj[0] + nx * a.Lx) - xi);
+        g.dy = (float)((xj[1] + ny * a.Ly) - yi);
+        g.dz = (float)((xj[2] + nz * a.Lz) - zi);
+    }
     const float r2 = g.dx * g.dx + g.dy * g.dy + g.dz * g.dz + kEpsReg * kEpsReg;
     g.rho = sqrtf(r2);
     if (!(g.rho < a.d.rc)) return g;       // skin-shell edge: zero weight

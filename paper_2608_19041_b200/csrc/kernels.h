@@ -11,8 +11,8 @@ namespace umd {
 // Full build: fold + bin + sort + count + scan + fill + reverse map.  Synchronises once
 // (to learn the edge count and grow the edge arrays).  Returns a UMLMD_* code.
 int neighbor_build(NeighborDev* nb, int64_t N, const double* d_pos, const int32_t* d_type,
-                   const double L[3], const int pbc[3], double skin, double rc, int* d_err,
-                   cudaStream_t st, std::string* err);
+                   const double cell[9], const int pbc[3], double skin, double rc, int* d_err,
+                   cudaStream_t st, std::string* err);   // cell: the three cell vectors as rows
 void neighbor_free(NeighborDev* nb);
 // Export the list in caller numbering (device buffers of the caller).
 int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
@@ -32,6 +32,8 @@ struct EdgeArgs {
     const int* src;
     const int* shift;
     double Lx, Ly, Lz;
+    double H[9];            // cell vectors as rows, used instead of Lx, Ly, Lz when tri
+    int tri;
     int a0, a1;             // destination range [a0, a1) of this tile
     float* state;           // [a1-a0][SP]: forward writes sums; backward reads dE/d(sums)
     float* g;               // [E][3] per-edge gradient (backward)

@@ -23,9 +23,12 @@ namespace umd {
 namespace {
 
 struct Grid {
-    double L[3];        // cell edge lengths
-    double lo[3];       // binning origin
-    double inv_cw[3];   // 1 / bin width
+    double L[3];        // cell edge lengths (orthorhombic cells)
+    double H[9];        // cell vectors as rows; H[3 k + k] = L[k] for an orthorhombic cell
+    double Hinv[9];     // inverse of H (general cells): fractional coordinates f = r Hinv
+    int tri;            // general cell: fold and bin in fractional coordinates
+    double lo[3];       // binning origin (Cartesian; fractional when tri)
+    double inv_cw[3];   // 1 / bin width (per unit of the binning coordinate)
     int nc[3];          // bins per direction
     int m[3];           // bin reach per direction
     int pbc[3];
@@ -52,6 +55,8 @@ __device__ __forceinline__ int pack_shift(int nx, int ny, int nz) {
     return (nx & 0xff) | ((ny & 0xff) << 8) | ((nz & 0xff) << 16);
 }
 
+struct CellRows { double h[9]; int tri; };
+
 // fold positions into the cell, bin them
 __global__ void k_fold_bin(int N, const double* __restrict__ pos, Grid g, double* __restrict__ wpos,
                            int* __restrict__ img_o, int* __restrict__ key, int* __restrict__ idx,
@@ -60,7 +65,27 @@ __global__ void k_fold_bin(int N, const double* __restrict__ pos, Grid g, double
     if (i >= N) return;
     int c[3];
     bool bad = false;
-    for (int k = 0; k < 3; ++k) {
+    if (g.tri) {
+        // general cell: f = r Hinv, fold by whole cell vectors along periodic directions (the same
+        // arithmetic k_gather_positions applies later), bin by the folded fractional coordinate
+        const double x = pos[3 * (size_t)i], y = pos[3 * (size_t)i + 1], z = pos[3 * (size_t)i + 2];
+        if (!isfinite(x) || !isfinite(y) || !isfinite(z)) bad = true;
+        double f[3], fl[3];
+        for (int k = 0; k < 3; ++k) {
+            f[k] = x * g.Hinv[k] + y * g.Hinv[3 + k] + z * g.Hinv[6 + k];
+            fl[k] = g.pbc[k] ? floor(f[k]) : 0.0;
+            if (fabs(fl[k]) > 1.0e6) bad = true;
+            img_o[3 * (size_t)i + k] = bad ? 0 : (int)fl[k];
+        }
+        for (int k = 0; k < 3; ++k) {
+            const double r = k == 0 ? x : (k == 1 ? y : z);
+            wpos[3 * (size_t)i + k] = r - ((fl[0] * g.H[k] + fl[1] * g.H[3 + k]) + fl[2] * g.H[6 + k]);
+            int ck = (int)floor(((f[k] - fl[k]) - g.lo[k]) * g.inv_cw[k]);
+            ck = ck < 0 ? 0 : (ck >= g.nc[k] ? g.nc[k] - 1 : ck);
+            c[k] = ck;
+        }
+    }
+    for (int k = 0; k < 3 && !g.tri; ++k) {
         const double x = pos[3 * (size_t)i + k];
         if (!isfinite(x)) bad = true;
         double w = x;
@@ -140,21 +165,26 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
         int zc = cz + dz, nz = 0;
         if (g.pbc[2]) { nz = floor_div(zc, g.nc[2]); zc -= nz * g.nc[2]; }
         else if (zc < 0 || zc >= g.nc[2]) continue;
-        const double sz = __dmul_rn((double)nz, g.L[2]);
+        // shift vector n . H, built up one cell vector per loop level without fused multiply-add;
+        // for an orthorhombic cell all but one term of each component are exact zeros
+        const double szx = __dmul_rn((double)nz, g.H[6]), szy = __dmul_rn((double)nz, g.H[7]),
+                     szz = __dmul_rn((double)nz, g.H[8]);
         for (int ty = 0; ty < wy; ++ty) {
             int dy = sy0 + ty;
             if (dy > g.m[1]) dy -= wy;
             int yc = cy + dy, ny = 0;
             if (g.pbc[1]) { ny = floor_div(yc, g.nc[1]); yc -= ny * g.nc[1]; }
             else if (yc < 0 || yc >= g.nc[1]) continue;
-            const double sy = __dmul_rn((double)ny, g.L[1]);
+            const double syx = __dadd_rn(szx, __dmul_rn((double)ny, g.H[3])), syy = __dadd_rn(szy, __dmul_rn((double)ny, g.H[4])),
+                         syz = __dadd_rn(szz, __dmul_rn((double)ny, g.H[5]));
             for (int tx = 0; tx < wx; ++tx) {
                 int dx = sx0 + tx;
                 if (dx > g.m[0]) dx -= wx;
                 int xc = cx + dx, nx = 0;
                 if (g.pbc[0]) { nx = floor_div(xc, g.nc[0]); xc -= nx * g.nc[0]; }
                 else if (xc < 0 || xc >= g.nc[0]) continue;
-                const double sx = __dmul_rn((double)nx, g.L[0]);
+                const double sx = __dadd_rn(syx, __dmul_rn((double)nx, g.H[0])), sy = __dadd_rn(syy, __dmul_rn((double)nx, g.H[1])),
+                             sz = __dadd_rn(syz, __dmul_rn((double)nx, g.H[2]));
                 const int cell = (zc * g.nc[1] + yc) * g.nc[0] + xc;
                 const int beg = cell_start[cell], end = cell_start[cell + 1];
                 const bool self_img = (nx == 0 && ny == 0 && nz == 0);
@@ -225,16 +255,17 @@ __global__ void k_reverse_map(int N, int sorted, const eidx_t* __restrict__ row_
 
 __global__ void k_gather_positions(int N, const int* __restrict__ perm, const int* __restrict__ img,
                                    const double* __restrict__ pos, const double* __restrict__ xs0,
-                                   double Lx, double Ly, double Lz, double max_disp2,
+                                   CellRows H, double max_disp2,
                                    double* __restrict__ xs, int* __restrict__ err) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const int o = perm[i];
-    const double L[3] = {Lx, Ly, Lz};
+    const double n0 = (double)img[3 * (size_t)i], n1 = (double)img[3 * (size_t)i + 1], n2 = (double)img[3 * (size_t)i + 2];
     double d2 = 0;
     bool bad = false;
     for (int k = 0; k < 3; ++k) {
-        const double x = pos[3 * (size_t)o + k] - (double)img[3 * (size_t)i + k] * L[k];
+        const double x = H.tri ? pos[3 * (size_t)o + k] - ((n0 * H.h[k] + n1 * H.h[3 + k]) + n2 * H.h[6 + k])
+                               : pos[3 * (size_t)o + k] - (double)img[3 * (size_t)i + k] * H.h[4 * k];
         if (!isfinite(x)) bad = true;
         xs[3 * (size_t)i + k] = x;
         const double d = x - xs0[3 * (size_t)i + k];
@@ -297,32 +328,58 @@ void neighbor_free(NeighborDev* nb) {
 }
 
 int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int32_t* d_type,
-                   const double L[3], const int pbc[3], double skin, double rc, int* d_err,
+                   const double cell[9], const int pbc[3], double skin, double rc, int* d_err,
                    cudaStream_t st, std::string* err) {
     if (N64 > 0x7fff0000LL) { *err = "too many atoms for 32-bit indices"; return UMLMD_E_INVALID_ARG; }
     const int N = (int)N64;
     const double r_list = rc + skin;
     Grid g;
+    const double L[3] = {cell[0], cell[4], cell[8]};
+    g.tri = 0;
+    for (int k = 0; k < 9; ++k) { g.H[k] = cell[k]; g.Hinv[k] = 0; if (k % 4 != 0 && cell[k] != 0.0) g.tri = 1; }
+    // perpendicular height of the cell along each cell vector (the edge length when orthorhombic)
+    double height[3] = {L[0], L[1], L[2]};
+    if (g.tri) {
+        const double* h = cell;
+        const double c00 = h[4] * h[8] - h[5] * h[7], c01 = h[5] * h[6] - h[3] * h[8], c02 = h[3] * h[7] - h[4] * h[6];
+        const double det = h[0] * c00 + h[1] * c01 + h[2] * c02;
+        const double scale = std::fabs(h[0]) + std::fabs(h[1]) + std::fabs(h[2]) + std::fabs(h[3]) + std::fabs(h[4]) +
+                             std::fabs(h[5]) + std::fabs(h[6]) + std::fabs(h[7]) + std::fabs(h[8]);
+        if (!(std::fabs(det) > 1e-12 * scale * scale * scale)) { *err = "singular cell"; return UMLMD_E_UNSUPPORTED_CELL; }
+        const double id = 1.0 / det;
+        g.Hinv[0] = c00 * id; g.Hinv[3] = c01 * id; g.Hinv[6] = c02 * id;
+        g.Hinv[1] = (h[2] * h[7] - h[1] * h[8]) * id; g.Hinv[4] = (h[0] * h[8] - h[2] * h[6]) * id; g.Hinv[7] = (h[1] * h[6] - h[0] * h[7]) * id;
+        g.Hinv[2] = (h[1] * h[5] - h[2] * h[4]) * id; g.Hinv[5] = (h[2] * h[3] - h[0] * h[5]) * id; g.Hinv[8] = (h[0] * h[4] - h[1] * h[3]) * id;
+        for (int k = 0; k < 3; ++k)     // f_k = r . column k of Hinv: planes of constant f_k are 1 / |column| apart
+            height[k] = 1.0 / std::sqrt(g.Hinv[k] * g.Hinv[k] + g.Hinv[3 + k] * g.Hinv[3 + k] + g.Hinv[6 + k] * g.Hinv[6 + k]);
+    }
     // per-direction bounding interval for non-periodic directions (host reduction of a
     // device min/max would cost a sync as well; the list build synchronises anyway)
-    double lo[3] = {0, 0, 0}, ext[3] = {L[0], L[1], L[2]};
+    // binning coordinate: Cartesian for an orthorhombic cell, fractional for a general one; `ext` is
+    // the extent along it, `unit` the perpendicular length of one unit of it
+    double lo[3] = {0, 0, 0}, ext[3] = {L[0], L[1], L[2]}, unit[3] = {1, 1, 1};
+    if (g.tri) for (int k = 0; k < 3; ++k) { ext[k] = 1.0; unit[k] = height[k]; }
     if (!(pbc[0] && pbc[1] && pbc[2]) && N > 0) {
         std::vector<double> hp((size_t)N * 3);
         NB_CHECK(cudaMemcpyAsync(hp.data(), d_pos, sizeof(double) * 3 * (size_t)N, cudaMemcpyDeviceToHost, st));
         NB_CHECK(cudaStreamSynchronize(st));
         for (int k = 0; k < 3; ++k) {
             if (pbc[k]) continue;
-            double mn = hp[k], mx = hp[k];
-            for (int i = 1; i < N; ++i) { const double v = hp[3 * (size_t)i + k]; if (v < mn) mn = v; if (v > mx) mx = v; }
+            auto coord = [&](int i) {
+                const double* r = &hp[3 * (size_t)i];
+                return g.tri ? r[0] * g.Hinv[k] + r[1] * g.Hinv[3 + k] + r[2] * g.Hinv[6 + k] : r[k];
+            };
+            double mn = coord(0), mx = mn;
+            for (int i = 1; i < N; ++i) { const double v = coord(i); if (v < mn) mn = v; if (v > mx) mx = v; }
             if (!std::isfinite(mn) || !std::isfinite(mx)) { *err = "non-finite position"; return UMLMD_E_NONFINITE; }
-            lo[k] = mn; ext[k] = (mx - mn) + 1e-6;
+            lo[k] = mn; ext[k] = (mx - mn) + 1e-6 / unit[k];
         }
     }
     int64_t ncell = 1;
     const double rl_pad = r_list * (1.0 + 1e-9) + 1e-12;
     for (int k = 0; k < 3; ++k) {
         g.L[k] = L[k]; g.lo[k] = lo[k]; g.pbc[k] = pbc[k] ? 1 : 0;
-        int nc = (int)std::floor(ext[k] / rl_pad);
+        int nc = (int)std::floor(ext[k] * unit[k] / rl_pad);
         if (nc < 1) nc = 1;
         if (nc > 1024) nc = 1024;
         g.nc[k] = nc;
@@ -337,7 +394,7 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     for (int k = 0; k < 3; ++k) {
         const double cw = ext[k] / g.nc[k];
         g.inv_cw[k] = 1.0 / cw;
-        g.m[k] = pbc[k] || g.nc[k] > 1 ? (int)std::ceil(r_list / cw) : 0;
+        g.m[k] = pbc[k] || g.nc[k] > 1 ? (int)std::ceil(r_list / (cw * unit[k])) : 0;
         if (!pbc[k] && g.m[k] > g.nc[k] - 1) g.m[k] = g.nc[k] - 1;
         if (g.m[k] > 127) { *err = "cell much smaller than the list radius (more than 127 images)"; return UMLMD_E_UNSUPPORTED_CELL; }
         ncell *= g.nc[k];
@@ -348,6 +405,8 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
 
     nb->N = N; nb->skin = skin; nb->r_list = r_list;
     for (int k = 0; k < 3; ++k) { nb->L[k] = L[k]; nb->pbc[k] = pbc[k] ? 1 : 0; }
+    for (int k = 0; k < 9; ++k) nb->H[k] = cell[k];
+    nb->tri = g.tri;
     if (N == 0) { nb->E = 0; return UMLMD_OK; }
 
     // per-atom arrays (all sized from one capacity)
@@ -449,8 +508,10 @@ cudaError_t launch_gather_positions(const NeighborDev& nb, const double* d_pos, 
     const double half = 0.5 * nb.skin;
     // a tiny slack keeps a fresh build with zero skin from tripping on its own rounding
     const double max_disp2 = half * half + 1e-20;
-    k_gather_positions<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, nb.img, d_pos, nb.xs0, nb.L[0], nb.L[1],
-                                                        nb.L[2], max_disp2, nb.xs, d_err);
+    CellRows H;
+    for (int k = 0; k < 9; ++k) H.h[k] = nb.H[k];
+    H.tri = nb.tri;
+    k_gather_positions<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, nb.img, d_pos, nb.xs0, H, max_disp2, nb.xs, d_err);
     return cudaGetLastError();
 }
 

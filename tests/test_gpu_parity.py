@@ -358,3 +358,66 @@ def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
     d2 = (a["atom_energy"] - outs[1]["atom_energy"]).abs().max().item()
     d3 = (a["atom_energy"] - outs[2]["atom_energy"]).abs().max().item()
     print(f"max|dE_i| vs CUDA-core path: path 2 {d2 / e_scale:.2e}, path 3 {d3 / e_scale:.2e} of max|E_i|")
+
+
+# ------------------------------------------------------------------ general (triclinic) cells
+
+def _sheared(desc, tilt, flip=False):
+    """The random box of `desc` mapped into a general cell: same fractional coordinates, cell rows
+    a = (ex, 0, 0), b = (t0 ey, ey, 0), c = (t1 ez, t2 ez, ez); `flip` swaps two rows (left-handed)."""
+    s = make_system(desc)
+    e = np.diag(np.asarray(s["cell"], dtype=np.float64))
+    cell = np.array([[e[0], 0.0, 0.0], [tilt[0] * e[1], e[1], 0.0], [tilt[1] * e[2], tilt[2] * e[2], e[2]]])
+    frac = s["pos"] / e
+    if flip:
+        cell, frac = cell[[1, 0, 2]], frac[:, [1, 0, 2]]
+        s["pbc"] = [s["pbc"][1], s["pbc"][0], s["pbc"][2]]
+    s["pos"] = frac @ cell
+    s["cell"] = cell.tolist()
+    return s
+
+
+TRI = [
+    (dict(kind="random_box", atoms=14, edges=(9.0, 13.0, 12.5), min_dist=1.4, seed=52, n_types=1, masses=[1.0], shift=True), (0.3, -0.2, 0.25), False),
+    (dict(kind="random_box", atoms=8, edges=(4.1, 14.0, 7.3), min_dist=1.4, seed=53, n_types=1, masses=[1.0]), (0.45, 0.1, -0.35), False),
+    (dict(kind="random_box", atoms=300, edges=(21.0, 22.5, 30.0), min_dist=1.6, seed=57, n_types=1, masses=[1.0], shift=True), (-0.4, 0.3, 0.2), False),
+    (dict(kind="random_box", atoms=30, edges=(20.0, 7.0, 9.0), min_dist=1.6, seed=56, n_types=1, masses=[1.0], pbc=[0, 1, 1]), (0.2, 0.2, -0.3), False),
+    (dict(kind="random_box", atoms=40, edges=(14.5, 12.1, 19.0), min_dist=1.4, seed=54, n_types=1, masses=[1.0]), (0.25, 0.15, 0.3), True),
+]
+
+
+@pytest.mark.parametrize("case", range(len(TRI)))
+@pytest.mark.parametrize("skin", [0.0, 1.0])
+def test_neighbor_lists_in_general_cells(case, skin):
+    desc, tilt, flip = TRI[case]
+    s = _sheared(desc, tilt, flip)
+    blob = make_blob(SMALL_PROFILES["p8_2_0"], seed=1)
+    m, _ = _build(blob, s, skin=skin)
+    got = _rows_from_gpu(m, len(s["pos"]))
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    ref = orc.neighbor_rows(pos, s["cell"], s["pbc"], 6.0 + skin)
+    assert m.query()["n_edges"] == sum(len(r) for r in ref)
+    for a, b in zip(got, ref):
+        assert np.array_equal(a, b)
+    m.close()
+
+
+@pytest.mark.parametrize("name,case", [("p16_3_2", 0), ("p32_2_4", 1), ("p32_3_2", 2), ("p8_2_0", 3), ("p16_2_0", 4)])
+def test_parity_in_general_cells(name, case):
+    p = SMALL_PROFILES[name]
+    desc, tilt, flip = TRI[case]
+    blob = make_blob(p, seed=48, bias_scale=0.2)
+    s = _sheared(dict(desc, n_types=p["T"], masses=[1.0] * p["T"]), tilt, flip)
+    _compare(blob, s, skin=0.5 * (case % 2))
+
+
+def test_singular_cell_is_refused():
+    p = SMALL_PROFILES["p8_2_0"]
+    blob = make_blob(p, seed=1)
+    s = make_system(dict(SYS_SMALL, n_types=p["T"]))
+    m, pos = _build(blob, s)
+    bad = [[9.5, 0.0, 0.0], [19.0, 0.0, 0.0], [0.0, 0.0, 12.0]]
+    with pytest.raises(_binding().UmlmdError) as e:
+        m.build_neighbors(pos, _dev(s["types"], torch.int32), bad, s["pbc"], 0.0)
+    assert e.value.code == -4
+    m.close()
