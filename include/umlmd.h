@@ -196,6 +196,19 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
                    double t_damp_ps, double* e_pot, double* e_kin, double* e_conserved);
 
 /*
+ * Per-atom virial of the last evaluation that produced forces or the virial (umlmd_compute with
+ * d_force or virial given, or umlmd_step / umlmd_step_nvt): every directed edge e = (i <- j, n)
+ * with gradient g_e = dE/dr_ij and vector r_e shares -g_e (x) r_e equally between its two atoms,
+ *   W_k = -1/2 sum over the edges with k as centre or as neighbour of g_e (x) r_e,
+ * so that sum_k W_k is the virial umlmd_compute returns (the paper lists atomic virials as an
+ * optional per-atom output without fixing the split; this is the usual half-and-half one).
+ *   d_atom_virial [N, 9] double, row-major 3 x 3 per atom (component [a][b] = force-like index a,
+ *   vector index b), caller's numbering, eV.
+ * UMLMD_E_INVALID_ARG if no such evaluation has run since the last build.
+ */
+int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial);
+
+/*
  * Diagnostics used by the parity tests: copy out per-atom intermediates of the last
  * umlmd_compute, in the caller's numbering.  Each pointer may be NULL.
  *   d_state  [N, S+2] float: unnormalised sums A (degree, then m, then channel), s0, s1

@@ -535,6 +535,17 @@ class Oracle:
         return dict(E=float(Ei.sum()), E_i=Ei, F=F, virial=virial, rows=rows, n_edges=len(dst),
                     D_raw=Dt, g=g, dst=dst, src=src, rij=rij)
 
+    def atom_virials(self, res):
+        """Per-atom shares [N,3,3] of the virial from a `compute` result.  READING (the paper names
+        atomic virials as an optional output but not the split): each directed edge gives half of
+        -g_e (x) r_e to its centre and half to its neighbour."""
+        N = len(res["E_i"])
+        contrib = -0.5 * res["g"][:, :, None] * res["rij"][:, None, :]
+        W = np.zeros((N, 3, 3))
+        np.add.at(W, res["dst"], contrib)
+        np.add.at(W, res["src"], contrib)
+        return W
+
     def force_on(self, pos, types, cell, pbc, k):
         """Force on a single atom k of a large system: needs the rows of k and of every
         atom that has k as a neighbour (the same atoms, the list being symmetric)."""

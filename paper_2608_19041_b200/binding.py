@@ -23,7 +23,7 @@ ERRORS = {
 EXPORTS = [
     "umlmd_profile_widths", "umlmd_create", "umlmd_destroy", "umlmd_query", "umlmd_last_error",
     "umlmd_build_neighbors", "umlmd_get_neighbors", "umlmd_compute", "umlmd_set_md_state", "umlmd_step",
-    "umlmd_step_nvt",
+    "umlmd_step_nvt", "umlmd_atom_virial",
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
     "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
 ]
@@ -69,6 +69,7 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_step.argtypes = [vp, ctypes.c_int, dbl, ctypes.c_int, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.umlmd_step_nvt.argtypes = [vp, ctypes.c_int, dbl, ctypes.c_int, dbl, dbl, ctypes.POINTER(dbl), ctypes.POINTER(dbl),
                                    ctypes.POINTER(dbl)]
+    lib.umlmd_atom_virial.argtypes = [vp, vp]
     lib.umlmd_get_intermediates.argtypes = [vp, vp, vp]
     lib.umlmd_eval_radial_table.argtypes = [vp, i64, ctypes.POINTER(dbl), ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.umlmd_eval_pair_cache.argtypes = [vp, i32, i32, ctypes.POINTER(dbl)]
@@ -179,6 +180,14 @@ class Model:
         if rc != OK:
             self._raise(rc)
         return row_ptr, src[:E], shift[:E]
+
+    def atom_virial(self):
+        """[N, 3, 3] CUDA tensor: per-atom shares of the virial of the last evaluation with forces."""
+        out = torch.empty((max(self.n_atoms, 1), 3, 3), dtype=torch.float64, device="cuda")
+        rc = self._lib.umlmd_atom_virial(self._h, _ptr(out))
+        if rc != OK:
+            self._raise(rc)
+        return out[:self.n_atoms]
 
     def compute(self, pos, forces=True, virial=True, atom_energy=False):
         """Returns dict(energy=float, forces=CUDA tensor or None, virial=np [3,3] or None,

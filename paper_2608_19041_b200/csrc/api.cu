@@ -42,6 +42,7 @@ struct umlmd {
     double* md_pos = nullptr; double* md_vel = nullptr; double* md_force = nullptr; int64_t md_cap = 0;
     double* d_mass = nullptr; double* d_inv_mass = nullptr;
     bool have_md = false, have_force = false;
+    bool have_edge_grad = false;     // h->g holds the edge gradients of the positions in nb.xs
     int steps_since_build = 0;
     double* d_nhc = nullptr;      // thermostat chain on the device: eta[M], v_eta[M], scale, kinetic energy
     bool nhc_reset = true;
@@ -197,6 +198,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
             vpart_used += blocks;
         }
     }
+    h->have_edge_grad = want_grad;
     if (want_grad) {
         Scope sc(h, kForce, 1);
         API_CUDA(h, launch_force_assembly(nb, h->g, d_force ? nullptr : h->f_sorted, d_force, h->d_err, h->st));
@@ -257,6 +259,7 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
     { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, d_pos, d_type, cell, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
     h->have_list = true;
+    h->have_edge_grad = false;       // edges were renumbered
     h->steps_since_build = 0;
     return ensure_workspace(h);
 }
@@ -573,6 +576,16 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
         for (int k = 1; k < M; ++k) e += p.kT * chain[k];
         *e_conserved = e;
     }
+    return UMLMD_OK;
+}
+
+int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
+    if (!h->have_edge_grad) return fail(h, UMLMD_E_INVALID_ARG, "no evaluation with forces or virial since the last build");
+    if (h->nb.N > 0 && !d_atom_virial) return fail(h, UMLMD_E_INVALID_ARG, "null output buffer");
+    { Scope sc(h, kForce, 1); API_CUDA(h, launch_atom_virial(h->nb, h->g, d_atom_virial, h->st)); }
+    API_CUDA(h, cudaStreamSynchronize(h->st));
     return UMLMD_OK;
 }
 

@@ -48,6 +48,52 @@ __global__ void k_force_rows(int N, const eidx_t* __restrict__ row_ptr, const ei
     }
 }
 
+// Per-atom share of the virial, one warp per atom over its own row: every directed edge gives half
+// of -g_e (x) r_e to its centre and half to its neighbour, so atom i collects
+// -1/2 sum_{e in row(i)} (g_e - g_rev(e)) (x) r_e (the reverse edge has the opposite vector).
+// Edge vectors are recomputed in double from the positions of the last evaluation.
+struct CellRowsA { double h[9]; };
+__global__ void k_atom_virial(int N, const eidx_t* __restrict__ row_ptr, const int* __restrict__ src,
+                              const int* __restrict__ shift, const eidx_t* __restrict__ rev,
+                              const float* __restrict__ g, const double* __restrict__ xs, CellRowsA H,
+                              const int* __restrict__ perm, double* __restrict__ out) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const eidx_t e0 = row_ptr[warp];
+    const int len = (int)(row_ptr[warp + 1] - e0);
+    const double xi = xs[3 * (size_t)warp], yi = xs[3 * (size_t)warp + 1], zi = xs[3 * (size_t)warp + 2];
+    double w[9];
+#pragma unroll
+    for (int k = 0; k < 9; ++k) w[k] = 0.0;
+    for (int k = lane; k < len; k += 32) {
+        const eidx_t e = e0 + k;
+        const float* a = g + 3 * (size_t)e;
+        double d[3] = {(double)a[0], (double)a[1], (double)a[2]};
+        const eidx_t r = rev[e];
+        if (r >= 0) { const float* b = g + 3 * (size_t)r; d[0] -= (double)b[0]; d[1] -= (double)b[1]; d[2] -= (double)b[2]; }
+        const int j = src[e], s = shift[e];
+        const double nx = (double)(signed char)(s & 0xff), ny = (double)(signed char)((s >> 8) & 0xff),
+                     nz = (double)(signed char)((s >> 16) & 0xff);
+        const double* xj = xs + 3 * (size_t)j;
+        const double rx = (xj[0] + ((nx * H.h[0] + ny * H.h[3]) + nz * H.h[6])) - xi;
+        const double ry = (xj[1] + ((nx * H.h[1] + ny * H.h[4]) + nz * H.h[7])) - yi;
+        const double rz = (xj[2] + ((nx * H.h[2] + ny * H.h[5]) + nz * H.h[8])) - zi;
+#pragma unroll
+        for (int p = 0; p < 3; ++p) { w[3 * p] += d[p] * rx; w[3 * p + 1] += d[p] * ry; w[3 * p + 2] += d[p] * rz; }
+    }
+#pragma unroll
+    for (int k = 0; k < 9; ++k) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) w[k] += __shfl_xor_sync(0xffffffffu, w[k], off);
+    }
+    if (lane < 9) {
+        double v = 0.0;
+#pragma unroll
+        for (int k = 0; k < 9; ++k) if (lane == k) v = w[k];
+        out[9 * (size_t)perm[warp] + lane] = -0.5 * v;
+    }
+}
+
 __global__ void k_scatter3(int N, const int* __restrict__ perm, const double* __restrict__ in,
                            double* __restrict__ out, int* __restrict__ err) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -232,6 +278,15 @@ cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double*
     const int N = (int)nb.N;
     if (N == 0) return cudaSuccess;
     k_force_rows<<<(N + 7) / 8, 256, 0, st>>>(N, nb.row_ptr, nb.rev, g, f_sorted, nb.perm, d_force, d_err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_atom_virial(const NeighborDev& nb, const float* g, double* d_out, cudaStream_t st) {
+    const int N = (int)nb.N;
+    if (N == 0) return cudaSuccess;
+    CellRowsA H;
+    for (int k = 0; k < 9; ++k) H.h[k] = nb.H[k];
+    k_atom_virial<<<(N + 7) / 8, 256, 0, st>>>(N, nb.row_ptr, nb.src, nb.shift, nb.rev, g, nb.xs, H, nb.perm, d_out);
     return cudaGetLastError();
 }
 

@@ -98,6 +98,9 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a 
 cudaError_t launch_species_present(int64_t N, const int* type, int T, int* d_flags, int* d_err, cudaStream_t st);
 cudaError_t launch_force_assembly(const NeighborDev& nb, const float* g, double* d_force_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
+// per-atom virial shares [N][9] in the caller's numbering from the edge gradients of the last
+// backward pass: W_i = -1/2 sum over the edges that touch atom i of g_e (x) r_e
+cudaError_t launch_atom_virial(const NeighborDev& nb, const float* g, double* d_out, cudaStream_t st);
 cudaError_t launch_scatter_forces(const NeighborDev& nb, const double* f_sorted, double* d_force,
                                   int* d_err, cudaStream_t st);
 cudaError_t launch_scatter_atom_energy(const NeighborDev& nb, const double* e_sorted, double* d_out,

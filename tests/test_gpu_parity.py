@@ -421,3 +421,27 @@ def test_singular_cell_is_refused():
         m.build_neighbors(pos, _dev(s["types"], torch.int32), bad, s["pbc"], 0.0)
     assert e.value.code == -4
     m.close()
+
+
+@pytest.mark.parametrize("general_cell", [False, True])
+def test_atom_virials(general_cell):
+    p = SMALL_PROFILES["p32_3_2"]
+    blob = make_blob(p, seed=49, bias_scale=0.2)
+    desc = dict(SYS_SMALL, n_types=p["T"])
+    s = _sheared(desc, (0.3, -0.2, 0.25)) if general_cell else make_system(desc)
+    o = orc.Oracle(blob)
+    ref = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    Wref = o.atom_virials(ref)
+    m, pos = _build(blob, s, skin=0.7)
+    with pytest.raises(_binding().UmlmdError):
+        m.atom_virial()                            # nothing evaluated yet
+    out = m.compute(pos)
+    W = m.atom_virial().cpu().numpy()
+    scale = max(np.abs(Wref).max(), 1e-12)
+    assert np.abs(W - Wref).max() <= 2e-5 * scale
+    # the total is accumulated from single-precision products in the edge kernel
+    assert np.abs(W.sum(axis=0) - out["virial"]).max() <= 1e-5 * np.abs(out["virial"]).max() + 1e-5 * scale
+    m.compute(pos, forces=False, virial=False)     # an energy-only evaluation leaves no edge gradients
+    with pytest.raises(_binding().UmlmdError):
+        m.atom_virial()
+    m.close()

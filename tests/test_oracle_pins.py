@@ -543,3 +543,21 @@ def test_force_on_single_atom_matches_whole_system():
     Fk, Ei = o.force_on(s["pos"], s["types"], s["cell"], s["pbc"], 4)
     assert np.abs(Fk - out["F"][4]).max() < 1e-12 * max(1.0, np.abs(out["F"]).max())
     assert abs(Ei[4] - out["E_i"][4]) < 1e-13 * max(1.0, abs(out["E_i"][4]))
+
+
+def test_atom_virials_sum_to_the_virial_and_split_a_dimer_evenly():
+    p = SMALL_PROFILES["p8_2_0"]
+    o = orc.Oracle(make_blob(p, seed=9))
+    s = make_system(dict(kind="random_box", atoms=20, edges=(7.5, 8.0, 9.0), min_dist=1.6, seed=4, n_types=p["T"],
+                         masses=[1.0] * p["T"]))
+    res = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])
+    W = o.atom_virials(res)
+    assert np.allclose(W.sum(axis=0), res["virial"], rtol=0, atol=1e-12 * max(1.0, np.abs(res["virial"]).max()))
+    # an isolated pair of equal atoms: the two shares are equal, and each is -1/2 of the sum over
+    # both directed edges; with F the force on atom 1 and d = r_1 - r_0 the virial is F (x) d
+    pos = np.array([[10.0, 10.0, 10.0], [11.1, 10.4, 9.3]])
+    big = [[40.0, 0, 0], [0, 40.0, 0], [0, 0, 40.0]]
+    r2 = o.compute(pos, np.zeros(2, dtype=np.int64), big, (0, 0, 0))
+    W2 = o.atom_virials(r2)
+    assert np.allclose(W2[0], W2[1], rtol=1e-12, atol=1e-15)
+    assert np.allclose(W2[0] + W2[1], np.outer(r2["F"][1], pos[1] - pos[0]), rtol=1e-10, atol=1e-14)
