@@ -1,7 +1,9 @@
 /*
  * umlmd.h -- C ABI of libumlmd: energy, force and virial evaluation of the DPA4C
- * machine-learning interatomic potential on one NVIDIA B200 (sm_100a), plus a
- * velocity-Verlet NVE driver.
+ * machine-learning interatomic potential on one NVIDIA B200 (sm_100a) over a cutoff neighbor
+ * list that the library builds itself (orthorhombic or general cells, any mix of periodic
+ * directions), plus velocity-Verlet NVE and Nose-Hoover-chain NVT drivers and per-atom
+ * energies and virials.
  *
  * Conventions
  *   - Every function returns an int status: UMLMD_OK (0) or a negative UMLMD_E_* code.
