@@ -91,8 +91,9 @@ int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out);
  *   {Theta_t[F,F], b_t[F]} t = 2..n_hidden, w_head[F], b_head, E_ref[T].
  * The create step evaluates, once and in double precision on the host, everything the
  * paper's compressed inference precomputes: the Hermite radial table of the shared radial
- * map and modes on [0, rc] (the cubic through value and first derivative at each knot; the
- * paper stores the quintic that also matches the second derivative), the
+ * map and modes on [0, rc] (the cubic through value and first derivative at each knot, its
+ * quadratic and cubic coefficients stored as 20- and 12-bit fixed-point numbers on the
+ * table's own scale; the paper stores the quintic that also matches the second derivative), the
  * ordered type-pair scale / shift / mode-mixing cache, and the unit-norm Gaunt coupling
  * tensors of the admissible degree triples.
  *   stream: a cudaStream_t passed as void* (NULL = the default stream).
@@ -125,7 +126,7 @@ const char* umlmd_last_error(const umlmd_t* h);
  * reproducible bit for bit.  Atoms are renumbered internally in cell order; all outputs
  * of this library are in the caller's numbering.
  * The call also finds which species occur.  When the P species present are few enough that
- * P^2 tables of table_rows x 4 x C0 floats fit in umlmd_options.pair_table_mb, the edge
+ * P^2 tables of table_rows x 3 x C0 words fit in umlmd_options.pair_table_mb, the edge
  * amplitude of every ordered pair (s, s') among them, psi_c(rho) = gamma_c g_c(rho) + beta_c +
  * sum_mu U_c,mu q_mu(rho), is tabulated as a cubic table of its own (the same linear
  * combination of the coefficient rows of the radial table), and umlmd_compute reads one row of

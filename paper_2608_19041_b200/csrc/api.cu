@@ -35,7 +35,8 @@ struct umlmd {
     int64_t pair_table_budget = 192ll << 20;            // bytes; negative = never build them
     bool pair_tables = false;                           // in use for the current system
     std::vector<int> present;                           // species the tables were built for, ascending
-    float* table_uni = nullptr; size_t table_uni_cap = 0;   // [present^2][n_rows][4][C0], capacity in floats
+    float* table_uni = nullptr; size_t table_uni_cap = 0;   // [present^2][n_rows][3][C0], capacity in floats
+    float* uni_scale = nullptr;                         // [2] largest |c2|, |c3| of those tables
     int* d_species = nullptr;                           // [3T]: occurrence flags, species -> slot, present list
     int* h_species = nullptr;                           // pinned [T]
     // MD
@@ -164,6 +165,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         EdgeArgs ea;
         ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.type_s = nb.type_s;
         ea.table_uni = h->pair_tables ? h->table_uni : nullptr;
+        ea.uni_scale = h->uni_scale;
         ea.species_slot = h->d_species + d.T; ea.n_present = (int)h->present.size();
         ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
@@ -272,7 +274,7 @@ int setup_pair_tables(umlmd_t* h) {
     std::vector<int> present;
     for (int t = 0; t < d.T; ++t) if (h->h_species[t]) present.push_back(t);
     const size_t np = present.size();
-    const size_t floats = np * np * (size_t)d.n_rows * 4 * d.C0;
+    const size_t floats = np * np * (size_t)d.n_rows * 3 * d.C0;
     h->pair_tables = np > 0 && h->pair_table_budget >= 0 && floats * sizeof(float) <= (size_t)h->pair_table_budget;
     if (!h->pair_tables || present == h->present) return UMLMD_OK;
     if (floats > h->table_uni_cap) {
@@ -284,9 +286,10 @@ int setup_pair_tables(umlmd_t* h) {
     std::vector<int> up(2 * (size_t)d.T, 0);          // species -> slot, then the present list
     for (size_t k = 0; k < np; ++k) { up[present[k]] = (int)k; up[d.T + k] = present[k]; }
     API_CUDA(h, cudaMemcpyAsync(h->d_species + d.T, up.data(), sizeof(int) * up.size(), cudaMemcpyHostToDevice, h->st));
-    API_CUDA(h, launch_fuse_pair_tables(d, h->md.table, h->md.pairmod, h->d_species + 2 * d.T, (int)np, h->table_uni, h->st));
+    if (!h->uni_scale) { void* p = nullptr; API_CUDA(h, dev_malloc(&p, 4 * sizeof(float))); h->uni_scale = (float*)p; }
+    API_CUDA(h, launch_fuse_pair_tables(d, h->md.table, h->md.pairmod, h->d_species + 2 * d.T, (int)np, h->uni_scale, h->table_uni, h->st));
     API_CUDA(h, cudaStreamSynchronize(h->st));       // `up` is pageable host memory
-    h->launches_total += 1;
+    h->launches_total += 2;
     h->present = present;
     return UMLMD_OK;
 }
@@ -332,7 +335,7 @@ int umlmd_destroy(umlmd_t* h) {
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
     void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
-                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni, h->d_species};
+                    h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni, h->d_species, h->uni_scale};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
@@ -608,9 +611,13 @@ int umlmd_eval_radial_table(const umlmd_t* h, int64_t n, const double* rho, doub
         if (row < 0) row = 0;
         if (row > d.n_rows - 1) row = d.n_rows - 1;
         const double t = rho[i] - row * h->hm.dx;
-        const float* p = &h->hm.table[(size_t)row * 4 * d.CP];
+        const float* p = &h->hm.table[(size_t)row * 3 * d.CP];
         for (int c = 0; c < NC; ++c) {
-            const double c0 = p[c], c1 = p[d.CP + c], c2 = p[2 * d.CP + c], c3 = p[3 * d.CP + c];
+            unsigned w;
+            std::memcpy(&w, &p[2 * d.CP + c], sizeof(w));
+            float h2, h3;
+            tab_unpack(w, d.tab_k2, d.tab_k3, &h2, &h3);
+            const double c0 = p[c], c1 = p[d.CP + c], c2 = h2, c3 = h3;
             out_g[i * NC + c] = ((c3 * t + c2) * t + c1) * t + c0;
             if (out_dg) out_dg[i * NC + c] = (3 * c3 * t + 2 * c2) * t + c1;
         }

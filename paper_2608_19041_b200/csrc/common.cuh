@@ -38,6 +38,7 @@ struct Dims {
     int H, Hp;
     int CP;                  // table channels C0+R rounded up to 4
     int n_rows;              // table intervals
+    float tab_k2, tab_k3;    // steps of the packed quadratic and cubic coefficients of the radial table
     float rc, dx, inv_dx;
 };
 
@@ -49,7 +50,7 @@ struct GauntSparse {         // non-zeros of one unit-norm coupling tensor
 
 // Device-resident constants of one model.
 struct ModelDev {
-    float* table;     // [n_rows][4][CP] cubic Hermite coefficients c0..c3 of [g, q]
+    float* table;     // [n_rows][3][CP] cubic Hermite pieces of [g, q]: c0, c1 (fp32), packed (c2, c3)
     float* pairmod;   // [T*T][2+R][C0]: scale gamma, shift beta, mode mixing U[:, mu]
     float* X0;        // [T][C0]
     float* W1p;       // [C1][C1]  I + W_1
@@ -76,6 +77,27 @@ struct Handle;  // defined in api.cu
 // ---- launchers (each enqueues on `st`; none synchronises) ---------------------------
 
 typedef long long eidx_t;      // edge offsets are 64-bit: a list may hold more than 2^31 edges
+
+// Packed high-order coefficients of a cubic table piece.  c2 and c3 only enter through c2 t^2 and
+// c3 t^3 with t below the table spacing, so a 20-bit and a 12-bit fixed-point number on the table's
+// own scale (c2 = k2 I2, c3 = k3 I3; k = largest magnitude in the table / largest integer) cost
+// nothing in the value and leave the derivative within a few 1e-7 of its largest entry at the
+// default spacing (the error grows with the spacing like the interpolation error itself).
+// One 32-bit word: I2 in the upper 20 bits, I3 in the lower 12, both two's complement.
+constexpr int kTabI2Max = (1 << 19) - 1, kTabI3Max = (1 << 11) - 1;
+__host__ __device__ inline float tab_step2(float max_abs_c2) { return max_abs_c2 * (1.0f / (float)kTabI2Max); }
+__host__ __device__ inline float tab_step3(float max_abs_c3) { return max_abs_c3 * (1.0f / (float)kTabI3Max); }
+__host__ __device__ inline unsigned tab_pack(float c2, float c3, float k2, float k3) {
+    float q2 = k2 > 0.f ? c2 / k2 : 0.f, q3 = k3 > 0.f ? c3 / k3 : 0.f;
+    q2 = q2 > (float)kTabI2Max ? (float)kTabI2Max : (q2 < -(float)kTabI2Max ? -(float)kTabI2Max : q2);
+    q3 = q3 > (float)kTabI3Max ? (float)kTabI3Max : (q3 < -(float)kTabI3Max ? -(float)kTabI3Max : q3);
+    const int i2 = (int)(q2 < 0.f ? q2 - 0.5f : q2 + 0.5f), i3 = (int)(q3 < 0.f ? q3 - 0.5f : q3 + 0.5f);
+    return ((unsigned)i2 << 12) | ((unsigned)i3 & 0xfffu);
+}
+__host__ __device__ inline void tab_unpack(unsigned w, float k2, float k3, float* c2, float* c3) {
+    *c2 = k2 * (float)((int)w >> 12);
+    *c3 = k3 * (float)((int)(w << 20) >> 20);
+}
 
 struct NeighborDev {
     int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;

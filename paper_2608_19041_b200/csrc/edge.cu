@@ -125,26 +125,35 @@ __device__ __forceinline__ void harmonics_grad_contract(float x, float y, float 
     *gx = ax; *gy = ay; *gz = az;
 }
 
-// value (and derivative) of four consecutive table channels at offset t in row `row`
+// value (and derivative) of four consecutive table channels at offset t in row `row`: three
+// 16-byte loads, c0, c1 and the packed (c2, c3) words with steps k2, k3 (common.cuh, tab_pack)
 template <bool DERIV>
 __device__ __forceinline__ void table_eval4(const float* __restrict__ table, int CP, int row, int c, float t,
-                                            float* v, float* dv) {
-    const float* p = table + (size_t)row * 4 * CP + c;
-    const float4 c0 = ldg4(p), c1 = ldg4(p + CP), c2 = ldg4(p + 2 * CP), c3 = ldg4(p + 3 * CP);
-#define UMLMD_HORNER(k, f)                                                                             \
-    v[k] = ((c3.f * t + c2.f) * t + c1.f) * t + c0.f;                                                  \
-    if (DERIV) dv[k] = (3.0f * c3.f * t + 2.0f * c2.f) * t + c1.f;
-    UMLMD_HORNER(0, x) UMLMD_HORNER(1, y) UMLMD_HORNER(2, z) UMLMD_HORNER(3, w)
-#undef UMLMD_HORNER
+                                            float k2, float k3, float* v, float* dv) {
+    const float* p = table + (size_t)row * 3 * CP + c;
+    const float4 c0 = ldg4(p), c1 = ldg4(p + CP);
+    const int4 w = __ldg(reinterpret_cast<const int4*>(p + 2 * CP));
+    const float u2 = k2 * t * t, u3 = k3 * t * t * t;           // c2 t^2 = I2 u2, c3 t^3 = I3 u3
+    const float v2 = 2.0f * k2 * t, v3 = 3.0f * k3 * t * t;
+#define UMLMD_PIECE(k, f)                                                                              \
+    {                                                                                                  \
+        const float i2 = (float)(w.f >> 12), i3 = (float)((w.f << 20) >> 20);                          \
+        v[k] = fmaf(i3, u3, fmaf(i2, u2, fmaf(c1.f, t, c0.f)));                                        \
+        if (DERIV) dv[k] = fmaf(i3, v3, fmaf(i2, v2, c1.f));                                           \
+    }
+    UMLMD_PIECE(0, x) UMLMD_PIECE(1, y) UMLMD_PIECE(2, z) UMLMD_PIECE(3, w)
+#undef UMLMD_PIECE
 }
 
 template <bool DERIV>
 __device__ __forceinline__ void table_eval1(const float* __restrict__ table, int CP, int row, int c, float t,
-                                            float* v, float* dv) {
-    const float* p = table + (size_t)row * 4 * CP + c;
-    const float c0 = __ldg(p), c1 = __ldg(p + CP), c2 = __ldg(p + 2 * CP), c3 = __ldg(p + 3 * CP);
-    *v = ((c3 * t + c2) * t + c1) * t + c0;
-    if (DERIV) *dv = (3.0f * c3 * t + 2.0f * c2) * t + c1;
+                                            float k2, float k3, float* v, float* dv) {
+    const float* p = table + (size_t)row * 3 * CP + c;
+    const float c0 = __ldg(p), c1 = __ldg(p + CP);
+    const int w = __ldg(reinterpret_cast<const int*>(p + 2 * CP));
+    const float i2 = (float)(w >> 12), i3 = (float)((w << 20) >> 20);
+    *v = fmaf(i3, k3 * t * t * t, fmaf(i2, k2 * t * t, fmaf(c1, t, c0)));
+    if (DERIV) *dv = fmaf(i3, 3.0f * k3 * t * t, fmaf(i2, 2.0f * k2 * t, c1));
 }
 
 // Shared radial modes q_mu(rho) (and derivatives) of the first nb queued edges, one (edge, mode)
@@ -157,7 +166,7 @@ __device__ __forceinline__ void eval_modes(const EdgeArgs& a, const int4* qes, i
         const int b = idx / R, q = idx - b * R;
         const int4 es = qes[b];
         float qv, dqv = 0.f;
-        table_eval1<DERIV>(a.table, a.d.CP, es.x, a.d.C0 + q, __int_as_float(es.z), &qv, &dqv);
+        table_eval1<DERIV>(a.table, a.d.CP, es.x, a.d.C0 + q, __int_as_float(es.z), a.d.tab_k2, a.d.tab_k3, &qv, &dqv);
         qm[b * kMaxR + q] = qv;
         if (DERIV) dqm[b * kMaxR + q] = dqv;
     }
@@ -166,16 +175,17 @@ __device__ __forceinline__ void eval_modes(const EdgeArgs& a, const int4* qes, i
 // amplitude psi (and d psi / d rho) of this lane's four channels for one edge; qm / dqm: the
 // edge's parked radial modes (only read when HASR).  UNI: psi_c(rho) of every ordered pair of
 // species present is tabulated by itself (a.table_uni, row pitch C0; `row` already points into
-// the edge's pair), so neither pair rows nor modes are read
+// the edge's pair), so neither pair rows nor modes are read.  k2, k3: steps of the packed
+// coefficients of the table that is read
 template <int C0, bool HASR, bool DERIV, bool UNI>
 __device__ __forceinline__ void amplitude4(const EdgeArgs& a, int row, float t, int pair, int c, float* psi,
-                                           float* dpsi, const float* qm, const float* dqm) {
+                                           float* dpsi, const float* qm, const float* dqm, float k2, float k3) {
     if (UNI) {
-        table_eval4<DERIV>(a.table_uni, C0, row, c, t, psi, dpsi);
+        table_eval4<DERIV>(a.table_uni, C0, row, c, t, k2, k3, psi, dpsi);
         return;
     }
     float g[4], dg[4];
-    table_eval4<DERIV>(a.table, a.d.CP, row, c, t, g, dg);
+    table_eval4<DERIV>(a.table, a.d.CP, row, c, t, k2, k3, g, dg);
     const int R = HASR ? a.d.R : 0;
     const float* pm = a.pairmod + (size_t)pair * (2 + R) * C0 + c;
     const float4 ga = ldg4(pm), be = ldg4(pm + C0);
@@ -271,6 +281,7 @@ k_edge_forward(const EdgeArgs a) {
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
     const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
     const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
+    const float k2 = UNI ? tab_step2(__ldg(a.uni_scale)) : a.d.tab_k2, k3 = UNI ? tab_step3(__ldg(a.uni_scale + 1)) : a.d.tab_k3;
     const eidx_t e0 = a.row_ptr[i];
     const int len = (int)(a.row_ptr[i + 1] - e0);      // edge offsets are 64-bit, offsets inside a row are not
     const unsigned lt_mask = (1u << lane) - 1u;
@@ -292,8 +303,8 @@ k_edge_forward(const EdgeArgs a) {
             for (; it + 1 < nb; it += 2) {
                 const int4 ea = qes[it], eb = qes[it + 1];
                 float pa[4], pb[4];
-                amplitude4<C0, HASR, false, UNI>(a, ea.x, __int_as_float(ea.z), ea.y, c, pa, nullptr, nullptr, nullptr);
-                amplitude4<C0, HASR, false, UNI>(a, eb.x, __int_as_float(eb.z), eb.y, c, pb, nullptr, nullptr, nullptr);
+                amplitude4<C0, HASR, false, UNI>(a, ea.x, __int_as_float(ea.z), ea.y, c, pa, nullptr, nullptr, nullptr, k2, k3);
+                amplitude4<C0, HASR, false, UNI>(a, eb.x, __int_as_float(eb.z), eb.y, c, pb, nullptr, nullptr, nullptr, k2, k3);
                 const float ca = __int_as_float(ea.w), cb = __int_as_float(eb.w);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) acc0[k] += ca * pa[k];
@@ -312,7 +323,7 @@ k_edge_forward(const EdgeArgs a) {
             const int row = es.x, pair = es.y;
             const float t = __int_as_float(es.z), chi = __int_as_float(es.w);
             float psi[4];
-            amplitude4<C0, HASR, false, UNI>(a, row, t, pair, c, psi, nullptr, qm + b * kMaxR, nullptr);
+            amplitude4<C0, HASR, false, UNI>(a, row, t, pair, c, psi, nullptr, qm + b * kMaxR, nullptr, k2, k3);
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc0[k] += chi * psi[k];
             if (cl < W::NL1)
@@ -459,6 +470,7 @@ k_edge_backward(const EdgeArgs a) {
     if (active) {
         const double xi = a.xs[3 * (size_t)i], yi = a.xs[3 * (size_t)i + 1], zi = a.xs[3 * (size_t)i + 2];
         const int ti = UNI ? a.species_slot[a.type_s[i]] : a.type_s[i];
+        const float k2 = UNI ? tab_step2(__ldg(a.uni_scale)) : a.d.tab_k2, k3 = UNI ? tab_step3(__ldg(a.uni_scale + 1)) : a.d.tab_k3;
         const eidx_t e0 = a.row_ptr[i];
         const int len = (int)(a.row_ptr[i + 1] - e0);
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
@@ -492,7 +504,7 @@ k_edge_backward(const EdgeArgs a) {
 #pragma unroll
                     for (int gq = 0; gq < G; ++gq)
                         amplitude4<C0, HASR, true, UNI>(a, row, t, pair, c + gq * W::GOFF, psi + 4 * gq, dpsi + 4 * gq,
-                                                        qm + b * kMaxR, qm + (32 + b) * kMaxR);
+                                                        qm + b * kMaxR, qm + (32 + b) * kMaxR, k2, k3);
 #pragma unroll
                     for (int k = 0; k < 4 * G; ++k) { pa += h0[k] * dpsi[k]; pb += h0[k] * psi[k]; }
                     if (cl < W::NL1) {       // the leading C1 channels all sit in group 0
@@ -654,34 +666,72 @@ cudaError_t dispatch(const EdgeArgs& a, int blocks, cudaStream_t st) {
 }
 
 // Tables of psi_c(rho) = gamma_c g_c(rho) + beta_c + sum_mu U_c,mu q_mu(rho) for the ordered
-// pairs (present[a], present[b]), stored as [a * n_present + b][row][k][c]: the cubic
-// coefficients are linear in the tabulated functions, so the same combination of the
-// coefficient rows of [g, q] gives them exactly.
+// pairs (present[a], present[b]), stored as [a * n_present + b][row][3][C0] in the format of the
+// radial table: the cubic coefficients are linear in the tabulated functions, so the same
+// combination of the coefficient rows of [g, q] gives them.  Two passes: the first finds the
+// largest |c2| and |c3| (the scale of the packed words), the second writes the rows.
+template <bool WRITE>
 __global__ void k_fuse_pair_tables(Dims d, const float* __restrict__ table, const float* __restrict__ pairmod,
-                                   const int* __restrict__ present, int n_present, float* __restrict__ out) {
-    const int64_t per_pair = (int64_t)d.n_rows * 4 * d.C0;
-    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;   // over [pair][row][k][c]
-    if (idx >= per_pair * n_present * n_present) return;
-    const int pr = (int)(idx / per_pair);
-    const int64_t in_pair = idx - pr * per_pair;
-    const int c = (int)(in_pair % d.C0);
-    const int64_t rk = in_pair / d.C0;          // row * 4 + k
-    const int si = present[pr / n_present], sj = present[pr % n_present];
-    const float* pm = pairmod + (size_t)(si * d.T + sj) * (2 + d.R) * d.C0 + c;
-    const float* tr = table + (size_t)rk * d.CP;
-    double v = (double)pm[0] * (double)tr[c];
-    if ((rk & 3) == 0) v += (double)pm[d.C0];
-    for (int q = 0; q < d.R; ++q) v += (double)pm[(size_t)(2 + q) * d.C0] * (double)tr[d.C0 + q];
-    out[idx] = (float)v;
+                                   const int* __restrict__ present, int n_present, float* __restrict__ scale,
+                                   float* __restrict__ out) {
+    const int64_t per_pair = (int64_t)d.n_rows * d.C0;
+    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;   // over [pair][row][c]
+    float c2 = 0.f, c3 = 0.f;
+    if (idx < per_pair * n_present * n_present) {
+        const int pr = (int)(idx / per_pair);
+        const int64_t in_pair = idx - pr * per_pair;
+        const int c = (int)(in_pair % d.C0);
+        const int64_t row = in_pair / d.C0;
+        const int si = present[pr / n_present], sj = present[pr % n_present];
+        const float* pm = pairmod + (size_t)(si * d.T + sj) * (2 + d.R) * d.C0 + c;
+        const float* tr = table + (size_t)row * 3 * d.CP;
+        auto coef = [&](int col, double* o) {     // the four coefficients of column col of the radial table
+            float h2, h3;
+            tab_unpack(__float_as_uint(tr[2 * d.CP + col]), d.tab_k2, d.tab_k3, &h2, &h3);
+            o[0] = (double)tr[col]; o[1] = (double)tr[d.CP + col]; o[2] = (double)h2; o[3] = (double)h3;
+        };
+        double v[4], o[4];
+        coef(c, o);
+        for (int k = 0; k < 4; ++k) v[k] = (double)pm[0] * o[k];
+        v[0] += (double)pm[d.C0];
+        for (int q = 0; q < d.R; ++q) {
+            coef(d.C0 + q, o);
+            const double u = (double)pm[(size_t)(2 + q) * d.C0];
+            for (int k = 0; k < 4; ++k) v[k] += u * o[k];
+        }
+        c2 = (float)v[2]; c3 = (float)v[3];
+        if (WRITE) {
+            float* orow = out + ((size_t)pr * d.n_rows + row) * 3 * d.C0;
+            orow[c] = (float)v[0];
+            orow[d.C0 + c] = (float)v[1];
+            orow[2 * d.C0 + c] = __uint_as_float(tab_pack(c2, c3, tab_step2(scale[0]), tab_step3(scale[1])));
+        }
+    }
+    if (!WRITE) {        // non-negative floats order like their bit patterns
+        float a2 = fabsf(c2), a3 = fabsf(c3);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            a2 = fmaxf(a2, __shfl_xor_sync(0xffffffffu, a2, off));
+            a3 = fmaxf(a3, __shfl_xor_sync(0xffffffffu, a3, off));
+        }
+        if ((threadIdx.x & 31) == 0) {
+            atomicMax(reinterpret_cast<unsigned*>(scale), __float_as_uint(a2));
+            atomicMax(reinterpret_cast<unsigned*>(scale) + 1, __float_as_uint(a3));
+        }
+    }
 }
 
 }  // namespace
 
 cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
-                                    int n_present, float* out, cudaStream_t st) {
-    const int64_t n = (int64_t)d.n_rows * 4 * d.C0 * n_present * n_present;
+                                    int n_present, float* scale, float* out, cudaStream_t st) {
+    const int64_t n = (int64_t)d.n_rows * d.C0 * n_present * n_present;
     if (n == 0) return cudaSuccess;
-    k_fuse_pair_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(d, table, pairmod, present, n_present, out);
+    cudaError_t e = cudaMemsetAsync(scale, 0, 2 * sizeof(float), st);
+    if (e != cudaSuccess) return e;
+    const unsigned blocks = (unsigned)((n + 255) / 256);
+    k_fuse_pair_tables<false><<<blocks, 256, 0, st>>>(d, table, pairmod, present, n_present, scale, out);
+    k_fuse_pair_tables<true><<<blocks, 256, 0, st>>>(d, table, pairmod, present, n_present, scale, out);
     return cudaGetLastError();
 }
 

@@ -39,15 +39,17 @@ struct EdgeArgs {
     float* g;               // [E][3] per-edge gradient (backward)
     double* virial_part;    // [blocks][9] partial virial sums (backward)
     // non-null when the species present are few enough for per-pair amplitude tables:
-    // [n_present^2][n_rows][4][C0] cubic coefficients of psi_c(rho) of each ordered pair
-    // (launch_fuse_pair_tables), read instead of table, pairmod and the radial modes
+    // [n_present^2][n_rows][3][C0] cubic pieces of psi_c(rho) of each ordered pair, in the format
+    // of the radial table (launch_fuse_pair_tables), read instead of table, pairmod and the radial
+    // modes; uni_scale[0..1] = largest |c2|, |c3| of these tables (scale of their packed words)
     const float* table_uni;
+    const float* uni_scale;
     const int* species_slot;    // [T] species -> index among the species present
     int n_present;
 };
 // present: device array of the n_present species indices, ascending
 cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
-                                    int n_present, float* out, cudaStream_t st);
+                                    int n_present, float* scale, float* out, cudaStream_t st);
 cudaError_t launch_edge_forward(const EdgeArgs& a, cudaStream_t st);
 cudaError_t launch_edge_backward(const EdgeArgs& a, int* n_blocks, cudaStream_t st);
 int edge_backward_blocks(int n_rows_in_tile);

@@ -269,23 +269,34 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
             }
         }
     }
-    m->table.assign((size_t)n_rows * 4 * CP, 0.0f);
+    m->table.assign((size_t)n_rows * 3 * CP, 0.0f);
     {
-        // p(t) = c0 + c1 t + c2 t^2 + c3 t^3, t = rho - rho_s, matching value and slope at both knots
+        // p(t) = c0 + c1 t + c2 t^2 + c3 t^3, t = rho - rho_s, matching value and slope at both knots;
+        // c2 and c3 are stored packed on the table's own scale (common.cuh, tab_pack)
         const double D1 = m->dx, D2 = D1 * D1, D3 = D2 * D1;
+        std::vector<float> hi((size_t)n_rows * 2 * NC);
+        float m2 = 0.f, m3 = 0.f;
         for (int s = 0; s < n_rows; ++s) {
             const double* ya = &Y[(size_t)s * 2 * NC];
             const double* yb = &Y[(size_t)(s + 1) * 2 * NC];
-            float* row = &m->table[(size_t)s * 4 * CP];
+            float* row = &m->table[(size_t)s * 3 * CP];
             for (int c = 0; c < NC; ++c) {
                 const double y0 = ya[c], p0 = ya[NC + c], y1 = yb[c], p1 = yb[NC + c];
                 const double del = y1 - y0;
                 row[0 * CP + c] = (float)y0;
                 row[1 * CP + c] = (float)p0;
-                row[2 * CP + c] = (float)((3 * del - (2 * p0 + p1) * D1) / D2);
-                row[3 * CP + c] = (float)((-2 * del + (p0 + p1) * D1) / D3);
+                const float c2 = (float)((3 * del - (2 * p0 + p1) * D1) / D2), c3 = (float)((-2 * del + (p0 + p1) * D1) / D3);
+                hi[((size_t)s * NC + c) * 2] = c2; hi[((size_t)s * NC + c) * 2 + 1] = c3;
+                if (std::fabs(c2) > m2) m2 = std::fabs(c2);
+                if (std::fabs(c3) > m3) m3 = std::fabs(c3);
             }
         }
+        d.tab_k2 = tab_step2(m2); d.tab_k3 = tab_step3(m3);
+        for (int s = 0; s < n_rows; ++s)
+            for (int c = 0; c < NC; ++c) {
+                const unsigned w = tab_pack(hi[((size_t)s * NC + c) * 2], hi[((size_t)s * NC + c) * 2 + 1], d.tab_k2, d.tab_k3);
+                std::memcpy(&m->table[(size_t)s * 3 * CP + 2 * CP + c], &w, sizeof(w));
+            }
     }
 
     // ---- ordered type-pair cache -----------------------------------------------------

@@ -13,7 +13,7 @@ namespace umd {
 struct HostModel {
     Dims d;
     double rc = 0, dx = 0;
-    std::vector<float> table;      // [n_rows][4][CP]
+    std::vector<float> table;      // [n_rows][3][CP]: c0, c1, packed (c2, c3) (see tab_pack)
     std::vector<float> pairmod;    // [T*T][2+R][C0]
     std::vector<float> X0, W1p, W2p, A1, A2, mu, inv_sigma;
     std::vector<std::vector<float>> theta, thetaT, bias;   // per hidden layer
