@@ -304,6 +304,33 @@ def test_neighbor_rows_match_kdtree_counts():
     assert (np.array([len(r) for r in rows]) == counts).all()
 
 
+@pytest.mark.parametrize("pbc", [(1, 1, 1), (1, 0, 1)])
+def test_general_cell_rows_match_plain_loops_and_a_rotated_box_keeps_its_energy(pbc):
+    # a sheared cell against plain loops over images, and a rigidly rotated orthorhombic box (its
+    # cell matrix is then full) against the unrotated one: same edge multiset, same energies
+    s = make_system(dict(kind="random_box", atoms=10, edges=(6.0, 7.5, 8.0), min_dist=1.4, seed=31, n_types=1,
+                         masses=[1.0], shift=True, pbc=list(pbc)))
+    e = np.diag(np.asarray(s["cell"], dtype=np.float64))
+    cell = np.array([[e[0], 0.0, 0.0], [0.3 * e[1], e[1], 0.0], [-0.2 * e[2], 0.25 * e[2], e[2]]])
+    pos = orc.wrap_positions((s["pos"] / e) @ cell, cell, pbc)
+    frac = pos @ np.linalg.inv(cell)
+    per = np.asarray(pbc, bool)
+    assert (frac[:, per] > -1e-12).all() and (frac[:, per] < 1 + 1e-12).all()
+    rows = orc.neighbor_rows(pos, cell, pbc, 6.0)
+    ref = _python_neighbors(pos, cell, pbc, 6.0)
+    for a, b in zip(rows, ref):
+        assert [tuple(x) for x in a.tolist()] == b
+
+    o, s2 = _small_case(n=16, edges=(6.5, 7.0, 8.2), seed=33, pbc=pbc)
+    base = o.compute(s2["pos"], s2["types"], s2["cell"], pbc)
+    Rm = _random_rotation(8)
+    rot = o.compute(s2["pos"] @ Rm.T, s2["types"], np.asarray(s2["cell"]) @ Rm.T, pbc)
+    assert rot["n_edges"] == base["n_edges"]
+    assert np.allclose(rot["E_i"], base["E_i"], rtol=1e-11, atol=1e-13)
+    assert np.allclose(rot["F"], base["F"] @ Rm.T, rtol=1e-9, atol=1e-12)
+    assert np.allclose(rot["virial"], Rm @ base["virial"] @ Rm.T, rtol=1e-9, atol=1e-11)
+
+
 def test_non_periodic_cluster_has_no_images():
     s = make_system(dict(kind="random_box", atoms=12, edges=(6.0, 6.0, 6.0), min_dist=1.5, seed=13,
                          n_types=1, masses=[1.0], pbc=[0, 0, 0]))
