@@ -346,7 +346,8 @@ def run_ours(args):
     dom = dict(kernels[0]) if kernels else None
     if dom:
         dom["peak_source"] = peaks["source"]
-        dom["traffic"] = load_traffic(args.workload, dom["kernel"])
+        tile = args.node_tile if args.node_tile > 0 else DEFAULT_NODE_TILE
+        dom["traffic"] = load_traffic(args.workload, dom["kernel"], N / max(1, -(-N // tile)))
 
     # ---- end to end from host buffers: upload positions, evaluate, download forces
     k_e2e = max(1, min(args.steps, 10))
@@ -404,10 +405,17 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def load_traffic(workload, kernel):
+CAPTURE_ATOMS = 131072          # size of the box the stored ncu capture ran on
+DEFAULT_NODE_TILE = 524288       # the library's default workspace tile (atoms per launch of the tiled kernels)
+
+
+def load_traffic(workload, kernel, atoms_per_launch):
     """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of one kernel class on
     one workload, from the stored summary of an ncu capture: lines "workload class bytes" in
-    profiles/dram_traffic_per_launch.txt.  None when no capture is stored."""
+    profiles/dram_traffic_per_launch.txt hold the bytes of one launch over CAPTURE_ATOMS atoms of
+    the same recipe; the traffic of these kernels is proportional to the atoms (and their edges)
+    a launch covers, so it is scaled to the launch size of the timed run.  None when no capture
+    is stored."""
     path = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")
     if not os.path.exists(path):
         return None
@@ -415,7 +423,7 @@ def load_traffic(workload, kernel):
         for ln in f:
             w = ln.split()
             if len(w) >= 3 and not ln.startswith("#") and w[0] == workload and w[1] == kernel:
-                return float(w[2])
+                return float(w[2]) * atoms_per_launch / CAPTURE_ATOMS
     return None
 
 

@@ -56,7 +56,7 @@ enum {
 typedef struct umlmd_options {
     uint32_t struct_bytes;
     double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
-    int32_t  node_tile;  /* atoms per workspace tile; 0 = 131072                            */
+    int32_t  node_tile;  /* atoms per workspace tile; 0 = 524288                            */
     int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM, persistent, 3 = tcgen05 3xTF32 GEMM, one tile per CTA */
     int32_t  pair_table_mb;  /* device memory, MiB, that per-pair amplitude tables may take
                                 (see umlmd_build_neighbors); 0 = 192, negative = never build them */
@@ -216,7 +216,7 @@ int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial);
  * umlmd_compute, in the caller's numbering.  Each pointer may be NULL.
  *   d_state  [N, S+2] float: unnormalised sums A (degree, then m, then channel), s0, s1
  *   d_desc   [N, D_out] float: calibrated feature vector D
- * Only valid when N <= node tile (single-tile evaluation); otherwise UMLMD_E_CAPACITY.
+ * Only valid for a single-tile evaluation of fewer than 65536 atoms; otherwise UMLMD_E_CAPACITY.
  * These hold forward values only if umlmd_compute was called with d_force == NULL and
  * virial == NULL (the backward pass reuses both buffers).
  */

@@ -17,7 +17,7 @@ struct umlmd {
     cudaStream_t st = nullptr;
     std::string err;
     NeighborDev nb;
-    int node_tile = 131072;
+    int node_tile = 524288;
     int mlp_path = 2;   // tensor-core GEMM wherever it applies, CUDA-core GEMM otherwise
     bool have_list = false;
     bool on_device = false;
@@ -113,6 +113,11 @@ void fill_info(const Dims& d, umlmd_info* o) {
     o->H = d.H; o->H_pair = d.Hp; o->table_rows = d.n_rows;
 }
 
+// the fp32 feature rows and the state of a small single-tile system stay readable after an
+// evaluation (umlmd_get_intermediates); larger systems skip the copy nothing else reads
+constexpr int64_t kIntermediatesMaxAtoms = 65536;
+bool keeps_intermediates(const umlmd_t* h) { return h->nb.N < kIntermediatesMaxAtoms && h->nb.N <= h->node_tile; }
+
 int ensure_workspace(umlmd_t* h) {
     const Dims& d = h->d;
     const int64_t N = h->nb.N, E = h->nb.E;
@@ -182,7 +187,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         // system smaller than one node tile)
         const bool presplit = h->mlp_path >= 2 && gemm_tc_available();
         ia.desc_hi = presplit ? h->tc_hi : nullptr; ia.desc_lo = presplit ? h->tc_lo : nullptr;
-        ia.write_desc = !presplit || d.D_out == d.F || N < h->node_tile;
+        ia.write_desc = !presplit || d.D_out == d.F || keeps_intermediates(h);
         const bool fold_x0 = presplit && d.D_out != d.F;      // first GEMM skips the per-species constant columns
         ia.skip_x0_split = fold_x0;
         { Scope sc(h, kInvFwd, 1); API_CUDA(h, launch_invariants_forward(ia, h->st)); }
@@ -595,7 +600,7 @@ int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial) {
 int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc) {
     if (!h) return UMLMD_E_INVALID_ARG;
     if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "no neighbor list built");
-    if (h->nb.N >= h->node_tile) return fail(h, UMLMD_E_CAPACITY, "intermediates are only kept for systems smaller than one node tile");
+    if (!keeps_intermediates(h)) return fail(h, UMLMD_E_CAPACITY, "intermediates are only kept for systems of one tile and fewer than 65536 atoms");
     if (d_state) API_CUDA(h, launch_unsort_state(h->nb, h->state, h->d.SP, h->d.S + 2, d_state, h->st));
     if (d_desc) API_CUDA(h, launch_unsort_state(h->nb, h->desc, h->d.DP, h->d.D_out, d_desc, h->st));
     API_CUDA(h, cudaStreamSynchronize(h->st));
