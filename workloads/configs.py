@@ -134,6 +134,11 @@ SMALL_PROFILES = {
                         Hp=176, S=76, D_out=144),
     "p32_3_2": _profile(32, 3, 2, 16, 2, 64, 3, C1=8, C2=4, K1=4, K2=2, H=88,
                         Hp=176, S=83, D_out=155),
+    # the widest set of shared radial modes, at a narrow and at a wide scalar width
+    "p16_2_8": _profile(16, 2, 8, 8, 2, 48, 3, C1=4, C2=4, K1=4, K2=2, H=48,
+                        Hp=88, S=48, D_out=86),
+    "p64_3_8": _profile(64, 3, 8, 16, 2, 96, 2, C1=8, C2=4, K1=4, K2=2, H=176,
+                        Hp=344, S=115, D_out=219),
     # D_out == F: the first MLP layer carries the identity residual
     "p32_2_0_res": _profile(32, 2, 0, 8, 2, 144, 2, C1=8, C2=4, K1=4, K2=2, H=88,
                             Hp=176, S=76, D_out=144),
