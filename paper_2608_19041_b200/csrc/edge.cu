@@ -233,10 +233,12 @@ template <int C0, int L, int G = 1> struct Widths {
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
 };
 
-// the backward pass keeps two channel groups per lane from C0 = 32 up: twice as many table and
-// pair loads are in flight per lane, which is what this latency-bound phase lacks at two blocks
-// per SM (measured: 3 % at C0 = 128, 11 % at C0 = 32)
-template <int C0> struct BwdGroups { static constexpr int G = C0 >= 32 ? 2 : 1; };
+// the backward pass keeps several channel groups per lane (four from C0 = 64 up, two at C0 = 32):
+// that many times the table and pair loads are in flight per lane, which is what this
+// latency-bound phase lacks at two blocks per SM (measured: edge backward 10 % faster with four
+// groups than with two at C0 = 128 and 64, 11 % faster with two than with one at C0 = 32, where
+// four are slower again)
+template <int C0> struct BwdGroups { static constexpr int G = C0 >= 64 ? 4 : (C0 >= 32 ? 2 : 1); };
 
 template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L, BwdGroups<C0>::G>;
