@@ -260,8 +260,11 @@ template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared 
 //   3. lane = edge again: harmonics and the chi^2 psi_c B_lm products of degree >= 1 for the
 //      lane's own edge, summed over the batch by a shared-memory transpose (32 values at a
 //      time), so that lane v ends up owning sums v, v+32, v+64 of the flattened block.
+// Up to C0 = 64 a fourth resident block per SM (64 registers, a few spilled words) is worth more
+// than the registers: the channel-parallel phase waits on load latency (measured: 6-10 % on the
+// forward kernel at C0 = 8 .. 64, 2 % the other way at C0 = 128, which stays at three blocks).
 template <int C0, int L, bool HASR, bool UNI>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, C0 <= 64 ? 4 : 3)
 k_edge_forward(const EdgeArgs a) {
     using W = Widths<C0, L>;
     // one 32 x 33 float scratch per warp: first the parked amplitudes (row pitch PF), then,
