@@ -233,12 +233,13 @@ template <int C0, int L, int G = 1> struct Widths {
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
 };
 
-// the backward pass keeps several channel groups per lane (four from C0 = 64 up, two at C0 = 32):
-// that many times the table and pair loads are in flight per lane, which is what this
-// latency-bound phase lacks at two blocks per SM (measured: edge backward 10 % faster with four
-// groups than with two at C0 = 128 and 64, 11 % faster with two than with one at C0 = 32, where
-// four are slower again)
-template <int C0> struct BwdGroups { static constexpr int G = C0 >= 64 ? 4 : (C0 >= 32 ? 2 : 1); };
+// The channel-parallel phase of the backward pass waits on load latency, and what hides it best
+// depends on the width (all measured on the edge backward kernel).  C0 = 128: four channel groups
+// per lane, that many times the table and pair loads in flight, at two resident blocks per SM (128
+// registers): 10 % faster than two groups, and than two groups at three blocks.  C0 = 32 and 64:
+// two groups at three blocks (85 registers, a few spilled words): 9-13 % faster than two blocks,
+// four groups being slower again.  C0 <= 16: one group, three blocks (13 % faster than two).
+template <int C0> struct BwdGroups { static constexpr int G = C0 >= 128 ? 4 : (C0 >= 32 ? 2 : 1); };
 
 template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
     using W = Widths<C0, L, BwdGroups<C0>::G>;
@@ -450,7 +451,7 @@ k_edge_forward(const EdgeArgs a) {
 // destination's gradient block held in shared memory, and assembles dE/dr_ij.  Edges in the
 // skin shell get a zero gradient as soon as their geometry is known.
 template <int C0, int L, bool HASR, bool UNI>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, C0 <= 64 ? 3 : 2)
 k_edge_backward(const EdgeArgs a) {
     constexpr int G = BwdGroups<C0>::G;
     using W = Widths<C0, L, G>;
