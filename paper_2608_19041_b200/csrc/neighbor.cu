@@ -177,16 +177,28 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
             else if (yc < 0 || yc >= g.nc[1]) continue;
             const double syx = __dadd_rn(szx, __dmul_rn((double)ny, g.H[3])), syy = __dadd_rn(szy, __dmul_rn((double)ny, g.H[4])),
                          syz = __dadd_rn(szz, __dmul_rn((double)ny, g.H[5]));
-            for (int tx = 0; tx < wx; ++tx) {
+            for (int tx = 0, run = 1; tx < wx; tx += run) {
                 int dx = sx0 + tx;
                 if (dx > g.m[0]) dx -= wx;
                 int xc = cx + dx, nx = 0;
+                run = 1;
                 if (g.pbc[0]) { nx = floor_div(xc, g.nc[0]); xc -= nx * g.nc[0]; }
                 else if (xc < 0 || xc >= g.nc[0]) continue;
+                // bins that follow one another along x with the same image hold consecutive atoms:
+                // they are scanned as one range (same candidates in the same order, fuller warps)
+                while (g.sorted && tx + run < wx) {
+                    int dx2 = sx0 + tx + run;
+                    if (dx2 > g.m[0]) dx2 -= wx;
+                    int xc2 = cx + dx2, nx2 = 0;
+                    if (g.pbc[0]) { nx2 = floor_div(xc2, g.nc[0]); xc2 -= nx2 * g.nc[0]; }
+                    else if (xc2 < 0 || xc2 >= g.nc[0]) break;
+                    if (nx2 != nx || xc2 != xc + run) break;
+                    ++run;
+                }
                 const double sx = __dadd_rn(syx, __dmul_rn((double)nx, g.H[0])), sy = __dadd_rn(syy, __dmul_rn((double)nx, g.H[1])),
                              sz = __dadd_rn(syz, __dmul_rn((double)nx, g.H[2]));
                 const int cell = (zc * g.nc[1] + yc) * g.nc[0] + xc;
-                const int beg = cell_start[cell], end = cell_start[cell + 1];
+                const int beg = cell_start[cell], end = cell_start[cell + run];
                 const bool self_img = (nx == 0 && ny == 0 && nz == 0);
                 for (int b = beg; b < end; b += 32) {
                     const int j = b + lane;
