@@ -514,6 +514,158 @@ def test_pair_modulation_ranges_and_order():
     assert U.shape == (p["T"], p["T"], p["C0"], p["R"])
 
 
+def test_swiglu_gate_is_the_first_half_of_the_columns():
+    # Eq. "swiglu": [x_g, x_v] = x W, output SiLU(x_g) * x_v with the gate in the FIRST H columns.
+    # One input row, H = 2, every product written out by hand; swapping the halves would give
+    # SiLU(x_v) * x_g = (-0.5249791874789399 * ..., ...) instead.
+    x = torch.tensor([[0.5, -1.0, 2.0]], dtype=torch.float64)
+    W = torch.tensor([[1.0, -2.0, 0.5, 3.0],
+                      [0.0, 1.0, -1.0, 2.0],
+                      [0.25, 0.5, 1.5, -0.5]], dtype=torch.float64)
+    a_gate = np.array([0.5 * 1.0 + (-1.0) * 0.0 + 2.0 * 0.25, 0.5 * (-2.0) + (-1.0) * 1.0 + 2.0 * 0.5])   # 1.0, -1.0
+    a_val = np.array([0.5 * 0.5 + (-1.0) * (-1.0) + 2.0 * 1.5, 0.5 * 3.0 + (-1.0) * 2.0 + 2.0 * (-0.5)])  # 4.25, -1.5
+    expected = a_gate * scipy.special.expit(a_gate) * a_val
+    got = orc.swiglu(x, W).numpy()[0]
+    assert np.allclose(got, expected, rtol=1e-15, atol=0)
+    # the same numbers as decimals: SiLU(1) = 0.7310585786300049, SiLU(-1) = -0.2689414213699951
+    assert np.allclose(got, [0.7310585786300049 * 4.25, -0.2689414213699951 * -1.5], rtol=1e-14, atol=0)
+    swapped = a_val * scipy.special.expit(a_val) * a_gate
+    assert np.abs(got - swapped).max() > 0.5
+
+
+def test_pair_modulation_against_a_hand_built_network():
+    # Eq. "pairfilm" with C0 = 2, R = 1, T = 2 and weights chosen so that two hidden units carry
+    # everything: h0 = SiLU(X0_a[0]) X0_b[0] (gate reads the centre, value the neighbour) and
+    # h1 = SiLU(X0_b[1]) X0_a[1].  Then [s | t | w] = 0.1 (h0 row0 + h1 row1), gamma = 1 + tanh s,
+    # beta = X0_a + X0_b + tanh t, U = tanh w.  A missing 0.1, a different block order or the
+    # neighbour-first concatenation each change these numbers.
+    C0, R, T = 2, 1, 2
+    Hp = 8 * math.ceil(2 * C0 / 3)
+    X0 = np.array([[0.8, -0.3], [-1.2, 0.6]])
+    W_in = np.zeros((2 * C0, 2 * Hp))
+    W_in[0, 0] = 1.0            # gate 0 <- centre feature 0 (z = [X0_a, X0_b])
+    W_in[2, Hp + 0] = 1.0       # value 0 <- neighbour feature 0
+    W_in[3, 1] = 1.0            # gate 1 <- neighbour feature 1
+    W_in[1, Hp + 1] = 1.0       # value 1 <- centre feature 1
+    row0 = np.array([1.0, -2.0, 3.0, 0.5, -1.5, 2.5])
+    row1 = np.array([0.7, 1.1, -0.9, 2.0, 0.3, -0.6])
+    W_out = np.zeros((Hp, C0 * (2 + R)))
+    W_out[0], W_out[1] = row0, row1
+    prm = dict(X0=torch.from_numpy(X0), W_p_in=torch.from_numpy(W_in), W_p_out=torch.from_numpy(W_out))
+    gamma, beta, U = orc.pair_modulation(dict(T=T, C0=C0, R=R), prm)
+    assert U.shape == (T, T, C0, R)
+
+    def silu_(v):
+        return v * scipy.special.expit(v)
+
+    for a in range(T):
+        for b in range(T):
+            h0 = silu_(X0[a, 0]) * X0[b, 0]
+            h1 = silu_(X0[b, 1]) * X0[a, 1]
+            o = 0.1 * (h0 * row0 + h1 * row1)
+            assert np.allclose(gamma[a, b].numpy(), 1.0 + np.tanh(o[0:2]), rtol=1e-14, atol=0)
+            assert np.allclose(beta[a, b].numpy(), X0[a] + X0[b] + np.tanh(o[2:4]), rtol=1e-14, atol=0)
+            assert np.allclose(U[a, b, :, 0].numpy(), np.tanh(o[4:6]), rtol=1e-13, atol=0)
+    # one entry as plain decimals, centre species 0, neighbour species 1:
+    # h0 = SiLU(0.8)(-1.2) = -0.662381, h1 = SiLU(0.6)(-0.3) = -0.116218, s_0 = 0.1 (h0 + 0.7 h1) = -0.0743734
+    h0, h1 = -1.2 * 0.8 / (1 + math.exp(-0.8)), -0.3 * 0.6 / (1 + math.exp(-0.6))
+    assert abs(gamma[0, 1, 0].item() - (1 + math.tanh(0.1 * (h0 * 1.0 + h1 * 0.7)))) < 1e-15
+    assert abs(gamma[0, 1, 0].item() - 0.925764) < 1e-6
+    # ordered pairs: (0, 1) and (1, 0) differ
+    assert abs(gamma[0, 1, 0].item() - gamma[1, 0, 0].item()) > 1e-3
+
+
+def _beta_only_oracle(profile, seed):
+    """Oracle of a small profile with the learned radial map and the pair network's output layer
+    zeroed (psi = beta = X0_i + X0_j), no alignment (W_l = 0) and probes that select the leading
+    channels (A_l = leading columns of the identity)."""
+    p = SMALL_PROFILES[profile]
+    o = orc.Oracle(make_blob(p, seed=seed))
+    for k in ("W_out", "W_mode", "W_p_out", "W_1", "W_2", "A_1", "A_2"):
+        o.prm[k].zero_()
+    for l in (1, 2):
+        A = o.prm[f"A_{l}"]
+        for k in range(A.shape[1]):
+            A[k, k] = 1.0
+    with torch.no_grad():
+        o.pair = orc.pair_modulation(o.p, o.prm)
+    return p, o
+
+
+def test_higher_degree_gram_blocks_follow_the_addition_theorem():
+    # With psi = beta the degree-l moments are X_l[m, c] = sum_j chi_j^2 beta_jc B_lm(u_j) / M_1 for
+    # the LEADING C_l channels, and the addition theorem turns the Gram block into
+    #   G_l[c, c'] = sum_jk chi_j^2 chi_k^2 beta_jc beta_kc' P_l(u_j . u_k) / M_1^2,
+    # which needs only distances, directions and scipy's Legendre polynomials.  Pins the weight
+    # chi^2 for every l >= 1, the shared normaliser M_1, the leading-channel rule (C_2 < C_1 here)
+    # and the positions of vech(G_2), vech(G_3) in the feature vector.
+    p, o = _beta_only_oracle("p32_3_2", 52)
+    s = make_system(dict(kind="random_box", atoms=18, edges=(8.0, 8.5, 9.0), min_dist=1.6, seed=53,
+                         n_types=p["T"], masses=[1.0] * p["T"]))
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"], want_grad=False)
+    X0 = o.prm["X0"].numpy()
+    C0, Cs = p["C0"], {1: p["C1"], 2: p["C2"], 3: 1}
+    assert Cs[2] < Cs[1]
+    for i in (0, 6, 17):
+        sel = out["dst"] == i
+        d = np.sqrt((out["rij"][sel] ** 2).sum(1))
+        chi = 1.0 - scipy.special.betainc(5, 4, np.clip(d / p["rc"], 0, 1))
+        beta = X0[s["types"][i]][None, :] + X0[s["types"][out["src"][sel]]]
+        M1sq = 0.25 + (chi ** 4).sum()
+        u = out["rij"][sel] / d[:, None]
+        cosjk = np.clip(u @ u.T, -1.0, 1.0)
+        off = 2 * C0 + 2
+        for l in (1, 2, 3):
+            C = Cs[l]
+            wb = (chi ** 2)[:, None] * beta[:, :C]                        # [edges, C_l]
+            G = wb.T @ scipy.special.eval_legendre(l, cosjk) @ wb / M1sq
+            vech = np.array([G[a, b] * (1 if a == b else math.sqrt(2)) for a in range(C) for b in range(a, C)])
+            got = out["D_raw"][i][off:off + len(vech)]
+            assert np.allclose(got, vech, rtol=1e-9, atol=1e-12 * np.abs(vech).max()), (i, l)
+            off += len(vech)
+
+
+def test_bispectrum_and_quartic_blocks_from_cartesian_tensors():
+    # Same setting: the probes are v_k = sum_j chi_j^2 beta_jk u_j / M_1 and, by Eq. "stf",
+    # Q_h = sum_j chi_j^2 beta_jh sqrt(3/2) (u_j u_j^T - I/3) / M_1, built here from directions
+    # alone.  Eq. "closed-forms" then gives the (1,1,2) and (2,2,2) blocks and Eq. "quartic"
+    # Pi[h, k] = |Q_h v_k|^2; the feature vector holds J(1,1,2) right after the Gram blocks,
+    # J(2,2,2) after it (L = 2) and Pi, h-major, in its last K_1 K_2 entries.
+    p, o = _beta_only_oracle("p32_2_4", 54)
+    s = make_system(dict(kind="random_box", atoms=16, edges=(8.0, 8.5, 9.0), min_dist=1.6, seed=55,
+                         n_types=p["T"], masses=[1.0] * p["T"]))
+    out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"], want_grad=False)
+    X0 = o.prm["X0"].numpy()
+    C0, C1, C2, K1, K2, D = p["C0"], p["C1"], p["C2"], p["K1"], p["K2"], p["D_out"]
+    for i in (1, 9, 15):
+        sel = out["dst"] == i
+        d = np.sqrt((out["rij"][sel] ** 2).sum(1))
+        chi = 1.0 - scipy.special.betainc(5, 4, np.clip(d / p["rc"], 0, 1))
+        beta = X0[s["types"][i]][None, :] + X0[s["types"][out["src"][sel]]]
+        M1 = math.sqrt(0.25 + (chi ** 4).sum())
+        u = out["rij"][sel] / d[:, None]
+        w = chi ** 2
+        v = np.einsum("e,ek,ea->ka", w, beta[:, :K1], u) / M1                          # [K1, 3]
+        quad = math.sqrt(1.5) * (u[:, :, None] * u[:, None, :] - np.eye(3)[None] / 3.0)
+        Q = np.einsum("e,eh,eab->hab", w, beta[:, :K2], quad) / M1                    # [K2, 3, 3]
+        Dr = out["D_raw"][i]
+        Pi = np.array([[np.sum((Q[h] @ v[k]) ** 2) for k in range(K1)] for h in range(K2)])
+        assert np.allclose(Dr[D - K1 * K2:], Pi.reshape(-1), rtol=1e-9, atol=1e-13 * np.abs(Pi).max())
+        off = 2 * C0 + 2 + C1 * (C1 + 1) // 2 + C2 * (C2 + 1) // 2
+        j112 = [-(1 / math.sqrt(5)) * (v[a] @ Q[h] @ v[b]) * (1.0 if a == b else math.sqrt(2))
+                for a in range(K1) for b in range(a, K1) for h in range(K2)]
+        assert np.allclose(Dr[off:off + len(j112)], j112, rtol=1e-9, atol=1e-13 * np.abs(j112).max())
+        off += len(j112)
+        j222 = []
+        for a in range(K2):
+            for b in range(a, K2):
+                for c in range(b, K2):
+                    fam = len(set(itertools.permutations((a, b, c))))
+                    j222.append(-math.sqrt(12 / 35) * np.trace(Q[a] @ Q[b] @ Q[c]) * math.sqrt(fam))
+        assert np.allclose(Dr[off:off + len(j222)], j222, rtol=1e-9, atol=1e-13 * np.abs(j222).max())
+        assert off + len(j222) == D - K1 * K2
+
+
 # ---------------------------------------------------------------- forces and virial
 
 def _energy(o, pos, s, cell=None):
