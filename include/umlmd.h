@@ -57,7 +57,9 @@ typedef struct umlmd_options {
     uint32_t struct_bytes;
     double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
     int32_t  node_tile;  /* atoms per workspace tile; 0 = 524288                            */
-    int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 3xTF32 GEMM, persistent, 3 = tcgen05 3xTF32 GEMM, one tile per CTA */
+    int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 GEMM on split half-precision operands
+                            (three products, 22 significant bits), persistent, 3 = the same, one tile per CTA;
+                            2 and 3 need F % 8 == 0 and fall back to 1 otherwise */
     int32_t  pair_table_mb;  /* device memory, MiB, that per-pair amplitude tables may take
                                 (see umlmd_build_neighbors); 0 = 192, negative = never build them */
 } umlmd_options;

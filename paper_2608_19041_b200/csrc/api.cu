@@ -24,7 +24,7 @@ struct umlmd {
     std::vector<void*> model_allocs;
     // workspace
     float* state = nullptr; float* desc = nullptr; float* pre = nullptr; float* hbuf = nullptr;
-    float* tc_hi = nullptr; float* tc_lo = nullptr;   // TF32 split of the current GEMM's activations
+    __half* tc_hi = nullptr; __half* tc_lo = nullptr;   // half-precision split of the current GEMM's activations
     int64_t tile_cap = 0;
     float* g = nullptr; int64_t g_cap = 0;
     double* e_atom = nullptr; double* f_sorted = nullptr; int* type_o = nullptr; int64_t n_cap = 0;
@@ -185,7 +185,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         // fp32 feature rows are then only kept where something still reads them (the identity
         // residual of a first layer as wide as the feature vector, or the intermediates query of a
         // system smaller than one node tile)
-        const bool presplit = h->mlp_path >= 2 && gemm_tc_available();
+        const bool presplit = mlp_uses_tc(d.F, h->mlp_path);
         ia.desc_hi = presplit ? h->tc_hi : nullptr; ia.desc_lo = presplit ? h->tc_lo : nullptr;
         ia.write_desc = !presplit || d.D_out == d.F || keeps_intermediates(h);
         const bool fold_x0 = presplit && d.D_out != d.F;      // first GEMM skips the per-species constant columns
@@ -196,7 +196,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit; ma.fold_x0 = fold_x0;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
-        { Scope sc(h, kMlpFwd, d.n_hidden + (presplit ? 1 : (h->mlp_path >= 2 ? 2 : 1))); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
+        { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
             { Scope sc(h, kInvBwd, 1); API_CUDA(h, launch_invariants_backward(ia, h->st)); }
@@ -233,12 +233,15 @@ int ensure_device_model(umlmd_t* h) {
     ModelDev& md = h->md;
     cudaError_t e = cudaSuccess;
     auto up = [&](const std::vector<float>& v, float** p) { if (e == cudaSuccess) e = upload(h, v, p); };
+    auto uph = [&](const std::vector<__half>& v, __half** p) { if (e == cudaSuccess) e = upload(h, v, p); };
     up(m.table, &md.table); up(m.pairmod, &md.pairmod); up(m.X0, &md.X0); up(m.W1p, &md.W1p); up(m.W2p, &md.W2p);
     up(m.A1, &md.A1); up(m.A2, &md.A2); up(m.mu, &md.mu); up(m.inv_sigma, &md.inv_sigma);
     up(m.type_bias, &md.type_bias);
     for (int t = 0; t < h->d.n_hidden; ++t) { up(m.theta[t], &md.theta[t]); up(m.thetaT[t], &md.thetaT[t]); up(m.bias[t], &md.bias[t]);
-        up(m.theta_hi[t], &md.theta_hi[t]); up(m.theta_lo[t], &md.theta_lo[t]);
-        up(m.thetaT_hi[t], &md.thetaT_hi[t]); up(m.thetaT_lo[t], &md.thetaT_lo[t]); }
+        uph(m.theta_hi[t], &md.theta_hi[t]); uph(m.theta_lo[t], &md.theta_lo[t]);
+        uph(m.thetaT_hi[t], &md.thetaT_hi[t]); uph(m.thetaT_lo[t], &md.thetaT_lo[t]);
+        md.w_scale_inv[t] = 1.0f / m.w_scale[t]; }
+    md.grad_scale = m.grad_scale;
     up(m.w_head, &md.w_head); up(m.e_ref, &md.e_ref);
     md.b_head = m.b_head;
     if (e == cudaSuccess && h->d.L >= 3) {

@@ -2,6 +2,7 @@
 // device-resident model constants, the per-handle workspace and the kernel launchers.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -61,8 +62,13 @@ struct ModelDev {
     float* inv_sigma; // [D_out]
     float* theta[8];  // Theta_t, row-major [K_in (padded)][F]; theta[0] has DP rows
     float* thetaT[8]; // transposes, [F][K_in (padded)]
-    float* theta_hi[8];  float* theta_lo[8];    // TF32 split of theta  (x = hi + lo)
-    float* thetaT_hi[8]; float* thetaT_lo[8];   // TF32 split of thetaT
+    // half-precision split (x = hi + lo) of w_scale[t] * theta and of its transpose; w_scale[t] is
+    // the power of two that brings the largest |weight| of the layer to [2^9, 2^10), so that the
+    // low parts are normal half-precision numbers; w_scale_inv[t] undoes it on the accumulator
+    __half* theta_hi[8];  __half* theta_lo[8];
+    __half* thetaT_hi[8]; __half* thetaT_lo[8];
+    float w_scale_inv[8];
+    float grad_scale; // power of two the tensor-core backward chain multiplies its gradients by (from max |w_head|)
     float* bias[8];   // b_t [F]
     float* type_bias; // [T][F] first-layer bias with the centre's initial features folded in
     float* w_head;    // [F]

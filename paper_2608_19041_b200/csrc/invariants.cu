@@ -228,10 +228,10 @@ struct Front {
     }
 };
 
-// one calibrated feature-vector entry: fp32 and / or its TF32 split
+// one calibrated feature-vector entry: fp32 and / or its half-precision split
 __device__ __forceinline__ void put_feature(const InvArgs& a, size_t off, float v, bool split_ok) {
     if (a.write_desc) a.desc[off] = v;
-    if (a.desc_hi && split_ok) split_tf32(v, a.desc_hi[off], a.desc_lo[off]);
+    if (a.desc_hi && split_ok) split_f16(v, a.desc_hi[off], a.desc_lo[off]);
 }
 
 template <int C1, int C2, int L>

@@ -62,10 +62,10 @@ struct InvArgs {
     int a0, n;              // tile start (sorted index) and atom count
     float* state;           // [n][SP]
     float* desc;            // [n][DP]
-    // forward only: when non-null the feature rows are also written as their TF32 split (row pitch
-    // DP), the form the tensor-core MLP reads; write_desc = false then skips the fp32 copy
-    float* desc_hi;
-    float* desc_lo;
+    // forward only: when non-null the feature rows are also written as their half-precision split
+    // (row pitch DP), the form the tensor-core MLP reads; write_desc = false then skips the fp32 copy
+    __half* desc_hi;
+    __half* desc_lo;
     bool write_desc;
     bool skip_x0_split;     // the split omits the first C0 columns (the MLP folds them into a per-species bias)
 };
@@ -84,11 +84,11 @@ struct MlpArgs {
     double* e_atom;         // [N] sorted order, eV (written at a0..a0+n)
     int path;               // 1 = CUDA-core fp32, 2 = tcgen05
     bool want_grad;
-    float* tc_hi;           // two slots of [n][max(DP, F)]: TF32 splits of the activations (tensor-core path)
-    float* tc_lo;
+    __half* tc_hi;          // two slots of [n][max(DP, F)]: half-precision splits of the activations (tensor-core path)
+    __half* tc_lo;
     bool desc_presplit;     // slot 0 already holds the split of desc (written by the invariants kernel)
     bool fold_x0;           // tensor-core path: the first C0 feature columns enter through m.type_bias instead of the GEMM
-    size_t tc_slot;         // floats per slot
+    size_t tc_slot;         // elements per slot
     int* err;               // device error word
 };
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)

@@ -61,11 +61,10 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
 }
 
 // scalar head: E_i = h . w_head + b_head + E_ref[type]; seeds the backward pass with
-// dE/dY_last = w_head * SiLU'(Y_last) (also as a TF32 split for the tensor-core path)
+// dE/dY_last = w_head * SiLU'(Y_last)
 __global__ void k_head(int n, int F, const float* __restrict__ h, const float* __restrict__ w, float b_head,
                        const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
-                       float* __restrict__ pre_last, float* __restrict__ seed_hi, float* __restrict__ seed_lo,
-                       double* __restrict__ e_atom, bool want_grad) {
+                       float* __restrict__ pre_last, double* __restrict__ e_atom, bool want_grad) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= n) return;
     const float* hr = h + (size_t)warp * F;
@@ -80,7 +79,6 @@ __global__ void k_head(int n, int F, const float* __restrict__ h, const float* _
         for (int f = lane; f < F; f += 32) {
             const float v = __ldg(w + f) * silu_grad(pr[f]);
             pr[f] = v;
-            if (seed_hi) split_tf32(v, seed_hi[(size_t)warp * F + f], seed_lo[(size_t)warp * F + f]);
         }
     }
 }
@@ -105,9 +103,11 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-static cudaError_t run_gemm(const GemmArgs& g, int path, cudaStream_t st) {
-    if (path >= 2 && gemm_tc_supported(g)) return launch_gemm_tc(g, st);
-    return launch_gemm_simt(g, st);
+// a model runs all of its layers on one kind of GEMM (the two keep gradients on different scales)
+static cudaError_t run_gemm(const GemmArgs& g, bool tc, cudaStream_t st) {
+    if (!tc) return launch_gemm_simt(g, st);
+    if (!gemm_tc_supported(g)) return cudaErrorInvalidValue;
+    return launch_gemm_tc(g, st);
 }
 
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
@@ -117,7 +117,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     const size_t layer = (size_t)n * F;
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
-    const bool tc = a.path >= 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    const bool tc = a.tc_hi && a.tc_lo && mlp_uses_tc(F, a.path);
     const int variant = tc ? gemm_tc_pick_variant(n, F, a.path) : a.path;
     // the backward seed goes to the slot the last layer does not read its input from
     const int seed_slot = NH & 1;
@@ -126,6 +126,8 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     for (int t = 0; t < NH; ++t) {
         GemmArgs g = {};
         g.mode = 0;
+        g.acc_scale = tc ? a.m.w_scale_inv[t] : 1.0f; g.rvec_scale = 1.0f; g.out_scale = 1.0f;
+        g.seed_scale = tc ? a.m.grad_scale : 1.0f;
         g.M = n; g.N = F;
         if (t == 0) { g.A = a.desc; g.lda = d.DP; g.K = d.DP; g.res = res0 ? a.desc : nullptr; g.ldres = d.DP; }
         else { g.A = hb[(t - 1) & 1]; g.lda = F; g.K = F; g.res = hb[(t - 1) & 1]; g.ldres = F; }
@@ -149,6 +151,12 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         }
         g.pre = a.want_grad ? a.pre + (size_t)t * layer : nullptr; g.ldpre = F;
         g.out = hb[t & 1]; g.ldout = F;
+        if (tc) {
+            // the activations travel as their split only: the residual of layer t is the split this
+            // layer reads as its A operand, and no fp32 copy of the output is stored
+            g.out = nullptr;
+            if (t > 0) { g.res = nullptr; g.res_hi = g.A_hi; g.res_lo = g.A_lo; g.ldres = F; }
+        }
         if (tc && t == NH - 1) {
             // last layer: the epilogue takes the head's dot product and the backward seed, so
             // neither the activations nor the pre-activations of this layer are stored
@@ -159,7 +167,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
                 g.ldnxt = F;
             }
         }
-        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+        if ((e = run_gemm(g, tc, st)) != cudaSuccess) return e;
     }
     if (tc) {
         const int parts = gemm_tc_head_parts(F, variant);
@@ -170,7 +178,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         const int warps = 8, blocks = (n + warps - 1) / warps;
         k_head<<<blocks, warps * 32, 0, st>>>(n, F, hb[(NH - 1) & 1], a.m.w_head, a.m.b_head, a.m.e_ref, a.type_s,
                                              a.a0, a.want_grad ? a.pre + (size_t)(NH - 1) * layer : nullptr,
-                                             nullptr, nullptr, a.e_atom, a.want_grad);
+                                             a.e_atom, a.want_grad);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -185,14 +193,18 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
     float* hb[2] = {a.hbuf, a.hbuf + layer};
     const bool res0 = (d.D_out == F);
     cudaError_t e;
-    const bool tc = a.path >= 2 && a.tc_hi && a.tc_lo && gemm_tc_available();
+    const bool tc = a.tc_hi && a.tc_lo && mlp_uses_tc(F, a.path);
     const int variant = tc ? gemm_tc_pick_variant(n, F, a.path) : a.path;
-    int sp = NH & 1;           // tensor-core path: slot with the TF32 split of pre[t] (the forward pass left the seed here)
+    // tensor-core path: every gradient of the chain is carried multiplied by grad_scale (the seed
+    // came that way); the head weights join it with the same factor and the last GEMM removes it
+    const float gs = tc ? a.m.grad_scale : 1.0f;
+    int sp = NH & 1;           // tensor-core path: slot with the half-precision split of pre[t] (the forward pass left the seed here)
     int slot = 0;              // slot holding dE/dh_t (unused while the gradient is w_head itself)
     bool vec_grad = true;      // dE/dh_t == w_head for every atom (top layer)
     for (int t = NH - 1; t >= 1; --t) {
         GemmArgs g = {};
         g.mode = 1;
+        g.acc_scale = tc ? a.m.w_scale_inv[t] : 1.0f; g.rvec_scale = gs; g.out_scale = 1.0f; g.seed_scale = 1.0f;
         g.M = n; g.N = F; g.K = F;
         g.A = a.pre + (size_t)t * layer; g.lda = F;
         g.B = a.m.thetaT[t]; g.ldb = F;
@@ -206,12 +218,13 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         const bool need_dh = (t - 1 >= 1) || res0;
         g.out = need_dh ? hb[out_slot] : nullptr; g.ldout = F;
         g.pre = a.pre + (size_t)(t - 1) * layer; g.ldpre = F;
-        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+        if ((e = run_gemm(g, tc, st)) != cudaSuccess) return e;
         slot = out_slot; vec_grad = false;
     }
     {
         GemmArgs g = {};
         g.mode = 1;
+        g.acc_scale = tc ? a.m.w_scale_inv[0] : 1.0f; g.rvec_scale = gs; g.out_scale = 1.0f / gs; g.seed_scale = 1.0f;
         g.M = n; g.N = d.DP; g.K = F;
         g.A = a.pre; g.lda = F;
         g.B = a.m.thetaT[0]; g.ldb = d.DP;
@@ -228,7 +241,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
             g.Bt_hi += (size_t)d.C0 * F; g.Bt_lo += (size_t)d.C0 * F;
             g.out = a.desc + d.C0;
         }
-        if ((e = run_gemm(g, a.path, st)) != cudaSuccess) return e;
+        if ((e = run_gemm(g, tc, st)) != cudaSuccess) return e;
     }
     return cudaSuccess;
 }

@@ -2,6 +2,7 @@
 // GEMM kernels of the MLP.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -20,16 +21,27 @@ struct GemmArgs {
     int mode;
     const float* bias;
     const float* res; int ldres; int res_n;
+    // tensor-core path, mode 0: the residual given as a half-precision split (row pitch ldres)
+    // instead of res: the split the previous layer left for this layer's A operand
+    const __half* res_hi; const __half* res_lo;
     const float* rvec; int rvec_n;
     float* pre; int ldpre;
     float* out; int ldout;
-    // tensor-core path only: pre-split copies of B (hi / lo TF32 parts), K-major [N][K]
-    const float* Bt_hi; const float* Bt_lo; int ldbt;
-    float* A_hi; float* A_lo;     // [M][K] TF32 split of A: filled by the caller if a_presplit, else by a split kernel
+    // tensor-core path only: pre-split copies of B (hi / lo half-precision parts, scaled by a power
+    // of two, see acc_scale), K-major [N][K]
+    const __half* Bt_hi; const __half* Bt_lo; int ldbt;
+    __half* A_hi; __half* A_lo;   // [M][K] half-precision split of A: filled by the caller if a_presplit, else by a split kernel
     int a_presplit;
-    // TF32 split of the value the next GEMM of the chain consumes (mode 0: out, mode 1: the new
-    // pre), written by the epilogue with row pitch ldnxt when non-null
-    float* nxt_hi; float* nxt_lo; int ldnxt;
+    // half-precision split of the value the next GEMM of the chain consumes (mode 0: out, mode 1:
+    // the new pre), written by the epilogue with row pitch ldnxt when non-null
+    __half* nxt_hi; __half* nxt_lo; int ldnxt;
+    // tensor-core path: powers of two that keep the low parts of the splits out of the subnormal
+    // range of half precision.  The accumulator is multiplied by acc_scale (the inverse of the
+    // weights' scale) before anything else; the backward chain carries gradients multiplied by a
+    // common factor, so rvec is multiplied by rvec_scale (that factor) on its way in, `out` by
+    // out_scale on its way out (its inverse at the end of the chain), and the seed the last
+    // forward layer leaves for the backward pass by seed_scale.  The CUDA-core path sets all to 1.
+    float acc_scale, rvec_scale, out_scale, seed_scale;
     // tensor-core path, mode 0, last layer: instead of storing out (and pre), the epilogue dots
     // each output row with head_w over the CTA's columns, head_part[m * head_parts + column
     // tile], and, when nxt_hi is set, leaves the split of head_w[n] * SiLU'(y[m,n]) there (the
@@ -42,26 +54,39 @@ struct GemmArgs {
     int* err;                     // device error word (bounded-wait expiry)
 };
 
-__device__ __forceinline__ float sigmoidf_(float x) { return 1.0f / (1.0f + expf(-x)); }
+// Logistic function from the hardware base-2 exponential and reciprocal (two transcendental
+// instructions instead of some twenty for expf and a correctly rounded division, in every element
+// of every GEMM epilogue).  The exponent -x log2(e) is rounded once, which leaves a relative error
+// of about 4e-8 |x| in exp(-x); the logistic function damps it by s (1 - s) <= min(1/4, exp(-|x|)),
+// so the result stays within two single-precision roundings for every x.
+__device__ __forceinline__ float sigmoidf_(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float silu(float x) { return x * sigmoidf_(x); }
 __device__ __forceinline__ float silu_grad(float x) {
     const float s = sigmoidf_(x);
     return s * (1.0f + x * (1.0f - s));
 }
 
-// x = hi + lo with hi = round-to-nearest TF32 of x and lo = round-to-nearest TF32 of (x - hi)
-__device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
-    uint32_t hb, lb;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hb) : "f"(x));
-    hi = __uint_as_float(hb);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lb) : "f"(x - hi));
-    lo = __uint_as_float(lb);
+// x = hi + lo with hi = x rounded to half precision and lo = (x - hi) rounded to half precision:
+// 22 significant bits, as long as lo stays a normal number (|x| above 2^-3 or so; below that the
+// absolute error is the subnormal spacing, 2^-25, which is why gradients and weights are carried
+// multiplied by a power of two)
+__device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo) {
+    hi = __float2half_rn(x);
+    lo = __float2half_rn(x - __half2float(hi));
 }
-__device__ __forceinline__ void store_split4(float* hi, float* lo, size_t off, float4 v) {
-    float4 h, l;
-    split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
-    *reinterpret_cast<float4*>(hi + off) = h;
-    *reinterpret_cast<float4*>(lo + off) = l;
+// four consecutive columns (off a multiple of 4): one 8-byte store per part.  The conversions are
+// the packed ones (two floats to a half2, a half2 to two floats): those run on the FMA pipes,
+// whereas the scalar float-to-half conversion shares the transcendental unit with the
+// exponential and the reciprocal of SiLU, which is what the fused epilogue is bound by.
+__device__ __forceinline__ void store_split4(__half* hi, __half* lo, size_t off, float4 v) {
+    const __half2 h01 = __floats2half2_rn(v.x, v.y), h23 = __floats2half2_rn(v.z, v.w);
+    const float2 f01 = __half22float2(h01), f23 = __half22float2(h23);
+    const __half2 l01 = __floats2half2_rn(v.x - f01.x, v.y - f01.y), l23 = __floats2half2_rn(v.z - f23.x, v.w - f23.y);
+    uint2 hw, lw;
+    hw.x = *reinterpret_cast<const uint32_t*>(&h01); hw.y = *reinterpret_cast<const uint32_t*>(&h23);
+    lw.x = *reinterpret_cast<const uint32_t*>(&l01); lw.y = *reinterpret_cast<const uint32_t*>(&l23);
+    *reinterpret_cast<uint2*>(hi + off) = hw;
+    *reinterpret_cast<uint2*>(lo + off) = lw;
 }
 
 // epilogue for four consecutive columns n..n+3 of row m (n multiple of 4, n < N)
@@ -96,13 +121,24 @@ __device__ __forceinline__ void gemm_epilogue4(const GemmArgs& g, int m, int n, 
     }
 }
 
+// hi + lo of four consecutive columns, through the read-only path
+__device__ __forceinline__ float4 load_split4(const __half* hi, const __half* lo, size_t off) {
+    const uint2 hw = __ldg(reinterpret_cast<const uint2*>(hi + off)), lw = __ldg(reinterpret_cast<const uint2*>(lo + off));
+    const float2 h0 = __half22float2(*reinterpret_cast<const __half2*>(&hw.x)), h1 = __half22float2(*reinterpret_cast<const __half2*>(&hw.y));
+    const float2 l0 = __half22float2(*reinterpret_cast<const __half2*>(&lw.x)), l1 = __half22float2(*reinterpret_cast<const __half2*>(&lw.y));
+    return make_float4(h0.x + l0.x, h0.y + l0.y, h1.x + l1.x, h1.y + l1.y);
+}
+
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 bool gemm_tc_supported(const GemmArgs& g);
 bool gemm_tc_available();      // the driver's tensor-map encoder could be resolved
+// whether a model of hidden width F runs its MLP on the tensor-core GEMM under `path` (the
+// half-precision operand rows must be multiples of 16 bytes)
+inline bool mlp_uses_tc(int F, int path) { return path >= 2 && (F & 7) == 0 && gemm_tc_available(); }
 int gemm_tc_pick_variant(int M, int N, int requested);   // 2 (persistent) or 3 (one tile per CTA) for path 2
 constexpr int kGemmTcBN = 128;  // column tile of the tensor-core GEMM
 // partial head sums per row that the fused last-layer epilogue of a variant leaves
-inline int gemm_tc_head_parts(int N, int variant) { return (variant == 3 ? 1 : 2) * ((N + kGemmTcBN - 1) / kGemmTcBN); }
+inline int gemm_tc_head_parts(int N, int variant) { return (variant == 3 ? 1 : 4) * ((N + kGemmTcBN - 1) / kGemmTcBN); }
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st);
 
 }  // namespace umd

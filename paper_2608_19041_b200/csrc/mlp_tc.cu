@@ -1,20 +1,26 @@
 // Tensor-core GEMM for the MLP layers on sm_100a: TMA loads into 64-byte-swizzled shared
-// memory, tcgen05.mma (kind::tf32) issued by one thread, fp32 accumulator in tensor memory,
+// memory, tcgen05.mma (kind::f16) issued by one thread, fp32 accumulator in tensor memory,
 // tcgen05.ld epilogue with the fused bias / SiLU / residual (or SiLU-derivative) step.
 //
-// Precision: a single TF32 product carries 11 significant bits, far short of the 1e-5
-// parity target, so every operand is split into two TF32 numbers, x = hi + lo with
-// hi = round_tf32(x) and lo = round_tf32(x - hi), and each K step issues three MMAs,
-// A_lo B_hi + A_hi B_lo + A_hi B_hi (the lo*lo term, ~2^-22, is dropped).  Both parts are
-// exactly representable in TF32, so the result does not depend on how the tensor core
-// treats the low mantissa bits.  Weights are split once on the host; activations are split
-// by the kernel that produces them (the invariants kernel, a GEMM epilogue; a small split kernel
-// remains for callers that hand in an unsplit operand).
+// Precision: a single half-precision (or TF32) product carries 11 significant bits, far short
+// of the 1e-5 parity target, so every operand is split into two half-precision numbers,
+// x = hi + lo with hi = half(x) and lo = half(x - hi), and each K step issues three MMAs,
+// A_lo B_hi + A_hi B_lo + A_hi B_hi (the lo*lo term, ~2^-22, is dropped): the same 22
+// significant bits as a split into two TF32 numbers, at twice the tensor-core rate (K = 16 per
+// instruction instead of 8) and half the operand bytes (hi and lo together are as large as the
+// fp32 value).  Half precision has the narrower exponent: a low part below 2^-14 is subnormal
+// and keeps an absolute error of 2^-25.  Activations are O(1), where that is at the level of
+// single-precision rounding; weights and back-propagated gradients are small numbers, so the
+// weights are stored multiplied by a power of two chosen per layer at create time and the
+// backward chain carries its gradients multiplied by one chosen from the head weights
+// (GemmArgs::acc_scale, rvec_scale, out_scale, seed_scale); powers of two change no mantissa.
+// Weights are split once on the host; activations are split by the kernel that produces them
+// (the invariants kernel, a GEMM epilogue; a small split kernel remains for callers that hand in
+// an unsplit operand).
 //
-// Tiling of the first kernel below: one CTA computes a 128 x 128 output tile; K advances in blocks of 16 floats (one
+// Tiling of the first kernel below: one CTA computes a 128 x 128 output tile; K advances in blocks of 32 halves (one
 // 64-byte swizzle span) through a 3-stage ring of {A_hi, A_lo, B_hi, B_lo} tiles (32 KB per
-// stage), so two CTAs fit on an SM and one CTA's epilogue overlaps the other's main loop
-// (a 128 x 128 x 8 TF32 MMA reads 8 KB of shared memory and is bound by that, ~94 cycles).
+// stage), so two CTAs fit on an SM and one CTA's epilogue overlaps the other's main loop.
 // This kernel keeps the hi*hi sum and the cross terms in two accumulators (256 columns of
 // tensor memory per CTA); the persistent kernel further down, which needs all 512 columns
 // for its double buffering, sums all three products into one.
@@ -34,8 +40,9 @@ namespace umd {
 
 namespace {
 
-constexpr int BM = 128, BN = kGemmTcBN, BK = 16, STAGES = 3;
-constexpr uint32_t TILE_BYTES = BM * BK * 4;          // 8 KB, also BN * BK * 4
+constexpr int BM = 128, BN = kGemmTcBN, BK = 32, STAGES = 3;   // BK in half-precision elements
+constexpr int MMA_K = 16;                              // K of one kind::f16 instruction (32 bytes of a row)
+constexpr uint32_t TILE_BYTES = BM * BK * 2;          // 8 KB, also BN * BK * 2
 constexpr uint32_t STAGE_BYTES = 4 * TILE_BYTES;      // A_hi, A_lo, B_hi, B_lo
 constexpr uint32_t BAR_BYTES = 128;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + BAR_BYTES;
@@ -79,11 +86,11 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
     return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(512 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)4 << 61);
 }
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -108,8 +115,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// instruction descriptor: D = F32, A = B = TF32, both K-major, N = 128, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// instruction descriptor: D = F32, A = B = F16 (format code 0), both K-major, N = 128, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // MODE 0: forward layer, 1: backward layer, 2: last forward layer with the fused head
 template <int MODE>
@@ -162,16 +169,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                 tc_fence_after();
                 const uint32_t sa = tiles + s * STAGE_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / 8; ++k) {
+                for (int k = 0; k < BK / MMA_K; ++k) {
                     const uint64_t ah = umma_desc(sa + k * 32), al = umma_desc(sa + TILE_BYTES + k * 32);
                     const uint64_t bh = umma_desc(sa + 2 * TILE_BYTES + k * 32), bl = umma_desc(sa + 3 * TILE_BYTES + k * 32);
                     // The accumulator truncates once per instruction.  The cross terms, 2^-11 of
                     // the result, get an accumulator of their own, where that loss is 2^-11 as
                     // small, and the main sum sees a third of the instructions.
                     const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                    umma_tf32(tmem + BN, al, bh, kIdesc, acc);
-                    umma_tf32(tmem + BN, ah, bl, kIdesc, 1u);
-                    umma_tf32(tmem, ah, bh, kIdesc, acc);
+                    umma_f16(tmem + BN, al, bh, kIdesc, acc);
+                    umma_f16(tmem + BN, ah, bl, kIdesc, 1u);
+                    umma_f16(tmem, ah, bh, kIdesc, acc);
                 }
                 umma_commit(bars + 8 * (STAGES + s));      // frees the stage when these MMAs retire
             }
@@ -187,6 +194,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
         mbar_wait(accum_bar, 0, g.err);
         tc_fence_after();
         float* stage = reinterpret_cast<float*>(smem_raw + (tiles - raw)) + (size_t)q * 32 * EPITCH;
+        const float sc = g.acc_scale;
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += 32) {
             float v[32], w[32];
@@ -195,7 +203,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 *reinterpret_cast<float4*>(stage + lane * EPITCH + c0 + 4 * j) =
-                    make_float4(v[4 * j] + w[4 * j], v[4 * j + 1] + w[4 * j + 1], v[4 * j + 2] + w[4 * j + 2], v[4 * j + 3] + w[4 * j + 3]);
+                    make_float4(sc * (v[4 * j] + w[4 * j]), sc * (v[4 * j + 1] + w[4 * j + 1]), sc * (v[4 * j + 2] + w[4 * j + 2]),
+                                sc * (v[4 * j + 3] + w[4 * j + 3]));
         }
         __syncwarp();
         const int n = n0 + 4 * lane;
@@ -204,8 +213,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
             float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
             if (valid && MODE != 1 && !g.bias_rows) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
             if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
-            const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
-            if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+            const bool use_res = valid && (g.res || g.res_hi) && (MODE != 1 || g.res_n == 0 || n < g.res_n);
+            if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) {
+                rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+                rvec.x *= g.rvec_scale; rvec.y *= g.rvec_scale; rvec.z *= g.rvec_scale; rvec.w *= g.rvec_scale;
+            }
             const int rows = min(32, g.M - (m0 + q * 32));
             // The stores below may alias the loads as far as the compiler knows, so the rows
             // are taken in batches: all global loads of a batch are issued before its first
@@ -221,8 +233,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                     res[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                     y[j] = res[j];
                     if (r0 + j < rows) {
-                        if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + m * g.ldres + n);
-                        if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n);
+                        if (use_res) {
+                            if (MODE != 1 && g.res_hi) res[j] = load_split4(g.res_hi, g.res_lo, m * g.ldres + n);
+                            else res[j] = __ldg(reinterpret_cast<const float4*>(g.res + m * g.ldres + n));
+                        }
+                        if (MODE == 1 && rd_pre) y[j] = __ldg(reinterpret_cast<const float4*>(g.pre + m * g.ldpre + n));
                         if (MODE != 1 && valid && g.bias_rows)      // per-species bias: carried in the y slot
                             y[j] = __ldg(reinterpret_cast<const float4*>(g.bias_rows + (size_t)g.row_type[m] * g.N + n));
                     }
@@ -244,23 +259,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                             if (lane == 0) g.head_part[m * g.head_parts + blockIdx.x] = part;
                             if (valid && g.nxt_hi)
                                 store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n,
-                                             make_float4(hw.x * silu_grad(a.x), hw.y * silu_grad(a.y), hw.z * silu_grad(a.z),
-                                                         hw.w * silu_grad(a.w)));
+                                             make_float4(g.seed_scale * hw.x * silu_grad(a.x), g.seed_scale * hw.y * silu_grad(a.y),
+                                                         g.seed_scale * hw.z * silu_grad(a.z), g.seed_scale * hw.w * silu_grad(a.w)));
                         } else if (valid) {
                             if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
-                            *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
+                            if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
                             if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
                         }
                     } else if (valid) {
                         a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
-                        if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
+                        if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = make_float4(g.out_scale * a.x, g.out_scale * a.y, g.out_scale * a.z, g.out_scale * a.w);
                         if (g.pre) {
                             const float4 o = make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y),
                                                          a.z * silu_grad(y[j].z), a.w * silu_grad(y[j].w));
-                            // the next GEMM of the chain reads the split; the fp32 copy is only
-                            // kept when nothing else will carry the value
-                            if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
-                            else *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
+                            // the next GEMM of the chain reads the split (gemm_tc_supported insists on it)
+                            store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
                         }
                     }
                 }
@@ -279,13 +292,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
 // uses two accumulators (rows 0..127 and 128..255) that share every B tile, so the weights
 // cross L2 -> shared memory half as often as with one 128 x 128 tile per CTA; tensor memory
 // holds two such pairs (512 columns), so the epilogue of item i overlaps the main loop of
-// item i + 1.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2..9: epilogue (warp % 4 =
-// lane quarter of tensor memory, (warp - 2) / 4 = which accumulator of the pair).
-// The epilogue turns the tile through a staging area of its own, 64 columns at a time.
+// item i + 1.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2..17: epilogue (warp % 4 =
+// lane quarter of tensor memory; of the four warps of a quarter, one per accumulator of the
+// pair and per 64-column half).  The fused epilogue is a few dozen dependent instructions per
+// element (exponential, reciprocal, conversions) and is bound by instruction latency, not by
+// memory: with eight warps (two per scheduler) it took twice as long as an item's MMAs; sixteen
+// hide that latency.  The epilogue turns the tile through a staging area of its own, 32 columns
+// at a time.
 constexpr int P_STAGES = 3;
 constexpr uint32_t P_STAGE_BYTES = 6 * TILE_BYTES;    // A0_hi, A0_lo, A1_hi, A1_lo, B_hi, B_lo
-constexpr int P_EPW = 8;                               // epilogue warps
-constexpr int P_SPITCH = 64 + 4;                       // staging row pitch (floats)
+constexpr int P_EPW = 16;                              // epilogue warps
+constexpr int P_SPITCH = 32 + 4;                       // staging row pitch (floats)
 constexpr uint32_t P_STAGING_BYTES = P_EPW * 32 * P_SPITCH * 4;
 constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_STAGING_BYTES + 1024 + BAR_BYTES;
 constexpr int P_THREADS = (2 + P_EPW) * 32;
@@ -367,20 +384,20 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                     tc_fence_after();
                     const uint32_t sa = tiles + s * P_STAGE_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / 8; ++k) {
+                    for (int k = 0; k < BK / MMA_K; ++k) {
                         const uint64_t bh = umma_desc(sa + 4 * TILE_BYTES + k * 32), bl = umma_desc(sa + 5 * TILE_BYTES + k * 32);
                         const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
                         {
                             const uint64_t ah = umma_desc(sa + k * 32), al = umma_desc(sa + TILE_BYTES + k * 32);
-                            umma_tf32(d0, al, bh, kIdesc, acc);
-                            umma_tf32(d0, ah, bl, kIdesc, 1u);
-                            umma_tf32(d0, ah, bh, kIdesc, 1u);
+                            umma_f16(d0, al, bh, kIdesc, acc);
+                            umma_f16(d0, ah, bl, kIdesc, 1u);
+                            umma_f16(d0, ah, bh, kIdesc, 1u);
                         }
                         {
                             const uint64_t ah = umma_desc(sa + 2 * TILE_BYTES + k * 32), al = umma_desc(sa + 3 * TILE_BYTES + k * 32);
-                            umma_tf32(d1, al, bh, kIdesc, acc);
-                            umma_tf32(d1, ah, bl, kIdesc, 1u);
-                            umma_tf32(d1, ah, bh, kIdesc, 1u);
+                            umma_f16(d1, al, bh, kIdesc, acc);
+                            umma_f16(d1, ah, bl, kIdesc, 1u);
+                            umma_f16(d1, ah, bh, kIdesc, 1u);
                         }
                     }
                     umma_commit(bars + 8 * (P_STAGES + s));    // frees the stage when these MMAs retire
@@ -389,96 +406,102 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
             }
         }
     } else {                                               // epilogue
-        const int e = warp - 2, q = warp & 3, h = e >> 2;
+        const int e = warp - 2, q = warp & 3, h = (e >> 2) & 1, p = e >> 3;
         float* stage = reinterpret_cast<float*>(smem_raw + (staging - raw)) + (size_t)e * 32 * P_SPITCH;
-        const int hr = lane >> 4, c4 = (lane & 15) * 4;      // half-warp per row, four columns per lane
+        const int rr = lane >> 3, c4 = (lane & 7) * 4;       // eight lanes per row, four columns per lane
+        const float sc = g.acc_scale;
         int li = 0;
         for (int it = blockIdx.x; it < items; it += gridDim.x, ++li) {
             const int b = li & 1, v = li >> 1;
             const int ct = it % ntn;
-            const int mrow0 = (it / ntn) * 2 * BM + h * BM + q * 32, n0 = ct * BN;
+            const int mrow0 = (it / ntn) * 2 * BM + h * BM + q * 32, n0 = ct * BN + p * 64;
             mbar_wait_a(acc_full + 8 * b, v & 1, g.err, abort_flag);
             tc_fence_after();
-            const uint32_t tacc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 256 + h * 128);
+            const uint32_t tacc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 256 + h * 128 + p * 64);
 #pragma unroll 1
-            for (int pass = 0; pass < 2; ++pass) {
-#pragma unroll 1
-                for (int c0 = 0; c0 < 64; c0 += 32) {
+            for (int ch = 0; ch < 2; ++ch) {               // two chunks of 32 columns
+                {
                     float vv[32];
-                    tmem_ld32(tacc + (uint32_t)(pass * 64 + c0), vv);
+                    tmem_ld32(tacc + (uint32_t)(ch * 32), vv);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<float4*>(stage + lane * P_SPITCH + c0 + 4 * j) =
-                            make_float4(vv[4 * j], vv[4 * j + 1], vv[4 * j + 2], vv[4 * j + 3]);
+                        *reinterpret_cast<float4*>(stage + lane * P_SPITCH + 4 * j) =
+                            make_float4(sc * vv[4 * j], sc * vv[4 * j + 1], sc * vv[4 * j + 2], sc * vv[4 * j + 3]);
                 }
-                if (pass == 1) {                           // the accumulator has been read out: hand it back
+                if (ch == 1) {                             // the accumulator has been read out: hand it back
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty + 8 * b) : "memory");
                 }
                 __syncwarp();
-                const int n = n0 + pass * 64 + c4;
+                const int n = n0 + ch * 32 + c4;
                 const bool valid = n < g.N;
                 float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), rvec = bias, hw = bias;
                 if (valid && MODE != 1 && !g.bias_rows) bias = __ldg(reinterpret_cast<const float4*>(g.bias + n));
                 if (valid && MODE == 2) hw = __ldg(reinterpret_cast<const float4*>(g.head_w + n));
-                const bool use_res = valid && g.res && (MODE != 1 || g.res_n == 0 || n < g.res_n);
-                if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+                const bool use_res = valid && (g.res || g.res_hi) && (MODE != 1 || g.res_n == 0 || n < g.res_n);
+                if (valid && MODE == 1 && g.rvec && (g.rvec_n == 0 || n < g.rvec_n)) {
+                    rvec = __ldg(reinterpret_cast<const float4*>(g.rvec + n));
+                    rvec.x *= g.rvec_scale; rvec.y *= g.rvec_scale; rvec.z *= g.rvec_scale; rvec.w *= g.rvec_scale;
+                }
                 const bool rd_pre = valid && MODE == 1 && g.pre;
-                constexpr int RB = 4;                      // iterations (two rows each) whose loads are issued together
+                constexpr int RB = 4;                      // iterations (four rows each) whose loads are issued together
 #pragma unroll 1
-                for (int i0 = 0; i0 < 16; i0 += RB) {
+                for (int i0 = 0; i0 < 8; i0 += RB) {
                     float4 res[RB], y[RB];
 #pragma unroll
                     for (int j = 0; j < RB; ++j) {
-                        const int m = mrow0 + 2 * (i0 + j) + hr;
+                        const int m = mrow0 + 4 * (i0 + j) + rr;
                         res[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                         y[j] = res[j];
                         if (m < g.M) {
-                            if (use_res) res[j] = *reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n);
-                            if (MODE == 1 && rd_pre) y[j] = *reinterpret_cast<const float4*>(g.pre + (size_t)m * g.ldpre + n);
+                            if (use_res) {
+                                if (MODE != 1 && g.res_hi) res[j] = load_split4(g.res_hi, g.res_lo, (size_t)m * g.ldres + n);
+                                else res[j] = __ldg(reinterpret_cast<const float4*>(g.res + (size_t)m * g.ldres + n));
+                            }
+                            if (MODE == 1 && rd_pre) y[j] = __ldg(reinterpret_cast<const float4*>(g.pre + (size_t)m * g.ldpre + n));
                             if (MODE != 1 && valid && g.bias_rows)  // per-species bias: carried in the y slot
-                                y[j] = __ldg(reinterpret_cast<const float4*>(g.bias_rows + (size_t)g.row_type[m] * g.N + n));
+                                y[j] = __ldg(reinterpret_cast<const float4*>(g.bias_rows + (size_t)__ldg(g.row_type + m) * g.N + n));
                         }
                     }
 #pragma unroll
                     for (int j = 0; j < RB; ++j) {
-                        const int r = 2 * (i0 + j) + hr;
+                        const int r = 4 * (i0 + j) + rr;
                         const size_t m = (size_t)(mrow0 + r);
                         const bool okm = mrow0 + r < g.M;
+                        const float4 rj = res[j], yj = y[j];
                         float4 a = *reinterpret_cast<const float4*>(stage + r * P_SPITCH + c4);
                         if (MODE != 1) {
-                            const float4 bb = g.bias_rows ? y[j] : bias;
+                            const float4 bb = g.bias_rows ? yj : bias;
                             a.x += bb.x; a.y += bb.y; a.z += bb.z; a.w += bb.w;
-                            const float4 o = make_float4(silu(a.x) + res[j].x, silu(a.y) + res[j].y, silu(a.z) + res[j].z,
-                                                         silu(a.w) + res[j].w);
-                            if (MODE == 2) {               // last layer: row . w_head over these 64 columns, and the seed
+                            const float4 o = make_float4(silu(a.x) + rj.x, silu(a.y) + rj.y, silu(a.z) + rj.z, silu(a.w) + rj.w);
+                            if (MODE == 2) {               // last layer: row . w_head over these 32 columns, and the seed
                                 float part = valid ? o.x * hw.x + o.y * hw.y + o.z * hw.z + o.w * hw.w : 0.f;
 #pragma unroll
-                                for (int off = 8; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-                                if ((lane & 15) == 0 && okm) g.head_part[m * g.head_parts + 2 * ct + pass] = part;
+                                for (int off = 4; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                                if ((lane & 7) == 0 && okm) g.head_part[m * g.head_parts + 4 * ct + 2 * p + ch] = part;
                                 if (valid && okm && g.nxt_hi)
                                     store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n,
-                                                 make_float4(hw.x * silu_grad(a.x), hw.y * silu_grad(a.y), hw.z * silu_grad(a.z),
-                                                             hw.w * silu_grad(a.w)));
+                                                 make_float4(g.seed_scale * hw.x * silu_grad(a.x), g.seed_scale * hw.y * silu_grad(a.y),
+                                                             g.seed_scale * hw.z * silu_grad(a.z), g.seed_scale * hw.w * silu_grad(a.w)));
                             } else if (valid && okm) {
                                 if (g.pre) *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = a;
-                                *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
+                                if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = o;
                                 if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
                             }
                         } else if (valid && okm) {
-                            a.x += res[j].x + rvec.x; a.y += res[j].y + rvec.y; a.z += res[j].z + rvec.z; a.w += res[j].w + rvec.w;
-                            if (g.out) *reinterpret_cast<float4*>(g.out + m * g.ldout + n) = a;
-                            if (g.pre) {
-                                const float4 o = make_float4(a.x * silu_grad(y[j].x), a.y * silu_grad(y[j].y),
-                                                             a.z * silu_grad(y[j].z), a.w * silu_grad(y[j].w));
-                                if (g.nxt_hi) store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n, o);
-                                else *reinterpret_cast<float4*>(g.pre + m * g.ldpre + n) = o;
-                            }
+                            a.x += rj.x + rvec.x; a.y += rj.y + rvec.y; a.z += rj.z + rvec.z; a.w += rj.w + rvec.w;
+                            if (g.out)
+                                *reinterpret_cast<float4*>(g.out + m * g.ldout + n) =
+                                    make_float4(g.out_scale * a.x, g.out_scale * a.y, g.out_scale * a.z, g.out_scale * a.w);
+                            if (g.pre)                     // the next GEMM of the chain reads the split (gemm_tc_supported insists on it)
+                                store_split4(g.nxt_hi, g.nxt_lo, m * g.ldnxt + n,
+                                             make_float4(a.x * silu_grad(yj.x), a.y * silu_grad(yj.y), a.z * silu_grad(yj.z),
+                                                         a.w * silu_grad(yj.w)));
                         }
                     }
                 }
-                __syncwarp();                              // staging rows are rewritten by the next pass
+                __syncwarp();                              // staging rows are rewritten by the next chunk
             }
         }
     }
@@ -489,9 +512,9 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
     }
 }
 
-// hi = round-to-nearest TF32 of x, lo = round-to-nearest TF32 of (x - hi); rows [M][K]
-__global__ void k_split_tf32(const float* __restrict__ A, int lda, int M, int K, float* __restrict__ hi,
-                             float* __restrict__ lo) {
+// half-precision split of an fp32 matrix, rows [M][K] (K a multiple of 4)
+__global__ void k_split_f16(const float* __restrict__ A, int lda, int M, int K, __half* __restrict__ hi,
+                            __half* __restrict__ lo) {
     const int k4 = K >> 2;
     const size_t total = (size_t)M * k4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -519,15 +542,16 @@ EncodeFn encode_fn() {
     return fn;
 }
 
-// 2-D map over a row-major [rows][cols] float matrix with row pitch ld; box = 16 cols x 128 rows
-bool make_map(CUtensorMap* map, const float* ptr, int rows, int cols, int ld) {
+// 2-D map over a row-major [rows][cols] half-precision matrix with row pitch ld (elements); box =
+// 32 cols x 128 rows
+bool make_map(CUtensorMap* map, const __half* ptr, int rows, int cols, int ld) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {BK, BM};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(ptr), dims, strides, box, estr,
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -551,8 +575,15 @@ int gemm_tc_pick_variant(int M, int N, int requested) {
 }
 
 bool gemm_tc_supported(const GemmArgs& g) {
-    return g.A_hi && g.A_lo && g.Bt_hi && g.Bt_lo && g.M > 0 && g.N >= 4 && g.K >= 4 && (g.K & 3) == 0 &&
-           (g.N & 3) == 0 && (g.lda & 3) == 0 && (g.ldbt & 3) == 0 && encode_fn() != nullptr;
+    // rows of the half-precision operands start on 16-byte boundaries (tensor-map strides, and the
+    // column offset of a folded first layer); the epilogue works on four fp32 columns at a time
+    const int lda_s = g.lda_split ? g.lda_split : g.K;
+    if (g.mode == 1 && g.pre && !g.nxt_hi) return false;     // pre is read through the read-only path, never rewritten
+    return g.A_hi && g.A_lo && g.Bt_hi && g.Bt_lo && g.M > 0 && g.N >= 4 && g.K >= 8 && (g.K & 3) == 0 &&
+           (g.N & 3) == 0 && (lda_s & 7) == 0 && (g.ldbt & 7) == 0 &&
+           (reinterpret_cast<uintptr_t>(g.A_hi) & 15) == 0 && (reinterpret_cast<uintptr_t>(g.A_lo) & 15) == 0 &&
+           (reinterpret_cast<uintptr_t>(g.Bt_hi) & 15) == 0 && (reinterpret_cast<uintptr_t>(g.Bt_lo) & 15) == 0 &&
+           encode_fn() != nullptr;
 }
 
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
@@ -575,7 +606,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st) {
         const size_t total = (size_t)g.M * (g.K >> 2);
         int blocks = (int)((total + 255) / 256);
         if (blocks > 148 * 16) blocks = 148 * 16;
-        k_split_tf32<<<blocks, 256, 0, st>>>(g.A, g.lda, g.M, g.K, g.A_hi, g.A_lo);
+        k_split_f16<<<blocks, 256, 0, st>>>(g.A, g.lda, g.M, g.K, g.A_hi, g.A_lo);
     }
     CUtensorMap mAh, mAl, mBh, mBl;
     const int lda_s = g.lda_split ? g.lda_split : g.K;

@@ -388,30 +388,44 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
                 m->type_bias[(size_t)t * F + f] = (float)s;
             }
     }
-    // TF32 splits for the tensor-core GEMM: hi = round-to-nearest-even to 10 mantissa bits,
-    // lo = the same rounding of (x - hi); both are exactly representable in TF32
-    auto tf32 = [](float x) {
-        uint32_t u;
-        std::memcpy(&u, &x, 4);
-        u += 0x00000FFFu + ((u >> 13) & 1u);
-        u &= 0xFFFFE000u;
-        float y;
-        std::memcpy(&y, &u, 4);
-        return y;
+    // Half-precision splits for the tensor-core GEMM: x = hi + lo, hi = half(x), lo = half(x - hi).
+    // The low part of a small number would be subnormal in half precision, so each layer's weights
+    // are split after multiplication by the power of two that brings the layer's largest magnitude
+    // into [2^9, 2^10) (the GEMM epilogue multiplies the accumulator by the inverse).
+    auto pow2_scale = [](double max_abs, int target_exp) {
+        if (!(max_abs > 0)) return 1.0f;
+        int e;
+        std::frexp(max_abs, &e);                 // max_abs = f * 2^e, f in [0.5, 1)
+        return (float)std::ldexp(1.0, target_exp - e);
     };
-    auto split = [&](const std::vector<float>& w, std::vector<float>* hi, std::vector<float>* lo) {
+    auto split = [&](const std::vector<float>& w, float sc, std::vector<__half>* hi, std::vector<__half>* lo) {
         hi->resize(w.size()); lo->resize(w.size());
-        for (size_t i = 0; i < w.size(); ++i) { (*hi)[i] = tf32(w[i]); (*lo)[i] = tf32(w[i] - (*hi)[i]); }
+        for (size_t i = 0; i < w.size(); ++i) {
+            const float x = w[i] * sc;
+            (*hi)[i] = __float2half_rn(x);
+            (*lo)[i] = __float2half_rn(x - __half2float((*hi)[i]));
+        }
     };
     m->theta_hi.resize(NH); m->theta_lo.resize(NH); m->thetaT_hi.resize(NH); m->thetaT_lo.resize(NH);
+    m->w_scale.resize(NH);
     for (int t = 0; t < NH; ++t) {
-        split(m->theta[t], &m->theta_hi[t], &m->theta_lo[t]);
-        split(m->thetaT[t], &m->thetaT_hi[t], &m->thetaT_lo[t]);
+        double mx = 0;
+        for (float v : m->theta[t]) mx = std::fmax(mx, std::fabs((double)v));
+        m->w_scale[t] = pow2_scale(mx, 10);
+        split(m->theta[t], m->w_scale[t], &m->theta_hi[t], &m->theta_lo[t]);
+        split(m->thetaT[t], m->w_scale[t], &m->thetaT_hi[t], &m->thetaT_lo[t]);
     }
     const size_t tail = 13 + 2 * NH;
     m->w_head = to_f(arr[tail]);
     m->b_head = (float)arr[tail + 1][0];
     m->e_ref = to_f(arr[tail + 2]);
+    {
+        // the backward pass starts from w_head * SiLU' and stays on that scale: carry it times the
+        // power of two that brings max |w_head| into [2^5, 2^6)
+        double mx = 0;
+        for (float v : m->w_head) mx = std::fmax(mx, std::fabs((double)v));
+        m->grad_scale = pow2_scale(mx, 6);
+    }
 
     // ---- Gaunt couplings of the generic triples ------------------------------------
     m->g123.n = 0; m->g233.n = 0;

@@ -6,6 +6,8 @@
 #include <string>
 #include <vector>
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace umd {
@@ -17,7 +19,10 @@ struct HostModel {
     std::vector<float> pairmod;    // [T*T][2+R][C0]
     std::vector<float> X0, W1p, W2p, A1, A2, mu, inv_sigma;
     std::vector<std::vector<float>> theta, thetaT, bias;   // per hidden layer
-    std::vector<std::vector<float>> theta_hi, theta_lo, thetaT_hi, thetaT_lo;   // TF32 splits
+    // half-precision splits of w_scale[t] * theta[t] (and of the transposes) for the tensor-core GEMM
+    std::vector<std::vector<__half>> theta_hi, theta_lo, thetaT_hi, thetaT_lo;
+    std::vector<float> w_scale;    // per layer, a power of two
+    float grad_scale = 1.0f;       // power of two for the back-propagated gradients
     std::vector<float> type_bias;  // [T][F]: b_1 plus the first layer's image of the centre's calibrated initial features
     std::vector<float> w_head, e_ref;
     float b_head = 0;

@@ -19,7 +19,8 @@ def _binding():
 
 @pytest.mark.parametrize("name,n_force,n_rows,modes", [("cfg3_water32400", 3, 48, None), ("cfg4_hea128k", 3, 48, None),
                                                        ("cfg5_amorphous1m", 2, 24, None),
-                                                       ("cfg3_water32400", 2, 24, 4)])   # R = 4: the profile with shared radial modes
+                                                       ("cfg3_water32400", 2, 24, 4),    # R = 4: the profile with shared radial modes
+                                                       ("cfg5_amorphous1m", 1, 12, 4)])  # R = 4 with 64 species: modes read through the pair cache
 def test_fullsize_sampled_parity(name, n_force, n_rows, modes):
     cfg = CONFIGS[name]
     s = make_system(cfg["system"])

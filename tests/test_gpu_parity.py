@@ -330,13 +330,12 @@ def test_paper_variants_on_small_diamond_cell(name):
     s = make_system(dict(cfg["system"], cells=4))
     blob = make_blob(cfg["profile"], seed=cfg["weights_seed"], calibration=load_calibration(name), bias_scale=0.1,
                      e_ref_scale=0.5)
-    # Twice the usual tolerance: on this nearly perfect lattice the odd-degree invariants almost
-    # cancel (single-precision noise amplified by the calibration, as on the 108-atom Al cell), and
-    # the tensor-core accumulator truncates once per MMA instruction, a one-sided bias of about half
-    # an ulp times the 100-150 instructions per output (~4e-6 of a pre-activation); together they
-    # sit at 0.5-1.1e-5 of the largest atomic energy here, while the CUDA-core path shows 5e-6.
-    _compare(blob, s, check_intermediates=False, tol_scale=2.0)
-    _compare(blob, s, check_intermediates=False, skin=1.0, tol_scale=2.0)
+    # a nearly perfect lattice, like the 108-atom Al cell: the odd-degree invariants almost cancel and
+    # single-precision noise in them is amplified by the calibration; the per-variant error is printed
+    for skin in (0.0, 1.0):
+        ref, out = _compare(blob, s, check_intermediates=False, skin=skin)
+        err = np.abs(out["atom_energy"].cpu().numpy() - ref["E_i"]).max() / np.abs(ref["E_i"]).max()
+        print(f"{name} skin {skin}: max|dE_i| / max|E_i| = {err:.2e}")
 
 
 def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():

@@ -142,4 +142,9 @@ SMALL_PROFILES = {
     # D_out == F: the first MLP layer carries the identity residual
     "p32_2_0_res": _profile(32, 2, 0, 8, 2, 144, 2, C1=8, C2=4, K1=4, K2=2, H=88,
                             Hp=176, S=76, D_out=144),
+    # the widest scalar width, with and without shared radial modes, three species
+    "p128_3_4": _profile(128, 3, 4, 16, 2, 96, 3, C1=16, C2=8, K1=8, K2=2, H=344,
+                         Hp=688, S=223, D_out=541),
+    "p128_2_0": _profile(128, 2, 0, 16, 2, 96, 3, C1=16, C2=8, K1=8, K2=2, H=344,
+                         Hp=688, S=216, D_out=522),
 }
