@@ -17,10 +17,18 @@ the 126 MB L2, so consecutive timed steps cannot serve each other from cache.  S
 workloads can be selected with --workload; they fit in L2 and are launch-bound.
 
 The line also carries: "e2e" (same metric driven from host buffers: positions copied from
-pinned host memory and forces copied back every step), "roofline" (dominant kernel class:
-algorithmic FLOPs or bytes over its CUDA-event time, against the measured peaks),
-"kernels" (every class with launches, time share and roofline fraction), "cpu_baseline"
-(the fp64 oracle on a bounded sample, on this box's host cores) and "clocks".
+pinned host memory and forces copied back every step, the list rebuilt at the workload's
+cadence inside the timed region), "roofline" (dominant kernel class: algorithmic FLOPs or
+bytes over its CUDA-event time, against the measured peaks), "kernels" (every class with
+launches, time share and roofline fraction), "workloads" (short runs of the other four of the
+five benchmark systems: rate, time per step, dominant class), "cpu_baseline" (the fp64 oracle
+on a bounded sample, on this box's host cores) and "clocks".
+
+Peaks: HBM and the tensor rate are the measured numbers of MEASURED_PEAKS.json (the MLP
+multiplies half-precision operands, so its roof is the measured 16-bit tensor rate, sustained,
+and its work is the algorithmic 2 flops per multiply-add: the three products per
+multiply-add that carry single precision are this implementation's overhead, not work); the
+FP32 rate is measured in this run by the library's FMA probe.
 """
 
 import argparse
@@ -130,8 +138,10 @@ def work_model(p, n_atoms, e_rc, e_list, one_species=False):
     return {
         "edge_forward": dict(flops=fwd_edge * e_rc, bytes=8 * e_list + n_atoms * (28 + 4 * (S + 2)), pipe="alu"),
         "edge_backward": dict(flops=bwd_edge * e_rc, bytes=(8 + 12) * e_list + n_atoms * (28 + 4 * (S + 2)), pipe="alu"),
-        "mlp_forward": dict(flops=mlp * n_atoms, bytes=4 * n_atoms * (D + 2 * NH * F), pipe="tensor"),
-        "mlp_backward": dict(flops=mlp * n_atoms, bytes=4 * n_atoms * (D + 2 * NH * F), pipe="tensor"),
+        # compulsory bytes of the MLP: the feature rows in, one energy out (forward); the gradient
+        # rows out (backward).  Activations that travel between layers are the implementation's.
+        "mlp_forward": dict(flops=mlp * n_atoms, bytes=n_atoms * (4 * D + 8), pipe="tensor"),
+        "mlp_backward": dict(flops=mlp * n_atoms, bytes=n_atoms * 4 * D, pipe="tensor"),
         "invariants_forward": dict(flops=0, bytes=4 * n_atoms * (S + 2 + D), pipe="hbm"),
         "invariants_backward": dict(flops=0, bytes=4 * n_atoms * (2 * (S + 2) + D), pipe="hbm"),
         "force_assembly": dict(flops=0, bytes=e_list * (12 + 12 + 8) + n_atoms * 72, pipe="hbm"),
@@ -145,20 +155,22 @@ def work_model(p, n_atoms, e_rc, e_list, one_species=False):
 def roofline_entry(name, ms, launches, evals, work, peaks):
     """achieved = algorithmic work of `evals` evaluations / time; against the binding peak."""
     w = work[name]
-    alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12          # TFLOP/s
-    tf32_peak = 0.5 * peaks["bf16_tflops_sustained"]
+    alu_peak = peaks["fp32_tflops"]
+    tensor_peak = peaks["bf16_tflops_sustained"]          # half-precision operands: the 16-bit tensor rate
     t = ms * 1e-3
     if t <= 0:
         return None
     flops, byts = w["flops"] * evals, w["bytes"] * evals
-    t_flop = flops / ((tf32_peak if w["pipe"] == "tensor" else alu_peak) * 1e12) if flops else 0.0
+    t_flop = flops / ((tensor_peak if w["pipe"] == "tensor" else alu_peak) * 1e12) if flops else 0.0
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
     if flops and t_flop >= t_hbm:
-        bound, ach, peak, unit = w["pipe"], flops / t / 1e12, (tf32_peak if w["pipe"] == "tensor" else alu_peak), "TFLOP/s"
+        bound, ach, peak, unit = w["pipe"], flops / t / 1e12, (tensor_peak if w["pipe"] == "tensor" else alu_peak), "TFLOP/s"
+        src = peaks["source"] if w["pipe"] == "tensor" else peaks["fp32_source"]
     else:
-        bound, ach, peak, unit = "hbm", byts / t / 1e9, peaks["hbm_gbs"], "GB/s"
+        bound, ach, peak, unit, src = "hbm", byts / t / 1e9, peaks["hbm_gbs"], "GB/s", peaks["source"]
     return dict(kernel=name, bound=bound, achieved=round(ach, 3), peak=round(peak, 1), unit=unit,
-                frac=round(ach / peak, 4), launches=int(launches), ms_total=round(ms, 3), traffic=None)
+                frac=round(ach / peak, 4), launches=int(launches), ms_total=round(ms, 3), traffic=None,
+                peak_source=src)
 
 
 # ------------------------------------------------------------------ CPU oracle leg
@@ -240,6 +252,141 @@ def job_rate(units_per_rank, ms, world):
 
 # ------------------------------------------------------------------ our arm
 
+class Workload:
+    """One benchmark system on this rank's GPU: model, device state, and the timed loops."""
+
+    def __init__(self, args, name, atoms=0, modes=None, nvt=False):
+        import torch
+
+        from paper_2608_19041_b200 import binding
+        self.torch = torch
+        self.args, self.base_name, self.nvt = args, name, nvt
+        cfg = CONFIGS[name]
+        self.cfg = cfg
+        self.modes = modes
+        self.p = workload_profile(name, modes)
+        # a workload without an MD recipe is timed as repeated single evaluations (energy + forces +
+        # virial of the same frame, list built once): velocities are zero and nothing moves
+        self.static = cfg["md"] is None
+        self.md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=0.0, seed=1, rebuild_every=1 << 30, skin=0.0)
+        desc = dict(cfg["system"])
+        label = name
+        if atoms:
+            # a smaller box of the same recipe (density, exclusion radius, species mix): the size one
+            # node tile of the full workload has, for profiler captures that must stay small
+            if desc.get("kind") == "poisson_disk":
+                desc["atoms"] = int(atoms)
+            elif desc.get("kind") in ("fcc", "bcc", "diamond"):
+                per_cell = {"fcc": 4, "bcc": 2, "diamond": 8}[desc["kind"]]
+                desc["cells"] = max(1, round((atoms / per_cell) ** (1.0 / 3.0)))
+            else:
+                raise SystemExit("--atoms applies to the amorphous and the lattice workloads only")
+            label = f"{label}[atoms={int(atoms)}]"
+        if modes is not None:
+            label = f"{label}[R={modes}]"
+        self.label = label
+        s = make_system(desc, None if self.static else self.md)
+        self.s = s
+        self.N = len(s["pos"])
+        self.model = binding.Model(workload_blob(name, modes), mlp_path=args.mlp_path, node_tile=args.node_tile,
+                                   pair_table_mb=args.pair_table_mb, table_dx=args.table_dx)
+        self.pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
+        self.vel = None if self.static else torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
+        self.types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+        self.skin, self.every, self.dt = self.md["skin"], self.md["rebuild_every"], self.md["dt_ps"]
+        m = self.model
+        m.build_neighbors(self.pos, self.types, s["cell"], s["pbc"], 0.0)
+        self.e_rc = m.query()["n_edges"]
+        m.build_neighbors(self.pos, self.types, s["cell"], s["pbc"], self.skin)
+        self.e_list = m.query()["n_edges"]
+        if not self.static:
+            m.set_md_state(self.pos, self.vel, s["masses"])
+
+    def run_steps(self, k):
+        m = self.model
+        if not self.static:
+            if self.nvt:
+                ep, ek, _ = m.step_nvt(k, self.dt, self.md["temperature"], 100.0 * self.dt, self.every)
+                return ep, ek
+            return m.step(k, self.dt, self.every)
+        out = None
+        for _ in range(k):
+            out = m.compute(self.pos, forces=True, virial=True)
+        return (out["energy"] if out else 0.0), 0.0
+
+    def timed(self, steps, warmup, sync_all, sampler=None):
+        """(ms, e_pot, e_kin, launches): exactly `steps` steps after `warmup`, CUDA events."""
+        torch = self.torch
+        self.run_steps(warmup)
+        l0 = self.model.query()["kernel_launches"]
+        sync_all()
+        if sampler:
+            sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        e_pot, e_kin = self.run_steps(steps)
+        ev1.record()
+        sync_all()
+        return ev0.elapsed_time(ev1), e_pot, e_kin, self.model.query()["kernel_launches"] - l0
+
+    def classes(self, steps, peaks):
+        """Per-class CUDA-event times of `steps` more steps, with each class's roofline entry."""
+        m = self.model
+        m.get_profile()
+        m.set_profiling(True)
+        self.run_steps(steps)
+        prof = m.get_profile()
+        m.set_profiling(False)
+        work = work_model(self.p, self.N, self.e_rc, self.e_list, one_species=len(np.unique(self.s["types"])) == 1)
+        total_ms = sum(v[0] for v in prof.values()) or 1.0
+        kernels = []
+        for cname, (kms, kl) in prof.items():
+            if kl == 0 or cname not in work:
+                continue
+            evals = steps if cname != "neighbor_build" else max(1, kl // 7)
+            ent = roofline_entry(cname, kms, kl, evals, work, peaks)
+            if ent:
+                ent["share"] = round(kms / total_ms, 4)
+                kernels.append(ent)
+        kernels.sort(key=lambda k: -k["ms_total"])
+        return kernels
+
+    def e2e(self, steps, sync_all):
+        """The same metric driven from host buffers through the public calls: every iteration
+        uploads the positions from pinned host memory, evaluates energy, forces and virial, and
+        downloads the forces; the neighbor list is rebuilt at the workload's cadence inside the
+        timed region (the host owns the integrator here, so none runs on the device)."""
+        torch = self.torch
+        m, s, N = self.model, self.s, self.N
+        every = self.every if self.every < (1 << 20) else 0
+        k_e2e = 2 * every if every else max(1, min(steps, 10))
+        host_pos = self.pos.cpu().pin_memory()
+        host_f = torch.empty((N, 3), dtype=torch.float64).pin_memory()
+        dpos = torch.empty_like(self.pos)
+        dpos.copy_(host_pos)
+        m.build_neighbors(dpos, self.types, s["cell"], s["pbc"], self.skin)
+        m.compute(dpos)
+        sync_all()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        builds = 0
+        t0.record()
+        for k in range(1, k_e2e + 1):
+            dpos.copy_(host_pos, non_blocking=True)
+            if every and k % every == 0:
+                m.build_neighbors(dpos, self.types, s["cell"], s["pbc"], self.skin)
+                builds += 1
+            out = m.compute(dpos, forces=True, virial=True)
+            host_f.copy_(out["forces"], non_blocking=True)
+        t1.record()
+        sync_all()
+        return t0.elapsed_time(t1), k_e2e, builds
+
+    def close(self):
+        self.model.close()
+        del self.pos, self.vel, self.types
+        self.torch.cuda.empty_cache()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -252,45 +399,6 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    name = args.workload
-    cfg = CONFIGS[name]
-    modes = args.modes if args.modes >= 0 else None
-    p = workload_profile(name, modes)
-    # a workload without an MD recipe is timed as repeated single evaluations (energy + forces +
-    # virial of the same frame, list built once): velocities are zero and nothing moves
-    static = cfg["md"] is None
-    md = cfg["md"] or dict(steps=1, dt_ps=0.001, temperature=0.0, seed=1, rebuild_every=1 << 30, skin=0.0)
-    desc = dict(cfg["system"])
-    if args.atoms:
-        # a smaller box of the same recipe (density, exclusion radius, species mix): the size one
-        # node tile of the full workload has, for profiler captures that must stay small
-        if desc.get("kind") == "poisson_disk":
-            desc["atoms"] = int(args.atoms)
-        elif desc.get("kind") in ("fcc", "bcc", "diamond"):
-            per_cell = {"fcc": 4, "bcc": 2, "diamond": 8}[desc["kind"]]
-            desc["cells"] = max(1, round((args.atoms / per_cell) ** (1.0 / 3.0)))
-        else:
-            raise SystemExit("--atoms applies to the amorphous and the lattice workloads only")
-        name = f"{name}[atoms={int(args.atoms)}]"
-    s = make_system(desc, None if static else md)
-    N = len(s["pos"])
-    blob = workload_blob(args.workload, modes)
-    if modes is not None:
-        name = f"{name}[R={modes}]"
-    model = binding.Model(blob, mlp_path=args.mlp_path, node_tile=args.node_tile, pair_table_mb=args.pair_table_mb,
-                          table_dx=args.table_dx)
-    pos0 = torch.as_tensor(s["pos"], dtype=torch.float64)
-    pos = pos0.cuda().contiguous()
-    vel = None if static else torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
-    types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
-    skin, every, dt = md["skin"], md["rebuild_every"], md["dt_ps"]
-
-    model.build_neighbors(pos, types, s["cell"], s["pbc"], 0.0)
-    e_rc = model.query()["n_edges"]
-    model.build_neighbors(pos, types, s["cell"], s["pbc"], skin)
-    e_list = model.query()["n_edges"]
-    if not static:
-        model.set_md_state(pos, vel, s["masses"])
 
     def sync_all():
         torch.cuda.synchronize()
@@ -298,81 +406,68 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def run_steps(k):
-        if not static:
-            if args.nvt:
-                ep, ek, _ = model.step_nvt(k, dt, md["temperature"], 100.0 * dt, every)
-                return ep, ek
-            return model.step(k, dt, every)
-        for _ in range(k):
-            out = model.compute(pos, forces=True, virial=True)
-        return out["energy"], 0.0
+    peaks = measured_peaks()
+    # FP32 roof: measured here by the library's FMA probe; the figure derived from unit counts and
+    # the maximum clock (SMs x 128 lanes x 2 x clock) is kept beside it
+    derived = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    try:
+        peaks["fp32_tflops"], peaks["fp32_source"] = binding.probe_fma_peak(), "measured (FMA probe of this run)"
+    except Exception:
+        peaks["fp32_tflops"], peaks["fp32_source"] = derived, "derived (SMs x 128 lanes x 2 x max clock)"
+    peaks["fp32_tflops_derived"] = derived
 
-    run_steps(args.warmup)
-    launches0 = model.query()["kernel_launches"]
+    modes = args.modes if args.modes >= 0 else None
+    w = Workload(args, args.workload, atoms=args.atoms, modes=modes, nvt=args.nvt)
+    N, name, cfg = w.N, w.label, w.cfg
     sampler = ClockSampler(local)
-    sync_all()
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    e_pot, e_kin = run_steps(args.steps)
-    ev1.record()
-    sync_all()
+    ms, e_pot, e_kin, launches = w.timed(args.steps, args.warmup, sync_all, sampler)
     clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    launches = model.query()["kernel_launches"] - launches0
     ms = max_over_ranks(ms, "cuda")
     value = job_rate(N * args.steps, ms, world)
 
     # ---- second pass with per-class events: where the time goes, roofline per class
-    model.get_profile()
-    model.set_profiling(True)
-    run_steps(args.steps)
-    prof = model.get_profile()
-    model.set_profiling(False)
-    peaks = measured_peaks()
-    work = work_model(p, N, e_rc, e_list, one_species=len(np.unique(s["types"])) == 1)
-    total_ms = sum(v[0] for v in prof.values()) or 1.0
-    kernels = []
-    for cname, (kms, kl) in prof.items():
-        if kl == 0 or cname not in work:
-            continue
-        evals = args.steps if cname != "neighbor_build" else max(1, kl // 6)
-        ent = roofline_entry(cname, kms, kl, evals, work, peaks)
-        if ent:
-            ent["share"] = round(kms / total_ms, 4)
-            kernels.append(ent)
-    kernels.sort(key=lambda k: -k["ms_total"])
+    kernels = w.classes(args.steps, peaks)
     dom = dict(kernels[0]) if kernels else None
     if dom:
-        dom["peak_source"] = peaks["source"]
         tile = args.node_tile if args.node_tile > 0 else DEFAULT_NODE_TILE
         dom["traffic"] = load_traffic(args.workload, dom["kernel"], N / max(1, -(-N // tile)))
+        if dom["bound"] == "alu" and clocks["sm_mhz"]:
+            # the same fraction against the FP32 rate at the clock the sampler saw during the run
+            at_clock = peaks["fp32_tflops"] * clocks["sm_mhz"] / peaks["sm_max_mhz"]
+            dom["frac_at_sampled_clock"] = round(dom["achieved"] / at_clock, 4)
+        dom["fp32_peak_derived"] = round(derived, 1)
 
-    # ---- end to end from host buffers: upload positions, evaluate, download forces
-    k_e2e = max(1, min(args.steps, 10))
-    host_pos = pos.cpu().pin_memory()
-    host_f = torch.empty((N, 3), dtype=torch.float64).pin_memory()
-    dpos = torch.empty_like(pos)
-    dpos.copy_(host_pos)
-    model.build_neighbors(dpos, types, s["cell"], s["pbc"], skin)
-    model.compute(dpos)
-    sync_all()
-    t0 = torch.cuda.Event(enable_timing=True)
-    t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for k in range(k_e2e):
-        dpos.copy_(host_pos, non_blocking=True)
-        if k % every == 0 and k > 0:
-            model.build_neighbors(dpos, types, s["cell"], s["pbc"], skin)
-        out = model.compute(dpos, forces=True, virial=True)
-        host_f.copy_(out["forces"], non_blocking=True)
-    t1.record()
-    sync_all()
-    ms_e2e = t0.elapsed_time(t1)
+    # ---- end to end from host buffers
+    ms_e2e, k_e2e, builds = w.e2e(args.steps, sync_all)
     ms_e2e = max_over_ranks(ms_e2e, "cuda")
     e2e = dict(value=job_rate(N * k_e2e, ms_e2e, world), unit="atom-steps/s", h2d_bytes_per_step=N * 24,
-               d2h_bytes_per_step=N * 24 + 80, steps=k_e2e)
+               d2h_bytes_per_step=N * 24 + 80, steps=k_e2e, neighbor_builds=builds,
+               note="host-driven loop: upload positions, evaluate, download forces; list rebuilt at the workload's cadence")
+    static, md, p = w.static, w.md, w.p
+    skin, every, dt = w.skin, w.every, w.dt
+    e_rc, e_list = w.e_rc, w.e_list
+    w.close()
+
+    # ---- the other benchmark systems, short runs (rank 0 of a single-GPU run only)
+    others = None
+    if rank == 0 and world == 1 and not args.no_workloads and not args.atoms and modes is None:
+        others = []
+        for oname in FIVE:
+            if oname == args.workload:
+                continue
+            ow = Workload(args, oname)
+            k = OTHER_STEPS[oname]
+            osamp = ClockSampler(local)
+            oms, _, _, ol = ow.timed(k, max(3, args.warmup), sync_all, osamp)
+            ocl = osamp.stop()
+            ok = ow.classes(k, peaks)
+            top = ok[0] if ok else None
+            others.append(dict(workload=oname, n_atoms=ow.N, value=ow.N * k / (oms * 1e-3), unit="atom-steps/s",
+                               steps=k, ms_per_step=oms / k, gpu_launches=int(ol),
+                               dominant=dict(kernel=top["kernel"], bound=top["bound"], frac=top["frac"],
+                                             share=top["share"]) if top else None,
+                               clocks=dict(sm_mhz=ocl["sm_mhz"], reasons=ocl["reasons"])))
+            ow.close()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -397,13 +492,20 @@ def run_ours(args):
                                 **({"published": pub} if pub else {}),
                                 cache="working set per step exceeds L2" if N >= 100000 else "fits in L2 (launch-bound)"),
                     e_pot_per_atom=e_pot / N, e_kin_per_atom=e_kin / N,
-                    gpu_launches=int(launches), e2e=e2e, roofline=dom, kernels=kernels, cpu_baseline=cpu,
+                    gpu_launches=int(launches), e2e=e2e, roofline=dom, kernels=kernels, workloads=others, cpu_baseline=cpu,
+                    peaks=dict(hbm_gbs=peaks["hbm_gbs"], tensor_16bit_tflops_sustained=peaks["bf16_tflops_sustained"],
+                               fp32_tflops=round(peaks["fp32_tflops"], 2), fp32_source=peaks["fp32_source"],
+                               fp32_tflops_derived=round(derived, 1), source=peaks["source"]),
                     clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"],
                                 samples=clocks["samples"]))
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
+
+FIVE = ["cfg1_al108", "cfg2_cu4000", "cfg3_water32400", "cfg4_hea128k", "cfg5_amorphous1m"]
+# timed steps of the short runs of the other systems (cfg1: single evaluations of one frame)
+OTHER_STEPS = {"cfg1_al108": 200, "cfg2_cu4000": 200, "cfg3_water32400": 100, "cfg4_hea128k": 40, "cfg5_amorphous1m": 10}
 
 CAPTURE_ATOMS = 131072          # size of the box the stored ncu capture ran on
 DEFAULT_NODE_TILE = 524288       # the library's default workspace tile (atoms per launch of the tiled kernels)
@@ -444,6 +546,7 @@ def main():
     ap.add_argument("--nvt", action="store_true", help="time the Nose-Hoover-chain NVT driver instead of NVE")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the short runs of the other benchmark systems")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

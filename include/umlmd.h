@@ -62,6 +62,13 @@ typedef struct umlmd_options {
                             2 and 3 need F % 8 == 0 and fall back to 1 otherwise */
     int32_t  pair_table_mb;  /* device memory, MiB, that per-pair amplitude tables may take
                                 (see umlmd_build_neighbors); 0 = 192, negative = never build them */
+    int32_t  gemm_spin_limit;       /* polls after which a wait inside the tensor-core GEMM's operand
+                                       pipeline gives up (the kernel then finishes with garbage, and the
+                                       call returns UMLMD_E_CUDA "pipeline wait expired"); 0 = 4,000,000 */
+    int32_t  fault_skip_gemm_stage; /* diagnostic for that error path: k > 0 makes the first evaluation
+                                       after umlmd_create leave the k-th operand stage of the first MLP
+                                       layer unloaded, so that exactly such a wait runs out (nothing
+                                       faults or hangs; the handle stays usable); 0 = off */
 } umlmd_options;
 
 /* Structural widths of a model, all derived from (C0, L, R) by the paper's formulas
@@ -106,8 +113,23 @@ int umlmd_profile_widths(int32_t C0, int32_t L, int32_t R, umlmd_info* out);
 int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, void* stream,
                  umlmd_t** out);
 int umlmd_destroy(umlmd_t* h);
+/* Library plumbing, no counterpart in the paper: the model's structural widths (derived by the
+ * paper's width formulas, see umlmd_info), the size of the current list, the device memory the
+ * library holds in this process and the number of kernels this handle has launched. */
 int umlmd_query(const umlmd_t* h, umlmd_info* out);
 const char* umlmd_last_error(const umlmd_t* h);
+
+/*
+ * Device memory, in bytes, that a handle of this model holds after umlmd_build_neighbors,
+ * umlmd_compute and umlmd_set_md_state on a system of N atoms whose list has n_edges entries
+ * (list radius rc + skin): model constants, the neighbor list and its build scratch, one node
+ * tile of evaluation workspace, per-edge gradients and per-atom results.  Known before anything
+ * is allocated (library plumbing, no counterpart in the paper; the paper's memory-scaling note is
+ * the model: a fixed tile workspace plus terms linear in atoms and in edges).  An upper estimate
+ * within a few per cent; per-pair amplitude tables, when the species present are few enough for
+ * them, add at most umlmd_options.pair_table_mb on top.
+ */
+int umlmd_workspace_bytes(const umlmd_t* h, int64_t N, int64_t n_edges, int64_t* bytes);
 
 /*
  * Build the directed neighbor graph of the paper's neighbor-set definition with list
@@ -151,6 +173,18 @@ int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* 
                         int64_t cap, int64_t* n_edges);
 
 /*
+ * The same export (the edge set of the paper's neighbor-set definition, for verification) for the
+ * centres first_row .. first_row + n_rows - 1 only, with 64-bit offsets, so that rows of a list of
+ * any length can be compared entry by entry:
+ *   d_row_ptr [n_rows + 1] int64, always filled: offsets of the rows inside d_src / d_shift
+ *   d_src [cap] int32, d_shift [cap, 3] int8: the neighbor instances (j, n), caller's numbering
+ * *n_edges receives the number of edges of those rows.  Pass cap = 0 (edge buffers may be NULL) to
+ * learn it; UMLMD_E_CAPACITY if the rows hold more than cap edges (what fits has been written).
+ */
+int umlmd_get_neighbor_rows(umlmd_t* h, int64_t first_row, int64_t n_rows, int64_t* d_row_ptr,
+                            int32_t* d_src, int8_t* d_shift, int64_t cap, int64_t* n_edges);
+
+/*
  * Energy, forces and virial for positions d_pos [N,3] (same atoms, species and cell as
  * the last build; each atom within skin/2 of where it was at the build, else
  * UMLMD_E_STALE_NEIGHBORS).
@@ -169,14 +203,19 @@ int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_for
                   double virial[9], double* d_atom_energy);
 
 /*
+ * (Not in the paper, which drives its model from LAMMPS: the integrators here exist because the
+ * benchmark's workloads are MD runs.)
  * Register MD state for umlmd_step: d_pos and d_vel [N,3] double (Angstrom, Angstrom/ps)
  * are advanced in place; mass_per_type is T doubles (amu, host; copied).  N, species and
- * cell are those of the last umlmd_build_neighbors call.
+ * cell are those of the last umlmd_build_neighbors call.  The library keeps the forces of the
+ * registered positions between calls: after editing d_pos by hand, register the state again.
  */
 int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* mass_per_type);
 
 /*
- * Advance nsteps of velocity-Verlet NVE with time step dt_ps.  The neighbor list is
+ * Advance nsteps of velocity-Verlet NVE with time step dt_ps (not in the paper, whose timed runs
+ * are LAMMPS NVT steps; each step runs the paper's whole evaluation path once: v += dt/2 F/m,
+ * r += dt v, evaluate, v += dt/2 F/m, in double precision).  The neighbor list is
  * rebuilt (with the skin of the last build) every rebuild_every steps, counted from the
  * last build; rebuild_every == 0 never rebuilds (a step in which an atom has moved more
  * than skin/2 since the build then fails with UMLMD_E_STALE_NEIGHBORS); rebuild_every < 0
@@ -199,6 +238,17 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
  */
 int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double temperature_K,
                    double t_damp_ps, double* e_pot, double* e_kin, double* e_conserved);
+
+/*
+ * Thermostat state of umlmd_step_nvt, for checkpoints (not in the paper): the chain's positions
+ * eta[3] followed by its velocities v_eta[3] (1/ps).  umlmd_get_nvt_state reads them (zeros
+ * while the chain is at rest); umlmd_set_nvt_state, called after umlmd_set_md_state, restores
+ * them, so that a run continued from saved positions, velocities and chain state repeats the
+ * uninterrupted run exactly when it restarts on a step at which that run rebuilt its list.
+ */
+#define UMLMD_NVT_STATE_DOUBLES 6
+int umlmd_get_nvt_state(umlmd_t* h, double state[UMLMD_NVT_STATE_DOUBLES]);
+int umlmd_set_nvt_state(umlmd_t* h, const double state[UMLMD_NVT_STATE_DOUBLES]);
 
 /*
  * Per-atom virial of the last evaluation that produced forces or the virial (umlmd_compute with
@@ -247,6 +297,15 @@ int umlmd_get_profile(umlmd_t* h, int32_t max_classes, double* ms, int64_t* laun
 const char* umlmd_profile_class_name(int32_t cls);
 
 /*
+ * Measurement aid, not part of the model (the paper has no counterpart): the FP32 fused
+ * multiply-add rate of the current device, in TFLOP/s (2 flops per FMA), from a register-resident
+ * chain of FMAs on every lane, timed with CUDA events on `stream` (best of four launches of about
+ * a millisecond).  The benchmark divides the edge kernels' arithmetic rate by this number.
+ * Allocates four bytes of device memory for the duration of the call and synchronises.
+ */
+int umlmd_probe_fma_peak(double* tflops, void* stream);
+
+/*
  * Kinetic energy sum_i m_i |v_i|^2 / 2 (eV) for callers that must not allocate.  (The
  * paper has no counterpart: its integrator is LAMMPS'.)
  *
@@ -262,13 +321,17 @@ const char* umlmd_profile_class_name(int32_t cls);
  *   N                 atoms, at most UMLMD_STATIC_MAX_ATOMS; more is rejected with
  *                     UMLMD_E_CAPACITY and a message (umlmd_static_last_error)
  *   d_vel             [N,3] double, Angstrom/ps           (device, caller-owned)
- *   d_type            [N] int32 species                   (device, caller-owned)
+ *   d_type            [N] int32 species                   (device, caller-owned); every entry must
+ *                     be a valid index into d_mass_per_type: there is no handle here to check it
+ *                     against, and an entry outside the mass array is an out-of-bounds read
  *   d_mass_per_type   masses in amu indexed by species    (device, caller-owned)
  *   d_e_kin           one double, receives the result     (device, caller-owned)
  *   stream            cudaStream_t as void*; the call only enqueues work
  * The first call on each device looks up the device address of the fixed array (current
  * device = the one the stream belongs to); make that first call before starting any
- * stream capture.  All calls on a device share the array: it keeps the previous call's
+ * stream capture.  The address is remembered per device for the life of the process and
+ * belongs to the device's primary context: do not call this after cudaDeviceReset in the same
+ * process.  All calls on a device share the array: it keeps the previous call's
  * partial sums, every entry that a call reads is first written by that same call so
  * nothing needs clearing, and two calls whose kernels overlap on the GPU (different
  * streams) race on it -- serialise them.

@@ -26,6 +26,7 @@ EXPORTS = [
     "umlmd_step_nvt", "umlmd_atom_virial",
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
     "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
+    "umlmd_probe_fma_peak", "umlmd_get_neighbor_rows", "umlmd_workspace_bytes", "umlmd_get_nvt_state", "umlmd_set_nvt_state",
 ]
 
 
@@ -37,7 +38,8 @@ class UmlmdError(RuntimeError):
 
 class Options(ctypes.Structure):
     _fields_ = [("struct_bytes", ctypes.c_uint32), ("table_dx", ctypes.c_double),
-                ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32), ("pair_table_mb", ctypes.c_int32)]
+                ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32), ("pair_table_mb", ctypes.c_int32),
+                ("gemm_spin_limit", ctypes.c_int32), ("fault_skip_gemm_stage", ctypes.c_int32)]
 
 
 class Info(ctypes.Structure):
@@ -78,6 +80,11 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_profile_class_name.argtypes = [i32]
     lib.umlmd_profile_class_name.restype = ctypes.c_char_p
     lib.umlmd_kinetic_energy_static.argtypes = [i64, vp, vp, vp, vp, vp]
+    lib.umlmd_get_neighbor_rows.argtypes = [vp, i64, i64, vp, vp, vp, i64, ctypes.POINTER(i64)]
+    lib.umlmd_workspace_bytes.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
+    lib.umlmd_get_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
+    lib.umlmd_set_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
+    lib.umlmd_probe_fma_peak.argtypes = [ctypes.POINTER(dbl), vp]
     lib.umlmd_static_last_error.argtypes = []
     lib.umlmd_static_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -105,6 +112,16 @@ def profile_widths(C0, L, R=0):
             ("C1", "C2", "K1", "K2", "S", "D_out", "H", "H_pair")}
 
 
+def probe_fma_peak(stream=None):
+    """FP32 fused multiply-add rate of the current device in TFLOP/s (measured by the library)."""
+    out = ctypes.c_double()
+    st = stream if stream is not None else torch.cuda.current_stream()
+    rc = lib().umlmd_probe_fma_peak(ctypes.byref(out), ctypes.c_void_p(st.cuda_stream))
+    if rc != OK:
+        raise UmlmdError(rc, "umlmd_probe_fma_peak failed")
+    return out.value
+
+
 def _ptr(t):
     return ctypes.c_void_p(t.data_ptr()) if t is not None else None
 
@@ -117,10 +134,12 @@ def _check_dev(t, dtype, name):
 class Model:
     """A DPA4C model on the current CUDA device, created from a weight blob."""
 
-    def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, pair_table_mb=0, stream=None):
+    def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, pair_table_mb=0, stream=None,
+                 gemm_spin_limit=0, fault_skip_gemm_stage=0):
         self._lib = lib()
         self._h = ctypes.c_void_p()
-        opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path), int(pair_table_mb))
+        opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path), int(pair_table_mb),
+                      int(gemm_spin_limit), int(fault_skip_gemm_stage))
         # creation is host-only; a stream is only meaningful when a device is present
         self._stream = stream if stream is not None else (
             torch.cuda.current_stream() if torch.cuda.is_available() else None)
@@ -180,6 +199,43 @@ class Model:
         if rc != OK:
             self._raise(rc)
         return row_ptr, src[:E], shift[:E]
+
+    def get_neighbor_rows(self, first_row, n_rows):
+        """(row_ptr [n_rows+1] int64, src [E], shift [E,3]) of the centres first_row .. first_row+n_rows-1."""
+        ne = ctypes.c_int64()
+        row_ptr = torch.empty(n_rows + 1, dtype=torch.int64, device="cuda")
+        rc = self._lib.umlmd_get_neighbor_rows(self._h, int(first_row), int(n_rows), _ptr(row_ptr), None, None, 0,
+                                               ctypes.byref(ne))
+        if rc != OK:
+            self._raise(rc)
+        E = ne.value
+        src = torch.empty(max(E, 1), dtype=torch.int32, device="cuda")
+        shift = torch.empty((max(E, 1), 3), dtype=torch.int8, device="cuda")
+        rc = self._lib.umlmd_get_neighbor_rows(self._h, int(first_row), int(n_rows), _ptr(row_ptr), _ptr(src), _ptr(shift),
+                                               max(E, 1), ctypes.byref(ne))
+        if rc != OK:
+            self._raise(rc)
+        return row_ptr, src[:E], shift[:E]
+
+    def workspace_bytes(self, n_atoms, n_edges):
+        out = ctypes.c_int64()
+        rc = self._lib.umlmd_workspace_bytes(self._h, int(n_atoms), int(n_edges), ctypes.byref(out))
+        if rc != OK:
+            self._raise(rc)
+        return out.value
+
+    def get_nvt_state(self):
+        st = (ctypes.c_double * 6)()
+        rc = self._lib.umlmd_get_nvt_state(self._h, st)
+        if rc != OK:
+            self._raise(rc)
+        return np.array(list(st), dtype=np.float64)
+
+    def set_nvt_state(self, state):
+        st = (ctypes.c_double * 6)(*[float(x) for x in state])
+        rc = self._lib.umlmd_set_nvt_state(self._h, st)
+        if rc != OK:
+            self._raise(rc)
 
     def atom_virial(self):
         """[N, 3, 3] CUDA tensor: per-atom shares of the virial of the last evaluation with forces."""

@@ -19,6 +19,8 @@ struct umlmd {
     NeighborDev nb;
     int node_tile = 524288;
     int mlp_path = 2;   // tensor-core GEMM wherever it applies, CUDA-core GEMM otherwise
+    int gemm_spin_limit = 0;      // polls before a tensor-core pipeline wait gives up (0 = default)
+    int fault_skip_stage = 0;     // diagnostic, consumed by the first evaluation: see umlmd_options
     bool have_list = false;
     bool on_device = false;
     std::vector<void*> model_allocs;
@@ -196,6 +198,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.hbuf = h->hbuf; ma.e_atom = h->e_atom; ma.path = h->mlp_path; ma.want_grad = want_grad;
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit; ma.fold_x0 = fold_x0;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
+        ma.spin_limit = h->gemm_spin_limit; ma.test_skip_kblock = h->fault_skip_stage;
+        h->fault_skip_stage = 0;                      // one shot
         { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
             { Scope sc(h, kMlpBwd, d.n_hidden); API_CUDA(h, launch_mlp_backward(ma, h->st)); }
@@ -329,6 +333,9 @@ int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, 
         if (opt->node_tile > 0) h->node_tile = opt->node_tile;
         if (opt->mlp_path > 0) h->mlp_path = opt->mlp_path;
         if (opt->pair_table_mb != 0) h->pair_table_budget = opt->pair_table_mb < 0 ? -1 : (int64_t)opt->pair_table_mb << 20;
+        if (opt->gemm_spin_limit < 0 || opt->fault_skip_gemm_stage < 0) { delete h; return UMLMD_E_INVALID_ARG; }
+        h->gemm_spin_limit = opt->gemm_spin_limit;
+        h->fault_skip_stage = opt->fault_skip_gemm_stage;
     }
     int rc = build_host_model(blob, blob_bytes, dx_override, &h->hm, &h->err);
     if (rc != UMLMD_OK) { delete h; return rc; }
@@ -422,6 +429,85 @@ int umlmd_get_neighbors(umlmd_t* h, int32_t* d_row_ptr, int32_t* d_src, int8_t* 
     return UMLMD_OK;
 }
 
+int umlmd_get_neighbor_rows(umlmd_t* h, int64_t first_row, int64_t n_rows, int64_t* d_row_ptr, int32_t* d_src,
+                            int8_t* d_shift, int64_t cap, int64_t* n_edges) {
+    if (!h || !n_edges) return UMLMD_E_INVALID_ARG;
+    if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "no neighbor list built");
+    if (first_row < 0 || n_rows < 0 || first_row + n_rows > h->nb.N) return fail(h, UMLMD_E_INVALID_ARG, "row range outside [0, N)");
+    if (!d_row_ptr) return fail(h, UMLMD_E_INVALID_ARG, "null row offsets");
+    if (cap < 0 || (cap > 0 && (!d_src || !d_shift))) return fail(h, UMLMD_E_INVALID_ARG, "null edge buffers");
+    int rc = neighbor_export_rows(&h->nb, first_row, n_rows, d_row_ptr, d_src, d_shift, cap, h->st, &h->err);
+    if (rc != UMLMD_OK) return rc;
+    int64_t total = 0;
+    API_CUDA(h, cudaMemcpyAsync(&total, d_row_ptr + n_rows, sizeof(total), cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    *n_edges = total;
+    if (cap > 0 && cap < total) return fail(h, UMLMD_E_CAPACITY, "edge buffers smaller than the rows asked for");
+    return UMLMD_OK;
+}
+
+int umlmd_workspace_bytes(const umlmd_t* h, int64_t N, int64_t n_edges, int64_t* bytes) {
+    if (!h || !bytes || N < 0 || n_edges < 0) return UMLMD_E_INVALID_ARG;
+    const Dims& d = h->d;
+    const HostModel& m = h->hm;
+    auto buf = [](int64_t n, int64_t elem) { return (n + 16) * elem; };          // dev_ensure pads by 16 elements
+    auto grown = [](int64_t n, int64_t elem) { return ((int64_t)(n * 1.1) + 16) * elem; };
+    int64_t t = 0;
+    // model constants (uploaded by the first build)
+    auto vec = [&](size_t n, size_t elem) { t += (int64_t)(n * elem + 16); };
+    vec(m.table.size(), 4); vec(m.pairmod.size(), 4); vec(m.X0.size(), 4); vec(m.W1p.size(), 4); vec(m.W2p.size(), 4);
+    vec(m.A1.size(), 4); vec(m.A2.size(), 4); vec(m.mu.size(), 4); vec(m.inv_sigma.size(), 4); vec(m.type_bias.size(), 4);
+    for (int k = 0; k < d.n_hidden; ++k) {
+        vec(m.theta[k].size(), 4); vec(m.thetaT[k].size(), 4); vec(m.bias[k].size(), 4);
+        vec(m.theta_hi[k].size(), 2); vec(m.theta_lo[k].size(), 2); vec(m.thetaT_hi[k].size(), 2); vec(m.thetaT_lo[k].size(), 2);
+    }
+    vec(m.w_head.size(), 4); vec(m.e_ref.size(), 4);
+    if (d.L >= 3) t += 2 * (int64_t)(sizeof(GauntSparse) + 16);
+    t += 8 * (reduce_scratch_doubles(0) + 16) + 8 * 16 + 4 * 4 + 4 * 3 * d.T + 16;
+    // neighbor list: per-atom arrays, cell table (at most 8 N + 64 cells), edges, sort / scan scratch
+    const int64_t A = N + 1;
+    t += buf(3 * A, 8) * 3 + buf(6 * A, 4) + buf(A, 4) * 2 + buf(A + 1, 8) + buf(A, 4) * 4 + buf(A + 1, 4);
+    t += buf(8 * N + 64 + 2, 4);
+    t += grown(n_edges, 4) * 2 + grown(n_edges, 8);
+    t += 16 * A + (2 << 20);
+    // evaluation workspace of one node tile, per-edge gradients, per-atom results, MD forces
+    const int64_t Bt = N < h->node_tile ? N : h->node_tile;
+    const int64_t wmax = d.DP > d.F ? d.DP : d.F;
+    t += buf(Bt * d.SP, 4) + buf(Bt * d.DP, 4) + buf(Bt * d.F * d.n_hidden, 4) + buf(Bt * d.F * 2, 4) + 2 * buf(2 * Bt * wmax, 2);
+    t += grown(3 * n_edges, 4);
+    t += buf(N, 8) + buf(3 * N, 8) + buf(N, 4);
+    const int64_t tiles = Bt > 0 ? (N + Bt - 1) / Bt : 0;
+    t += buf((N / 8 + tiles + 2) * 9, 8);
+    t += buf(3 * N, 8) + 2 * buf(d.T, 8) + buf(2 * kNhcChain + 2, 8);
+    *bytes = t;
+    return UMLMD_OK;
+}
+
+int umlmd_get_nvt_state(umlmd_t* h, double state[UMLMD_NVT_STATE_DOUBLES]) {
+    if (!h || !state) return UMLMD_E_INVALID_ARG;
+    static_assert(UMLMD_NVT_STATE_DOUBLES == 2 * kNhcChain, "thermostat state size");
+    for (int k = 0; k < UMLMD_NVT_STATE_DOUBLES; ++k) state[k] = 0.0;
+    if (!h->d_nhc || h->nhc_reset) return UMLMD_OK;            // chain at rest
+    API_CUDA(h, cudaMemcpyAsync(state, h->d_nhc, sizeof(double) * UMLMD_NVT_STATE_DOUBLES, cudaMemcpyDeviceToHost, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    return UMLMD_OK;
+}
+
+int umlmd_set_nvt_state(umlmd_t* h, const double state[UMLMD_NVT_STATE_DOUBLES]) {
+    if (!h || !state) return UMLMD_E_INVALID_ARG;
+    if (!h->have_md) return fail(h, UMLMD_E_NO_MD_STATE, "umlmd_set_md_state must be called first");
+    for (int k = 0; k < UMLMD_NVT_STATE_DOUBLES; ++k)
+        if (!std::isfinite(state[k])) return fail(h, UMLMD_E_INVALID_ARG, "non-finite thermostat state");
+    if (!h->d_nhc) { int64_t c = 0; API_CUDA(h, dev_ensure(&h->d_nhc, &c, 2 * kNhcChain + 2)); }
+    double full[2 * kNhcChain + 2] = {0};
+    for (int k = 0; k < UMLMD_NVT_STATE_DOUBLES; ++k) full[k] = state[k];
+    full[2 * kNhcChain] = 1.0;
+    API_CUDA(h, cudaMemcpyAsync(h->d_nhc, full, sizeof(full), cudaMemcpyHostToDevice, h->st));
+    API_CUDA(h, cudaStreamSynchronize(h->st));
+    h->nhc_reset = false;
+    return UMLMD_OK;
+}
+
 int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_force, double virial[9],
                   double* d_atom_energy) {
     if (!h) return UMLMD_E_INVALID_ARG;
@@ -489,9 +575,27 @@ static int maybe_rebuild(umlmd_t* h, int rebuild_every) {
         double cell[9];
         for (int k = 0; k < 9; ++k) cell[k] = h->nb.H[k];
         const int pbc[3] = {h->nb.pbc[0], h->nb.pbc[1], h->nb.pbc[2]};
-        return build_list(h, N, h->md_pos, h->type_o, cell, pbc, skin);
+        // The build synchronises the stream anyway (it reads the edge count), so this is the place
+        // to look at what the steps since the previous build reported: a list that went stale, or a
+        // non-finite value, ends the run here instead of after the last step.
+        API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+        int rc = build_list(h, N, h->md_pos, h->type_o, cell, pbc, skin);
+        if (rc != UMLMD_OK) return rc;
+        const int word = *h->h_err;                  // the build has synchronised the stream since the copy
+        if (word) {
+            API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+            return decode_device_errors(h, word);
+        }
     }
     return UMLMD_OK;
+}
+
+// error exit of a stepping loop: the error word must not leak into the next call, and the forces
+// kept for the next step's opening kick no longer match the positions
+static int stop_run(umlmd_t* h, int rc) {
+    h->have_force = false;
+    if (h->d_err) cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st);
+    return rc;
 }
 
 int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* e_pot, double* e_kin) {
@@ -510,14 +614,14 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
         // step's closing half kick
         if (s == 0) { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, nullptr, h->st)); }
         ++h->steps_since_build;
-        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return rc;
-        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return stop_run(h, rc);
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return stop_run(h, rc);
         const bool last = s + 1 == nsteps;
         { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, nullptr, h->st)); }
     }
     { Scope sc(h, kIntegrate, 2); API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st)); }
     rc = fetch_results(h, 11);
-    if (rc != UMLMD_OK) return rc;
+    if (rc != UMLMD_OK) return stop_run(h, rc);
     if (e_pot) *e_pot = h->h_out[0];
     if (e_kin) *e_kin = h->h_out[10];
     return UMLMD_OK;
@@ -557,8 +661,8 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
     for (int s = 0; s < nsteps; ++s) {
         { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, d_scale, h->st)); }
         ++h->steps_since_build;
-        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return rc;
-        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return rc;
+        if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return stop_run(h, rc);
+        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return stop_run(h, rc);
         const bool last = s + 1 == nsteps;
         Scope sc(h, kIntegrate, 4);
         API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, false, nullptr, h->st));
@@ -577,7 +681,7 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
     double chain[2 * M + 2];
     API_CUDA(h, cudaMemcpyAsync(chain, h->d_nhc, sizeof(chain), cudaMemcpyDeviceToHost, h->st));
     rc = fetch_results(h, 10);
-    if (rc != UMLMD_OK) return rc;
+    if (rc != UMLMD_OK) return stop_run(h, rc);
     const double ke = chain[2 * M + 1];
     if (e_pot) *e_pot = h->h_out[0];
     if (e_kin) *e_kin = ke;

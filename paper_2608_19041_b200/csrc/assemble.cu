@@ -4,6 +4,7 @@
 // row, the gradient of each edge minus the gradient of its reverse edge (the reverse-edge
 // map turns the source-sorted view into a gather).  No floating-point atomics anywhere,
 // sums in double, fixed order, so results are bitwise reproducible.
+#include <atomic>
 #include "kernels.h"
 
 namespace umd {
@@ -371,8 +372,11 @@ constexpr int kMaxDevices = 64;
 static __device__ __align__(256) double g_static_partials[kRedMaxBlocks];
 
 // g_static_partials is only a host-side handle in host code; the device address has to be
-// asked for, once per device, with that device current.
-double* g_static_partials_dev[kMaxDevices] = {nullptr};
+// asked for, once per device, with that device current.  The cached addresses are atomics: two
+// host threads may make the first call on a device at the same time (both resolve the same
+// address).  They belong to the device's primary context: after cudaDeviceReset they are stale,
+// which the header states.
+std::atomic<double*> g_static_partials_dev[kMaxDevices];
 thread_local char g_static_err[256] = "";
 
 int static_fail(int code, const char* msg) {
@@ -397,7 +401,8 @@ extern "C" int umlmd_kinetic_energy_static(int64_t N, const double* d_vel, const
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
         return static_fail(UMLMD_E_CUDA, "umlmd_kinetic_energy_static: no current CUDA device");
-    if (!g_static_partials_dev[dev]) {
+    double* partials = g_static_partials_dev[dev].load(std::memory_order_acquire);
+    if (!partials) {
         double* p = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void**)&p, g_static_partials);
         if (e != cudaSuccess || !p) {
@@ -405,12 +410,13 @@ extern "C" int umlmd_kinetic_energy_static(int64_t N, const double* d_vel, const
             snprintf(msg, sizeof(msg), "umlmd_kinetic_energy_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
             return static_fail(UMLMD_E_CUDA, msg);
         }
-        g_static_partials_dev[dev] = p;
+        g_static_partials_dev[dev].store(p, std::memory_order_release);
+        partials = p;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // every partial that the final pass reads is written by the first pass of the same call,
     // so nothing left over from an earlier call needs clearing
-    cudaError_t e = launch_kinetic_energy(N, d_vel, d_type, d_mass_per_type, g_static_partials_dev[dev], d_e_kin, st);
+    cudaError_t e = launch_kinetic_energy(N, d_vel, d_type, d_mass_per_type, partials, d_e_kin, st);
     if (e != cudaSuccess) {
         char msg[200];
         snprintf(msg, sizeof(msg), "umlmd_kinetic_energy_static: launch failed: %s", cudaGetErrorString(e));

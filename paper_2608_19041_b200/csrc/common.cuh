@@ -22,7 +22,7 @@ constexpr double kAccelUnit = 9648.53321;   // (eV/Angstrom/amu) in Angstrom/ps^
 constexpr double kBoltzmann = 8.617333262e-5;
 
 // error word bits set by kernels (read back at synchronisation points)
-enum : int { kErrStale = 1, kErrNonFinite = 2, kErrEdgeOverflow = 4, kErrShiftRange = 8, kErrPipelineTimeout = 16, kErrSpecies = 32 };
+enum : int { kErrStale = 1, kErrNonFinite = 2, kErrShiftRange = 8, kErrPipelineTimeout = 16, kErrSpecies = 32 };
 
 // Widths derived from (C0, L, R): degree-wise channels, probe ranks, feature-state width
 // S, feature-vector width D_out, gated hidden widths, and the flat offsets used by the

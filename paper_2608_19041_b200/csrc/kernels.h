@@ -17,6 +17,10 @@ void neighbor_free(NeighborDev* nb);
 // Export the list in caller numbering (device buffers of the caller).
 int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
                     cudaStream_t st, std::string* err);
+// Rows first .. first + n - 1 of the caller's numbering with 64-bit offsets: d_row_ptr [n + 1] is
+// always filled; edges are copied while they fit `cap` (cap = 0 or null buffers: offsets only).
+int neighbor_export_rows(NeighborDev* nb, int64_t first, int64_t n, int64_t* d_row_ptr, int32_t* d_src,
+                         int8_t* d_shift, int64_t cap, cudaStream_t st, std::string* err);
 // xs[i] = pos[perm[i]] - img[i]*L; flags stale / non-finite atoms in *d_err.
 cudaError_t launch_gather_positions(const NeighborDev& nb, const double* d_pos, int* d_err,
                                     cudaStream_t st);
@@ -90,6 +94,8 @@ struct MlpArgs {
     bool fold_x0;           // tensor-core path: the first C0 feature columns enter through m.type_bias instead of the GEMM
     size_t tc_slot;         // elements per slot
     int* err;               // device error word
+    int spin_limit;         // tensor-core path: polls before a pipeline wait gives up (0 = default)
+    int test_skip_kblock;   // diagnostic, first layer of the forward pass only: see GemmArgs
 };
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad

@@ -137,6 +137,7 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
         // the split kernel), and the epilogue leaves the split of its output in the other slot
         g.A_hi = a.tc_hi + (size_t)(t & 1) * a.tc_slot; g.A_lo = a.tc_lo + (size_t)(t & 1) * a.tc_slot;
         g.a_presplit = t > 0 || (tc && a.desc_presplit); g.err = a.err; g.variant = variant;
+        g.spin_limit = a.spin_limit; g.test_skip_kblock = t == 0 ? a.test_skip_kblock : 0;
         if (tc && t + 1 < NH) {
             g.nxt_hi = a.tc_hi + (size_t)((t + 1) & 1) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)((t + 1) & 1) * a.tc_slot;
             g.ldnxt = F;
@@ -210,7 +211,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.B = a.m.thetaT[t]; g.ldb = F;
         g.Bt_hi = a.m.theta_hi[t]; g.Bt_lo = a.m.theta_lo[t]; g.ldbt = F;
         g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
-        g.a_presplit = tc; g.err = a.err; g.variant = variant;
+        g.a_presplit = tc; g.err = a.err; g.variant = variant; g.spin_limit = a.spin_limit;
         if (tc) { g.nxt_hi = a.tc_hi + (size_t)(1 - sp) * a.tc_slot; g.nxt_lo = a.tc_lo + (size_t)(1 - sp) * a.tc_slot; g.ldnxt = F; }
         sp = 1 - sp;
         if (vec_grad) g.rvec = a.m.w_head; else { g.res = hb[slot]; g.ldres = F; }
@@ -230,7 +231,7 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.B = a.m.thetaT[0]; g.ldb = d.DP;
         g.Bt_hi = a.m.theta_hi[0]; g.Bt_lo = a.m.theta_lo[0]; g.ldbt = F;
         g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
-        g.a_presplit = tc; g.err = a.err; g.variant = variant;
+        g.a_presplit = tc; g.err = a.err; g.variant = variant; g.spin_limit = a.spin_limit;
         if (res0) {
             if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }

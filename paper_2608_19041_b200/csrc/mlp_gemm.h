@@ -52,6 +52,11 @@ struct GemmArgs {
     int lda_split;                // row pitch of A_hi / A_lo (0 = K)
     int variant;                  // tensor-core kernel: 3 = one tile per CTA, otherwise the persistent one
     int* err;                     // device error word (bounded-wait expiry)
+    // tensor-core path: polls before a wait on the operand pipeline gives up (0 = the default, a
+    // fraction of a second), and a diagnostic that makes every CTA leave its k-th operand stage
+    // unloaded (0 = off), so that the give-up path can be exercised: the wait for that stage then
+    // runs out, the kernel returns with kErrPipelineTimeout set, and nothing hangs
+    int spin_limit, test_skip_kblock;
 };
 
 // Logistic function from the hardware base-2 exponential and reciprocal (two transcendental

@@ -67,13 +67,26 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait: flags the error word and returns after kSpinLimit polls
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, int* err) {
-    for (int i = 0; i < kSpinLimit; ++i) {
+// Bounded wait.  After `limit` polls it gives up: the CTA's abort flag is raised, the error word
+// gets kErrPipelineTimeout, and from then on every wait of the CTA returns at once, the producer
+// stops issuing copies and the MMA warp stops issuing instructions, so that a wedged pipeline
+// ends with a wrong result and an error code instead of a hang.  Returns false on that path.
+__device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, int* err, volatile int* abort_flag, int limit) {
+    if (*abort_flag) return false;
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (i > 64) __nanosleep(32);
+    }
+    *abort_flag = 1;
+    if (err) atomicOr(err, kErrPipelineTimeout);
+    return false;
+}
+// plain bounded wait of the shutdown path (no flag, no error: the caller is already giving up)
+__device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity, int limit) {
+    for (int i = 0; i < limit; ++i) {
         if (mbar_try(bar, parity)) return;
         if (i > 64) __nanosleep(32);
     }
-    if (err) atomicOr(err, kErrPipelineTimeout);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
     asm volatile(
@@ -127,8 +140,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t bars = tiles + STAGES * STAGE_BYTES;       // full[s], empty[s], accum, then the tmem slot
-    const uint32_t accum_bar = bars + 8 * (2 * STAGES);
+    const uint32_t accum_bar = bars + 8 * (2 * STAGES), drain_bar = accum_bar + 24;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars - raw) + 8 * (2 * STAGES + 1));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (bars - raw) + 8 * (2 * STAGES + 2));
+    const int limit = g.spin_limit > 0 ? g.spin_limit : kSpinLimit;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int KB = (g.K + BK - 1) / BK;
@@ -136,6 +151,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(bars + 8 * s, 1); mbar_init(bars + 8 * (STAGES + s), 1); }
         mbar_init(accum_bar, 1);
+        mbar_init(drain_bar, 1);
+        *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -150,22 +167,30 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
 
     if (warp == 0) {
         if (lane == 0) {                                   // TMA producer
+            int issued[STAGES];                           // k-block last loaded into each stage (-1: none)
+            for (int s = 0; s < STAGES; ++s) issued[s] = -1;
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % STAGES, u = kb / STAGES;
-                if (u > 0) mbar_wait(bars + 8 * (STAGES + s), (u - 1) & 1, g.err);
+                if (u > 0 && !mbar_wait_a(bars + 8 * (STAGES + s), (u - 1) & 1, g.err, abort_flag, limit)) break;
+                if (*abort_flag) break;
+                if (g.test_skip_kblock && kb == g.test_skip_kblock - 1) continue;   // diagnostic: this stage never arrives
                 const uint32_t full = bars + 8 * s, sa = tiles + s * STAGE_BYTES;
                 mbar_expect_tx(full, STAGE_BYTES);
                 tma_load_2d(sa, &mAh, kb * BK, m0, full);
                 tma_load_2d(sa + TILE_BYTES, &mAl, kb * BK, m0, full);
                 tma_load_2d(sa + 2 * TILE_BYTES, &mBh, kb * BK, n0, full);
                 tma_load_2d(sa + 3 * TILE_BYTES, &mBl, kb * BK, n0, full);
+                issued[s] = kb;
             }
+            if (*abort_flag)                              // giving up: let the copies still in flight land first
+                for (int s = 0; s < STAGES; ++s)
+                    if (issued[s] >= 0) mbar_wait_quiet(bars + 8 * s, (issued[s] / STAGES) & 1, limit);
         }
     } else if (warp == 1) {
         if (lane == 0) {                                   // MMA issuer
             for (int kb = 0; kb < KB; ++kb) {
                 const int s = kb % STAGES, u = kb / STAGES;
-                mbar_wait(bars + 8 * s, u & 1, g.err);
+                if (!mbar_wait_a(bars + 8 * s, u & 1, g.err, abort_flag, limit)) break;
                 tc_fence_after();
                 const uint32_t sa = tiles + s * STAGE_BYTES;
 #pragma unroll
@@ -183,6 +208,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
                 umma_commit(bars + 8 * (STAGES + s));      // frees the stage when these MMAs retire
             }
             umma_commit(accum_bar);
+            if (*abort_flag) {                             // every instruction issued so far has to retire before the
+                umma_commit(drain_bar);                    // tensor memory goes back
+                mbar_wait_quiet(drain_bar, 0, limit);
+            }
         }
     } else {                                               // epilogue: warps 2..5 -> lane quarters 2,3,0,1
         // Tensor memory hands each thread one accumulator row; global memory wants a warp
@@ -191,7 +220,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUten
         // rows with a padded pitch, then walks them row by row, lanes across columns, so
         // every global access of the fused epilogue is one contiguous 512-byte segment.
         const int q = warp & 3;
-        mbar_wait(accum_bar, 0, g.err);
+        mbar_wait_a(accum_bar, 0, g.err, abort_flag, limit);
         tc_fence_after();
         float* stage = reinterpret_cast<float*>(smem_raw + (tiles - raw)) + (size_t)q * 32 * EPITCH;
         const float sc = g.acc_scale;
@@ -307,17 +336,6 @@ constexpr uint32_t P_STAGING_BYTES = P_EPW * 32 * P_SPITCH * 4;
 constexpr int P_SMEM_BYTES = P_STAGES * P_STAGE_BYTES + P_STAGING_BYTES + 1024 + BAR_BYTES;
 constexpr int P_THREADS = (2 + P_EPW) * 32;
 
-// bounded wait that gives up at once after any wait of this CTA has expired
-__device__ __forceinline__ void mbar_wait_a(uint32_t bar, uint32_t parity, int* err, volatile int* abort_flag) {
-    if (*abort_flag) return;
-    for (int i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try(bar, parity)) return;
-        if (i > 64) __nanosleep(32);
-    }
-    *abort_flag = 1;
-    if (err) atomicOr(err, kErrPipelineTimeout);
-}
-
 template <int MODE>
 __global__ void __launch_bounds__(P_THREADS, 1)
 k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUtensorMap mAl,
@@ -330,6 +348,8 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
     const uint32_t acc_full = bars + 8 * (2 * P_STAGES), acc_empty = acc_full + 16;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + (acc_empty + 16 - raw));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (acc_empty + 24 - raw));
+    const uint32_t drain_bar = acc_empty + 32;
+    const int limit = g.spin_limit > 0 ? g.spin_limit : kSpinLimit;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = (g.K + BK - 1) / BK;
     const int ntn = (g.N + BN - 1) / BN, ntm = (g.M + 2 * BM - 1) / (2 * BM);
@@ -338,6 +358,7 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) { mbar_init(bars + 8 * s, 1); mbar_init(bars + 8 * (P_STAGES + s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full + 8 * b, 1); mbar_init(acc_empty + 8 * b, P_EPW); }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -354,11 +375,16 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
     if (warp == 0) {
         if (lane == 0) {                                   // TMA producer
             int gk = 0;
-            for (int it = blockIdx.x; it < items; it += gridDim.x) {
+            int issued[P_STAGES];                         // k-block count of the last load into each stage (-1: none)
+            for (int s = 0; s < P_STAGES; ++s) issued[s] = -1;
+            for (int it = blockIdx.x; it < items && !*abort_flag; it += gridDim.x) {
                 const int m0 = (it / ntn) * 2 * BM, n0 = (it % ntn) * BN;
                 for (int kb = 0; kb < KB; ++kb, ++gk) {
                     const int s = gk % P_STAGES, u = gk / P_STAGES;
-                    if (u > 0) mbar_wait_a(bars + 8 * (P_STAGES + s), (u - 1) & 1, g.err, abort_flag);
+                    if (u > 0 && !mbar_wait_a(bars + 8 * (P_STAGES + s), (u - 1) & 1, g.err, abort_flag, limit)) break;
+                    if (*abort_flag) break;
+                    if (g.test_skip_kblock && gk == g.test_skip_kblock - 1) continue;   // diagnostic: this stage never arrives
+                    issued[s] = gk;
                     const uint32_t full = bars + 8 * s, sa = tiles + s * P_STAGE_BYTES;
                     mbar_expect_tx(full, P_STAGE_BYTES);
                     tma_load_2d(sa, &mAh, kb * BK, m0, full);
@@ -369,18 +395,21 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                     tma_load_2d(sa + 5 * TILE_BYTES, &mBl, kb * BK, n0, full);
                 }
             }
+            if (*abort_flag)                              // giving up: let the copies still in flight land first
+                for (int s = 0; s < P_STAGES; ++s)
+                    if (issued[s] >= 0) mbar_wait_quiet(bars + 8 * s, (issued[s] / P_STAGES) & 1, limit);
         }
     } else if (warp == 1) {
         if (lane == 0) {                                   // MMA issuer
             int gk = 0, li = 0;
-            for (int it = blockIdx.x; it < items; it += gridDim.x, ++li) {
+            for (int it = blockIdx.x; it < items && !*abort_flag; it += gridDim.x, ++li) {
                 const int b = li & 1, v = li >> 1;
-                if (v > 0) mbar_wait_a(acc_empty + 8 * b, (v - 1) & 1, g.err, abort_flag);
+                if (v > 0 && !mbar_wait_a(acc_empty + 8 * b, (v - 1) & 1, g.err, abort_flag, limit)) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem + (uint32_t)(b * 256), d1 = d0 + 128u;
                 for (int kb = 0; kb < KB; ++kb, ++gk) {
                     const int s = gk % P_STAGES, u = gk / P_STAGES;
-                    mbar_wait_a(bars + 8 * s, u & 1, g.err, abort_flag);
+                    if (!mbar_wait_a(bars + 8 * s, u & 1, g.err, abort_flag, limit)) break;
                     tc_fence_after();
                     const uint32_t sa = tiles + s * P_STAGE_BYTES;
 #pragma unroll
@@ -404,6 +433,10 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
                 }
                 umma_commit(acc_full + 8 * b);
             }
+            if (*abort_flag) {                             // every instruction issued so far has to retire before the
+                umma_commit(drain_bar);                    // tensor memory goes back
+                mbar_wait_quiet(drain_bar, 0, limit);
+            }
         }
     } else {                                               // epilogue
         const int e = warp - 2, q = warp & 3, h = (e >> 2) & 1, p = e >> 3;
@@ -415,7 +448,7 @@ k_gemm_tcp(const __grid_constant__ CUtensorMap mAh, const __grid_constant__ CUte
             const int b = li & 1, v = li >> 1;
             const int ct = it % ntn;
             const int mrow0 = (it / ntn) * 2 * BM + h * BM + q * 32, n0 = ct * BN + p * 64;
-            mbar_wait_a(acc_full + 8 * b, v & 1, g.err, abort_flag);
+            mbar_wait_a(acc_full + 8 * b, v & 1, g.err, abort_flag, limit);
             tc_fence_after();
             const uint32_t tacc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 256 + h * 128 + p * 64);
 #pragma unroll 1

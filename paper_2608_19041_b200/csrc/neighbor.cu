@@ -315,6 +315,39 @@ __global__ void k_export_rows(int N, const int* __restrict__ perm, const eidx_t*
     }
 }
 
+// the same export restricted to the centres first .. first + n - 1 of the caller's numbering, with
+// 64-bit row offsets (a list may hold more than 2^31 edges; a range of rows rarely does)
+__global__ void k_export_deg_range(int N, int first, int n, const int* __restrict__ perm,
+                                   const eidx_t* __restrict__ row_ptr, int* __restrict__ deg_o) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) deg_o[n] = 0;
+    if (i >= N) return;
+    const int o = perm[i] - first;
+    if (o >= 0 && o < n) deg_o[o] = (int)(row_ptr[i + 1] - row_ptr[i]);
+}
+
+__global__ void k_export_rows_range(int N, int first, int n, const int* __restrict__ perm,
+                                    const eidx_t* __restrict__ row_ptr, const int* __restrict__ src,
+                                    const int* __restrict__ shift, const long long* __restrict__ row_ptr_o,
+                                    long long cap, int* __restrict__ src_o, signed char* __restrict__ shift_o) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int o = perm[warp] - first;
+    if (o < 0 || o >= n) return;
+    const eidx_t e0 = row_ptr[warp];
+    const int len = (int)(row_ptr[warp + 1] - e0);
+    const long long q0 = row_ptr_o[o];
+    for (int k = lane; k < len; k += 32) {
+        if (q0 + k >= cap) break;
+        const int s = shift[e0 + k];
+        src_o[q0 + k] = perm[src[e0 + k]];
+        shift_o[3 * (size_t)(q0 + k)] = (signed char)(s & 0xff);
+        shift_o[3 * (size_t)(q0 + k) + 1] = (signed char)((s >> 8) & 0xff);
+        shift_o[3 * (size_t)(q0 + k) + 2] = (signed char)((s >> 16) & 0xff);
+    }
+}
+
 struct WidenDeg {
     __host__ __device__ eidx_t operator()(int v) const { return (eidx_t)v; }
 };
@@ -510,6 +543,29 @@ int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t*
     if (nb->E > 0)
         k_export_rows<<<wb, TB, 0, st>>>(N, nb->perm, nb->row_ptr, nb->src, nb->shift, d_row_ptr, d_src,
                                          (signed char*)d_shift);
+    NB_CHECK(cudaGetLastError());
+    return UMLMD_OK;
+}
+
+int neighbor_export_rows(NeighborDev* nb, int64_t first, int64_t n, int64_t* d_row_ptr, int32_t* d_src,
+                         int8_t* d_shift, int64_t cap, cudaStream_t st, std::string* err) {
+    const int N = (int)nb->N;
+    if (n == 0 || N == 0) {
+        NB_CHECK(cudaMemsetAsync(d_row_ptr, 0, sizeof(int64_t), st));
+        return UMLMD_OK;
+    }
+    const int TB = 256;
+    k_export_deg_range<<<(N + TB - 1) / TB, TB, 0, st>>>(N, (int)first, (int)n, nb->perm, nb->row_ptr, nb->deg);
+    auto deg_wide = thrust::make_transform_iterator(static_cast<const int*>(nb->deg), WidenDeg());
+    size_t tmp_bytes = nb->cub_bytes;
+    NB_CHECK(cub::DeviceScan::ExclusiveScan(nb->cub_tmp, tmp_bytes, deg_wide, reinterpret_cast<eidx_t*>(d_row_ptr), cub::Sum(),
+                                            (eidx_t)0, (int)n + 1, st));
+    if (cap > 0 && d_src && d_shift) {
+        const int wb = (N + TB / 32 - 1) / (TB / 32);
+        k_export_rows_range<<<wb, TB, 0, st>>>(N, (int)first, (int)n, nb->perm, nb->row_ptr, nb->src, nb->shift,
+                                               reinterpret_cast<const long long*>(d_row_ptr), (long long)cap, d_src,
+                                               (signed char*)d_shift);
+    }
     NB_CHECK(cudaGetLastError());
     return UMLMD_OK;
 }

@@ -1,0 +1,149 @@
+"""GPU tests of the boundary calls that are not the evaluation itself: the row-range export of the
+neighbor list, the workspace estimate, the thermostat checkpoint, and the give-up path of the
+tensor-core GEMM's bounded waits."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dpa4c as orc
+from workloads import CONFIGS, SMALL_PROFILES, make_blob, make_system, workload_blob
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_19041_b200 import binding
+    return binding
+
+
+def _dev(a, dtype):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=dtype).cuda().contiguous()
+
+
+def _build(blob, s, skin=0.0, **kw):
+    m = _binding().Model(blob, **kw)
+    pos = _dev(s["pos"], torch.float64)
+    types = _dev(s["types"], torch.int32)
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], skin)
+    return m, pos
+
+
+def test_neighbor_rows_by_range_equal_the_full_export():
+    s = make_system(dict(kind="random_box", atoms=300, edges=(21.0, 22.5, 30.0), min_dist=1.5, seed=17, n_types=1,
+                         masses=[1.0], shift=True))
+    N = len(s["pos"])
+    m, _ = _build(make_blob(SMALL_PROFILES["p8_2_0"], seed=1), s, skin=1.0)
+    rp, src, shift = [t.cpu().numpy() for t in m.get_neighbors()]
+    for first, n in [(0, N), (17, 23), (N - 5, 5), (40, 1), (100, 0)]:
+        rp2, src2, shift2 = [t.cpu().numpy() for t in m.get_neighbor_rows(first, n)]
+        assert rp2.dtype == np.int64 and rp2[0] == 0
+        assert np.array_equal(rp2, rp[first:first + n + 1].astype(np.int64) - rp[first])
+        a, b = rp[first], rp[first + n]
+        assert np.array_equal(src2, src[a:b]) and np.array_equal(shift2, shift[a:b])
+    # brute force for a few centres, through the range call alone
+    pos = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    for c, ref in zip((0, 123, N - 1), orc.neighbor_rows(pos, s["cell"], s["pbc"], 7.0, centers=[0, 123, N - 1])):
+        rp2, src2, shift2 = [t.cpu().numpy() for t in m.get_neighbor_rows(c, 1)]
+        ent = np.concatenate([src2[:, None].astype(np.int64), shift2.astype(np.int64)], axis=1)
+        assert np.array_equal(ent[np.lexsort((ent[:, 3], ent[:, 2], ent[:, 1], ent[:, 0]))], ref)
+    # a buffer that is too small is reported, the offsets still come back
+    B = _binding()
+    import ctypes
+    ne = ctypes.c_int64()
+    rp3 = torch.empty(11, dtype=torch.int64, device="cuda")
+    small_src = torch.empty(4, dtype=torch.int32, device="cuda")
+    small_shift = torch.empty((4, 3), dtype=torch.int8, device="cuda")
+    rc = m._lib.umlmd_get_neighbor_rows(m._h, 0, 10, B._ptr(rp3), B._ptr(small_src), B._ptr(small_shift), 4, ctypes.byref(ne))
+    assert rc == -9 and ne.value == rp[10] and rp3[-1].item() == rp[10]
+    with pytest.raises(B.UmlmdError):
+        m.get_neighbor_rows(N - 3, 5)                      # range past the end
+    m.close()
+
+
+def test_workspace_estimate_covers_what_a_run_allocates():
+    name = "cfg2_cu4000"
+    cfg = CONFIGS[name]
+    s = make_system(cfg["system"], cfg["md"])
+    torch.cuda.synchronize()
+    m = _binding().Model(workload_blob(name), pair_table_mb=-1)
+    before = m.query()["device_bytes"]
+    pos, vel = _dev(s["pos"], torch.float64), _dev(s["vel"], torch.float64)
+    types = _dev(s["types"], torch.int32)
+    m.build_neighbors(pos, types, s["cell"], s["pbc"], cfg["md"]["skin"])
+    E = m.query()["n_edges"]
+    est = m.workspace_bytes(len(s["pos"]), E)
+    m.compute(pos)
+    m.set_md_state(pos, vel, s["masses"])
+    m.step_nvt(2, 0.001, 300.0, 0.1, 10)
+    held = m.query()["device_bytes"] - before
+    print(f"workspace of {name}: held {held / 2**20:.1f} MiB, estimate {est / 2**20:.1f} MiB")
+    assert held <= est <= 1.15 * held + (4 << 20)
+    m.close()
+
+
+@pytest.mark.parametrize("variant", ["one_tile", "persistent"])
+def test_expired_pipeline_wait_is_reported_and_the_handle_recovers(variant):
+    # The diagnostic option leaves one operand stage of the first MLP layer unloaded; nothing sets
+    # the barrier the MMA warp then waits on, the shortened wait runs out, the kernel finishes and
+    # the call reports it.  The next evaluation on the same handle is a normal one.
+    if variant == "one_tile":
+        p = SMALL_PROFILES["p32_2_4"]
+        s = make_system(dict(kind="random_box", atoms=150, edges=(12.5, 13.5, 14.0), min_dist=1.7, seed=31,
+                             n_types=p["T"], masses=[1.0] * p["T"]))
+        path = 3
+    else:   # enough rows for the persistent kernel: more than half an item per SM
+        p = SMALL_PROFILES["p8_2_0"]
+        s = make_system(dict(kind="fcc", cells=18, a=4.05, jitter=0.05, seed=5, n_types=p["T"], masses=[1.0] * p["T"]))
+        path = 2
+    blob = make_blob(p, seed=45, bias_scale=0.2, e_ref_scale=0.5)
+    B = _binding()
+    good, pos = _build(blob, s, mlp_path=path)
+    ref = good.compute(pos, atom_energy=True)
+    m, _ = _build(blob, s, mlp_path=path, gemm_spin_limit=20000, fault_skip_gemm_stage=2)
+    with pytest.raises(B.UmlmdError) as e:
+        m.compute(pos)
+    assert e.value.code == -8 and "pipeline wait expired" in str(e.value)
+    out = m.compute(pos, atom_energy=True)                 # the diagnostic is one shot
+    assert out["energy"] == ref["energy"] and torch.equal(out["forces"], ref["forces"])
+    good.close()
+    m.close()
+
+
+def test_thermostat_state_round_trip_continues_a_run_exactly():
+    name = "cfg2_cu4000"
+    cfg = CONFIGS[name]
+    md = cfg["md"]
+    s = make_system(cfg["system"], md)
+    blob = workload_blob(name)
+    T, damp, every = 300.0, 0.05, 10
+
+    def start(p0, v0, chain=None):
+        m = _binding().Model(blob)
+        pos, vel = _dev(p0, torch.float64), _dev(v0, torch.float64)
+        m.build_neighbors(pos, _dev(s["types"], torch.int32), s["cell"], s["pbc"], md["skin"])
+        m.set_md_state(pos, vel, s["masses"])
+        if chain is not None:
+            m.set_nvt_state(chain)
+        return m, pos, vel
+
+    m, pos, vel = start(s["pos"], s["vel"])
+    assert np.all(m.get_nvt_state() == 0.0)                 # at rest
+    m.step_nvt(every, md["dt_ps"], T, damp, every)          # ends on a rebuild step
+    chain = m.get_nvt_state()
+    assert np.abs(chain).max() > 0
+    p_mid, v_mid = pos.cpu().numpy().copy(), vel.cpu().numpy().copy()
+    a = m.step_nvt(every, md["dt_ps"], T, damp, every)
+    pa, va = pos.cpu().numpy(), vel.cpu().numpy()
+    chain_a = m.get_nvt_state()
+    m.close()
+    m2, pos2, vel2 = start(p_mid, v_mid, chain)
+    b = m2.step_nvt(every, md["dt_ps"], T, damp, every)
+    assert np.array_equal(pos2.cpu().numpy(), pa) and np.array_equal(vel2.cpu().numpy(), va)
+    assert a == b and np.array_equal(m2.get_nvt_state(), chain_a)
+    m2.close()
+    # without the chain state the continuation differs
+    m3, pos3, vel3 = start(p_mid, v_mid)
+    m3.step_nvt(every, md["dt_ps"], T, damp, every)
+    assert not np.array_equal(vel3.cpu().numpy(), va)
+    m3.close()

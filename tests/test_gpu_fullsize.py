@@ -180,6 +180,14 @@ def test_more_than_2_31_edges():
     with pytest.raises(_binding().UmlmdError) as e:
         m.get_neighbors()
     assert e.value.code == -9
+    # the row-range export has 64-bit offsets: rows from the start, the middle and the end of the
+    # caller's numbering against brute force
+    pos_w0 = orc.wrap_positions(s["pos"], s["cell"], s["pbc"])
+    for c, ref_row in zip((0, N // 2 + 1, N - 1),
+                          orc.neighbor_rows(pos_w0, s["cell"], s["pbc"], rc + cfg["md"]["skin"], centers=[0, N // 2 + 1, N - 1])):
+        _, rsrc, rshift = m.get_neighbor_rows(c, 1)
+        ent = np.concatenate([rsrc.cpu().numpy()[:, None].astype(np.int64), rshift.cpu().numpy().astype(np.int64)], axis=1)
+        assert np.array_equal(ent[np.lexsort((ent[:, 3], ent[:, 2], ent[:, 1], ent[:, 0]))], ref_row), c
     out = m.compute(pos, atom_energy=True)
     Ei = out["atom_energy"].cpu().numpy()
     F = out["forces"].cpu().numpy()
