@@ -38,7 +38,7 @@ enum {
     UMLMD_OK = 0,
     UMLMD_E_INVALID_ARG = -1,         /* NULL pointer, negative size, bad option            */
     UMLMD_E_BAD_BLOB = -2,            /* magic / version / size mismatch, non-finite weight */
-    UMLMD_E_UNSUPPORTED_PROFILE = -3, /* C0 not in {8,16,32,64,128}, L not in {2,3},
+    UMLMD_E_UNSUPPORTED_PROFILE = -3, /* C0 not in {8,16,32,64,128}, L not in {2,3,4},
                                          R not in {0,2,4,8}, F % 4 != 0, ...                */
     UMLMD_E_UNSUPPORTED_CELL = -4,    /* singular or non-finite cell, non-positive edge,
                                          more than 127 periodic images along a direction     */

@@ -170,7 +170,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
     for (int a0 = 0; a0 < N; a0 += B) {
         const int n = N - a0 < B ? N - a0 : B;
         EdgeArgs ea;
-        ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.type_s = nb.type_s;
+        ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.rec = nb.rec; ea.type_s = nb.type_s;
         ea.table_uni = h->pair_tables ? h->table_uni : nullptr;
         ea.uni_scale = h->uni_scale;
         ea.species_slot = h->d_species + d.T; ea.n_present = (int)h->present.size();
@@ -253,6 +253,7 @@ int ensure_device_model(umlmd_t* h) {
         e = upload(h, g1, &md.g123);
         if (e == cudaSuccess) e = upload(h, g2, &md.g233);
     }
+    if (e == cudaSuccess && h->d.L >= 4) e = upload(h, m.g4, &md.g4);
     void* p = nullptr;
     if (e == cudaSuccess) { e = dev_malloc(&p, sizeof(double) * (reduce_scratch_doubles(0) + 16)); h->scratch = (double*)p; }
     if (e == cudaSuccess) { e = dev_malloc(&p, sizeof(double) * 16); h->d_out = (double*)p; }
@@ -463,6 +464,7 @@ int umlmd_workspace_bytes(const umlmd_t* h, int64_t N, int64_t n_edges, int64_t*
     }
     vec(m.w_head.size(), 4); vec(m.e_ref.size(), 4);
     if (d.L >= 3) t += 2 * (int64_t)(sizeof(GauntSparse) + 16);
+    if (d.L >= 4) t += (int64_t)(5 * sizeof(GauntSparseBig) + 16);
     t += 8 * (reduce_scratch_doubles(0) + 16) + 8 * 16 + 4 * 4 + 4 * 3 * d.T + 16;
     // neighbor list: per-atom arrays, cell table (at most 8 N + 64 cells), edges, sort / scan scratch
     const int64_t A = N + 1;

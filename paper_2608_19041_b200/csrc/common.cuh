@@ -15,9 +15,10 @@
 namespace umd {
 
 constexpr float kEpsReg = 1.0e-7f;     // direction regulariser, Angstrom (edge geometry)
-constexpr int kMaxDeg = 3;             // highest angular degree compiled in
+constexpr int kMaxDeg = 4;             // highest angular degree compiled in
 constexpr int kMaxR = 8;               // most shared radial modes
-constexpr int kMaxGaunt = 96;          // non-zeros kept per generic coupling tensor
+constexpr int kMaxGaunt = 96;          // non-zeros kept per coupling tensor of the degree <= 3 triples
+constexpr int kMaxGauntBig = 256;      // the same for the triples that involve degree 4 (up to 9 x 9 x 9 entries)
 constexpr double kAccelUnit = 9648.53321;   // (eV/Angstrom/amu) in Angstrom/ps^2
 constexpr double kBoltzmann = 8.617333262e-5;
 
@@ -36,6 +37,7 @@ struct Dims {
     int D_out, DP;           // feature-vector width; row stride (multiple of 32)
     int oG[kMaxDeg + 1];     // offsets of vech(G_l) in D
     int oJ112, oJ123, oJ222, oJ233, oPi;
+    int oJ134, oJ224, oJ244, oJ334, oJ444;   // blocks of the triples that exist only for L = 4
     int H, Hp;
     int CP;                  // table channels C0+R rounded up to 4
     int n_rows;              // table intervals
@@ -47,6 +49,11 @@ struct GauntSparse {         // non-zeros of one unit-norm coupling tensor
     int n;
     unsigned char m1[kMaxGaunt], m2[kMaxGaunt], m3[kMaxGaunt];
     float v[kMaxGaunt];
+};
+struct GauntSparseBig {      // the same with room for the degree-4 triples
+    int n;
+    unsigned char m1[kMaxGauntBig], m2[kMaxGauntBig], m3[kMaxGauntBig];
+    float v[kMaxGauntBig];
 };
 
 // Device-resident constants of one model.
@@ -76,6 +83,7 @@ struct ModelDev {
     float b_head;
     GauntSparse* g123;   // device copies (NULL when L < 3)
     GauntSparse* g233;
+    GauntSparseBig* g4;  // [5] device copies of (1,3,4), (2,2,4), (2,4,4), (3,3,4), (4,4,4) (NULL when L < 4)
 };
 
 struct Handle;  // defined in api.cu
@@ -118,6 +126,10 @@ struct NeighborDev {
     int* type_s = nullptr;       // [N] species, sorted order
     double* xs0 = nullptr;       // [N][3] folded positions at build time, sorted order
     double* xs = nullptr;        // [N][3] current positions minus img*L, sorted order
+    // [N][2] the same positions and the species as one 32-byte record per atom for the edge kernels'
+    // neighbour gathers (one sector and two 16-byte loads instead of four scattered loads):
+    // (x_hi, y_hi, z_hi, species bits), (x_lo, y_lo, z_lo, 0) with x = (double)x_hi + (double)x_lo
+    float4* rec = nullptr;
     eidx_t* row_ptr = nullptr;   // [N+1]
     int* src = nullptr;          // [E] sorted index of the neighbour
     int* shift = nullptr;        // [E] packed int8 x3 image n

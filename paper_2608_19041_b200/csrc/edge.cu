@@ -45,7 +45,10 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool 
     const int s = a.shift[e];
     const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff),
               nz = (int)(signed char)((s >> 16) & 0xff);
-    const double* xj = a.xs + 3 * (size_t)j;
+    // the neighbour's record: position as float pairs (exact to 2^-48 of the coordinate) and species
+    const float4 r0 = __ldg(a.rec + 2 * (size_t)j), r1 = __ldg(a.rec + 2 * (size_t)j + 1);
+    const double xj[3] = {(double)r0.x + (double)r1.x, (double)r0.y + (double)r1.y, (double)r0.z + (double)r1.z};
+    const int tj = __float_as_int(r0.w);
     if (a.tri) {        // general cell: the image offset is n . H
         g.dx = (float)((xj[0] + ((nx * a.H[0] + ny * a.H[3]) + nz * a.H[6])) - xi);
         g.dy = (float)((xj[1] + ((nx * a.H[1] + ny * a.H[4]) + nz * a.H[7])) - yi);
@@ -75,17 +78,17 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool 
         // per-pair amplitude tables, one after another: the pair selects the table (ti is
         // already the compact index of the centre's species)
         if (a.n_present > 1) {           // with one species there is one table and no lookup
-            g.pair = ti * a.n_present + a.species_slot[a.type_s[j]];
+            g.pair = ti * a.n_present + a.species_slot[tj];
             g.row += g.pair * a.d.n_rows;
         }
     } else {
-        g.pair = ti * a.d.T + a.type_s[j];
+        g.pair = ti * a.d.T + tj;
     }
     return g;
 }
 
 template <int L>
-__device__ __forceinline__ void harmonics_s1(float x, float y, float z, float* B1, float* B2, float* B3) {
+__device__ __forceinline__ void harmonics_s1(float x, float y, float z, float* B1, float* B2, float* B3, float* B4) {
     const float r3 = 1.7320508075688772f;
     B1[0] = x; B1[1] = y; B1[2] = z;
     B2[0] = r3 * x * y; B2[1] = r3 * y * z; B2[2] = 0.5f * (3.0f * z * z - 1.0f); B2[3] = r3 * x * z;
@@ -100,12 +103,26 @@ __device__ __forceinline__ void harmonics_s1(float x, float y, float z, float* B
         B3[5] = 0.5f * b * z * (x * x - y * y);
         B3[6] = a * x * (x * x - 3.0f * y * y);
     }
+    if (L >= 4) {   // degree four of the supplementary note, |u|^2 = 1
+        const float xx = x * x, yy = y * y, zz = z * z;
+        const float a0 = 2.958039891549808f, a1 = 2.0916500663351889f, a2 = 1.118033988749895f, a3 = 0.7905694150420949f,
+                    a6 = 0.5590169943749475f, a8 = 0.739509972887452f;
+        B4[0] = a0 * x * y * (xx - yy);
+        B4[1] = a1 * y * z * (3.0f * xx - yy);
+        B4[2] = a2 * x * y * (7.0f * zz - 1.0f);
+        B4[3] = a3 * y * z * (7.0f * zz - 3.0f);
+        B4[4] = 0.125f * (35.0f * zz * zz - 30.0f * zz + 3.0f);
+        B4[5] = a3 * x * z * (7.0f * zz - 3.0f);
+        B4[6] = a6 * (xx - yy) * (7.0f * zz - 1.0f);
+        B4[7] = a1 * x * z * (xx - 3.0f * yy);
+        B4[8] = a8 * (xx * xx - 6.0f * xx * yy + yy * yy);
+    }
 }
 
 // sum over l >= 1 of t_lm * grad_u B_lm (|u|^2 = 1 convention)
 template <int L>
 __device__ __forceinline__ void harmonics_grad_contract(float x, float y, float z, const float* t1,
-                                                        const float* t2, const float* t3, float* gx,
+                                                        const float* t2, const float* t3, const float* t4, float* gx,
                                                         float* gy, float* gz) {
     const float r3 = 1.7320508075688772f;
     float ax = t1[0], ay = t1[1], az = t1[2];
@@ -121,6 +138,19 @@ __device__ __forceinline__ void harmonics_grad_contract(float x, float y, float 
               t3[5] * (b * y * z) - t3[6] * (6.0f * a * x * y);
         az += t3[1] * (b * x * y) + t3[2] * (10.0f * c * y * z) + t3[3] * (0.5f * (15.0f * zz - 3.0f)) +
               t3[4] * (10.0f * c * x * z) + t3[5] * (0.5f * b * (xx - yy));
+    }
+    if (L >= 4) {
+        const float xx = x * x, yy = y * y, zz = z * z;
+        const float a0 = 2.958039891549808f, a1 = 2.0916500663351889f, a2 = 1.118033988749895f, a3 = 0.7905694150420949f,
+                    a6 = 0.5590169943749475f, a8 = 0.739509972887452f;
+        const float s7 = 7.0f * zz - 1.0f, s73 = 7.0f * zz - 3.0f, s21 = 21.0f * zz - 3.0f;
+        ax += t4[0] * (a0 * y * (3.0f * xx - yy)) + t4[1] * (6.0f * a1 * x * y * z) + t4[2] * (a2 * y * s7) + t4[5] * (a3 * z * s73) +
+              t4[6] * (2.0f * a6 * x * s7) + t4[7] * (3.0f * a1 * z * (xx - yy)) + t4[8] * (4.0f * a8 * x * (xx - 3.0f * yy));
+        ay += t4[0] * (a0 * x * (xx - 3.0f * yy)) + t4[1] * (3.0f * a1 * z * (xx - yy)) + t4[2] * (a2 * x * s7) + t4[3] * (a3 * z * s73) -
+              t4[6] * (2.0f * a6 * y * s7) - t4[7] * (6.0f * a1 * x * y * z) + t4[8] * (4.0f * a8 * y * (yy - 3.0f * xx));
+        az += t4[1] * (a1 * y * (3.0f * xx - yy)) + t4[2] * (14.0f * a2 * x * y * z) + t4[3] * (a3 * y * s21) +
+              t4[4] * (z * (17.5f * zz - 7.5f)) + t4[5] * (a3 * x * s21) + t4[6] * (14.0f * a6 * z * (xx - yy)) +
+              t4[7] * (a1 * x * (xx - 3.0f * yy));
     }
     *gx = ax; *gy = ay; *gz = az;
 }
@@ -225,7 +255,7 @@ template <int C0, int L, int G = 1> struct Widths {
     static constexpr int LH = LPE / 2;          // parked partial dot products per edge (lanes paired)
     static constexpr int EPI = 32 / LPE;        // edges per replay step
     static constexpr int NL1 = C1 / 4;          // lanes of a group that hold degree-1 channels
-    static constexpr int NHI = 3 * C1 + 5 * C2 + (L >= 3 ? 7 : 0);   // sums of degree >= 1
+    static constexpr int NHI = 3 * C1 + 5 * C2 + (L >= 3 ? 7 : 0) + (L >= 4 ? 9 : 0);   // sums of degree >= 1
     static constexpr int NCH = (NHI + 31) / 32;
     // row pitch (floats) of the per-edge amplitude staging; pitch/4 odd keeps 16-byte
     // accesses of 8 consecutive lanes on distinct bank groups
@@ -339,7 +369,7 @@ k_edge_forward(const EdgeArgs a) {
         __syncwarp();
         // lane = edge: products of degree >= 1, then batch sums by transposition
         float ps[W::C1];
-        float B1[3], B2[5], B3[7];
+        float B1[3], B2[5], B3[7], B4[9];
         float w = 0.f;
         if (lane < nb) {
 #pragma unroll
@@ -349,7 +379,7 @@ k_edge_forward(const EdgeArgs a) {
             }
             const float dx = qd[lane], dy = qd[32 + lane], dz = qd[64 + lane];
             const float inv_rho = 1.0f / sqrtf(dx * dx + dy * dy + dz * dz + kEpsReg * kEpsReg);
-            harmonics_s1<L>(dx * inv_rho, dy * inv_rho, dz * inv_rho, B1, B2, B3);
+            harmonics_s1<L>(dx * inv_rho, dy * inv_rho, dz * inv_rho, B1, B2, B3, B4);
             const float chi = __int_as_float(qes[lane].w);
             w = chi * chi;
         } else {
@@ -361,6 +391,8 @@ k_edge_forward(const EdgeArgs a) {
             for (int q = 0; q < 5; ++q) B2[q] = 0.f;
 #pragma unroll
             for (int q = 0; q < 7; ++q) B3[q] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 9; ++q) B4[q] = 0.f;
         }
         __syncwarp();                           // amplitudes are in registers: reuse the scratch
         int vv = 0;
@@ -391,6 +423,10 @@ k_edge_forward(const EdgeArgs a) {
         if (L >= 3) {
 #pragma unroll
             for (int m = 0; m < 7; ++m) emit(w * B3[m] * ps[0]);
+        }
+        if (L >= 4) {
+#pragma unroll
+            for (int m = 0; m < 9; ++m) emit(w * B4[m] * ps[0]);
         }
     };
 
@@ -493,6 +529,7 @@ k_edge_backward(const EdgeArgs a) {
         const float* H1 = hi_s;
         const float* H2 = H1 + 3 * W::C1;
         const float* H3 = H2 + 5 * W::C2;
+        const float* H4 = H3 + (L >= 3 ? 7 : 0);
 
         auto run_batch = [&](const int nb) {     // the first nb queue slots
             if (HASR) {
@@ -548,8 +585,8 @@ k_edge_backward(const EdgeArgs a) {
                 }
 #pragma unroll
                 for (int k = 0; k < W::C1; ++k) ec[k] = 0.f;
-                float B1[3], B2[5], B3[7], t1[3], t2[5], t3[7];
-                harmonics_s1<L>(gux, guy, guz, B1, B2, B3);
+                float B1[3], B2[5], B3[7], B4[9], t1[3], t2[5], t3[7], t4[9];
+                harmonics_s1<L>(gux, guy, guz, B1, B2, B3, B4);
                 float bt = 0.f;    // sum_lm B_lm t_lm,  t_lm = sum_c psi_c G_lmc
 #pragma unroll
                 for (int m = 0; m < 3; ++m) {
@@ -571,12 +608,18 @@ k_edge_backward(const EdgeArgs a) {
                     if (L >= 3) { const float hv = H3[m]; tm = ps[0] * hv; ec[0] += B3[m] * hv; bt += B3[m] * tm; }
                     t3[m] = tm;
                 }
+#pragma unroll
+                for (int m = 0; m < 9; ++m) {
+                    float tm = 0.f;
+                    if (L >= 4) { const float hv = H4[m]; tm = ps[0] * hv; ec[0] += B4[m] * hv; bt += B4[m] * tm; }
+                    t4[m] = tm;
+                }
                 const float w = chi * chi;
                 float pr1 = 0.f;
 #pragma unroll
                 for (int k = 0; k < W::C1; ++k) pr1 += ec[k] * dps[k];
                 float ux, uy, uz;
-                harmonics_grad_contract<L>(gux, guy, guz, t1, t2, t3, &ux, &uy, &uz);
+                harmonics_grad_contract<L>(gux, guy, guz, t1, t2, t3, t4, &ux, &uy, &uz);
                 const float pux = w * ux, puy = w * uy, puz = w * uz;
                 const float p_rho = chi * sa + w * pr1;
                 const float p_chi = sb + 2.0f * chi * bt;
@@ -668,6 +711,7 @@ cudaError_t dispatch(const EdgeArgs& a, int blocks, cudaStream_t st) {
         return FWD ? launch_fwd_r<C0v, Lv>(a, blocks, st) : launch_bwd_r<C0v, Lv>(a, blocks, st);
     UMLMD_CASE(8, 2) UMLMD_CASE(8, 3) UMLMD_CASE(16, 2) UMLMD_CASE(16, 3) UMLMD_CASE(32, 2)
     UMLMD_CASE(32, 3) UMLMD_CASE(64, 2) UMLMD_CASE(64, 3) UMLMD_CASE(128, 2) UMLMD_CASE(128, 3)
+    UMLMD_CASE(8, 4) UMLMD_CASE(16, 4) UMLMD_CASE(32, 4) UMLMD_CASE(64, 4) UMLMD_CASE(128, 4)
 #undef UMLMD_CASE
     return cudaErrorInvalidValue;
 }

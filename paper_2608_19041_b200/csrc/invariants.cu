@@ -79,10 +79,33 @@ __device__ __forceinline__ float fam3(int a, int b, int c) {
 __device__ __forceinline__ int tri(int p, int q, int C) { return p * C - (p * (p - 1)) / 2 + (q - p); }
 __device__ __forceinline__ int tri_sym(int p, int q, int C) { return p <= q ? tri(p, q, C) : tri(q, p, C); }
 
+// The couplings that involve degree 4 (only present for L = 4, which no timed workload uses) are
+// contracted entry by entry over their non-zeros, all by one warp (lane = atom): operands are
+// [m][atom] columns, X[m * stride].
+__device__ __forceinline__ float contract3(const GauntSparseBig* G, const float* A, int sa, const float* B, int sb,
+                                           const float* C, int sc) {
+    float s = 0.f;
+    const int nn = G->n;
+    for (int n = 0; n < nn; ++n) s += G->v[n] * A[G->m1[n] * sa] * B[G->m2[n] * sb] * C[G->m3[n] * sc];
+    return s;
+}
+// dA += g dJ/dA and likewise for B, C (the operands may be the same array: the shares add up)
+__device__ __forceinline__ void contract3_grad(const GauntSparseBig* G, float g, const float* A, int sa, const float* B,
+                                               int sb, const float* C, int sc, float* dA, float* dB, float* dC) {
+    const int nn = G->n;
+    for (int n = 0; n < nn; ++n) {
+        const int m1 = G->m1[n], m2 = G->m2[n], m3 = G->m3[n];
+        const float v = g * G->v[n], av = A[m1 * sa], bv = B[m2 * sb], cv = C[m3 * sc];
+        dA[m1 * sa] += v * bv * cv;
+        dB[m2 * sb] += v * av * cv;
+        dC[m3 * sc] += v * av * bv;
+    }
+}
+
 template <int C1, int C2, int L>
 struct Plan {                                 // widths and the shared-memory plan, in rows of P floats
     static constexpr int K1 = C2, K2 = 2;
-    static constexpr int nX1 = 3 * C1, nX2 = 5 * C2, nX3 = L >= 3 ? 7 : 0, nX = nX1 + nX2 + nX3;
+    static constexpr int nX1 = 3 * C1, nX2 = 5 * C2, nX3 = L >= 3 ? 7 : 0, nX4 = L >= 4 ? 9 : 0, nX = nX1 + nX2 + nX3 + nX4;
     static constexpr int nZ1 = 3 * K1, nZ2 = 5 * K2, nZ = nZ1 + nZ2;
     static constexpr int nU = L >= 3 ? 3 * K2 : 0, nY = L >= 3 ? 5 : 0;          // forward intermediates
     static constexpr int nPreF = nU + nY;
@@ -92,8 +115,10 @@ struct Plan {                                 // widths and the shared-memory pl
     static constexpr int nMat = C1 * C1 + C2 * C2 + C1 * K1 + C2 * K2;
     static constexpr int nGaunt = L >= 3 ? 2 * (int)((sizeof(GauntSparse) + 3) / 4) : 0;
     static constexpr int nMatP = (nMat + nGaunt + 3) / 4 * 4;                    // matrices come first: 16-byte rows
+    // backward, L = 4: gradient shares of the degree-4 couplings with respect to Z1, Z2, X3 and X4
+    static constexpr int nE4 = L >= 4 ? nZ1 + nZ2 + 7 + 9 : 0;
     static int rows(int TW, int nDS, bool bwd) {
-        return TW + nX + nZ + nDS + (bwd ? nPreB + nX + nX3 + nZ + 18 + nAux : nPreF);
+        return TW + nX + nZ + nDS + (bwd ? nPreB + nX + nX3 + nZ + 18 + nAux + nE4 : nPreF);
     }
     static size_t bytes(int TW, int nDS, bool bwd) { return sizeof(float) * ((size_t)rows(TW, nDS, bwd) * P + nMatP); }
 };
@@ -108,7 +133,7 @@ struct Front {
     float *ST, *XT, *ZZ;
     float *mW1, *mW2, *mA1, *mA2;
     const GauntSparse *G123, *G233;
-    int nv, b0, lane, warp, C0, TW, o1, o2, o3, oS;
+    int nv, b0, lane, warp, C0, TW, o1, o2, o3, o4, oS;
     float iM1;
     double M1d;
 
@@ -161,7 +186,7 @@ struct Front {
         b0 = blockIdx.x * AT;
         nv = a.n - b0 < AT ? a.n - b0 : AT;
         C0 = d.C0; TW = d.SP - C0;
-        o1 = d.offA[1] - C0; o2 = d.offA[2] - C0; o3 = d.offA[3] - C0; oS = d.S - C0;
+        o1 = d.offA[1] - C0; o2 = d.offA[2] - C0; o3 = d.offA[3] - C0; o4 = d.offA[4] - C0; oS = d.S - C0;
         // state slice: a warp reads 32 consecutive entries of one atom's row; four atoms'
         // loads are issued before the first store
         const float* src = a.state + (size_t)b0 * d.SP + C0;
@@ -181,14 +206,17 @@ struct Front {
         __syncthreads();
         M1d = sqrt(0.25 + (double)ST[(oS + 1) * P + lane] + (double)ST[(oS + 3) * P + lane]);
         iM1 = (float)(1.0 / M1d);
-        for (int u = warp; u < 9; u += NW) {
+        for (int u = warp; u < 10; u += NW) {
             if (u < 3) align_row<C1, K1>(ST + (o1 + u * C1) * P + lane, mW1, mA1, XT + u * C1 * P + lane, ZZ + u * K1 * P + lane);
             else if (u < 8)
                 align_row<C2, K2>(ST + (o2 + (u - 3) * C2) * P + lane, mW2, mA2, XT + (PL::nX1 + (u - 3) * C2) * P + lane,
                                   ZZ + (PL::nZ1 + (u - 3) * K2) * P + lane);
-            else if (L >= 3) {
+            else if (u == 8 && L >= 3) {
 #pragma unroll
                 for (int mm = 0; mm < 7; ++mm) XT[(PL::nX1 + PL::nX2 + mm) * P + lane] = ST[(o3 + mm) * P + lane] * iM1;
+            } else if (u == 9 && L >= 4) {
+#pragma unroll
+                for (int mm = 0; mm < 9; ++mm) XT[(PL::nX1 + PL::nX2 + PL::nX3 + mm) * P + lane] = ST[(o4 + mm) * P + lane] * iM1;
             }
         }
         __syncthreads();
@@ -409,6 +437,24 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
             }
         }
     }
+    if (L >= 4) {   // squared norm of the degree-4 row and the five couplings that involve it
+        if (TAKE()) {
+            const float* X4 = XT + (PL::nX1 + PL::nX2 + PL::nX3) * P + lane;
+            const GauntSparseBig* G4 = m.g4;
+            float s = 0.f;
+#pragma unroll
+            for (int mm = 0; mm < 9; ++mm) s += X4[mm * P] * X4[mm * P];
+            DSK(d.oG[4]) = s;
+            for (int k1 = 0; k1 < K1; ++k1) DSK(d.oJ134 + k1) = contract3(G4 + 0, Z1 + k1 * P, K1 * P, X3, P, X4, P);
+            int k = d.oJ224;
+            for (int e1 = 0; e1 < K2; ++e1)
+                for (int e2 = e1; e2 < K2; ++e2)
+                    DSK(k++) = (e1 == e2 ? 1.0f : kR2) * contract3(G4 + 1, Z2 + e1 * P, K2 * P, Z2 + e2 * P, K2 * P, X4, P);
+            for (int e = 0; e < K2; ++e) DSK(d.oJ244 + e) = contract3(G4 + 2, Z2 + e * P, K2 * P, X4, P, X4, P);
+            DSK(d.oJ334) = contract3(G4 + 3, X3, P, X3, P, X4, P);
+            DSK(d.oJ444) = contract3(G4 + 4, X4, P, X4, P, X4, P);
+        }
+    }
     if (TAKE()) {   // (2,2,2): -sqrt(12/35) tr(Q Q Q), non-decreasing index triples
         int k = d.oJ222;
 #pragma unroll
@@ -500,7 +546,11 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     float* GX = PRE + PL::nPreB * P;               // dE/dXt (degree-3 rows twice: the two couplings' shares)
     float* DZ = GX + (PL::nX + PL::nX3) * P;
     float* DQ = DZ + PL::nZ * P;
-    float* AUX = DQ + 18 * P;                      // row 0: sum_c X_0 dE/dX_0; rows 1..9: partial dots
+    float* AUX = DQ + 18 * P;                      // row 0: sum_c X_0 dE/dX_0; rows 1..10: partial dots
+    float* E1 = AUX + PL::nAux * P;                // L = 4: shares of the degree-4 couplings in dE/dZ1, dE/dZ2,
+    float* E2 = E1 + PL::nZ1 * P;                  // dE/dX3 and the whole of dE/dX4
+    float* E3 = E2 + PL::nZ2 * P;
+    float* E4 = E3 + 7 * P;
     float* Ws = PRE + PL::nPreF * P;               // [m1 * K2 + e]
     float* Zg = Ws + PL::nW * P;                   // [m1]
     float* YQ = Zg + PL::nZg * P;                  // [(e * K1 + k) * 3 + m]
@@ -564,6 +614,29 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
             const float g0 = DSK(d.oJ233), g1 = DSK(d.oJ233 + 1);
 #pragma unroll
             for (int m1 = 0; m1 < 5; ++m1) Zg[m1 * P + lane] = g0 * Z2[(m1 * K2) * P] + g1 * Z2[(m1 * K2 + 1) * P];
+        }
+    }
+    if (L >= 4) {
+        if (TAKE()) {      // all gradient shares of the couplings that involve degree 4, by this one warp
+            const float* X4 = XT + (PL::nX1 + PL::nX2 + PL::nX3) * P + lane;
+            const GauntSparseBig* G4 = m.g4;
+            float* e1 = E1 + lane; float* e2 = E2 + lane; float* e3 = E3 + lane; float* e4 = E4 + lane;
+            for (int r = 0; r < PL::nZ1; ++r) e1[r * P] = 0.f;
+            for (int r = 0; r < PL::nZ2; ++r) e2[r * P] = 0.f;
+            for (int r = 0; r < 7; ++r) e3[r * P] = 0.f;
+            const float g4n = 2.0f * DSK(d.oG[4]);
+            for (int mm = 0; mm < 9; ++mm) e4[mm * P] = g4n * X4[mm * P];
+            for (int k1 = 0; k1 < K1; ++k1)
+                contract3_grad(G4 + 0, DSK(d.oJ134 + k1), Z1 + k1 * P, K1 * P, X3, P, X4, P, e1 + k1 * P, e3, e4);
+            int k = d.oJ224;
+            for (int ea = 0; ea < K2; ++ea)
+                for (int eb = ea; eb < K2; ++eb)
+                    contract3_grad(G4 + 1, DSK(k++) * (ea == eb ? 1.0f : kR2), Z2 + ea * P, K2 * P, Z2 + eb * P, K2 * P, X4, P,
+                                   e2 + ea * P, e2 + eb * P, e4);
+            for (int e = 0; e < K2; ++e)
+                contract3_grad(G4 + 2, DSK(d.oJ244 + e), Z2 + e * P, K2 * P, X4, P, X4, P, e2 + e * P, e4, e4);
+            contract3_grad(G4 + 3, DSK(d.oJ334), X3, P, X3, P, X4, P, e3, e3, e4);
+            contract3_grad(G4 + 4, DSK(d.oJ444), X4, P, X4, P, X4, P, e4, e4, e4);
         }
     }
 #pragma unroll
@@ -698,6 +771,10 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
                 for (int mm = 0; mm < 3; ++mm) acc[mm] += g * PRE[(mm * K2 + e) * P + lane];
             }
         }
+        if (L >= 4) {
+#pragma unroll
+            for (int mm = 0; mm < 3; ++mm) acc[mm] += E1[(mm * K1 + k) * P + lane];
+        }
 #pragma unroll
         for (int mm = 0; mm < 3; ++mm) DZ[(mm * K1 + k) * P + lane] = acc[mm];
     }
@@ -773,13 +850,14 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
             else if (m2 == 2) add = kInvR6 * (2.0f * q[8 * P] - q[0] - q[4 * P]);
             else if (m2 == 3) add = kInvR2 * (q[2 * P] + q[6 * P]);
             else add = kInvR2 * (q[0] - q[4 * P]);
+            if (L >= 4) add += E2[(m2 * K2 + e) * P + lane];
             DZ[(PL::nZ1 + m2 * K2 + e) * P + lane] = acc[e] + add;
         }
     }
     __syncthreads();
 
     // ---- probes and alignment transposed, row by row; dot1 = sum dXt . Xt = sum dX . X --
-    for (int u = 0; u < 9; ++u) {
+    for (int u = 0; u < 10; ++u) {
         if (!TAKE()) continue;
         float dot = 0.f;
         if (u < 3)
@@ -788,12 +866,21 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
         else if (u < 8)
             dot = back_row<C2, K2>(GX + (PL::nX1 + (u - 3) * C2) * P + lane, DZ + (PL::nZ1 + (u - 3) * K2) * P + lane, f.mA2,
                                    f.mW2, X2 + ((u - 3) * C2) * P, ST + (f.o2 + (u - 3) * C2) * P + lane, f.iM1);
-        else if (L >= 3) {
+        else if (u == 8 && L >= 3) {
 #pragma unroll
             for (int mm = 0; mm < 7; ++mm) {
-                const float g = GX[(PL::nX1 + PL::nX2 + mm) * P + lane] + GX[(PL::nX + mm) * P + lane];
+                float g = GX[(PL::nX1 + PL::nX2 + mm) * P + lane] + GX[(PL::nX + mm) * P + lane];
+                if (L >= 4) g += E3[mm * P + lane];
                 dot += g * X3[mm * P];
                 ST[(f.o3 + mm) * P + lane] = g * f.iM1;
+            }
+        } else if (u == 9 && L >= 4) {
+            const float* X4 = XT + (PL::nX1 + PL::nX2 + PL::nX3) * P + lane;
+#pragma unroll
+            for (int mm = 0; mm < 9; ++mm) {
+                const float g = E4[mm * P + lane];
+                dot += g * X4[mm * P];
+                ST[(f.o4 + mm) * P + lane] = g * f.iM1;
             }
         }
         AUX[(1 + u) * P + lane] = dot;
@@ -802,7 +889,7 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     if (warp == 0) {   // gradients of the two sums of squared envelopes, fixed summation order
         float dot1 = 0.f;
 #pragma unroll
-        for (int u = 0; u < 9; ++u) dot1 += AUX[(1 + u) * P + lane];
+        for (int u = 0; u < 10; ++u) dot1 += AUX[(1 + u) * P + lane];
         const float iM0 = (float)(1.0 / f.M0_of(lane));
         const float dM0 = DSK(2 * C0), dM1 = DSK(2 * C0 + 1), dot0 = AUX[lane];
         ST[f.oS * P + lane] = (dM0 - dot0 * iM0) * 0.5f * iM0;
@@ -840,7 +927,7 @@ cudaError_t dispatch(const InvArgs& a, cudaStream_t st) {
         return cudaGetLastError();                                                              \
     }
     UMLMD_CASE(4, 4, 2) UMLMD_CASE(4, 4, 3) UMLMD_CASE(8, 4, 2) UMLMD_CASE(8, 4, 3)
-    UMLMD_CASE(16, 8, 2) UMLMD_CASE(16, 8, 3)
+    UMLMD_CASE(16, 8, 2) UMLMD_CASE(16, 8, 3) UMLMD_CASE(4, 4, 4) UMLMD_CASE(8, 4, 4) UMLMD_CASE(16, 8, 4)
 #undef UMLMD_CASE
     return cudaErrorInvalidValue;
 }

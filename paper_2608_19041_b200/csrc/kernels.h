@@ -31,6 +31,7 @@ struct EdgeArgs {
     const float* table;
     const float* pairmod;
     const double* xs;       // [N][3] sorted positions
+    const float4* rec;      // [N][2] positions (as float pairs) and species, one record per atom
     const int* type_s;
     const eidx_t* row_ptr;
     const int* src;

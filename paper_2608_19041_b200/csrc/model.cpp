@@ -42,8 +42,8 @@ inline void j0_derivs(double x, double* j, double* j1) {
     }
 }
 
-// real Cartesian harmonics up to degree 3 for a unit vector, s = |u|^2 kept
-void harmonics_host(const double u[3], double B1[3], double B2[5], double B3[7]) {
+// real Cartesian harmonics up to degree 4 for a unit vector, s = |u|^2 kept
+void harmonics_host(const double u[3], double B1[3], double B2[5], double B3[7], double B4[9]) {
     const double x = u[0], y = u[1], z = u[2], s = x * x + y * y + z * z;
     B1[0] = x; B1[1] = y; B1[2] = z;
     const double r3 = std::sqrt(3.0);
@@ -57,6 +57,16 @@ void harmonics_host(const double u[3], double B1[3], double B2[5], double B3[7])
     B3[4] = c * x * (5 * z * z - s);
     B3[5] = 0.5 * b * z * (x * x - y * y);
     B3[6] = a * x * (x * x - 3 * y * y);
+    const double r35 = std::sqrt(35.0), r70 = std::sqrt(70.0), r10 = std::sqrt(10.0), r5 = std::sqrt(5.0);
+    B4[0] = 0.5 * r35 * x * y * (x * x - y * y);
+    B4[1] = 0.25 * r70 * y * z * (3 * x * x - y * y);
+    B4[2] = 0.5 * r5 * x * y * (7 * z * z - s);
+    B4[3] = 0.25 * r10 * y * z * (7 * z * z - 3 * s);
+    B4[4] = 0.125 * (35 * z * z * z * z - 30 * z * z * s + 3 * s * s);
+    B4[5] = 0.25 * r10 * x * z * (7 * z * z - 3 * s);
+    B4[6] = 0.25 * r5 * (x * x - y * y) * (7 * z * z - s);
+    B4[7] = 0.25 * r70 * x * z * (x * x - 3 * y * y);
+    B4[8] = 0.125 * r35 * (x * x * x * x - 6 * x * x * y * y + y * y * y * y);
 }
 
 // Gauss-Legendre nodes and weights on [-1, 1] by Newton iteration
@@ -81,7 +91,11 @@ void gauss_legendre(int n, std::vector<double>* xs, std::vector<double>* ws) {
     }
 }
 
-bool gaunt_sparse(int l1, int l2, int l3, GauntSparse* out) {
+// non-zeros of the unit-norm coupling of degrees (l1, l2, l3), sign -1: the product of three
+// harmonics has degree at most 12, which 16 Gauss-Legendre nodes in cos(theta) times 32 equally
+// spaced azimuths integrate exactly
+template <typename Sparse, int CAP>
+bool gaunt_sparse(int l1, int l2, int l3, Sparse* out) {
     const int n1 = 2 * l1 + 1, n2 = 2 * l2 + 1, n3 = 2 * l3 + 1;
     std::vector<double> I(n1 * n2 * n3, 0.0), xs, ws;
     const int nth = 16, nph = 32;
@@ -92,9 +106,9 @@ bool gaunt_sparse(int l1, int l2, int l3, GauntSparse* out) {
             const double ph = (b + 0.5) * (2.0 * M_PI / nph);
             const double u[3] = {st * std::cos(ph), st * std::sin(ph), ct};
             const double w = ws[a] * (2.0 * M_PI / nph);
-            double B1[3], B2[5], B3[7];
-            harmonics_host(u, B1, B2, B3);
-            const double* Bs[4] = {nullptr, B1, B2, B3};
+            double B1[3], B2[5], B3[7], B4[9];
+            harmonics_host(u, B1, B2, B3, B4);
+            const double* Bs[5] = {nullptr, B1, B2, B3, B4};
             for (int i = 0; i < n1; ++i)
                 for (int j = 0; j < n2; ++j)
                     for (int k = 0; k < n3; ++k)
@@ -110,7 +124,7 @@ bool gaunt_sparse(int l1, int l2, int l3, GauntSparse* out) {
             for (int k = 0; k < n3; ++k) {
                 const double v = -I[(i * n2 + j) * n3 + k] / nrm;
                 if (std::fabs(v) > 1e-12) {
-                    if (out->n >= kMaxGaunt) return false;
+                    if (out->n >= CAP) return false;
                     out->m1[out->n] = (unsigned char)i;
                     out->m2[out->n] = (unsigned char)j;
                     out->m3[out->n] = (unsigned char)k;
@@ -135,8 +149,8 @@ bool derive_dims(int C0, int L, int R, Dims* d) {
     if (!(R == 0 || R == 2 || R == 4 || R == 8)) return false;
     std::memset(d, 0, sizeof(*d));
     d->C0 = C0; d->L = L; d->R = R;
-    d->C[0] = C0; d->C[1] = C1; d->C[2] = C1 / 2 > 4 ? C1 / 2 : 4; d->C[3] = 1;
-    d->K[0] = 0; d->K[1] = d->C[2]; d->K[2] = 2; d->K[3] = 1;
+    d->C[0] = C0; d->C[1] = C1; d->C[2] = C1 / 2 > 4 ? C1 / 2 : 4; d->C[3] = 1; d->C[4] = 1;
+    d->K[0] = 0; d->K[1] = d->C[2]; d->K[2] = 2; d->K[3] = 1; d->K[4] = 1;
     int off = 0;
     for (int l = 0; l <= L; ++l) { d->offA[l] = off; off += (2 * l + 1) * d->C[l]; }
     d->S = off;
@@ -144,10 +158,16 @@ bool derive_dims(int C0, int L, int R, Dims* d) {
     int o = 2 * C0 + 2;
     for (int l = 1; l <= L; ++l) { d->oG[l] = o; o += d->C[l] * (d->C[l] + 1) / 2; }
     const int K1 = d->K[1], K2 = d->K[2];
+    // bispectrum blocks in lexicographic order of the degree triples; single probes at degrees 3, 4
     d->oJ112 = o; o += K1 * (K1 + 1) / 2 * K2;
     d->oJ123 = o; if (L >= 3) o += K1 * K2;
+    d->oJ134 = o; if (L >= 4) o += K1;
     d->oJ222 = o; o += K2 * (K2 + 1) * (K2 + 2) / 6;
+    d->oJ224 = o; if (L >= 4) o += K2 * (K2 + 1) / 2;
     d->oJ233 = o; if (L >= 3) o += K2;
+    d->oJ244 = o; if (L >= 4) o += K2;
+    d->oJ334 = o; if (L >= 4) o += 1;
+    d->oJ444 = o; if (L >= 4) o += 1;
     d->oPi = o; o += K1 * K2;
     d->D_out = o;
     d->DP = round_up(o, 32);
@@ -173,7 +193,7 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
     const bool gaussian = u[8] == 1;
     Dims& d = m->d;
     if (!derive_dims(C0, L, R, &d)) {
-        *err = "unsupported (C0, L, R): C0 in {8,16,32,64,128}, L in {2,3}, R in {0,2,4,8}";
+        *err = "unsupported (C0, L, R): C0 in {8,16,32,64,128}, L in {2,3,4}, R in {0,2,4,8}";
         return UMLMD_E_UNSUPPORTED_PROFILE;
     }
     if (N_rbf < 1 || N_rbf > 64 || NH < 1 || NH > 8 || F < 4 || F % 4 != 0 || F > 4096 || T < 1 ||
@@ -430,10 +450,20 @@ int build_host_model(const void* blob_v, size_t bytes, double dx_override, HostM
     // ---- Gaunt couplings of the generic triples ------------------------------------
     m->g123.n = 0; m->g233.n = 0;
     if (L >= 3) {
-        if (!gaunt_sparse(1, 2, 3, &m->g123) || !gaunt_sparse(2, 3, 3, &m->g233)) {
+        if (!gaunt_sparse<GauntSparse, kMaxGaunt>(1, 2, 3, &m->g123) || !gaunt_sparse<GauntSparse, kMaxGaunt>(2, 3, 3, &m->g233)) {
             *err = "coupling tensor has more non-zeros than reserved";
             return UMLMD_E_UNSUPPORTED_PROFILE;
         }
+    }
+    m->g4.clear();
+    if (L >= 4) {
+        const int tr[5][3] = {{1, 3, 4}, {2, 2, 4}, {2, 4, 4}, {3, 3, 4}, {4, 4, 4}};
+        m->g4.resize(5);
+        for (int k = 0; k < 5; ++k)
+            if (!gaunt_sparse<GauntSparseBig, kMaxGauntBig>(tr[k][0], tr[k][1], tr[k][2], &m->g4[k])) {
+                *err = "coupling tensor has more non-zeros than reserved";
+                return UMLMD_E_UNSUPPORTED_PROFILE;
+            }
     }
     return UMLMD_OK;
 }

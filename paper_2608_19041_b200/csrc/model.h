@@ -27,6 +27,7 @@ struct HostModel {
     std::vector<float> w_head, e_ref;
     float b_head = 0;
     GauntSparse g123, g233;
+    std::vector<GauntSparseBig> g4;   // (1,3,4), (2,2,4), (2,4,4), (3,3,4), (4,4,4) when L = 4
 };
 
 // Fills `d` widths for (C0, L, R); false when the triple is unsupported.

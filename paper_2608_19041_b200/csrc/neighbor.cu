@@ -267,22 +267,27 @@ __global__ void k_reverse_map(int N, int sorted, const eidx_t* __restrict__ row_
 
 __global__ void k_gather_positions(int N, const int* __restrict__ perm, const int* __restrict__ img,
                                    const double* __restrict__ pos, const double* __restrict__ xs0,
-                                   CellRows H, double max_disp2,
-                                   double* __restrict__ xs, int* __restrict__ err) {
+                                   CellRows H, double max_disp2, const int* __restrict__ type_s,
+                                   double* __restrict__ xs, float4* __restrict__ rec, int* __restrict__ err) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     const int o = perm[i];
     const double n0 = (double)img[3 * (size_t)i], n1 = (double)img[3 * (size_t)i + 1], n2 = (double)img[3 * (size_t)i + 2];
     double d2 = 0;
     bool bad = false;
+    float hi[3], lo[3];
     for (int k = 0; k < 3; ++k) {
         const double x = H.tri ? pos[3 * (size_t)o + k] - ((n0 * H.h[k] + n1 * H.h[3 + k]) + n2 * H.h[6 + k])
                                : pos[3 * (size_t)o + k] - (double)img[3 * (size_t)i + k] * H.h[4 * k];
         if (!isfinite(x)) bad = true;
         xs[3 * (size_t)i + k] = x;
+        hi[k] = (float)x;
+        lo[k] = (float)(x - (double)hi[k]);
         const double d = x - xs0[3 * (size_t)i + k];
         d2 += d * d;
     }
+    rec[2 * (size_t)i] = make_float4(hi[0], hi[1], hi[2], __int_as_float(type_s[i]));
+    rec[2 * (size_t)i + 1] = make_float4(lo[0], lo[1], lo[2], 0.f);
     if (bad) atomicOr(err, kErrNonFinite);
     else if (d2 > max_disp2) atomicOr(err, kErrStale);
 }
@@ -364,7 +369,7 @@ struct WidenDeg {
 }  // namespace
 
 void neighbor_free(NeighborDev* nb) {
-    void* ptrs[] = {nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
+    void* ptrs[] = {nb->rec, nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
                     nb->shift, nb->rev, nb->key, nb->key2, nb->idx, nb->idx2, nb->cell_start, nb->deg,
                     nb->cub_tmp};
     for (void* p : ptrs)
@@ -461,6 +466,7 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
         c = 0; NB_CHECK(dev_ensure(&nb->wpos, &c, need * 3));
         c = 0; NB_CHECK(dev_ensure(&nb->xs0, &c, need * 3));
         c = 0; NB_CHECK(dev_ensure(&nb->xs, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->rec, &c, need * 2));
         c = 0; NB_CHECK(dev_ensure(&nb->img, &c, need * 6));   // sorted-order and caller-order halves
         c = 0; NB_CHECK(dev_ensure(&nb->perm, &c, need));
         c = 0; NB_CHECK(dev_ensure(&nb->type_s, &c, need));
@@ -579,7 +585,7 @@ cudaError_t launch_gather_positions(const NeighborDev& nb, const double* d_pos, 
     CellRows H;
     for (int k = 0; k < 9; ++k) H.h[k] = nb.H[k];
     H.tri = nb.tri;
-    k_gather_positions<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, nb.img, d_pos, nb.xs0, H, max_disp2, nb.xs, d_err);
+    k_gather_positions<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, nb.img, d_pos, nb.xs0, H, max_disp2, nb.type_s, nb.xs, nb.rec, d_err);
     return cudaGetLastError();
 }
 

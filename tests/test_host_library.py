@@ -38,7 +38,7 @@ def test_profile_widths_match_printed_table():
             if l.strip() and not l.startswith("#")]
     for row in rows:
         C0, C1, C2, K1, K2 = map(int, row[:5])
-        for k, L in enumerate((2, 3)):
+        for k, L in enumerate((2, 3, 4)):
             w = binding.profile_widths(C0, L)
             assert (w["C1"], w["C2"], w["K1"], w["K2"]) == (C1, C2, K1, K2)
             assert w["S"] == int(row[5 + k]) and w["D_out"] == int(row[8 + k])

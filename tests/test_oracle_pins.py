@@ -592,19 +592,20 @@ def _beta_only_oracle(profile, seed):
     return p, o
 
 
-def test_higher_degree_gram_blocks_follow_the_addition_theorem():
+@pytest.mark.parametrize("profile", ["p32_3_2", "p32_4_2"])
+def test_higher_degree_gram_blocks_follow_the_addition_theorem(profile):
     # With psi = beta the degree-l moments are X_l[m, c] = sum_j chi_j^2 beta_jc B_lm(u_j) / M_1 for
     # the LEADING C_l channels, and the addition theorem turns the Gram block into
     #   G_l[c, c'] = sum_jk chi_j^2 chi_k^2 beta_jc beta_kc' P_l(u_j . u_k) / M_1^2,
     # which needs only distances, directions and scipy's Legendre polynomials.  Pins the weight
     # chi^2 for every l >= 1, the shared normaliser M_1, the leading-channel rule (C_2 < C_1 here)
     # and the positions of vech(G_2), vech(G_3) in the feature vector.
-    p, o = _beta_only_oracle("p32_3_2", 52)
+    p, o = _beta_only_oracle(profile, 52)
     s = make_system(dict(kind="random_box", atoms=18, edges=(8.0, 8.5, 9.0), min_dist=1.6, seed=53,
                          n_types=p["T"], masses=[1.0] * p["T"]))
     out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"], want_grad=False)
     X0 = o.prm["X0"].numpy()
-    C0, Cs = p["C0"], {1: p["C1"], 2: p["C2"], 3: 1}
+    C0, Cs = p["C0"], {1: p["C1"], 2: p["C2"], 3: 1, 4: 1}
     assert Cs[2] < Cs[1]
     for i in (0, 6, 17):
         sel = out["dst"] == i
@@ -615,7 +616,7 @@ def test_higher_degree_gram_blocks_follow_the_addition_theorem():
         u = out["rij"][sel] / d[:, None]
         cosjk = np.clip(u @ u.T, -1.0, 1.0)
         off = 2 * C0 + 2
-        for l in (1, 2, 3):
+        for l in range(1, p["L"] + 1):
             C = Cs[l]
             wb = (chi ** 2)[:, None] * beta[:, :C]                        # [edges, C_l]
             G = wb.T @ scipy.special.eval_legendre(l, cosjk) @ wb / M1sq
@@ -672,7 +673,7 @@ def _energy(o, pos, s, cell=None):
     return o.compute(pos, s["types"], s["cell"] if cell is None else cell, s["pbc"], want_grad=False)["E"]
 
 
-@pytest.mark.parametrize("profile", ["p16_3_2", "p32_2_4"])
+@pytest.mark.parametrize("profile", ["p16_3_2", "p32_2_4", "p8_4_0"])
 def test_forces_sum_to_zero_and_match_finite_differences(profile):
     o, s = _small_case(profile=profile, n=16, edges=(7.0, 7.7, 8.1), seed=80)
     out = o.compute(s["pos"], s["types"], s["cell"], s["pbc"])

@@ -147,4 +147,11 @@ SMALL_PROFILES = {
                          Hp=688, S=223, D_out=541),
     "p128_2_0": _profile(128, 2, 0, 16, 2, 96, 3, C1=16, C2=8, K1=8, K2=2, H=344,
                          Hp=688, S=216, D_out=522),
+    # maximum degree four, at the three degree-wise channel layouts
+    "p8_4_0": _profile(8, 4, 0, 8, 2, 32, 2, C1=4, C2=4, K1=4, K2=2, H=24, Hp=48,
+                       S=56, D_out=93),
+    "p32_4_2": _profile(32, 4, 2, 16, 2, 64, 3, C1=8, C2=4, K1=4, K2=2, H=88,
+                        Hp=176, S=92, D_out=167),
+    "p128_4_4": _profile(128, 4, 4, 16, 2, 96, 2, C1=16, C2=8, K1=8, K2=2, H=344,
+                         Hp=688, S=232, D_out=557),
 }
