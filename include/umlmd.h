@@ -203,6 +203,31 @@ int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_for
                   double virial[9], double* d_atom_energy);
 
 /*
+ * Batched evaluation of many independent frames of one model in one call: the paper's execution
+ * note evaluates several frames at once and reduces the atomic energies per frame (its
+ * "segmented" energy reduction); small systems are bound by the fixed cost of a step's launches,
+ * which a batch pays once.  The atoms of all frames are concatenated:
+ *   frame_offsets  host, n_frames + 1 int64: frame f holds atoms frame_offsets[f] .. [f+1] - 1
+ *   d_pos [N,3], d_type [N]   device, N = frame_offsets[n_frames]
+ *   cells          host, n_frames x 9 doubles: each frame's cell vectors as rows (any non-singular cell)
+ *   pbc            3 ints, the same for every frame
+ *   energies       host, n_frames doubles (may be NULL)
+ *   d_force        [N,3] double, device (may be NULL)
+ *   virials        host, n_frames x 9 doubles (may be NULL)
+ *   d_atom_energy  [N] double, device (may be NULL)
+ * The neighbor lists (radius rc, no skin) are found by exhaustive search inside each frame, which
+ * suits frames of up to a few thousand atoms (limit UMLMD_BATCH_MAX_FRAME_ATOMS, else
+ * UMLMD_E_CAPACITY); edges never cross frames.  The whole batch then runs through the same kernels
+ * as one system, and one block per frame sums the frame's atomic energies and edge virials in a
+ * fixed order.  The call replaces the handle's neighbor list and MD state: call
+ * umlmd_build_neighbors again before umlmd_compute or umlmd_step.
+ */
+#define UMLMD_BATCH_MAX_FRAME_ATOMS 16384
+int umlmd_compute_batch(umlmd_t* h, int32_t n_frames, const int64_t* frame_offsets, const double* d_pos,
+                        const int32_t* d_type, const double* cells, const int pbc[3], double* energies,
+                        double* d_force, double* virials, double* d_atom_energy);
+
+/*
  * (Not in the paper, which drives its model from LAMMPS: the integrators here exist because the
  * benchmark's workloads are MD runs.)
  * Register MD state for umlmd_step: d_pos and d_vel [N,3] double (Angstrom, Angstrom/ps)

@@ -27,6 +27,7 @@ EXPORTS = [
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
     "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
     "umlmd_probe_fma_peak", "umlmd_get_neighbor_rows", "umlmd_workspace_bytes", "umlmd_get_nvt_state", "umlmd_set_nvt_state",
+    "umlmd_compute_batch",
 ]
 
 
@@ -81,6 +82,8 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_profile_class_name.restype = ctypes.c_char_p
     lib.umlmd_kinetic_energy_static.argtypes = [i64, vp, vp, vp, vp, vp]
     lib.umlmd_get_neighbor_rows.argtypes = [vp, i64, i64, vp, vp, vp, i64, ctypes.POINTER(i64)]
+    lib.umlmd_compute_batch.argtypes = [vp, i32, ctypes.POINTER(i64), vp, vp, ctypes.POINTER(dbl), ctypes.POINTER(ctypes.c_int),
+                                        ctypes.POINTER(dbl), vp, ctypes.POINTER(dbl), vp]
     lib.umlmd_workspace_bytes.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
     lib.umlmd_get_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
     lib.umlmd_set_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
@@ -259,6 +262,29 @@ class Model:
             self._raise(rc)
         return dict(energy=e.value, forces=f, atom_energy=ea,
                     virial=np.array(list(vir), dtype=np.float64).reshape(3, 3) if virial else None)
+
+    def compute_batch(self, frame_offsets, pos, types, cells, pbc=(1, 1, 1), forces=True, virial=True, atom_energy=False):
+        """Energies [n_frames] (numpy), forces (CUDA tensor or None), virials [n_frames,3,3] (numpy or
+        None) and atomic energies of concatenated frames; replaces the handle's neighbor list."""
+        _check_dev(pos, torch.float64, "pos")
+        _check_dev(types, torch.int32, "types")
+        off = np.ascontiguousarray(frame_offsets, dtype=np.int64)
+        nf = len(off) - 1
+        n = int(off[-1])
+        cl = np.ascontiguousarray(cells, dtype=np.float64).reshape(nf, 9)
+        e = np.zeros(nf, dtype=np.float64)
+        vir = np.zeros((nf, 9), dtype=np.float64) if virial else None
+        f = torch.empty((n, 3), dtype=torch.float64, device="cuda") if forces else None
+        ea = torch.empty(n, dtype=torch.float64, device="cuda") if atom_energy else None
+        P = ctypes.POINTER(ctypes.c_double)
+        pbc3 = (ctypes.c_int * 3)(*[int(x) for x in pbc])
+        rc = self._lib.umlmd_compute_batch(self._h, nf, off.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), _ptr(pos),
+                                           _ptr(types), cl.ctypes.data_as(P), pbc3, e.ctypes.data_as(P), _ptr(f),
+                                           vir.ctypes.data_as(P) if virial else None, _ptr(ea))
+        if rc != OK:
+            self._raise(rc)
+        self.n_atoms = 0
+        return dict(energies=e, forces=f, atom_energy=ea, virials=vir.reshape(nf, 3, 3) if virial else None)
 
     def set_md_state(self, pos, vel, masses):
         _check_dev(pos, torch.float64, "pos")

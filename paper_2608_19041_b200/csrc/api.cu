@@ -31,6 +31,7 @@ struct umlmd {
     float* g = nullptr; int64_t g_cap = 0;
     double* e_atom = nullptr; double* f_sorted = nullptr; int* type_o = nullptr; int64_t n_cap = 0;
     double* virial_part = nullptr; int64_t vpart_cap = 0;
+    double* frame_out = nullptr; int64_t frame_out_cap = 0;     // batched evaluation: [n_frames][10] energy, virial
     double* scratch = nullptr; double* d_out = nullptr; int* d_err = nullptr;
     double* h_out = nullptr; int* h_err = nullptr;      // pinned
     // per-pair amplitude tables of the species present (set up by umlmd_build_neighbors)
@@ -164,7 +165,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
     const Dims& d = h->d;
     NeighborDev& nb = h->nb;
     const int N = (int)nb.N;
-    { Scope sc(h, kGather, 1); API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st)); }
+    // (a batched list was built from these very positions: nothing to gather)
+    if (!nb.batch) { Scope sc(h, kGather, 1); API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st)); }
     const int B = N < h->node_tile ? N : h->node_tile;
     int vpart_used = 0;
     for (int a0 = 0; a0 < N; a0 += B) {
@@ -174,6 +176,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ea.table_uni = h->pair_tables ? h->table_uni : nullptr;
         ea.uni_scale = h->uni_scale;
         ea.species_slot = h->d_species + d.T; ea.n_present = (int)h->present.size();
+        ea.frames = nb.batch ? nb.frames : nullptr; ea.frame_of = nb.frame_of;
         ea.row_ptr = nb.row_ptr; ea.src = nb.src; ea.shift = nb.shift;
         ea.Lx = nb.L[0]; ea.Ly = nb.L[1]; ea.Lz = nb.L[2];
         for (int k = 0; k < 9; ++k) ea.H[k] = nb.H[k];
@@ -350,7 +353,7 @@ int umlmd_destroy(umlmd_t* h) {
     if (h->on_device) cudaStreamSynchronize(h->st);
     for (void* p : h->model_allocs) dev_free(p);
     neighbor_free(&h->nb);
-    void* ptrs[] = {h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
+    void* ptrs[] = {h->frame_out, h->state, h->desc, h->pre, h->hbuf, h->tc_hi, h->tc_lo, h->g, h->e_atom, h->f_sorted, h->type_o, h->virial_part,
                     h->scratch, h->d_out, h->d_err, h->md_force, h->d_mass, h->d_inv_mass, h->d_nhc, h->table_uni, h->d_species, h->uni_scale};
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
@@ -527,6 +530,66 @@ int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_for
     if (rc != UMLMD_OK) return rc;
     if (energy) *energy = h->h_out[0];
     if (virial) for (int k = 0; k < 9; ++k) virial[k] = h->h_out[1 + k];
+    return UMLMD_OK;
+}
+
+int umlmd_compute_batch(umlmd_t* h, int32_t n_frames, const int64_t* frame_offsets, const double* d_pos,
+                        const int32_t* d_type, const double* cells, const int pbc[3], double* energies, double* d_force,
+                        double* virials, double* d_atom_energy) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    if (n_frames < 0 || (n_frames > 0 && (!frame_offsets || !cells)) || !pbc)
+        return fail(h, UMLMD_E_INVALID_ARG, "bad argument to umlmd_compute_batch");
+    if (n_frames == 0) return UMLMD_OK;
+    if (frame_offsets[0] != 0) return fail(h, UMLMD_E_INVALID_ARG, "frame_offsets must start at 0");
+    for (int f = 0; f < n_frames; ++f) {
+        const int64_t n = frame_offsets[f + 1] - frame_offsets[f];
+        if (n < 0) return fail(h, UMLMD_E_INVALID_ARG, "frame_offsets must not decrease");
+        if (n > UMLMD_BATCH_MAX_FRAME_ATOMS)
+            return fail(h, UMLMD_E_CAPACITY, "a frame of a batch holds more atoms than the exhaustive per-frame search is meant for; use umlmd_build_neighbors");
+    }
+    const int64_t N = frame_offsets[n_frames];
+    if (N > 0x7fff0000LL) return fail(h, UMLMD_E_INVALID_ARG, "too many atoms for 32-bit indices");
+    if (N > 0 && (!d_pos || !d_type)) return fail(h, UMLMD_E_INVALID_ARG, "null positions or species");
+    int rc = ensure_device_model(h);
+    if (rc != UMLMD_OK) return rc;
+    h->have_list = false; h->have_md = false; h->have_edge_grad = false;     // the handle's list is replaced
+    { Scope sc(h, kNeighbor, 5); rc = neighbor_build_batch(&h->nb, n_frames, frame_offsets, cells, pbc, d_pos, d_type, h->d.T, h->hm.rc, h->d_err, h->st, &h->err); }
+    if (rc != UMLMD_OK) return rc;
+    const bool want_grad = d_force != nullptr || virials != nullptr;
+    if (N > 0) {
+        if ((rc = ensure_workspace(h)) != UMLMD_OK) return rc;
+        const int T = h->d.T;
+        if (!h->d_species) {
+            void* p = nullptr;
+            API_CUDA(h, dev_malloc(&p, sizeof(int) * 3 * (size_t)T));
+            h->d_species = (int*)p;
+            API_CUDA(h, cudaMallocHost((void**)&h->h_species, sizeof(int) * (size_t)T));
+        }
+        API_CUDA(h, launch_species_present(N, h->nb.type_s, T, h->d_species, h->d_err, h->st));
+        h->launches_total += 1;
+        API_CUDA(h, cudaMemcpyAsync(h->h_species, h->d_species, sizeof(int) * (size_t)T, cudaMemcpyDeviceToHost, h->st));
+        API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
+        API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+        API_CUDA(h, cudaStreamSynchronize(h->st));
+        if ((rc = decode_device_errors(h, *h->h_err)) != UMLMD_OK) return rc;
+        if ((rc = setup_pair_tables(h)) != UMLMD_OK) return rc;
+        if ((rc = enqueue_compute(h, d_pos, want_grad, d_force, d_atom_energy)) != UMLMD_OK) return rc;
+    }
+    API_CUDA(h, dev_ensure(&h->frame_out, &h->frame_out_cap, (int64_t)n_frames * 10));
+    if (N > 0) {
+        Scope sc(h, kReduce, 1);
+        API_CUDA(h, launch_frame_reduce(h->nb, h->e_atom, h->g, virials != nullptr, h->frame_out, h->st));
+    } else {
+        API_CUDA(h, cudaMemsetAsync(h->frame_out, 0, sizeof(double) * 10 * (size_t)n_frames, h->st));
+    }
+    std::vector<double> host((size_t)n_frames * 10);
+    API_CUDA(h, cudaMemcpyAsync(host.data(), h->frame_out, sizeof(double) * host.size(), cudaMemcpyDeviceToHost, h->st));
+    if (N > 0) { if ((rc = fetch_results(h, 10)) != UMLMD_OK) return rc; }
+    else API_CUDA(h, cudaStreamSynchronize(h->st));
+    for (int f = 0; f < n_frames; ++f) {
+        if (energies) energies[f] = host[10 * (size_t)f];
+        if (virials) for (int k = 0; k < 9; ++k) virials[9 * (size_t)f + k] = host[10 * (size_t)f + 1 + k];
+    }
     return UMLMD_OK;
 }
 

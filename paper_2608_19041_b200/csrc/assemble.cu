@@ -147,6 +147,40 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
     return s;   // valid in thread 0
 }
 
+// Segmented reduction of a batched evaluation: block f sums the atomic energies of frame f and,
+// when asked, -g (x) r over the edges of the frame's rows (edge vectors recomputed from the
+// positions and the frame's cell); thread-strided partial sums, then one fixed-order block sum.
+__global__ void __launch_bounds__(kRedBlock) k_frame_reduce(const FrameCell* __restrict__ frames, const double* __restrict__ e_atom,
+                                                            const eidx_t* __restrict__ row_ptr, const int* __restrict__ src,
+                                                            const int* __restrict__ shift, const float* __restrict__ g,
+                                                            const double* __restrict__ xs, bool want_virial,
+                                                            double* __restrict__ out) {
+    __shared__ double sh[kRedBlock / 32];
+    const FrameCell& fc = frames[blockIdx.x];
+    double e = 0, v[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    for (int i = fc.a0 + threadIdx.x; i < fc.a1; i += kRedBlock) {
+        e += e_atom[i];
+        if (!want_virial) continue;
+        const double xi = xs[3 * (size_t)i], yi = xs[3 * (size_t)i + 1], zi = xs[3 * (size_t)i + 2];
+        for (eidx_t k = row_ptr[i]; k < row_ptr[i + 1]; ++k) {
+            const int j = src[k], s = shift[k];
+            const int nx = (int)(signed char)(s & 0xff), ny = (int)(signed char)((s >> 8) & 0xff), nz = (int)(signed char)((s >> 16) & 0xff);
+            const double r[3] = {(xs[3 * (size_t)j] + ((nx * fc.H[0] + ny * fc.H[3]) + nz * fc.H[6])) - xi,
+                                 (xs[3 * (size_t)j + 1] + ((nx * fc.H[1] + ny * fc.H[4]) + nz * fc.H[7])) - yi,
+                                 (xs[3 * (size_t)j + 2] + ((nx * fc.H[2] + ny * fc.H[5]) + nz * fc.H[8])) - zi};
+            const double gg[3] = {(double)g[3 * (size_t)k], (double)g[3 * (size_t)k + 1], (double)g[3 * (size_t)k + 2]};
+            for (int a = 0; a < 3; ++a)
+                for (int b = 0; b < 3; ++b) v[3 * a + b] += gg[a] * r[b];
+        }
+    }
+    const double es = block_sum(e, sh);
+    if (threadIdx.x == 0) out[10 * (size_t)blockIdx.x] = es;
+    for (int k = 0; k < 9; ++k) {
+        const double s = want_virial ? block_sum(v[k], sh) : 0.0;
+        if (threadIdx.x == 0) out[10 * (size_t)blockIdx.x + 1 + k] = -s;
+    }
+}
+
 // pass 1: block b sums the contiguous slice [b*chunk, (b+1)*chunk) of x
 __global__ void __launch_bounds__(kRedBlock) k_sum_slices(const double* __restrict__ x, int64_t N, int64_t chunk,
                                                           double* __restrict__ part) {
@@ -303,6 +337,13 @@ cudaError_t launch_scatter_atom_energy(const NeighborDev& nb, const double* e_so
     const int N = (int)nb.N;
     if (N == 0) return cudaSuccess;
     k_scatter1<<<(N + 255) / 256, 256, 0, st>>>(N, nb.perm, e_sorted, d_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_frame_reduce(const NeighborDev& nb, const double* e_atom, const float* g, bool want_virial,
+                                double* d_out, cudaStream_t st) {
+    if (nb.n_frames <= 0) return cudaSuccess;
+    k_frame_reduce<<<nb.n_frames, kRedBlock, 0, st>>>(nb.frames, e_atom, nb.row_ptr, nb.src, nb.shift, g, nb.xs, want_virial, d_out);
     return cudaGetLastError();
 }
 

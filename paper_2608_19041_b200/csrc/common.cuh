@@ -113,6 +113,16 @@ __host__ __device__ inline void tab_unpack(unsigned w, float k2, float k3, float
     *c3 = k3 * (float)((int)(w << 20) >> 20);
 }
 
+// One frame of a batched evaluation (umlmd_compute_batch): its own cell and its slice of the
+// concatenated atom arrays.
+struct FrameCell {
+    double H[9];      // cell vectors as rows
+    double Hinv[9];   // inverse (fractional coordinates f = r Hinv)
+    int m[3];         // periodic images to visit along each cell vector (0 for an open direction)
+    int pbc[3];
+    int a0, a1;       // atoms [a0, a1) of the concatenated arrays
+};
+
 struct NeighborDev {
     int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;
     double L[3] = {0, 0, 0};     // cell edge lengths (the diagonal of H)
@@ -134,6 +144,10 @@ struct NeighborDev {
     int* src = nullptr;          // [E] sorted index of the neighbour
     int* shift = nullptr;        // [E] packed int8 x3 image n
     eidx_t* rev = nullptr;       // [E] index of the reverse edge, -1 if absent
+    // batched evaluation: per-frame cells and the frame of every atom (null for a single system)
+    FrameCell* frames = nullptr; int64_t frames_cap = 0; int n_frames = 0;
+    int* frame_of = nullptr;
+    bool batch = false;          // the list in here is the union of per-frame lists
     // scratch
     int* key = nullptr; int* key2 = nullptr; int* idx = nullptr; int* idx2 = nullptr;
     int* cell_start = nullptr; int64_t ncell_cap = 0;

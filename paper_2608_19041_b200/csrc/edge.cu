@@ -34,8 +34,9 @@ struct Geom {
 };
 
 // phase 1: one lane, one edge
+// Hf: cell of the destination's frame in a batched evaluation (rows), null for a single system
 __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool in_range, double xi, double yi,
-                                              double zi, int ti) {
+                                              double zi, int ti, const double* __restrict__ Hf) {
     Geom g;
     g.valid = false;
     g.dx = g.dy = g.dz = 0.f; g.rho = 1.f; g.inv_rho = 1.f; g.ux = g.uy = g.uz = 0.f;
@@ -49,7 +50,11 @@ __device__ __forceinline__ Geom edge_geometry(const EdgeArgs& a, eidx_t e, bool 
     const float4 r0 = __ldg(a.rec + 2 * (size_t)j), r1 = __ldg(a.rec + 2 * (size_t)j + 1);
     const double xj[3] = {(double)r0.x + (double)r1.x, (double)r0.y + (double)r1.y, (double)r0.z + (double)r1.z};
     const int tj = __float_as_int(r0.w);
-    if (a.tri) {        // general cell: the image offset is n . H
+    if (Hf) {
+        g.dx = (float)((xj[0] + ((nx * __ldg(Hf + 0) + ny * __ldg(Hf + 3)) + nz * __ldg(Hf + 6))) - xi);
+        g.dy = (float)((xj[1] + ((nx * __ldg(Hf + 1) + ny * __ldg(Hf + 4)) + nz * __ldg(Hf + 7))) - yi);
+        g.dz = (float)((xj[2] + ((nx * __ldg(Hf + 2) + ny * __ldg(Hf + 5)) + nz * __ldg(Hf + 8))) - zi);
+    } else if (a.tri) {        // general cell: the image offset is n . H
         g.dx = (float)((xj[0] + ((nx * a.H[0] + ny * a.H[3]) + nz * a.H[6])) - xi);
         g.dy = (float)((xj[1] + ((nx * a.H[1] + ny * a.H[4]) + nz * a.H[7])) - yi);
         g.dz = (float)((xj[2] + ((nx * a.H[2] + ny * a.H[5]) + nz * a.H[8])) - zi);
@@ -321,6 +326,7 @@ k_edge_forward(const EdgeArgs a) {
     const float k2 = UNI ? tab_step2(__ldg(a.uni_scale)) : a.d.tab_k2, k3 = UNI ? tab_step3(__ldg(a.uni_scale + 1)) : a.d.tab_k3;
     const eidx_t e0 = a.row_ptr[i];
     const int len = (int)(a.row_ptr[i + 1] - e0);      // edge offsets are 64-bit, offsets inside a row are not
+    const double* Hf = a.frames ? a.frames[a.frame_of[i]].H : nullptr;
     const unsigned lt_mask = (1u << lane) - 1u;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
     float accH[W::NCH];
@@ -432,7 +438,7 @@ k_edge_forward(const EdgeArgs a) {
 
     int qn = 0;
     for (int base = 0; base < len; base += 32) {
-        const Geom g = edge_geometry(a, e0 + base + lane, base + lane < len, xi, yi, zi, ti);
+        const Geom g = edge_geometry(a, e0 + base + lane, base + lane < len, xi, yi, zi, ti, Hf);
         const unsigned vmask = __ballot_sync(kFull, g.valid);
         const int p = qn + __popc(vmask & lt_mask);       // queue slot of this lane's edge, if it has one
         if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
@@ -516,6 +522,7 @@ k_edge_backward(const EdgeArgs a) {
         const float k2 = UNI ? tab_step2(__ldg(a.uni_scale)) : a.d.tab_k2, k3 = UNI ? tab_step3(__ldg(a.uni_scale + 1)) : a.d.tab_k3;
         const eidx_t e0 = a.row_ptr[i];
         const int len = (int)(a.row_ptr[i + 1] - e0);
+        const double* Hf = a.frames ? a.frames[a.frame_of[i]].H : nullptr;
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
         float h0[4 * G];
 #pragma unroll
@@ -640,7 +647,7 @@ k_edge_backward(const EdgeArgs a) {
         int qn = 0;
         for (int base = 0; base < len; base += 32) {
             const int e = base + lane;                                // offset inside the row
-            const Geom g = edge_geometry(a, e0 + e, e < len, xi, yi, zi, ti);
+            const Geom g = edge_geometry(a, e0 + e, e < len, xi, yi, zi, ti, Hf);
             const unsigned vmask = __ballot_sync(kFull, g.valid);
             const int p = qn + __popc(vmask & lt_mask);   // queue slot of this lane's edge, if it has one
             if (g.valid && p < 32) {

@@ -17,6 +17,16 @@ void neighbor_free(NeighborDev* nb);
 // Export the list in caller numbering (device buffers of the caller).
 int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t* d_shift,
                     cudaStream_t st, std::string* err);
+// Union of the neighbor lists of n_frames independent frames (atoms concatenated, frame f = atoms
+// offsets[f] .. offsets[f+1]-1 with cell cells[9 f ..]), list radius rc, by exhaustive search inside
+// each frame (meant for many small frames); atoms keep the caller's order.  Returns a UMLMD_* code.
+int neighbor_build_batch(NeighborDev* nb, int n_frames, const int64_t* offsets, const double* cells, const int pbc[3],
+                         const double* d_pos, const int32_t* d_type, int T, double rc, int* d_err, cudaStream_t st,
+                         std::string* err);
+// per-frame energy and virial: out[10 f] = sum of e_atom over the frame, out[10 f + 1 ..] = -sum over
+// the frame's edges of g (x) r, each by one block in a fixed order
+cudaError_t launch_frame_reduce(const NeighborDev& nb, const double* e_atom, const float* g, bool want_virial,
+                                double* d_out, cudaStream_t st);
 // Rows first .. first + n - 1 of the caller's numbering with 64-bit offsets: d_row_ptr [n + 1] is
 // always filled; edges are copied while they fit `cap` (cap = 0 or null buffers: offsets only).
 int neighbor_export_rows(NeighborDev* nb, int64_t first, int64_t n, int64_t* d_row_ptr, int32_t* d_src,
@@ -47,6 +57,9 @@ struct EdgeArgs {
     // [n_present^2][n_rows][3][C0] cubic pieces of psi_c(rho) of each ordered pair, in the format
     // of the radial table (launch_fuse_pair_tables), read instead of table, pairmod and the radial
     // modes; uni_scale[0..1] = largest |c2|, |c3| of these tables (scale of their packed words)
+    // batched evaluation: the image offsets of a row come from the cell of the destination's frame
+    const FrameCell* frames;    // null for a single system
+    const int* frame_of;
     const float* table_uni;
     const float* uni_scale;
     const int* species_slot;    // [T] species -> index among the species present

@@ -265,6 +265,89 @@ __global__ void k_reverse_map(int N, int sorted, const eidx_t* __restrict__ row_
     }
 }
 
+// ---- batched frames -------------------------------------------------------------------------
+// fold the atoms of frame blockIdx.x into its cell, write positions, records, species, frame index
+__global__ void k_batch_fold(const FrameCell* __restrict__ frames, const double* __restrict__ pos,
+                             const int* __restrict__ type, int T, double* __restrict__ xs, float4* __restrict__ rec,
+                             int* __restrict__ type_s, int* __restrict__ frame_of, int* __restrict__ perm,
+                             int* __restrict__ err) {
+    const FrameCell& fc = frames[blockIdx.x];
+    for (int i = fc.a0 + threadIdx.x; i < fc.a1; i += blockDim.x) {
+        const double x = pos[3 * (size_t)i], y = pos[3 * (size_t)i + 1], z = pos[3 * (size_t)i + 2];
+        bool bad = !isfinite(x) || !isfinite(y) || !isfinite(z);
+        double fl[3];
+        for (int k = 0; k < 3; ++k) {
+            const double f = x * fc.Hinv[k] + y * fc.Hinv[3 + k] + z * fc.Hinv[6 + k];
+            fl[k] = fc.pbc[k] ? floor(f) : 0.0;
+            if (!(fabs(fl[k]) <= 1.0e6)) { bad = true; fl[k] = 0.0; }
+        }
+        float hi[3], lo[3];
+        for (int k = 0; k < 3; ++k) {
+            const double r = k == 0 ? x : (k == 1 ? y : z);
+            const double w = bad ? 0.0 : r - ((fl[0] * fc.H[k] + fl[1] * fc.H[3 + k]) + fl[2] * fc.H[6 + k]);
+            xs[3 * (size_t)i + k] = w;
+            hi[k] = (float)w;
+            lo[k] = (float)(w - (double)hi[k]);
+        }
+        int t = type[i];
+        if (t < 0 || t >= T) { atomicOr(err, kErrSpecies); t = 0; }
+        if (bad) atomicOr(err, kErrNonFinite);
+        rec[2 * (size_t)i] = make_float4(hi[0], hi[1], hi[2], __int_as_float(t));
+        rec[2 * (size_t)i + 1] = make_float4(lo[0], lo[1], lo[2], 0.f);
+        type_s[i] = t;
+        frame_of[i] = blockIdx.x;
+        perm[i] = i;
+    }
+}
+
+// One warp per centre: every atom of the centre's frame under every image within reach, in the
+// order image (z slowest), then atom; the same double-precision predicate as the cell-list scan.
+template <bool FILL>
+__global__ void k_batch_scan(int N, const FrameCell* __restrict__ frames, const int* __restrict__ frame_of, double rl2,
+                             const double* __restrict__ xs, int* __restrict__ deg, const eidx_t* __restrict__ row_ptr,
+                             int* __restrict__ src, int* __restrict__ shift) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= N) return;
+    const int i = warp;
+    const FrameCell& fc = frames[frame_of[i]];
+    const double xi = xs[3 * (size_t)i], yi = xs[3 * (size_t)i + 1], zi = xs[3 * (size_t)i + 2];
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const eidx_t base_out = FILL ? row_ptr[i] : 0;
+    int count = 0;
+    for (int nz = -fc.m[2]; nz <= fc.m[2]; ++nz) {
+        const double szx = __dmul_rn((double)nz, fc.H[6]), szy = __dmul_rn((double)nz, fc.H[7]), szz = __dmul_rn((double)nz, fc.H[8]);
+        for (int ny = -fc.m[1]; ny <= fc.m[1]; ++ny) {
+            const double syx = __dadd_rn(szx, __dmul_rn((double)ny, fc.H[3])), syy = __dadd_rn(szy, __dmul_rn((double)ny, fc.H[4])),
+                         syz = __dadd_rn(szz, __dmul_rn((double)ny, fc.H[5]));
+            for (int nx = -fc.m[0]; nx <= fc.m[0]; ++nx) {
+                const double sx = __dadd_rn(syx, __dmul_rn((double)nx, fc.H[0])), sy = __dadd_rn(syy, __dmul_rn((double)nx, fc.H[1])),
+                             sz = __dadd_rn(syz, __dmul_rn((double)nx, fc.H[2]));
+                const bool self_img = nx == 0 && ny == 0 && nz == 0;
+                for (int b = fc.a0; b < fc.a1; b += 32) {
+                    const int j = b + lane;
+                    bool ok = false;
+                    if (j < fc.a1) {
+                        const double ddx = __dsub_rn(__dadd_rn(xs[3 * (size_t)j], sx), xi);
+                        const double ddy = __dsub_rn(__dadd_rn(xs[3 * (size_t)j + 1], sy), yi);
+                        const double ddz = __dsub_rn(__dadd_rn(xs[3 * (size_t)j + 2], sz), zi);
+                        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(ddx, ddx), __dmul_rn(ddy, ddy)), __dmul_rn(ddz, ddz));
+                        ok = (d2 < rl2) && !(self_img && j == i);
+                    }
+                    const unsigned mask = __ballot_sync(0xffffffffu, ok);
+                    if (FILL && ok) {
+                        const eidx_t p = base_out + count + __popc(mask & lt_mask);
+                        src[p] = j;
+                        shift[p] = pack_shift(nx, ny, nz);
+                    }
+                    count += __popc(mask);
+                }
+            }
+        }
+    }
+    if (!FILL && lane == 0) deg[i] = count;
+}
+
 __global__ void k_gather_positions(int N, const int* __restrict__ perm, const int* __restrict__ img,
                                    const double* __restrict__ pos, const double* __restrict__ xs0,
                                    CellRows H, double max_disp2, const int* __restrict__ type_s,
@@ -369,7 +452,7 @@ struct WidenDeg {
 }  // namespace
 
 void neighbor_free(NeighborDev* nb) {
-    void* ptrs[] = {nb->rec, nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
+    void* ptrs[] = {nb->frames, nb->rec, nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
                     nb->shift, nb->rev, nb->key, nb->key2, nb->idx, nb->idx2, nb->cell_start, nb->deg,
                     nb->cub_tmp};
     for (void* p : ptrs)
@@ -383,6 +466,7 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     if (N64 > 0x7fff0000LL) { *err = "too many atoms for 32-bit indices"; return UMLMD_E_INVALID_ARG; }
     const int N = (int)N64;
     const double r_list = rc + skin;
+    nb->batch = false; nb->n_frames = 0; nb->frame_of = nullptr;
     Grid g;
     const double L[3] = {cell[0], cell[4], cell[8]};
     g.tri = 0;
@@ -549,6 +633,100 @@ int neighbor_export(NeighborDev* nb, int32_t* d_row_ptr, int32_t* d_src, int8_t*
     if (nb->E > 0)
         k_export_rows<<<wb, TB, 0, st>>>(N, nb->perm, nb->row_ptr, nb->src, nb->shift, d_row_ptr, d_src,
                                          (signed char*)d_shift);
+    NB_CHECK(cudaGetLastError());
+    return UMLMD_OK;
+}
+
+int neighbor_build_batch(NeighborDev* nb, int n_frames, const int64_t* offsets, const double* cells, const int pbc[3],
+                         const double* d_pos, const int32_t* d_type, int T, double rc, int* d_err, cudaStream_t st,
+                         std::string* err) {
+    const int64_t N = offsets[n_frames];
+    std::vector<FrameCell> fr((size_t)n_frames);
+    for (int f = 0; f < n_frames; ++f) {
+        FrameCell& c = fr[f];
+        const double* H = cells + 9 * (size_t)f;
+        for (int k = 0; k < 9; ++k) {
+            if (!std::isfinite(H[k])) { *err = "non-finite cell in a frame"; return UMLMD_E_UNSUPPORTED_CELL; }
+            c.H[k] = H[k];
+        }
+        const double cx[3] = {H[4] * H[8] - H[5] * H[7], H[5] * H[6] - H[3] * H[8], H[3] * H[7] - H[4] * H[6]};   // b x c
+        const double cy[3] = {H[7] * H[2] - H[8] * H[1], H[8] * H[0] - H[6] * H[2], H[6] * H[1] - H[7] * H[0]};   // c x a
+        const double cz[3] = {H[1] * H[5] - H[2] * H[4], H[2] * H[3] - H[0] * H[5], H[0] * H[4] - H[1] * H[3]};   // a x b
+        const double det = H[0] * cx[0] + H[1] * cx[1] + H[2] * cx[2];
+        double scale = 0;
+        for (int k = 0; k < 9; ++k) scale = std::fmax(scale, std::fabs(H[k]));
+        if (!(std::fabs(det) > 1e-12 * scale * scale * scale)) { *err = "singular cell in a frame"; return UMLMD_E_UNSUPPORTED_CELL; }
+        const double* cr[3] = {cx, cy, cz};
+        for (int k = 0; k < 3; ++k) {           // column k of the inverse = (cross product k) / det
+            for (int r = 0; r < 3; ++r) c.Hinv[3 * r + k] = cr[k][r] / det;
+            const double nrm = std::sqrt(cr[k][0] * cr[k][0] + cr[k][1] * cr[k][1] + cr[k][2] * cr[k][2]);
+            const double height = std::fabs(det) / nrm;
+            c.pbc[k] = pbc[k] ? 1 : 0;
+            c.m[k] = pbc[k] ? (int)std::ceil(rc / height) : 0;
+            if (c.m[k] > 127) { *err = "frame cell much smaller than the cutoff (more than 127 images)"; return UMLMD_E_UNSUPPORTED_CELL; }
+        }
+        c.a0 = (int)offsets[f]; c.a1 = (int)offsets[f + 1];
+    }
+    nb->N = N; nb->skin = 0; nb->r_list = rc; nb->tri = 1; nb->batch = true; nb->n_frames = n_frames;
+    for (int k = 0; k < 3; ++k) { nb->pbc[k] = pbc[k] ? 1 : 0; nb->L[k] = 0; }
+    for (int k = 0; k < 9; ++k) nb->H[k] = 0;
+    nb->E = 0;
+    if (N == 0) return UMLMD_OK;
+    if (N > nb->N_cap || !nb->xs) {
+        const int64_t need = N + 1;
+        int64_t c;
+        // the same per-atom arrays as the cell-list build sizes (the two builds may alternate on one handle)
+        c = 0; NB_CHECK(dev_ensure(&nb->wpos, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->xs0, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->xs, &c, need * 3));
+        c = 0; NB_CHECK(dev_ensure(&nb->rec, &c, need * 2));
+        c = 0; NB_CHECK(dev_ensure(&nb->img, &c, need * 6));
+        c = 0; NB_CHECK(dev_ensure(&nb->perm, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->type_s, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->row_ptr, &c, need + 1));
+        c = 0; NB_CHECK(dev_ensure(&nb->key, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->key2, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->idx, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->idx2, &c, need));
+        c = 0; NB_CHECK(dev_ensure(&nb->deg, &c, need + 1));
+        nb->N_cap = N;
+    }
+    nb->frame_of = nb->key;                    // scratch of the cell-list build, free here
+    NB_CHECK(dev_ensure(&nb->frames, &nb->frames_cap, (int64_t)n_frames));
+    NB_CHECK(cudaMemcpyAsync(nb->frames, fr.data(), sizeof(FrameCell) * (size_t)n_frames, cudaMemcpyHostToDevice, st));
+    NB_CHECK(cudaStreamSynchronize(st));       // `fr` is pageable host memory
+    auto deg_wide = thrust::make_transform_iterator(static_cast<const int*>(nb->deg), WidenDeg());
+    size_t need_scan = 0;
+    cub::DeviceScan::ExclusiveScan(nullptr, need_scan, deg_wide, nb->row_ptr, cub::Sum(), (eidx_t)0, (int)N + 1, st);
+    if (need_scan > nb->cub_bytes) {
+        if (nb->cub_tmp) dev_free(nb->cub_tmp);
+        nb->cub_tmp = nullptr; nb->cub_bytes = 0;
+        NB_CHECK(dev_malloc(&nb->cub_tmp, need_scan + 256));
+        nb->cub_bytes = need_scan + 256;
+    }
+    const int TB = 256;
+    k_batch_fold<<<n_frames, TB, 0, st>>>(nb->frames, d_pos, d_type, T, nb->xs, nb->rec, nb->type_s, nb->frame_of, nb->perm, d_err);
+    const double rl2 = rc * rc;
+    const int wb = (int)((N + TB / 32 - 1) / (TB / 32));
+    k_batch_scan<false><<<wb, TB, 0, st>>>((int)N, nb->frames, nb->frame_of, rl2, nb->xs, nb->deg, nullptr, nullptr, nullptr);
+    NB_CHECK(cudaMemsetAsync(nb->deg + N, 0, sizeof(int), st));
+    size_t tmp_bytes = nb->cub_bytes;
+    NB_CHECK(cub::DeviceScan::ExclusiveScan(nb->cub_tmp, tmp_bytes, deg_wide, nb->row_ptr, cub::Sum(), (eidx_t)0, (int)N + 1, st));
+    eidx_t total = 0;
+    NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(total), cudaMemcpyDeviceToHost, st));
+    NB_CHECK(cudaStreamSynchronize(st));
+    nb->E = total;
+    if (total > nb->E_cap) {
+        int64_t c;
+        c = 0; NB_CHECK(dev_ensure(&nb->src, &c, total, 1.1));
+        c = 0; NB_CHECK(dev_ensure(&nb->shift, &c, total, 1.1));
+        c = 0; NB_CHECK(dev_ensure(&nb->rev, &c, total, 1.1));
+        nb->E_cap = c;
+    }
+    if (total > 0) {
+        k_batch_scan<true><<<wb, TB, 0, st>>>((int)N, nb->frames, nb->frame_of, rl2, nb->xs, nullptr, nb->row_ptr, nb->src, nb->shift);
+        k_reverse_map<<<wb, TB, 0, st>>>((int)N, 0, nb->row_ptr, nb->src, nb->shift, nb->rev);
+    }
     NB_CHECK(cudaGetLastError());
     return UMLMD_OK;
 }
