@@ -143,6 +143,9 @@ int umlmd_workspace_bytes(const umlmd_t* h, int64_t N, int64_t n_edges, int64_t*
  *   cell    9 doubles, rows are the cell vectors a, b, c; any non-singular cell.  A diagonal
  *           (orthorhombic) cell takes the exactly reproducible path below; a general cell is
  *           folded with f = r cell^-1, r - floor(f) . cell, and images are offset by n . cell
+ *           (an implementation that folds with (f - floor f) . cell gets the same points to the
+ *           last bit or two: in a sheared cell two implementations agree on the edge set except
+ *           for a pair whose distance lies within rounding of the list radius)
  *   pbc     3 ints, non-zero = periodic along that cell vector
  *   skin    extra list radius in Angstrom (>= 0); edges beyond rc carry zero weight
  * The predicate is evaluated in double precision as ((xj + n*L) - xi), d2 = (dx*dx +
