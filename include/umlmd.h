@@ -58,8 +58,10 @@ typedef struct umlmd_options {
     double   table_dx;   /* radial table spacing in Angstrom; 0 = the blob's value         */
     int32_t  node_tile;  /* atoms per workspace tile; 0 = 524288                            */
     int32_t  mlp_path;   /* 0 = default (2), 1 = CUDA-core fp32 GEMM, 2 = tcgen05 GEMM on split half-precision operands
-                            (three products, 22 significant bits), persistent, 3 = the same, one tile per CTA;
-                            2 and 3 need F % 8 == 0 and fall back to 1 otherwise */
+                            (three products, 22 significant bits), persistent, 3 = the same, one tile per CTA,
+                            4 = the same on pairs of CTAs (tcgen05 cta_group::2, 256 rows x up to 256 columns per
+                            pair) for every GEMM; path 2 uses that kernel only where it is the faster one, the
+                            last GEMM of the backward pass; 2, 3 and 4 need F % 8 == 0 and fall back to 1 otherwise */
     int32_t  pair_table_mb;  /* device memory, MiB, that per-pair amplitude tables may take
                                 (see umlmd_build_neighbors); 0 = 192, negative = never build them */
     int32_t  gemm_spin_limit;       /* polls after which a wait inside the tensor-core GEMM's operand

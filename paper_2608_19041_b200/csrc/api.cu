@@ -332,7 +332,7 @@ int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, 
     double dx_override = 0;
     if (opt) {
         if (opt->struct_bytes != sizeof(umlmd_options)) { delete h; return UMLMD_E_INVALID_ARG; }
-        if (opt->table_dx < 0 || opt->node_tile < 0 || opt->mlp_path < 0 || opt->mlp_path > 3) { delete h; return UMLMD_E_INVALID_ARG; }
+        if (opt->table_dx < 0 || opt->node_tile < 0 || opt->mlp_path < 0 || opt->mlp_path > 4) { delete h; return UMLMD_E_INVALID_ARG; }
         dx_override = opt->table_dx;
         if (opt->node_tile > 0) h->node_tile = opt->node_tile;
         if (opt->mlp_path > 0) h->mlp_path = opt->mlp_path;

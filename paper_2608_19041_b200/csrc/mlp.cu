@@ -232,6 +232,9 @@ cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st) {
         g.Bt_hi = a.m.theta_hi[0]; g.Bt_lo = a.m.theta_lo[0]; g.ldbt = F;
         g.A_hi = a.tc_hi + (size_t)sp * a.tc_slot; g.A_lo = a.tc_lo + (size_t)sp * a.tc_slot;
         g.a_presplit = tc; g.err = a.err; g.variant = variant; g.spin_limit = a.spin_limit;
+        // this GEMM's epilogue is a plain store, so its main loop sets the pace, and the two-CTA
+        // kernel's is the faster one (measured: 122 against 147 us on 131072 rows, N = 416, K = 384)
+        if (tc && a.path == 2 && variant == 2) g.variant = gemm_tc_pick_variant(n, d.DP, 4);
         if (res0) {
             if (vec_grad) { g.rvec = a.m.w_head; g.rvec_n = F; }
             else { g.res = hb[slot]; g.ldres = F; g.res_n = F; }

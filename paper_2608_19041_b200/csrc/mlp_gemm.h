@@ -50,7 +50,7 @@ struct GemmArgs {
     // tensor-core path, mode 0 / head: per-row bias bias_rows[row_type[m] * N + n] instead of bias[n]
     const float* bias_rows; const int* row_type;
     int lda_split;                // row pitch of A_hi / A_lo (0 = K)
-    int variant;                  // tensor-core kernel: 3 = one tile per CTA, otherwise the persistent one
+    int variant;                  // tensor-core kernel: 3 = one tile per CTA, 4 = two-CTA persistent, otherwise the one-CTA persistent one
     int* err;                     // device error word (bounded-wait expiry)
     // tensor-core path: polls before a wait on the operand pipeline gives up (0 = the default, a
     // fraction of a second), and a diagnostic that makes every CTA leave its k-th operand stage
@@ -143,7 +143,10 @@ inline bool mlp_uses_tc(int F, int path) { return path >= 2 && (F & 7) == 0 && g
 int gemm_tc_pick_variant(int M, int N, int requested);   // 2 (persistent) or 3 (one tile per CTA) for path 2
 constexpr int kGemmTcBN = 128;  // column tile of the tensor-core GEMM
 // partial head sums per row that the fused last-layer epilogue of a variant leaves
-inline int gemm_tc_head_parts(int N, int variant) { return (variant == 3 ? 1 : 4) * ((N + kGemmTcBN - 1) / kGemmTcBN); }
+inline int gemm_tc_head_parts(int N, int variant) {
+    if (variant == 4) return (N + 31) / 32;        // one per 32-column chunk
+    return (variant == 3 ? 1 : 4) * ((N + kGemmTcBN - 1) / kGemmTcBN);
+}
 cudaError_t launch_gemm_tc(const GemmArgs& g, cudaStream_t st);
 
 }  // namespace umd

@@ -82,7 +82,7 @@ def test_workspace_estimate_covers_what_a_run_allocates():
     m.close()
 
 
-@pytest.mark.parametrize("variant", ["one_tile", "persistent"])
+@pytest.mark.parametrize("variant", ["one_tile", "persistent", "cta_pairs"])
 def test_expired_pipeline_wait_is_reported_and_the_handle_recovers(variant):
     # The diagnostic option leaves one operand stage of the first MLP layer unloaded; nothing sets
     # the barrier the MMA warp then waits on, the shortened wait runs out, the kernel finishes and
@@ -95,7 +95,7 @@ def test_expired_pipeline_wait_is_reported_and_the_handle_recovers(variant):
     else:   # enough rows for the persistent kernel: more than half an item per SM
         p = SMALL_PROFILES["p8_2_0"]
         s = make_system(dict(kind="fcc", cells=18, a=4.05, jitter=0.05, seed=5, n_types=p["T"], masses=[1.0] * p["T"]))
-        path = 2
+        path = 2 if variant == "persistent" else 4
     blob = make_blob(p, seed=45, bias_scale=0.2, e_ref_scale=0.5)
     B = _binding()
     good, pos = _build(blob, s, mlp_path=path)

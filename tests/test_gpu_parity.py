@@ -362,6 +362,31 @@ def test_tensor_core_mlp_path_matches_cuda_core_path_on_cu4000():
     print(f"max|dE_i| vs CUDA-core path: path 2 {d2 / e_scale:.2e}, path 3 {d3 / e_scale:.2e} of max|E_i|")
 
 
+@pytest.mark.parametrize("name", ["p32_2_4", "p128_3_4"])
+def test_persistent_tensor_core_kernels_match_the_cuda_core_path(name):
+    # enough rows that path 2 takes the one-CTA persistent kernel and path 4 the two-CTA one (both
+    # fall back to one tile per CTA on small systems); ragged last row tile, widths that are not
+    # multiples of the column tile
+    p = SMALL_PROFILES[name]
+    blob = make_blob(p, seed=50, bias_scale=0.2, e_ref_scale=0.5)
+    s = make_system(dict(kind="fcc", cells=18, a=4.05, jitter=0.05, seed=6, n_types=p["T"], masses=[1.0] * p["T"]))
+    outs = {}
+    for path in (1, 2, 4):
+        m, pos = _build(blob, s, mlp_path=path)
+        outs[path] = m.compute(pos, atom_energy=True)
+        m.close()
+    a = outs[1]
+    e_scale = a["atom_energy"].abs().max().item()
+    f_scale = a["forces"].abs().max().item()
+    for path in (2, 4):
+        b = outs[path]
+        de = (a["atom_energy"] - b["atom_energy"]).abs().max().item()
+        print(f"{name} path {path}: max|dE_i| vs CUDA-core path {de / e_scale:.2e} of max|E_i|")
+        assert de <= 5e-6 * e_scale
+        assert (a["forces"] - b["forces"]).abs().max().item() <= 1e-5 * f_scale
+        assert np.abs(a["virial"] - b["virial"]).max() <= 1e-5 * np.abs(a["virial"]).max()
+
+
 # ------------------------------------------------------------------ general (triclinic) cells
 
 def _sheared(desc, tilt, flip=False):
