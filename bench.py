@@ -289,10 +289,12 @@ class Workload:
         self.s = s
         self.N = len(s["pos"])
         self.model = binding.Model(workload_blob(name, modes), mlp_path=args.mlp_path, node_tile=args.node_tile,
-                                   pair_table_mb=args.pair_table_mb, table_dx=args.table_dx)
+                                   pair_table_mb=args.pair_table_mb, table_dx=args.table_dx,
+                                   launch_graphs=args.launch_graphs)
         self.pos = torch.as_tensor(s["pos"], dtype=torch.float64).cuda().contiguous()
         self.vel = None if self.static else torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
         self.types = torch.as_tensor(s["types"], dtype=torch.int32).cuda().contiguous()
+        self.forces = torch.empty((self.N, 3), dtype=torch.float64, device="cuda")     # result buffer of every evaluation
         self.skin, self.every, self.dt = self.md["skin"], self.md["rebuild_every"], self.md["dt_ps"]
         m = self.model
         m.build_neighbors(self.pos, self.types, s["cell"], s["pbc"], 0.0)
@@ -311,14 +313,15 @@ class Workload:
             return m.step(k, self.dt, self.every)
         out = None
         for _ in range(k):
-            out = m.compute(self.pos, forces=True, virial=True)
+            out = m.compute(self.pos, forces=True, virial=True, out_forces=self.forces)
         return (out["energy"] if out else 0.0), 0.0
 
     def timed(self, steps, warmup, sync_all, sampler=None):
         """(ms, e_pot, e_kin, launches): exactly `steps` steps after `warmup`, CUDA events."""
         torch = self.torch
         self.run_steps(warmup)
-        l0 = self.model.query()["kernel_launches"]
+        q0 = self.model.query()
+        l0 = q0["kernel_launches"]
         sync_all()
         if sampler:
             sampler.start()
@@ -327,7 +330,9 @@ class Workload:
         e_pot, e_kin = self.run_steps(steps)
         ev1.record()
         sync_all()
-        return ev0.elapsed_time(ev1), e_pot, e_kin, self.model.query()["kernel_launches"] - l0
+        q1 = self.model.query()
+        self.graph_replays = q1["graph_replays"] - q0["graph_replays"]     # of the timed steps
+        return ev0.elapsed_time(ev1), e_pot, e_kin, q1["kernel_launches"] - l0
 
     def classes(self, steps, peaks):
         """Per-class CUDA-event times of `steps` more steps, with each class's roofline entry."""
@@ -365,7 +370,7 @@ class Workload:
         dpos = torch.empty_like(self.pos)
         dpos.copy_(host_pos)
         m.build_neighbors(dpos, self.types, s["cell"], s["pbc"], self.skin)
-        m.compute(dpos)
+        m.compute(dpos, out_forces=self.forces)
         sync_all()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         builds = 0
@@ -375,7 +380,7 @@ class Workload:
             if every and k % every == 0:
                 m.build_neighbors(dpos, self.types, s["cell"], s["pbc"], self.skin)
                 builds += 1
-            out = m.compute(dpos, forces=True, virial=True)
+            out = m.compute(dpos, forces=True, virial=True, out_forces=self.forces)
             host_f.copy_(out["forces"], non_blocking=True)
         t1.record()
         sync_all()
@@ -383,7 +388,7 @@ class Workload:
 
     def close(self):
         self.model.close()
-        del self.pos, self.vel, self.types
+        del self.pos, self.vel, self.types, self.forces
         self.torch.cuda.empty_cache()
 
 
@@ -421,6 +426,7 @@ def run_ours(args):
     N, name, cfg = w.N, w.label, w.cfg
     sampler = ClockSampler(local)
     ms, e_pot, e_kin, launches = w.timed(args.steps, args.warmup, sync_all, sampler)
+    graph_replays = w.graph_replays
     clocks = sampler.stop()
     ms = max_over_ranks(ms, "cuda")
     value = job_rate(N * args.steps, ms, world)
@@ -463,7 +469,7 @@ def run_ours(args):
             ok = ow.classes(k, peaks)
             top = ok[0] if ok else None
             others.append(dict(workload=oname, n_atoms=ow.N, value=ow.N * k / (oms * 1e-3), unit="atom-steps/s",
-                               steps=k, ms_per_step=oms / k, gpu_launches=int(ol),
+                               steps=k, ms_per_step=oms / k, gpu_launches=int(ol), graph_replays=int(ow.graph_replays),
                                dominant=dict(kernel=top["kernel"], bound=top["bound"], frac=top["frac"],
                                              share=top["share"]) if top else None,
                                clocks=dict(sm_mhz=ocl["sm_mhz"], reasons=ocl["reasons"])))
@@ -492,11 +498,11 @@ def run_ours(args):
                                 profile={k: p[k] for k in ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T")},
                                 dt_ps=dt, rebuild_every=every, skin=skin,
                                 ensemble="nvt (Nose-Hoover chain, period 100 dt)" if (args.nvt and not static) else "nve",
-                                mlp_path=args.mlp_path, pair_table_mb=args.pair_table_mb, table_dx=args.table_dx, parallelism="replicas" if world > 1 else "single",
+                                mlp_path=args.mlp_path, launch_graphs=args.launch_graphs, pair_table_mb=args.pair_table_mb, table_dx=args.table_dx, parallelism="replicas" if world > 1 else "single",
                                 **({"published": pub} if pub else {}),
                                 cache="working set per step exceeds L2" if N >= 100000 else "fits in L2 (launch-bound)"),
                     e_pot_per_atom=e_pot / N, e_kin_per_atom=e_kin / N,
-                    gpu_launches=int(launches), e2e=e2e, roofline=dom, kernels=kernels, workloads=others, cpu_baseline=cpu,
+                    gpu_launches=int(launches), graph_replays=int(graph_replays), e2e=e2e, roofline=dom, kernels=kernels, workloads=others, cpu_baseline=cpu,
                     peaks=dict(hbm_gbs=peaks["hbm_gbs"], tensor_16bit_tflops_sustained=peaks["bf16_tflops_sustained"],
                                fp32_tflops=round(peaks["fp32_tflops"], 2), fp32_source=peaks["fp32_source"],
                                fp32_tflops_derived=round(derived, 1), source=peaks["source"]),
@@ -507,13 +513,92 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_domain(args):
+    """One system cut into bricks, one per rank (paper_2608_19041_b200/domain.py): per step a forward
+    exchange of ghost coordinates, one evaluation per brick, a reverse exchange of ghost forces.
+    Strong scaling: the system is fixed, `value` is its atoms x steps over the slowest rank's time.
+    With one rank the brick is the whole cell and its ghosts are its own periodic images."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_19041_b200 import binding
+    from paper_2608_19041_b200.domain import Domain, SerialComm, TorchComm, brick_grid
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    comm = TorchComm() if world > 1 else SerialComm()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    name = args.workload
+    cfg = CONFIGS[name]
+    if cfg["md"] is None:
+        raise SystemExit("--domain needs a workload with an MD recipe")
+    md = cfg["md"]
+    desc = dict(cfg["system"])
+    if args.atoms:
+        if desc.get("kind") != "poisson_disk":
+            raise SystemExit("--atoms with --domain applies to the amorphous workload only")
+        desc["atoms"] = int(args.atoms)
+    s = make_system(desc, md)                      # the same seeded system on every rank
+    N = len(s["pos"])
+    grid = brick_grid(world)
+    model = binding.Model(workload_blob(name), mlp_path=args.mlp_path, node_tile=args.node_tile,
+                          pair_table_mb=args.pair_table_mb, launch_graphs=args.launch_graphs)
+    d = Domain(model, comm, np.diag(s["cell"]), grid, model.query()["rc"], md["skin"], s["masses"])
+    d.distribute(s["pos"], s["vel"], s["types"])
+    d.start()
+    e_start = d.totals()
+    d.step(args.warmup, md["dt_ps"], md["rebuild_every"])
+    l0 = model.query()["kernel_launches"]
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    d.step(args.steps, md["dt_ps"], md["rebuild_every"])
+    ev1.record()
+    sync_all()
+    clocks = sampler.stop()
+    ms = max_over_ranks(ev0.elapsed_time(ev1), "cuda")
+    launches = model.query()["kernel_launches"] - l0
+    e_end = d.totals()
+    counts = torch.tensor([d.n_own, d.n_ghost], dtype=torch.float64, device="cuda")
+    counts = comm.all_reduce_sum(counts).tolist()
+    if rank == 0:
+        line = dict(metric="atom-steps/s (energy+forces+virial)", value=N * args.steps / (ms * 1e-3), unit="atom-steps/s",
+                    n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=ms / args.steps, higher_is_better=True,
+                    scaling="strong", vs_baseline=None, dtype="f32", data="synthetic",
+                    config=dict(workload=name if not args.atoms else f"{name}[atoms={N}]", n_atoms=N,
+                                parallelism=f"domain {grid[0]}x{grid[1]}x{grid[2]} (bricks with ghost atoms)",
+                                ghosts_total=int(counts[1]), ghost_bytes_per_step=int(counts[1]) * 48,
+                                dt_ps=md["dt_ps"], rebuild_every=md["rebuild_every"], skin=md["skin"], ensemble="nve",
+                                cache="working set per step exceeds L2" if N >= 100000 else "fits in L2 (launch-bound)"),
+                    e_total_per_atom_start=(e_start[0] + e_start[1]) / N, e_total_per_atom_end=(e_end[0] + e_end[1]) / N,
+                    gpu_launches=int(launches), e2e=None, roofline=None, cpu_baseline=None,
+                    clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"],
+                                samples=clocks["samples"]))
+        print(json.dumps(line))
+    model.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def batched_frames(args, name, n_frames, calls, sync_all):
     import torch
 
     from paper_2608_19041_b200 import binding
     s = make_system(CONFIGS[name]["system"])
     n = len(s["pos"])
-    m = binding.Model(workload_blob(name), mlp_path=args.mlp_path, pair_table_mb=args.pair_table_mb)
+    m = binding.Model(workload_blob(name), mlp_path=args.mlp_path, launch_graphs=args.launch_graphs, pair_table_mb=args.pair_table_mb)
     off = np.arange(n_frames + 1) * n
     pos = torch.as_tensor(np.tile(s["pos"], (n_frames, 1)), dtype=torch.float64).cuda().contiguous()
     types = torch.as_tensor(np.tile(s["types"], n_frames), dtype=torch.int32).cuda().contiguous()
@@ -574,17 +659,23 @@ def main():
     ap.add_argument("--pair-table-mb", type=int, default=0,
                     help="memory for per-pair amplitude tables in MiB (0 = library default, negative = off)")
     ap.add_argument("--node-tile", type=int, default=0)
+    ap.add_argument("--launch-graphs", type=int, default=0, choices=[-1, 0, 1],
+                    help="replay of repeated launch sequences as CUDA graphs: 0 = the library's rule (systems of at most 65536 atoms), 1 = always, -1 = never")
     ap.add_argument("--atoms", type=int, default=0, help="amorphous and lattice workloads: (about) this many atoms in a smaller box of the same recipe")
     ap.add_argument("--modes", type=int, default=-1, help="override the number R of shared radial modes of the workload's profile")
     ap.add_argument("--nvt", action="store_true", help="time the Nose-Hoover-chain NVT driver instead of NVE")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--domain", action="store_true",
+                    help="cut the workload into one brick per rank (ghost-atom exchange each step) instead of running replicas")
     ap.add_argument("--no-workloads", action="store_true", help="skip the short runs of the other benchmark systems")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.domain:
+        run_domain(args)
     else:
         run_ours(args)
 

@@ -71,6 +71,13 @@ typedef struct umlmd_options {
                                        after umlmd_create leave the k-th operand stage of the first MLP
                                        layer unloaded, so that exactly such a wait runs out (nothing
                                        faults or hangs; the handle stays usable); 0 = off */
+    int32_t  launch_graphs;         /* replay of repeated launch sequences as CUDA graphs (an evaluation
+                                       of the same buffers as the one before it; the middle steps of an MD
+                                       run between two list builds): 0 = for systems of at most 65536
+                                       atoms, where the time between two dozen short kernels exceeds the
+                                       time inside them, 1 = always, -1 = never.  Results are those of
+                                       the plain launches, bit for bit (same kernels, same order).  Not
+                                       in the paper. */
 } umlmd_options;
 
 /* Structural widths of a model, all derived from (C0, L, R) by the paper's formulas
@@ -84,6 +91,7 @@ typedef struct umlmd_info {
     int64_t n_atoms, n_edges;          /* of the current neighbor list (0 before a build)  */
     int64_t device_bytes;              /* device memory currently held by the library      */
     int64_t kernel_launches;           /* kernels of this library launched by the handle   */
+    int64_t graph_replays;             /* launch sequences replayed as graphs (their kernels are counted above) */
 } umlmd_info;
 
 /* Widths for a (C0, L, R) triple without a handle; fills only the width fields.
@@ -279,6 +287,46 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
 #define UMLMD_NVT_STATE_DOUBLES 6
 int umlmd_get_nvt_state(umlmd_t* h, double state[UMLMD_NVT_STATE_DOUBLES]);
 int umlmd_set_nvt_state(umlmd_t* h, const double state[UMLMD_NVT_STATE_DOUBLES]);
+
+/*
+ * Ghost atoms, for a system cut into spatial domains (the paper's distributed runs: each rank owns
+ * the atoms of its region, holds copies -- ghosts -- of the atoms within the list radius around it,
+ * receives their coordinates before an evaluation and sends the forces on them back afterwards; no
+ * learned quantity crosses a boundary because the model has a single aggregation layer).
+ * After this call the atoms with index >= n_owned (caller's numbering) of every evaluation are
+ * ghosts: they are neighbours only.  No atomic energy is computed for them (their entries of
+ * d_atom_energy are 0, the energy is the sum over the owned atoms), only the edges that end on an
+ * owned atom carry a gradient, and d_force holds for every atom, owned or ghost, minus the derivative
+ * of that energy: the forces on ghosts are what has to be added to their owners' forces, and the
+ * virial is the owned atoms' share, -sum over their edges of g (x) r.  Summed over all domains these
+ * are the energy, forces and virial of the whole system.  The neighbor list is built over all
+ * atoms as usual (give the domain's box as a non-periodic cell); ghosts cost their rows of the
+ * per-atom stages but none of the per-edge work.
+ *   n_owned   number of owned atoms, placed first; negative or >= N: every atom is owned (default)
+ * umlmd_step and umlmd_step_nvt move every atom of the handle and refuse to run while ghosts are
+ * set; a domain's driver uses umlmd_compute and umlmd_vv_update.  Not in the paper as an interface
+ * (it delegates this to its MD host code).
+ */
+int umlmd_set_owned_atoms(umlmd_t* h, int64_t n_owned);
+
+/*
+ * One piece of a velocity Verlet step on caller-owned arrays (no handle: for drivers that own the
+ * integrator state themselves, e.g. one spatial domain's owned atoms):
+ *   v += half_kicks * (dt/2) * F / m   (half_kicks in {0, 1, 2}; 2 = the closing kick of one step and
+ *                                        the opening kick of the next in one pass)
+ *   r += dt * v                        (if drift != 0, after the kick)
+ * with 1 eV/(Angstrom amu) = 9648.533 Angstrom/ps^2 (metal units, as umlmd_step).
+ *   d_pos, d_vel   [N,3] double, Angstrom and Angstrom/ps   (device, caller-owned, updated in place)
+ *   d_force        [N,3] double, eV/Angstrom                (device; may be null if half_kicks == 0)
+ *   d_type         [N] int32 species; every entry must index d_inv_mass_per_type (not checked:
+ *                  there is no handle to check it against)
+ *   d_inv_mass_per_type   1/mass in 1/amu by species        (device)
+ *   stream         cudaStream_t as void*; the call only enqueues work
+ * Returns UMLMD_E_INVALID_ARG for null pointers, a bad count or time step; UMLMD_E_CUDA if the
+ * launch fails.  Not in the paper (it integrates with LAMMPS).
+ */
+int umlmd_vv_update(int64_t N, double* d_pos, double* d_vel, const double* d_force, const int32_t* d_type,
+                    const double* d_inv_mass_per_type, double dt_ps, int32_t half_kicks, int32_t drift, void* stream);
 
 /*
  * Per-atom virial of the last evaluation that produced forces or the virial (umlmd_compute with

@@ -27,7 +27,7 @@ EXPORTS = [
     "umlmd_get_intermediates", "umlmd_eval_radial_table", "umlmd_eval_pair_cache", "umlmd_set_profiling",
     "umlmd_get_profile", "umlmd_profile_class_name", "umlmd_kinetic_energy_static", "umlmd_static_last_error",
     "umlmd_probe_fma_peak", "umlmd_get_neighbor_rows", "umlmd_workspace_bytes", "umlmd_get_nvt_state", "umlmd_set_nvt_state",
-    "umlmd_compute_batch",
+    "umlmd_compute_batch", "umlmd_set_owned_atoms", "umlmd_vv_update",
 ]
 
 
@@ -40,7 +40,8 @@ class UmlmdError(RuntimeError):
 class Options(ctypes.Structure):
     _fields_ = [("struct_bytes", ctypes.c_uint32), ("table_dx", ctypes.c_double),
                 ("node_tile", ctypes.c_int32), ("mlp_path", ctypes.c_int32), ("pair_table_mb", ctypes.c_int32),
-                ("gemm_spin_limit", ctypes.c_int32), ("fault_skip_gemm_stage", ctypes.c_int32)]
+                ("gemm_spin_limit", ctypes.c_int32), ("fault_skip_gemm_stage", ctypes.c_int32),
+                ("launch_graphs", ctypes.c_int32)]
 
 
 class Info(ctypes.Structure):
@@ -48,7 +49,8 @@ class Info(ctypes.Structure):
                 ("C0", "L", "R", "N_rbf", "n_hidden", "F", "T", "C1", "C2", "K1", "K2", "S", "D_out", "H",
                  "H_pair", "table_rows")] + \
                [("rc", ctypes.c_double), ("table_dx", ctypes.c_double), ("n_atoms", ctypes.c_int64),
-                ("n_edges", ctypes.c_int64), ("device_bytes", ctypes.c_int64), ("kernel_launches", ctypes.c_int64)]
+                ("n_edges", ctypes.c_int64), ("device_bytes", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
+                ("graph_replays", ctypes.c_int64)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -88,6 +90,8 @@ def load_library(path=_LIB_PATH):
     lib.umlmd_get_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
     lib.umlmd_set_nvt_state.argtypes = [vp, ctypes.POINTER(dbl)]
     lib.umlmd_probe_fma_peak.argtypes = [ctypes.POINTER(dbl), vp]
+    lib.umlmd_set_owned_atoms.argtypes = [vp, i64]
+    lib.umlmd_vv_update.argtypes = [i64, vp, vp, vp, vp, vp, dbl, i32, i32, vp]
     lib.umlmd_static_last_error.argtypes = []
     lib.umlmd_static_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -115,6 +119,40 @@ def profile_widths(C0, L, R=0):
             ("C1", "C2", "K1", "K2", "S", "D_out", "H", "H_pair")}
 
 
+def _stream_ptr(stream):
+    st = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(st.cuda_stream)
+
+
+def vv_update(pos, vel, force, types, inv_mass, dt_ps, half_kicks, drift, stream=None):
+    """One piece of a velocity Verlet step on caller-owned CUDA arrays (umlmd_vv_update):
+    half_kicks half kicks, then a drift if asked; inv_mass = 1/mass by species (CUDA, float64)."""
+    _check_dev(vel, torch.float64, "vel")
+    _check_dev(types, torch.int32, "types")
+    _check_dev(inv_mass, torch.float64, "inv_mass")
+    if drift:
+        _check_dev(pos, torch.float64, "pos")
+    if half_kicks:
+        _check_dev(force, torch.float64, "force")
+    rc = lib().umlmd_vv_update(vel.shape[0], _ptr(pos), _ptr(vel), _ptr(force), _ptr(types), _ptr(inv_mass),
+                               float(dt_ps), int(half_kicks), int(bool(drift)), _stream_ptr(stream))
+    if rc != OK:
+        raise UmlmdError(rc, "umlmd_vv_update failed")
+
+
+def kinetic_energy(vel, types, mass, out=None, stream=None):
+    """Kinetic energy in eV of caller-owned CUDA arrays (umlmd_kinetic_energy_static): returns a
+    one-element CUDA tensor; mass = mass by species (CUDA, float64)."""
+    _check_dev(vel, torch.float64, "vel")
+    _check_dev(types, torch.int32, "types")
+    _check_dev(mass, torch.float64, "mass")
+    out = out if out is not None else torch.zeros(1, dtype=torch.float64, device="cuda")
+    rc = lib().umlmd_kinetic_energy_static(vel.shape[0], _ptr(vel), _ptr(types), _ptr(mass), _ptr(out), _stream_ptr(stream))
+    if rc != OK:
+        raise UmlmdError(rc, lib().umlmd_static_last_error().decode())
+    return out
+
+
 def probe_fma_peak(stream=None):
     """FP32 fused multiply-add rate of the current device in TFLOP/s (measured by the library)."""
     out = ctypes.c_double()
@@ -138,11 +176,11 @@ class Model:
     """A DPA4C model on the current CUDA device, created from a weight blob."""
 
     def __init__(self, blob, table_dx=0.0, node_tile=0, mlp_path=0, pair_table_mb=0, stream=None,
-                 gemm_spin_limit=0, fault_skip_gemm_stage=0):
+                 gemm_spin_limit=0, fault_skip_gemm_stage=0, launch_graphs=0):
         self._lib = lib()
         self._h = ctypes.c_void_p()
         opt = Options(ctypes.sizeof(Options), float(table_dx), int(node_tile), int(mlp_path), int(pair_table_mb),
-                      int(gemm_spin_limit), int(fault_skip_gemm_stage))
+                      int(gemm_spin_limit), int(fault_skip_gemm_stage), int(launch_graphs))
         # creation is host-only; a stream is only meaningful when a device is present
         self._stream = stream if stream is not None else (
             torch.cuda.current_stream() if torch.cuda.is_available() else None)
@@ -248,14 +286,26 @@ class Model:
             self._raise(rc)
         return out[:self.n_atoms]
 
-    def compute(self, pos, forces=True, virial=True, atom_energy=False):
+    def compute(self, pos, forces=True, virial=True, atom_energy=False, out_forces=None, out_atom_energy=None):
         """Returns dict(energy=float, forces=CUDA tensor or None, virial=np [3,3] or None,
-        atom_energy=CUDA tensor or None)."""
+        atom_energy=CUDA tensor or None).  out_forces [n,3] / out_atom_energy [n] (float64, CUDA):
+        buffers to write into instead of new ones (a repeated call with the same buffers is
+        replayed as one graph launch for small systems)."""
         _check_dev(pos, torch.float64, "pos")
         n = self.n_atoms
         e = ctypes.c_double()
-        f = torch.empty((n, 3), dtype=torch.float64, device="cuda") if forces else None
-        ea = torch.empty(n, dtype=torch.float64, device="cuda") if atom_energy else None
+        if out_forces is not None:
+            _check_dev(out_forces, torch.float64, "out_forces")
+            if out_forces.numel() != 3 * n:
+                raise ValueError("out_forces must hold n_atoms x 3 values")
+        if out_atom_energy is not None:
+            _check_dev(out_atom_energy, torch.float64, "out_atom_energy")
+            if out_atom_energy.numel() != n:
+                raise ValueError("out_atom_energy must hold n_atoms values")
+        f = out_forces if out_forces is not None else (
+            torch.empty((n, 3), dtype=torch.float64, device="cuda") if forces else None)
+        ea = out_atom_energy if out_atom_energy is not None else (
+            torch.empty(n, dtype=torch.float64, device="cuda") if atom_energy else None)
         vir = (ctypes.c_double * 9)() if virial else None
         rc = self._lib.umlmd_compute(self._h, _ptr(pos), ctypes.byref(e), _ptr(f), vir, _ptr(ea))
         if rc != OK:
@@ -285,6 +335,12 @@ class Model:
             self._raise(rc)
         self.n_atoms = 0
         return dict(energies=e, forces=f, atom_energy=ea, virials=vir.reshape(nf, 3, 3) if virial else None)
+
+    def set_owned_atoms(self, n_owned):
+        """Atoms with index >= n_owned are ghosts (neighbours only) from now on; negative: none."""
+        rc = self._lib.umlmd_set_owned_atoms(self._h, int(n_owned))
+        if rc != OK:
+            self._raise(rc)
 
     def set_md_state(self, pos, vel, masses):
         _check_dev(pos, torch.float64, "pos")

@@ -58,6 +58,20 @@ struct umlmd {
     double prof_ms[16] = {0};
     int64_t prof_launches[16] = {0};
     int64_t launches_total = 0;
+    // replay of repeated launch sequences as CUDA graphs (see run_replayed)
+    struct Replay {
+        cudaGraphExec_t exec = nullptr;
+        const void* key[4] = {nullptr, nullptr, nullptr, nullptr}; double key_dt = 0; int64_t key_serial = -1; int key_flags = 0;
+        bool seen = false;                           // the key's sequence has run once as plain launches
+        int64_t launches[16] = {0}; int64_t total = 0;   // what one replay launches, per class
+    };
+    Replay rp_compute, rp_step;
+    int launch_graphs = 0;                           // option: 0 = automatic, 1 = always, -1 = never
+    bool graphs_broken = false;                      // a capture failed on this handle: plain launches from then on
+    cudaStream_t cap_st = nullptr;                   // stream the sequences are captured on
+    int64_t n_owned = -1;                            // atoms [n_owned, N) are ghosts (neighbours only); negative = none
+    int64_t graph_replays = 0;
+    int64_t list_serial = 0;                         // bumped by everything that changes what a sequence launches
 };
 
 enum KernelClass { kGather = 0, kEdgeFwd, kInvFwd, kMlpFwd, kMlpBwd, kInvBwd, kEdgeBwd, kForce, kReduce, kIntegrate,
@@ -182,6 +196,8 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         for (int k = 0; k < 9; ++k) ea.H[k] = nb.H[k];
         ea.tri = nb.tri;
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
+        const bool ghosts = h->n_owned >= 0 && h->n_owned < N;
+        ea.perm = ghosts ? nb.perm : nullptr; ea.n_owned = ghosts ? (int)h->n_owned : N;
         ea.virial_part = h->virial_part + (size_t)vpart_used * 9;
         { Scope sc(h, kEdgeFwd, 1); API_CUDA(h, launch_edge_forward(ea, h->st)); }
         InvArgs ia;
@@ -202,6 +218,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit; ma.fold_x0 = fold_x0;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
         ma.spin_limit = h->gemm_spin_limit; ma.test_skip_kblock = h->fault_skip_stage;
+        ma.perm = ea.perm; ma.n_owned = ea.n_owned;
         h->fault_skip_stage = 0;                      // one shot
         { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
@@ -224,13 +241,87 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
     return UMLMD_OK;
 }
 
-// copy results and the error word to the host, synchronise, clear the error word
-int fetch_results(umlmd_t* h, int n_out) {
+// copy results and the error word to the host and clear the error word (enqueue_fetch), then
+// synchronise and decode (finish_fetch)
+int enqueue_fetch(umlmd_t* h, int n_out) {
     API_CUDA(h, cudaMemcpyAsync(h->h_out, h->d_out, sizeof(double) * n_out, cudaMemcpyDeviceToHost, h->st));
     API_CUDA(h, cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, h->st));
     API_CUDA(h, cudaMemsetAsync(h->d_err, 0, sizeof(int), h->st));
+    return UMLMD_OK;
+}
+int finish_fetch(umlmd_t* h) {
     API_CUDA(h, cudaStreamSynchronize(h->st));
     return decode_device_errors(h, *h->h_err);
+}
+int fetch_results(umlmd_t* h, int n_out) {
+    int rc = enqueue_fetch(h, n_out);
+    return rc != UMLMD_OK ? rc : finish_fetch(h);
+}
+
+// Replay of a repeated launch sequence.  A system of a few thousand atoms spends more time between
+// its two dozen kernels than inside them, so a sequence that recurs with the same arguments (an
+// evaluation of the same buffers, a middle step of an MD run between two list builds) is recorded
+// once as a CUDA graph and replayed with one launch.  `body` enqueues the sequence on h->st; `key`
+// names everything its launches depend on besides the handle's own state, which list_serial covers.
+// The first occurrence of a key runs as plain launches (it also performs every lazy one-time
+// initialisation of the launch helpers), the second is captured on a stream of the handle's own
+// (the caller's may be the legacy default stream, which cannot capture) and every later one
+// replayed.  A capture that fails for any reason leaves the handle on plain launches for good.
+bool replay_allowed(const umlmd_t* h) {
+    if (h->graphs_broken || h->prof_on || h->fault_skip_stage || h->launch_graphs < 0) return false;
+    if (h->launch_graphs > 0) return true;
+    return h->nb.N <= 65536 && h->nb.N <= h->node_tile;       // automatic: systems where launch latency shows
+}
+void replay_drop(umlmd_t::Replay& r) {
+    if (r.exec) cudaGraphExecDestroy(r.exec);
+    r.exec = nullptr;
+}
+template <class Body>
+int run_replayed(umlmd_t* h, umlmd_t::Replay& r, const void* k0, const void* k1, const void* k2, const void* k3,
+                 double dt, int flags, Body body) {
+    if (!replay_allowed(h)) return body();
+    const bool same = r.key[0] == k0 && r.key[1] == k1 && r.key[2] == k2 && r.key[3] == k3 && r.key_dt == dt &&
+                      r.key_flags == flags && r.key_serial == h->list_serial;
+    if (!same) {
+        replay_drop(r);
+        r.key[0] = k0; r.key[1] = k1; r.key[2] = k2; r.key[3] = k3; r.key_dt = dt; r.key_flags = flags;
+        r.key_serial = h->list_serial; r.seen = true;
+        return body();
+    }
+    if (!r.exec) {
+        if (!h->cap_st && cudaStreamCreateWithFlags(&h->cap_st, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError(); h->graphs_broken = true;
+            return body();
+        }
+        int64_t before[16], total = h->launches_total;
+        for (int c = 0; c < 16; ++c) before[c] = h->prof_launches[c];
+        cudaStream_t real = h->st;
+        h->st = h->cap_st;
+        int rc = UMLMD_OK;
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamBeginCapture(h->cap_st, cudaStreamCaptureModeRelaxed);
+        if (e == cudaSuccess) {
+            rc = body();
+            e = cudaStreamEndCapture(h->cap_st, &graph);
+            if (rc == UMLMD_OK && e == cudaSuccess) e = cudaGraphInstantiate(&r.exec, graph, 0);
+            if (graph) cudaGraphDestroy(graph);
+        }
+        h->st = real;
+        for (int c = 0; c < 16; ++c) { r.launches[c] = h->prof_launches[c] - before[c]; h->prof_launches[c] = before[c]; }
+        r.total = h->launches_total - total; h->launches_total = total;      // nothing has run yet
+        if (rc != UMLMD_OK || e != cudaSuccess || !r.exec) {
+            cudaGetLastError();
+            replay_drop(r);
+            h->graphs_broken = true;
+            h->err.clear();
+            return body();
+        }
+    }
+    for (int c = 0; c < 16; ++c) h->prof_launches[c] += r.launches[c];
+    h->launches_total += r.total;
+    ++h->graph_replays;
+    API_CUDA(h, cudaGraphLaunch(r.exec, h->st));
+    return UMLMD_OK;
 }
 
 // first use on a device: upload the model constants and allocate the small result buffers
@@ -279,6 +370,7 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
     h->have_list = true;
     h->have_edge_grad = false;       // edges were renumbered
     h->steps_since_build = 0;
+    ++h->list_serial;                // recorded launch sequences name the old list
     return ensure_workspace(h);
 }
 
@@ -340,6 +432,8 @@ int umlmd_create(const void* blob, size_t blob_bytes, const umlmd_options* opt, 
         if (opt->gemm_spin_limit < 0 || opt->fault_skip_gemm_stage < 0) { delete h; return UMLMD_E_INVALID_ARG; }
         h->gemm_spin_limit = opt->gemm_spin_limit;
         h->fault_skip_stage = opt->fault_skip_gemm_stage;
+        if (opt->launch_graphs < -1 || opt->launch_graphs > 1) { delete h; return UMLMD_E_INVALID_ARG; }
+        h->launch_graphs = opt->launch_graphs;
     }
     int rc = build_host_model(blob, blob_bytes, dx_override, &h->hm, &h->err);
     if (rc != UMLMD_OK) { delete h; return rc; }
@@ -358,6 +452,9 @@ int umlmd_destroy(umlmd_t* h) {
     for (void* p : ptrs) dev_free(p);
     for (auto& sp : h->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
+    if (h->rp_compute.exec) cudaGraphExecDestroy(h->rp_compute.exec);
+    if (h->rp_step.exec) cudaGraphExecDestroy(h->rp_step.exec);
+    if (h->cap_st) cudaStreamDestroy(h->cap_st);
     if (h->h_out) cudaFreeHost(h->h_out);
     if (h->h_err) cudaFreeHost(h->h_err);
     if (h->h_species) cudaFreeHost(h->h_species);
@@ -374,6 +471,7 @@ int umlmd_query(const umlmd_t* h, umlmd_info* out) {
     out->n_edges = h->have_list ? h->nb.E : 0;
     out->device_bytes = dev_bytes_held();
     out->kernel_launches = h->launches_total;
+    out->graph_replays = h->graph_replays;
     return UMLMD_OK;
 }
 
@@ -524,9 +622,12 @@ int umlmd_compute(umlmd_t* h, const double* d_pos, double* energy, double* d_for
         if (virial) for (int k = 0; k < 9; ++k) virial[k] = 0;
         return UMLMD_OK;
     }
-    int rc = enqueue_compute(h, d_pos, want_grad, d_force, d_atom_energy);
+    int rc = run_replayed(h, h->rp_compute, d_pos, d_force, d_atom_energy, nullptr, 0.0, want_grad ? 1 : 0, [&]() {
+        int r = enqueue_compute(h, d_pos, want_grad, d_force, d_atom_energy);
+        return r != UMLMD_OK ? r : enqueue_fetch(h, 10);
+    });
     if (rc != UMLMD_OK) return rc;
-    rc = fetch_results(h, 10);
+    rc = finish_fetch(h);
     if (rc != UMLMD_OK) return rc;
     if (energy) *energy = h->h_out[0];
     if (virial) for (int k = 0; k < 9; ++k) virial[k] = h->h_out[1 + k];
@@ -553,6 +654,7 @@ int umlmd_compute_batch(umlmd_t* h, int32_t n_frames, const int64_t* frame_offse
     int rc = ensure_device_model(h);
     if (rc != UMLMD_OK) return rc;
     h->have_list = false; h->have_md = false; h->have_edge_grad = false;     // the handle's list is replaced
+    ++h->list_serial;
     { Scope sc(h, kNeighbor, 5); rc = neighbor_build_batch(&h->nb, n_frames, frame_offsets, cells, pbc, d_pos, d_type, h->d.T, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) return rc;
     const bool want_grad = d_force != nullptr || virials != nullptr;
@@ -611,6 +713,7 @@ int umlmd_set_md_state(umlmd_t* h, double* d_pos, double* d_vel, const double* m
     if (h->nb.N > h->md_cap || !h->md_force) API_CUDA(h, dev_ensure(&h->md_force, &h->md_cap, h->nb.N * 3));
     h->md_pos = d_pos; h->md_vel = d_vel;
     h->have_md = true; h->have_force = false; h->nhc_reset = true;
+    ++h->list_serial;                // masses and buffers of the recorded step sequence may have changed
     return UMLMD_OK;
 }
 
@@ -668,6 +771,8 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
     if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
     if (!h->have_md) return fail(h, UMLMD_E_NO_MD_STATE, "umlmd_set_md_state must be called first");
     if (nsteps < 0 || !(dt_ps > 0) || !std::isfinite(dt_ps)) return fail(h, UMLMD_E_INVALID_ARG, "bad step count or time step");
+    if (h->n_owned >= 0 && h->n_owned < h->nb.N)
+        return fail(h, UMLMD_E_INVALID_ARG, "this driver integrates every atom of the handle; with ghost atoms use umlmd_compute and umlmd_vv_update");
     const int64_t N = h->nb.N;
     int rc;
     if (!h->have_force) {
@@ -680,9 +785,17 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
         if (s == 0) { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, nullptr, h->st)); }
         ++h->steps_since_build;
         if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return stop_run(h, rc);
-        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return stop_run(h, rc);
         const bool last = s + 1 == nsteps;
-        { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, nullptr, h->st)); }
+        auto body = [&]() {
+            int r = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr);
+            if (r != UMLMD_OK) return r;
+            Scope sc(h, kIntegrate, 1);
+            API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, last ? 1 : 2, !last, nullptr, h->st));
+            return (int)UMLMD_OK;
+        };
+        // a middle step between two list builds launches the same sequence as the one before it
+        rc = last ? body() : run_replayed(h, h->rp_step, h->md_pos, h->md_vel, h->md_force, nullptr, dt_ps, 0, body);
+        if (rc != UMLMD_OK) return stop_run(h, rc);
     }
     { Scope sc(h, kIntegrate, 2); API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, h->d_out + 10, h->st)); }
     rc = fetch_results(h, 11);
@@ -701,6 +814,8 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
         !(t_damp_ps > 0) || !std::isfinite(t_damp_ps))
         return fail(h, UMLMD_E_INVALID_ARG, "bad step count, time step, temperature or damping time");
     const int64_t N = h->nb.N;
+    if (h->n_owned >= 0 && h->n_owned < N)
+        return fail(h, UMLMD_E_INVALID_ARG, "this driver integrates every atom of the handle; with ghost atoms use umlmd_compute and umlmd_vv_update");
     if (N < 2) return fail(h, UMLMD_E_INVALID_ARG, "the thermostat needs at least two atoms");
     constexpr int M = kNhcChain;
     int rc;
@@ -767,6 +882,25 @@ int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial) {
     { Scope sc(h, kForce, 1); API_CUDA(h, launch_atom_virial(h->nb, h->g, d_atom_virial, h->st)); }
     API_CUDA(h, cudaStreamSynchronize(h->st));
     return UMLMD_OK;
+}
+
+int umlmd_set_owned_atoms(umlmd_t* h, int64_t n_owned) {
+    if (!h) return UMLMD_E_INVALID_ARG;
+    h->n_owned = n_owned < 0 ? -1 : n_owned;
+    h->have_force = false; h->have_edge_grad = false;
+    ++h->list_serial;                // recorded launch sequences carry the old count
+    return UMLMD_OK;
+}
+
+int umlmd_vv_update(int64_t N, double* d_pos, double* d_vel, const double* d_force, const int32_t* d_type,
+                    const double* d_inv_mass_per_type, double dt_ps, int32_t half_kicks, int32_t drift, void* stream) {
+    if (N < 0 || half_kicks < 0 || half_kicks > 2 || !(dt_ps > 0) || !std::isfinite(dt_ps)) return UMLMD_E_INVALID_ARG;
+    if (N > 0 && (!d_vel || !d_type || !d_inv_mass_per_type || (half_kicks > 0 && !d_force) || (drift && !d_pos)))
+        return UMLMD_E_INVALID_ARG;
+    if (N == 0 || (half_kicks == 0 && !drift)) return UMLMD_OK;
+    cudaError_t e = launch_vv_kick_drift(N, d_pos, d_vel, d_force, d_type, d_inv_mass_per_type, dt_ps, half_kicks, drift != 0,
+                                         nullptr, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? UMLMD_OK : UMLMD_E_CUDA;
 }
 
 int umlmd_get_intermediates(umlmd_t* h, float* d_state, float* d_desc) {

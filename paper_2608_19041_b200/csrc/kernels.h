@@ -64,6 +64,11 @@ struct EdgeArgs {
     const float* uni_scale;
     const int* species_slot;    // [T] species -> index among the species present
     int n_present;
+    // ghost atoms (copies of atoms another spatial domain owns): rows whose atom has caller index
+    // >= n_owned are neighbours only -- the forward pass leaves their sums at zero and the backward
+    // pass gives their edges a zero gradient.  perm: sorted -> caller index; null when every atom is owned
+    const int* perm;
+    int n_owned;
 };
 // present: device array of the n_present species indices, ascending
 cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
@@ -110,6 +115,8 @@ struct MlpArgs {
     int* err;               // device error word
     int spin_limit;         // tensor-core path: polls before a pipeline wait gives up (0 = default)
     int test_skip_kblock;   // diagnostic, first layer of the forward pass only: see GemmArgs
+    const int* perm;        // ghost atoms (see EdgeArgs): their atomic energy is zero; null when every atom is owned
+    int n_owned;
 };
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad

@@ -1,6 +1,6 @@
 """GPU tests of the boundary calls that are not the evaluation itself: the row-range export of the
-neighbor list, the workspace estimate, the thermostat checkpoint, and the give-up path of the
-tensor-core GEMM's bounded waits."""
+neighbor list, the workspace estimate, the thermostat checkpoint, the give-up path of the
+tensor-core GEMM's bounded waits, and the replay of repeated launch sequences as graphs."""
 
 import numpy as np
 import pytest
@@ -147,3 +147,57 @@ def test_thermostat_state_round_trip_continues_a_run_exactly():
     m3.step_nvt(every, md["dt_ps"], T, damp, every)
     assert not np.array_equal(vel3.cpu().numpy(), va)
     m3.close()
+
+
+@pytest.mark.parametrize("own_stream", [False, True])
+def test_replayed_launch_sequences_repeat_the_plain_launches_bit_for_bit(own_stream):
+    # Two handles on the same system, one with graph replay switched off and one with it forced on.
+    # Repeated evaluations into the same buffers (first plain, then recorded, then replayed) and an
+    # MD run that crosses two list builds must agree in every bit, and both handles must count
+    # the same kernel launches.  The caller's stream is the legacy default stream in one case (the
+    # sequence is then recorded on a stream of the handle's own) and a stream of its own in the other.
+    p = SMALL_PROFILES["p32_3_2"]
+    s = make_system(dict(kind="fcc", cells=4, a=4.05, jitter=0.05, seed=9, n_types=p["T"], masses=[20.0] * p["T"]))
+    blob = make_blob(p, seed=46, bias_scale=0.2, e_ref_scale=0.5)
+    stream = torch.cuda.Stream() if own_stream else None
+    with torch.cuda.stream(stream) if own_stream else torch.cuda.stream(torch.cuda.current_stream()):
+        plain, pos_a = _build(blob, s, skin=1.0, launch_graphs=-1, stream=stream)
+        graph, pos_b = _build(blob, s, skin=1.0, launch_graphs=1, stream=stream)
+        n = plain.n_atoms
+        fa = torch.empty((n, 3), dtype=torch.float64, device="cuda")
+        fb = torch.empty_like(fa)
+        ea = torch.empty(n, dtype=torch.float64, device="cuda")
+        eb = torch.empty_like(ea)
+        gen = torch.Generator(device="cuda").manual_seed(3)
+        for it in range(5):
+            oa = plain.compute(pos_a, out_forces=fa, out_atom_energy=ea)
+            ob = graph.compute(pos_b, out_forces=fb, out_atom_energy=eb)
+            torch.cuda.synchronize()
+            assert oa["energy"] == ob["energy"], it
+            assert np.array_equal(oa["virial"], ob["virial"]), it
+            assert torch.equal(fa, fb) and torch.equal(ea, eb), it
+            d = 0.01 * torch.randn(pos_a.shape, dtype=torch.float64, device="cuda", generator=gen)
+            pos_a += d                                         # same buffers, new contents
+            pos_b += d
+        assert plain.query()["kernel_launches"] == graph.query()["kernel_launches"]
+        # an energy-only evaluation is a different sequence: recorded separately, same results
+        for it in range(3):
+            assert plain.compute(pos_a, forces=False, virial=False)["energy"] == \
+                graph.compute(pos_b, forces=False, virial=False)["energy"]
+        vel = 0.5 * torch.randn(pos_a.shape, dtype=torch.float64, device="cuda", generator=gen)
+        va, vb = vel.clone(), vel.clone()
+        plain.set_md_state(pos_a, va, [20.0] * p["T"])
+        graph.set_md_state(pos_b, vb, [20.0] * p["T"])
+        for chunk in (7, 1, 25):                               # 33 steps: builds at steps 10, 20, 30
+            ra = plain.step(chunk, 0.001, rebuild_every=10)
+            rb = graph.step(chunk, 0.001, rebuild_every=10)
+            assert ra == rb
+            torch.cuda.synchronize()
+            assert torch.equal(pos_a, pos_b) and torch.equal(va, vb)
+        assert plain.query()["kernel_launches"] == graph.query()["kernel_launches"]
+        # 5 evaluations (one plain, four replayed), 3 energy-only (one plain), and of the 33 steps
+        # the three that end a call, the three with a list build (each the first with its list) and
+        # the first after the change of MD state run as plain launches
+        assert plain.query()["graph_replays"] == 0 and graph.query()["graph_replays"] == 4 + 2 + (33 - 3 - 3 - 1)
+    plain.close()
+    graph.close()
