@@ -293,15 +293,16 @@ int umlmd_set_nvt_state(umlmd_t* h, const double state[UMLMD_NVT_STATE_DOUBLES])
  * the atoms of its region, holds copies -- ghosts -- of the atoms within the list radius around it,
  * receives their coordinates before an evaluation and sends the forces on them back afterwards; no
  * learned quantity crosses a boundary because the model has a single aggregation layer).
- * After this call the atoms with index >= n_owned (caller's numbering) of every evaluation are
- * ghosts: they are neighbours only.  No atomic energy is computed for them (their entries of
+ * From the next umlmd_build_neighbors on (the call drops the current list: the library's internal
+ * order puts owned atoms first), the atoms with index >= n_owned (caller's numbering) are ghosts:
+ * they are neighbours only.  No atomic energy is computed for them (their entries of
  * d_atom_energy are 0, the energy is the sum over the owned atoms), only the edges that end on an
  * owned atom carry a gradient, and d_force holds for every atom, owned or ghost, minus the derivative
  * of that energy: the forces on ghosts are what has to be added to their owners' forces, and the
  * virial is the owned atoms' share, -sum over their edges of g (x) r.  Summed over all domains these
  * are the energy, forces and virial of the whole system.  The neighbor list is built over all
- * atoms as usual (give the domain's box as a non-periodic cell); ghosts cost their rows of the
- * per-atom stages but none of the per-edge work.
+ * atoms as usual (give the domain's box as a non-periodic cell); ghosts cost their share of the list
+ * build and of the force assembly, nothing else: no per-edge or per-atom stage visits their rows.
  *   n_owned   number of owned atoms, placed first; negative or >= N: every atom is owned (default)
  * umlmd_step and umlmd_step_nvt move every atom of the handle and refuse to run while ghosts are
  * set; a domain's driver uses umlmd_compute and umlmd_vv_update.  Not in the paper as an interface

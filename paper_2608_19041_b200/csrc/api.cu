@@ -179,12 +179,13 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
     const Dims& d = h->d;
     NeighborDev& nb = h->nb;
     const int N = (int)nb.N;
+    const int NR = (int)nb.n_owned;      // rows that are evaluated: the owned atoms, first in the internal order
     // (a batched list was built from these very positions: nothing to gather)
     if (!nb.batch) { Scope sc(h, kGather, 1); API_CUDA(h, launch_gather_positions(nb, d_pos, h->d_err, h->st)); }
     const int B = N < h->node_tile ? N : h->node_tile;
     int vpart_used = 0;
-    for (int a0 = 0; a0 < N; a0 += B) {
-        const int n = N - a0 < B ? N - a0 : B;
+    for (int a0 = 0; a0 < NR; a0 += B) {
+        const int n = NR - a0 < B ? NR - a0 : B;
         EdgeArgs ea;
         ea.d = d; ea.table = h->md.table; ea.pairmod = h->md.pairmod; ea.xs = nb.xs; ea.rec = nb.rec; ea.type_s = nb.type_s;
         ea.table_uni = h->pair_tables ? h->table_uni : nullptr;
@@ -196,8 +197,6 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         for (int k = 0; k < 9; ++k) ea.H[k] = nb.H[k];
         ea.tri = nb.tri;
         ea.a0 = a0; ea.a1 = a0 + n; ea.state = h->state; ea.g = h->g;
-        const bool ghosts = h->n_owned >= 0 && h->n_owned < N;
-        ea.perm = ghosts ? nb.perm : nullptr; ea.n_owned = ghosts ? (int)h->n_owned : N;
         ea.virial_part = h->virial_part + (size_t)vpart_used * 9;
         { Scope sc(h, kEdgeFwd, 1); API_CUDA(h, launch_edge_forward(ea, h->st)); }
         InvArgs ia;
@@ -218,7 +217,6 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         ma.tc_hi = h->tc_hi; ma.tc_lo = h->tc_lo; ma.err = h->d_err; ma.desc_presplit = presplit; ma.fold_x0 = fold_x0;
         ma.tc_slot = (size_t)h->tile_cap * (size_t)(d.DP > d.F ? d.DP : d.F);
         ma.spin_limit = h->gemm_spin_limit; ma.test_skip_kblock = h->fault_skip_stage;
-        ma.perm = ea.perm; ma.n_owned = ea.n_owned;
         h->fault_skip_stage = 0;                      // one shot
         { Scope sc(h, kMlpFwd, d.n_hidden + 1); API_CUDA(h, launch_mlp_forward(ma, h->st)); }
         if (want_grad) {
@@ -365,13 +363,22 @@ int build_list(umlmd_t* h, int64_t N, const double* d_pos, const int32_t* d_type
                const int pbc[3], double skin) {
     int rc = ensure_device_model(h);
     if (rc != UMLMD_OK) return rc;
-    { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, d_pos, d_type, cell, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
+    { Scope sc(h, kNeighbor, 7); rc = neighbor_build(&h->nb, N, h->n_owned, d_pos, d_type, cell, pbc, skin, h->hm.rc, h->d_err, h->st, &h->err); }
     if (rc != UMLMD_OK) { h->have_list = false; return rc; }
     h->have_list = true;
     h->have_edge_grad = false;       // edges were renumbered
     h->steps_since_build = 0;
     ++h->list_serial;                // recorded launch sequences name the old list
-    return ensure_workspace(h);
+    rc = ensure_workspace(h);
+    if (rc != UMLMD_OK) return rc;
+    if (h->nb.n_owned < h->nb.N) {
+        // ghost atoms come last in the internal order and no stage visits their rows: their atomic
+        // energies and the gradients of their edges are zero from here until the next build
+        API_CUDA(h, cudaMemsetAsync(h->e_atom + h->nb.n_owned, 0, sizeof(double) * (size_t)(h->nb.N - h->nb.n_owned), h->st));
+        if (h->nb.E > h->nb.E_owned)
+            API_CUDA(h, cudaMemsetAsync(h->g + 3 * (size_t)h->nb.E_owned, 0, sizeof(float) * 3 * (size_t)(h->nb.E - h->nb.E_owned), h->st));
+    }
+    return UMLMD_OK;
 }
 
 // With few species present, psi_c(rho) of every ordered pair among them is tabulated by itself,
@@ -771,7 +778,7 @@ int umlmd_step(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, double* 
     if (!h->have_list) return fail(h, UMLMD_E_NO_NEIGHBORS, "umlmd_build_neighbors must be called first");
     if (!h->have_md) return fail(h, UMLMD_E_NO_MD_STATE, "umlmd_set_md_state must be called first");
     if (nsteps < 0 || !(dt_ps > 0) || !std::isfinite(dt_ps)) return fail(h, UMLMD_E_INVALID_ARG, "bad step count or time step");
-    if (h->n_owned >= 0 && h->n_owned < h->nb.N)
+    if (h->nb.n_owned < h->nb.N)
         return fail(h, UMLMD_E_INVALID_ARG, "this driver integrates every atom of the handle; with ghost atoms use umlmd_compute and umlmd_vv_update");
     const int64_t N = h->nb.N;
     int rc;
@@ -814,7 +821,7 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
         !(t_damp_ps > 0) || !std::isfinite(t_damp_ps))
         return fail(h, UMLMD_E_INVALID_ARG, "bad step count, time step, temperature or damping time");
     const int64_t N = h->nb.N;
-    if (h->n_owned >= 0 && h->n_owned < N)
+    if (h->nb.n_owned < N)
         return fail(h, UMLMD_E_INVALID_ARG, "this driver integrates every atom of the handle; with ghost atoms use umlmd_compute and umlmd_vv_update");
     if (N < 2) return fail(h, UMLMD_E_INVALID_ARG, "the thermostat needs at least two atoms");
     constexpr int M = kNhcChain;
@@ -887,8 +894,9 @@ int umlmd_atom_virial(umlmd_t* h, double* d_atom_virial) {
 int umlmd_set_owned_atoms(umlmd_t* h, int64_t n_owned) {
     if (!h) return UMLMD_E_INVALID_ARG;
     h->n_owned = n_owned < 0 ? -1 : n_owned;
-    h->have_force = false; h->have_edge_grad = false;
-    ++h->list_serial;                // recorded launch sequences carry the old count
+    // the internal order of the atoms depends on it: the next evaluation needs a new list
+    h->have_list = false; h->have_md = false; h->have_force = false; h->have_edge_grad = false;
+    ++h->list_serial;
     return UMLMD_OK;
 }
 

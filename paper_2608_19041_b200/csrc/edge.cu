@@ -327,7 +327,6 @@ k_edge_forward(const EdgeArgs a) {
     const eidx_t e0 = a.row_ptr[i];
     const int len = (int)(a.row_ptr[i + 1] - e0);      // edge offsets are 64-bit, offsets inside a row are not
     const double* Hf = a.frames ? a.frames[a.frame_of[i]].H : nullptr;
-    const bool ghost = a.perm && a.perm[i] >= a.n_owned;    // a neighbour only: its own sums stay zero
     const unsigned lt_mask = (1u << lane) - 1u;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
     float accH[W::NCH];
@@ -439,7 +438,7 @@ k_edge_forward(const EdgeArgs a) {
 
     int qn = 0;
     for (int base = 0; base < len; base += 32) {
-        const Geom g = edge_geometry(a, e0 + base + lane, base + lane < len && !ghost, xi, yi, zi, ti, Hf);
+        const Geom g = edge_geometry(a, e0 + base + lane, base + lane < len, xi, yi, zi, ti, Hf);
         const unsigned vmask = __ballot_sync(kFull, g.valid);
         const int p = qn + __popc(vmask & lt_mask);       // queue slot of this lane's edge, if it has one
         if (g.valid) { const double c2 = (double)g.chi * (double)g.chi; s0 += c2; s1 += c2 * c2; }
@@ -524,7 +523,6 @@ k_edge_backward(const EdgeArgs a) {
         const eidx_t e0 = a.row_ptr[i];
         const int len = (int)(a.row_ptr[i + 1] - e0);
         const double* Hf = a.frames ? a.frames[a.frame_of[i]].H : nullptr;
-        const bool ghost = a.perm && a.perm[i] >= a.n_owned;    // a neighbour only: its edges carry no gradient
         const float* grow = a.state + (size_t)(i - a.a0) * a.d.SP;
         float h0[4 * G];
 #pragma unroll
@@ -649,7 +647,7 @@ k_edge_backward(const EdgeArgs a) {
         int qn = 0;
         for (int base = 0; base < len; base += 32) {
             const int e = base + lane;                                // offset inside the row
-            const Geom g = edge_geometry(a, e0 + e, e < len && !ghost, xi, yi, zi, ti, Hf);
+            const Geom g = edge_geometry(a, e0 + e, e < len, xi, yi, zi, ti, Hf);
             const unsigned vmask = __ballot_sync(kFull, g.valid);
             const int p = qn + __popc(vmask & lt_mask);   // queue slot of this lane's edge, if it has one
             if (g.valid && p < 32) {

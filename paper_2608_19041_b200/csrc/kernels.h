@@ -10,7 +10,10 @@ namespace umd {
 // ---- neighbor.cu ---------------------------------------------------------------------
 // Full build: fold + bin + sort + count + scan + fill + reverse map.  Synchronises once
 // (to learn the edge count and grow the edge arrays).  Returns a UMLMD_* code.
-int neighbor_build(NeighborDev* nb, int64_t N, const double* d_pos, const int32_t* d_type,
+// n_owned < N: the atoms with caller index >= n_owned are ghosts; they come after all owned atoms
+// in the internal order (owned atoms in cell order, then ghosts in cell order), so that rows
+// [0, n_owned) are the owned atoms' and nb->E_owned edges belong to them.
+int neighbor_build(NeighborDev* nb, int64_t N, int64_t n_owned, const double* d_pos, const int32_t* d_type,
                    const double cell[9], const int pbc[3], double skin, double rc, int* d_err,
                    cudaStream_t st, std::string* err);   // cell: the three cell vectors as rows
 void neighbor_free(NeighborDev* nb);
@@ -64,11 +67,6 @@ struct EdgeArgs {
     const float* uni_scale;
     const int* species_slot;    // [T] species -> index among the species present
     int n_present;
-    // ghost atoms (copies of atoms another spatial domain owns): rows whose atom has caller index
-    // >= n_owned are neighbours only -- the forward pass leaves their sums at zero and the backward
-    // pass gives their edges a zero gradient.  perm: sorted -> caller index; null when every atom is owned
-    const int* perm;
-    int n_owned;
 };
 // present: device array of the n_present species indices, ascending
 cudaError_t launch_fuse_pair_tables(const Dims& d, const float* table, const float* pairmod, const int* present,
@@ -115,8 +113,6 @@ struct MlpArgs {
     int* err;               // device error word
     int spin_limit;         // tensor-core path: polls before a pipeline wait gives up (0 = default)
     int test_skip_kblock;   // diagnostic, first layer of the forward pass only: see GemmArgs
-    const int* perm;        // ghost atoms (see EdgeArgs): their atomic energy is zero; null when every atom is owned
-    int n_owned;
 };
 cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st);   // layers + head (+ backward seed)
 cudaError_t launch_mlp_backward(const MlpArgs& a, cudaStream_t st);  // needs a forward with want_grad

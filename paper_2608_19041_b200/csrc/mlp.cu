@@ -64,18 +64,16 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const GemmArgs g) {
 // dE/dY_last = w_head * SiLU'(Y_last)
 __global__ void k_head(int n, int F, const float* __restrict__ h, const float* __restrict__ w, float b_head,
                        const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
-                       float* __restrict__ pre_last, double* __restrict__ e_atom, bool want_grad,
-                       const int* __restrict__ perm, int n_owned) {
+                       float* __restrict__ pre_last, double* __restrict__ e_atom, bool want_grad) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= n) return;
-    const bool ghost = perm && perm[a0 + warp] >= n_owned;
     const float* hr = h + (size_t)warp * F;
     float s = 0.f;
     for (int f = lane; f < F; f += 32) s += hr[f] * __ldg(w + f);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
     if (lane == 0)
-        e_atom[a0 + warp] = ghost ? 0.0 : (double)s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + warp]);
+        e_atom[a0 + warp] = (double)s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + warp]);
     if (want_grad) {
         float* pr = pre_last + (size_t)warp * F;
         for (int f = lane; f < F; f += 32) {
@@ -88,10 +86,9 @@ __global__ void k_head(int n, int F, const float* __restrict__ h, const float* _
 // tensor-core path: the last layer's epilogue left one partial dot product per column tile
 __global__ void k_head_finish(int n, int parts, const float* __restrict__ part, float b_head,
                               const float* __restrict__ e_ref, const int* __restrict__ type_s, int a0,
-                              double* __restrict__ e_atom, const int* __restrict__ perm, int n_owned) {
+                              double* __restrict__ e_atom) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    if (perm && perm[a0 + i] >= n_owned) { e_atom[a0 + i] = 0.0; return; }     // a ghost atom has no energy of its own here
     double s = 0.0;
     for (int p = 0; p < parts; ++p) s += (double)part[(size_t)i * parts + p];
     e_atom[a0 + i] = s + (double)b_head + (double)__ldg(e_ref + type_s[a0 + i]);
@@ -176,13 +173,13 @@ cudaError_t launch_mlp_forward(const MlpArgs& a, cudaStream_t st) {
     if (tc) {
         const int parts = gemm_tc_head_parts(F, variant);
         k_head_finish<<<(n + 255) / 256, 256, 0, st>>>(n, parts, hb[(NH - 1) & 1], a.m.b_head, a.m.e_ref, a.type_s, a.a0,
-                                                        a.e_atom, a.perm, a.n_owned);
+                                                        a.e_atom);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     } else {
         const int warps = 8, blocks = (n + warps - 1) / warps;
         k_head<<<blocks, warps * 32, 0, st>>>(n, F, hb[(NH - 1) & 1], a.m.w_head, a.m.b_head, a.m.e_ref, a.type_s,
                                              a.a0, a.want_grad ? a.pre + (size_t)(NH - 1) * layer : nullptr,
-                                             a.e_atom, a.want_grad, a.perm, a.n_owned);
+                                             a.e_atom, a.want_grad);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -32,6 +32,9 @@ struct Grid {
     int nc[3];          // bins per direction
     int m[3];           // bin reach per direction
     int pbc[3];
+    int ncell;          // bins in all
+    int halves;         // 2 when ghost atoms are binned apart from owned ones (keys ncell .. 2 ncell - 1), else 1
+    int n_owned;        // caller indices >= n_owned are ghosts
     int sorted;         // every periodic direction has at least 2 m + 1 bins: bins are visited in
                         // increasing bin index, so each row comes out sorted by neighbour index
 };
@@ -107,7 +110,7 @@ __global__ void k_fold_bin(int N, const double* __restrict__ pos, Grid g, double
         atomicOr(err, kErrNonFinite);
         c[0] = c[1] = c[2] = 0;
     }
-    key[i] = (c[2] * g.nc[1] + c[1]) * g.nc[0] + c[0];
+    key[i] = (c[2] * g.nc[1] + c[1]) * g.nc[0] + c[0] + (i >= g.n_owned ? g.ncell : 0);
     idx[i] = i;
 }
 
@@ -149,7 +152,8 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     const int lane = threadIdx.x & 31;
     if (warp >= N) return;
     const int i = warp;
-    const int key = skey[i];
+    int key = skey[i];
+    if (key >= g.ncell) key -= g.ncell;         // a ghost's own bin
     const int cx = key % g.nc[0], cy = (key / g.nc[0]) % g.nc[1], cz = key / (g.nc[0] * g.nc[1]);
     const double xi = xs0[3 * (size_t)i], yi = xs0[3 * (size_t)i + 1], zi = xs0[3 * (size_t)i + 2];
     int count = 0;
@@ -159,6 +163,9 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
     const int sz0 = walk_start(cz, g.m[2], g.nc[2], g.pbc[2], g.sorted);
     const int sy0 = walk_start(cy, g.m[1], g.nc[1], g.pbc[1], g.sorted);
     const int sx0 = walk_start(cx, g.m[0], g.nc[0], g.pbc[0], g.sorted);
+    // with ghosts the bins are walked twice, owned atoms first: ghosts follow every owned atom in
+    // the internal order, so the row still ascends in the neighbour index
+    for (int half = 0; half < g.halves; ++half)
     for (int tz = 0; tz < wz; ++tz) {
         int dz = sz0 + tz;
         if (dz > g.m[2]) dz -= wz;
@@ -197,7 +204,7 @@ __global__ void k_scan_cells(int N, Grid g, double rl2, const int* __restrict__ 
                 }
                 const double sx = __dadd_rn(syx, __dmul_rn((double)nx, g.H[0])), sy = __dadd_rn(syy, __dmul_rn((double)nx, g.H[1])),
                              sz = __dadd_rn(syz, __dmul_rn((double)nx, g.H[2]));
-                const int cell = (zc * g.nc[1] + yc) * g.nc[0] + xc;
+                const int cell = (zc * g.nc[1] + yc) * g.nc[0] + xc + half * g.ncell;
                 const int beg = cell_start[cell], end = cell_start[cell + run];
                 const bool self_img = (nx == 0 && ny == 0 && nz == 0);
                 for (int b = beg; b < end; b += 32) {
@@ -460,11 +467,12 @@ void neighbor_free(NeighborDev* nb) {
     *nb = NeighborDev();
 }
 
-int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int32_t* d_type,
+int neighbor_build(NeighborDev* nb, int64_t N64, int64_t n_owned64, const double* d_pos, const int32_t* d_type,
                    const double cell[9], const int pbc[3], double skin, double rc, int* d_err,
                    cudaStream_t st, std::string* err) {
     if (N64 > 0x7fff0000LL) { *err = "too many atoms for 32-bit indices"; return UMLMD_E_INVALID_ARG; }
     const int N = (int)N64;
+    const int n_owned = n_owned64 < 0 || n_owned64 > N64 ? N : (int)n_owned64;
     const double r_list = rc + skin;
     nb->batch = false; nb->n_frames = 0; nb->frame_of = nullptr;
     Grid g;
@@ -536,8 +544,10 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     g.sorted = 1;
     for (int k = 0; k < 3; ++k)
         if (g.pbc[k] && g.nc[k] < 2 * g.m[k] + 1) g.sorted = 0;
+    g.ncell = (int)ncell; g.n_owned = n_owned; g.halves = n_owned < N ? 2 : 1;
+    const int64_t nkeys = (int64_t)g.halves * ncell;
 
-    nb->N = N; nb->skin = skin; nb->r_list = r_list;
+    nb->N = N; nb->skin = skin; nb->r_list = r_list; nb->n_owned = n_owned; nb->E_owned = 0;
     for (int k = 0; k < 3; ++k) { nb->L[k] = L[k]; nb->pbc[k] = pbc[k] ? 1 : 0; }
     for (int k = 0; k < 9; ++k) nb->H[k] = cell[k];
     nb->tri = g.tri;
@@ -562,13 +572,13 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
         c = 0; NB_CHECK(dev_ensure(&nb->deg, &c, need + 1));
         nb->N_cap = N;
     }
-    NB_CHECK(dev_ensure(&nb->cell_start, &nb->ncell_cap, ncell + 2));
+    NB_CHECK(dev_ensure(&nb->cell_start, &nb->ncell_cap, nkeys + 2));
     int* img_o = nb->img + 3 * (size_t)(N + 1);
 
     const int TB = 256;
     k_fold_bin<<<(N + TB - 1) / TB, TB, 0, st>>>(N, d_pos, g, nb->wpos, img_o, nb->key, nb->idx, d_err);
     int end_bit = 1;
-    while ((1LL << end_bit) < ncell) ++end_bit;
+    while ((1LL << end_bit) < nkeys) ++end_bit;
     size_t need_tmp = 0, need_scan = 0;
     cub::DeviceRadixSort::SortPairs(nullptr, need_tmp, nb->key, nb->key2, nb->idx, nb->idx2, N, 0, end_bit, st);
     // row offsets are accumulated in 64 bits from the 32-bit row lengths
@@ -587,7 +597,7 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     size_t tmp_bytes = nb->cub_bytes;
     NB_CHECK(cub::DeviceRadixSort::SortPairs(nb->cub_tmp, tmp_bytes, nb->key, nb->key2, nb->idx, nb->idx2, N,
                                              0, end_bit, st));
-    k_cell_start<<<(int)((ncell + 1 + TB - 1) / TB), TB, 0, st>>>((int)ncell, N, nb->key2, nb->cell_start);
+    k_cell_start<<<(int)((nkeys + 1 + TB - 1) / TB), TB, 0, st>>>((int)nkeys, N, nb->key2, nb->cell_start);
     k_gather_sorted<<<(N + TB - 1) / TB, TB, 0, st>>>(N, nb->idx2, nb->wpos, img_o, d_type, nb->perm, nb->xs0,
                                                       nb->xs, nb->img, nb->type_s);
     const double rl2 = r_list * r_list;
@@ -598,10 +608,12 @@ int neighbor_build(NeighborDev* nb, int64_t N64, const double* d_pos, const int3
     NB_CHECK(cudaMemsetAsync(nb->deg + N, 0, sizeof(int), st));
     tmp_bytes = nb->cub_bytes;
     NB_CHECK(cub::DeviceScan::ExclusiveScan(nb->cub_tmp, tmp_bytes, deg_wide, nb->row_ptr, cub::Sum(), (eidx_t)0, N + 1, st));
-    eidx_t total = 0;
+    eidx_t total = 0, total_owned = 0;
     NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(total), cudaMemcpyDeviceToHost, st));
+    if (n_owned < N) NB_CHECK(cudaMemcpyAsync(&total_owned, nb->row_ptr + n_owned, sizeof(total_owned), cudaMemcpyDeviceToHost, st));
     NB_CHECK(cudaStreamSynchronize(st));
     nb->E = total;
+    nb->E_owned = n_owned < N ? total_owned : total;
     if (total > nb->E_cap) {
         int64_t c;
         c = 0; NB_CHECK(dev_ensure(&nb->src, &c, total, 1.1));
@@ -716,6 +728,7 @@ int neighbor_build_batch(NeighborDev* nb, int n_frames, const int64_t* offsets, 
     NB_CHECK(cudaMemcpyAsync(&total, nb->row_ptr + N, sizeof(total), cudaMemcpyDeviceToHost, st));
     NB_CHECK(cudaStreamSynchronize(st));
     nb->E = total;
+    nb->n_owned = N; nb->E_owned = total;
     if (total > nb->E_cap) {
         int64_t c;
         c = 0; NB_CHECK(dev_ensure(&nb->src, &c, total, 1.1));

@@ -142,10 +142,14 @@ def test_ghost_atoms_have_no_energy_and_owned_forces_need_their_return():
     full = m.compute(pos, atom_energy=True)
     n_own = 25
     m.set_owned_atoms(n_own)
+    with pytest.raises(B.UmlmdError):                    # the list has to be rebuilt: owned atoms come first inside
+        m.compute(pos)
+    m.build_neighbors(pos, types, s["cell"], (0, 0, 0), 0.5)
     part = m.compute(pos, atom_energy=True)
-    assert torch.equal(part["atom_energy"][:n_own], full["atom_energy"][:n_own])
+    # (the rows list their neighbours in another order now: fp32 sums differ in the last bits)
+    assert (part["atom_energy"][:n_own] - full["atom_energy"][:n_own]).abs().max().item() < 2e-6 * full["atom_energy"].abs().max().item()
     assert part["atom_energy"][n_own:].abs().max().item() == 0.0
-    assert abs(part["energy"] - full["atom_energy"][:n_own].sum().item()) < 1e-9 * abs(full["energy"])
+    assert abs(part["energy"] - part["atom_energy"].sum().item()) < 1e-9 * abs(full["energy"])
     h = 2e-3
     for k, ax in ((3, 0), (n_own + 4, 1), (n_own + 20, 2)):      # an owned atom and two ghosts
         pp, pm = pos.clone(), pos.clone()
@@ -158,6 +162,7 @@ def test_ghost_atoms_have_no_energy_and_owned_forces_need_their_return():
         m.set_md_state(pos, vel, s["masses"])
         m.step(1, 0.001, 0)
     m.set_owned_atoms(-1)
+    m.build_neighbors(pos, types, s["cell"], (0, 0, 0), 0.5)
     again = m.compute(pos, atom_energy=True)
     assert again["energy"] == full["energy"] and torch.equal(again["forces"], full["forces"])
     m.close()
