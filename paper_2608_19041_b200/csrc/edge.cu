@@ -266,6 +266,15 @@ template <int C0, int L, int G = 1> struct Widths {
     // accesses of 8 consecutive lanes on distinct bank groups
     static constexpr int PF = ((C1 / 4 + 1) & 1) ? C1 + 4 : C1 + 8;          // forward: psi
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
+    // forward, sums of degree >= 1: a job is four consecutive channels of one harmonic component
+    // (degrees 1 and 2) or one component of a one-channel degree (3, 4); a lane owns up to SLOTS jobs
+    static constexpr int J1 = 3 * (C1 / 4), J2 = 5 * (C2 / 4), J3 = L >= 3 ? 7 : 0, J4 = L >= 4 ? 9 : 0;
+    static constexpr int NJ = J1 + J2 + J3 + J4;
+    static constexpr int SLOTS = (NJ + 31) / 32;
+    static constexpr int NM = 3 + 5 + J3 + J4;  // harmonic components of all degrees >= 1
+    static constexpr int PW = NM | 1;           // odd row pitch of the parked weights
+    static constexpr int WOFF = 32 * PF;        // they sit behind the parked amplitudes (where the radial modes were)
+    static constexpr int SCRATCH = 32 * PF + (32 * PW > 32 * kMaxR ? 32 * PW : 32 * kMaxR);
 };
 
 // The channel-parallel phase of the backward pass waits on load latency, and what hides it best
@@ -293,9 +302,11 @@ template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared 
 //   2. lanes = channels (a group of C0/4 lanes per edge): amplitude psi of all C0 channels,
 //      degree-0 sums accumulated in registers; the leading C1 amplitudes of each edge are
 //      parked in shared memory.
-//   3. lane = edge again: harmonics and the chi^2 psi_c B_lm products of degree >= 1 for the
-//      lane's own edge, summed over the batch by a shared-memory transpose (32 values at a
-//      time), so that lane v ends up owning sums v, v+32, v+64 of the flattened block.
+//   3. lane = edge again: harmonics of the lane's own edge, parked as weights chi^2 B_lm; then
+//      lane = job: a lane owns four consecutive channels of one harmonic component (or one
+//      component of a one-channel degree) for the whole row, and for every edge of the batch adds
+//      weight x amplitudes from the two parked rows: two shared-memory reads per edge and warp,
+//      where summing per-edge products by transposition took six.
 // Up to C0 = 64 a fourth resident block per SM (64 registers, a few spilled words) is worth more
 // than the registers: the channel-parallel phase waits on load latency (measured: 6-10 % on the
 // forward kernel at C0 = 8 .. 64, 2 % the other way at C0 = 128, which stays at three blocks).
@@ -303,9 +314,9 @@ template <int C0, int L, bool HASR, bool UNI>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, C0 <= 64 ? 4 : 3)
 k_edge_forward(const EdgeArgs a) {
     using W = Widths<C0, L>;
-    // one 32 x 33 float scratch per warp: first the parked amplitudes (row pitch PF), then,
-    // once every lane has read its own row, the transpose buffer
-    __shared__ __align__(16) float scratch[kWarpsPerBlock][32 * 33];
+    // scratch per warp: the parked amplitudes of the batch (row pitch PF), and behind them first the
+    // radial modes, then (once the amplitudes are done) the harmonic weights chi^2 B_lm (row pitch PW)
+    __shared__ __align__(16) float scratch[kWarpsPerBlock][W::SCRATCH];
     // queue of edges inside the cutoff: row, pair, t, chi (fetched with one 16-byte broadcast
     // load in the channel-parallel phase; shuffles would go through the same L1 data pipe as
     // the table reads) and the edge vector
@@ -315,9 +326,8 @@ k_edge_forward(const EdgeArgs a) {
     const int i = a.a0 + blockIdx.x * kWarpsPerBlock + wid;
     if (i >= a.a1) return;
     float* const psi_s = scratch[wid];      // [32][PF]
-    float* const tr = scratch[wid];         // [32][33]
-    float* const qm = scratch[wid] + 32 * W::PF;   // [32][kMaxR] radial modes, behind the parked amplitudes
-    static_assert(32 * W::PF + 32 * kMaxR <= 32 * 33, "scratch too small for the parked radial modes");
+    float* const qm = scratch[wid] + W::WOFF;      // [32][kMaxR] radial modes, behind the parked amplitudes
+    float* const wbs = scratch[wid] + W::WOFF;     // [32][PW] harmonic weights, in the same place later
     int4* const qes = q_es[wid];
     float* const qd = q_d[wid];
     const int sub = lane / W::LPE, cl = lane % W::LPE, c = 4 * cl;
@@ -329,9 +339,27 @@ k_edge_forward(const EdgeArgs a) {
     const double* Hf = a.frames ? a.frames[a.frame_of[i]].H : nullptr;
     const unsigned lt_mask = (1u << lane) - 1u;
     float acc0[4] = {0.f, 0.f, 0.f, 0.f};
-    float accH[W::NCH];
+    // this lane's jobs of the degree >= 1 sums: offset of the four channels in an amplitude row,
+    // of the component in a weight row, of the result in the output block (negative: no job)
+    float accJ[W::SLOTS][4];
+    int j_psi[W::SLOTS], j_w[W::SLOTS], j_out[W::SLOTS];
 #pragma unroll
-    for (int j = 0; j < W::NCH; ++j) accH[j] = 0.f;
+    for (int sl = 0; sl < W::SLOTS; ++sl) {
+        accJ[sl][0] = accJ[sl][1] = accJ[sl][2] = accJ[sl][3] = 0.f;
+        const int j = lane + 32 * sl;
+        if (j < W::J1) {
+            const int m = j / (W::C1 / 4), cb = j % (W::C1 / 4);
+            j_psi[sl] = 4 * cb; j_w[sl] = m; j_out[sl] = m * W::C1 + 4 * cb;
+        } else if (j < W::J1 + W::J2) {
+            const int jj = j - W::J1, m = jj / (W::C2 / 4), cb = jj % (W::C2 / 4);
+            j_psi[sl] = 4 * cb; j_w[sl] = 3 + m; j_out[sl] = 3 * W::C1 + m * W::C2 + 4 * cb;
+        } else if (j < W::NJ) {
+            const int m = j - W::J1 - W::J2;             // degrees 3 and 4 follow each other in both layouts
+            j_psi[sl] = 0; j_w[sl] = 8 + m; j_out[sl] = 3 * W::C1 + 5 * W::C2 + m;
+        } else {
+            j_psi[sl] = 0; j_w[sl] = 0; j_out[sl] = -1;
+        }
+    }
     double s0 = 0.0, s1 = 0.0;   // normaliser sums in double: the calibration subtracts their mean
 
     auto run_batch = [&](const int nb) {     // the first nb queue slots
@@ -373,67 +401,41 @@ k_edge_forward(const EdgeArgs a) {
                 *reinterpret_cast<float4*>(psi_s + b * W::PF + c) = make_float4(psi[0], psi[1], psi[2], psi[3]);
         }
         __syncwarp();
-        // lane = edge: products of degree >= 1, then batch sums by transposition
-        float ps[W::C1];
-        float B1[3], B2[5], B3[7], B4[9];
-        float w = 0.f;
+        // lane = edge: the harmonic weights chi^2 B_lm of the lane's edge, parked next to the amplitudes
         if (lane < nb) {
-#pragma unroll
-            for (int q = 0; q < W::C1 / 4; ++q) {
-                const float4 p4 = *reinterpret_cast<const float4*>(psi_s + lane * W::PF + 4 * q);
-                ps[4 * q] = p4.x; ps[4 * q + 1] = p4.y; ps[4 * q + 2] = p4.z; ps[4 * q + 3] = p4.w;
-            }
+            float B1[3], B2[5], B3[7], B4[9];
             const float dx = qd[lane], dy = qd[32 + lane], dz = qd[64 + lane];
             const float inv_rho = 1.0f / sqrtf(dx * dx + dy * dy + dz * dz + kEpsReg * kEpsReg);
             harmonics_s1<L>(dx * inv_rho, dy * inv_rho, dz * inv_rho, B1, B2, B3, B4);
             const float chi = __int_as_float(qes[lane].w);
-            w = chi * chi;
-        } else {
+            const float w = chi * chi;
+            float* wr = wbs + lane * W::PW;
 #pragma unroll
-            for (int q = 0; q < W::C1; ++q) ps[q] = 0.f;
+            for (int m = 0; m < 3; ++m) wr[m] = w * B1[m];
 #pragma unroll
-            for (int q = 0; q < 3; ++q) B1[q] = 0.f;
+            for (int m = 0; m < 5; ++m) wr[3 + m] = w * B2[m];
+            if (L >= 3) {
 #pragma unroll
-            for (int q = 0; q < 5; ++q) B2[q] = 0.f;
-#pragma unroll
-            for (int q = 0; q < 7; ++q) B3[q] = 0.f;
-#pragma unroll
-            for (int q = 0; q < 9; ++q) B4[q] = 0.f;
-        }
-        __syncwarp();                           // amplitudes are in registers: reuse the scratch
-        int vv = 0;
-        auto emit = [&](float val) {
-            tr[(vv & 31) * 33 + lane] = val;
-            ++vv;
-            if ((vv & 31) == 0 || vv == W::NHI) {
-                __syncwarp();
-                float s = 0.f;
-#pragma unroll
-                for (int l = 0; l < 32; ++l) s += tr[lane * 33 + l];
-                accH[(vv - 1) >> 5] += s;
-                __syncwarp();
+                for (int m = 0; m < 7; ++m) wr[8 + m] = w * B3[m];
             }
-        };
+            if (L >= 4) {
 #pragma unroll
-        for (int m = 0; m < 3; ++m) {
-            const float wb = w * B1[m];
-#pragma unroll
-            for (int k = 0; k < W::C1; ++k) emit(wb * ps[k]);
+                for (int m = 0; m < 9; ++m) wr[15 + m] = w * B4[m];
+            }
         }
+        __syncwarp();
+        // lane = job: the sums over the batch stay in the lane's registers for the whole row; per edge
+        // a lane reads its four amplitudes and its weight (every lane inside the same two rows)
+#pragma unroll 4
+        for (int e = 0; e < nb; ++e) {
 #pragma unroll
-        for (int m = 0; m < 5; ++m) {
-            const float wb = w * B2[m];
-#pragma unroll
-            for (int k = 0; k < W::C2; ++k) emit(wb * ps[k]);
+            for (int sl = 0; sl < W::SLOTS; ++sl) {
+                const float4 p4 = *reinterpret_cast<const float4*>(psi_s + e * W::PF + j_psi[sl]);
+                const float wv = wbs[e * W::PW + j_w[sl]];
+                accJ[sl][0] += wv * p4.x; accJ[sl][1] += wv * p4.y; accJ[sl][2] += wv * p4.z; accJ[sl][3] += wv * p4.w;
+            }
         }
-        if (L >= 3) {
-#pragma unroll
-            for (int m = 0; m < 7; ++m) emit(w * B3[m] * ps[0]);
-        }
-        if (L >= 4) {
-#pragma unroll
-            for (int m = 0; m < 9; ++m) emit(w * B4[m] * ps[0]);
-        }
+        __syncwarp();                           // the next batch overwrites both
     };
 
     int qn = 0;
@@ -473,9 +475,11 @@ k_edge_forward(const EdgeArgs a) {
     float* row_out = a.state + (size_t)(i - a.a0) * a.d.SP;
     if (sub == 0) *reinterpret_cast<float4*>(row_out + c) = make_float4(acc0[0], acc0[1], acc0[2], acc0[3]);
 #pragma unroll
-    for (int j = 0; j < W::NCH; ++j) {
-        const int v = lane + 32 * j;
-        if (v < W::NHI) row_out[a.d.offA[1] + v] = accH[j];
+    for (int sl = 0; sl < W::SLOTS; ++sl) {
+        if (j_out[sl] < 0) continue;
+        float* o = row_out + a.d.offA[1] + j_out[sl];
+        if (lane + 32 * sl < W::J1 + W::J2) *reinterpret_cast<float4*>(o) = make_float4(accJ[sl][0], accJ[sl][1], accJ[sl][2], accJ[sl][3]);
+        else o[0] = accJ[sl][0];
     }
     if (lane == 0) {
         const float h0 = (float)s0, h1 = (float)s1;
