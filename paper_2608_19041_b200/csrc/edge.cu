@@ -264,7 +264,9 @@ template <int C0, int L, int G = 1> struct Widths {
     static constexpr int NCH = (NHI + 31) / 32;
     // row pitch (floats) of the per-edge amplitude staging; pitch/4 odd keeps 16-byte
     // accesses of 8 consecutive lanes on distinct bank groups
-    static constexpr int PF = ((C1 / 4 + 1) & 1) ? C1 + 4 : C1 + 8;          // forward: psi
+    // (forward, C0 = 128: a whole warp works on one edge, rows are written one or two at a time and
+    // read one at a time, so no padding is needed, and with degree 4 none fits in 48 KB)
+    static constexpr int PF = C0 / (4 * G) == 32 ? C1 : (((C1 / 4 + 1) & 1) ? C1 + 4 : C1 + 8);   // forward: psi
     static constexpr int PB = ((2 * C1 / 4 + 1) & 1) ? 2 * C1 + 4 : 2 * C1 + 8;   // backward: psi, dpsi
     // forward, sums of degree >= 1: a job is four consecutive channels of one harmonic component
     // (degrees 1 and 2) or one component of a one-channel degree (3, 4); a lane owns up to SLOTS jobs
