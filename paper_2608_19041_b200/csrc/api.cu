@@ -61,11 +61,11 @@ struct umlmd {
     // replay of repeated launch sequences as CUDA graphs (see run_replayed)
     struct Replay {
         cudaGraphExec_t exec = nullptr;
-        const void* key[4] = {nullptr, nullptr, nullptr, nullptr}; double key_dt = 0; int64_t key_serial = -1; int key_flags = 0;
+        const void* key[4] = {nullptr, nullptr, nullptr, nullptr}; double key_dt = 0, key_x0 = 0, key_x1 = 0; int64_t key_serial = -1; int key_flags = 0;
         bool seen = false;                           // the key's sequence has run once as plain launches
         int64_t launches[16] = {0}; int64_t total = 0;   // what one replay launches, per class
     };
-    Replay rp_compute, rp_step;
+    Replay rp_compute, rp_step, rp_nvt;
     int launch_graphs = 0;                           // option: 0 = automatic, 1 = always, -1 = never
     bool graphs_broken = false;                      // a capture failed on this handle: plain launches from then on
     cudaStream_t cap_st = nullptr;                   // stream the sequences are captured on
@@ -276,13 +276,13 @@ void replay_drop(umlmd_t::Replay& r) {
 }
 template <class Body>
 int run_replayed(umlmd_t* h, umlmd_t::Replay& r, const void* k0, const void* k1, const void* k2, const void* k3,
-                 double dt, int flags, Body body) {
+                 double dt, int flags, Body body, double x0 = 0.0, double x1 = 0.0) {
     if (!replay_allowed(h)) return body();
-    const bool same = r.key[0] == k0 && r.key[1] == k1 && r.key[2] == k2 && r.key[3] == k3 && r.key_dt == dt &&
+    const bool same = r.key[0] == k0 && r.key[1] == k1 && r.key[2] == k2 && r.key[3] == k3 && r.key_dt == dt && r.key_x0 == x0 && r.key_x1 == x1 &&
                       r.key_flags == flags && r.key_serial == h->list_serial;
     if (!same) {
         replay_drop(r);
-        r.key[0] = k0; r.key[1] = k1; r.key[2] = k2; r.key[3] = k3; r.key_dt = dt; r.key_flags = flags;
+        r.key[0] = k0; r.key[1] = k1; r.key[2] = k2; r.key[3] = k3; r.key_dt = dt; r.key_x0 = x0; r.key_x1 = x1; r.key_flags = flags;
         r.key_serial = h->list_serial; r.seen = true;
         return body();
     }
@@ -461,6 +461,7 @@ int umlmd_destroy(umlmd_t* h) {
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
     if (h->rp_compute.exec) cudaGraphExecDestroy(h->rp_compute.exec);
     if (h->rp_step.exec) cudaGraphExecDestroy(h->rp_step.exec);
+    if (h->rp_nvt.exec) cudaGraphExecDestroy(h->rp_nvt.exec);
     if (h->cap_st) cudaStreamDestroy(h->cap_st);
     if (h->h_out) cudaFreeHost(h->h_out);
     if (h->h_err) cudaFreeHost(h->h_err);
@@ -849,13 +850,22 @@ int umlmd_step_nvt(umlmd_t* h, int nsteps, double dt_ps, int rebuild_every, doub
         { Scope sc(h, kIntegrate, 1); API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, true, d_scale, h->st)); }
         ++h->steps_since_build;
         if ((rc = maybe_rebuild(h, rebuild_every)) != UMLMD_OK) return stop_run(h, rc);
-        if ((rc = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr)) != UMLMD_OK) return stop_run(h, rc);
         const bool last = s + 1 == nsteps;
-        Scope sc(h, kIntegrate, 4);
-        API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, false, nullptr, h->st));
-        API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, d_ke, h->st));
-        // closing half step of the chain, and the next step's opening one in the same launch
-        API_CUDA(h, launch_nhc(h->d_nhc, d_ke, last ? 1 : 2, p, h->st));
+        auto body = [&]() {
+            int r = enqueue_compute(h, h->md_pos, true, h->md_force, nullptr);
+            if (r != UMLMD_OK) return r;
+            Scope sc(h, kIntegrate, 4);
+            API_CUDA(h, launch_vv_kick_drift(N, h->md_pos, h->md_vel, h->md_force, h->type_o, h->d_inv_mass, dt_ps, 1, false, nullptr, h->st));
+            API_CUDA(h, launch_kinetic_energy(N, h->md_vel, h->type_o, h->d_mass, h->scratch, d_ke, h->st));
+            // closing half step of the chain, and the next step's opening one in the same launch
+            API_CUDA(h, launch_nhc(h->d_nhc, d_ke, last ? 1 : 2, p, h->st));
+            return (int)UMLMD_OK;
+        };
+        // a middle step between two list builds launches the same sequence as the one before it (the
+        // opening kick and drift above differ between the first step of a call and the others: plain)
+        rc = last ? body() : run_replayed(h, h->rp_nvt, h->md_pos, h->md_vel, h->md_force, h->d_nhc, dt_ps, 0, body,
+                                          temperature_K, t_damp_ps);
+        if (rc != UMLMD_OK) return stop_run(h, rc);
     }
     if (nsteps > 0) {      // the last scale factor has not been applied to the velocities yet
         Scope sc(h, kIntegrate, 1);

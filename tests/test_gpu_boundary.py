@@ -199,5 +199,16 @@ def test_replayed_launch_sequences_repeat_the_plain_launches_bit_for_bit(own_str
         # the three that end a call, the three with a list build (each the first with its list) and
         # the first after the change of MD state run as plain launches
         assert plain.query()["graph_replays"] == 0 and graph.query()["graph_replays"] == 4 + 2 + (33 - 3 - 3 - 1)
+        # the thermostatted driver replays its middle steps too
+        r0 = graph.query()["graph_replays"]
+        for chunk in (4, 19):
+            ra = plain.step_nvt(chunk, 0.001, 300.0, 0.05, rebuild_every=10)
+            rb = graph.step_nvt(chunk, 0.001, 300.0, 0.05, rebuild_every=10)
+            assert ra == rb
+            torch.cuda.synchronize()
+            assert torch.equal(pos_a, pos_b) and torch.equal(va, vb)
+        assert np.array_equal(plain.get_nvt_state(), graph.get_nvt_state())
+        assert graph.query()["graph_replays"] > r0 + 10
+        assert plain.query()["kernel_launches"] == graph.query()["kernel_launches"]
     plain.close()
     graph.close()
