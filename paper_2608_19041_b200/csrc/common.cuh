@@ -125,6 +125,7 @@ struct FrameCell {
 
 struct NeighborDev {
     int64_t N = 0, E = 0, E_cap = 0, N_cap = 0;
+    unsigned long long* bounds = nullptr;   // [6] scratch of the extent reduction (open directions)
     int64_t n_owned = 0, E_owned = 0;   // rows [0, n_owned) and edges [0, E_owned) belong to owned atoms (all of them without ghosts)
     double L[3] = {0, 0, 0};     // cell edge lengths (the diagonal of H)
     double H[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};   // cell vectors as rows

@@ -14,6 +14,7 @@
 #include <thrust/iterator/transform_iterator.h>
 
 #include <cmath>
+#include <cstring>
 
 #include "alloc.h"
 #include "kernels.h"
@@ -59,6 +60,50 @@ __device__ __forceinline__ int pack_shift(int nx, int ny, int nz) {
 }
 
 struct CellRows { double h[9]; int tri; };
+
+// order-preserving map of a double onto an unsigned integer, for atomicMin / atomicMax
+__device__ __forceinline__ unsigned long long ordered_key(double x) {
+    const long long b = __double_as_longlong(x);
+    return b < 0 ? ~(unsigned long long)b : (unsigned long long)b | 0x8000000000000000ull;
+}
+inline double ordered_value(unsigned long long k) {
+    const unsigned long long b = (k & 0x8000000000000000ull) ? (k & 0x7fffffffffffffffull) : ~k;
+    double x;
+    std::memcpy(&x, &b, sizeof(x));
+    return x;
+}
+// smallest and largest binning coordinate of the atoms along each direction (Cartesian for an
+// orthorhombic cell, fractional for a general one): keys[k] = min, keys[3 + k] = max
+__global__ void k_bounds(int N, const double* __restrict__ pos, Grid g, unsigned long long* __restrict__ keys) {
+    __shared__ unsigned long long smin[3][8], smax[3][8];
+    unsigned long long mn[3] = {~0ull, ~0ull, ~0ull}, mx[3] = {0ull, 0ull, 0ull};
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
+        const double x = pos[3 * (size_t)i], y = pos[3 * (size_t)i + 1], z = pos[3 * (size_t)i + 2];
+        for (int k = 0; k < 3; ++k) {
+            const double v = g.tri ? x * g.Hinv[k] + y * g.Hinv[3 + k] + z * g.Hinv[6 + k] : (k == 0 ? x : (k == 1 ? y : z));
+            const unsigned long long key = ordered_key(v);
+            if (key < mn[k]) mn[k] = key;
+            if (key > mx[k]) mx[k] = key;
+        }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int k = 0; k < 3; ++k) {
+        for (int off = 16; off > 0; off >>= 1) {
+            const unsigned long long a = __shfl_xor_sync(0xffffffffu, mn[k], off), b = __shfl_xor_sync(0xffffffffu, mx[k], off);
+            if (a < mn[k]) mn[k] = a;
+            if (b > mx[k]) mx[k] = b;
+        }
+        if (lane == 0) { smin[k][warp] = mn[k]; smax[k][warp] = mx[k]; }
+    }
+    __syncthreads();
+    if (threadIdx.x < 3) {
+        const int k = threadIdx.x;
+        unsigned long long a = smin[k][0], b = smax[k][0];
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) { if (smin[k][w] < a) a = smin[k][w]; if (smax[k][w] > b) b = smax[k][w]; }
+        atomicMin(keys + k, a);
+        atomicMax(keys + 3 + k, b);
+    }
+}
 
 // fold positions into the cell, bin them
 __global__ void k_fold_bin(int N, const double* __restrict__ pos, Grid g, double* __restrict__ wpos,
@@ -461,7 +506,7 @@ struct WidenDeg {
 void neighbor_free(NeighborDev* nb) {
     void* ptrs[] = {nb->frames, nb->rec, nb->wpos, nb->img, nb->perm, nb->type_s, nb->xs0, nb->xs, nb->row_ptr, nb->src,
                     nb->shift, nb->rev, nb->key, nb->key2, nb->idx, nb->idx2, nb->cell_start, nb->deg,
-                    nb->cub_tmp};
+                    nb->cub_tmp, nb->bounds};
     for (void* p : ptrs)
         dev_free(p);
     *nb = NeighborDev();
@@ -502,17 +547,19 @@ int neighbor_build(NeighborDev* nb, int64_t N64, int64_t n_owned64, const double
     double lo[3] = {0, 0, 0}, ext[3] = {L[0], L[1], L[2]}, unit[3] = {1, 1, 1};
     if (g.tri) for (int k = 0; k < 3; ++k) { ext[k] = 1.0; unit[k] = height[k]; }
     if (!(pbc[0] && pbc[1] && pbc[2]) && N > 0) {
-        std::vector<double> hp((size_t)N * 3);
-        NB_CHECK(cudaMemcpyAsync(hp.data(), d_pos, sizeof(double) * 3 * (size_t)N, cudaMemcpyDeviceToHost, st));
+        // the extent of the atoms along the open directions, reduced on the device (six keys come back)
+        if (!nb->bounds) { int64_t c = 0; NB_CHECK(dev_ensure(&nb->bounds, &c, 6)); }
+        const unsigned long long init[6] = {~0ull, ~0ull, ~0ull, 0ull, 0ull, 0ull};
+        unsigned long long keys[6];
+        NB_CHECK(cudaMemcpyAsync(nb->bounds, init, sizeof(init), cudaMemcpyHostToDevice, st));
+        int blocks = (N + 255) / 256;
+        if (blocks > 1184) blocks = 1184;
+        k_bounds<<<blocks, 256, 0, st>>>(N, d_pos, g, nb->bounds);
+        NB_CHECK(cudaMemcpyAsync(keys, nb->bounds, sizeof(keys), cudaMemcpyDeviceToHost, st));
         NB_CHECK(cudaStreamSynchronize(st));
         for (int k = 0; k < 3; ++k) {
             if (pbc[k]) continue;
-            auto coord = [&](int i) {
-                const double* r = &hp[3 * (size_t)i];
-                return g.tri ? r[0] * g.Hinv[k] + r[1] * g.Hinv[3 + k] + r[2] * g.Hinv[6 + k] : r[k];
-            };
-            double mn = coord(0), mx = mn;
-            for (int i = 1; i < N; ++i) { const double v = coord(i); if (v < mn) mn = v; if (v > mx) mx = v; }
+            const double mn = ordered_value(keys[k]), mx = ordered_value(keys[3 + k]);
             if (!std::isfinite(mn) || !std::isfinite(mx)) { *err = "non-finite position"; return UMLMD_E_NONFINITE; }
             lo[k] = mn; ext[k] = (mx - mn) + 1e-6 / unit[k];
         }
