@@ -126,6 +126,42 @@ def test_bricks_with_ghosts_reproduce_the_undivided_evaluation(grid):
     ref_model.close()
 
 
+def test_a_brick_without_atoms_of_its_own_takes_part_in_the_exchange():
+    # a slab with 17 A of vacuum along x, cut into three bricks along x: the third owns nothing and
+    # holds only images of the slab's first layers; energies and forces are those of the whole cell
+    from paper_2608_19041_b200.domain import Domain
+    p = SMALL_PROFILES["p16_3_2"]
+    s = make_system(dict(kind="fcc", cells=6, a=4.05, jitter=0.08, seed=13, n_types=p["T"], masses=[20.0] * p["T"]))
+    s["cell"] = np.array(s["cell"], dtype=np.float64)
+    s["cell"][0, 0] *= 1.7
+    blob = make_blob(p, seed=49, bias_scale=0.2, e_ref_scale=0.5)
+    ref_model, pos, types = _reference(blob, s, 1.0)
+    ref = ref_model.compute(pos, atom_energy=True)
+    grid = (3, 1, 1)
+    B = _binding()
+
+    def rank_fn(comm):
+        m = B.Model(blob)
+        d = Domain(m, comm, np.diag(s["cell"]), grid, p["rc"], 1.0, s["masses"])
+        d.distribute(s["pos"], np.zeros_like(s["pos"]), s["types"])
+        d.start()
+        e_pot, _, virial = d.totals()
+        _, _, force = d.gather()
+        res = dict(e_pot=e_pot, virial=virial, force=force.clone(), n_own=d.n_own, n_ghost=d.n_ghost)
+        m.close()
+        return res
+
+    out = _run_ranks(3, rank_fn)
+    assert out[2]["n_own"] == 0 and out[2]["n_ghost"] > 0
+    assert sum(o["n_own"] for o in out) == len(s["pos"])
+    f_ref = ref["forces"]
+    for o in out:
+        assert abs(o["e_pot"] - ref["energy"]) <= 2e-6 * ref["atom_energy"].abs().sum().item()
+        assert (o["force"] - f_ref).abs().max().item() <= 2e-5 * f_ref.abs().max().item()
+        assert np.abs(o["virial"] - ref["virial"]).max() <= 2e-5 * max(1.0, np.abs(ref["virial"]).max())
+    ref_model.close()
+
+
 def test_ghost_atoms_have_no_energy_and_owned_forces_need_their_return():
     # one handle, hand-made ghosts: the first half of a small cluster is owned, the rest are ghosts.
     # The energy is the owned atoms' share, and the forces are the derivative of that share
