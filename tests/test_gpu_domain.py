@@ -134,6 +134,8 @@ def test_a_brick_without_atoms_of_its_own_takes_part_in_the_exchange():
     s = make_system(dict(kind="fcc", cells=6, a=4.05, jitter=0.08, seed=13, n_types=p["T"], masses=[20.0] * p["T"]))
     s["cell"] = np.array(s["cell"], dtype=np.float64)
     s["cell"][0, 0] *= 1.7
+    s["pos"] = np.array(s["pos"], dtype=np.float64)
+    s["pos"][:, 0] += 1.0                               # keeps the jittered first layer from wrapping to the far side
     blob = make_blob(p, seed=49, bias_scale=0.2, e_ref_scale=0.5)
     ref_model, pos, types = _reference(blob, s, 1.0)
     ref = ref_model.compute(pos, atom_energy=True)
