@@ -164,6 +164,52 @@ def test_a_brick_without_atoms_of_its_own_takes_part_in_the_exchange():
     ref_model.close()
 
 
+def test_exchange_over_an_nccl_process_group_of_one_rank():
+    # the production communicator (torch.distributed over NCCL) with a single rank: the brick's
+    # ghosts are its own periodic images and every exchange is a message to itself, through the
+    # same all_to_all_single / all_gather / all_reduce calls that several GPUs would use
+    import socket
+
+    import torch.distributed as dist
+
+    from paper_2608_19041_b200.domain import Domain, TorchComm
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        name = "cfg2_cu4000"
+        cfg = CONFIGS[name]
+        desc = dict(cfg["system"])
+        desc["cells"] = 6
+        s = make_system(desc, cfg["md"])
+        md = cfg["md"]
+        blob = workload_blob(name)
+        B = _binding()
+        ref_model, pos, types = _reference(blob, s, md["skin"])
+        vel = torch.as_tensor(s["vel"], dtype=torch.float64).cuda().contiguous()
+        ref_model.set_md_state(pos, vel, s["masses"])
+        e_pot_ref, e_kin_ref = ref_model.step(12, md["dt_ps"], md["rebuild_every"])
+        m = B.Model(blob)
+        d = Domain(m, TorchComm(), np.diag(s["cell"]), (1, 1, 1), ref_model.query()["rc"], md["skin"], s["masses"])
+        d.distribute(s["pos"], s["vel"], s["types"])
+        d.start()
+        d.step(12, md["dt_ps"], md["rebuild_every"])
+        e_pot, e_kin, _ = d.totals()
+        p, v, _ = d.gather()
+        L = torch.as_tensor(np.array(np.diag(s["cell"]))).cuda()
+        dp = p - pos
+        dp -= torch.round(dp / L) * L
+        assert dp.abs().max().item() < 2e-6 and (v - vel).abs().max().item() < 2e-4
+        assert abs(e_pot - e_pot_ref) < 2e-6 * len(s["pos"]) and abs(e_kin - e_kin_ref) < 2e-6 * len(s["pos"])
+        assert d.n_ghost > 0
+        m.close()
+        ref_model.close()
+    finally:
+        dist.destroy_process_group()
+
+
 def test_ghost_atoms_have_no_energy_and_owned_forces_need_their_return():
     # one handle, hand-made ghosts: the first half of a small cluster is owned, the rest are ghosts.
     # The energy is the owned atoms' share, and the forces are the derivative of that share
