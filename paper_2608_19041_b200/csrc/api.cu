@@ -232,7 +232,7 @@ int enqueue_compute(umlmd_t* h, const double* d_pos, bool want_grad, double* d_f
         Scope sc(h, kForce, 1);
         API_CUDA(h, launch_force_assembly(nb, h->g, d_force ? nullptr : h->f_sorted, d_force, h->d_err, h->st));
     }
-    Scope sc(h, kReduce, d_atom_energy ? 3 : 2);
+    Scope sc(h, kReduce, (N <= 4096 ? 1 : 2) + (d_atom_energy ? 1 : 0));      // one reduction launch for a single slice of energies
     API_CUDA(h, launch_reduce_energy_virial(h->e_atom, N, h->virial_part, vpart_used, h->scratch, h->d_out,
                                             h->d_err, h->st));
     if (d_atom_energy) API_CUDA(h, launch_scatter_atom_energy(nb, h->e_atom, d_atom_energy, h->st));

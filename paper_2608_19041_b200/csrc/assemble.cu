@@ -351,6 +351,12 @@ cudaError_t launch_reduce_energy_virial(const double* e_atom, int64_t N, const d
                                         double* scratch, double* out, int* d_err, cudaStream_t st) {
     int blocks; int64_t chunk;
     slices(N, &blocks, &chunk);
+    if (blocks == 1) {
+        // a single slice: the second pass sums the atomic energies itself, in the order the first
+        // pass would have used (its own sum over one partial only adds zeros), and one launch less
+        k_final_reduce<<<10, kRedBlock, 0, st>>>(e_atom, (int)N, virial_part, n_part, out, d_err);
+        return cudaGetLastError();
+    }
     k_sum_slices<<<blocks, kRedBlock, 0, st>>>(e_atom, N, chunk, scratch);
     k_final_reduce<<<10, kRedBlock, 0, st>>>(scratch, blocks, virial_part, n_part, out, d_err);
     return cudaGetLastError();
