@@ -159,7 +159,7 @@ int ensure_workspace(umlmd_t* h) {
         h->n_cap = N;
     }
     const int64_t n_tiles = B > 0 ? (N + B - 1) / B : 0;
-    const int64_t vneed = (N / 8 + n_tiles + 2) * 9;
+    const int64_t vneed = (N / 4 + n_tiles + 2) * 9;
     if (vneed > h->vpart_cap || !h->virial_part) API_CUDA(h, dev_ensure(&h->virial_part, &h->vpart_cap, vneed));
     return UMLMD_OK;
 }
@@ -588,7 +588,7 @@ int umlmd_workspace_bytes(const umlmd_t* h, int64_t N, int64_t n_edges, int64_t*
     t += grown(3 * n_edges, 4);
     t += buf(N, 8) + buf(3 * N, 8) + buf(N, 4);
     const int64_t tiles = Bt > 0 ? (N + Bt - 1) / Bt : 0;
-    t += buf((N / 8 + tiles + 2) * 9, 8);
+    t += buf((N / 4 + tiles + 2) * 9, 8);
     t += buf(3 * N, 8) + 2 * buf(d.T, 8) + buf(2 * kNhcChain + 2, 8);
     *bytes = t;
     return UMLMD_OK;

@@ -22,7 +22,11 @@ namespace umd {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 8;
+// A block is done when its slowest row is: with fewer rows per block fewer finished warps sit on
+// registers and shared memory waiting for it (measured at eight / four / two warps per block, 131072
+// atoms of the 64-species workload: backward 1.535 / 1.487 / 1.479 ms, forward 1.318 / 1.301 / 1.294 ms;
+// four keeps the per-block virial partials at a quarter of the atom count).
+constexpr int kWarpsPerBlock = 4;
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
@@ -281,10 +285,10 @@ template <int C0, int L, int G = 1> struct Widths {
 
 // The channel-parallel phase of the backward pass waits on load latency, and what hides it best
 // depends on the width (all measured on the edge backward kernel).  C0 = 128: four channel groups
-// per lane, that many times the table and pair loads in flight, at two resident blocks per SM (128
-// registers): 10 % faster than two groups, and than two groups at three blocks.  C0 = 32 and 64:
-// two groups at three blocks (85 registers, a few spilled words): 9-13 % faster than two blocks,
-// four groups being slower again.  C0 <= 16: one group, three blocks (13 % faster than two).
+// per lane, that many times the table and pair loads in flight, at 16 resident warps per SM (128
+// registers): 10 % faster than two groups, and than two groups at 24 warps.  C0 = 32 and 64:
+// two groups at 24 warps (85 registers, a few spilled words): 9-13 % faster than 16 warps,
+// four groups being slower again.  C0 <= 16: one group, 24 warps (13 % faster than 16).
 template <int C0> struct BwdGroups { static constexpr int G = C0 >= 128 ? 4 : (C0 >= 32 ? 2 : 1); };
 
 template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared memory of the backward kernel
@@ -309,11 +313,11 @@ template <int C0, int L, bool HASR> struct BwdSmem {          // dynamic shared 
 //      component of a one-channel degree) for the whole row, and for every edge of the batch adds
 //      weight x amplitudes from the two parked rows: two shared-memory reads per edge and warp,
 //      where summing per-edge products by transposition took six.
-// Up to C0 = 64 a fourth resident block per SM (64 registers, a few spilled words) is worth more
+// Up to C0 = 64 a fourth group of eight resident warps per SM (64 registers, a few spilled words) is worth more
 // than the registers: the channel-parallel phase waits on load latency (measured: 6-10 % on the
-// forward kernel at C0 = 8 .. 64, 2 % the other way at C0 = 128, which stays at three blocks).
+// forward kernel at C0 = 8 .. 64, 2 % the other way at C0 = 128, which stays at 24 warps).
 template <int C0, int L, bool HASR, bool UNI>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, C0 <= 64 ? 4 : 3)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, (C0 <= 64 ? 4 : 3) * 8 / kWarpsPerBlock)
 k_edge_forward(const EdgeArgs a) {
     using W = Widths<C0, L>;
     // scratch per warp: the parked amplitudes of the batch (row pitch PF), and behind them first the
@@ -499,7 +503,7 @@ k_edge_forward(const EdgeArgs a) {
 // destination's gradient block held in shared memory, and assembles dE/dr_ij.  Edges in the
 // skin shell get a zero gradient as soon as their geometry is known.
 template <int C0, int L, bool HASR, bool UNI>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, C0 <= 64 ? 3 : 2)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, (C0 <= 64 ? 3 : 2) * 8 / kWarpsPerBlock)
 k_edge_backward(const EdgeArgs a) {
     constexpr int G = BwdGroups<C0>::G;
     using W = Widths<C0, L, G>;
