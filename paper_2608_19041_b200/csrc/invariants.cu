@@ -117,8 +117,9 @@ struct Plan {                                 // widths and the shared-memory pl
     static constexpr int nMatP = (nMat + nGaunt + 3) / 4 * 4;                    // matrices come first: 16-byte rows
     // backward, L = 4: gradient shares of the degree-4 couplings with respect to Z1, Z2, X3 and X4
     static constexpr int nE4 = L >= 4 ? nZ1 + nZ2 + 7 + 9 : 0;
+    // forward: the staged state slice shares the rows of the feature staging area (nDS counts the larger)
     static int rows(int TW, int nDS, bool bwd) {
-        return TW + nX + nZ + nDS + (bwd ? nPreB + nX + nX3 + nZ + 18 + nAux + nE4 : nPreF);
+        return bwd ? TW + nX + nZ + nDS + nPreB + nX + nX3 + nZ + 18 + nAux + nE4 : nX + nZ + nDS + nPreF;
     }
     static size_t bytes(int TW, int nDS, bool bwd) { return sizeof(float) * ((size_t)rows(TW, nDS, bwd) * P + nMatP); }
 };
@@ -272,17 +273,23 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
     const int C0 = d.C0, TW = d.SP - C0;
     const int c_full = (2 * C0 / 32) * 32;         // columns [0, c_full) go straight from global to global
     float* mats = sm;
-    float* ST = sm + PL::nMatP;
-    float* XT = ST + TW * P;
+    float* XT = sm + PL::nMatP;
     float* ZZ = XT + PL::nX * P;
     float* PRE = ZZ + PL::nZ * P;
-    float* DS = PRE + PL::nPreF * P;               // feature columns [c_full, DP), [column][atom]
+    // staging area of the feature columns, [column][atom], filled and written out in two portions
+    // (columns [c_full, oG[2]) and [oG[2], DP)); before that it holds the state slice, which is only
+    // needed until the harmonic rows are aligned and the first 2 C0 columns are out
+    float* DS = PRE + PL::nPreF * P;
+    float* ST = DS;
+    (void)TW;
     Front<C1, C2, L> f;
     f.setup(a, ST, XT, ZZ, mats);
     const int lane = f.lane, warp = f.warp, nv = f.nv, b0 = f.b0;
+    const double M0lane = f.M0_of(lane);           // kept: the state slice is overwritten below
     int uctr = 0;
+    int dbase = c_full;                            // first column of the portion in the staging area
 #define TAKE() ((uctr++ % NW) == warp)
-#define DSK(k) DS[((k) - c_full) * P + lane]
+#define DSK(k) DS[((k) - dbase) * P + lane]
 
     f.gaunt_pre(PRE, uctr);
 
@@ -346,15 +353,13 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
         float v = 0.f;
         if (lane < nv) {
             if (c < C0) v = __ldg(m.X0 + a.type_s[a.a0 + b0 + lane] * C0 + c);
-            else v = a.state[(size_t)(b0 + lane) * d.SP + (c - C0)] * (float)(1.0 / f.M0_of(lane));
+            else v = a.state[(size_t)(b0 + lane) * d.SP + (c - C0)] * (float)(1.0 / M0lane);
         }
         DSK(c) = v;
     }
     if (TAKE()) {   // the two normalising scales, calibrated here in double precision
-        const double M0d = f.M0_of(lane);
-        DSK(kM0) = (float)((M0d - (double)__ldg(m.mu + kM0)) * (double)__ldg(m.inv_sigma + kM0));
+        DSK(kM0) = (float)((M0lane - (double)__ldg(m.mu + kM0)) * (double)__ldg(m.inv_sigma + kM0));
         DSK(kM1) = (float)((f.M1d - (double)__ldg(m.mu + kM1)) * (double)__ldg(m.inv_sigma + kM1));
-        for (int k = d.D_out; k < d.DP; ++k) DSK(k) = 0.f;
     }
     // Gram blocks, row-major upper triangle, strict off-diagonals times sqrt 2; a unit is
     // rows u and C-1-u, which together hold C+1 entries
@@ -371,6 +376,28 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
                 DSK(k) = kR2 * (x0 * X1[q * P] + x1 * X1[(C1 + q) * P] + x2 * X1[(2 * C1 + q) * P]);
             }
         }
+    }
+    // ---- first portion out: calibrate and write, lane = column ---------------------------
+    auto write_out = [&](const int lo, const int hi) {
+        __syncthreads();
+        for (int cb = lo; cb < hi; cb += 32) {
+            const int col = cb + lane;
+            if (col >= hi) continue;
+            float mu_c = 0.f, is_c = 1.f;
+            if (col < d.D_out && col != kM0 && col != kM1) { mu_c = __ldg(m.mu + col); is_c = __ldg(m.inv_sigma + col); }
+            const bool split_col = !(a.skip_x0_split && col < C0);
+#pragma unroll
+            for (int i = 0; i < AT / NW; ++i) {
+                const int aa = warp + i * NW;
+                if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (DS[(col - lo) * P + aa] - mu_c) * is_c, split_col);
+            }
+        }
+        __syncthreads();
+    };
+    write_out(c_full, d.oG[2]);
+    dbase = d.oG[2];
+    if (TAKE()) {
+        for (int k = d.D_out; k < d.DP; ++k) DSK(k) = 0.f;      // padding columns
     }
     for (int u = 0; u < C2 / 2; ++u) {
         if (!TAKE()) continue;
@@ -479,20 +506,7 @@ __global__ void __launch_bounds__(NT) k_inv_forward(const InvArgs a) {
             DSK(d.oPi + e * K1 + k1) = y[0] * y[0] + y[1] * y[1] + y[2] * y[2];
         }
     }
-    __syncthreads();
-
-    // ---- calibrate and write out, lane = column ----------------------------------------
-    for (int cb = c_full; cb < d.DP; cb += 32) {
-        const int col = cb + lane;
-        float mu_c = 0.f, is_c = 1.f;
-        if (col < d.D_out && col != kM0 && col != kM1) { mu_c = __ldg(m.mu + col); is_c = __ldg(m.inv_sigma + col); }
-        const bool split_col = !(a.skip_x0_split && col < C0);
-#pragma unroll
-        for (int i = 0; i < AT / NW; ++i) {
-            const int aa = warp + i * NW;
-            if (aa < nv) put_feature(a, (size_t)(b0 + aa) * d.DP + col, (DS[(col - c_full) * P + aa] - mu_c) * is_c, split_col);
-        }
-    }
+    write_out(d.oG[2], d.DP);
 #undef TAKE
 #undef DSK
 }
@@ -916,7 +930,13 @@ cudaError_t dispatch(const InvArgs& a, cudaStream_t st) {
     if (a.n <= 0) return cudaSuccess;
     const int blocks = (a.n + AT - 1) / AT;
     const int C1 = a.d.C[1], C2 = a.d.C[2], L = a.d.L;
-    const int TW = a.d.SP - a.d.C0, nDS = a.d.DP - (2 * a.d.C0 / 32) * 32;
+    const int TW = a.d.SP - a.d.C0;
+    int nDS = a.d.DP - (2 * a.d.C0 / 32) * 32;
+    if (FWD) {      // the larger of the two portions of staged columns and of the state slice they replace
+        const int na = a.d.oG[2] - (2 * a.d.C0 / 32) * 32, nb = a.d.DP - a.d.oG[2];
+        nDS = na > nb ? na : nb;
+        if (TW > nDS) nDS = TW;
+    }
 #define UMLMD_CASE(c1, c2, l)                                                                   \
     if (C1 == c1 && C2 == c2 && L == l) {                                                       \
         const size_t bytes = Plan<c1, c2, l>::bytes(TW, nDS, !FWD);                             \
