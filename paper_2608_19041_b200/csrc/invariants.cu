@@ -117,9 +117,11 @@ struct Plan {                                 // widths and the shared-memory pl
     static constexpr int nMatP = (nMat + nGaunt + 3) / 4 * 4;                    // matrices come first: 16-byte rows
     // backward, L = 4: gradient shares of the degree-4 couplings with respect to Z1, Z2, X3 and X4
     static constexpr int nE4 = L >= 4 ? nZ1 + nZ2 + 7 + 9 : 0;
-    // forward: the staged state slice shares the rows of the feature staging area (nDS counts the larger)
+    // the staged state slice shares the rows of the staging area of the feature columns (nDS counts the
+    // larger of the slice and of the two portions the columns are staged in)
     static int rows(int TW, int nDS, bool bwd) {
-        return bwd ? TW + nX + nZ + nDS + nPreB + nX + nX3 + nZ + 18 + nAux + nE4 : nX + nZ + nDS + nPreF;
+        (void)TW;
+        return bwd ? nX + nZ + nDS + nPreB + nX + nX3 + nZ + 18 + nAux + nE4 : nX + nZ + nDS + nPreF;
     }
     static size_t bytes(int TW, int nDS, bool bwd) { return sizeof(float) * ((size_t)rows(TW, nDS, bwd) * P + nMatP); }
 };
@@ -542,7 +544,7 @@ __device__ __forceinline__ float back_row(const float* dxt, const float* dz, con
 }
 
 template <int C1, int C2, int L>
-__global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
+__global__ void __launch_bounds__(NT, 3) k_inv_backward(const InvArgs a) {
     using PL = Plan<C1, C2, L>;
     constexpr int K1 = C2, K2 = 2;
     extern __shared__ float sm[];
@@ -550,12 +552,16 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     const ModelDev& m = a.m;
     const int C0 = d.C0, TW = d.SP - C0;
     const int c_full = (2 * C0 / 32) * 32;
-    const int nDS = d.DP - c_full;
+    const int nA = d.oG[2] - c_full, nB = d.DP - d.oG[2];
+    const int nDS = TW > (nA > nB ? nA : nB) ? TW : (nA > nB ? nA : nB);
     float* mats = sm;
-    float* ST = sm + PL::nMatP;
-    float* XT = ST + TW * P;
+    float* XT = sm + PL::nMatP;
     float* ZZ = XT + PL::nX * P;
-    float* DS = ZZ + PL::nZ * P;                   // dE/dD / sigma, columns [c_full, DP), [column][atom]
+    // One area, four uses one after the other: the state slice (until the harmonic rows are aligned),
+    // dE/dD / sigma of the columns [oG[2], DP), then of the columns [c_full, oG[2]) ([column][atom]),
+    // and at the end the gradient of the state slice on its way out.
+    float* DS = ZZ + PL::nZ * P;
+    float* ST = DS;
     float* PRE = DS + nDS * P;                     // U, Y, W, Zg, Q v
     float* GX = PRE + PL::nPreB * P;               // dE/dXt (degree-3 rows twice: the two couplings' shares)
     float* DZ = GX + (PL::nX + PL::nX3) * P;
@@ -570,10 +576,11 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     float* YQ = Zg + PL::nZg * P;                  // [(e * K1 + k) * 3 + m]
     const int b0 = blockIdx.x * AT;
     const float* dDg = a.desc + (size_t)b0 * d.DP;
-    {   // stage the gradient rows, lane = column, divided by sigma (zero beyond D_out)
+    // stage the gradient columns [lo, hi), lane = column, divided by sigma (zero beyond D_out)
+    auto stage = [&](const int lo, const int hi) {
         const int ln = threadIdx.x & 31, wp = threadIdx.x >> 5;
         const int nv0 = a.n - b0 < AT ? a.n - b0 : AT;
-        for (int cb = c_full; cb < d.DP; cb += 64) {
+        for (int cb = lo; cb < hi; cb += 64) {
             float v[2][AT / NW];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -581,25 +588,30 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
 #pragma unroll
                 for (int i = 0; i < AT / NW; ++i) {
                     const int aa = wp + i * NW;
-                    v[h][i] = (col < d.DP && aa < nv0) ? dDg[(size_t)aa * d.DP + col] : 0.f;
+                    v[h][i] = (col < hi && aa < nv0) ? dDg[(size_t)aa * d.DP + col] : 0.f;
                 }
             }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int col = cb + 32 * h + ln;
-                if (col >= d.DP) continue;
+                if (col >= hi) continue;
                 const float is_c = col < d.D_out ? __ldg(m.inv_sigma + col) : 0.f;
 #pragma unroll
-                for (int i = 0; i < AT / NW; ++i) DS[(col - c_full) * P + wp + i * NW] = v[h][i] * is_c;
+                for (int i = 0; i < AT / NW; ++i) DS[(col - lo) * P + wp + i * NW] = v[h][i] * is_c;
             }
         }
-    }
+    };
     Front<C1, C2, L> f;
-    f.setup(a, ST, XT, ZZ, mats);                  // its barriers also publish DS
+    f.setup(a, ST, XT, ZZ, mats);
     const int lane = f.lane, warp = f.warp, nv = f.nv;
+    const double M0lane = f.M0_of(lane);           // kept: the state slice is overwritten next
+    __syncthreads();
+    stage(d.oG[2], d.DP);
+    __syncthreads();
     int uctr = 0;
+    int dbase = d.oG[2];                           // first column of the staged portion
 #define TAKE() ((uctr++ % NW) == warp)
-#define DSK(k) DS[((k) - c_full) * P + lane]
+#define DSK(k) DS[((k) - dbase) * P + lane]
 
     const float* X1 = XT + lane;
     const float* X2 = XT + PL::nX1 * P + lane;
@@ -688,7 +700,7 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
 #pragma unroll
         for (int u = 0; u < UA; ++u) {
             const int aa = warp + u * NW;
-            const float im0 = (float)(1.0 / f.M0_of(aa));
+            const float im0 = (float)(1.0 / __shfl_sync(kFull, M0lane, aa));
             float part = 0.f;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -705,18 +717,6 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     __syncthreads();
 
     // ---- gradients of the aligned rows, the probes and the two matrices Q --------------
-    for (int p = 0; p < C1; ++p) {                 // Gram of degree 1: a symmetric matrix-vector product per row
-        if (!TAKE()) continue;
-        float acc[3] = {0.f, 0.f, 0.f};
-#pragma unroll 4
-        for (int q = 0; q < C1; ++q) {
-            const float g = DSK(d.oG[1] + tri_sym(p, q, C1)) * (p == q ? 2.0f : kR2);
-#pragma unroll
-            for (int mm = 0; mm < 3; ++mm) acc[mm] += g * X1[(mm * C1 + q) * P];
-        }
-#pragma unroll
-        for (int mm = 0; mm < 3; ++mm) GX[(mm * C1 + p) * P + lane] = acc[mm];
-    }
     for (int p = 0; p < C2; ++p) {
         if (!TAKE()) continue;
         float acc[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
@@ -870,6 +870,25 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
     }
     __syncthreads();
 
+    // ---- the columns [c_full, oG[2]): the two normalising scales and the Gram block of degree 1 ----
+    stage(c_full, d.oG[2]);
+    dbase = c_full;
+    __syncthreads();
+    const float dM0 = DSK(2 * C0), dM1 = DSK(2 * C0 + 1);      // kept: the area takes the outgoing slice next
+    for (int p = 0; p < C1; ++p) {                 // Gram of degree 1: a symmetric matrix-vector product per row
+        if (!TAKE()) continue;
+        float acc[3] = {0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int q = 0; q < C1; ++q) {
+            const float g = DSK(d.oG[1] + tri_sym(p, q, C1)) * (p == q ? 2.0f : kR2);
+#pragma unroll
+            for (int mm = 0; mm < 3; ++mm) acc[mm] += g * X1[(mm * C1 + q) * P];
+        }
+#pragma unroll
+        for (int mm = 0; mm < 3; ++mm) GX[(mm * C1 + p) * P + lane] = acc[mm];
+    }
+    __syncthreads();
+
     // ---- probes and alignment transposed, row by row; dot1 = sum dXt . Xt = sum dX . X --
     for (int u = 0; u < 10; ++u) {
         if (!TAKE()) continue;
@@ -904,10 +923,12 @@ __global__ void __launch_bounds__(NT) k_inv_backward(const InvArgs a) {
         float dot1 = 0.f;
 #pragma unroll
         for (int u = 0; u < 10; ++u) dot1 += AUX[(1 + u) * P + lane];
-        const float iM0 = (float)(1.0 / f.M0_of(lane));
-        const float dM0 = DSK(2 * C0), dM1 = DSK(2 * C0 + 1), dot0 = AUX[lane];
+        const float iM0 = (float)(1.0 / M0lane);
+        const float dot0 = AUX[lane];
         ST[f.oS * P + lane] = (dM0 - dot0 * iM0) * 0.5f * iM0;
         ST[(f.oS + 1) * P + lane] = (dM1 - dot1 * f.iM1) * 0.5f * f.iM1;
+        ST[(f.oS + 2) * P + lane] = 0.f;
+        ST[(f.oS + 3) * P + lane] = 0.f;
     }
     __syncthreads();
     // write the block's slice back, lane = state entry
@@ -932,7 +953,7 @@ cudaError_t dispatch(const InvArgs& a, cudaStream_t st) {
     const int C1 = a.d.C[1], C2 = a.d.C[2], L = a.d.L;
     const int TW = a.d.SP - a.d.C0;
     int nDS = a.d.DP - (2 * a.d.C0 / 32) * 32;
-    if (FWD) {      // the larger of the two portions of staged columns and of the state slice they replace
+    {               // the larger of the two portions of staged columns and of the state slice that shares their rows
         const int na = a.d.oG[2] - (2 * a.d.C0 / 32) * 32, nb = a.d.DP - a.d.oG[2];
         nDS = na > nb ? na : nb;
         if (TW > nDS) nDS = TW;
